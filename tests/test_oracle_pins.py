@@ -1,0 +1,340 @@
+"""Pins for the CPU oracle: what the paper and the mathematics fix, checked on the CPU.
+
+Every check here compares the oracle with something other than itself: a textbook
+formulation written separately, an identity the paper proves, a number the paper prints,
+a closed form, or brute-force loops on tiny inputs.
+"""
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import rap_oracle as O
+from paper_2602_02599_b200 import synth
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _small(pairing=O.PAIR_HALF, rho=0.75, D=16, Hq=4, Hkv=2, hidden=24, n=7, seed=3, L=1):
+    """Tiny full-weight model: everything needed for both (R) and (F)."""
+    rng = np.random.default_rng(seed)
+    P, dv = O.retained_counts(rho, D)
+    ks = rng.lognormal(0, 1, (L, Hkv, D // 2))
+    vs = rng.lognormal(0, 1, (L, Hkv, D))
+    tabs = O.build_tables(ks, vs, [P] * L, [dv] * L, D, 10000.0, pairing)
+    Wq = rng.normal(0, 0.3, (Hq * D, hidden))
+    Wk = rng.normal(0, 0.3, (Hkv * D, hidden))
+    Wv = rng.normal(0, 0.3, (Hkv * D, hidden))
+    X = rng.normal(0, 1, (n, hidden))
+    return dict(P=P, dv=dv, tabs=tabs, Wq=Wq, Wk=Wk, Wv=Wv, X=X, D=D, Hq=Hq, Hkv=Hkv,
+                pairing=pairing, theta=10000.0)
+
+
+def _reduced(m, layer=0, **kw):
+    w = O.gather_weights(m["Wq"], m["Wk"], m["Wv"], m["tabs"], layer, m["P"], m["dv"], m["D"])
+    return O.reduced_attention_from_hidden(m["X"], w, m["tabs"]["inv_freq"][layer], m["Hq"], m["Hkv"],
+                                           m["P"], m["dv"], m["D"], **kw)
+
+
+def _full(m, layer=0, **kw):
+    return O.full_masked_attention(m["X"], m["Wq"], m["Wk"], m["Wv"], m["tabs"]["k_pair_idx"][layer],
+                                   m["tabs"]["v_idx"][layer], m["D"], m["theta"], m["pairing"],
+                                   m["Hq"], m["Hkv"], m["P"], m["dv"], **kw)
+
+
+# ---- storage rounding ------------------------------------------------------------------
+def test_round_bf16_matches_library_rounding():
+    rng = np.random.default_rng(0)
+    x = np.concatenate([rng.normal(0, 1, 5000), rng.normal(0, 1e-3, 2000), rng.normal(0, 1e4, 2000),
+                        [0.0, -0.0, 1.0, 1.00390625, 1.01171875, 3.3895314e38, 1e-40]]).astype(np.float32)
+    want = torch.from_numpy(x).to(torch.bfloat16).to(torch.float64).numpy()
+    got = O.round_bf16(x)
+    assert np.array_equal(got, want)
+    # ties go to even: 1 + 2^-8 is halfway between 1 and 1 + 2^-7
+    assert O.round_bf16(np.float32(1.00390625)) == 1.0
+    assert O.round_bf16(np.float32(1.01171875)) == 1.015625
+
+
+# ---- tables ----------------------------------------------------------------------------
+def test_counts_match_table13():
+    rows = [l.split() for l in open(os.path.join(GOLD, "table13_retained_fraction.txt"))
+            if l.strip() and not l.startswith("#")]
+    assert len(rows) == 5
+    for rho, frac in rows:
+        P, dv = O.retained_counts(float(rho), 128)
+        assert f"{P / 64:.3f}" == frac or abs(P / 64 - float(frac)) < 5.1e-4
+    # the budgets the workloads name
+    assert O.retained_counts(0.75, 64) == (24, 48)
+    assert O.retained_counts(0.9, 128) == (58, 115)
+    assert O.retained_counts(0.7, 128) == (45, 90)
+    assert O.retained_counts(1.0, 128) == (64, 128)
+    for rho, (P, dv) in synth.SWEEP_COUNTS.items():
+        assert O.retained_counts(rho, 128) == (P, dv)
+
+
+def test_bytes_per_token_table15():
+    rows = dict(l.split() for l in open(os.path.join(GOLD, "table15_bytes_per_token.txt"))
+                if l.strip() and not l.startswith("#"))
+    dense = O.kv_bytes_per_token(32, 8, 128, 128, 2)
+    assert dense == int(rows["dense"]) * 1024
+    P, dv = O.retained_counts(0.7, 128)
+    rap = O.kv_bytes_per_token(32, 8, 2 * P, dv, 2)
+    assert rap == 92160
+    assert abs(rap / 1024 - float(rows["rap0.7"])) < 1.0 and rap / dense < 0.705
+
+
+def test_cost_model_table3():
+    rows = dict((l.split()[0], l.split()[1:]) for l in open(os.path.join(GOLD, "table3_cost_model.txt"))
+                if l.strip() and not l.startswith("#"))
+    # RAP: cache, params and FLOPs of the K/V side all scale with the retained fraction.
+    S, H, D = 1000, 32, 128
+    for rho in (0.9, 0.7, 0.5):
+        P, dv = O.retained_counts(rho, D)
+        assert O.attn_read_bytes(1, 1, S, 2 * P, dv, 1) / (2 * S * D) == pytest.approx(rho, abs=0.007)
+        assert (H * D) * (2 * P + dv) / (2 * H * D * D) == pytest.approx(rho, abs=0.007)
+    assert 0.7 / (2 * 32) == pytest.approx(float(rows["palu_leftover_rho0.7_H32"][0]), abs=5e-4)
+    assert 4096 * 4096 / 1e6 == pytest.approx(float(rows["wq_millions"][0]), abs=5e-3)
+    assert 4096 * 1024 / 1e6 == pytest.approx(float(rows["wk_millions"][0]), abs=5e-3)
+
+
+def test_topk_brute_force_and_ties():
+    rng = np.random.default_rng(1)
+    for _ in range(50):
+        n = int(rng.integers(1, 12))
+        k = int(rng.integers(1, n + 1))
+        s = rng.integers(0, 4, n).astype(np.float64)          # many ties
+        got = O.top_k_ascending(s, k)
+        # brute force: repeatedly take the largest remaining, lowest index on ties
+        left, pick = list(range(n)), []
+        for _ in range(k):
+            best = left[0]
+            for i in left:
+                if s[i] > s[best]:
+                    best = i
+            pick.append(best)
+            left.remove(best)
+        assert list(got) == sorted(pick)
+    s = rng.lognormal(0, 1, 64)
+    assert list(O.top_k_ascending(s, 20)) == sorted(np.argsort(-s, kind="stable")[:20].tolist())
+    assert list(O.top_k_ascending([1.0, 5.0, 5.0, 5.0, 0.0], 2)) == [1, 2]
+
+
+@pytest.mark.parametrize("pairing", [O.PAIR_HALF, O.PAIR_ADJACENT])
+def test_selection_matrix_properties(pairing):
+    m = _small(pairing=pairing, D=16, rho=0.6)
+    D, P = m["D"], m["P"]
+    for h in range(m["Hkv"]):
+        pairs = m["tabs"]["k_pair_idx"][0, h, :P]
+        idx = m["tabs"]["k_dim_idx"][0, h, :2 * P]
+        assert np.all(np.diff(pairs) > 0) and pairs.min() >= 0 and pairs.max() < D // 2
+        assert np.all(m["tabs"]["k_pair_idx"][0, h, P:] == -1)
+        assert np.all(m["tabs"]["k_dim_idx"][0, h, 2 * P:] == -1)
+        E = O.selection_matrix(idx, D)
+        assert np.array_equal(E @ E.T, np.eye(2 * P))                 # E_k E_k^T = I
+        M = E.T @ E
+        assert np.array_equal(M, np.diag(np.diag(M))) and set(np.diag(M)) <= {0.0, 1.0}
+        # whole pairs only: both members kept or both dropped
+        for i in range(D // 2):
+            a, b = (i, i + D // 2) if pairing == O.PAIR_HALF else (2 * i, 2 * i + 1)
+            assert M[a, a] == M[b, b] == (1.0 if i in pairs else 0.0)
+        # E_k R_t = R_(t,S) E_k : selecting after the full rotation == index-aware rotation
+        x = np.random.default_rng(h).normal(size=D)
+        for t in (0, 1, 17, 4097):
+            lhs = E @ O.textbook_rope(x, t, D, m["theta"], pairing)
+            rhs = O.rope_reduced(E @ x, t, m["tabs"]["inv_freq"][0, h])
+            assert np.allclose(lhs, rhs, rtol=0, atol=1e-12)
+        # frequencies are those of the ORIGINAL pair indices
+        want = np.array([m["theta"] ** (-2.0 * i / D) for i in pairs])
+        assert np.allclose(m["tabs"]["inv_freq"][0, h, :P], want, rtol=1e-15, atol=0)
+        v = m["tabs"]["v_idx"][0, h, :m["dv"]]
+        assert np.all(np.diff(v) > 0) and v.min() >= 0 and v.max() < D
+
+
+# ---- rho = 1: nothing removed -> textbook RoPE GQA attention ----------------------------
+def _textbook_gqa(X, Wq, Wk, Wv, D, Hq, Hkv, theta):
+    """Plain rotate-half RoPE attention written with array ops, no RAP objects at all."""
+    n = X.shape[0]
+    inv = 1.0 / (theta ** (np.arange(0, D, 2) / D))
+    ang = np.arange(n)[:, None] * inv[None, :]
+    cos = np.concatenate([np.cos(ang), np.cos(ang)], axis=1)
+    sin = np.concatenate([np.sin(ang), np.sin(ang)], axis=1)
+
+    def rot(x):   # x [n][heads][D]
+        x1, x2 = x[..., : D // 2], x[..., D // 2:]
+        return x * cos[:, None, :] + np.concatenate([-x2, x1], axis=-1) * sin[:, None, :]
+
+    q = rot((X @ Wq.T).reshape(n, Hq, D))[-1]
+    k = rot((X @ Wk.T).reshape(n, Hkv, D))
+    v = (X @ Wv.T).reshape(n, Hkv, D)
+    out = np.zeros((Hq, D))
+    for g in range(Hq):
+        h = g // (Hq // Hkv)
+        s = k[:, h, :] @ q[g] / np.sqrt(D)
+        p = np.exp(s - s.max())
+        out[g] = (p / p.sum()) @ v[:, h, :]
+    return out
+
+
+def test_rho1_equals_textbook_attention():
+    m = _small(rho=1.0, D=16, Hq=6, Hkv=2, n=9)
+    out, _, _, _ = _reduced(m)
+    ref = _textbook_gqa(m["X"], m["Wq"], m["Wk"], m["Wv"], m["D"], m["Hq"], m["Hkv"], m["theta"])
+    # reduced V coordinates at rho=1 are all channels in ascending order
+    assert np.allclose(out, ref, rtol=0, atol=1e-12)
+
+
+# ---- rho < 1: reduced path == full-dimensional masked path ------------------------------
+@pytest.mark.parametrize("pairing", [O.PAIR_HALF, O.PAIR_ADJACENT])
+@pytest.mark.parametrize("rho", [0.75, 0.4])
+def test_reduced_equals_full_masked(pairing, rho):
+    m = _small(pairing=pairing, rho=rho, D=16, Hq=4, Hkv=2, n=8, seed=11)
+    out, _, _, _ = _reduced(m)
+    ref = _full(m)
+    assert np.allclose(out, ref, rtol=0, atol=1e-12)
+
+
+def test_negative_controls_break_the_identity():
+    m = _small(rho=0.5, D=16, n=8, seed=5)
+    out, _, _, _ = _reduced(m)
+    # a 1/sqrt(2P) scale is NOT what the method computes
+    wrong_scale = _full(m, scale_dim=2 * m["P"])
+    assert np.abs(out - wrong_scale).max() > 1e-4
+    # re-indexed frequencies theta^(-2c/D) (c = reduced index) are not index-aware
+    w = O.gather_weights(m["Wq"], m["Wk"], m["Wv"], m["tabs"], 0, m["P"], m["dv"], m["D"])
+    reidx = np.tile(O.textbook_inv_freq(m["D"], m["theta"])[None, :], (m["Hkv"], 1))
+    bad, _, _, _ = O.reduced_attention_from_hidden(m["X"], w, reidx, m["Hq"], m["Hkv"], m["P"], m["dv"], m["D"])
+    assert np.abs(bad - _full(m)).max() > 1e-4
+    # gathering W_q with another KV head's indices breaks it as well
+    tabs2 = {k: v.copy() for k, v in m["tabs"].items()}
+    tabs2["k_dim_idx"][0, 0], tabs2["k_dim_idx"][0, 1] = m["tabs"]["k_dim_idx"][0, 1], m["tabs"]["k_dim_idx"][0, 0]
+    assert not np.array_equal(tabs2["k_dim_idx"], m["tabs"]["k_dim_idx"])
+    w_bad = O.gather_weights(m["Wq"], m["Wk"], m["Wv"], m["tabs"], 0, m["P"], m["dv"], m["D"])
+    w_swapped = O.gather_weights(m["Wq"], m["Wk"], m["Wv"], tabs2, 0, m["P"], m["dv"], m["D"])
+    nq = m["Hq"] * 2 * m["P"]
+    w_bad[:nq] = w_swapped[:nq]          # q rows follow the wrong head, k rows the right one
+    bad, _, _, _ = O.reduced_attention_from_hidden(m["X"], w_bad, m["tabs"]["inv_freq"][0], m["Hq"], m["Hkv"],
+                                                   m["P"], m["dv"], m["D"])
+    assert np.abs(bad - _full(m)).max() > 1e-4
+
+
+# ---- R_m^T R_n = R_(n-m): per-pair relative formula, shift invariance ---------------------
+def test_per_pair_relative_rotation_identity():
+    rng = np.random.default_rng(7)
+    P = 5
+    inv = 10000.0 ** (-2.0 * np.array([0, 3, 4, 9, 15]) / 32)
+    q, k = rng.normal(size=2 * P), rng.normal(size=2 * P)
+    for m_pos, n_pos in [(0, 0), (5, 2), (100, 131), (4096, 17)]:
+        lhs = O.rope_reduced(q, m_pos, inv) @ O.rope_reduced(k, n_pos, inv)
+        rhs = 0.0
+        for c in range(P):
+            aq, bq, ak, bk = q[2 * c], q[2 * c + 1], k[2 * c], k[2 * c + 1]
+            d = (n_pos - m_pos) * inv[c]
+            rhs += (aq * ak + bq * bk) * math.cos(d) + (bq * ak - aq * bk) * math.sin(d)
+        assert lhs == pytest.approx(rhs, abs=1e-11)
+    # rotation by 0 is the identity; rotation preserves the norm of every pair
+    assert np.array_equal(O.rope_reduced(q, 0, inv), q)
+    r = O.rope_reduced(q, 77, inv)
+    assert np.allclose(r[0::2] ** 2 + r[1::2] ** 2, q[0::2] ** 2 + q[1::2] ** 2, atol=1e-12)
+    # quarter turn: (a, b) -> (-b, a) when pos * inv_freq = pi / 2
+    r = O.rope_reduced([2.0, 3.0], 1, [math.pi / 2])
+    assert r == pytest.approx([-3.0, 2.0], abs=1e-15)
+
+
+def test_position_shift_invariance():
+    m = _small(rho=0.75, D=16, n=6, seed=2)
+    w = O.gather_weights(m["Wq"], m["Wk"], m["Wv"], m["tabs"], 0, m["P"], m["dv"], m["D"])
+    n = m["X"].shape[0]
+
+    def logits(offset):
+        q, k, _ = O.qkv_rope(m["X"], w, None, np.arange(n) + offset, m["tabs"]["inv_freq"][0],
+                             m["Hq"], m["Hkv"], m["P"], m["dv"])
+        return np.array([[q[-1, g] @ k[j, g // 2] for j in range(n)] for g in range(m["Hq"])])
+
+    base = logits(0)
+    for off in (1, 1000, 100000):
+        assert np.allclose(logits(off), base, rtol=0, atol=1e-9)
+
+
+# ---- attention: brute force and closed forms ---------------------------------------------
+def test_attention_brute_force_tiny():
+    rng = np.random.default_rng(4)
+    B, Hq, Hkv, P2, dv, cap, D = 2, 4, 2, 4, 3, 5, 8
+    q = rng.normal(size=(B, Hq, P2))
+    K = rng.normal(size=(B, Hkv, cap, P2))
+    V = rng.normal(size=(B, Hkv, cap, dv))
+    lens = [3, 5]
+    got = O.decode_attn(q, K, V, lens, D)
+    for b in range(B):
+        for g in range(Hq):
+            h = g // 2
+            s = []
+            for j in range(lens[b]):
+                acc = 0.0
+                for d in range(P2):
+                    acc += q[b, g, d] * K[b, h, j, d]
+                s.append(acc / math.sqrt(D))
+            mx = max(s)
+            e = [math.exp(x - mx) for x in s]
+            z = sum(e)
+            for c in range(dv):
+                want = sum(e[j] / z * V[b, h, j, c] for j in range(lens[b]))
+                assert got[b, g, c] == pytest.approx(want, abs=1e-14)
+
+
+def test_attention_closed_forms():
+    V = np.array([[[[1.0, 2.0], [5.0, -2.0], [9.0, 9.0]]]])
+    K = np.array([[[[0.3, 0.1], [0.3, 0.1], [7.0, 7.0]]]])
+    q = np.array([[[1.0, -2.0]]])
+    # one cached token: the output is that token's V row
+    assert np.array_equal(O.decode_attn(q, K, V, [1], 4)[0, 0], [1.0, 2.0])
+    # two tokens with equal logits: the mean of the two V rows; the third row is not read
+    assert O.decode_attn(q, K, V, [2], 4)[0, 0] == pytest.approx([3.0, 0.0], abs=1e-15)
+    # scale 1/sqrt(D): logits (ln 3) * sqrt(D) / sqrt(D) -> weights 3:1
+    D = 16
+    K2 = np.array([[[[math.log(3.0) * math.sqrt(D)], [0.0]]]])
+    V2 = np.array([[[[1.0], [0.0]]]])
+    assert O.decode_attn(np.array([[[1.0]]]), K2, V2, [2], D)[0, 0, 0] == pytest.approx(0.75, abs=1e-15)
+
+
+def test_split_combine_invariance():
+    rng = np.random.default_rng(9)
+    n, P2, dv, D = 53, 6, 5, 16
+    q, K, V = rng.normal(size=P2) * 3, rng.normal(size=(n, P2)), rng.normal(size=(n, dv))
+    ref = O.decode_attn(q[None, None], K[None, None], V[None, None], [n], D)[0, 0]
+    for cuts in ([0, 53], [0, 1, 53], [0, 10, 10, 31, 53], [0, 0, 20, 53, 53]):
+        parts = [O.attn_partial(q, K[a:b], V[a:b], D) for a, b in zip(cuts[:-1], cuts[1:])]
+        assert np.allclose(O.combine_partials(parts), ref, rtol=0, atol=1e-13)
+
+
+def test_append_layout():
+    K = np.full((2, 2, 4, 2), -7.0)
+    V = np.full((2, 2, 4, 3), -7.0)
+    k_new = np.arange(8, dtype=np.float64).reshape(2, 2, 2) + 1.00390625
+    v_new = np.arange(12, dtype=np.float64).reshape(2, 2, 3)
+    O.append(K, V, k_new, v_new, seq_id=[1, 0], slot=[3, 0], dtype="bf16")
+    assert np.array_equal(K[1, :, 3, :], O.round_bf16(k_new[0])) and np.array_equal(V[0, :, 0, :], v_new[1])
+    touched = np.zeros((2, 2, 4), bool)
+    touched[1, :, 3] = touched[0, :, 0] = True
+    assert np.all(K[~touched] == -7.0) and np.all(V[~touched] == -7.0)
+
+
+# ---- low-rank comparator ------------------------------------------------------------------
+def test_lowrank_comparator_reduces_to_textbook():
+    """With B_k = E_k (a selection) and latent = unrotated reduced K, rebuilding + full RoPE
+    equals the masked full-dim attention, i.e. the RAP result."""
+    m = _small(rho=0.5, D=16, Hq=4, Hkv=2, n=6, seed=21)
+    D, P, Hkv, Hq = m["D"], m["P"], m["Hkv"], m["Hq"]
+    n = m["X"].shape[0]
+    w = O.gather_weights(m["Wq"], m["Wk"], m["Wv"], m["tabs"], 0, P, m["dv"], D)
+    y = O.project(m["X"], w)
+    off = Hq * 2 * P
+    latent = np.stack([y[:, off + h * 2 * P: off + (h + 1) * 2 * P] for h in range(Hkv)])[None]
+    off += Hkv * 2 * P
+    V = np.stack([y[:, off + h * m["dv"]: off + (h + 1) * m["dv"]] for h in range(Hkv)])[None]
+    Bk = np.stack([O.selection_matrix(m["tabs"]["k_dim_idx"][0, h, :2 * P], D) for h in range(Hkv)])
+    qfull = (m["Wq"] @ m["X"][-1]).reshape(Hq, D)
+    qrot = np.stack([O.textbook_rope(qfull[g], n - 1, D, m["theta"], m["pairing"]) for g in range(Hq)])[None]
+    got = O.lowrank_decode_attn(qrot, latent, Bk, V, [n], D, m["theta"], m["pairing"])[0]
+    assert np.allclose(got, _full(m), rtol=0, atol=1e-12)
