@@ -1,0 +1,199 @@
+/*
+ * rap.h -- C ABI of the B200-native RAP (RoPE-Aligned Pruning) decode path.
+ *
+ * The library implements the online consequence of RAP: attention over a KV cache whose
+ * K rows keep only whole retained RoPE pairs (2P dims) and whose V rows keep only
+ * retained channels (d_v' dims); the pair selection E_k is fused offline into a shrunken
+ * W~_q = W_q E_k^T, so no decode step ever rebuilds a full-width K (Section 4, Step 3;
+ * Eq. 6, Eq. 7; Algorithm 1).
+ *
+ * Conventions
+ *   - plain C; every entry point returns rap_status (0 = OK) and never throws, aborts or
+ *     traps.  Arguments are validated on the host BEFORE anything is launched.
+ *   - pointers named d_* are DEVICE pointers, h_* are HOST pointers; all are owned by the
+ *     caller.  The library owns only what rap_create allocates (a device status word, the
+ *     split-KV / projection workspace and the staging buffers of rap_decode_step_host),
+ *     released by rap_destroy.
+ *   - all GPU work is enqueued on the caller's stream (`stream` is a cudaStream_t passed as
+ *     void*, NULL = the legacy default stream) and is asynchronous unless stated otherwise.
+ *   - device buffers must be 16-byte aligned (RAP_EALIGN otherwise).
+ *   - weights are stored [out][in] row-major, so y = W x.
+ *   - notation: L layers, hidden = model width, H_q / H_kv query / KV heads, G = H_q/H_kv,
+ *     D = original head_dim, P_l retained pairs and d_v'_l retained V channels of layer l,
+ *     B batch, S_cap cache capacity in rows.
+ *   - layouts are dense-packed, no padding:
+ *       q~      [T][H_q][2P]                       (storage dtype)
+ *       K cache [B][H_kv][S_cap][2P]   per layer   (storage dtype)
+ *       V cache [B][H_kv][S_cap][d_v'] per layer   (storage dtype)
+ *       out     [B][H_q][d_v']                     (fp32, reduced V coordinates)
+ *     Reduced K/q dims are pair-interleaved: reduced dims (2c, 2c+1) are the two members of
+ *     the c-th retained pair, pairs in ascending original index.
+ */
+#ifndef RAP_H_
+#define RAP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  RAP_OK = 0,
+  RAP_EINVAL = 1,       /* NULL required pointer, bad enum, value out of range          */
+  RAP_ESHAPE = 2,       /* shape outside what the context was created for               */
+  RAP_ECAPACITY = 3,    /* a cache slot / sequence length exceeds S_cap                 */
+  RAP_EALIGN = 4,       /* device pointer not 16-byte aligned, or S_cap not multiple of 8 */
+  RAP_EUNSUPPORTED = 5, /* valid request this build does not implement                  */
+  RAP_ECUDA = 6,        /* a CUDA runtime call failed (see rap_last_cuda_error)          */
+  RAP_ETIMEOUT = 7,     /* a bounded device-side wait gave up (device status word)      */
+  RAP_ESTATE = 8        /* call order: tables not built yet for this context            */
+} rap_status;
+
+typedef enum { RAP_F32 = 0, RAP_BF16 = 1 } rap_dtype;
+
+/* RoPE pairing of the model (Section 3): pair i = dims (i, i + D/2), or (2i, 2i + 1). */
+typedef enum { RAP_PAIR_HALF = 0, RAP_PAIR_ADJACENT = 1 } rap_pairing;
+
+typedef struct {
+  int32_t n_layers, hidden, n_q_heads, n_kv_heads, head_dim; /* D even, H_q % H_kv == 0, G <= 8 */
+  double rope_theta;                                         /* theta_base of Eq. 3           */
+  int32_t pairing;                                           /* rap_pairing                   */
+  int32_t dtype;                                             /* rap_dtype of X, W~, q~, caches */
+  int32_t max_batch;                                         /* largest B of a decode call    */
+  int32_t max_rows;                                          /* largest T of an append call   */
+} rap_model_desc;
+
+typedef struct rap_ctx rap_ctx;
+
+/* Create / destroy a context.  rap_create validates the description, selects the current
+ * device and allocates the library-owned device buffers (cudaMalloc).  RAP_EINVAL on a bad
+ * description, RAP_ECUDA when no sm_100 device or an allocation fails. */
+rap_status rap_create(const rap_model_desc* desc, rap_ctx** out);
+rap_status rap_destroy(rap_ctx* ctx);
+
+const char* rap_status_string(rap_status s);
+/* Text of the last CUDA error seen by this context ("" if none). Host memory owned by ctx. */
+const char* rap_last_cuda_error(const rap_ctx* ctx);
+
+/* Per-head budget at retain ratio rho (Section 4.2 "Balanced K/V"; Table 13): whole pairs
+ * P = floor(rho*D/2 + 1/2) and V channels d_v' = floor(rho*D + 1/2), rounded independently.
+ * RAP_EINVAL unless 0 < rho <= 1 and D even. */
+rap_status rap_retained_counts(double rho, int32_t head_dim, int32_t* n_pairs, int32_t* n_vch);
+
+/* Element offset of (b, h, pos, c) in a cache of row width W: ((b*H_kv + h)*S_cap + pos)*W + c. */
+size_t rap_cache_elem_offset(int32_t n_kv_heads, int32_t S_cap, int32_t W, int32_t b, int32_t h,
+                             int32_t pos, int32_t c);
+
+/* ---- a1. tables (Algorithm 2, selection lines; Eq. 6 RAPIndex; Eq. 3 frequencies) --------
+ * For every (layer l, KV head h): keep the n_pairs[l] RoPE pairs with the largest score and
+ * the n_vch[l] V channels with the largest score (ties: lower index), each list ascending.
+ *   h_k_pair_scores [L][H_kv][D/2], h_v_chan_scores [L][H_kv][D]  HOST fp64
+ *   h_n_pairs[L] in [1, D/2], h_n_vch[L] in [1, D]                HOST
+ * Outputs are DEVICE buffers with fixed strides (unused tail = -1 / 0.0):
+ *   d_k_pair_idx int32 [L][H_kv][D/2]   retained original pair indices i_c
+ *   d_k_dim_idx  int32 [L][H_kv][D]     RAPIndex: original in-head dim of reduced dim r
+ *   d_v_idx      int32 [L][H_kv][D]     retained original V channels
+ *   d_inv_freq   fp64  [L][H_kv][D/2]   theta^(-2 i_c / D): the ORIGINAL pair's frequency
+ * The per-layer counts are recorded in the context and used by every later call.
+ * Deterministic.  Work: host selection, then async copies on `stream` from context-owned
+ * pinned memory (a later rap_build_tables on the same context first synchronizes `stream`). */
+rap_status rap_build_tables(rap_ctx* ctx, const double* h_k_pair_scores, const double* h_v_chan_scores,
+                            const int32_t* h_n_pairs, const int32_t* h_n_vch,
+                            int32_t* d_k_pair_idx, int32_t* d_k_dim_idx, int32_t* d_v_idx,
+                            double* d_inv_freq, void* stream);
+
+/* ---- a0. offline weight gather (Algorithm 1: W~_k, W~_q = W_q E_k^T, W~_v) ----------------
+ * Index selection, no arithmetic.  d_wq [H_q*D][hidden], d_wk / d_wv [H_kv*D][hidden] are the
+ * dense weights of `layer`; d_w_qkv [N_out][hidden] receives the rows
+ *   q head g: RAPIndex of KV head g/G (2P rows) | k head h: RAPIndex of h | v head h: v_idx of h,
+ * N_out = (H_q + H_kv)*2P + H_kv*d_v'.  Optional bias vectors are gathered the same way
+ * (d_bq/d_bk/d_bv -> d_bias [N_out]; pass NULL for all four when there is no bias). */
+rap_status rap_pack_weights(rap_ctx* ctx, int32_t layer, const void* d_wq, const void* d_wk,
+                            const void* d_wv, const int32_t* d_k_dim_idx, const int32_t* d_v_idx,
+                            void* d_w_qkv, const void* d_bq, const void* d_bk, const void* d_bv,
+                            void* d_bias, void* stream);
+
+/* ---- a2-a4. pruned QKV projection + index-aware RoPE + append (Eq. 1, Eq. 3, Section 4) ---
+ * T rows of hidden states.  Row r belongs to sequence d_seq_id[r] (0..B-1), sits at position
+ * d_pos[r] and is written to cache row d_slot[r].  For every row:
+ *   y = W~_qkv x (+ bias), fp32 accumulate;
+ *   q~ and k~ pairs c rotate by the angle pos * inv_freq[l][h][c] (q head g uses KV head g/G);
+ *   q~, k~, v~ are rounded once to the storage dtype; q~ -> d_q_out [T][H_q][2P],
+ *   k~ -> K cache row (seq, h, slot), v~ -> V cache row (seq, h, slot).
+ * d_bias may be NULL.  d_k_cache / d_v_cache are THIS layer's buffers with B_cache sequences.
+ * h_slot_max: the caller's upper bound on every d_slot value (RAP_ECAPACITY if >= S_cap);
+ * the kernel also skips, and records in the device status word, any row whose slot or
+ * sequence id is out of range.  T <= max_rows. */
+rap_status rap_qkv_rope_append(rap_ctx* ctx, int32_t layer, int32_t T, const void* d_x,
+                               const void* d_w_qkv, const void* d_bias, const int32_t* d_seq_id,
+                               const int32_t* d_pos, const int32_t* d_slot, int32_t h_slot_max,
+                               const double* d_inv_freq, void* d_q_out, void* d_k_cache,
+                               void* d_v_cache, int32_t B_cache, int32_t S_cap, void* stream);
+
+/* ---- a5. split-KV decode attention on the reduced dims (Eq. 2, Eq. 7, scale 1/sqrt(D)) ----
+ * For each sequence b and query head g (KV head h = g/G):
+ *   s_j = q~_g . K[b,h,j] / sqrt(D),  j in [0, d_seq_len[b]);  p = softmax(s);
+ *   out[b,g,:] = sum_j p_j V[b,h,j,:].
+ * d_seq_len[b] counts valid cache rows INCLUDING the row just appended (>= 1; a sequence
+ * with length 0 produces zeros).  h_seq_len_max: caller's bound on d_seq_len (<= S_cap).
+ * The scale uses the ORIGINAL head_dim.  n_split = 0 lets the library choose the number of
+ * sequence splits; partial (max, sum, accumulator) triples live in the context workspace,
+ * so two calls on the same context must not overlap on the GPU.  B <= max_batch. */
+rap_status rap_decode_attn(rap_ctx* ctx, int32_t layer, int32_t B, const void* d_q,
+                           const void* d_k_cache, const void* d_v_cache, int32_t S_cap,
+                           const int32_t* d_seq_len, int32_t h_seq_len_max, int32_t n_split,
+                           float* d_out, void* stream);
+
+/* ---- one decode step over all layers (a2-a5 per layer) -------------------------------------
+ * Layer l consumes d_x + l*B*hidden (one hidden-state row per sequence) and produces
+ * d_out + l*out_layer_stride ([B][H_q][d_v'_l] fp32).  d_seq_len[b] = rows cached BEFORE the
+ * step: the new token takes position = slot = d_seq_len[b] and attends over d_seq_len[b]+1
+ * rows (Eq. 2 runs over the prefix including t).  h_seq_len_max bounds d_seq_len (< S_cap).
+ * h_w_qkv / h_bias / h_k_cache / h_v_cache are HOST arrays of L device pointers (h_bias may be
+ * NULL).  d_q_scratch: caller's [B][H_q][D] storage-dtype scratch for q~.  If advance != 0 a
+ * final kernel adds 1 to every d_seq_len[b]. */
+rap_status rap_decode_step(rap_ctx* ctx, int32_t B, const void* d_x, const void* const* h_w_qkv,
+                           const void* const* h_bias, const double* d_inv_freq,
+                           void* const* h_k_cache, void* const* h_v_cache, int32_t S_cap,
+                           int32_t* d_seq_len, int32_t h_seq_len_max, int32_t n_split,
+                           void* d_q_scratch, float* d_out, size_t out_layer_stride,
+                           int32_t advance, void* stream);
+
+/* Same step with HOST input and output: h_x [L][B][hidden] (storage dtype) is copied to the
+ * device, the step runs, out is copied back to h_out [L][out_layer_stride] and the stream is
+ * synchronized before returning.  Pinned host memory makes the copies asynchronous. */
+rap_status rap_decode_step_host(rap_ctx* ctx, int32_t B, const void* h_x, const void* const* h_w_qkv,
+                                const void* const* h_bias, const double* d_inv_freq,
+                                void* const* h_k_cache, void* const* h_v_cache, int32_t S_cap,
+                                int32_t* d_seq_len, int32_t h_seq_len_max, int32_t n_split,
+                                float* h_out, size_t out_layer_stride, int32_t advance, void* stream);
+
+/* ---- comparator: low-rank cache with per-step reconstruction (Section 3) ------------------
+ * Measurement-only counterpart of a weight-side low-rank method at equal cached dims: the K
+ * cache holds UNROTATED latents [B][H_kv][S_cap][r]; every call rebuilds K_j = latent_j B_k[h]
+ * (d_bk [H_kv][r][D], storage dtype), applies full-width RoPE at position j, and attends with
+ * the full-width, already rotated d_q_full [B][H_q][D].  V side as in rap_decode_attn with
+ * row width d_v.  Output [B][H_q][d_v] fp32. */
+rap_status rap_lowrank_decode_attn(rap_ctx* ctx, int32_t B, int32_t r, int32_t d_v, const void* d_q_full,
+                                   const void* d_k_latent, const void* d_bk, const void* d_v_cache,
+                                   int32_t S_cap, const int32_t* d_seq_len, int32_t h_seq_len_max,
+                                   int32_t n_split, float* d_out, void* stream);
+
+/* Reads (and clears) the device status word after synchronizing `stream`.  code is a
+ * rap_status (RAP_OK, RAP_ECAPACITY for a skipped out-of-range row, RAP_ETIMEOUT for a bounded
+ * wait that gave up); detail identifies the row / stage. */
+rap_status rap_get_last_device_status(rap_ctx* ctx, int32_t* code, int32_t* detail, void* stream);
+
+/* Number of kernels this context has launched since creation (for launch accounting). */
+int64_t rap_kernel_launch_count(const rap_ctx* ctx);
+
+/* Forces a kernel variant for rap_decode_attn: 0 = automatic, 1 = generic kernel only.
+ * Meant for tests and profiling. */
+rap_status rap_set_attn_variant(rap_ctx* ctx, int32_t variant);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RAP_H_ */

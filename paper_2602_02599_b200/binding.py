@@ -1,0 +1,219 @@
+"""ctypes binding of the RAP decode C ABI (include/rap.h): argument marshalling only.
+
+Every function has the name of the C entry point it calls.  Tensors are torch CUDA tensors
+used as device buffers (data_ptr()), the stream is torch's current stream.  Nothing is
+computed in Python and there is no CPU fallback: a missing library raises at first use.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from ctypes import POINTER, byref, c_char_p, c_double, c_int32, c_int64, c_size_t, c_void_p
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "librap_b200.so")
+
+RAP_OK, RAP_EINVAL, RAP_ESHAPE, RAP_ECAPACITY, RAP_EALIGN, RAP_EUNSUPPORTED, RAP_ECUDA, RAP_ETIMEOUT, RAP_ESTATE = range(9)
+RAP_F32, RAP_BF16 = 0, 1
+RAP_PAIR_HALF, RAP_PAIR_ADJACENT = 0, 1
+
+EXPORTS = [
+    "rap_create", "rap_destroy", "rap_status_string", "rap_last_cuda_error", "rap_retained_counts",
+    "rap_cache_elem_offset", "rap_build_tables", "rap_pack_weights", "rap_qkv_rope_append",
+    "rap_decode_attn", "rap_decode_step", "rap_decode_step_host", "rap_lowrank_decode_attn",
+    "rap_get_last_device_status", "rap_kernel_launch_count", "rap_set_attn_variant",
+]
+
+
+class rap_model_desc(ctypes.Structure):
+    _fields_ = [("n_layers", c_int32), ("hidden", c_int32), ("n_q_heads", c_int32), ("n_kv_heads", c_int32),
+                ("head_dim", c_int32), ("rope_theta", c_double), ("pairing", c_int32), ("dtype", c_int32),
+                ("max_batch", c_int32), ("max_rows", c_int32)]
+
+
+class RapError(RuntimeError):
+    def __init__(self, status, where, detail=""):
+        self.status = status
+        msg = f"{where}: {_lib().rap_status_string(status).decode()}"
+        if detail:
+            msg += f" ({detail})"
+        super().__init__(msg)
+
+
+_LIB = None
+
+
+def _lib():
+    """Load librap_b200.so (built in-tree by build.py); raises if it is not there."""
+    global _LIB
+    if _LIB is not None:
+        return _LIB
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} is missing: run `python -m paper_2602_02599_b200.build` "
+                           "(there is no fallback path)")
+    lib = ctypes.CDLL(LIB_PATH)
+    P = c_void_p
+    lib.rap_create.argtypes = [POINTER(rap_model_desc), POINTER(P)]
+    lib.rap_destroy.argtypes = [P]
+    lib.rap_status_string.argtypes = [c_int32]
+    lib.rap_status_string.restype = c_char_p
+    lib.rap_last_cuda_error.argtypes = [P]
+    lib.rap_last_cuda_error.restype = c_char_p
+    lib.rap_retained_counts.argtypes = [c_double, c_int32, POINTER(c_int32), POINTER(c_int32)]
+    lib.rap_cache_elem_offset.argtypes = [c_int32] * 7
+    lib.rap_cache_elem_offset.restype = c_size_t
+    lib.rap_build_tables.argtypes = [P] * 10
+    lib.rap_pack_weights.argtypes = [P, c_int32] + [P] * 11
+    lib.rap_qkv_rope_append.argtypes = [P, c_int32, c_int32, P, P, P, P, P, P, c_int32, P, P, P, P, c_int32, c_int32, P]
+    lib.rap_decode_attn.argtypes = [P, c_int32, c_int32, P, P, P, c_int32, P, c_int32, c_int32, P, P]
+    lib.rap_decode_step.argtypes = [P, c_int32, P, P, P, P, P, P, c_int32, P, c_int32, c_int32, P, P, c_size_t, c_int32, P]
+    lib.rap_decode_step_host.argtypes = [P, c_int32, P, P, P, P, P, P, c_int32, P, c_int32, c_int32, P, c_size_t, c_int32, P]
+    lib.rap_lowrank_decode_attn.argtypes = [P, c_int32, c_int32, c_int32, P, P, P, P, c_int32, P, c_int32, c_int32, P, P]
+    lib.rap_get_last_device_status.argtypes = [P, POINTER(c_int32), POINTER(c_int32), P]
+    lib.rap_kernel_launch_count.argtypes = [P]
+    lib.rap_kernel_launch_count.restype = c_int64
+    lib.rap_set_attn_variant.argtypes = [P, c_int32]
+    for name in EXPORTS:
+        fn = getattr(lib, name)
+        if fn.restype is ctypes.c_int:       # default: every other entry point returns rap_status
+            fn.restype = c_int32
+    _LIB = lib
+    return lib
+
+
+def _ptr(t):
+    """Device (or host) address of a torch tensor / numpy array / raw int; None -> NULL."""
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return c_void_p(t)
+    if isinstance(t, np.ndarray):
+        return c_void_p(t.ctypes.data)
+    return c_void_p(t.data_ptr())
+
+
+def _stream():
+    import torch
+    return c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _ptr_array(tensors):
+    arr = (c_void_p * len(tensors))()
+    for i, t in enumerate(tensors):
+        arr[i] = None if t is None else (t if isinstance(t, int) else t.data_ptr())
+    return arr
+
+
+def rap_retained_counts(rho, head_dim):
+    P, dv = c_int32(), c_int32()
+    s = _lib().rap_retained_counts(rho, head_dim, byref(P), byref(dv))
+    if s:
+        raise RapError(s, "rap_retained_counts")
+    return P.value, dv.value
+
+
+def rap_cache_elem_offset(n_kv_heads, S_cap, W, b, h, pos, c):
+    return _lib().rap_cache_elem_offset(n_kv_heads, S_cap, W, b, h, pos, c)
+
+
+class RapContext:
+    """Owns one rap_ctx.  Methods are the C entry points with the ctx argument bound."""
+
+    def __init__(self, n_layers, hidden, n_q_heads, n_kv_heads, head_dim, rope_theta, pairing, dtype,
+                 max_batch, max_rows=None):
+        self.desc = rap_model_desc(n_layers, hidden, n_q_heads, n_kv_heads, head_dim, float(rope_theta),
+                                   int(pairing), int(dtype), max_batch, max_rows or max_batch)
+        self._ctx = c_void_p()
+        s = _lib().rap_create(byref(self.desc), byref(self._ctx))
+        if s:
+            detail = _lib().rap_last_cuda_error(self._ctx).decode() if self._ctx else ""
+            if self._ctx:
+                _lib().rap_destroy(self._ctx)
+                self._ctx = c_void_p()
+            raise RapError(s, "rap_create", detail)
+
+    def _check(self, s, where):
+        if s:
+            raise RapError(s, where, _lib().rap_last_cuda_error(self._ctx).decode())
+
+    def close(self):
+        if self._ctx:
+            _lib().rap_destroy(self._ctx)
+            self._ctx = c_void_p()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # ---- entry points --------------------------------------------------------------------
+    def rap_build_tables(self, k_pair_scores, v_chan_scores, n_pairs, n_vch, d_k_pair_idx, d_k_dim_idx,
+                         d_v_idx, d_inv_freq):
+        ks = np.ascontiguousarray(k_pair_scores, dtype=np.float64)
+        vs = np.ascontiguousarray(v_chan_scores, dtype=np.float64)
+        npairs = np.ascontiguousarray(n_pairs, dtype=np.int32)
+        nvch = np.ascontiguousarray(n_vch, dtype=np.int32)
+        self._check(_lib().rap_build_tables(self._ctx, _ptr(ks), _ptr(vs), _ptr(npairs), _ptr(nvch),
+                                            _ptr(d_k_pair_idx), _ptr(d_k_dim_idx), _ptr(d_v_idx),
+                                            _ptr(d_inv_freq), _stream()), "rap_build_tables")
+
+    def rap_pack_weights(self, layer, d_wq, d_wk, d_wv, d_k_dim_idx, d_v_idx, d_w_qkv,
+                         d_bq=None, d_bk=None, d_bv=None, d_bias=None):
+        self._check(_lib().rap_pack_weights(self._ctx, layer, _ptr(d_wq), _ptr(d_wk), _ptr(d_wv),
+                                            _ptr(d_k_dim_idx), _ptr(d_v_idx), _ptr(d_w_qkv), _ptr(d_bq),
+                                            _ptr(d_bk), _ptr(d_bv), _ptr(d_bias), _stream()), "rap_pack_weights")
+
+    def rap_qkv_rope_append(self, layer, T, d_x, d_w_qkv, d_bias, d_seq_id, d_pos, d_slot, h_slot_max,
+                            d_inv_freq, d_q_out, d_k_cache, d_v_cache, B_cache, S_cap):
+        self._check(_lib().rap_qkv_rope_append(self._ctx, layer, T, _ptr(d_x), _ptr(d_w_qkv), _ptr(d_bias),
+                                               _ptr(d_seq_id), _ptr(d_pos), _ptr(d_slot), h_slot_max,
+                                               _ptr(d_inv_freq), _ptr(d_q_out), _ptr(d_k_cache), _ptr(d_v_cache),
+                                               B_cache, S_cap, _stream()), "rap_qkv_rope_append")
+
+    def rap_decode_attn(self, layer, B, d_q, d_k_cache, d_v_cache, S_cap, d_seq_len, h_seq_len_max, n_split, d_out):
+        self._check(_lib().rap_decode_attn(self._ctx, layer, B, _ptr(d_q), _ptr(d_k_cache), _ptr(d_v_cache), S_cap,
+                                           _ptr(d_seq_len), h_seq_len_max, n_split, _ptr(d_out), _stream()),
+                    "rap_decode_attn")
+
+    def rap_decode_step(self, B, d_x, w_qkv, bias, d_inv_freq, k_cache, v_cache, S_cap, d_seq_len,
+                        h_seq_len_max, n_split, d_q_scratch, d_out, out_layer_stride, advance):
+        """w_qkv / bias / k_cache / v_cache: per-layer lists of tensors, or prebuilt pointer arrays."""
+        args = [a if isinstance(a, ctypes.Array) or a is None else _ptr_array(a) for a in (w_qkv, bias, k_cache, v_cache)]
+        self._check(_lib().rap_decode_step(self._ctx, B, _ptr(d_x), args[0], args[1], _ptr(d_inv_freq), args[2],
+                                           args[3], S_cap, _ptr(d_seq_len), h_seq_len_max, n_split,
+                                           _ptr(d_q_scratch), _ptr(d_out), out_layer_stride, advance, _stream()),
+                    "rap_decode_step")
+
+    def rap_decode_step_host(self, B, h_x, w_qkv, bias, d_inv_freq, k_cache, v_cache, S_cap, d_seq_len,
+                             h_seq_len_max, n_split, h_out, out_layer_stride, advance):
+        args = [a if isinstance(a, ctypes.Array) or a is None else _ptr_array(a) for a in (w_qkv, bias, k_cache, v_cache)]
+        self._check(_lib().rap_decode_step_host(self._ctx, B, _ptr(h_x), args[0], args[1], _ptr(d_inv_freq), args[2],
+                                                args[3], S_cap, _ptr(d_seq_len), h_seq_len_max, n_split,
+                                                _ptr(h_out), out_layer_stride, advance, _stream()),
+                    "rap_decode_step_host")
+
+    def rap_lowrank_decode_attn(self, B, r, d_v, d_q_full, d_k_latent, d_bk, d_v_cache, S_cap, d_seq_len,
+                                h_seq_len_max, n_split, d_out):
+        self._check(_lib().rap_lowrank_decode_attn(self._ctx, B, r, d_v, _ptr(d_q_full), _ptr(d_k_latent), _ptr(d_bk),
+                                                   _ptr(d_v_cache), S_cap, _ptr(d_seq_len), h_seq_len_max, n_split,
+                                                   _ptr(d_out), _stream()), "rap_lowrank_decode_attn")
+
+    def rap_get_last_device_status(self):
+        code, detail = c_int32(), c_int32()
+        self._check(_lib().rap_get_last_device_status(self._ctx, byref(code), byref(detail), _stream()),
+                    "rap_get_last_device_status")
+        return code.value, detail.value
+
+    def rap_kernel_launch_count(self):
+        return int(_lib().rap_kernel_launch_count(self._ctx))
+
+    def rap_set_attn_variant(self, variant):
+        self._check(_lib().rap_set_attn_variant(self._ctx, variant), "rap_set_attn_variant")
+
+
+def ptr_array(tensors):
+    """Host array of device pointers for the per-layer arguments of rap_decode_step."""
+    return _ptr_array(tensors)

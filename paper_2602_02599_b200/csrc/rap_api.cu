@@ -1,0 +1,374 @@
+// Host side of the C ABI: context life cycle, argument validation, table construction
+// (Algorithm 2 selection lines, Eq. 6, Eq. 3) and the per-layer decode loop.
+#include <algorithm>
+#include <cmath>
+#include <cstring>
+#include <new>
+#include <numeric>
+
+#include "rap_internal.h"
+
+namespace {
+
+bool desc_ok(const rap_model_desc& d) {
+  if (d.n_layers < 1 || d.hidden < 1 || d.n_q_heads < 1 || d.n_kv_heads < 1) return false;
+  if (d.head_dim < 2 || (d.head_dim & 1) || d.head_dim > 256) return false;
+  if (d.n_q_heads % d.n_kv_heads) return false;
+  if (d.n_q_heads / d.n_kv_heads > RAP_MAX_GROUP) return false;
+  if (!(d.rope_theta > 1.0) || !std::isfinite(d.rope_theta)) return false;
+  if (d.pairing != RAP_PAIR_HALF && d.pairing != RAP_PAIR_ADJACENT) return false;
+  if (d.dtype != RAP_F32 && d.dtype != RAP_BF16) return false;
+  if (d.max_batch < 1 || d.max_rows < 1) return false;
+  if ((d.hidden * rap_elem_bytes(d.dtype)) % 16) return false;   // rows of X / W~ stay 16-byte aligned
+  return true;
+}
+
+void free_all(rap_ctx* c) {
+  if (c->d_status) cudaFree(c->d_status);
+  if (c->d_attn_ws) cudaFree(c->d_attn_ws);
+  if (c->d_proj_ws) cudaFree(c->d_proj_ws);
+  if (c->d_stage_x) cudaFree(c->d_stage_x);
+  if (c->d_stage_out) cudaFree(c->d_stage_out);
+  if (c->d_stage_q) cudaFree(c->d_stage_q);
+  if (c->h_tables) cudaFreeHost(c->h_tables);
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* rap_status_string(rap_status s) {
+  switch (s) {
+    case RAP_OK: return "RAP_OK";
+    case RAP_EINVAL: return "RAP_EINVAL: invalid argument";
+    case RAP_ESHAPE: return "RAP_ESHAPE: shape outside what the context was created for";
+    case RAP_ECAPACITY: return "RAP_ECAPACITY: cache capacity exceeded";
+    case RAP_EALIGN: return "RAP_EALIGN: pointer not 16-byte aligned or S_cap not a multiple of 8";
+    case RAP_EUNSUPPORTED: return "RAP_EUNSUPPORTED: not implemented in this build";
+    case RAP_ECUDA: return "RAP_ECUDA: CUDA runtime error";
+    case RAP_ETIMEOUT: return "RAP_ETIMEOUT: bounded device wait gave up";
+    case RAP_ESTATE: return "RAP_ESTATE: rap_build_tables has not run on this context";
+  }
+  return "unknown rap_status";
+}
+
+const char* rap_last_cuda_error(const rap_ctx* ctx) { return ctx ? ctx->cuda_error.c_str() : ""; }
+
+int64_t rap_kernel_launch_count(const rap_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+rap_status rap_set_attn_variant(rap_ctx* ctx, int32_t variant) {
+  if (!ctx || variant < 0 || variant > 1) return RAP_EINVAL;
+  ctx->attn_variant = variant;
+  return RAP_OK;
+}
+
+rap_status rap_retained_counts(double rho, int32_t head_dim, int32_t* n_pairs, int32_t* n_vch) {
+  if (!n_pairs || !n_vch || !(rho > 0.0) || rho > 1.0 || head_dim < 2 || (head_dim & 1)) return RAP_EINVAL;
+  *n_pairs = (int32_t)std::floor(rho * (double)(head_dim / 2) + 0.5);
+  *n_vch = (int32_t)std::floor(rho * (double)head_dim + 0.5);
+  return RAP_OK;
+}
+
+size_t rap_cache_elem_offset(int32_t n_kv_heads, int32_t S_cap, int32_t W, int32_t b, int32_t h,
+                             int32_t pos, int32_t c) {
+  return (((size_t)b * (size_t)n_kv_heads + (size_t)h) * (size_t)S_cap + (size_t)pos) * (size_t)W + (size_t)c;
+}
+
+rap_status rap_create(const rap_model_desc* desc, rap_ctx** out) {
+  if (!desc || !out) return RAP_EINVAL;
+  *out = nullptr;
+  if (!desc_ok(*desc)) return RAP_EINVAL;
+  rap_ctx* c = new (std::nothrow) rap_ctx();
+  if (!c) return RAP_EINVAL;
+  c->desc = *desc;
+  c->n_pairs.assign(desc->n_layers, 0);
+  c->n_vch.assign(desc->n_layers, 0);
+  // From here on errors are reported through a context the caller can inspect and destroy.
+  *out = c;
+  RAP_CUDA_TRY(c, cudaGetDevice(&c->device));
+  cudaDeviceProp prop;
+  RAP_CUDA_TRY(c, cudaGetDeviceProperties(&prop, c->device));
+  if (prop.major != 10) {
+    c->cuda_error = "device is not sm_100 (B200) -- this library carries sm_100a code only";
+    return RAP_ECUDA;
+  }
+  c->sm_count = prop.multiProcessorCount;
+  const rap_model_desc& d = c->desc;
+  const size_t e = rap_elem_bytes(d.dtype);
+  const size_t n_out_max = (size_t)(d.n_q_heads + 2 * d.n_kv_heads) * d.head_dim;
+  c->attn_ws_bytes = (size_t)d.max_batch * d.n_q_heads * RAP_MAX_SPLIT * (size_t)(d.head_dim + 2) * sizeof(float);
+  c->proj_ws_bytes = (size_t)d.max_rows * n_out_max * sizeof(float) * RAP_MAX_KSPLIT;
+  c->stage_x_bytes = (size_t)d.n_layers * d.max_batch * d.hidden * e;
+  c->stage_out_bytes = (size_t)d.n_layers * d.max_batch * d.n_q_heads * d.head_dim * sizeof(float);
+  RAP_CUDA_TRY(c, cudaMalloc(&c->d_status, 2 * sizeof(int32_t)));
+  RAP_CUDA_TRY(c, cudaMemset(c->d_status, 0, 2 * sizeof(int32_t)));
+  RAP_CUDA_TRY(c, cudaMalloc(&c->d_attn_ws, c->attn_ws_bytes));
+  RAP_CUDA_TRY(c, cudaMalloc(&c->d_proj_ws, c->proj_ws_bytes));
+  RAP_CUDA_TRY(c, cudaMalloc(&c->d_stage_x, c->stage_x_bytes));
+  RAP_CUDA_TRY(c, cudaMalloc(&c->d_stage_out, c->stage_out_bytes));
+  RAP_CUDA_TRY(c, cudaMalloc(&c->d_stage_q, (size_t)d.max_batch * d.n_q_heads * d.head_dim * e));
+  const size_t units = (size_t)d.n_layers * d.n_kv_heads;
+  c->h_tables_bytes = units * ((size_t)(d.head_dim / 2 + 2 * d.head_dim) * sizeof(int32_t) +
+                               (size_t)(d.head_dim / 2) * sizeof(double));
+  RAP_CUDA_TRY(c, cudaMallocHost(&c->h_tables, c->h_tables_bytes));
+  return RAP_OK;
+}
+
+rap_status rap_destroy(rap_ctx* ctx) {
+  if (!ctx) return RAP_EINVAL;
+  if (ctx->tables_inflight) cudaStreamSynchronize((cudaStream_t)ctx->tables_stream);
+  free_all(ctx);
+  delete ctx;
+  return RAP_OK;
+}
+
+rap_status rap_build_tables(rap_ctx* ctx, const double* ks, const double* vs, const int32_t* n_pairs,
+                            const int32_t* n_vch, int32_t* d_k_pair_idx, int32_t* d_k_dim_idx,
+                            int32_t* d_v_idx, double* d_inv_freq, void* stream) {
+  if (!ctx || !ks || !vs || !n_pairs || !n_vch || !d_k_pair_idx || !d_k_dim_idx || !d_v_idx || !d_inv_freq)
+    return RAP_EINVAL;
+  if (!rap_aligned16(d_k_pair_idx) || !rap_aligned16(d_k_dim_idx) || !rap_aligned16(d_v_idx) ||
+      !rap_aligned16(d_inv_freq))
+    return RAP_EALIGN;
+  const rap_model_desc& d = ctx->desc;
+  const int L = d.n_layers, H = d.n_kv_heads, D = d.head_dim, half = D / 2;
+  for (int l = 0; l < L; ++l) {
+    if (n_pairs[l] < 1 || n_pairs[l] > half || n_vch[l] < 1 || n_vch[l] > D) return RAP_EINVAL;
+  }
+  const size_t units = (size_t)L * H;
+  for (size_t i = 0; i < units * half; ++i) if (std::isnan(ks[i])) return RAP_EINVAL;
+  for (size_t i = 0; i < units * D; ++i) if (std::isnan(vs[i])) return RAP_EINVAL;
+  cudaStream_t st = (cudaStream_t)stream;
+  if (ctx->tables_inflight) {
+    RAP_CUDA_TRY(ctx, cudaStreamSynchronize((cudaStream_t)ctx->tables_stream));
+    ctx->tables_inflight = false;
+  }
+  int32_t* h_pair = (int32_t*)ctx->h_tables;
+  int32_t* h_dim = h_pair + units * half;
+  int32_t* h_v = h_dim + units * D;
+  double* h_freq = (double*)(h_v + units * D);   // offset is a multiple of 8 bytes: (half + 2D) * 4 * units
+  std::fill(h_pair, h_pair + units * half, -1);
+  std::fill(h_dim, h_dim + units * D, -1);
+  std::fill(h_v, h_v + units * D, -1);
+  std::fill(h_freq, h_freq + units * half, 0.0);
+
+  std::vector<int32_t> order;
+  auto top_k = [&order](const double* s, int n, int k, int32_t* dst) {
+    order.resize(n);
+    std::iota(order.begin(), order.end(), 0);
+    // larger score first; equal scores keep the lower index first
+    std::stable_sort(order.begin(), order.end(), [s](int32_t a, int32_t b) { return s[a] > s[b]; });
+    std::sort(order.begin(), order.begin() + k);
+    std::copy(order.begin(), order.begin() + k, dst);
+  };
+  for (int l = 0; l < L; ++l) {
+    const int P = n_pairs[l], dv = n_vch[l];
+    for (int h = 0; h < H; ++h) {
+      const size_t u = (size_t)l * H + h;
+      int32_t* pr = h_pair + u * half;
+      top_k(ks + u * half, half, P, pr);
+      for (int c = 0; c < P; ++c) {
+        const int i = pr[c];
+        if (d.pairing == RAP_PAIR_HALF) {
+          h_dim[u * D + 2 * c] = i;
+          h_dim[u * D + 2 * c + 1] = i + half;
+        } else {
+          h_dim[u * D + 2 * c] = 2 * i;
+          h_dim[u * D + 2 * c + 1] = 2 * i + 1;
+        }
+        h_freq[u * half + c] = std::pow(d.rope_theta, -2.0 * (double)i / (double)D);
+      }
+      top_k(vs + u * D, D, dv, h_v + u * D);
+    }
+  }
+  RAP_CUDA_TRY(ctx, cudaMemcpyAsync(d_k_pair_idx, h_pair, units * half * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+  RAP_CUDA_TRY(ctx, cudaMemcpyAsync(d_k_dim_idx, h_dim, units * D * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+  RAP_CUDA_TRY(ctx, cudaMemcpyAsync(d_v_idx, h_v, units * D * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+  RAP_CUDA_TRY(ctx, cudaMemcpyAsync(d_inv_freq, h_freq, units * half * sizeof(double), cudaMemcpyHostToDevice, st));
+  ctx->tables_inflight = true;
+  ctx->tables_stream = stream;
+  for (int l = 0; l < L; ++l) {
+    ctx->n_pairs[l] = n_pairs[l];
+    ctx->n_vch[l] = n_vch[l];
+  }
+  ctx->tables_built = true;
+  return RAP_OK;
+}
+
+rap_status rap_pack_weights(rap_ctx* ctx, int32_t layer, const void* d_wq, const void* d_wk, const void* d_wv,
+                            const int32_t* d_k_dim_idx, const int32_t* d_v_idx, void* d_w_qkv,
+                            const void* d_bq, const void* d_bk, const void* d_bv, void* d_bias, void* stream) {
+  if (!ctx || !d_wq || !d_wk || !d_wv || !d_k_dim_idx || !d_v_idx || !d_w_qkv) return RAP_EINVAL;
+  if (!ctx->tables_built) return RAP_ESTATE;
+  if (layer < 0 || layer >= ctx->desc.n_layers) return RAP_EINVAL;
+  const bool any_b = d_bq || d_bk || d_bv || d_bias, all_b = d_bq && d_bk && d_bv && d_bias;
+  if (any_b && !all_b) return RAP_EINVAL;
+  if (!rap_aligned16(d_wq) || !rap_aligned16(d_wk) || !rap_aligned16(d_wv) || !rap_aligned16(d_w_qkv))
+    return RAP_EALIGN;
+  return rap_launch_pack(ctx, layer, d_wq, d_wk, d_wv, d_k_dim_idx, d_v_idx, d_w_qkv, d_bq, d_bk, d_bv,
+                         d_bias, (cudaStream_t)stream);
+}
+
+rap_status rap_qkv_rope_append(rap_ctx* ctx, int32_t layer, int32_t T, const void* d_x, const void* d_w_qkv,
+                               const void* d_bias, const int32_t* d_seq_id, const int32_t* d_pos,
+                               const int32_t* d_slot, int32_t h_slot_max, const double* d_inv_freq,
+                               void* d_q_out, void* d_k_cache, void* d_v_cache, int32_t B_cache,
+                               int32_t S_cap, void* stream) {
+  if (!ctx || !d_x || !d_w_qkv || !d_seq_id || !d_pos || !d_slot || !d_inv_freq || !d_q_out || !d_k_cache ||
+      !d_v_cache)
+    return RAP_EINVAL;
+  if (!ctx->tables_built) return RAP_ESTATE;
+  const rap_model_desc& d = ctx->desc;
+  if (layer < 0 || layer >= d.n_layers || T < 0 || B_cache < 1 || S_cap < 1) return RAP_EINVAL;
+  if (T > d.max_rows) return RAP_ESHAPE;
+  if (S_cap % 8) return RAP_EALIGN;
+  if (h_slot_max < 0) return RAP_EINVAL;
+  if (h_slot_max >= S_cap) return RAP_ECAPACITY;
+  if (!rap_aligned16(d_x) || !rap_aligned16(d_w_qkv) || !rap_aligned16(d_q_out) || !rap_aligned16(d_k_cache) ||
+      !rap_aligned16(d_v_cache) || !rap_aligned16(d_inv_freq) || (d_bias && !rap_aligned16(d_bias)))
+    return RAP_EALIGN;
+  if (T == 0) return RAP_OK;
+  rap_proj_args a;
+  a.x = d_x; a.w = d_w_qkv; a.bias = d_bias;
+  a.seq_id = d_seq_id; a.pos = d_pos; a.slot = d_slot;
+  a.inv_freq = d_inv_freq + (size_t)layer * d.n_kv_heads * (d.head_dim / 2);
+  a.q_out = d_q_out; a.k_cache = d_k_cache; a.v_cache = d_v_cache;
+  a.T = T; a.hidden = d.hidden; a.Hq = d.n_q_heads; a.Hkv = d.n_kv_heads;
+  a.P2 = 2 * ctx->n_pairs[layer]; a.dv = ctx->n_vch[layer]; a.half_dim = d.head_dim / 2;
+  a.B_cache = B_cache; a.S_cap = S_cap; a.dtype = d.dtype;
+  return rap_launch_qkv_rope_append(ctx, a, (cudaStream_t)stream);
+}
+
+rap_status rap_decode_attn(rap_ctx* ctx, int32_t layer, int32_t B, const void* d_q, const void* d_k_cache,
+                           const void* d_v_cache, int32_t S_cap, const int32_t* d_seq_len,
+                           int32_t h_seq_len_max, int32_t n_split, float* d_out, void* stream) {
+  if (!ctx || !d_q || !d_k_cache || !d_v_cache || !d_seq_len || !d_out) return RAP_EINVAL;
+  if (!ctx->tables_built) return RAP_ESTATE;
+  const rap_model_desc& d = ctx->desc;
+  if (layer < 0 || layer >= d.n_layers || B < 0 || S_cap < 1 || n_split < 0 || h_seq_len_max < 0) return RAP_EINVAL;
+  if (B > d.max_batch || n_split > RAP_MAX_SPLIT) return RAP_ESHAPE;
+  if (S_cap % 8) return RAP_EALIGN;
+  if (h_seq_len_max > S_cap) return RAP_ECAPACITY;
+  if (!rap_aligned16(d_q) || !rap_aligned16(d_k_cache) || !rap_aligned16(d_v_cache) || !rap_aligned16(d_out) ||
+      !rap_aligned16(d_seq_len))
+    return RAP_EALIGN;
+  if (B == 0) return RAP_OK;
+  rap_attn_args a;
+  a.q = d_q; a.k = d_k_cache; a.v = d_v_cache; a.seq_len = d_seq_len; a.len_add = 0;
+  a.B = B; a.Hq = d.n_q_heads; a.Hkv = d.n_kv_heads; a.P2 = 2 * ctx->n_pairs[layer]; a.dv = ctx->n_vch[layer];
+  a.S_cap = S_cap; a.head_dim = d.head_dim; a.dtype = d.dtype; a.n_split = n_split; a.h_len_max = h_seq_len_max;
+  a.out = d_out;
+  return rap_launch_attn(ctx, a, (cudaStream_t)stream);
+}
+
+rap_status rap_decode_step(rap_ctx* ctx, int32_t B, const void* d_x, const void* const* h_w_qkv,
+                           const void* const* h_bias, const double* d_inv_freq, void* const* h_k_cache,
+                           void* const* h_v_cache, int32_t S_cap, int32_t* d_seq_len, int32_t h_seq_len_max,
+                           int32_t n_split, void* d_q_scratch, float* d_out, size_t out_layer_stride,
+                           int32_t advance, void* stream) {
+  if (!ctx || !d_x || !h_w_qkv || !d_inv_freq || !h_k_cache || !h_v_cache || !d_seq_len || !d_q_scratch || !d_out)
+    return RAP_EINVAL;
+  if (!ctx->tables_built) return RAP_ESTATE;
+  const rap_model_desc& d = ctx->desc;
+  if (B < 0 || S_cap < 1 || n_split < 0 || h_seq_len_max < 0) return RAP_EINVAL;
+  if (B > d.max_batch || B > d.max_rows || n_split > RAP_MAX_SPLIT) return RAP_ESHAPE;
+  if (S_cap % 8) return RAP_EALIGN;
+  if (h_seq_len_max >= S_cap) return RAP_ECAPACITY;
+  if (!rap_aligned16(d_x) || !rap_aligned16(d_inv_freq) || !rap_aligned16(d_seq_len) || !rap_aligned16(d_q_scratch) ||
+      !rap_aligned16(d_out) || (out_layer_stride % 4))
+    return RAP_EALIGN;
+  for (int l = 0; l < d.n_layers; ++l) {
+    if (!h_w_qkv[l] || !h_k_cache[l] || !h_v_cache[l]) return RAP_EINVAL;
+    if (out_layer_stride < (size_t)B * d.n_q_heads * ctx->n_vch[l]) return RAP_ESHAPE;
+    if (!rap_aligned16(h_w_qkv[l]) || !rap_aligned16(h_k_cache[l]) || !rap_aligned16(h_v_cache[l]) ||
+        (h_bias && h_bias[l] && !rap_aligned16(h_bias[l])))
+      return RAP_EALIGN;
+  }
+  if (B == 0) return RAP_OK;
+  cudaStream_t st = (cudaStream_t)stream;
+  const size_t e = rap_elem_bytes(d.dtype);
+  for (int l = 0; l < d.n_layers; ++l) {
+    rap_proj_args p;
+    p.x = (const char*)d_x + (size_t)l * B * d.hidden * e;
+    p.w = h_w_qkv[l]; p.bias = h_bias ? h_bias[l] : nullptr;
+    p.seq_id = nullptr; p.pos = d_seq_len; p.slot = nullptr;   // decode mode: row r = sequence r at pos = slot = len
+    p.inv_freq = d_inv_freq + (size_t)l * d.n_kv_heads * (d.head_dim / 2);
+    p.q_out = d_q_scratch; p.k_cache = h_k_cache[l]; p.v_cache = h_v_cache[l];
+    p.T = B; p.hidden = d.hidden; p.Hq = d.n_q_heads; p.Hkv = d.n_kv_heads;
+    p.P2 = 2 * ctx->n_pairs[l]; p.dv = ctx->n_vch[l]; p.half_dim = d.head_dim / 2;
+    p.B_cache = B; p.S_cap = S_cap; p.dtype = d.dtype;
+    rap_status s = rap_launch_qkv_rope_append(ctx, p, st);
+    if (s != RAP_OK) return s;
+    rap_attn_args a;
+    a.q = d_q_scratch; a.k = h_k_cache[l]; a.v = h_v_cache[l]; a.seq_len = d_seq_len; a.len_add = 1;
+    a.B = B; a.Hq = d.n_q_heads; a.Hkv = d.n_kv_heads; a.P2 = p.P2; a.dv = p.dv; a.S_cap = S_cap;
+    a.head_dim = d.head_dim; a.dtype = d.dtype; a.n_split = n_split; a.h_len_max = h_seq_len_max + 1;
+    a.out = d_out + (size_t)l * out_layer_stride;
+    s = rap_launch_attn(ctx, a, st);
+    if (s != RAP_OK) return s;
+  }
+  if (advance) return rap_launch_advance(ctx, d_seq_len, B, st);
+  return RAP_OK;
+}
+
+rap_status rap_decode_step_host(rap_ctx* ctx, int32_t B, const void* h_x, const void* const* h_w_qkv,
+                                const void* const* h_bias, const double* d_inv_freq, void* const* h_k_cache,
+                                void* const* h_v_cache, int32_t S_cap, int32_t* d_seq_len, int32_t h_seq_len_max,
+                                int32_t n_split, float* h_out, size_t out_layer_stride, int32_t advance,
+                                void* stream) {
+  if (!ctx || !h_x || !h_out) return RAP_EINVAL;
+  const rap_model_desc& d = ctx->desc;
+  if (B < 0) return RAP_EINVAL;
+  if (B > d.max_batch) return RAP_ESHAPE;
+  if (out_layer_stride > (size_t)d.max_batch * d.n_q_heads * d.head_dim) return RAP_ESHAPE;
+  cudaStream_t st = (cudaStream_t)stream;
+  const size_t xb = (size_t)d.n_layers * B * d.hidden * rap_elem_bytes(d.dtype);
+  const size_t ob = (size_t)d.n_layers * out_layer_stride * sizeof(float);
+  if (B == 0) return RAP_OK;
+  RAP_CUDA_TRY(ctx, cudaMemcpyAsync(ctx->d_stage_x, h_x, xb, cudaMemcpyHostToDevice, st));
+  rap_status s = rap_decode_step(ctx, B, ctx->d_stage_x, h_w_qkv, h_bias, d_inv_freq, h_k_cache, h_v_cache, S_cap,
+                                 d_seq_len, h_seq_len_max, n_split, ctx->d_stage_q, ctx->d_stage_out,
+                                 out_layer_stride, advance, stream);
+  if (s != RAP_OK) return s;
+  RAP_CUDA_TRY(ctx, cudaMemcpyAsync(h_out, ctx->d_stage_out, ob, cudaMemcpyDeviceToHost, st));
+  RAP_CUDA_TRY(ctx, cudaStreamSynchronize(st));
+  return RAP_OK;
+}
+
+rap_status rap_lowrank_decode_attn(rap_ctx* ctx, int32_t B, int32_t r, int32_t d_v, const void* d_q_full,
+                                   const void* d_k_latent, const void* d_bk, const void* d_v_cache, int32_t S_cap,
+                                   const int32_t* d_seq_len, int32_t h_seq_len_max, int32_t n_split, float* d_out,
+                                   void* stream) {
+  if (!ctx || !d_q_full || !d_k_latent || !d_bk || !d_v_cache || !d_seq_len || !d_out) return RAP_EINVAL;
+  const rap_model_desc& d = ctx->desc;
+  if (B < 0 || r < 1 || r > d.head_dim || d_v < 1 || d_v > d.head_dim || S_cap < 1 || n_split < 0 ||
+      h_seq_len_max < 0)
+    return RAP_EINVAL;
+  if (B > d.max_batch || n_split > RAP_MAX_SPLIT) return RAP_ESHAPE;
+  if (S_cap % 8) return RAP_EALIGN;
+  if (h_seq_len_max > S_cap) return RAP_ECAPACITY;
+  if (!rap_aligned16(d_q_full) || !rap_aligned16(d_k_latent) || !rap_aligned16(d_bk) || !rap_aligned16(d_v_cache) ||
+      !rap_aligned16(d_out) || !rap_aligned16(d_seq_len))
+    return RAP_EALIGN;
+  if (B == 0) return RAP_OK;
+  rap_lowrank_args a;
+  a.q_full = d_q_full; a.k_latent = d_k_latent; a.bk = d_bk; a.v = d_v_cache; a.seq_len = d_seq_len;
+  a.B = B; a.Hq = d.n_q_heads; a.Hkv = d.n_kv_heads; a.r = r; a.dv = d_v; a.S_cap = S_cap;
+  a.head_dim = d.head_dim; a.dtype = d.dtype; a.pairing = d.pairing; a.rope_theta = d.rope_theta;
+  a.n_split = n_split; a.h_len_max = h_seq_len_max; a.out = d_out;
+  return rap_launch_lowrank_attn(ctx, a, (cudaStream_t)stream);
+}
+
+rap_status rap_get_last_device_status(rap_ctx* ctx, int32_t* code, int32_t* detail, void* stream) {
+  if (!ctx || !code || !detail) return RAP_EINVAL;
+  int32_t h[2] = {0, 0};
+  cudaStream_t st = (cudaStream_t)stream;
+  RAP_CUDA_TRY(ctx, cudaMemcpyAsync(h, ctx->d_status, sizeof(h), cudaMemcpyDeviceToHost, st));
+  RAP_CUDA_TRY(ctx, cudaMemsetAsync(ctx->d_status, 0, sizeof(h), st));
+  RAP_CUDA_TRY(ctx, cudaStreamSynchronize(st));
+  *code = h[0];
+  *detail = h[1];
+  return RAP_OK;
+}
+
+}  // extern "C"

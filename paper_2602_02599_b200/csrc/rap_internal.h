@@ -1,0 +1,87 @@
+// Internal declarations shared by the translation units of the RAP decode library.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+#include <string>
+#include <vector>
+
+#include "rap.h"
+
+#define RAP_MAX_SPLIT 64     // upper bound on sequence splits of the attention scan
+#define RAP_MAX_GROUP 8      // largest G = H_q / H_kv
+#define RAP_MAX_KSPLIT 8     // upper bound on reduction splits of the projection
+
+struct rap_ctx {
+  rap_model_desc desc;
+  int device = 0;
+  int sm_count = 0;
+  bool tables_built = false;
+  std::vector<int32_t> n_pairs;   // P_l
+  std::vector<int32_t> n_vch;     // d_v'_l
+  // library-owned device memory
+  int32_t* d_status = nullptr;    // [2] = {code, detail}
+  float* d_attn_ws = nullptr;     // split-KV partials
+  size_t attn_ws_bytes = 0;
+  float* d_proj_ws = nullptr;     // fp32 projection results / split-K partials
+  size_t proj_ws_bytes = 0;
+  void* d_stage_x = nullptr;      // staging for rap_decode_step_host
+  float* d_stage_out = nullptr;
+  void* d_stage_q = nullptr;
+  size_t stage_x_bytes = 0, stage_out_bytes = 0;
+  // pinned host staging for rap_build_tables
+  void* h_tables = nullptr;
+  size_t h_tables_bytes = 0;
+  void* tables_stream = nullptr;
+  bool tables_inflight = false;
+  int32_t attn_variant = 0;
+  int64_t launches = 0;
+  std::string cuda_error;
+  // lazily created tensor maps / per-device attributes live in the .cu files
+  bool smem_attr_set = false;
+};
+
+static inline int rap_elem_bytes(int32_t dtype) { return dtype == RAP_F32 ? 4 : 2; }
+static inline bool rap_aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+#define RAP_CUDA_TRY(ctx, expr)                                         \
+  do {                                                                  \
+    cudaError_t _e = (expr);                                            \
+    if (_e != cudaSuccess) {                                            \
+      (ctx)->cuda_error = std::string(#expr) + ": " + cudaGetErrorString(_e); \
+      return RAP_ECUDA;                                                 \
+    }                                                                   \
+  } while (0)
+
+// Launchers implemented in the kernel files.  All return RAP_OK or RAP_ECUDA.
+struct rap_attn_args {
+  const void* q; const void* k; const void* v;
+  const int32_t* seq_len; int32_t len_add;      // effective length = seq_len[b] + len_add
+  int32_t B, Hq, Hkv, P2, dv, S_cap, head_dim, dtype;
+  int32_t n_split, h_len_max;
+  float* out;
+};
+rap_status rap_launch_attn(rap_ctx* ctx, const rap_attn_args& a, cudaStream_t st);
+
+struct rap_proj_args {
+  const void* x; const void* w; const void* bias;
+  const int32_t* seq_id; const int32_t* pos; const int32_t* slot;   // seq_id/slot NULL => decode mode
+  const double* inv_freq;   // this layer's [H_kv][D/2]
+  void* q_out; void* k_cache; void* v_cache;
+  int32_t T, hidden, Hq, Hkv, P2, dv, half_dim, B_cache, S_cap, dtype;
+};
+rap_status rap_launch_qkv_rope_append(rap_ctx* ctx, const rap_proj_args& a, cudaStream_t st);
+
+struct rap_lowrank_args {
+  const void* q_full; const void* k_latent; const void* bk; const void* v;
+  const int32_t* seq_len; int32_t B, Hq, Hkv, r, dv, S_cap, head_dim, dtype, pairing;
+  double rope_theta; int32_t n_split, h_len_max; float* out;
+};
+rap_status rap_launch_lowrank_attn(rap_ctx* ctx, const rap_lowrank_args& a, cudaStream_t st);
+
+rap_status rap_launch_pack(rap_ctx* ctx, int32_t layer, const void* wq, const void* wk, const void* wv,
+                           const int32_t* k_dim_idx, const int32_t* v_idx, void* w_qkv,
+                           const void* bq, const void* bk, const void* bv, void* bias, cudaStream_t st);
+rap_status rap_launch_advance(rap_ctx* ctx, int32_t* seq_len, int32_t B, cudaStream_t st);

@@ -1,0 +1,278 @@
+"""Parity of the CUDA path (through the C ABI) against the CPU oracle, on the same seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import rap_oracle as O
+from paper_2602_02599_b200 import binding, synth
+from paper_2602_02599_b200.stack import DecodeStack
+
+import util
+
+pytestmark = pytest.mark.gpu
+
+
+def _tables_equal(st, tabs):
+    torch.cuda.synchronize()
+    assert np.array_equal(st.k_pair_idx.cpu().numpy(), tabs["k_pair_idx"])
+    assert np.array_equal(st.k_dim_idx.cpu().numpy(), tabs["k_dim_idx"])
+    assert np.array_equal(st.v_idx.cpu().numpy(), tabs["v_idx"])
+    got, want = st.inv_freq.cpu().numpy(), tabs["inv_freq"]
+    assert np.allclose(got, want, rtol=4e-16, atol=0)
+
+
+@pytest.mark.parametrize("name", ["tiny", "3b", "8b", "14b", "sweep0.5", "sweep1.0"])
+def test_tables_bit_exact_all_layers(name):
+    w = synth.CONFIGS[name]
+    ks, vs = synth.draw_scores(w)
+    st = DecodeStack(w, batch=1, s_cap=8, alloc_cache=False)
+    st.build_tables(ks, vs)
+    _tables_equal(st, util.oracle_tables(w, ks, vs))
+    st.close()
+
+
+def test_tables_ties_adjacent_pairing_and_per_layer_budgets():
+    from dataclasses import replace
+    w = replace(synth.TINY, n_layers=3, pairing=1)
+    rng = np.random.default_rng(5)
+    ks = rng.integers(0, 3, (3, 2, 32)).astype(np.float64)        # heavy ties
+    vs = rng.integers(0, 3, (3, 2, 64)).astype(np.float64)
+    n_pairs, n_vch = [32, 1, 17], [1, 64, 33]
+    st = DecodeStack(w, n_pairs=n_pairs, n_vch=n_vch, batch=1, s_cap=8, alloc_cache=False)
+    st.build_tables(ks, vs)
+    _tables_equal(st, util.oracle_tables(w, ks, vs, n_pairs, n_vch))
+    st.close()
+
+
+def test_pack_weights_bit_exact():
+    w = synth.scaled_down(synth.LLAMA_8B, n_layers=2, batch=1, seq=8, hidden=256)
+    ks, vs = synth.draw_scores(w)
+    st, tabs, w_host = util.build_small_stack(w, ks, vs, full_weights=True)
+    for l in range(w.n_layers):
+        assert np.array_equal(util.to_np64(st.w_qkv[l]), w_host[l])
+    st.close()
+
+
+def _end_to_end(w, lens_before, n_split=0, with_bias=False, chunk=None):
+    """Prefill lens_before[b] tokens per sequence, then one decode step; compare every stage."""
+    ks, vs = synth.draw_scores(w)
+    T_pre = int(np.sum(lens_before))
+    st, tabs, w_host = util.build_small_stack(w, ks, vs, full_weights=True, max_rows=max(chunk or T_pre, w.batch))
+    B, Hq, Hkv, D = w.batch, w.n_q_heads, w.n_kv_heads, w.head_dim
+    bias_host = None
+    if with_bias:
+        bias_host, st.bias = [], []
+        for l in range(w.n_layers):
+            b = synth.draw_bias(w, l, st.n_out(l))
+            st.bias.append(torch.from_numpy(b).to(st.device).to(st.dt))
+            bias_host.append(O.round_storage(b, w.dtype))
+    caches = util.prefill_both(st, tabs, w_host, w, lens_before, chunk=chunk) if not with_bias else None
+    if with_bias:   # bias path: empty caches, first token only
+        caches = [(np.zeros((B, Hkv, st.s_cap, 2 * st.n_pairs[l])), np.zeros((B, Hkv, st.s_cap, st.n_vch[l])))
+                  for l in range(w.n_layers)]
+        for l in range(w.n_layers):
+            st.k_cache[l].zero_(); st.v_cache[l].zero_()
+        lens_before = np.zeros(B, dtype=np.int32)
+    lens_before = np.asarray(lens_before, dtype=np.int32)
+    st.seq_len.copy_(torch.from_numpy(lens_before))
+    X = np.stack([synth.draw_hidden(w, l, 1, B) for l in range(w.n_layers)])
+    dx = torch.from_numpy(X).to(st.device).to(st.dt).contiguous()
+    # canaries around what the step may write
+    for l in range(w.n_layers):
+        for b in range(B):
+            st.k_cache[l][b, :, lens_before[b] + 1:, :] = -77.0
+            st.v_cache[l][b, :, lens_before[b] + 1:, :] = -77.0
+    before = [(st.k_cache[l].clone(), st.v_cache[l].clone()) for l in range(w.n_layers)]
+    st.decode_step(dx, int(lens_before.max()), n_split=n_split, advance=1)
+    torch.cuda.synchronize()
+    assert st.ctx.rap_get_last_device_status() == (0, 0)
+    assert np.array_equal(st.seq_len.cpu().numpy(), lens_before + 1)
+    worst = 0.0
+    for l in range(w.n_layers):
+        P, dv = st.n_pairs[l], st.n_vch[l]
+        Xr = O.round_storage(X[l], w.dtype)
+        q, k, v = O.qkv_rope(Xr, w_host[l], None if bias_host is None else bias_host[l], lens_before,
+                             tabs["inv_freq"][l], Hq, Hkv, P, dv)
+        Kd, Vd = util.to_np64(st.k_cache[l]), util.to_np64(st.v_cache[l])
+        Kb, Vb = util.to_np64(before[l][0]), util.to_np64(before[l][1])
+        # slot layout: exactly the rows (b, :, len_b) changed
+        changed_k = np.any(Kd != Kb, axis=-1)
+        changed_v = np.any(Vd != Vb, axis=-1)
+        expect = np.zeros_like(changed_k)
+        for b in range(B):
+            expect[b, :, lens_before[b]] = True
+        assert np.array_equal(changed_k | expect, expect) and np.array_equal(changed_v | expect, expect)
+        k_dev = np.stack([Kd[b, :, lens_before[b], :] for b in range(B)])
+        v_dev = np.stack([Vd[b, :, lens_before[b], :] for b in range(B)])
+        util.check_projection(k_dev, O.round_storage(k, w.dtype), w.dtype, f"k layer {l}")
+        util.check_projection(v_dev, O.round_storage(v, w.dtype), w.dtype, f"v layer {l}")
+        # attention judged on the device's own rounded q~ and cache rows (a2-a4 judged above)
+        # -> recompute q~ on the device into a separate buffer
+        dq = torch.empty((B, Hq, 2 * P), dtype=st.dt, device=st.device)
+        tmp_k, tmp_v = st.k_cache[l].clone(), st.v_cache[l].clone()
+        dpos = torch.from_numpy(lens_before).to(st.device)
+        dsid = torch.arange(B, dtype=torch.int32, device=st.device)
+        st.qkv_rope_append(l, dx[l], dsid, dpos, dpos, int(lens_before.max()), q_out=dq)
+        torch.cuda.synchronize()
+        assert torch.equal(tmp_k, st.k_cache[l]) and torch.equal(tmp_v, st.v_cache[l])   # idempotent rewrite
+        util.check_projection(util.to_np64(dq), O.round_storage(q, w.dtype), w.dtype, f"q layer {l}")
+        want = O.decode_attn(util.to_np64(dq), Kd, Vd, lens_before + 1, D)
+        got = util.to_np64(st.out[l][: B * Hq * dv]).reshape(B, Hq, dv)
+        worst = max(worst, util.check_attn(got, want, w.dtype))
+        # and the whole chain against the oracle's own caches (looser: rounding of k/v may differ by an ulp)
+        if w.dtype == "f32":
+            Ko, Vo = caches[l]
+            O.append(Ko, Vo, k, v, np.arange(B), lens_before, w.dtype)
+            want2 = O.decode_attn(O.round_storage(q, w.dtype), Ko, Vo, lens_before + 1, D)
+            assert np.abs(got - want2).max() <= util.F32_MAX_ABS
+    st.close()
+    return worst
+
+
+def test_config1_tiny_fp32_end_to_end():
+    w = synth.TINY
+    err = _end_to_end(w, [w.seq])
+    assert err <= 1e-5
+
+
+@pytest.mark.parametrize("n_split", [1, 3, 64])
+def test_config1_split_counts(n_split):
+    _end_to_end(synth.TINY, [synth.TINY.seq], n_split=n_split)
+
+
+def test_tiny_with_bias():
+    _end_to_end(synth.TINY, [0], with_bias=True)
+
+
+@pytest.mark.parametrize("name", ["3b", "8b", "14b", "sweep1.0", "sweep0.8", "sweep0.5"])
+def test_scaled_down_bf16_twins(name):
+    w = synth.scaled_down(synth.CONFIGS[name], n_layers=2, batch=2, seq=512, hidden=512)
+    _end_to_end(w, [512, 475], chunk=256)
+
+
+@pytest.mark.parametrize("lens", [[0, 1], [63, 64], [65, 127], [128, 129], [1, 300]])
+def test_ragged_and_tile_boundaries(lens):
+    w = synth.scaled_down(synth.LLAMA_8B, n_layers=1, batch=2, seq=320, hidden=256)
+    _end_to_end(w, lens, chunk=256)
+    _end_to_end(w, lens, n_split=7, chunk=256)
+
+
+def test_adjacent_pairing_end_to_end():
+    from dataclasses import replace
+    w = replace(synth.TINY, pairing=1, seq=40)
+    _end_to_end(w, [40])
+
+
+def _random_attn_case(w, lens, n_split, seed=0):
+    """rap_decode_attn alone on random caches (no projection), every unit checked."""
+    st = DecodeStack(w, s_cap=((max(lens) + 8 + 7) // 8) * 8)
+    ks, vs = synth.draw_scores(w)
+    st.build_tables(ks, vs)
+    g = torch.Generator(device=st.device).manual_seed(seed)
+    P2, dv = 2 * w.n_pairs, w.n_vch
+    sig = float(np.sqrt(w.hidden) * 0.02)
+    for l in range(w.n_layers):
+        st.k_cache[l].normal_(0, sig, generator=g)
+        st.v_cache[l].normal_(0, sig, generator=g)
+    q = torch.empty((w.batch, w.n_q_heads, P2), dtype=st.dt, device=st.device).normal_(0, sig, generator=g)
+    dl = torch.tensor(lens, dtype=torch.int32, device=st.device)
+    for l in range(w.n_layers):
+        out = st.decode_attn(l, q, dl, int(max(lens)), n_split=n_split)
+        torch.cuda.synchronize()
+        want = O.decode_attn(util.to_np64(q), util.to_np64(st.k_cache[l]), util.to_np64(st.v_cache[l]), lens, w.head_dim)
+        got = util.to_np64(out[: w.batch * w.n_q_heads * dv]).reshape(w.batch, w.n_q_heads, dv)
+        util.check_attn(got, want, w.dtype)
+    st.close()
+
+
+@pytest.mark.parametrize("name", ["3b", "8b", "14b", "sweep1.0", "sweep0.9", "sweep0.8", "sweep0.5"])
+@pytest.mark.parametrize("n_split", [0, 5])
+def test_attention_only_longer_sequences(name, n_split):
+    w = synth.scaled_down(synth.CONFIGS[name], n_layers=1, batch=3, seq=4096)
+    _random_attn_case(w, [4096, 2500, 1], n_split)
+
+
+def test_attention_generic_variant_matches():
+    w = synth.scaled_down(synth.LLAMA_8B, n_layers=1, batch=2, seq=1500)
+    st = DecodeStack(w, s_cap=1504)
+    st.build_tables(*synth.draw_scores(w))
+    g = torch.Generator(device=st.device).manual_seed(1)
+    st.k_cache[0].normal_(0, 1.3, generator=g)
+    st.v_cache[0].normal_(0, 1.3, generator=g)
+    q = torch.empty((2, w.n_q_heads, 2 * w.n_pairs), dtype=st.dt, device=st.device).normal_(0, 1.3, generator=g)
+    dl = torch.tensor([1500, 777], dtype=torch.int32, device=st.device)
+    a = st.decode_attn(0, q, dl, 1500).clone()
+    st.ctx.rap_set_attn_variant(1)
+    b = st.decode_attn(0, q, dl, 1500).clone()
+    torch.cuda.synchronize()
+    assert (a - b).abs().max().item() < 2e-5
+    st.close()
+
+
+def test_decode_step_host_matches_device_step():
+    w = synth.scaled_down(synth.LLAMA_8B, n_layers=2, batch=2, seq=256, hidden=256)
+    ks, vs = synth.draw_scores(w)
+    st, tabs, w_host = util.build_small_stack(w, ks, vs, full_weights=False)
+    g = torch.Generator(device=st.device).manual_seed(3)
+    for l in range(w.n_layers):
+        st.k_cache[l].normal_(0, 1.0, generator=g)
+        st.v_cache[l].normal_(0, 1.0, generator=g)
+    st.seq_len.fill_(256)
+    X = np.stack([synth.draw_hidden(w, l, 9, w.batch) for l in range(w.n_layers)])
+    hx = torch.from_numpy(X).to(st.dt).contiguous().pin_memory()
+    dx = hx.to(st.device)
+    ref = st.decode_step(dx, 256).clone()
+    kref = [c.clone() for c in st.k_cache]
+    for l in range(w.n_layers):                      # undo the append so the host step redoes the same work
+        st.k_cache[l][:, :, 256, :] = 0
+        st.v_cache[l][:, :, 256, :] = 0
+    h_out = torch.empty((w.n_layers, st.out_stride), dtype=torch.float32).pin_memory()
+    st.decode_step_host(hx, h_out, 256, advance=1)
+    assert torch.equal(h_out, ref.cpu())
+    assert all(torch.equal(a, b) for a, b in zip(kref, st.k_cache))
+    assert st.seq_len.cpu().tolist() == [257, 257]
+    assert st.ctx.rap_kernel_launch_count() > 0
+    st.close()
+
+
+def test_argument_validation_on_device_context():
+    w = synth.scaled_down(synth.LLAMA_8B, n_layers=1, batch=2, seq=64, hidden=256)
+    st = DecodeStack(w, s_cap=72)
+    lib = binding._lib()
+    ctx = st.ctx._ctx
+    P = binding._ptr
+    q = torch.zeros((2, w.n_q_heads, 90), dtype=st.dt, device=st.device)
+    sl = torch.ones(2, dtype=torch.int32, device=st.device)
+    # tables not built yet
+    assert lib.rap_decode_attn(ctx, 0, 2, P(q), P(st.k_cache[0]), P(st.v_cache[0]), 72, P(sl), 1, 0, P(st.out), None) == binding.RAP_ESTATE
+    st.build_tables(*synth.draw_scores(w))
+    call = lambda **kw: lib.rap_decode_attn(ctx, kw.get("layer", 0), kw.get("B", 2), kw.get("q", P(q)), P(st.k_cache[0]),
+                                            P(st.v_cache[0]), kw.get("cap", 72), P(sl), kw.get("lmax", 1),
+                                            kw.get("ns", 0), P(st.out), None)
+    assert call() == binding.RAP_OK
+    assert call(layer=1) == binding.RAP_EINVAL
+    assert call(B=3) == binding.RAP_ESHAPE
+    assert call(q=None) == binding.RAP_EINVAL
+    assert call(q=binding.c_void_p(q.data_ptr() + 2)) == binding.RAP_EALIGN
+    assert call(cap=70) == binding.RAP_EALIGN
+    assert call(lmax=73) == binding.RAP_ECAPACITY
+    assert call(ns=65) == binding.RAP_ESHAPE
+    x = torch.zeros((2, w.hidden), dtype=st.dt, device=st.device)
+    st.set_packed_weights(0, synth.draw_packed_weights(w, 0))
+    ids = torch.arange(2, dtype=torch.int32, device=st.device)
+    app = lambda slot_max, T=2: lib.rap_qkv_rope_append(ctx, 0, T, P(x), P(st.w_qkv[0]), None, P(ids), P(ids), P(ids),
+                                                        slot_max, P(st.inv_freq), P(st.q_scratch), P(st.k_cache[0]),
+                                                        P(st.v_cache[0]), 2, 72, None)
+    assert app(1) == binding.RAP_OK
+    assert app(72) == binding.RAP_ECAPACITY
+    assert app(1, T=3) == binding.RAP_ESHAPE
+    # a slot the host bound did not catch is skipped on the device and reported
+    bad = torch.tensor([0, 500], dtype=torch.int32, device=st.device)
+    st.k_cache[0].fill_(5.0)
+    assert lib.rap_qkv_rope_append(ctx, 0, 2, P(x), P(st.w_qkv[0]), None, P(ids), P(ids), P(bad), 1, P(st.inv_freq),
+                                   P(st.q_scratch), P(st.k_cache[0]), P(st.v_cache[0]), 2, 72, None) == binding.RAP_OK
+    code, detail = st.ctx.rap_get_last_device_status()
+    assert (code, detail) == (binding.RAP_ECAPACITY, 1)
+    assert torch.all(st.k_cache[0][1] == 5.0)
+    assert st.ctx.rap_get_last_device_status() == (0, 0)
+    st.close()
