@@ -1,0 +1,341 @@
+#!/usr/bin/env python
+"""Benchmark of the RAP decode hot path on B200: decode tokens/s and the attention scan's
+achieved HBM bandwidth on a synthetic, seeded, 8B-shaped stack (rho = 0.7, 32K-token cache).
+
+One step = every layer's rap_qkv_rope_append + rap_decode_attn for one batch of new tokens.
+`value` is timed with inputs resident in HBM; `e2e` goes through rap_decode_step_host with
+pinned host inputs and outputs.  `--impl reference` times the CPU oracle on a bounded sample.
+Prints ONE JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2602_02599_b200 import synth  # noqa: E402
+
+METRIC = "decode_tokens_per_s"
+UNIT = "tokens/s"
+T_PREFILL_TAIL = 256     # last cached positions of every sequence are written by the real append path
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return float(p["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+def load_traffic(workload):
+    """DRAM bytes per attention-scan launch from the committed ncu summary, if one exists."""
+    path = os.path.join(ROOT, "profiles", "attn_scan_traffic.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return d.get(workload)
+    return None
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        super().__init__(daemon=True)
+        self.index, self.rows, self.proc = index, [], None
+
+    def run(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            for line in self.proc.stdout:
+                self.rows.append([c.strip() for c in line.split(",")])
+        except Exception:
+            pass
+
+    def stop(self):
+        if self.proc is not None:
+            self.proc.terminate()
+        self.join(timeout=2)
+        sm = [float(r[0]) for r in self.rows if r and r[0].replace(".", "").isdigit()]
+        mx = [float(r[1]) for r in self.rows if len(r) > 1 and r[1].replace(".", "").isdigit()]
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [n for i, n in enumerate(names) if any(len(r) > 3 + i and r[3 + i] == "Active" for r in self.rows)]
+        busy = [s for s in sm if s > 0]
+        return {"sm_mhz": float(np.median(busy)) if busy else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": reasons, "samples": len(sm)}
+
+
+def build_stack(w, torch, seed_offset=0):
+    """Allocate the stack, build tables, upload weights and fill the caches (synthetic, seeded)."""
+    from paper_2602_02599_b200.stack import DecodeStack
+    st = DecodeStack(w, max_rows=max(w.batch, 2048))
+    ks, vs = synth.draw_scores(w)
+    st.build_tables(ks, vs)
+    for l in range(w.n_layers):
+        st.set_packed_weights(l, synth.draw_packed_weights(w, l))
+    g = torch.Generator(device=st.device).manual_seed(w.seed + seed_offset)
+    sigma = float(np.sqrt(w.hidden) * 0.02)
+    for l in range(w.n_layers):
+        st.k_cache[l].normal_(0.0, sigma, generator=g)
+        st.v_cache[l].normal_(0.0, sigma, generator=g)
+    # the last T_PREFILL_TAIL positions go through the real projection + RoPE + append path
+    tail = min(T_PREFILL_TAIL, w.seq)
+    rows_b = np.repeat(np.arange(w.batch, dtype=np.int32), tail)
+    rows_p = np.tile(np.arange(w.seq - tail, w.seq, dtype=np.int32), w.batch)
+    chunk = 2048
+    for l in range(w.n_layers):
+        xg = torch.Generator(device=st.device).manual_seed(w.seed + 7919 * (l + 1))
+        for c0 in range(0, len(rows_b), chunk):
+            c1 = min(len(rows_b), c0 + chunk)
+            x = torch.empty((c1 - c0, w.hidden), dtype=st.dt, device=st.device).normal_(0.0, 1.0, generator=xg)
+            sid = torch.from_numpy(rows_b[c0:c1]).to(st.device)
+            pos = torch.from_numpy(rows_p[c0:c1]).to(st.device)
+            qo = torch.empty((c1 - c0, w.n_q_heads, 2 * st.n_pairs[l]), dtype=st.dt, device=st.device)
+            st.qkv_rope_append(l, x, sid, pos, pos, int(rows_p[c0:c1].max()), q_out=qo)
+    torch.cuda.synchronize()
+    return st
+
+
+def attn_bytes(w, length):
+    return w.batch * w.n_kv_heads * length * (2 * w.n_pairs + w.n_vch) * w.elem_bytes
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
+    w = synth.CONFIGS[args.workload]
+    st = build_stack(w, torch, seed_offset=rank)
+    L, B, K, W = w.n_layers, w.batch, args.steps, args.warmup
+    n_steps = K + W
+    assert w.seq + 2 * n_steps + 2 < st.s_cap, "cache capacity too small for this many steps"
+    dev = st.device
+    # per-step inputs, resident in HBM before the timed region
+    xg = torch.Generator(device=dev).manual_seed(w.seed + 17 + rank)
+    x_all = torch.empty((n_steps, L, B, w.hidden), dtype=st.dt, device=dev).normal_(0.0, 1.0, generator=xg)
+    pos_all = (torch.arange(n_steps, dtype=torch.int32, device=dev)[:, None] + w.seq).expand(n_steps, B).contiguous()
+    len_all = pos_all + 1
+    seq_id = torch.arange(B, dtype=torch.int32, device=dev)
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    attn_ev = [[(ev(), ev()) for _ in range(L)] for _ in range(K)]
+    proj_ev = [[(ev(), ev()) for _ in range(L)] for _ in range(K)]
+
+    def step(i, timed_idx=None):
+        pos = int(w.seq + i)
+        for l in range(L):
+            if timed_idx is not None:
+                proj_ev[timed_idx][l][0].record()
+            st.qkv_rope_append(l, x_all[i, l], seq_id, pos_all[i], pos_all[i], pos)
+            if timed_idx is not None:
+                proj_ev[timed_idx][l][1].record()
+                attn_ev[timed_idx][l][0].record()
+            st.decode_attn(l, st.q_scratch, len_all[i], pos + 1)
+            if timed_idx is not None:
+                attn_ev[timed_idx][l][1].record()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(W):
+        step(i)
+    barrier()
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.3)
+    launches0 = st.ctx.rap_kernel_launch_count()
+    t0, t1 = ev(), ev()
+    barrier()
+    t0.record()
+    for i in range(K):
+        step(W + i, i)
+    t1.record()
+    barrier()
+    launches = st.ctx.rap_kernel_launch_count() - launches0
+    clocks = sampler.stop()
+    ms_total = t0.elapsed_time(t1)
+    attn_ms = float(np.mean([a.elapsed_time(b) for row in attn_ev for a, b in row]))
+    proj_ms = float(np.mean([a.elapsed_time(b) for row in proj_ev for a, b in row]))
+    code, detail = st.ctx.rap_get_last_device_status()
+    assert code == 0, f"device status {code} detail {detail}"
+
+    # ---- end to end through the host-buffer entry point ------------------------------------
+    st.seq_len.fill_(w.seq + n_steps)
+    hx = [torch.empty((L, B, w.hidden), dtype=st.dt).pin_memory() for _ in range(2)]
+    for h in hx:
+        h.copy_(x_all[0].cpu())
+    h_out = torch.empty((L, st.out_stride), dtype=torch.float32).pin_memory()
+    e2e_steps = max(2, min(K, 5))
+    st.decode_step_host(hx[0], h_out, w.seq + n_steps, advance=1)       # warm-up
+    barrier()
+    e0 = time.perf_counter()
+    d0, d1 = ev(), ev()
+    d0.record()
+    for i in range(e2e_steps):
+        st.decode_step_host(hx[i & 1], h_out, w.seq + n_steps + 1 + i, advance=1)
+    d1.record()
+    barrier()
+    e2e_ms = max(d0.elapsed_time(d1), (time.perf_counter() - e0) * 1e3) / e2e_steps
+
+    ms = torch.tensor([ms_total, e2e_ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(ms, op=dist.ReduceOp.MAX)
+    ms_total, e2e_ms = ms.tolist()
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+    ms_step = ms_total / K
+    peak, peak_kind = load_peaks()
+    mean_len = w.seq + W + (K + 1) / 2.0
+    alg = attn_bytes(w, mean_len)
+    achieved = alg / (attn_ms * 1e-3) / 1e9
+    line = {
+        "metric": METRIC, "value": world * B / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K,
+        "warmup": W, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic",
+        "config": {"workload": f"{w.name}: L={L} hidden={w.hidden} Hq/Hkv={w.n_q_heads}/{w.n_kv_heads} D={w.head_dim} "
+                               f"rho={w.rho} P={w.n_pairs} dv={w.n_vch} B={B} S={w.seq}",
+                   "per_gpu_batch": B, "global_batch": world * B, "context": w.seq,
+                   "l2": "inputs larger than L2 (%.1f GB of KV cache per step)" % (L * alg / 1e9),
+                   "parallelism": "replicas" if world > 1 else "single"},
+        "clocks": clocks, "gpu_launches": int(launches),
+        "e2e": {"value": world * B / (e2e_ms * 1e-3), "unit": UNIT,
+                "h2d_bytes_per_step": int(hx[0].numel() * hx[0].element_size()),
+                "d2h_bytes_per_step": int(h_out.numel() * 4)},
+        "roofline": {"bound": "hbm", "kernel": "rap_decode_attn (split-KV scan + combine)", "achieved": achieved,
+                     "peak": peak, "peak_source": peak_kind, "unit": "GB/s", "frac": achieved / peak,
+                     "frac_of_nominal_8000": achieved / 8000.0, "bytes_per_launch": alg, "ms_per_launch": attn_ms,
+                     "traffic": load_traffic(args.workload)},
+        "kernels": {"attn_ms_per_layer": attn_ms, "qkv_rope_append_ms_per_layer": proj_ms},
+    }
+    if args.cpu_baseline:
+        line["cpu_baseline"] = cpu_baseline(w, st, torch)
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def cpu_baseline(w, st, torch, budget_s=15.0):
+    """The oracle, as it stands, on the host cores: full-length scans of sampled (layer, b, kv-head)
+    units plus one layer's projection, extrapolated linearly to a whole step."""
+    from oracle import rap_oracle as O
+    from threadpoolctl import threadpool_info
+    cores = max([i.get("num_threads", 1) for i in threadpool_info()] + [1])
+    rng = np.random.default_rng(123)
+    L, B, Hkv, Hq, G = w.n_layers, w.batch, w.n_kv_heads, w.n_q_heads, w.group
+    n = w.seq + 1
+    torch.cuda.synchronize()
+    times, t_start = [], time.perf_counter()
+    while time.perf_counter() - t_start < budget_s and len(times) < 256:
+        l, b, h = int(rng.integers(L)), int(rng.integers(B)), int(rng.integers(Hkv))
+        K = st.k_cache[l][b, h, :n].to(torch.float64).cpu().numpy()[None, None]
+        V = st.v_cache[l][b, h, :n].to(torch.float64).cpu().numpy()[None, None]
+        q = rng.standard_normal((1, G, K.shape[-1]))
+        t = time.perf_counter()
+        O.decode_attn(q, K, V, [n], w.head_dim)
+        times.append(time.perf_counter() - t)
+    x = O.round_storage(synth.draw_hidden(w, 0, 0, B), w.dtype)
+    wq = st.w_qkv[0].to(torch.float64).cpu().numpy()
+    inv = st.inv_freq[0].cpu().numpy()
+    t = time.perf_counter()
+    O.qkv_rope(x, wq, None, np.full(B, w.seq), inv, Hq, Hkv, w.n_pairs, w.n_vch)
+    t_proj = time.perf_counter() - t
+    t_step = float(np.mean(times)) * L * B * Hkv + L * t_proj
+    return {"value": B / t_step, "unit": UNIT, "cores": int(cores), "kind": "oracle",
+            "sample": f"{len(times)} of {L * B * Hkv} (layer, sequence, kv-head) full-length scans + 1 of {L} layer "
+                      f"projections, extrapolated linearly to one step"}
+
+
+def run_reference(args):
+    """Reference arm: the CPU oracle on host cores, each step a bounded sample of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import rap_oracle as O
+    from threadpoolctl import threadpool_info
+    w = synth.CONFIGS[args.workload]
+    cores = max([i.get("num_threads", 1) for i in threadpool_info()] + [1])
+    L, B, Hkv, Hq, G = w.n_layers, w.batch, w.n_kv_heads, w.n_q_heads, w.group
+    n = w.seq + 1
+    units_per_step = 4
+    rng = np.random.default_rng(w.seed)
+    sigma = float(np.sqrt(w.hidden) * 0.02)
+    wq = O.round_storage(synth.draw_packed_weights(w, 0), w.dtype)
+    ks, vs = synth.draw_scores(synth.scaled_down(w, n_layers=1, batch=1, seq=8))
+    tabs = O.build_tables(ks, vs, [w.n_pairs], [w.n_vch], w.head_dim, w.rope_theta, w.pairing)
+
+    def sample_step(i):
+        t_units = 0.0
+        for u in range(units_per_step):
+            K = O.round_storage(synth.draw_cache_rows(w, 0, i, u, n, 2 * w.n_pairs, 0), w.dtype)[None, None]
+            V = O.round_storage(synth.draw_cache_rows(w, 0, i, u, n, w.n_vch, 1), w.dtype)[None, None]
+            q = O.round_storage(rng.standard_normal((1, G, 2 * w.n_pairs)) * sigma, w.dtype)
+            t = time.perf_counter()
+            O.decode_attn(q, K, V, [n], w.head_dim)
+            t_units += time.perf_counter() - t
+        x = O.round_storage(synth.draw_hidden(w, 0, i, B), w.dtype)
+        t = time.perf_counter()
+        O.qkv_rope(x, wq, None, np.full(B, w.seq), tabs["inv_freq"][0], Hq, Hkv, w.n_pairs, w.n_vch)
+        t_proj = time.perf_counter() - t
+        return t_units / units_per_step * L * B * Hkv + L * t_proj
+
+    for i in range(args.warmup):
+        sample_step(i)
+    est = [sample_step(args.warmup + i) for i in range(args.steps)]
+    t_step = float(np.mean(est))
+    val = B / t_step
+    sample = (f"per step: {units_per_step} of {L * B * Hkv} (layer, sequence, kv-head) full-length scans + 1 of {L} "
+              f"layer projections on synthetic rows, extrapolated linearly to the whole step")
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": t_step * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"{w.name}: L={L} hidden={w.hidden} Hq/Hkv={Hq}/{Hkv} D={w.head_dim} rho={w.rho} "
+                               f"P={w.n_pairs} dv={w.n_vch} B={B} S={w.seq}"},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": int(cores), "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="8b", choices=sorted(synth.CONFIGS))
+    ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "ours":
+        args.warmup = 3
+    if int(os.environ.get("WORLD_SIZE", "1")) > 1:
+        args.cpu_baseline = False
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -97,7 +97,13 @@ rap_status rap_create(const rap_model_desc* desc, rap_ctx** out) {
   const size_t e = rap_elem_bytes(d.dtype);
   const size_t n_out_max = (size_t)(d.n_q_heads + 2 * d.n_kv_heads) * d.head_dim;
   c->attn_ws_bytes = (size_t)d.max_batch * d.n_q_heads * RAP_MAX_SPLIT * (size_t)(d.head_dim + 2) * sizeof(float);
-  c->proj_ws_bytes = (size_t)d.max_rows * n_out_max * sizeof(float) * RAP_MAX_KSPLIT;
+  // full-size fp32 results for any row count, plus room for reduction splits on decode-sized calls
+  {
+    const size_t small_rows = d.max_rows < 256 ? d.max_rows : 256;
+    const size_t a = (size_t)d.max_rows * n_out_max * sizeof(float);
+    const size_t b = small_rows * n_out_max * sizeof(float) * RAP_MAX_KSPLIT;
+    c->proj_ws_bytes = a > b ? a : b;
+  }
   c->stage_x_bytes = (size_t)d.n_layers * d.max_batch * d.hidden * e;
   c->stage_out_bytes = (size_t)d.n_layers * d.max_batch * d.n_q_heads * d.head_dim * sizeof(float);
   RAP_CUDA_TRY(c, cudaMalloc(&c->d_status, 2 * sizeof(int32_t)));
