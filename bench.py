@@ -110,6 +110,14 @@ def build_stack(w, torch, seed_offset=0):
     return st
 
 
+def pick_workload(args):
+    """The named workload, optionally cut down (--layers/--batch/--seq) for profiler-sized runs."""
+    from dataclasses import replace
+    w = synth.CONFIGS[args.workload]
+    over = {k: v for k, v in (("n_layers", args.layers), ("batch", args.batch), ("seq", args.seq)) if v}
+    return replace(w, name=w.name + "-cut", **over) if over else w
+
+
 def attn_bytes(w, length):
     return w.batch * w.n_kv_heads * length * (2 * w.n_pairs + w.n_vch) * w.elem_bytes
 
@@ -123,7 +131,7 @@ def run_ours(args):
     torch.cuda.set_device(local)
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
-    w = synth.CONFIGS[args.workload]
+    w = pick_workload(args)
     st = build_stack(w, torch, seed_offset=rank)
     L, B, K, W = w.n_layers, w.batch, args.steps, args.warmup
     n_steps = K + W
@@ -274,7 +282,7 @@ def run_reference(args):
         return
     from oracle import rap_oracle as O
     from threadpoolctl import threadpool_info
-    w = synth.CONFIGS[args.workload]
+    w = pick_workload(args)
     cores = max([i.get("num_threads", 1) for i in threadpool_info()] + [1])
     L, B, Hkv, Hq, G = w.n_layers, w.batch, w.n_kv_heads, w.n_q_heads, w.group
     n = w.seq + 1
@@ -326,6 +334,9 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="8b", choices=sorted(synth.CONFIGS))
     ap.add_argument("--no-cpu-baseline", dest="cpu_baseline", action="store_false")
+    ap.add_argument("--layers", type=int, default=0, help="cut the workload to this many layers (profiling)")
+    ap.add_argument("--batch", type=int, default=0, help="cut the workload to this batch (profiling)")
+    ap.add_argument("--seq", type=int, default=0, help="cut the workload to this context (profiling)")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3

@@ -149,10 +149,10 @@ rap_status rap_build_tables(rap_ctx* ctx, const double* ks, const double* vs, co
     RAP_CUDA_TRY(ctx, cudaStreamSynchronize((cudaStream_t)ctx->tables_stream));
     ctx->tables_inflight = false;
   }
-  int32_t* h_pair = (int32_t*)ctx->h_tables;
+  double* h_freq = (double*)ctx->h_tables;          // doubles first so they stay 8-byte aligned
+  int32_t* h_pair = (int32_t*)(h_freq + units * half);
   int32_t* h_dim = h_pair + units * half;
   int32_t* h_v = h_dim + units * D;
-  double* h_freq = (double*)(h_v + units * D);   // offset is a multiple of 8 bytes: (half + 2D) * 4 * units
   std::fill(h_pair, h_pair + units * half, -1);
   std::fill(h_dim, h_dim + units * D, -1);
   std::fill(h_v, h_v + units * D, -1);
