@@ -146,6 +146,32 @@ rap_status rap_decode_attn(rap_ctx* ctx, int32_t layer, int32_t B, const void* d
                            const int32_t* d_seq_len, int32_t h_seq_len_max, int32_t n_split,
                            float* d_out, void* stream);
 
+/* ---- decode attention without any allocation (the paper has no counterpart) --------------
+ * Same result as rap_decode_attn, for callers that cannot allocate device memory: code running
+ * inside someone else's memory budget (a serving engine that hands out every byte of HBM up
+ * front), inside a region where cudaMalloc is forbidden or would synchronize the device, or
+ * before/without a rap_ctx (rap_create allocates).  It takes the shape directly instead of a
+ * context and calls no cudaMalloc / cudaFree or any other allocating routine.
+ *   dtype: rap_dtype of d_q and the caches; n_pairs = P, n_vch = d_v' of this layer;
+ *   d_q [B][H_q][2P], d_k_cache [B][H_kv][S_cap][2P], d_v_cache [B][H_kv][S_cap][d_v'],
+ *   d_seq_len[b] valid rows (as in rap_decode_attn), d_out [B][H_q][d_v'] fp32.
+ * Scratch: the split-KV partials go to a 4 MiB array that is part of the library image
+ * (RAP_NOALLOC_WS_FLOATS = 2^20 floats); every GPU that loads the library holds those 4 MiB
+ * until the process exits.  A call needs B * H_q * n_split * (d_v' + 2) floats: with
+ * n_split = 0 the library picks a split count that fits; RAP_ESHAPE if the requested n_split
+ * does not fit, or if even one split does not (B * H_q * (d_v' + 2) > 2^20).
+ * The first call on each device looks up the array's device address (with that device
+ * current); make that first call outside any stream capture.
+ * All calls on a device share the one array and it keeps the previous call's contents.  The
+ * kernels write every partial they later read, so nothing needs clearing, but two calls whose
+ * kernels overlap on the GPU (different streams, or a graph with parallel branches) race on
+ * it: serialize them.  Always uses the shape-generic kernel (any 2P, d_v' <= 256, G <= 8). */
+rap_status rap_decode_attn_noalloc(int32_t dtype, int32_t B, int32_t n_q_heads, int32_t n_kv_heads,
+                                   int32_t head_dim, int32_t n_pairs, int32_t n_vch, const void* d_q,
+                                   const void* d_k_cache, const void* d_v_cache, int32_t S_cap,
+                                   const int32_t* d_seq_len, int32_t h_seq_len_max, int32_t n_split,
+                                   float* d_out, void* stream);
+
 /* ---- one decode step over all layers (a2-a5 per layer) -------------------------------------
  * Layer l consumes d_x + l*B*hidden (one hidden-state row per sequence) and produces
  * d_out + l*out_layer_stride ([B][H_q][d_v'_l] fp32).  d_seq_len[b] = rows cached BEFORE the

@@ -24,6 +24,7 @@ EXPORTS = [
     "rap_cache_elem_offset", "rap_build_tables", "rap_pack_weights", "rap_qkv_rope_append",
     "rap_decode_attn", "rap_decode_step", "rap_decode_step_host", "rap_lowrank_decode_attn",
     "rap_get_last_device_status", "rap_kernel_launch_count", "rap_set_attn_variant",
+    "rap_decode_attn_noalloc",
 ]
 
 
@@ -75,6 +76,7 @@ def _lib():
     lib.rap_kernel_launch_count.argtypes = [P]
     lib.rap_kernel_launch_count.restype = c_int64
     lib.rap_set_attn_variant.argtypes = [P, c_int32]
+    lib.rap_decode_attn_noalloc.argtypes = [c_int32] * 7 + [P, P, P, c_int32, P, c_int32, c_int32, P, P]
     for name in EXPORTS:
         fn = getattr(lib, name)
         if fn.restype is ctypes.c_int:       # default: every other entry point returns rap_status
@@ -116,6 +118,22 @@ def rap_retained_counts(rho, head_dim):
 
 def rap_cache_elem_offset(n_kv_heads, S_cap, W, b, h, pos, c):
     return _lib().rap_cache_elem_offset(n_kv_heads, S_cap, W, b, h, pos, c)
+
+
+NOALLOC_WS_FLOATS = 1 << 20
+
+
+def rap_decode_attn_noalloc(dtype, B, n_q_heads, n_kv_heads, head_dim, n_pairs, n_vch, d_q, d_k_cache, d_v_cache,
+                            S_cap, d_seq_len, h_seq_len_max, n_split, d_out):
+    """Decode attention for callers that must not allocate: no context, scratch in the library's
+    own 4 MiB static device array (shared by all calls on a device; overlapping calls race)."""
+    s = _lib().rap_decode_attn_noalloc(dtype, B, n_q_heads, n_kv_heads, head_dim, n_pairs, n_vch, _ptr(d_q),
+                                       _ptr(d_k_cache), _ptr(d_v_cache), S_cap, _ptr(d_seq_len), h_seq_len_max,
+                                       n_split, _ptr(d_out), _stream())
+    if s:
+        need = B * n_q_heads * max(n_split, 1) * (n_vch + 2)
+        raise RapError(s, "rap_decode_attn_noalloc",
+                       f"needs {need} scratch floats, the static array holds {NOALLOC_WS_FLOATS}" if s == RAP_ESHAPE else "")
 
 
 class RapContext:

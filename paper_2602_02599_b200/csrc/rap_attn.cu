@@ -9,6 +9,8 @@
 // followed by (m, l): m = running max of the base-2 logits, l = sum 2^(s - m).
 #include <math.h>
 
+#include <mutex>
+
 #include "rap_internal.h"
 
 rap_status rap_launch_attn_fast(rap_ctx* ctx, const rap_attn_args& a, int n_split, cudaStream_t st);
@@ -191,5 +193,91 @@ rap_status rap_launch_attn(rap_ctx* ctx, const rap_attn_args& a, cudaStream_t st
   attn_combine_kernel<<<a.B * a.Hq, 128, 0, st>>>(ctx->d_attn_ws, n_split, a.dv, a.out);
   ctx->launches++;
   RAP_CUDA_TRY(ctx, cudaGetLastError());
+  return RAP_OK;
+}
+
+// ---- allocation-free variant ---------------------------------------------------------------
+// Split-KV partials of rap_decode_attn_noalloc live in this file-scope array instead of a
+// context workspace.  Every GPU that loads the library reserves it until the process exits.
+#define RAP_NOALLOC_WS_FLOATS (1u << 20)   // 4 MiB
+static __device__ __align__(256) float g_noalloc_ws[RAP_NOALLOC_WS_FLOATS];
+
+namespace {
+constexpr int NOALLOC_MAX_DEVICES = 64;
+std::mutex g_noalloc_mu;
+float* g_noalloc_addr[NOALLOC_MAX_DEVICES];   // device address of g_noalloc_ws, per device ordinal
+
+// In host code `g_noalloc_ws` names a host-side shadow, not device memory; the address a kernel
+// may use comes from cudaGetSymbolAddress, asked once per device with that device current.
+cudaError_t noalloc_ws_address(float** out) {
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= NOALLOC_MAX_DEVICES) return cudaErrorInvalidDevice;
+  std::lock_guard<std::mutex> lock(g_noalloc_mu);
+  if (!g_noalloc_addr[dev]) {
+    void* p = nullptr;
+    e = cudaGetSymbolAddress(&p, g_noalloc_ws);
+    if (e != cudaSuccess) return e;
+    g_noalloc_addr[dev] = static_cast<float*>(p);
+  }
+  *out = g_noalloc_addr[dev];
+  return cudaSuccess;
+}
+}  // namespace
+
+extern "C" rap_status rap_decode_attn_noalloc(int32_t dtype, int32_t B, int32_t n_q_heads, int32_t n_kv_heads,
+                                              int32_t head_dim, int32_t n_pairs, int32_t n_vch, const void* d_q,
+                                              const void* d_k_cache, const void* d_v_cache, int32_t S_cap,
+                                              const int32_t* d_seq_len, int32_t h_seq_len_max, int32_t n_split,
+                                              float* d_out, void* stream) {
+  if (!d_q || !d_k_cache || !d_v_cache || !d_seq_len || !d_out) return RAP_EINVAL;
+  if (dtype != RAP_F32 && dtype != RAP_BF16) return RAP_EINVAL;
+  if (B < 0 || n_q_heads < 1 || n_kv_heads < 1 || n_q_heads % n_kv_heads || head_dim < 2 || (head_dim & 1) ||
+      head_dim > GEN_THREADS || n_pairs < 1 || n_pairs > head_dim / 2 || n_vch < 1 || n_vch > head_dim ||
+      S_cap < 1 || n_split < 0 || h_seq_len_max < 0)
+    return RAP_EINVAL;
+  const int G = n_q_heads / n_kv_heads;
+  if (G > RAP_MAX_GROUP || n_split > RAP_MAX_SPLIT) return RAP_ESHAPE;
+  if (S_cap % 8) return RAP_EALIGN;
+  if (h_seq_len_max > S_cap) return RAP_ECAPACITY;
+  if (!rap_aligned16(d_q) || !rap_aligned16(d_k_cache) || !rap_aligned16(d_v_cache) || !rap_aligned16(d_out) ||
+      !rap_aligned16(d_seq_len))
+    return RAP_EALIGN;
+  if (B == 0) return RAP_OK;
+  // the partials of one split: B * H_q rows of d_v' accumulators + (m, l)
+  const size_t per_split = (size_t)B * n_q_heads * (size_t)(n_vch + 2);
+  if (per_split > RAP_NOALLOC_WS_FLOATS) return RAP_ESHAPE;
+  const int fit = (int)(RAP_NOALLOC_WS_FLOATS / per_split);
+  int ns = n_split;
+  if (ns == 0) {
+    // a few CTAs per SM, splits of at least four tiles, and no more than the static array holds
+    const int n_tiles = (h_seq_len_max + GEN_TILE - 1) / GEN_TILE;
+    ns = (1024 + B * n_kv_heads - 1) / (B * n_kv_heads);
+    if (ns > n_tiles / 4) ns = n_tiles / 4;
+    if (ns > RAP_MAX_SPLIT) ns = RAP_MAX_SPLIT;
+    if (ns > fit) ns = fit;
+    if (ns < 1) ns = 1;
+  } else if (ns > fit) {
+    return RAP_ESHAPE;
+  }
+  float* ws = nullptr;
+  if (noalloc_ws_address(&ws) != cudaSuccess) return RAP_ECUDA;
+  cudaStream_t st = (cudaStream_t)stream;
+  const int P2 = 2 * n_pairs;
+  const float qscale = (float)(1.4426950408889634 / sqrt((double)head_dim));
+  const size_t smem = (size_t)(G * P2 + G * GEN_TILE + G) * sizeof(float);
+  dim3 grid(ns, n_kv_heads, B);
+  if (dtype == RAP_F32)
+    attn_generic_kernel<float><<<grid, GEN_THREADS, smem, st>>>((const float*)d_q, (const float*)d_k_cache,
+                                                                (const float*)d_v_cache, d_seq_len, 0, n_q_heads,
+                                                                n_kv_heads, P2, n_vch, S_cap, qscale, ns, ws);
+  else
+    attn_generic_kernel<__nv_bfloat16><<<grid, GEN_THREADS, smem, st>>>(
+        (const __nv_bfloat16*)d_q, (const __nv_bfloat16*)d_k_cache, (const __nv_bfloat16*)d_v_cache, d_seq_len, 0,
+        n_q_heads, n_kv_heads, P2, n_vch, S_cap, qscale, ns, ws);
+  if (cudaGetLastError() != cudaSuccess) return RAP_ECUDA;
+  attn_combine_kernel<<<B * n_q_heads, 128, 0, st>>>(ws, ns, n_vch, d_out);
+  if (cudaGetLastError() != cudaSuccess) return RAP_ECUDA;
   return RAP_OK;
 }
