@@ -215,7 +215,8 @@ rap_status rap_get_last_device_status(rap_ctx* ctx, int32_t* code, int32_t* deta
 /* Number of kernels this context has launched since creation (for launch accounting). */
 int64_t rap_kernel_launch_count(const rap_ctx* ctx);
 
-/* Forces a kernel variant for rap_decode_attn: 0 = automatic, 1 = generic kernel only.
+/* Forces a kernel variant for rap_decode_attn: 0 = automatic (shape-specialised scan when the
+ * head shape has one), 1 = fully generic kernel only, 2 = skip the shape-specialised scan.
  * Meant for tests and profiling. */
 rap_status rap_set_attn_variant(rap_ctx* ctx, int32_t variant);
 

@@ -2,8 +2,9 @@
 // channels, Eq. 7; softmax scale 1/sqrt(D) with the ORIGINAL head_dim).
 //
 // This file holds the shape-generic scan kernel (any 2P, d_v', fp32 or bf16), the split
-// combine kernel and the launch heuristics.  The bandwidth-tuned bf16 scan lives in
-// rap_attn_fast.cu; rap_launch_attn picks it when its shape rules hold.
+// combine kernel and the launch heuristics.  The bandwidth-tuned bf16 scans live in
+// rap_attn_scan.cu (specialised per head shape) and rap_attn_fast.cu (run-time shape);
+// rap_launch_attn picks them when their shape rules hold.
 //
 // Partial results of split s for (b, g) live in the context workspace as d_v' accumulators
 // followed by (m, l): m = running max of the base-2 logits, l = sum 2^(s - m).
@@ -14,6 +15,7 @@
 #include "rap_internal.h"
 
 rap_status rap_launch_attn_fast(rap_ctx* ctx, const rap_attn_args& a, int n_split, cudaStream_t st);
+rap_status rap_launch_attn_scan(rap_ctx* ctx, const rap_attn_args& a, int n_split, cudaStream_t st);
 
 namespace {
 
@@ -172,7 +174,12 @@ static int choose_split(const rap_ctx* ctx, const rap_attn_args& a, int tile, in
 
 rap_status rap_launch_attn(rap_ctx* ctx, const rap_attn_args& a, cudaStream_t st) {
   const int G = a.Hq / a.Hkv;
-  if (ctx->attn_variant == 0 && a.dtype == RAP_BF16) {
+  if (a.dtype == RAP_BF16 && ctx->attn_variant != 1) {
+    // shape-specialised scan, then the shape-generic bf16 scan, then the fully generic kernel
+    if (ctx->attn_variant == 0) {
+      const rap_status s = rap_launch_attn_scan(ctx, a, a.n_split, st);
+      if (s != RAP_EUNSUPPORTED) return s;
+    }
     const rap_status s = rap_launch_attn_fast(ctx, a, a.n_split, st);
     if (s != RAP_EUNSUPPORTED) return s;
   }

@@ -1,0 +1,538 @@
+// Shape-specialised bf16 split-KV scan for rap_decode_attn (Eq. 2 on the retained dims, Eq. 7,
+// scale 1/sqrt(D)): the kernel the 3B / 8B / 14B-shaped workloads run.
+//
+// The scan reads every cache byte once and does G flops per byte, so HBM bandwidth bounds it;
+// what decides whether it gets there is the number of issue slots spent per cache word on the
+// plain FP32 pipes (tensor cores are not used for this scan).  Everything that depends on the
+// head shape -- K words per row (WK = P), V channels (DV = d_v'), group size G -- is a template
+// parameter, so the inner loops are fully unrolled with immediate shared-memory offsets and
+// no run-time predicates.
+//
+// One CTA (256 threads) owns a contiguous range of 64-position tiles of one (sequence, KV
+// head) unit and all G query heads of that KV head.
+//   * staging: K and V tiles are contiguous byte ranges of the dense-packed cache; warp 0
+//     moves them with bulk async copies (mbarrier complete_tx) into a 3-4 stage ring.  K rows
+//     whose byte length is a multiple of 32 are copied row by row to a padded stride so that
+//     lane-per-position reads stay bank-conflict free.
+//   * logits: warp c owns dim-chunk c (chunks are equal; the last one is shifted back into
+//     the row and its overlapped words meet zeroed q), lane l owns positions l and l + 32.
+//     q lives in registers pre-scaled by log2(e)/sqrt(D) as (even, odd) float pairs; each
+//     32-bit cache word is unpacked by shift / mask and fed to packed fma.rn.f32x2.
+//   * softmax: warp g < G adds the 8 chunk partials of head g.  The reference maximum is
+//     lazy: it is raised (with a warp max and a rescale factor for the accumulators) only when
+//     a logit exceeds it by more than 8, so p = 2^(s - m_ref) <= 256 and most tiles need neither
+//     shuffles nor a rescale; the row sum stays per lane until the end of the scan.
+//   * PV: thread (row group, channel pair) accumulates its rows two at a time per packed FMA.
+//   * partials (acc[d_v'], m, l) of the split go to the workspace; a combine kernel merges.
+// Every mbarrier wait is bounded: on timeout the CTA records RAP_ETIMEOUT and leaves.
+#include <math.h>
+
+#include "rap_internal.h"
+
+namespace {
+
+constexpr int ST = 64;           // positions per tile
+constexpr int STHREADS = 256;
+constexpr int SCHUNKS = 8;       // dim chunks of the logits phase (= warps)
+constexpr uint32_t WAIT_LIMIT = 1u << 21;
+constexpr int SMEM_BUDGET = 115712;   // two CTAs per SM
+constexpr float LAZY_MAX_SLACK = 8.f;
+
+constexpr int cround(int x, int m) { return (x + m - 1) / m * m; }
+
+template <int G, int WK, int DV>
+struct ScanCfg {
+  static constexpr int KV = (WK % 2) ? 1 : (WK % 4) ? 2 : 4;   // 32-bit words per K read
+  static constexpr bool KPAD = (WK % 8) == 0;                  // row-by-row copies to a padded stride
+  static constexpr int KS = KPAD ? WK + 4 : WK;                // K row stride in shared memory (words)
+  static constexpr int UNITS = WK / KV;
+  static constexpr int CLU = (UNITS + SCHUNKS - 1) / SCHUNKS;  // reads per lane, row and chunk
+  static constexpr int CL = CLU * KV;                          // words per chunk
+  static constexpr bool VODD = (DV & 1) != 0;
+  static constexpr int WVP = (DV + 1) / 2;                     // channel pairs per V row
+  static constexpr int NG = (STHREADS / WVP) > ST ? ST : (STHREADS / WVP);   // PV row groups
+  static constexpr int RPG = (ST + NG - 1) / NG;               // rows per group (largest)
+  static constexpr int LASTN = ST - (RPG - 1) * NG;            // groups that own a row in the last slot
+  static constexpr int IP = (RPG + 1) / 2;                     // row pairs per group
+  static constexpr int Gp = (G + 1) & ~1;
+  static constexpr int GS = cround(IP * Gp * 2, 32) + 8;       // p floats per group (bank-shifted)
+  static constexpr int OFF_SPART = 128;
+  static constexpr int OFF_PP = OFF_SPART + SCHUNKS * G * ST * 4;
+  static constexpr int OFF_ALPHA = OFF_PP + cround(NG * GS * 4, 16);
+  static constexpr int OFF_STAGE = cround(OFF_ALPHA + 32, 128);
+  static constexpr int V_OFF = cround(ST * KS * 4, 128);
+  static constexpr int STAGE_BYTES = cround(V_OFF + ST * DV * 2, 128);
+  static constexpr int NS_RAW = (SMEM_BUDGET - OFF_STAGE) / STAGE_BYTES;
+  static constexpr int NS = NS_RAW > 4 ? 4 : NS_RAW;
+  static constexpr int SMEM = OFF_STAGE + NS * STAGE_BYTES;
+  static_assert(NS >= 2, "tile ring needs two stages");
+  static_assert(NG * 2 * WVP * G <= SCHUNKS * G * ST, "row-group reduction reuses the partial-logit buffer");
+};
+
+struct ScanParams {
+  const uint32_t* q;          // [B][Hq][WK] bf16 pairs
+  const unsigned char* k;     // [B][Hkv][S_cap][WK * 4 bytes]
+  const unsigned char* v;     // [B][Hkv][S_cap][DV * 2 bytes]
+  const int32_t* seq_len;
+  float* ws;
+  int32_t* status;
+  int len_add, Hq, Hkv, S_cap, n_split;
+  float qscale;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ uint64_t pack2u(uint32_t lo, uint32_t hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+// d = a * b + c on two packed fp32 lanes
+__device__ __forceinline__ uint64_t ffma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t fmul2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
+  for (uint32_t i = 0; i < WAIT_LIMIT; ++i)
+    if (mbar_try_wait(bar, parity)) return true;
+  return false;
+}
+// global -> this CTA's shared memory, completion counted in bytes on the mbarrier (no multicast)
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+               "l"(src), "r"(bytes), "r"(bar)
+               : "memory");
+}
+
+template <int KV>
+__device__ __forceinline__ void ld_words(const uint32_t* p, uint32_t (&x)[KV]) {
+  if constexpr (KV == 1) {
+    x[0] = *p;
+  } else if constexpr (KV == 2) {
+    const uint2 v = *reinterpret_cast<const uint2*>(p);
+    x[0] = v.x; x[1] = v.y;
+  } else {
+    const uint4 v = *reinterpret_cast<const uint4*>(p);
+    x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w;
+  }
+}
+
+template <int G, int WK, int DV>
+__global__ void __launch_bounds__(STHREADS, 2) attn_scan_kernel(const ScanParams p) {
+  using C = ScanCfg<G, WK, DV>;
+  constexpr int Gp = C::Gp;
+  extern __shared__ __align__(128) unsigned char smem[];
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem);
+  float* s_part = reinterpret_cast<float*>(smem + C::OFF_SPART);   // [SCHUNKS][G][ST]; reused for the group reduction
+  float* pp = reinterpret_cast<float*>(smem + C::OFF_PP);
+  float* alpha_s = reinterpret_cast<float*>(smem + C::OFF_ALPHA);
+  unsigned char* stages = smem + C::OFF_STAGE;
+
+  const int split = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  int len = p.seq_len[b] + p.len_add;
+  len = min(max(len, 0), p.S_cap);
+  const int n_tiles = (len + ST - 1) / ST;
+  const int tps = (n_tiles + p.n_split - 1) / p.n_split;
+  const int t_begin = min(n_tiles, split * tps), t_end = min(n_tiles, t_begin + tps);
+  const int n_my = t_end - t_begin;
+  const int len8 = (len + 7) & ~7;      // rows a copy may touch: S_cap is a multiple of 8
+  float* ws_base = p.ws + (((size_t)b * p.Hq + (size_t)h * G) * p.n_split + split) * (size_t)(DV + 2);
+  const size_t ws_head = (size_t)p.n_split * (DV + 2);
+
+  if (n_my <= 0) {   // nothing to scan: neutral partials
+    for (int i = tid; i < G * (DV + 2); i += STHREADS) {
+      const int g = i / (DV + 2), c = i - g * (DV + 2);
+      ws_base[g * ws_head + c] = (c == DV) ? -INFINITY : 0.f;
+    }
+    return;
+  }
+
+  const size_t unit = (size_t)b * p.Hkv + h;
+  const unsigned char* kg = p.k + unit * (size_t)p.S_cap * (size_t)(WK * 4);
+  const unsigned char* vg = p.v + unit * (size_t)p.S_cap * (size_t)(DV * 2);
+  const uint32_t bar0 = smem_u32(bars);
+  const uint32_t stage0 = smem_u32(stages);
+
+  if (tid == 0) {
+#pragma unroll
+    for (int s = 0; s < C::NS; ++s) mbar_init(bar0 + 8 * s, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  for (int i = tid; i < C::NG * C::GS; i += STHREADS) pp[i] = 0.f;   // slots of rows that never exist stay zero
+  __syncthreads();
+
+  // issued by warp 0 (all lanes converged): tile tl of this CTA into stage st
+  auto issue_tile = [&](int tl, int st) {
+    const int j0 = (t_begin + tl) * ST;
+    const int rows = min(ST, len8 - j0);
+    const uint32_t bar = bar0 + 8 * st;
+    const uint32_t dst = stage0 + st * C::STAGE_BYTES;
+    const uint32_t kb = (uint32_t)rows * WK * 4, vb = (uint32_t)rows * DV * 2;
+    if (lane == 0) mbar_expect_tx(bar, kb + vb);
+    __syncwarp();
+    if constexpr (C::KPAD) {
+      for (int r = lane; r < rows; r += 32)
+        bulk_g2s(dst + r * C::KS * 4, kg + (size_t)(j0 + r) * (WK * 4), WK * 4, bar);
+    } else {
+      if (lane == 0) bulk_g2s(dst, kg + (size_t)j0 * (WK * 4), kb, bar);
+    }
+    if (lane == 0) bulk_g2s(dst + C::V_OFF, vg + (size_t)j0 * (DV * 2), vb, bar);
+  };
+  if (warp == 0) {
+    const int pre = min(n_my, C::NS - 1);
+    for (int tl = 0; tl < pre; ++tl) issue_tile(tl, tl);
+  }
+
+  // ---- this warp's dim chunk and its pre-scaled q registers ---------------------------------
+  const int u_nom = warp * C::CLU;                         // first unit this chunk is responsible for
+  const int u0 = min(u_nom, C::UNITS - C::CLU);            // first unit it reads (shifted back into the row)
+  const int w0 = u0 * C::KV;
+  uint64_t qr[G][C::CL];
+#pragma unroll
+  for (int g = 0; g < G; ++g) {
+    const uint32_t* qrow = p.q + ((size_t)b * p.Hq + (size_t)h * G + g) * WK;
+#pragma unroll
+    for (int i = 0; i < C::CL; ++i) {
+      const bool mine = (u0 + i / C::KV) >= u_nom;
+      const uint32_t x = mine ? qrow[w0 + i] : 0u;
+      qr[g][i] = pack2(__uint_as_float(x << 16) * p.qscale, __uint_as_float(x & 0xffff0000u) * p.qscale);
+    }
+  }
+
+  // ---- PV role ------------------------------------------------------------------------------
+  const int grp = tid / C::WVP, wch = tid - grp * C::WVP;
+  const bool pv_active = grp < C::NG;
+  const bool last_slot_ok = grp < C::LASTN;    // does this group own a row in slot RPG - 1 ?
+  const bool has_hi = 2 * wch + 1 < DV;        // odd DV: the last channel pair has one channel
+  uint64_t accLo[G], accHi[G];     // (even-slot rows, odd-slot rows) partial sums of channels 2*wch and 2*wch+1
+#pragma unroll
+  for (int g = 0; g < G; ++g) accLo[g] = accHi[g] = 0ull;
+  const float* ppg = pp + (pv_active ? grp : 0) * C::GS;
+
+  // softmax role: warp g < G, lanes own positions lane and lane + 32
+  float m_ref = -INFINITY, l_lane = 0.f;
+  int pidx0, pidx1;
+  {
+    const int g0 = lane % C::NG, i0 = lane / C::NG, g1 = (lane + 32) % C::NG, i1 = (lane + 32) / C::NG;
+    pidx0 = g0 * C::GS + (i0 >> 1) * Gp * 2 + (i0 & 1) + 2 * warp;
+    pidx1 = g1 * C::GS + (i1 >> 1) * Gp * 2 + (i1 & 1) + 2 * warp;
+  }
+  bool timed_out = false;
+  int st = 0;
+  uint32_t parity = 0;
+
+  for (int tl = 0; tl < n_my; ++tl) {
+    const bool ok = mbar_wait_bounded(bar0 + 8 * st, parity);
+    unsigned char* stage = stages + st * C::STAGE_BYTES;
+    const int j0 = (t_begin + tl) * ST;
+    const int nj = min(ST, len - j0);
+    if (nj < ST && ok) {
+      // last tile of the sequence: rows >= nj were not written by this sequence; zero their V so
+      // that the fixed-length PV loop meets 0 * 0 there
+      uint16_t* vz = reinterpret_cast<uint16_t*>(stage + C::V_OFF);
+      for (int i = nj * DV + tid; i < ST * DV; i += STHREADS) vz[i] = 0;
+    }
+
+    // ---- logits partials: rows lane, lane + 32; words [w0, w0 + CL) ------------------------
+    {
+      const uint32_t* r0 = reinterpret_cast<const uint32_t*>(stage) + lane * C::KS + w0;
+      const uint32_t* r1 = r0 + 32 * C::KS;
+      uint64_t a0[G], a1[G];
+#pragma unroll
+      for (int g = 0; g < G; ++g) a0[g] = a1[g] = 0ull;
+#pragma unroll
+      for (int u = 0; u < C::CLU; ++u) {
+        uint32_t x0[C::KV], x1[C::KV];
+        ld_words<C::KV>(r0 + u * C::KV, x0);
+        ld_words<C::KV>(r1 + u * C::KV, x1);
+#pragma unroll
+        for (int j = 0; j < C::KV; ++j) {
+          const uint64_t k0 = pack2u(x0[j] << 16, x0[j] & 0xffff0000u);
+          const uint64_t k1 = pack2u(x1[j] << 16, x1[j] & 0xffff0000u);
+#pragma unroll
+          for (int g = 0; g < G; ++g) {
+            a0[g] = ffma2(k0, qr[g][u * C::KV + j], a0[g]);
+            a1[g] = ffma2(k1, qr[g][u * C::KV + j], a1[g]);
+          }
+        }
+      }
+#pragma unroll
+      for (int g = 0; g < G; ++g) {
+        float e, o;
+        unpack2(a0[g], e, o);
+        s_part[(warp * G + g) * ST + lane] = e + o;
+        unpack2(a1[g], e, o);
+        s_part[(warp * G + g) * ST + lane + 32] = e + o;
+      }
+    }
+    if (__syncthreads_or(!ok)) {   // sync #1: partial logits visible; the previous tile's stage is free
+      timed_out = true;
+      break;
+    }
+    if (warp == 0 && tl + C::NS - 1 < n_my) issue_tile(tl + C::NS - 1, st == 0 ? C::NS - 1 : st - 1);
+
+    // ---- online softmax: warp g owns head g --------------------------------------------------
+    if (warp < G) {
+      const int g = warp;
+      float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+      for (int c = 0; c < SCHUNKS; ++c) {
+        s0 += s_part[(c * G + g) * ST + lane];
+        s1 += s_part[(c * G + g) * ST + lane + 32];
+      }
+      if (lane >= nj) s0 = -INFINITY;
+      if (lane + 32 >= nj) s1 = -INFINITY;
+      float mx = fmaxf(s0, s1);
+      float alpha = 1.f;
+      if (__any_sync(0xffffffffu, mx > m_ref + LAZY_MAX_SLACK)) {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+        const float m_new = fmaxf(m_ref, mx);
+        alpha = exp2f(m_ref - m_new);     // first tile: 2^(-inf) = 0
+        l_lane *= alpha;
+        m_ref = m_new;
+      }
+      const float p0 = exp2f(s0 - m_ref), p1 = exp2f(s1 - m_ref);
+      l_lane += p0 + p1;
+      pp[pidx0] = p0;
+      pp[pidx1] = p1;
+      if (lane == 0) alpha_s[g] = alpha;
+    }
+    __syncthreads();   // sync #2: p and alpha visible
+
+    // ---- PV: slots 0 .. RPG-1 of this thread's row group, two slots per packed FMA -----------
+    if (pv_active) {
+      {
+        bool resc = false;
+        float al[G];
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+          al[g] = alpha_s[g];
+          resc |= al[g] != 1.f;
+        }
+        if (resc) {
+#pragma unroll
+          for (int g = 0; g < G; ++g) {
+            const uint64_t aa = pack2(al[g], al[g]);
+            accLo[g] = fmul2(accLo[g], aa);
+            accHi[g] = fmul2(accHi[g], aa);
+          }
+        }
+      }
+      const unsigned char* vt = stage + C::V_OFF;
+#pragma unroll
+      for (int ip = 0; ip < C::IP; ++ip) {
+        const int iA = 2 * ip, iB = 2 * ip + 1;
+        const bool okA = (iA < C::RPG - 1) || (iA == C::RPG - 1 && last_slot_ok);
+        const bool okB = (iB < C::RPG - 1) || (iB == C::RPG - 1 && last_slot_ok);
+        uint64_t lo, hi;
+        if constexpr (!C::VODD) {
+          constexpr int WV = DV / 2;
+          const uint32_t* pa = reinterpret_cast<const uint32_t*>(vt) + grp * WV + wch;
+          const uint32_t xa = okA ? pa[iA * C::NG * WV] : 0u;
+          const uint32_t xb = okB ? pa[iB * C::NG * WV] : 0u;
+          lo = pack2u(xa << 16, xb << 16);
+          hi = pack2u(xa & 0xffff0000u, xb & 0xffff0000u);
+        } else {
+          const uint16_t* pa = reinterpret_cast<const uint16_t*>(vt) + grp * DV + 2 * wch;
+          const uint32_t la = okA ? pa[iA * C::NG * DV] : 0u, lb = okB ? pa[iB * C::NG * DV] : 0u;
+          const uint32_t ha = (okA && has_hi) ? pa[iA * C::NG * DV + 1] : 0u;
+          const uint32_t hb = (okB && has_hi) ? pa[iB * C::NG * DV + 1] : 0u;
+          lo = pack2u(la << 16, lb << 16);
+          hi = pack2u(ha << 16, hb << 16);
+        }
+        const float* pr = ppg + ip * Gp * 2;
+#pragma unroll
+        for (int g2 = 0; g2 < Gp / 2; ++g2) {
+          const float4 t = *reinterpret_cast<const float4*>(pr + 4 * g2);
+          const uint64_t pg0 = pack2(t.x, t.y);
+          accLo[2 * g2] = ffma2(lo, pg0, accLo[2 * g2]);
+          accHi[2 * g2] = ffma2(hi, pg0, accHi[2 * g2]);
+          if (2 * g2 + 1 < G) {
+            const uint64_t pg1 = pack2(t.z, t.w);
+            accLo[2 * g2 + 1] = ffma2(lo, pg1, accLo[2 * g2 + 1]);
+            accHi[2 * g2 + 1] = ffma2(hi, pg1, accHi[2 * g2 + 1]);
+          }
+        }
+      }
+    }
+    if (++st == C::NS) { st = 0; parity ^= 1u; }
+  }
+
+  if (timed_out) {
+    if (tid == 0) {
+      atomicCAS(&p.status[0], 0, (int)RAP_ETIMEOUT);
+      p.status[1] = (b * p.Hkv + h) * p.n_split + split;
+      // give copies still in flight a bounded chance to land before the shared memory is released
+      for (int s = 0; s < C::NS; ++s) {
+        mbar_wait_bounded(bar0 + 8 * s, 0);
+        mbar_wait_bounded(bar0 + 8 * s, 1);
+      }
+    }
+    __syncthreads();
+    return;
+  }
+
+  // ---- reduce the PV row groups and write this split's partials --------------------------------
+  __syncthreads();
+  float* red = s_part;              // [NG][G][2 * WVP]
+  constexpr int DVP = 2 * C::WVP;
+  if (pv_active) {
+#pragma unroll
+    for (int g = 0; g < G; ++g) {
+      float a, c;
+      unpack2(accLo[g], a, c);
+      red[(grp * G + g) * DVP + 2 * wch] = a + c;
+      unpack2(accHi[g], a, c);
+      red[(grp * G + g) * DVP + 2 * wch + 1] = a + c;
+    }
+  }
+  __syncthreads();
+  for (int i = tid; i < G * DV; i += STHREADS) {
+    const int g = i / DV, c = i - g * DV;
+    float s = 0.f;
+#pragma unroll
+    for (int r = 0; r < C::NG; ++r) s += red[(r * G + g) * DVP + c];
+    ws_base[g * ws_head + c] = s;
+  }
+  if (warp < G) {
+    float l = l_lane;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
+    if (lane == 0) {
+      ws_base[warp * ws_head + DV] = m_ref;
+      ws_base[warp * ws_head + DV + 1] = l;
+    }
+  }
+}
+
+// out[b][g][c] = sum_s 2^(m_s - M) acc_s[c] / sum_s 2^(m_s - M) l_s ; empty splits have l = 0.
+__global__ void __launch_bounds__(128) attn_scan_combine_kernel(const float* __restrict__ ws, int n_split, int dv,
+                                                                float* __restrict__ out) {
+  const size_t bg = blockIdx.x;
+  const float* base = ws + bg * n_split * (size_t)(dv + 2);
+  __shared__ float wgt[RAP_MAX_SPLIT];
+  __shared__ float inv_s;
+  if (threadIdx.x < 32) {
+    float M = -INFINITY;
+    for (int s = threadIdx.x; s < n_split; s += 32)
+      if (base[(size_t)s * (dv + 2) + dv + 1] > 0.f) M = fmaxf(M, base[(size_t)s * (dv + 2) + dv]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+    float den = 0.f;
+    for (int s = threadIdx.x; s < n_split; s += 32) {
+      const float l = base[(size_t)s * (dv + 2) + dv + 1];
+      const float w = l > 0.f ? exp2f(base[(size_t)s * (dv + 2) + dv] - M) : 0.f;
+      wgt[s] = w;
+      den += w * l;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) den += __shfl_xor_sync(0xffffffffu, den, o);
+    if (threadIdx.x == 0) inv_s = den > 0.f ? 1.f / den : 0.f;
+  }
+  __syncthreads();
+  const float inv = inv_s;
+  for (int c = threadIdx.x; c < dv; c += blockDim.x) {
+    float num = 0.f;
+    for (int s = 0; s < n_split; ++s) {
+      const float w = wgt[s];
+      if (w > 0.f) num += w * base[(size_t)s * (dv + 2) + c];
+    }
+    out[bg * dv + c] = num * inv;
+  }
+}
+
+typedef void (*scan_kernel_t)(const ScanParams);
+
+struct ScanEntry {
+  int G, WK, DV, smem;
+  scan_kernel_t fn;
+};
+
+template <int G, int WK, int DV>
+constexpr ScanEntry entry() {
+  return ScanEntry{G, WK, DV, ScanCfg<G, WK, DV>::SMEM, attn_scan_kernel<G, WK, DV>};
+}
+
+// head shapes of the workloads: D = 128 at retain ratios 1.0 / 0.9 / 0.8 / 0.7 / 0.5
+#define RAP_SCAN_SHAPES(G) entry<G, 58, 115>(), entry<G, 51, 102>(), entry<G, 45, 90>(), entry<G, 32, 64>()
+const ScanEntry kScanTable[] = {
+    RAP_SCAN_SHAPES(1), RAP_SCAN_SHAPES(2), RAP_SCAN_SHAPES(3), RAP_SCAN_SHAPES(4), RAP_SCAN_SHAPES(5),
+    entry<1, 64, 128>(), entry<2, 64, 128>(), entry<3, 64, 128>(), entry<4, 64, 128>(),
+};
+
+}  // namespace
+
+// Split count: fill two CTAs per SM a whole number of times with splits of at least 8 tiles.
+int rap_scan_choose_split(const rap_ctx* ctx, int B, int Hkv, int h_len_max) {
+  const long units_total = (long)B * Hkv;
+  const int n_tiles = (h_len_max + ST - 1) / ST;
+  const long slots = 2L * ctx->sm_count;
+  double best = 1e30;
+  int n_split = 1;
+  for (int ns = 1; ns <= RAP_MAX_SPLIT; ++ns) {
+    const int tiles_per = (n_tiles + ns - 1) / ns;
+    if (ns > 1 && tiles_per < 8) break;
+    const long waves = (units_total * ns + slots - 1) / slots;
+    const double cost = (double)waves * (tiles_per + 3);
+    if (cost < best - 1e-9) { best = cost; n_split = ns; }
+  }
+  return n_split;
+}
+
+rap_status rap_launch_attn_scan(rap_ctx* ctx, const rap_attn_args& a, int n_split_req, cudaStream_t st) {
+  if (a.dtype != RAP_BF16 || (a.P2 & 1)) return RAP_EUNSUPPORTED;
+  const int G = a.Hq / a.Hkv, WK = a.P2 / 2;
+  const ScanEntry* e = nullptr;
+  for (const ScanEntry& c : kScanTable)
+    if (c.G == G && c.WK == WK && c.DV == a.dv) { e = &c; break; }
+  if (!e) return RAP_EUNSUPPORTED;
+  const int n_split = n_split_req > 0 ? n_split_req : rap_scan_choose_split(ctx, a.B, a.Hkv, a.h_len_max);
+  ScanParams p;
+  p.q = (const uint32_t*)a.q; p.k = (const unsigned char*)a.k; p.v = (const unsigned char*)a.v;
+  p.seq_len = a.seq_len; p.ws = ctx->d_attn_ws; p.status = ctx->d_status;
+  p.len_add = a.len_add; p.Hq = a.Hq; p.Hkv = a.Hkv; p.S_cap = a.S_cap; p.n_split = n_split;
+  p.qscale = (float)(1.4426950408889634 / sqrt((double)a.head_dim));
+  RAP_CUDA_TRY(ctx, cudaFuncSetAttribute(e->fn, cudaFuncAttributeMaxDynamicSharedMemorySize, e->smem));
+  dim3 grid(n_split, a.Hkv, a.B);
+  e->fn<<<grid, STHREADS, e->smem, st>>>(p);
+  ctx->launches++;
+  RAP_CUDA_TRY(ctx, cudaGetLastError());
+  attn_scan_combine_kernel<<<a.B * a.Hq, 128, 0, st>>>(ctx->d_attn_ws, n_split, a.dv, a.out);
+  ctx->launches++;
+  RAP_CUDA_TRY(ctx, cudaGetLastError());
+  return RAP_OK;
+}
