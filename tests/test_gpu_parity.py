@@ -276,3 +276,36 @@ def test_argument_validation_on_device_context():
     assert torch.all(st.k_cache[0][1] == 5.0)
     assert st.ctx.rap_get_last_device_status() == (0, 0)
     st.close()
+
+
+@pytest.mark.parametrize("dtype,pairing", [("f32", 0), ("f32", 1), ("bf16", 0)])
+def test_lowrank_comparator_matches_oracle(dtype, pairing):
+    """rap_lowrank_decode_attn (latent K rebuilt and rotated at full width every call) against the
+    oracle's definition on the same storage-rounded inputs; ragged lengths, several splits."""
+    from dataclasses import replace
+    w = replace(synth.scaled_down(synth.LLAMA_8B, n_layers=1, batch=3, seq=300), dtype=dtype, pairing=pairing,
+                head_dim=64 if dtype == "f32" else 128)
+    D, Hq, Hkv, B = w.head_dim, w.n_q_heads, w.n_kv_heads, w.batch
+    r, dv = (44, 45) if D == 64 else (90, 90)
+    lens = [300, 129, 1]
+    cap = 304
+    dt = torch.float32 if dtype == "f32" else torch.bfloat16
+    rng = np.random.default_rng(77)
+    sig = float(np.sqrt(w.hidden) * 0.02)
+    lat = O.round_storage(rng.standard_normal((B, Hkv, cap, r)) * sig, dtype)
+    V = O.round_storage(rng.standard_normal((B, Hkv, cap, dv)) * sig, dtype)
+    Bk = O.round_storage(synth.draw_lowrank_factor(w, 0, r), dtype)
+    qf = O.round_storage(rng.standard_normal((B, Hq, D)) * sig, dtype)
+    ctx = binding.RapContext(1, w.hidden, Hq, Hkv, D, w.rope_theta, pairing,
+                             binding.RAP_F32 if dtype == "f32" else binding.RAP_BF16, B)
+    dev = torch.device("cuda:0")
+    up = lambda a: torch.from_numpy(np.ascontiguousarray(a)).to(dev).to(dt).contiguous()
+    d_lat, d_V, d_Bk, d_q = up(lat), up(V), up(Bk), up(qf)
+    dl = torch.tensor(lens, dtype=torch.int32, device=dev)
+    want = O.lowrank_decode_attn(qf, lat, Bk, V, lens, D, w.rope_theta, pairing)
+    for n_split in (0, 1, 3):
+        out = torch.full((B, Hq, dv), float("nan"), dtype=torch.float32, device=dev)
+        ctx.rap_lowrank_decode_attn(B, r, dv, d_q, d_lat, d_Bk, d_V, cap, dl, max(lens), n_split, out)
+        torch.cuda.synchronize()
+        util.check_attn(util.to_np64(out), want, dtype)
+    ctx.close()
