@@ -85,27 +85,7 @@ def build_stack(w, torch, seed_offset=0):
     st = DecodeStack(w, max_rows=max(w.batch, 2048))
     ks, vs = synth.draw_scores(w)
     st.build_tables(ks, vs)
-    for l in range(w.n_layers):
-        st.set_packed_weights(l, synth.draw_packed_weights(w, l))
-    g = torch.Generator(device=st.device).manual_seed(w.seed + seed_offset)
-    sigma = float(np.sqrt(w.hidden) * 0.02)
-    for l in range(w.n_layers):
-        st.k_cache[l].normal_(0.0, sigma, generator=g)
-        st.v_cache[l].normal_(0.0, sigma, generator=g)
-    # the last T_PREFILL_TAIL positions go through the real projection + RoPE + append path
-    tail = min(T_PREFILL_TAIL, w.seq)
-    rows_b = np.repeat(np.arange(w.batch, dtype=np.int32), tail)
-    rows_p = np.tile(np.arange(w.seq - tail, w.seq, dtype=np.int32), w.batch)
-    chunk = 2048
-    for l in range(w.n_layers):
-        xg = torch.Generator(device=st.device).manual_seed(w.seed + 7919 * (l + 1))
-        for c0 in range(0, len(rows_b), chunk):
-            c1 = min(len(rows_b), c0 + chunk)
-            x = torch.empty((c1 - c0, w.hidden), dtype=st.dt, device=st.device).normal_(0.0, 1.0, generator=xg)
-            sid = torch.from_numpy(rows_b[c0:c1]).to(st.device)
-            pos = torch.from_numpy(rows_p[c0:c1]).to(st.device)
-            qo = torch.empty((c1 - c0, w.n_q_heads, 2 * st.n_pairs[l]), dtype=st.dt, device=st.device)
-            st.qkv_rope_append(l, x, sid, pos, pos, int(rows_p[c0:c1].max()), q_out=qo)
+    st.fill_synthetic(w.seed + seed_offset, tail=T_PREFILL_TAIL)
     torch.cuda.synchronize()
     return st
 

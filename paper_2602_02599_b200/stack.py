@@ -114,5 +114,33 @@ class DecodeStack:
                                       n_split, h_out, self.out_stride, advance)
         return h_out
 
+    def fill_synthetic(self, seed, tail=256, chunk=2048):
+        """Seeded synthetic state for the large workloads: packed weights N(0, 0.02^2) from synth, cache
+        positions [0, seq) filled on the device with iid N(0, hidden * 0.02^2) (the law of projected
+        hidden states), then the last `tail` positions of every sequence rewritten through
+        rap_qkv_rope_append in `chunk`-row calls so the real append path is exercised at scale."""
+        from . import synth
+        w = self.w
+        for l in range(self.L):
+            self.set_packed_weights(l, synth.draw_packed_weights(w, l))
+        g = torch.Generator(device=self.device).manual_seed(seed)
+        sigma = float(np.sqrt(w.hidden) * 0.02)
+        for l in range(self.L):
+            self.k_cache[l].normal_(0.0, sigma, generator=g)
+            self.v_cache[l].normal_(0.0, sigma, generator=g)
+        tail = min(tail, w.seq)
+        rows_b = np.repeat(np.arange(self.B, dtype=np.int32), tail)
+        rows_p = np.tile(np.arange(w.seq - tail, w.seq, dtype=np.int32), self.B)
+        for l in range(self.L):
+            xg = torch.Generator(device=self.device).manual_seed(seed + 7919 * (l + 1))
+            for c0 in range(0, len(rows_b), chunk):
+                c1 = min(len(rows_b), c0 + chunk)
+                x = torch.empty((c1 - c0, w.hidden), dtype=self.dt, device=self.device).normal_(0.0, 1.0, generator=xg)
+                sid = torch.from_numpy(rows_b[c0:c1]).to(self.device)
+                pos = torch.from_numpy(rows_p[c0:c1]).to(self.device)
+                qo = torch.empty((c1 - c0, w.n_q_heads, 2 * self.n_pairs[l]), dtype=self.dt, device=self.device)
+                self.qkv_rope_append(l, x, sid, pos, pos, int(rows_p[c0:c1].max()), q_out=qo)
+        torch.cuda.synchronize()
+
     def close(self):
         self.ctx.close()
