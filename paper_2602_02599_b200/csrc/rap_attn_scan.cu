@@ -43,10 +43,16 @@ constexpr int cround(int x, int m) { return (x + m - 1) / m * m; }
 template <int G, int WK, int DV>
 struct ScanCfg {
   static constexpr int KV = (WK % 2) ? 1 : (WK % 4) ? 2 : 4;   // 32-bit words per K read
-  static constexpr bool KPAD = (WK % 8) == 0;                  // row-by-row copies to a padded stride
+  // Rows of 128 / 256 bytes put every row on the same banks.  For those the logits mapping is
+  // rotated: the 8 lanes of a quarter warp read 8 consecutive 16-byte units of ONE row (a contiguous
+  // 128 bytes), lane j of the quarter owns units j, j + 8, ..., and the chunk index of the partial
+  // logits is j instead of the warp.  Other multiples of 32 bytes fall back to padded row copies.
+  static constexpr bool KROT = (WK % 32) == 0;
+  static constexpr bool KPAD = (WK % 8) == 0 && !KROT;         // row-by-row copies to a padded stride
   static constexpr int KS = KPAD ? WK + 4 : WK;                // K row stride in shared memory (words)
   static constexpr int UNITS = WK / KV;
-  static constexpr int CLU = (UNITS + SCHUNKS - 1) / SCHUNKS;  // reads per lane, row and chunk
+  static constexpr int CLU = KROT ? UNITS / SCHUNKS : (UNITS + SCHUNKS - 1) / SCHUNKS;  // reads per lane and row
+  static constexpr int SPS = KROT ? G * ST + 4 : G * ST;       // partial-logit floats per chunk (bank-shifted when rotated)
   static constexpr int CL = CLU * KV;                          // words per chunk
   static constexpr bool VODD = (DV & 1) != 0;
   static constexpr int WVP = (DV + 1) / 2;                     // channel pairs per V row
@@ -57,7 +63,7 @@ struct ScanCfg {
   static constexpr int Gp = (G + 1) & ~1;
   static constexpr int GS = cround(IP * Gp * 2, 32) + 8;       // p floats per group (bank-shifted)
   static constexpr int OFF_SPART = 128;
-  static constexpr int OFF_PP = OFF_SPART + SCHUNKS * G * ST * 4;
+  static constexpr int OFF_PP = OFF_SPART + SCHUNKS * SPS * 4;
   static constexpr int OFF_ALPHA = OFF_PP + cround(NG * GS * 4, 16);
   static constexpr int OFF_STAGE = cround(OFF_ALPHA + 32, 128);
   static constexpr int V_OFF = cround(ST * KS * 4, 128);
@@ -66,7 +72,7 @@ struct ScanCfg {
   static constexpr int NS = NS_RAW > 4 ? 4 : NS_RAW;
   static constexpr int SMEM = OFF_STAGE + NS * STAGE_BYTES;
   static_assert(NS >= 2, "tile ring needs two stages");
-  static_assert(NG * 2 * WVP * G <= SCHUNKS * G * ST, "row-group reduction reuses the partial-logit buffer");
+  static_assert(NG * 2 * WVP * G <= SCHUNKS * SPS, "row-group reduction reuses the partial-logit buffer");
 };
 
 struct ScanParams {
@@ -224,15 +230,18 @@ __global__ void __launch_bounds__(STHREADS, 2) attn_scan_kernel(const ScanParams
   // ---- this warp's dim chunk and its pre-scaled q registers ---------------------------------
   const int u_nom = warp * C::CLU;                         // first unit this chunk is responsible for
   const int u0 = min(u_nom, C::UNITS - C::CLU);            // first unit it reads (shifted back into the row)
-  const int w0 = u0 * C::KV;
+  const int w0 = C::KROT ? (lane & 7) * 4 : u0 * C::KV;    // first word this thread reads in a row
+  const int ustep = C::KROT ? 32 : C::KV;                  // words between its consecutive reads
+  const int krow = C::KROT ? warp * 4 + (lane >> 3) : lane;   // its rows: krow and krow + 32
+  const int kchunk = C::KROT ? (lane & 7) : warp;          // which of the 8 partial sums it produces
   uint64_t qr[G][C::CL];
 #pragma unroll
   for (int g = 0; g < G; ++g) {
     const uint32_t* qrow = p.q + ((size_t)b * p.Hq + (size_t)h * G + g) * WK;
 #pragma unroll
     for (int i = 0; i < C::CL; ++i) {
-      const bool mine = (u0 + i / C::KV) >= u_nom;
-      const uint32_t x = mine ? qrow[w0 + i] : 0u;
+      const bool mine = C::KROT || (u0 + i / C::KV) >= u_nom;
+      const uint32_t x = mine ? qrow[w0 + (i / C::KV) * ustep + i % C::KV] : 0u;
       qr[g][i] = pack2(__uint_as_float(x << 16) * p.qscale, __uint_as_float(x & 0xffff0000u) * p.qscale);
     }
   }
@@ -273,7 +282,7 @@ __global__ void __launch_bounds__(STHREADS, 2) attn_scan_kernel(const ScanParams
 
     // ---- logits partials: rows lane, lane + 32; words [w0, w0 + CL) ------------------------
     {
-      const uint32_t* r0 = reinterpret_cast<const uint32_t*>(stage) + lane * C::KS + w0;
+      const uint32_t* r0 = reinterpret_cast<const uint32_t*>(stage) + krow * C::KS + w0;
       const uint32_t* r1 = r0 + 32 * C::KS;
       uint64_t a0[G], a1[G];
 #pragma unroll
@@ -281,8 +290,8 @@ __global__ void __launch_bounds__(STHREADS, 2) attn_scan_kernel(const ScanParams
 #pragma unroll
       for (int u = 0; u < C::CLU; ++u) {
         uint32_t x0[C::KV], x1[C::KV];
-        ld_words<C::KV>(r0 + u * C::KV, x0);
-        ld_words<C::KV>(r1 + u * C::KV, x1);
+        ld_words<C::KV>(r0 + u * ustep, x0);
+        ld_words<C::KV>(r1 + u * ustep, x1);
 #pragma unroll
         for (int j = 0; j < C::KV; ++j) {
           const uint64_t k0 = pack2u(x0[j] << 16, x0[j] & 0xffff0000u);
@@ -298,9 +307,9 @@ __global__ void __launch_bounds__(STHREADS, 2) attn_scan_kernel(const ScanParams
       for (int g = 0; g < G; ++g) {
         float e, o;
         unpack2(a0[g], e, o);
-        s_part[(warp * G + g) * ST + lane] = e + o;
+        s_part[kchunk * C::SPS + g * ST + krow] = e + o;
         unpack2(a1[g], e, o);
-        s_part[(warp * G + g) * ST + lane + 32] = e + o;
+        s_part[kchunk * C::SPS + g * ST + krow + 32] = e + o;
       }
     }
     if (__syncthreads_or(!ok)) {   // sync #1: partial logits visible; the previous tile's stage is free
@@ -315,8 +324,8 @@ __global__ void __launch_bounds__(STHREADS, 2) attn_scan_kernel(const ScanParams
       float s0 = 0.f, s1 = 0.f;
 #pragma unroll
       for (int c = 0; c < SCHUNKS; ++c) {
-        s0 += s_part[(c * G + g) * ST + lane];
-        s1 += s_part[(c * G + g) * ST + lane + 32];
+        s0 += s_part[c * C::SPS + g * ST + lane];
+        s1 += s_part[c * C::SPS + g * ST + lane + 32];
       }
       if (lane >= nj) s0 = -INFINITY;
       if (lane + 32 >= nj) s1 = -INFINITY;
