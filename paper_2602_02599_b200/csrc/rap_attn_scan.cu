@@ -31,7 +31,6 @@
 
 namespace {
 
-constexpr int ST = 64;           // positions per tile
 constexpr int STHREADS = 256;
 constexpr int SCHUNKS = 8;       // dim chunks of the logits phase (= warps)
 constexpr uint32_t WAIT_LIMIT = 1u << 21;
@@ -40,8 +39,22 @@ constexpr float LAZY_MAX_SLACK = 8.f;
 
 constexpr int cround(int x, int m) { return (x + m - 1) / m * m; }
 
+// positions per tile: the largest multiple of 32 (up to 192) whose two-stage ring fits beside the
+// partial-logit and p buffers of a CTA (two CTAs per SM).  Large tiles spread the per-tile costs
+// (barriers, waits, softmax bookkeeping) over more bytes and keep a whole tile in flight.
+constexpr int scan_smem_bound(int G, int row_bytes, int st) {
+  return 128 + SCHUNKS * (G * st + 4) * 4 + 3584 + 2 * (st * row_bytes + 256);
+}
+constexpr int scan_tile_rows(int G, int row_bytes) {
+  for (int st = 192; st > 64; st -= 32)
+    if (scan_smem_bound(G, row_bytes, st) <= SMEM_BUDGET) return st;
+  return 64;
+}
+
 template <int G, int WK, int DV>
 struct ScanCfg {
+  static constexpr int ST = scan_tile_rows(G, WK * 4 + DV * 2);   // positions per tile
+  static constexpr int RL = ST / 32;                           // rows per lane in the logits / softmax phases
   static constexpr int KV = (WK % 2) ? 1 : (WK % 4) ? 2 : 4;   // 32-bit words per K read
   // Rows of 128 / 256 bytes put every row on the same banks.  For those the logits mapping is
   // rotated: the 8 lanes of a quarter warp read 8 consecutive 16-byte units of ONE row (a contiguous
@@ -164,6 +177,7 @@ template <int G, int WK, int DV>
 __global__ void __launch_bounds__(STHREADS, 2) attn_scan_kernel(const ScanParams p) {
   using C = ScanCfg<G, WK, DV>;
   constexpr int Gp = C::Gp;
+  constexpr int ST = C::ST, RL = C::RL;
   extern __shared__ __align__(128) unsigned char smem[];
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem);
   float* s_part = reinterpret_cast<float*>(smem + C::OFF_SPART);   // [SCHUNKS][G][ST]; reused for the group reduction
@@ -258,11 +272,11 @@ __global__ void __launch_bounds__(STHREADS, 2) attn_scan_kernel(const ScanParams
 
   // softmax role: warp g < G, lanes own positions lane and lane + 32
   float m_ref = -INFINITY, l_lane = 0.f;
-  int pidx0, pidx1;
-  {
-    const int g0 = lane % C::NG, i0 = lane / C::NG, g1 = (lane + 32) % C::NG, i1 = (lane + 32) / C::NG;
-    pidx0 = g0 * C::GS + (i0 >> 1) * Gp * 2 + (i0 & 1) + 2 * warp;
-    pidx1 = g1 * C::GS + (i1 >> 1) * Gp * 2 + (i1 & 1) + 2 * warp;
+  int pidx[RL];
+#pragma unroll
+  for (int k = 0; k < RL; ++k) {
+    const int j = lane + 32 * k, gj = j % C::NG, ij = j / C::NG;
+    pidx[k] = gj * C::GS + (ij >> 1) * Gp * 2 + (ij & 1) + 2 * warp;
   }
   bool timed_out = false;
   int st = 0;
@@ -282,34 +296,42 @@ __global__ void __launch_bounds__(STHREADS, 2) attn_scan_kernel(const ScanParams
 
     // ---- logits partials: rows lane, lane + 32; words [w0, w0 + CL) ------------------------
     {
-      const uint32_t* r0 = reinterpret_cast<const uint32_t*>(stage) + krow * C::KS + w0;
-      const uint32_t* r1 = r0 + 32 * C::KS;
-      uint64_t a0[G], a1[G];
+      const uint32_t* rbase = reinterpret_cast<const uint32_t*>(stage) + krow * C::KS + w0;
 #pragma unroll
-      for (int g = 0; g < G; ++g) a0[g] = a1[g] = 0ull;
+      for (int rr = 0; rr < RL; rr += 2) {       // two rows (krow + 32 rr, krow + 32 rr + 32) per pass
+        const bool two = rr + 1 < RL;
+        const uint32_t* r0 = rbase + rr * 32 * C::KS;
+        const uint32_t* r1 = r0 + (two ? 32 * C::KS : 0);
+        uint64_t a0[G], a1[G];
 #pragma unroll
-      for (int u = 0; u < C::CLU; ++u) {
-        uint32_t x0[C::KV], x1[C::KV];
-        ld_words<C::KV>(r0 + u * ustep, x0);
-        ld_words<C::KV>(r1 + u * ustep, x1);
+        for (int g = 0; g < G; ++g) a0[g] = a1[g] = 0ull;
 #pragma unroll
-        for (int j = 0; j < C::KV; ++j) {
-          const uint64_t k0 = pack2u(x0[j] << 16, x0[j] & 0xffff0000u);
-          const uint64_t k1 = pack2u(x1[j] << 16, x1[j] & 0xffff0000u);
+        for (int u = 0; u < C::CLU; ++u) {
+          uint32_t x0[C::KV], x1[C::KV];
+          ld_words<C::KV>(r0 + u * ustep, x0);
+          if (two) ld_words<C::KV>(r1 + u * ustep, x1);
 #pragma unroll
-          for (int g = 0; g < G; ++g) {
-            a0[g] = ffma2(k0, qr[g][u * C::KV + j], a0[g]);
-            a1[g] = ffma2(k1, qr[g][u * C::KV + j], a1[g]);
+          for (int j = 0; j < C::KV; ++j) {
+            const uint64_t k0 = pack2u(x0[j] << 16, x0[j] & 0xffff0000u);
+#pragma unroll
+            for (int g = 0; g < G; ++g) a0[g] = ffma2(k0, qr[g][u * C::KV + j], a0[g]);
+            if (two) {
+              const uint64_t k1 = pack2u(x1[j] << 16, x1[j] & 0xffff0000u);
+#pragma unroll
+              for (int g = 0; g < G; ++g) a1[g] = ffma2(k1, qr[g][u * C::KV + j], a1[g]);
+            }
           }
         }
-      }
 #pragma unroll
-      for (int g = 0; g < G; ++g) {
-        float e, o;
-        unpack2(a0[g], e, o);
-        s_part[kchunk * C::SPS + g * ST + krow] = e + o;
-        unpack2(a1[g], e, o);
-        s_part[kchunk * C::SPS + g * ST + krow + 32] = e + o;
+        for (int g = 0; g < G; ++g) {
+          float e, o;
+          unpack2(a0[g], e, o);
+          s_part[kchunk * C::SPS + g * ST + krow + rr * 32] = e + o;
+          if (two) {
+            unpack2(a1[g], e, o);
+            s_part[kchunk * C::SPS + g * ST + krow + rr * 32 + 32] = e + o;
+          }
+        }
       }
     }
     if (__syncthreads_or(!ok)) {   // sync #1: partial logits visible; the previous tile's stage is free
@@ -321,15 +343,20 @@ __global__ void __launch_bounds__(STHREADS, 2) attn_scan_kernel(const ScanParams
     // ---- online softmax: warp g owns head g --------------------------------------------------
     if (warp < G) {
       const int g = warp;
-      float s0 = 0.f, s1 = 0.f;
+      float sv[RL];
+#pragma unroll
+      for (int k = 0; k < RL; ++k) sv[k] = 0.f;
 #pragma unroll
       for (int c = 0; c < SCHUNKS; ++c) {
-        s0 += s_part[c * C::SPS + g * ST + lane];
-        s1 += s_part[c * C::SPS + g * ST + lane + 32];
+#pragma unroll
+        for (int k = 0; k < RL; ++k) sv[k] += s_part[c * C::SPS + g * ST + lane + 32 * k];
       }
-      if (lane >= nj) s0 = -INFINITY;
-      if (lane + 32 >= nj) s1 = -INFINITY;
-      float mx = fmaxf(s0, s1);
+      float mx = -INFINITY;
+#pragma unroll
+      for (int k = 0; k < RL; ++k) {
+        if (lane + 32 * k >= nj) sv[k] = -INFINITY;
+        mx = fmaxf(mx, sv[k]);
+      }
       float alpha = 1.f;
       if (__any_sync(0xffffffffu, mx > m_ref + LAZY_MAX_SLACK)) {
 #pragma unroll
@@ -339,10 +366,12 @@ __global__ void __launch_bounds__(STHREADS, 2) attn_scan_kernel(const ScanParams
         l_lane *= alpha;
         m_ref = m_new;
       }
-      const float p0 = exp2f(s0 - m_ref), p1 = exp2f(s1 - m_ref);
-      l_lane += p0 + p1;
-      pp[pidx0] = p0;
-      pp[pidx1] = p1;
+#pragma unroll
+      for (int k = 0; k < RL; ++k) {
+        const float pk = exp2f(sv[k] - m_ref);
+        l_lane += pk;
+        pp[pidx[k]] = pk;
+      }
       if (lane == 0) alpha_s[g] = alpha;
     }
     __syncthreads();   // sync #2: p and alpha visible
@@ -492,13 +521,13 @@ __global__ void __launch_bounds__(128) attn_scan_combine_kernel(const float* __r
 typedef void (*scan_kernel_t)(const ScanParams);
 
 struct ScanEntry {
-  int G, WK, DV, smem;
+  int G, WK, DV, smem, tile;
   scan_kernel_t fn;
 };
 
 template <int G, int WK, int DV>
 constexpr ScanEntry entry() {
-  return ScanEntry{G, WK, DV, ScanCfg<G, WK, DV>::SMEM, attn_scan_kernel<G, WK, DV>};
+  return ScanEntry{G, WK, DV, ScanCfg<G, WK, DV>::SMEM, ScanCfg<G, WK, DV>::ST, attn_scan_kernel<G, WK, DV>};
 }
 
 // head shapes of the workloads: D = 128 at retain ratios 1.0 / 0.9 / 0.8 / 0.7 / 0.5
@@ -511,9 +540,9 @@ const ScanEntry kScanTable[] = {
 }  // namespace
 
 // Split count: fill two CTAs per SM a whole number of times with splits of at least 8 tiles.
-int rap_scan_choose_split(const rap_ctx* ctx, int B, int Hkv, int h_len_max) {
+int rap_scan_choose_split(const rap_ctx* ctx, int B, int Hkv, int h_len_max, int tile_rows) {
   const long units_total = (long)B * Hkv;
-  const int n_tiles = (h_len_max + ST - 1) / ST;
+  const int n_tiles = (h_len_max + tile_rows - 1) / tile_rows;
   const long slots = 2L * ctx->sm_count;
   double best = 1e30;
   int n_split = 1;
@@ -534,7 +563,7 @@ rap_status rap_launch_attn_scan(rap_ctx* ctx, const rap_attn_args& a, int n_spli
   for (const ScanEntry& c : kScanTable)
     if (c.G == G && c.WK == WK && c.DV == a.dv) { e = &c; break; }
   if (!e) return RAP_EUNSUPPORTED;
-  const int n_split = n_split_req > 0 ? n_split_req : rap_scan_choose_split(ctx, a.B, a.Hkv, a.h_len_max);
+  const int n_split = n_split_req > 0 ? n_split_req : rap_scan_choose_split(ctx, a.B, a.Hkv, a.h_len_max, e->tile);
   ScanParams p;
   p.q = (const uint32_t*)a.q; p.k = (const unsigned char*)a.k; p.v = (const unsigned char*)a.v;
   p.seq_len = a.seq_len; p.ws = ctx->d_attn_ws; p.status = ctx->d_status;
