@@ -38,11 +38,13 @@ def load_peaks():
 
 
 def load_traffic(workload):
-    """DRAM bytes per attention-scan launch from the committed ncu summary, if one exists."""
-    path = os.path.join(ROOT, "profiles", "attn_scan_traffic.json")
+    """DRAM bytes per attention-scan launch from the committed ncu summary, if it lists this workload."""
+    path = os.path.join(ROOT, "profiles", "attn_scan_traffic.txt")
     if os.path.exists(path):
-        d = json.load(open(path))
-        return d.get(workload)
+        for line in open(path):
+            f = line.split()
+            if len(f) == 2 and f[0] == workload:
+                return float(f[1])
     return None
 
 
