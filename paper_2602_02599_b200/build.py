@@ -12,7 +12,7 @@ INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "librap_b200.so")
 OBJ = os.path.join(HERE, "_build")
 SOURCES = ["rap_api.cu", "rap_proj.cu", "rap_proj_tc.cu", "rap_attn.cu", "rap_attn_fast.cu", "rap_attn_scan.cu",
-           "rap_lowrank.cu"]
+           "rap_lowrank.cu", "rap_lowrank_tc.cu"]
 
 
 def _stale():

@@ -535,6 +535,8 @@ constexpr ScanEntry entry() {
 const ScanEntry kScanTable[] = {
     RAP_SCAN_SHAPES(1), RAP_SCAN_SHAPES(2), RAP_SCAN_SHAPES(3), RAP_SCAN_SHAPES(4), RAP_SCAN_SHAPES(5),
     entry<1, 64, 128>(), entry<2, 64, 128>(), entry<3, 64, 128>(), entry<4, 64, 128>(),
+    // full-width K with a pruned V: the second pass of the low-rank comparator
+    entry<4, 64, 115>(), entry<4, 64, 102>(), entry<4, 64, 90>(), entry<4, 64, 64>(),
 };
 
 }  // namespace

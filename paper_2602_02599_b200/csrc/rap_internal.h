@@ -30,6 +30,11 @@ struct rap_ctx {
   void* d_stage_x = nullptr;      // staging for rap_decode_step_host
   float* d_stage_out = nullptr;
   void* d_stage_q = nullptr;
+  void* d_lr_k = nullptr;         // low-rank comparator: rebuilt, rotated full-width K (grown on demand)
+  size_t lr_k_bytes = 0;
+  void* d_lr_cs = nullptr;        // low-rank comparator: (cos, sin) table [positions][D/2]
+  size_t lr_cs_bytes = 0;
+  int lr_cs_len = 0;              // positions the table currently covers
   size_t stage_x_bytes = 0, stage_out_bytes = 0;
   // pinned host staging for rap_build_tables
   void* h_tables = nullptr;

@@ -180,7 +180,13 @@ __global__ void lowrank_combine_kernel(const float* __restrict__ ws, int n_split
 
 }  // namespace
 
+rap_status rap_launch_lowrank_fast(rap_ctx* ctx, const rap_lowrank_args& a, cudaStream_t st);
+
 rap_status rap_launch_lowrank_attn(rap_ctx* ctx, const rap_lowrank_args& a, cudaStream_t st) {
+  if (ctx->attn_variant == 0) {   // tensor-core rebuild + shape-specialised scan when the shape allows
+    const rap_status f = rap_launch_lowrank_fast(ctx, a, st);
+    if (f != RAP_EUNSUPPORTED) return f;
+  }
   const int G = a.Hq / a.Hkv, D = a.head_dim;
   if (a.dv > LR_THREADS) return RAP_EUNSUPPORTED;
   int n_split = a.n_split;

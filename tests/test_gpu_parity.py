@@ -303,9 +303,12 @@ def test_lowrank_comparator_matches_oracle(dtype, pairing):
     d_lat, d_V, d_Bk, d_q = up(lat), up(V), up(Bk), up(qf)
     dl = torch.tensor(lens, dtype=torch.int32, device=dev)
     want = O.lowrank_decode_attn(qf, lat, Bk, V, lens, D, w.rope_theta, pairing)
-    for n_split in (0, 1, 3):
-        out = torch.full((B, Hq, dv), float("nan"), dtype=torch.float32, device=dev)
-        ctx.rap_lowrank_decode_attn(B, r, dv, d_q, d_lat, d_Bk, d_V, cap, dl, max(lens), n_split, out)
-        torch.cuda.synchronize()
-        util.check_attn(util.to_np64(out), want, dtype)
+    for variant in (0, 1):      # 0: tensor-core rebuild + fast scan where the shape allows; 1: reference kernel
+        ctx.rap_set_attn_variant(variant)
+        for n_split in (0, 1, 3):
+            out = torch.full((B, Hq, dv), float("nan"), dtype=torch.float32, device=dev)
+            ctx.rap_lowrank_decode_attn(B, r, dv, d_q, d_lat, d_Bk, d_V, cap, dl, max(lens), n_split, out)
+            torch.cuda.synchronize()
+            util.check_attn(util.to_np64(out), want, dtype)
+    assert ctx.rap_get_last_device_status() == (0, 0)
     ctx.close()
