@@ -308,6 +308,64 @@ def run_reference(args):
     }), flush=True)
 
 
+def run_sweep(args):
+    """Retain-ratio sweep on the 8B shape (batch 16, 16384-token cache, two layers resident): time of
+    rap_decode_attn per layer at each rho against the same kernel at rho = 1 (dense), and against the
+    low-rank comparator at equal cached dims (latent K of width 2P rebuilt and rotated every call)."""
+    import torch
+    from dataclasses import replace
+    from paper_2602_02599_b200.stack import DecodeStack
+    torch.cuda.set_device(0)
+    rows, dense_ms = [], None
+    for rho in sorted(synth.SWEEP_COUNTS, reverse=True):
+        w = replace(synth.sweep_workload(rho), n_layers=2)
+        st = DecodeStack(w)
+        st.build_tables(*synth.draw_scores(w))
+        g = torch.Generator(device=st.device).manual_seed(w.seed)
+        sigma = float(np.sqrt(w.hidden) * 0.02)
+        for l in range(2):
+            st.k_cache[l].normal_(0.0, sigma, generator=g)
+            st.v_cache[l].normal_(0.0, sigma, generator=g)
+        n = w.seq + 1
+        q = torch.empty((w.batch, w.n_q_heads, 2 * w.n_pairs), dtype=st.dt, device=st.device).normal_(0, sigma, generator=g)
+        qf = torch.empty((w.batch, w.n_q_heads, w.head_dim), dtype=st.dt, device=st.device).normal_(0, sigma, generator=g)
+        bk = torch.from_numpy(synth.draw_lowrank_factor(w, 0, 2 * w.n_pairs)).to(st.device).to(st.dt).contiguous()
+        dl = torch.full((w.batch,), n, dtype=torch.int32, device=st.device)
+        out = torch.empty((w.batch, w.n_q_heads, w.n_vch), dtype=torch.float32, device=st.device)
+
+        def timed(fn):
+            for i in range(args.warmup):
+                fn(i & 1)
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for i in range(args.steps):
+                fn(i & 1)          # alternate the two layers: 2 x ~1 GB of cache, larger than L2
+            e1.record()
+            torch.cuda.synchronize()
+            return e0.elapsed_time(e1) / args.steps
+
+        rap_ms = timed(lambda l: st.decode_attn(l, q, dl, n))
+        low_ms = timed(lambda l: st.ctx.rap_lowrank_decode_attn(w.batch, 2 * w.n_pairs, w.n_vch, qf, st.k_cache[l], bk,
+                                                                st.v_cache[l], st.s_cap, dl, n, 0, out))
+        code, detail = st.ctx.rap_get_last_device_status()
+        assert code == 0, (code, detail)
+        if rho == 1.0:
+            dense_ms = rap_ms
+        by = attn_bytes(w, n)
+        rows.append({"rho": rho, "P": w.n_pairs, "dv": w.n_vch, "kv_bytes_per_layer": by, "rap_attn_ms": rap_ms,
+                     "rap_GBps": by / rap_ms / 1e6, "rap_vs_dense": rap_ms / dense_ms,
+                     "bytes_vs_dense": (2 * w.n_pairs + w.n_vch) / 256.0, "lowrank_attn_ms": low_ms,
+                     "lowrank_vs_dense": low_ms / dense_ms})
+        st.close()
+        del st, q, qf, bk, out
+        torch.cuda.empty_cache()
+    print(json.dumps({"metric": "attention_cost_ratio_vs_dense", "unit": "ratio", "n_gpus": 1, "steps": args.steps,
+                      "warmup": args.warmup, "dtype": "bf16", "data": "synthetic", "higher_is_better": False,
+                      "config": {"workload": "sweep on the 8B shape: 32q/8kv heads, D=128, B=16, S=16384, 2 layers resident"},
+                      "sweep": rows}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -319,6 +377,7 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="cut the workload to this many layers (profiling)")
     ap.add_argument("--batch", type=int, default=0, help="cut the workload to this batch (profiling)")
     ap.add_argument("--seq", type=int, default=0, help="cut the workload to this context (profiling)")
+    ap.add_argument("--sweep", action="store_true", help="retain-ratio sweep with the dense and low-rank comparators")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
@@ -326,6 +385,8 @@ def main():
         args.cpu_baseline = False
     if args.impl == "reference":
         run_reference(args)
+    elif args.sweep:
+        run_sweep(args)
     else:
         run_ours(args)
 

@@ -97,7 +97,44 @@ struct ScanParams {
   int32_t* status;
   int len_add, Hq, Hkv, S_cap, n_split;
   float qscale;
+  int B;           // sequences (used by the balanced mode)
+  int balanced;    // 0: grid (n_split, H_kv, B), equal tile ranges per split; 1: grid (CTAs), see SkPlan
 };
+
+// Balanced mode.  All tiles of all (sequence, KV head) units form one sequence, unit-major, of T
+// tiles; CTA c of NC scans the tiles [c T / NC, (c + 1) T / NC), whatever units they belong to, so
+// every CTA does the same amount of work for any batch, length mix and SM count.  A unit touched by
+// several CTAs gets one partial per CTA ("segment"); segment index = CTA - first CTA of the unit.
+// NC is capped so that no unit has more than RAP_MAX_SPLIT segments.  The scan and the combine
+// kernel derive the same plan from seq_len with the helpers below.
+struct SkPlan {
+  int T;           // total tiles (the host side keeps B * H_kv * S_cap / 64 below 2^31)
+  int nc;          // CTAs that take part (<= gridDim.x)
+};
+__device__ __forceinline__ int sk_tiles_of(const int32_t* seq_len, int b, int len_add, int S_cap, int tile_rows) {
+  const int len = min(max(seq_len[b] + len_add, 0), S_cap);
+  return (len + tile_rows - 1) / tile_rows;
+}
+__device__ __forceinline__ SkPlan sk_plan(const int32_t* seq_len, int B, int Hkv, int len_add, int S_cap, int tile_rows,
+                                          int grid) {
+  long long T = 0;
+  int n_max = 0;
+  for (int b = 0; b < B; ++b) {
+    const int n = sk_tiles_of(seq_len, b, len_add, S_cap, tile_rows);
+    T += (long long)n * Hkv;
+    n_max = max(n_max, n);
+  }
+  SkPlan pl;
+  pl.T = (int)T;
+  pl.nc = 0;
+  if (T > 0) {
+    const long long cap = (long long)(RAP_MAX_SPLIT - 2) * T / n_max;     // segments per unit <= n_max NC / T + 2
+    pl.nc = (int)max(1LL, min(min((long long)grid, cap), T));             // and every CTA owns at least one tile
+  }
+  return pl;
+}
+// first CTA whose range holds global tile s:  max c with floor(c T / NC) <= s
+__device__ __forceinline__ int sk_cta_of(int s, const SkPlan& pl) { return (int)((((long long)s + 1) * pl.nc - 1) / pl.T); }
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -185,29 +222,37 @@ __global__ void __launch_bounds__(STHREADS, 2) attn_scan_kernel(const ScanParams
   float* alpha_s = reinterpret_cast<float*>(smem + C::OFF_ALPHA);
   unsigned char* stages = smem + C::OFF_STAGE;
 
-  const int split = blockIdx.x, h = blockIdx.y, b = blockIdx.z;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  int len = p.seq_len[b] + p.len_add;
-  len = min(max(len, 0), p.S_cap);
-  const int n_tiles = (len + ST - 1) / ST;
-  const int tps = (n_tiles + p.n_split - 1) / p.n_split;
-  const int t_begin = min(n_tiles, split * tps), t_end = min(n_tiles, t_begin + tps);
-  const int n_my = t_end - t_begin;
-  const int len8 = (len + 7) & ~7;      // rows a copy may touch: S_cap is a multiple of 8
-  float* ws_base = p.ws + (((size_t)b * p.Hq + (size_t)h * G) * p.n_split + split) * (size_t)(DV + 2);
-  const size_t ws_head = (size_t)p.n_split * (DV + 2);
-
-  if (n_my <= 0) {   // nothing to scan: neutral partials
-    for (int i = tid; i < G * (DV + 2); i += STHREADS) {
-      const int g = i / (DV + 2), c = i - g * (DV + 2);
-      ws_base[g * ws_head + c] = (c == DV) ? -INFINITY : 0.f;
+  // what the current segment scans: tiles [t_begin, t_begin + n_my) of unit (b, h), partials to ws_base
+  int b = 0, h = 0, len = 0, len8 = 0, t_begin = 0, n_my = 0;
+  float* ws_base = nullptr;
+  size_t ws_head = 0;
+  const unsigned char* kg = nullptr;
+  const unsigned char* vg = nullptr;
+  // balanced mode: this CTA's range [cur, hi) of global tiles and the plan it comes from
+  SkPlan plan;
+  plan.T = 0; plan.nc = 0;
+  int cur = 0, hi = 0, unit_start = 0;
+  if (p.balanced) {
+    plan = sk_plan(p.seq_len, p.B, p.Hkv, p.len_add, p.S_cap, ST, (int)gridDim.x);
+    if ((int)blockIdx.x >= plan.nc) return;
+    cur = (int)((long long)blockIdx.x * plan.T / plan.nc);
+    hi = (int)((long long)(blockIdx.x + 1) * plan.T / plan.nc);
+    if (cur >= hi) return;
+    // the unit that holds tile `cur`
+    int pb = 0;
+    for (b = 0; b < p.B; ++b) {
+      const int nb = sk_tiles_of(p.seq_len, b, p.len_add, p.S_cap, ST) * p.Hkv;
+      if (cur < pb + nb) break;
+      pb += nb;
     }
-    return;
+    const int ntb = sk_tiles_of(p.seq_len, b, p.len_add, p.S_cap, ST);
+    h = (cur - pb) / ntb;
+    unit_start = pb + h * ntb;
+  } else {
+    b = blockIdx.z;
+    h = blockIdx.y;
   }
-
-  const size_t unit = (size_t)b * p.Hkv + h;
-  const unsigned char* kg = p.k + unit * (size_t)p.S_cap * (size_t)(WK * 4);
-  const unsigned char* vg = p.v + unit * (size_t)p.S_cap * (size_t)(DV * 2);
   const uint32_t bar0 = smem_u32(bars);
   const uint32_t stage0 = smem_u32(stages);
 
@@ -236,11 +281,6 @@ __global__ void __launch_bounds__(STHREADS, 2) attn_scan_kernel(const ScanParams
     }
     if (lane == 0) bulk_g2s(dst + C::V_OFF, vg + (size_t)j0 * (DV * 2), vb, bar);
   };
-  if (warp == 0) {
-    const int pre = min(n_my, C::NS - 1);
-    for (int tl = 0; tl < pre; ++tl) issue_tile(tl, tl);
-  }
-
   // ---- this warp's dim chunk and its pre-scaled q registers ---------------------------------
   const int u_nom = warp * C::CLU;                         // first unit this chunk is responsible for
   const int u0 = min(u_nom, C::UNITS - C::CLU);            // first unit it reads (shifted back into the row)
@@ -249,6 +289,62 @@ __global__ void __launch_bounds__(STHREADS, 2) attn_scan_kernel(const ScanParams
   const int krow = C::KROT ? warp * 4 + (lane >> 3) : lane;   // its rows: krow and krow + 32
   const int kchunk = C::KROT ? (lane & 7) : warp;          // which of the 8 partial sums it produces
   uint64_t qr[G][C::CL];
+
+  // ---- PV role ------------------------------------------------------------------------------
+  const int grp = tid / C::WVP, wch = tid - grp * C::WVP;
+  const bool pv_active = grp < C::NG;
+  const bool last_slot_ok = grp < C::LASTN;    // does this group own a row in slot RPG - 1 ?
+  const bool has_hi = 2 * wch + 1 < DV;        // odd DV: the last channel pair has one channel
+  uint64_t accLo[G], accHi[G];     // (even-slot rows, odd-slot rows) partial sums of channels 2*wch and 2*wch+1
+  const float* ppg = pp + (pv_active ? grp : 0) * C::GS;
+
+  // softmax role: warp g < G, lanes own positions lane and lane + 32
+  float m_ref, l_lane;
+  int pidx[RL];
+#pragma unroll
+  for (int k = 0; k < RL; ++k) {
+    const int j = lane + 32 * k, gj = j % C::NG, ij = j / C::NG;
+    pidx[k] = gj * C::GS + (ij >> 1) * Gp * 2 + (ij & 1) + 2 * warp;
+  }
+  bool timed_out = false;
+  int st = 0;                  // ring position and phase run on across segments
+  uint32_t parity = 0;
+
+  for (;;) {   // one pass per segment (a single one unless the mode is balanced)
+  int seg_tiles;               // tiles of the current unit
+  {
+    len = min(max(p.seq_len[b] + p.len_add, 0), p.S_cap);
+    len8 = (len + 7) & ~7;     // rows a copy may touch: S_cap is a multiple of 8
+    seg_tiles = (len + ST - 1) / ST;
+    if (p.balanced) {
+      t_begin = cur - unit_start;
+      n_my = min(seg_tiles - t_begin, hi - cur);
+      const int seg = (int)blockIdx.x - sk_cta_of(unit_start, plan);
+      ws_head = (size_t)RAP_MAX_SPLIT * (DV + 2);
+      ws_base = p.ws + (((size_t)b * p.Hq + (size_t)h * G) * RAP_MAX_SPLIT + seg) * (size_t)(DV + 2);
+    } else {
+      const int split = blockIdx.x;
+      const int tps = (seg_tiles + p.n_split - 1) / p.n_split;
+      t_begin = min(seg_tiles, split * tps);
+      n_my = min(seg_tiles, t_begin + tps) - t_begin;
+      ws_head = (size_t)p.n_split * (DV + 2);
+      ws_base = p.ws + (((size_t)b * p.Hq + (size_t)h * G) * p.n_split + split) * (size_t)(DV + 2);
+      if (n_my <= 0) {   // nothing to scan: neutral partials
+        for (int i = tid; i < G * (DV + 2); i += STHREADS) {
+          const int g = i / (DV + 2), c = i - g * (DV + 2);
+          ws_base[g * ws_head + c] = (c == DV) ? -INFINITY : 0.f;
+        }
+        return;
+      }
+    }
+    const size_t unit = (size_t)b * p.Hkv + h;
+    kg = p.k + unit * (size_t)p.S_cap * (size_t)(WK * 4);
+    vg = p.v + unit * (size_t)p.S_cap * (size_t)(DV * 2);
+  }
+  if (warp == 0) {
+    const int pre = min(n_my, C::NS - 1);
+    for (int tl = 0; tl < pre; ++tl) issue_tile(tl, (st + tl) % C::NS);
+  }
 #pragma unroll
   for (int g = 0; g < G; ++g) {
     const uint32_t* qrow = p.q + ((size_t)b * p.Hq + (size_t)h * G + g) * WK;
@@ -258,29 +354,10 @@ __global__ void __launch_bounds__(STHREADS, 2) attn_scan_kernel(const ScanParams
       const uint32_t x = mine ? qrow[w0 + (i / C::KV) * ustep + i % C::KV] : 0u;
       qr[g][i] = pack2(__uint_as_float(x << 16) * p.qscale, __uint_as_float(x & 0xffff0000u) * p.qscale);
     }
+    accLo[g] = accHi[g] = 0ull;
   }
-
-  // ---- PV role ------------------------------------------------------------------------------
-  const int grp = tid / C::WVP, wch = tid - grp * C::WVP;
-  const bool pv_active = grp < C::NG;
-  const bool last_slot_ok = grp < C::LASTN;    // does this group own a row in slot RPG - 1 ?
-  const bool has_hi = 2 * wch + 1 < DV;        // odd DV: the last channel pair has one channel
-  uint64_t accLo[G], accHi[G];     // (even-slot rows, odd-slot rows) partial sums of channels 2*wch and 2*wch+1
-#pragma unroll
-  for (int g = 0; g < G; ++g) accLo[g] = accHi[g] = 0ull;
-  const float* ppg = pp + (pv_active ? grp : 0) * C::GS;
-
-  // softmax role: warp g < G, lanes own positions lane and lane + 32
-  float m_ref = -INFINITY, l_lane = 0.f;
-  int pidx[RL];
-#pragma unroll
-  for (int k = 0; k < RL; ++k) {
-    const int j = lane + 32 * k, gj = j % C::NG, ij = j / C::NG;
-    pidx[k] = gj * C::GS + (ij >> 1) * Gp * 2 + (ij & 1) + 2 * warp;
-  }
-  bool timed_out = false;
-  int st = 0;
-  uint32_t parity = 0;
+  m_ref = -INFINITY;
+  l_lane = 0.f;
 
   for (int tl = 0; tl < n_my; ++tl) {
     const bool ok = mbar_wait_bounded(bar0 + 8 * st, parity);
@@ -438,7 +515,7 @@ __global__ void __launch_bounds__(STHREADS, 2) attn_scan_kernel(const ScanParams
   if (timed_out) {
     if (tid == 0) {
       atomicCAS(&p.status[0], 0, (int)RAP_ETIMEOUT);
-      p.status[1] = (b * p.Hkv + h) * p.n_split + split;
+      p.status[1] = (b * p.Hkv + h) * RAP_MAX_SPLIT + (int)(blockIdx.x % RAP_MAX_SPLIT);
       // give copies still in flight a bounded chance to land before the shared memory is released
       for (int s = 0; s < C::NS; ++s) {
         mbar_wait_bounded(bar0 + 8 * s, 0);
@@ -480,13 +557,40 @@ __global__ void __launch_bounds__(STHREADS, 2) attn_scan_kernel(const ScanParams
       ws_base[warp * ws_head + DV + 1] = l;
     }
   }
+  // ---- next segment: the following unit, from its first tile ---------------------------------------
+  if (!p.balanced) break;
+  cur += n_my;
+  if (cur >= hi) break;
+  unit_start += seg_tiles;
+  if (++h == p.Hkv) {
+    h = 0;
+    do { ++b; } while (b < p.B && sk_tiles_of(p.seq_len, b, p.len_add, p.S_cap, ST) == 0);
+    if (b >= p.B) break;
+  }
+  __syncthreads();   // the row-group reduction buffer is the next segment's partial-logit buffer
+  }   // segment loop
 }
 
 // out[b][g][c] = sum_s 2^(m_s - M) acc_s[c] / sum_s 2^(m_s - M) l_s ; empty splits have l = 0.
+// Balanced mode (seq_len != nullptr): the unit's segment count follows from the same plan the scan used.
 __global__ void __launch_bounds__(128) attn_scan_combine_kernel(const float* __restrict__ ws, int n_split, int dv,
-                                                                float* __restrict__ out) {
+                                                                float* __restrict__ out,
+                                                                const int32_t* __restrict__ seq_len, int B, int Hq,
+                                                                int Hkv, int len_add, int S_cap, int tile_rows,
+                                                                int scan_grid) {
   const size_t bg = blockIdx.x;
-  const float* base = ws + bg * n_split * (size_t)(dv + 2);
+  int stride = n_split;
+  if (seq_len != nullptr) {
+    const int b = (int)(bg / Hq), h = (int)(bg % Hq) / (Hq / Hkv);
+    const SkPlan pl = sk_plan(seq_len, B, Hkv, len_add, S_cap, tile_rows, scan_grid);
+    int pb = 0;
+    for (int bb = 0; bb < b; ++bb) pb += sk_tiles_of(seq_len, bb, len_add, S_cap, tile_rows) * Hkv;
+    const int n = sk_tiles_of(seq_len, b, len_add, S_cap, tile_rows);
+    const int start = pb + h * n;
+    n_split = n > 0 ? sk_cta_of(start + n - 1, pl) - sk_cta_of(start, pl) + 1 : 0;
+    stride = RAP_MAX_SPLIT;
+  }
+  const float* base = ws + bg * stride * (size_t)(dv + 2);
   __shared__ float wgt[RAP_MAX_SPLIT];
   __shared__ float inv_s;
   if (threadIdx.x < 32) {
@@ -541,23 +645,6 @@ const ScanEntry kScanTable[] = {
 
 }  // namespace
 
-// Split count: fill two CTAs per SM a whole number of times with splits of at least 8 tiles.
-int rap_scan_choose_split(const rap_ctx* ctx, int B, int Hkv, int h_len_max, int tile_rows) {
-  const long units_total = (long)B * Hkv;
-  const int n_tiles = (h_len_max + tile_rows - 1) / tile_rows;
-  const long slots = 2L * ctx->sm_count;
-  double best = 1e30;
-  int n_split = 1;
-  for (int ns = 1; ns <= RAP_MAX_SPLIT; ++ns) {
-    const int tiles_per = (n_tiles + ns - 1) / ns;
-    if (ns > 1 && tiles_per < 8) break;
-    const long waves = (units_total * ns + slots - 1) / slots;
-    const double cost = (double)waves * (tiles_per + 3);
-    if (cost < best - 1e-9) { best = cost; n_split = ns; }
-  }
-  return n_split;
-}
-
 rap_status rap_launch_attn_scan(rap_ctx* ctx, const rap_attn_args& a, int n_split_req, cudaStream_t st) {
   if (a.dtype != RAP_BF16 || (a.P2 & 1)) return RAP_EUNSUPPORTED;
   const int G = a.Hq / a.Hkv, WK = a.P2 / 2;
@@ -565,18 +652,29 @@ rap_status rap_launch_attn_scan(rap_ctx* ctx, const rap_attn_args& a, int n_spli
   for (const ScanEntry& c : kScanTable)
     if (c.G == G && c.WK == WK && c.DV == a.dv) { e = &c; break; }
   if (!e) return RAP_EUNSUPPORTED;
-  const int n_split = n_split_req > 0 ? n_split_req : rap_scan_choose_split(ctx, a.B, a.Hkv, a.h_len_max, e->tile);
+  // n_split = 0: balanced mode, one CTA per resident slot; an explicit n_split keeps equal ranges per split
+  const bool balanced = n_split_req <= 0 && (long long)a.B * a.Hkv * ((a.S_cap + 63) / 64) < (1LL << 31);
+  int n_split = balanced ? RAP_MAX_SPLIT : n_split_req;
+  if (n_split <= 0) {   // (only for tile counts beyond 2^31) equal ranges, a few waves of CTAs
+    n_split = (8 * ctx->sm_count + a.B * a.Hkv - 1) / (a.B * a.Hkv);
+    n_split = n_split > RAP_MAX_SPLIT ? RAP_MAX_SPLIT : n_split < 1 ? 1 : n_split;
+  }
   ScanParams p;
   p.q = (const uint32_t*)a.q; p.k = (const unsigned char*)a.k; p.v = (const unsigned char*)a.v;
   p.seq_len = a.seq_len; p.ws = ctx->d_attn_ws; p.status = ctx->d_status;
   p.len_add = a.len_add; p.Hq = a.Hq; p.Hkv = a.Hkv; p.S_cap = a.S_cap; p.n_split = n_split;
   p.qscale = (float)(1.4426950408889634 / sqrt((double)a.head_dim));
+  p.B = a.B; p.balanced = balanced ? 1 : 0;
   RAP_CUDA_TRY(ctx, cudaFuncSetAttribute(e->fn, cudaFuncAttributeMaxDynamicSharedMemorySize, e->smem));
+  const int scan_grid = 2 * ctx->sm_count;
   dim3 grid(n_split, a.Hkv, a.B);
+  if (balanced) grid = dim3(scan_grid, 1, 1);
   e->fn<<<grid, STHREADS, e->smem, st>>>(p);
   ctx->launches++;
   RAP_CUDA_TRY(ctx, cudaGetLastError());
-  attn_scan_combine_kernel<<<a.B * a.Hq, 128, 0, st>>>(ctx->d_attn_ws, n_split, a.dv, a.out);
+  attn_scan_combine_kernel<<<a.B * a.Hq, 128, 0, st>>>(ctx->d_attn_ws, n_split, a.dv, a.out,
+                                                       balanced ? a.seq_len : nullptr, a.B, a.Hq, a.Hkv, a.len_add,
+                                                       a.S_cap, e->tile, scan_grid);
   ctx->launches++;
   RAP_CUDA_TRY(ctx, cudaGetLastError());
   return RAP_OK;
