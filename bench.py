@@ -92,6 +92,22 @@ def build_stack(w, torch, seed_offset=0):
     return st
 
 
+def max_over_ranks(values, device, world):
+    """Element-wise maximum of per-rank timings (every rank gets the result): replicas share nothing
+    on the data path, the only exchange of a multi-GPU run is this one reduction of clock readings."""
+    import torch
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if world > 1:
+        import torch.distributed as dist
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
+def aggregate_throughput(per_rank_batch, world, ms_per_step):
+    """Whole-job tokens/s of `world` independent replicas that each decode per_rank_batch tokens per step."""
+    return world * per_rank_batch / (ms_per_step * 1e-3)
+
+
 def pick_workload(args):
     """The named workload, optionally cut down (--layers/--batch/--seq) for profiler-sized runs."""
     from dataclasses import replace
@@ -187,10 +203,7 @@ def run_ours(args):
     barrier()
     e2e_ms = max(d0.elapsed_time(d1), (time.perf_counter() - e0) * 1e3) / e2e_steps
 
-    ms = torch.tensor([ms_total, e2e_ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(ms, op=dist.ReduceOp.MAX)
-    ms_total, e2e_ms = ms.tolist()
+    ms_total, e2e_ms = max_over_ranks([ms_total, e2e_ms], dev, world)
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -201,7 +214,7 @@ def run_ours(args):
     alg = attn_bytes(w, mean_len)
     achieved = alg / (attn_ms * 1e-3) / 1e9
     line = {
-        "metric": METRIC, "value": world * B / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K,
+        "metric": METRIC, "value": aggregate_throughput(B, world, ms_step), "unit": UNIT, "n_gpus": world, "steps": K,
         "warmup": W, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic",
         "config": {"workload": f"{w.name}: L={L} hidden={w.hidden} Hq/Hkv={w.n_q_heads}/{w.n_kv_heads} D={w.head_dim} "
@@ -210,7 +223,7 @@ def run_ours(args):
                    "l2": "inputs larger than L2 (%.1f GB of KV cache per step)" % (L * alg / 1e9),
                    "parallelism": "replicas" if world > 1 else "single"},
         "clocks": clocks, "gpu_launches": int(launches),
-        "e2e": {"value": world * B / (e2e_ms * 1e-3), "unit": UNIT,
+        "e2e": {"value": aggregate_throughput(B, world, e2e_ms), "unit": UNIT,
                 "h2d_bytes_per_step": int(hx[0].numel() * hx[0].element_size()),
                 "d2h_bytes_per_step": int(h_out.numel() * 4)},
         "roofline": {"bound": "hbm", "kernel": "rap_decode_attn (split-KV scan + combine)", "achieved": achieved,

@@ -179,7 +179,12 @@ def _random_attn_case(w, lens, n_split, seed=0):
     for l in range(w.n_layers):
         out = st.decode_attn(l, q, dl, int(max(lens)), n_split=n_split)
         torch.cuda.synchronize()
-        want = O.decode_attn(util.to_np64(q), util.to_np64(st.k_cache[l]), util.to_np64(st.v_cache[l]), lens, w.head_dim)
+        # the definition needs at least one row; the library returns zeros for an empty sequence
+        want = O.decode_attn(util.to_np64(q), util.to_np64(st.k_cache[l]), util.to_np64(st.v_cache[l]),
+                             [max(1, n) for n in lens], w.head_dim)
+        for b, n in enumerate(lens):
+            if n == 0:
+                want[b] = 0.0
         got = util.to_np64(out[: w.batch * w.n_q_heads * dv]).reshape(w.batch, w.n_q_heads, dv)
         util.check_attn(got, want, w.dtype)
     st.close()
@@ -312,3 +317,11 @@ def test_lowrank_comparator_matches_oracle(dtype, pairing):
             util.check_attn(util.to_np64(out), want, dtype)
     assert ctx.rap_get_last_device_status() == (0, 0)
     ctx.close()
+
+
+@pytest.mark.parametrize("lens", [[0, 5000, 0, 1, 129, 0], [7000], [1, 1, 1, 1, 1, 1, 1, 1], [0, 0, 3]])
+def test_balanced_split_mixed_lengths(lens):
+    """n_split = 0 lets every CTA scan an equal share of the global tile sequence: empty sequences,
+    one long sequence (segment cap), many one-tile units and CTA ranges that cross unit boundaries."""
+    w = synth.scaled_down(synth.LLAMA_8B, n_layers=1, batch=len(lens), seq=max(lens))
+    _random_attn_case(w, lens, 0, seed=len(lens))
