@@ -215,8 +215,17 @@ rap_status rap_get_last_device_status(rap_ctx* ctx, int32_t* code, int32_t* deta
 /* Number of kernels this context has launched since creation (for launch accounting). */
 int64_t rap_kernel_launch_count(const rap_ctx* ctx);
 
+/* Timing of the attention launches inside rap_decode_step / rap_decode_step_host, for roofline
+ * reports: after rap_profile_attn(ctx, capacity) the next `capacity` attention launches (one per layer
+ * and step) are bracketed by CUDA events on the caller's stream; rap_profile_attn_read waits for them,
+ * returns the summed device time in milliseconds and the number of launches covered, and rearms the
+ * same events.  capacity = 0 switches the timing off.  Event creation happens in rap_profile_attn. */
+rap_status rap_profile_attn(rap_ctx* ctx, int32_t capacity);
+rap_status rap_profile_attn_read(rap_ctx* ctx, float* ms_sum, int32_t* n_calls);
+
 /* Forces a kernel variant for rap_decode_attn: 0 = automatic (shape-specialised scan when the
- * head shape has one), 1 = fully generic kernel only, 2 = skip the shape-specialised scan.
+ * head shape has one; the low-rank comparator's fast path), 1 = fully generic kernels only, 2 = skip the
+ * shape-specialised scan.
  * Meant for tests and profiling. */
 rap_status rap_set_attn_variant(rap_ctx* ctx, int32_t variant);
 

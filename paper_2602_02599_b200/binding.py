@@ -24,7 +24,7 @@ EXPORTS = [
     "rap_cache_elem_offset", "rap_build_tables", "rap_pack_weights", "rap_qkv_rope_append",
     "rap_decode_attn", "rap_decode_step", "rap_decode_step_host", "rap_lowrank_decode_attn",
     "rap_get_last_device_status", "rap_kernel_launch_count", "rap_set_attn_variant",
-    "rap_decode_attn_noalloc",
+    "rap_decode_attn_noalloc", "rap_profile_attn", "rap_profile_attn_read",
 ]
 
 
@@ -76,6 +76,8 @@ def _lib():
     lib.rap_kernel_launch_count.argtypes = [P]
     lib.rap_kernel_launch_count.restype = c_int64
     lib.rap_set_attn_variant.argtypes = [P, c_int32]
+    lib.rap_profile_attn.argtypes = [P, c_int32]
+    lib.rap_profile_attn_read.argtypes = [P, POINTER(ctypes.c_float), POINTER(c_int32)]
     lib.rap_decode_attn_noalloc.argtypes = [c_int32] * 7 + [P, P, P, c_int32, P, c_int32, c_int32, P, P]
     for name in EXPORTS:
         fn = getattr(lib, name)
@@ -227,6 +229,14 @@ class RapContext:
 
     def rap_kernel_launch_count(self):
         return int(_lib().rap_kernel_launch_count(self._ctx))
+
+    def rap_profile_attn(self, capacity):
+        self._check(_lib().rap_profile_attn(self._ctx, capacity), "rap_profile_attn")
+
+    def rap_profile_attn_read(self):
+        ms, n = ctypes.c_float(), c_int32()
+        self._check(_lib().rap_profile_attn_read(self._ctx, byref(ms), byref(n)), "rap_profile_attn_read")
+        return ms.value, n.value
 
     def rap_set_attn_variant(self, variant):
         self._check(_lib().rap_set_attn_variant(self._ctx, variant), "rap_set_attn_variant")

@@ -26,6 +26,7 @@ bool desc_ok(const rap_model_desc& d) {
 void free_all(rap_ctx* c) {
   if (c->d_status) cudaFree(c->d_status);
   if (c->d_attn_ws) cudaFree(c->d_attn_ws);
+  if (c->d_unit_cnt) cudaFree(c->d_unit_cnt);
   if (c->d_proj_ws) cudaFree(c->d_proj_ws);
   if (c->d_stage_x) cudaFree(c->d_stage_x);
   if (c->d_stage_out) cudaFree(c->d_stage_out);
@@ -33,6 +34,7 @@ void free_all(rap_ctx* c) {
   if (c->d_lr_k) cudaFree(c->d_lr_k);
   if (c->d_lr_cs) cudaFree(c->d_lr_cs);
   if (c->h_tables) cudaFreeHost(c->h_tables);
+  for (cudaEvent_t e : c->prof_ev) cudaEventDestroy(e);
 }
 
 }  // namespace
@@ -111,6 +113,8 @@ rap_status rap_create(const rap_model_desc* desc, rap_ctx** out) {
   RAP_CUDA_TRY(c, cudaMalloc(&c->d_status, 2 * sizeof(int32_t)));
   RAP_CUDA_TRY(c, cudaMemset(c->d_status, 0, 2 * sizeof(int32_t)));
   RAP_CUDA_TRY(c, cudaMalloc(&c->d_attn_ws, c->attn_ws_bytes));
+  RAP_CUDA_TRY(c, cudaMalloc(&c->d_unit_cnt, (size_t)d.max_batch * d.n_kv_heads * sizeof(int32_t)));
+  RAP_CUDA_TRY(c, cudaMemset(c->d_unit_cnt, 0, (size_t)d.max_batch * d.n_kv_heads * sizeof(int32_t)));
   RAP_CUDA_TRY(c, cudaMalloc(&c->d_proj_ws, c->proj_ws_bytes));
   RAP_CUDA_TRY(c, cudaMalloc(&c->d_stage_x, c->stage_x_bytes));
   RAP_CUDA_TRY(c, cudaMalloc(&c->d_stage_out, c->stage_out_bytes));
@@ -312,8 +316,14 @@ rap_status rap_decode_step(rap_ctx* ctx, int32_t B, const void* d_x, const void*
     a.B = B; a.Hq = d.n_q_heads; a.Hkv = d.n_kv_heads; a.P2 = p.P2; a.dv = p.dv; a.S_cap = S_cap;
     a.head_dim = d.head_dim; a.dtype = d.dtype; a.n_split = n_split; a.h_len_max = h_seq_len_max + 1;
     a.out = d_out + (size_t)l * out_layer_stride;
+    const bool timed = 2 * (ctx->prof_pairs + 1) <= (int)ctx->prof_ev.size();
+    if (timed) RAP_CUDA_TRY(ctx, cudaEventRecord(ctx->prof_ev[2 * ctx->prof_pairs], st));
     s = rap_launch_attn(ctx, a, st);
     if (s != RAP_OK) return s;
+    if (timed) {
+      RAP_CUDA_TRY(ctx, cudaEventRecord(ctx->prof_ev[2 * ctx->prof_pairs + 1], st));
+      ctx->prof_pairs++;
+    }
   }
   if (advance) return rap_launch_advance(ctx, d_seq_len, B, st);
   return RAP_OK;
@@ -367,6 +377,34 @@ rap_status rap_lowrank_decode_attn(rap_ctx* ctx, int32_t B, int32_t r, int32_t d
   return rap_launch_lowrank_attn(ctx, a, (cudaStream_t)stream);
 }
 
+rap_status rap_profile_attn(rap_ctx* ctx, int32_t capacity) {
+  if (!ctx || capacity < 0) return RAP_EINVAL;
+  for (cudaEvent_t e : ctx->prof_ev) cudaEventDestroy(e);
+  ctx->prof_ev.clear();
+  ctx->prof_pairs = 0;
+  for (int i = 0; i < 2 * capacity; ++i) {
+    cudaEvent_t e;
+    RAP_CUDA_TRY(ctx, cudaEventCreate(&e));
+    ctx->prof_ev.push_back(e);
+  }
+  return RAP_OK;
+}
+
+rap_status rap_profile_attn_read(rap_ctx* ctx, float* ms_sum, int32_t* n_calls) {
+  if (!ctx || !ms_sum || !n_calls) return RAP_EINVAL;
+  float sum = 0.f;
+  for (int i = 0; i < ctx->prof_pairs; ++i) {
+    float ms = 0.f;
+    RAP_CUDA_TRY(ctx, cudaEventSynchronize(ctx->prof_ev[2 * i + 1]));
+    RAP_CUDA_TRY(ctx, cudaEventElapsedTime(&ms, ctx->prof_ev[2 * i], ctx->prof_ev[2 * i + 1]));
+    sum += ms;
+  }
+  *ms_sum = sum;
+  *n_calls = ctx->prof_pairs;
+  ctx->prof_pairs = 0;
+  return RAP_OK;
+}
+
 rap_status rap_get_last_device_status(rap_ctx* ctx, int32_t* code, int32_t* detail, void* stream) {
   if (!ctx || !code || !detail) return RAP_EINVAL;
   int32_t h[2] = {0, 0};
@@ -374,6 +412,11 @@ rap_status rap_get_last_device_status(rap_ctx* ctx, int32_t* code, int32_t* deta
   RAP_CUDA_TRY(ctx, cudaMemcpyAsync(h, ctx->d_status, sizeof(h), cudaMemcpyDeviceToHost, st));
   RAP_CUDA_TRY(ctx, cudaMemsetAsync(ctx->d_status, 0, sizeof(h), st));
   RAP_CUDA_TRY(ctx, cudaStreamSynchronize(st));
+  if (h[0] != 0) {   // a kernel that gave up may have left unit arrival counters behind
+    const rap_model_desc& d = ctx->desc;
+    RAP_CUDA_TRY(ctx, cudaMemsetAsync(ctx->d_unit_cnt, 0, (size_t)d.max_batch * d.n_kv_heads * sizeof(int32_t), st));
+    RAP_CUDA_TRY(ctx, cudaStreamSynchronize(st));
+  }
   *code = h[0];
   *detail = h[1];
   return RAP_OK;

@@ -97,6 +97,8 @@ struct ScanParams {
   int32_t* status;
   int len_add, Hq, Hkv, S_cap, n_split;
   float qscale;
+  int32_t* unit_cnt;   // balanced mode: arrivals per (sequence, KV head) unit, zero between calls
+  float* out;          // balanced mode: [B][Hq][DV], written by the CTA that completes a unit
   int B;           // sequences (used by the balanced mode)
   int balanced;    // 0: grid (n_split, H_kv, B), equal tile ranges per split; 1: grid (CTAs), see SkPlan
 };
@@ -235,6 +237,11 @@ __global__ void __launch_bounds__(STHREADS, 2) attn_scan_kernel(const ScanParams
   int cur = 0, hi = 0, unit_start = 0;
   if (p.balanced) {
     plan = sk_plan(p.seq_len, p.B, p.Hkv, p.len_add, p.S_cap, ST, (int)gridDim.x);
+    if (blockIdx.x == 0) {   // sequences without any row are scanned by nobody: their output is zero
+      for (int bb = 0; bb < p.B; ++bb)
+        if (sk_tiles_of(p.seq_len, bb, p.len_add, p.S_cap, ST) == 0)
+          for (int i = tid; i < p.Hq * DV; i += STHREADS) p.out[(size_t)bb * p.Hq * DV + i] = 0.f;
+    }
     if ((int)blockIdx.x >= plan.nc) return;
     cur = (int)((long long)blockIdx.x * plan.T / plan.nc);
     hi = (int)((long long)(blockIdx.x + 1) * plan.T / plan.nc);
@@ -557,6 +564,54 @@ __global__ void __launch_bounds__(STHREADS, 2) attn_scan_kernel(const ScanParams
       ws_base[warp * ws_head + DV + 1] = l;
     }
   }
+  if (p.balanced) {
+    // ---- the CTA that delivers a unit's last partial merges them (no separate combine launch) ------
+    __shared__ int s_last;
+    __threadfence();           // this CTA's partials are visible before its arrival is counted
+    __syncthreads();
+    const int first = sk_cta_of(unit_start, plan);
+    const int nseg = sk_cta_of(unit_start + seg_tiles - 1, plan) - first + 1;
+    const int u = b * p.Hkv + h;
+    if (tid == 0) s_last = atomicAdd(&p.unit_cnt[u], 1) == nseg - 1;
+    __syncthreads();
+    if (s_last) {
+      __threadfence();
+      float* wgt = s_part;     // [G][64] segment weights, then G reciprocals of the denominators
+      const float* ub = p.ws + ((size_t)b * p.Hq + (size_t)h * G) * RAP_MAX_SPLIT * (size_t)(DV + 2);
+      if (warp < G) {
+        const float* gb = ub + (size_t)warp * ws_head;
+        float mv[2], lv[2];
+#pragma unroll
+        for (int k = 0; k < 2; ++k) {
+          const int sg = lane + 32 * k;
+          lv[k] = sg < nseg ? __ldcg(gb + (size_t)sg * (DV + 2) + DV + 1) : 0.f;
+          mv[k] = (sg < nseg && lv[k] > 0.f) ? __ldcg(gb + (size_t)sg * (DV + 2) + DV) : -INFINITY;
+        }
+        float M = fmaxf(mv[0], mv[1]);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+        float den = 0.f;
+#pragma unroll
+        for (int k = 0; k < 2; ++k) {
+          const float wk = lv[k] > 0.f ? exp2f(mv[k] - M) : 0.f;
+          wgt[warp * RAP_MAX_SPLIT + lane + 32 * k] = wk;
+          den += wk * lv[k];
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) den += __shfl_xor_sync(0xffffffffu, den, o);
+        if (lane == 0) wgt[G * RAP_MAX_SPLIT + warp] = den > 0.f ? 1.f / den : 0.f;
+      }
+      __syncthreads();
+      for (int i = tid; i < G * DV; i += STHREADS) {
+        const int g = i / DV, c = i - g * DV;
+        const float* gb = ub + (size_t)g * ws_head + c;
+        float num = 0.f;
+        for (int sg = 0; sg < nseg; ++sg) num += wgt[g * RAP_MAX_SPLIT + sg] * __ldcg(gb + (size_t)sg * (DV + 2));
+        p.out[((size_t)b * p.Hq + (size_t)h * G + g) * DV + c] = num * wgt[G * RAP_MAX_SPLIT + g];
+      }
+      if (tid == 0) p.unit_cnt[u] = 0;   // ready for the next call on this context
+    }
+  }
   // ---- next segment: the following unit, from its first tile ---------------------------------------
   if (!p.balanced) break;
   cur += n_my;
@@ -665,6 +720,7 @@ rap_status rap_launch_attn_scan(rap_ctx* ctx, const rap_attn_args& a, int n_spli
   p.len_add = a.len_add; p.Hq = a.Hq; p.Hkv = a.Hkv; p.S_cap = a.S_cap; p.n_split = n_split;
   p.qscale = (float)(1.4426950408889634 / sqrt((double)a.head_dim));
   p.B = a.B; p.balanced = balanced ? 1 : 0;
+  p.unit_cnt = ctx->d_unit_cnt; p.out = a.out;
   RAP_CUDA_TRY(ctx, cudaFuncSetAttribute(e->fn, cudaFuncAttributeMaxDynamicSharedMemorySize, e->smem));
   const int scan_grid = 2 * ctx->sm_count;
   dim3 grid(n_split, a.Hkv, a.B);
@@ -672,9 +728,11 @@ rap_status rap_launch_attn_scan(rap_ctx* ctx, const rap_attn_args& a, int n_spli
   e->fn<<<grid, STHREADS, e->smem, st>>>(p);
   ctx->launches++;
   RAP_CUDA_TRY(ctx, cudaGetLastError());
-  attn_scan_combine_kernel<<<a.B * a.Hq, 128, 0, st>>>(ctx->d_attn_ws, n_split, a.dv, a.out,
-                                                       balanced ? a.seq_len : nullptr, a.B, a.Hq, a.Hkv, a.len_add,
-                                                       a.S_cap, e->tile, scan_grid);
+  if (balanced) {
+    return RAP_OK;   // merged inside the scan kernel
+  }
+  attn_scan_combine_kernel<<<a.B * a.Hq, 128, 0, st>>>(ctx->d_attn_ws, n_split, a.dv, a.out, nullptr, a.B, a.Hq, a.Hkv,
+                                                       a.len_add, a.S_cap, e->tile, scan_grid);
   ctx->launches++;
   RAP_CUDA_TRY(ctx, cudaGetLastError());
   return RAP_OK;

@@ -25,6 +25,7 @@ struct rap_ctx {
   int32_t* d_status = nullptr;    // [2] = {code, detail}
   float* d_attn_ws = nullptr;     // split-KV partials
   size_t attn_ws_bytes = 0;
+  int32_t* d_unit_cnt = nullptr;  // [max_batch][H_kv] partial-arrival counters of the balanced scan (zero between calls)
   float* d_proj_ws = nullptr;     // fp32 projection results / split-K partials
   size_t proj_ws_bytes = 0;
   void* d_stage_x = nullptr;      // staging for rap_decode_step_host
@@ -41,6 +42,9 @@ struct rap_ctx {
   size_t h_tables_bytes = 0;
   void* tables_stream = nullptr;
   bool tables_inflight = false;
+  // optional timing of the attention launches of rap_decode_step (event pairs on the caller's stream)
+  std::vector<cudaEvent_t> prof_ev;   // 2 * capacity events
+  int prof_pairs = 0;                 // pairs recorded since the last read
   int32_t attn_variant = 0;
   int64_t launches = 0;
   std::string cuda_error;
