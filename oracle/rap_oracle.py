@@ -15,6 +15,10 @@ Two definitions of the same result live here:
       The paper proves (R) == (F) (Appendix "Full-dimensional representation",
       masked-logit equivalence); (F) exists only to pin (R).
 
+Output projection (gather_wo / out_proj): pinned by the identity W~_o o_reduced = W_o E_v^T o_reduced
+(expanding the reduced output back to D channels with zeros and using the dense W_o) and by a
+loop-written column gather.
+
 Pins (in tests/test_oracle_pins.py): rho=1 equals an independent textbook RoPE GQA
 attention; (R)==(F) for rho<1 in both pairings; the per-pair relative-rotation
 identity R_m^T R_n = R_(n-m); position-shift invariance; E_k E_k^T = I and
@@ -397,6 +401,28 @@ def lowrank_decode_attn(q_full, k_latent, B_k, v_cache, seq_len, head_dim, rope_
                 p /= p.sum()
                 out[b, g] = p @ V
     return out
+
+
+# --------------------------------------------------------------------------------------
+# output projection on the retained V channels (Algorithm 1: W~_o = E_v W_o absorbs the V selection)
+# --------------------------------------------------------------------------------------
+def gather_wo(Wo, tables, layer, n_vch_l, head_dim, Hq, Hkv):
+    """W~_o [hidden][H_q * d_v'] from the dense W_o [hidden][H_q * D] (weights stored [out][in]).
+
+    Input column g * D + u of W_o multiplies channel u of query head g's attention output; only
+    the retained channels u in S_v of KV head g // G ever carry a value, so W~_o keeps exactly
+    those columns, in the order of the reduced output (head-major, channels ascending)."""
+    D, G, dv = head_dim, Hq // Hkv, n_vch_l
+    cols = []
+    for g in range(Hq):
+        cols.append(g * D + np.asarray(tables["v_idx"][layer, g // G, :dv]))
+    return np.asarray(Wo)[:, np.concatenate(cols)]
+
+
+def out_proj(attn_out, wo_tilde):
+    """y[t] = W~_o o[t]: attn_out [T][H_q][d_v'] (reduced V coordinates) -> [T][hidden], fp64."""
+    o = np.asarray(attn_out, dtype=np.float64)
+    return o.reshape(o.shape[0], -1) @ np.asarray(wo_tilde, dtype=np.float64).T
 
 
 # --------------------------------------------------------------------------------------

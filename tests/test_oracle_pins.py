@@ -338,3 +338,31 @@ def test_lowrank_comparator_reduces_to_textbook():
     qrot = np.stack([O.textbook_rope(qfull[g], n - 1, D, m["theta"], m["pairing"]) for g in range(Hq)])[None]
     got = O.lowrank_decode_attn(qrot, latent, Bk, V, [n], D, m["theta"], m["pairing"])[0]
     assert np.allclose(got, _full(m), rtol=0, atol=1e-12)
+
+
+# ---- output projection on the retained V channels --------------------------------------------
+def test_out_proj_equals_dense_wo_on_zero_expanded_output():
+    """W~_o o_reduced == W_o (E_v^T o_reduced): expanding the reduced attention output back to D
+    channels (zeros where V was pruned) and applying the dense W_o gives the same hidden vector."""
+    m = _small(rho=0.5, D=16, Hq=4, Hkv=2, n=5, seed=31)
+    D, Hq, Hkv, dv, hidden = m["D"], m["Hq"], m["Hkv"], m["dv"], m["X"].shape[1]
+    rng = np.random.default_rng(8)
+    Wo = rng.normal(0, 0.05, (hidden, Hq * D))
+    o = rng.normal(0, 1.0, (3, Hq, dv))
+    wt = O.gather_wo(Wo, m["tabs"], 0, dv, D, Hq, Hkv)
+    assert wt.shape == (hidden, Hq * dv)
+    got = O.out_proj(o, wt)
+    G = Hq // Hkv
+    full = np.zeros((3, Hq, D))
+    for g in range(Hq):
+        for c in range(dv):
+            full[:, g, m["tabs"]["v_idx"][0, g // G, c]] = o[:, g, c]
+    want = full.reshape(3, Hq * D) @ Wo.T
+    assert np.allclose(got, want, rtol=0, atol=1e-13)
+    # the gather itself, column by column
+    for g in range(Hq):
+        for c in range(dv):
+            assert np.array_equal(wt[:, g * dv + c], Wo[:, g * D + m["tabs"]["v_idx"][0, g // G, c]])
+    # negative control: using another head's V selection breaks the identity
+    bad = O.gather_wo(Wo, m["tabs"], 0, dv, D, Hq, Hkv)[:, ::-1]
+    assert np.abs(O.out_proj(o, bad) - want).max() > 1e-3
