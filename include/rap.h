@@ -172,6 +172,19 @@ rap_status rap_decode_attn_noalloc(int32_t dtype, int32_t B, int32_t n_q_heads, 
                                    const int32_t* d_seq_len, int32_t h_seq_len_max, int32_t n_split,
                                    float* d_out, void* stream);
 
+/* ---- output projection on the retained V channels (Algorithm 1: W~_o = E_v W_o) ------------
+ * rap_pack_wo: offline column gather.  d_wo [hidden][H_q*D] is the dense W_o of `layer` (stored
+ * [out][in]); d_wo_tilde [hidden][H_q*d_v'] receives, for query head g and retained channel c, the
+ * column g*D + v_idx[g/G][c] -- the only columns a reduced attention output can reach.
+ * rap_out_proj: y[t] = W~_o o[t] for T <= max_batch rows; d_attn_out [T][H_q][d_v'] is the fp32 output
+ * of rap_decode_attn, d_y [T][hidden] is written in the storage dtype (fp32 accumulate, one rounding;
+ * for bf16 the attention output is first rounded to bf16, as a bf16 model would hand it to W_o).
+ * RAP_EUNSUPPORTED unless H_q*d_v' is a multiple of 8 (bf16) / 4 (fp32). */
+rap_status rap_pack_wo(rap_ctx* ctx, int32_t layer, const void* d_wo, const int32_t* d_v_idx, void* d_wo_tilde,
+                       void* stream);
+rap_status rap_out_proj(rap_ctx* ctx, int32_t layer, int32_t T, const float* d_attn_out, const void* d_wo_tilde,
+                        void* d_y, void* stream);
+
 /* ---- one decode step over all layers (a2-a5 per layer) -------------------------------------
  * Layer l consumes d_x + l*B*hidden (one hidden-state row per sequence) and produces
  * d_out + l*out_layer_stride ([B][H_q][d_v'_l] fp32).  d_seq_len[b] = rows cached BEFORE the

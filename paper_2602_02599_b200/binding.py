@@ -25,6 +25,7 @@ EXPORTS = [
     "rap_decode_attn", "rap_decode_step", "rap_decode_step_host", "rap_lowrank_decode_attn",
     "rap_get_last_device_status", "rap_kernel_launch_count", "rap_set_attn_variant",
     "rap_decode_attn_noalloc", "rap_profile_attn", "rap_profile_attn_read",
+    "rap_pack_wo", "rap_out_proj",
 ]
 
 
@@ -76,6 +77,8 @@ def _lib():
     lib.rap_kernel_launch_count.argtypes = [P]
     lib.rap_kernel_launch_count.restype = c_int64
     lib.rap_set_attn_variant.argtypes = [P, c_int32]
+    lib.rap_pack_wo.argtypes = [P, c_int32, P, P, P, P]
+    lib.rap_out_proj.argtypes = [P, c_int32, c_int32, P, P, P, P]
     lib.rap_profile_attn.argtypes = [P, c_int32]
     lib.rap_profile_attn_read.argtypes = [P, POINTER(ctypes.c_float), POINTER(c_int32)]
     lib.rap_decode_attn_noalloc.argtypes = [c_int32] * 7 + [P, P, P, c_int32, P, c_int32, c_int32, P, P]
@@ -229,6 +232,14 @@ class RapContext:
 
     def rap_kernel_launch_count(self):
         return int(_lib().rap_kernel_launch_count(self._ctx))
+
+    def rap_pack_wo(self, layer, d_wo, d_v_idx, d_wo_tilde):
+        self._check(_lib().rap_pack_wo(self._ctx, layer, _ptr(d_wo), _ptr(d_v_idx), _ptr(d_wo_tilde), _stream()),
+                    "rap_pack_wo")
+
+    def rap_out_proj(self, layer, T, d_attn_out, d_wo_tilde, d_y):
+        self._check(_lib().rap_out_proj(self._ctx, layer, T, _ptr(d_attn_out), _ptr(d_wo_tilde), _ptr(d_y), _stream()),
+                    "rap_out_proj")
 
     def rap_profile_attn(self, capacity):
         self._check(_lib().rap_profile_attn(self._ctx, capacity), "rap_profile_attn")

@@ -31,6 +31,7 @@ void free_all(rap_ctx* c) {
   if (c->d_stage_x) cudaFree(c->d_stage_x);
   if (c->d_stage_out) cudaFree(c->d_stage_out);
   if (c->d_stage_q) cudaFree(c->d_stage_q);
+  if (c->d_oproj_x) cudaFree(c->d_oproj_x);
   if (c->d_lr_k) cudaFree(c->d_lr_k);
   if (c->d_lr_cs) cudaFree(c->d_lr_cs);
   if (c->h_tables) cudaFreeHost(c->h_tables);
@@ -99,7 +100,8 @@ rap_status rap_create(const rap_model_desc* desc, rap_ctx** out) {
   c->sm_count = prop.multiProcessorCount;
   const rap_model_desc& d = c->desc;
   const size_t e = rap_elem_bytes(d.dtype);
-  const size_t n_out_max = (size_t)(d.n_q_heads + 2 * d.n_kv_heads) * d.head_dim;
+  size_t n_out_max = (size_t)(d.n_q_heads + 2 * d.n_kv_heads) * d.head_dim;
+  if ((size_t)d.hidden > n_out_max) n_out_max = d.hidden;       // the workspace also serves rap_out_proj
   c->attn_ws_bytes = (size_t)d.max_batch * d.n_q_heads * RAP_MAX_SPLIT * (size_t)(d.head_dim + 2) * sizeof(float);
   // full-size fp32 results for any row count, plus room for reduction splits on decode-sized calls
   {
@@ -119,6 +121,7 @@ rap_status rap_create(const rap_model_desc* desc, rap_ctx** out) {
   RAP_CUDA_TRY(c, cudaMalloc(&c->d_stage_x, c->stage_x_bytes));
   RAP_CUDA_TRY(c, cudaMalloc(&c->d_stage_out, c->stage_out_bytes));
   RAP_CUDA_TRY(c, cudaMalloc(&c->d_stage_q, (size_t)d.max_batch * d.n_q_heads * d.head_dim * e));
+  RAP_CUDA_TRY(c, cudaMalloc(&c->d_oproj_x, (size_t)d.max_batch * d.n_q_heads * d.head_dim * sizeof(__nv_bfloat16)));
   const size_t units = (size_t)d.n_layers * d.n_kv_heads;
   c->h_tables_bytes = units * ((size_t)(d.head_dim / 2 + 2 * d.head_dim) * sizeof(int32_t) +
                                (size_t)(d.head_dim / 2) * sizeof(double));
@@ -219,6 +222,26 @@ rap_status rap_pack_weights(rap_ctx* ctx, int32_t layer, const void* d_wq, const
     return RAP_EALIGN;
   return rap_launch_pack(ctx, layer, d_wq, d_wk, d_wv, d_k_dim_idx, d_v_idx, d_w_qkv, d_bq, d_bk, d_bv,
                          d_bias, (cudaStream_t)stream);
+}
+
+rap_status rap_pack_wo(rap_ctx* ctx, int32_t layer, const void* d_wo, const int32_t* d_v_idx, void* d_wo_tilde,
+                       void* stream) {
+  if (!ctx || !d_wo || !d_v_idx || !d_wo_tilde) return RAP_EINVAL;
+  if (!ctx->tables_built) return RAP_ESTATE;
+  if (layer < 0 || layer >= ctx->desc.n_layers) return RAP_EINVAL;
+  if (!rap_aligned16(d_wo) || !rap_aligned16(d_wo_tilde) || !rap_aligned16(d_v_idx)) return RAP_EALIGN;
+  return rap_launch_pack_wo(ctx, layer, d_wo, d_v_idx, d_wo_tilde, (cudaStream_t)stream);
+}
+
+rap_status rap_out_proj(rap_ctx* ctx, int32_t layer, int32_t T, const float* d_attn_out, const void* d_wo_tilde,
+                        void* d_y, void* stream) {
+  if (!ctx || !d_attn_out || !d_wo_tilde || !d_y) return RAP_EINVAL;
+  if (!ctx->tables_built) return RAP_ESTATE;
+  if (layer < 0 || layer >= ctx->desc.n_layers || T < 0) return RAP_EINVAL;
+  if (T > ctx->desc.max_batch) return RAP_ESHAPE;
+  if (!rap_aligned16(d_attn_out) || !rap_aligned16(d_wo_tilde) || !rap_aligned16(d_y)) return RAP_EALIGN;
+  if (T == 0) return RAP_OK;
+  return rap_launch_out_proj(ctx, layer, T, d_attn_out, d_wo_tilde, d_y, (cudaStream_t)stream);
 }
 
 rap_status rap_qkv_rope_append(rap_ctx* ctx, int32_t layer, int32_t T, const void* d_x, const void* d_w_qkv,

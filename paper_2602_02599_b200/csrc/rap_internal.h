@@ -31,6 +31,7 @@ struct rap_ctx {
   void* d_stage_x = nullptr;      // staging for rap_decode_step_host
   float* d_stage_out = nullptr;
   void* d_stage_q = nullptr;
+  void* d_oproj_x = nullptr;      // rap_out_proj: attention output rounded to the storage dtype
   void* d_lr_k = nullptr;         // low-rank comparator: rebuilt, rotated full-width K (grown on demand)
   size_t lr_k_bytes = 0;
   void* d_lr_cs = nullptr;        // low-rank comparator: (cos, sin) table [positions][D/2]
@@ -94,3 +95,6 @@ rap_status rap_launch_pack(rap_ctx* ctx, int32_t layer, const void* wq, const vo
                            const int32_t* k_dim_idx, const int32_t* v_idx, void* w_qkv,
                            const void* bq, const void* bk, const void* bv, void* bias, cudaStream_t st);
 rap_status rap_launch_advance(rap_ctx* ctx, int32_t* seq_len, int32_t B, cudaStream_t st);
+rap_status rap_launch_pack_wo(rap_ctx* ctx, int32_t layer, const void* wo, const int32_t* v_idx, void* dst, cudaStream_t st);
+rap_status rap_launch_out_proj(rap_ctx* ctx, int32_t layer, int32_t T, const float* attn_out, const void* wo_tilde,
+                               void* y, cudaStream_t st);

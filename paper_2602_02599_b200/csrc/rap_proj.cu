@@ -12,6 +12,8 @@
 #include "rap_internal.h"
 
 rap_status rap_launch_proj_tc(rap_ctx* ctx, const rap_proj_args& a, int* ksplit_out, cudaStream_t st);
+rap_status rap_launch_gemm_tc(rap_ctx* ctx, const void* x, const void* w, int T, int K, int N, int* ksplit_out,
+                              cudaStream_t st);
 
 namespace {
 
@@ -184,6 +186,35 @@ __global__ void pack_bias_kernel(const T* __restrict__ bq, const T* __restrict__
   }
 }
 
+// Offline column gather of the output projection (Algorithm 1: W~_o = E_v W_o): dst[n][g*dv + c] =
+// src[n][g*D + v_idx[g/G][c]], one block per output row n.
+template <typename T>
+__global__ void pack_wo_kernel(const T* __restrict__ wo, const int32_t* __restrict__ v_idx, T* __restrict__ dst, int Hq,
+                               int Hkv, int D, int dv) {
+  const int n = blockIdx.x, G = Hq / Hkv;
+  const T* src = wo + (size_t)n * Hq * D;
+  T* d = dst + (size_t)n * Hq * dv;
+  for (int i = threadIdx.x; i < Hq * dv; i += blockDim.x) {
+    const int g = i / dv, c = i - g * dv;
+    d[i] = src[g * D + v_idx[(g / G) * D + c]];
+  }
+}
+
+__global__ void cast_bf16_kernel(const float* __restrict__ src, __nv_bfloat16* __restrict__ dst, size_t n) {
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) dst[i] = __float2bfloat16_rn(src[i]);
+}
+
+// y[i] = storage( sum over the reduction splits of ws[ks][i] )
+template <typename T>
+__global__ void sum_splits_kernel(const float* __restrict__ ws, int ksplit, size_t n, T* __restrict__ y) {
+  const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  float a = 0.f;
+  for (int s = 0; s < ksplit; ++s) a += ws[(size_t)s * n + i];
+  y[i] = to_storage<T>(a);
+}
+
 __global__ void advance_kernel(int32_t* seq_len, int B) {
   const int b = blockIdx.x * blockDim.x + threadIdx.x;
   if (b < B) seq_len[b] += 1;
@@ -258,6 +289,59 @@ rap_status rap_launch_pack(rap_ctx* ctx, int32_t layer, const void* wq, const vo
 
 rap_status rap_launch_advance(rap_ctx* ctx, int32_t* seq_len, int32_t B, cudaStream_t st) {
   advance_kernel<<<(B + 127) / 128, 128, 0, st>>>(seq_len, B);
+  ctx->launches++;
+  RAP_CUDA_TRY(ctx, cudaGetLastError());
+  return RAP_OK;
+}
+
+rap_status rap_launch_pack_wo(rap_ctx* ctx, int32_t layer, const void* wo, const int32_t* v_idx, void* dst, cudaStream_t st) {
+  const rap_model_desc& d = ctx->desc;
+  const int dv = ctx->n_vch[layer], D = d.head_dim;
+  const int32_t* vi = v_idx + (size_t)layer * d.n_kv_heads * D;
+  if (d.dtype == RAP_F32)
+    pack_wo_kernel<float><<<d.hidden, 256, 0, st>>>((const float*)wo, vi, (float*)dst, d.n_q_heads, d.n_kv_heads, D, dv);
+  else
+    pack_wo_kernel<__nv_bfloat16><<<d.hidden, 256, 0, st>>>((const __nv_bfloat16*)wo, vi, (__nv_bfloat16*)dst,
+                                                            d.n_q_heads, d.n_kv_heads, D, dv);
+  ctx->launches++;
+  RAP_CUDA_TRY(ctx, cudaGetLastError());
+  return RAP_OK;
+}
+
+// y[T][hidden] = attn_out[T][Hq*dv] (fp32) * W~_o[hidden][Hq*dv]^T, result in the storage dtype
+rap_status rap_launch_out_proj(rap_ctx* ctx, int32_t layer, int32_t T, const float* attn_out, const void* wo_tilde,
+                               void* y, cudaStream_t st) {
+  const rap_model_desc& d = ctx->desc;
+  const int K = d.n_q_heads * ctx->n_vch[layer], N = d.hidden;
+  const size_t n = (size_t)T * N;
+  if ((size_t)T * N * sizeof(float) > ctx->proj_ws_bytes) return RAP_ESHAPE;
+  int ksplit = 1;
+  if (d.dtype == RAP_BF16) {
+    const size_t nx = (size_t)T * K;
+    cast_bf16_kernel<<<(unsigned)((nx + 255) / 256), 256, 0, st>>>(attn_out, (__nv_bfloat16*)ctx->d_oproj_x, nx);
+    ctx->launches++;
+    RAP_CUDA_TRY(ctx, cudaGetLastError());
+    rap_status s = rap_launch_gemm_tc(ctx, ctx->d_oproj_x, wo_tilde, T, K, N, &ksplit, st);
+    if (s == RAP_EUNSUPPORTED) {
+      if ((K * 2) % 16) return RAP_EUNSUPPORTED;
+      ksplit = 1;
+      dim3 grid((N + PROJ_WARPS - 1) / PROJ_WARPS, (T + PROJ_TT - 1) / PROJ_TT);
+      proj_generic_kernel<__nv_bfloat16><<<grid, PROJ_WARPS * 32, 0, st>>>(
+          (const __nv_bfloat16*)ctx->d_oproj_x, (const __nv_bfloat16*)wo_tilde, ctx->d_proj_ws, T, K, N);
+      ctx->launches++;
+      RAP_CUDA_TRY(ctx, cudaGetLastError());
+    } else if (s != RAP_OK) {
+      return s;
+    }
+    sum_splits_kernel<__nv_bfloat16><<<(unsigned)((n + 255) / 256), 256, 0, st>>>(ctx->d_proj_ws, ksplit, n, (__nv_bfloat16*)y);
+  } else {
+    if ((K * 4) % 16) return RAP_EUNSUPPORTED;
+    dim3 grid((N + PROJ_WARPS - 1) / PROJ_WARPS, (T + PROJ_TT - 1) / PROJ_TT);
+    proj_generic_kernel<float><<<grid, PROJ_WARPS * 32, 0, st>>>(attn_out, (const float*)wo_tilde, ctx->d_proj_ws, T, K, N);
+    ctx->launches++;
+    RAP_CUDA_TRY(ctx, cudaGetLastError());
+    sum_splits_kernel<float><<<(unsigned)((n + 255) / 256), 256, 0, st>>>(ctx->d_proj_ws, 1, n, (float*)y);
+  }
   ctx->launches++;
   RAP_CUDA_TRY(ctx, cudaGetLastError());
   return RAP_OK;

@@ -263,26 +263,27 @@ rap_status launch_tc(rap_ctx* ctx, const CUtensorMap& mw, const CUtensorMap& mx,
 
 }  // namespace
 
-rap_status rap_launch_proj_tc(rap_ctx* ctx, const rap_proj_args& a, int* ksplit_out, cudaStream_t st) {
-  if (a.dtype != RAP_BF16 || a.T < 1) return RAP_EUNSUPPORTED;
-  const int n_out = (a.Hq + a.Hkv) * a.P2 + a.Hkv * a.dv;
-  const int tn = a.T <= 32 ? 32 : a.T <= 64 ? 64 : 128;
+// Y[ks][T][N] (fp32, context workspace) = X[T][K] * W[N][K]^T, bf16 operands, K split over grid.z.
+rap_status rap_launch_gemm_tc(rap_ctx* ctx, const void* x, const void* w, int T, int K, int N, int* ksplit_out,
+                              cudaStream_t st) {
+  if (T < 1 || (K % 8) != 0) return RAP_EUNSUPPORTED;     // tensor-map rows must be multiples of 16 bytes
+  const int tn = T <= 32 ? 32 : T <= 64 ? 64 : 128;
   CUtensorMap mw, mx;
-  if (!make_map(&mw, a.w, (uint64_t)n_out, (uint64_t)a.hidden, TC_BM)) return RAP_EUNSUPPORTED;
-  if (!make_map(&mx, a.x, (uint64_t)a.T, (uint64_t)a.hidden, (uint32_t)tn)) return RAP_EUNSUPPORTED;
-  const int row_tiles = (n_out + TC_BM - 1) / TC_BM, tok_tiles = (a.T + tn - 1) / tn;
-  const int nkb = (a.hidden + TC_BK - 1) / TC_BK;
+  if (!make_map(&mw, w, (uint64_t)N, (uint64_t)K, TC_BM)) return RAP_EUNSUPPORTED;
+  if (!make_map(&mx, x, (uint64_t)T, (uint64_t)K, (uint32_t)tn)) return RAP_EUNSUPPORTED;
+  const int row_tiles = (N + TC_BM - 1) / TC_BM, tok_tiles = (T + tn - 1) / tn;
+  const int nkb = (K + TC_BK - 1) / TC_BK;
   // reduction split: enough CTAs for every SM on decode-sized calls, within the workspace
   int ksplit = ctx->sm_count / (row_tiles * tok_tiles);
   if (ksplit > RAP_MAX_KSPLIT) ksplit = RAP_MAX_KSPLIT;
   if (ksplit > nkb / 4) ksplit = nkb / 4;
-  while (ksplit > 1 && (size_t)ksplit * a.T * n_out * sizeof(float) > ctx->proj_ws_bytes) --ksplit;
+  while (ksplit > 1 && (size_t)ksplit * T * N * sizeof(float) > ctx->proj_ws_bytes) --ksplit;
   if (ksplit < 1) ksplit = 1;
   int per = (nkb + ksplit - 1) / ksplit;
   ksplit = (nkb + per - 1) / per;          // no empty split
-  if ((size_t)ksplit * a.T * n_out * sizeof(float) > ctx->proj_ws_bytes) return RAP_EUNSUPPORTED;
+  if ((size_t)ksplit * T * N * sizeof(float) > ctx->proj_ws_bytes) return RAP_EUNSUPPORTED;
   TcParams p;
-  p.y = ctx->d_proj_ws; p.status = ctx->d_status; p.T = a.T; p.n_out = n_out; p.nkb_total = nkb; p.nkb_per_split = per;
+  p.y = ctx->d_proj_ws; p.status = ctx->d_status; p.T = T; p.n_out = N; p.nkb_total = nkb; p.nkb_per_split = per;
   dim3 grid(row_tiles, tok_tiles, ksplit);
   *ksplit_out = ksplit;
   switch (tn) {
@@ -290,4 +291,10 @@ rap_status rap_launch_proj_tc(rap_ctx* ctx, const rap_proj_args& a, int* ksplit_
     case 64: return launch_tc<64>(ctx, mw, mx, p, grid, st);
     default: return launch_tc<128>(ctx, mw, mx, p, grid, st);
   }
+}
+
+rap_status rap_launch_proj_tc(rap_ctx* ctx, const rap_proj_args& a, int* ksplit_out, cudaStream_t st) {
+  if (a.dtype != RAP_BF16) return RAP_EUNSUPPORTED;
+  const int n_out = (a.Hq + a.Hkv) * a.P2 + a.Hkv * a.dv;
+  return rap_launch_gemm_tc(ctx, a.x, a.w, a.T, a.hidden, n_out, ksplit_out, st);
 }

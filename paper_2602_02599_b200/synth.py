@@ -7,7 +7,7 @@ It imports NumPy only.
 
 Streams: np.random.default_rng([seed, tag, layer(, extra)]) so every layer can be
 regenerated on its own.  Tags: 1 pair scores, 2 V-channel scores, 3 weights,
-4 hidden states, 5 cache fill, 6 low-rank comparator factors, 7 bias.
+4 hidden states, 5 cache fill, 6 low-rank comparator factors, 7 bias, 8 output projection.
 """
 from __future__ import annotations
 
@@ -15,7 +15,7 @@ from dataclasses import dataclass, replace
 
 import numpy as np
 
-TAG_KSCORE, TAG_VSCORE, TAG_W, TAG_X, TAG_CACHE, TAG_LOWRANK, TAG_BIAS = 1, 2, 3, 4, 5, 6, 7
+TAG_KSCORE, TAG_VSCORE, TAG_W, TAG_X, TAG_CACHE, TAG_LOWRANK, TAG_BIAS, TAG_WO = 1, 2, 3, 4, 5, 6, 7, 8
 
 
 @dataclass(frozen=True)
@@ -105,6 +105,12 @@ def draw_packed_weights(w, layer):
     """Shrunken W~_qkv [N_out][hidden] drawn directly (a row selection of iid rows is iid)."""
     rng = np.random.default_rng([w.seed, TAG_W, layer, 1])
     return rng.standard_normal((w.n_out, w.hidden), dtype=np.float32) * np.float32(0.02)
+
+
+def draw_wo(w, layer):
+    """Dense output projection W_o [hidden][H_q*D], N(0, 0.02^2), fp32 (weights stored [out][in])."""
+    rng = np.random.default_rng([w.seed, TAG_WO, layer])
+    return rng.standard_normal((w.hidden, w.n_q_heads * w.head_dim), dtype=np.float32) * np.float32(0.02)
 
 
 def draw_bias(w, layer, n):

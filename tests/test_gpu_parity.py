@@ -325,3 +325,32 @@ def test_balanced_split_mixed_lengths(lens):
     one long sequence (segment cap), many one-tile units and CTA ranges that cross unit boundaries."""
     w = synth.scaled_down(synth.LLAMA_8B, n_layers=1, batch=len(lens), seq=max(lens))
     _random_attn_case(w, lens, 0, seed=len(lens))
+
+
+@pytest.mark.parametrize("name,hidden,T", [("tiny", None, 1), ("8b", 512, 2), ("3b", 512, 5), ("14b", 512, 4), ("8b", None, 32)])
+def test_out_proj_matches_oracle(name, hidden, T):
+    """rap_pack_wo (column gather, bit-exact) and rap_out_proj (W~_o times the reduced attention output)
+    against the oracle on the same storage-rounded inputs; the last case is the 8B shape at batch 32."""
+    w = synth.scaled_down(synth.CONFIGS[name], n_layers=2, batch=T, seq=8, hidden=hidden)
+    ks, vs = synth.draw_scores(w)
+    st = DecodeStack(w, s_cap=16, alloc_cache=False)
+    st.build_tables(ks, vs)
+    tabs = util.oracle_tables(w, ks, vs)
+    rng = np.random.default_rng(12)
+    for l in range(w.n_layers):
+        Wo = synth.draw_wo(w, l)
+        d_wo = torch.from_numpy(Wo).to(st.device).to(st.dt).contiguous()
+        d_wt = torch.empty((w.hidden, w.n_q_heads * w.n_vch), dtype=st.dt, device=st.device)
+        st.ctx.rap_pack_wo(l, d_wo, st.v_idx, d_wt)
+        want_wt = O.gather_wo(O.round_storage(Wo, w.dtype), tabs, l, w.n_vch, w.head_dim, w.n_q_heads, w.n_kv_heads)
+        torch.cuda.synchronize()
+        assert np.array_equal(util.to_np64(d_wt), want_wt)
+        o = rng.standard_normal((T, w.n_q_heads, w.n_vch)).astype(np.float32)
+        d_o = torch.from_numpy(o).to(st.device)
+        d_y = torch.full((T, w.hidden), float("nan"), dtype=st.dt, device=st.device)
+        st.ctx.rap_out_proj(l, T, d_o, d_wt, d_y)
+        torch.cuda.synchronize()
+        want = O.out_proj(O.round_storage(o, w.dtype), want_wt)
+        util.check_projection(util.to_np64(d_y), O.round_storage(want, w.dtype), w.dtype, f"{name} out_proj layer {l}")
+    assert st.ctx.rap_get_last_device_status() == (0, 0)
+    st.close()
