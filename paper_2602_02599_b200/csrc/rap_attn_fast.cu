@@ -546,7 +546,7 @@ rap_status rap_launch_attn_fast(rap_ctx* ctx, const rap_attn_args& a, int n_spli
   p.seq_len = a.seq_len; p.ws = ctx->d_attn_ws; p.status = ctx->d_status;
   p.len_add = a.len_add; p.Hq = a.Hq; p.Hkv = a.Hkv; p.WK = WK; p.dv = dv; p.S_cap = a.S_cap; p.n_split = n_split;
   p.qscale = (float)(1.4426950408889634 / sqrt((double)a.head_dim));
-  RAP_CUDA_TRY(ctx, cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BUDGET));
+  RAP_CUDA_TRY(ctx, rap_raise_smem(ctx, kern, SMEM_BUDGET));
   dim3 grid(n_split, a.Hkv, a.B);
   kern<<<grid, FTHREADS, smem, st>>>(p);
   ctx->launches++;

@@ -721,7 +721,7 @@ rap_status rap_launch_attn_scan(rap_ctx* ctx, const rap_attn_args& a, int n_spli
   p.qscale = (float)(1.4426950408889634 / sqrt((double)a.head_dim));
   p.B = a.B; p.balanced = balanced ? 1 : 0;
   p.unit_cnt = ctx->d_unit_cnt; p.out = a.out;
-  RAP_CUDA_TRY(ctx, cudaFuncSetAttribute(e->fn, cudaFuncAttributeMaxDynamicSharedMemorySize, e->smem));
+  RAP_CUDA_TRY(ctx, rap_raise_smem(ctx, e->fn, e->smem));
   const int scan_grid = 2 * ctx->sm_count;
   dim3 grid(n_split, a.Hkv, a.B);
   if (balanced) grid = dim3(scan_grid, 1, 1);

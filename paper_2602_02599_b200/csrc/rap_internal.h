@@ -5,6 +5,7 @@
 #include <cuda_bf16.h>
 #include <stdint.h>
 
+#include <set>
 #include <string>
 #include <vector>
 
@@ -46,12 +47,23 @@ struct rap_ctx {
   // optional timing of the attention launches of rap_decode_step (event pairs on the caller's stream)
   std::vector<cudaEvent_t> prof_ev;   // 2 * capacity events
   int prof_pairs = 0;                 // pairs recorded since the last read
+  std::set<const void*> attr_done;    // kernels whose dynamic shared-memory limit has been raised on this device
+  struct MapSlot { const void* base; uint64_t rows, cols; uint32_t box; unsigned char map[128]; };
+  std::vector<MapSlot> tmaps;         // encoded tensor maps, reused while (pointer, shape, box) repeat
+  size_t tmap_next = 0;
   int32_t attn_variant = 0;
   int64_t launches = 0;
   std::string cuda_error;
   // lazily created tensor maps / per-device attributes live in the .cu files
   bool smem_attr_set = false;
 };
+
+// cudaFuncSetAttribute(MaxDynamicSharedMemorySize) once per kernel and context
+template <typename F>
+static inline cudaError_t rap_raise_smem(rap_ctx* ctx, F fn, int bytes) {
+  if (!ctx->attr_done.insert((const void*)fn).second) return cudaSuccess;
+  return cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+}
 
 static inline int rap_elem_bytes(int32_t dtype) { return dtype == RAP_F32 ? 4 : 2; }
 static inline bool rap_aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }

@@ -19,6 +19,7 @@ namespace {
 
 constexpr int LR_TILE = 64;
 constexpr int LR_THREADS = 256;
+constexpr int LR_SMEM_MAX = 227 * 1024;   // the dynamic shared-memory limit is raised once, to the device maximum
 
 template <typename T> __device__ __forceinline__ float ldf(const T* p);
 template <> __device__ __forceinline__ float ldf<float>(const float* p) { return *p; }
@@ -199,15 +200,16 @@ rap_status rap_launch_lowrank_attn(rap_ctx* ctx, const rap_lowrank_args& a, cuda
   }
   const size_t smem = (size_t)(D / 2) * sizeof(double) +
                       (size_t)(a.r * D + LR_TILE * a.r + LR_TILE * (D + 1) + G * D + G * LR_TILE + G) * sizeof(float);
+  if (smem > (size_t)LR_SMEM_MAX) return RAP_EUNSUPPORTED;
   const float qscale = (float)(1.4426950408889634 / sqrt((double)D));
   dim3 grid(n_split, a.Hkv, a.B);
   if (a.dtype == RAP_F32) {
-    RAP_CUDA_TRY(ctx, cudaFuncSetAttribute(lowrank_attn_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    RAP_CUDA_TRY(ctx, rap_raise_smem(ctx, lowrank_attn_kernel<float>, LR_SMEM_MAX));
     lowrank_attn_kernel<float><<<grid, LR_THREADS, smem, st>>>(
         (const float*)a.q_full, (const float*)a.k_latent, (const float*)a.bk, (const float*)a.v, a.seq_len, a.Hq, a.Hkv,
         a.r, a.dv, D, a.S_cap, a.pairing, a.rope_theta, qscale, n_split, ctx->d_attn_ws);
   } else {
-    RAP_CUDA_TRY(ctx, cudaFuncSetAttribute(lowrank_attn_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    RAP_CUDA_TRY(ctx, rap_raise_smem(ctx, lowrank_attn_kernel<__nv_bfloat16>, LR_SMEM_MAX));
     lowrank_attn_kernel<__nv_bfloat16><<<grid, LR_THREADS, smem, st>>>(
         (const __nv_bfloat16*)a.q_full, (const __nv_bfloat16*)a.k_latent, (const __nv_bfloat16*)a.bk,
         (const __nv_bfloat16*)a.v, a.seq_len, a.Hq, a.Hkv, a.r, a.dv, D, a.S_cap, a.pairing, a.rope_theta, qscale,

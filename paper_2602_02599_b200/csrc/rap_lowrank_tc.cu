@@ -129,7 +129,7 @@ lr_rebuild_kernel(const __nv_bfloat16* __restrict__ latent, const __nv_bfloat16*
 template <int RP>
 rap_status launch_rebuild(rap_ctx* ctx, const rap_lowrank_args& a, cudaStream_t st) {
   const size_t smem = (size_t)(RB_D * (RP + 8) + RB_TILE * RB_D + 16 + RB_TILE * (RB_D + 8)) * sizeof(__nv_bfloat16);
-  RAP_CUDA_TRY(ctx, cudaFuncSetAttribute(lr_rebuild_kernel<RP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+  RAP_CUDA_TRY(ctx, rap_raise_smem(ctx, lr_rebuild_kernel<RP>, (int)smem));
   // a few CTAs per SM, each looping over tiles so that the B_k^T staging is paid once per CTA
   const int n_tiles = (a.h_len_max + RB_TILE - 1) / RB_TILE;
   int gx = (4 * ctx->sm_count + a.B * a.Hkv - 1) / (a.B * a.Hkv);

@@ -23,6 +23,8 @@
 // RAP_ETIMEOUT in the device status word and the CTA winds down.
 #include <cuda.h>
 
+#include <string.h>
+
 #include <mutex>
 
 #include "rap_internal.h"
@@ -239,22 +241,39 @@ encode_tiled_t get_encode_fn() {
 }
 
 // [rows][cols] bf16 row-major -> tiles of box_rows x 64 elements, 128-byte swizzle, zero fill outside
-bool make_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+bool make_map(rap_ctx* ctx, CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+  static_assert(sizeof(CUtensorMap) == 128, "tensor map size");
+  for (const rap_ctx::MapSlot& m : ctx->tmaps)
+    if (m.base == base && m.rows == rows && m.cols == cols && m.box == box_rows) {
+      memcpy(map, m.map, sizeof(CUtensorMap));
+      return true;
+    }
   encode_tiled_t fn = get_encode_fn();
   if (!fn) return false;
   const cuuint64_t dims[2] = {cols, rows};
   const cuuint64_t strides[1] = {cols * 2};
   const cuuint32_t box[2] = {TC_BK, box_rows};
   const cuuint32_t estr[2] = {1, 1};
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  if (fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return false;
+  rap_ctx::MapSlot slot;
+  slot.base = base; slot.rows = rows; slot.cols = cols; slot.box = box_rows;
+  memcpy(slot.map, map, sizeof(CUtensorMap));
+  if (ctx->tmaps.size() < 256) {
+    ctx->tmaps.push_back(slot);
+  } else {
+    ctx->tmaps[ctx->tmap_next] = slot;
+    ctx->tmap_next = (ctx->tmap_next + 1) % 256;
+  }
+  return true;
 }
 
 template <int TN>
 rap_status launch_tc(rap_ctx* ctx, const CUtensorMap& mw, const CUtensorMap& mx, const TcParams& p, dim3 grid,
                      cudaStream_t st) {
-  RAP_CUDA_TRY(ctx, cudaFuncSetAttribute(proj_tc_kernel<TN>, cudaFuncAttributeMaxDynamicSharedMemorySize, TcCfg<TN>::SMEM));
+  RAP_CUDA_TRY(ctx, rap_raise_smem(ctx, proj_tc_kernel<TN>, TcCfg<TN>::SMEM));
   proj_tc_kernel<TN><<<grid, TC_THREADS, TcCfg<TN>::SMEM, st>>>(mw, mx, p);
   ctx->launches++;
   RAP_CUDA_TRY(ctx, cudaGetLastError());
@@ -269,8 +288,8 @@ rap_status rap_launch_gemm_tc(rap_ctx* ctx, const void* x, const void* w, int T,
   if (T < 1 || (K % 8) != 0) return RAP_EUNSUPPORTED;     // tensor-map rows must be multiples of 16 bytes
   const int tn = T <= 32 ? 32 : T <= 64 ? 64 : 128;
   CUtensorMap mw, mx;
-  if (!make_map(&mw, w, (uint64_t)N, (uint64_t)K, TC_BM)) return RAP_EUNSUPPORTED;
-  if (!make_map(&mx, x, (uint64_t)T, (uint64_t)K, (uint32_t)tn)) return RAP_EUNSUPPORTED;
+  if (!make_map(ctx, &mw, w, (uint64_t)N, (uint64_t)K, TC_BM)) return RAP_EUNSUPPORTED;
+  if (!make_map(ctx, &mx, x, (uint64_t)T, (uint64_t)K, (uint32_t)tn)) return RAP_EUNSUPPORTED;
   const int row_tiles = (N + TC_BM - 1) / TC_BM, tok_tiles = (T + tn - 1) / tn;
   const int nkb = (K + TC_BK - 1) / TC_BK;
   // reduction split: enough CTAs for every SM on decode-sized calls, within the workspace
