@@ -404,6 +404,63 @@ def lowrank_decode_attn(q_full, k_latent, B_k, v_cache, seq_len, head_dim, rope_
 
 
 # --------------------------------------------------------------------------------------
+# Budget-Alloc (Algorithm 2, layer-adaptive budgets with mean retain ratio rho)
+# --------------------------------------------------------------------------------------
+def budget_alloc(k_pair_scores, rho, head_dim):
+    """Per-layer pair budgets m_l proportional to the layer score with mean retain ratio rho.
+
+    sigma_l = mean over heads and pairs of the pair scores (Algorithm 2, layer score).
+    The paper fixes m_l ~ sigma_l and (1/L) sum m_l / (D/2) = rho but not the rounding; the
+    reading taken here: the integer total is round(rho * D/2 * L); real-valued targets are
+    proportional to sigma_l, layers whose target leaves [1, D/2] are pinned to the bound and the
+    rest re-shared (water-filling); targets are floored and the missing units go to the largest
+    fractional parts (ties: lower layer).  V keeps 2 m_l channels (Balanced K/V).
+    Returns (n_pairs [L], n_vch [L]) as int arrays."""
+    sc = np.asarray(k_pair_scores, dtype=np.float64)
+    L, P = sc.shape[0], head_dim // 2
+    sigma = sc.reshape(L, -1).mean(axis=1)
+    total = int(math.floor(rho * P * L + 0.5))
+    total = min(max(total, L), P * L)
+    fixed = {}
+    while True:
+        free = [l for l in range(L) if l not in fixed]
+        rest = total - sum(fixed.values())
+        ssum = sum(sigma[l] for l in free)
+        target = {l: (rest * sigma[l] / ssum if ssum > 0 else rest / len(free)) for l in free}
+        over = [l for l in free if target[l] > P]
+        under = [l for l in free if target[l] < 1]
+        if over:                       # pin the layers that want more than everything first
+            for l in over:
+                fixed[l] = P
+        elif under:
+            for l in under:
+                fixed[l] = 1
+        else:
+            break
+        if len(fixed) == L:
+            target = {}
+            break
+    m = np.zeros(L, dtype=np.int64)
+    for l, v in fixed.items():
+        m[l] = v
+    free = sorted(target)
+    for l in free:
+        m[l] = int(math.floor(target[l]))
+    missing = total - int(m.sum())
+    order = sorted(free, key=lambda l: (-(target[l] - math.floor(target[l])), l))
+    i = 0
+    while missing > 0 and order:
+        l = order[i % len(order)]
+        if m[l] < P:
+            m[l] += 1
+            missing -= 1
+        i += 1
+        if i > 4 * len(order) + missing:
+            break
+    return m.astype(np.int32), (2 * m).astype(np.int32)
+
+
+# --------------------------------------------------------------------------------------
 # output projection on the retained V channels (Algorithm 1: W~_o = E_v W_o absorbs the V selection)
 # --------------------------------------------------------------------------------------
 def gather_wo(Wo, tables, layer, n_vch_l, head_dim, Hq, Hkv):

@@ -366,3 +366,30 @@ def test_out_proj_equals_dense_wo_on_zero_expanded_output():
     # negative control: using another head's V selection breaks the identity
     bad = O.gather_wo(Wo, m["tabs"], 0, dv, D, Hq, Hkv)[:, ::-1]
     assert np.abs(O.out_proj(o, bad) - want).max() > 1e-3
+
+
+# ---- Budget-Alloc (Algorithm 2) ----------------------------------------------------------------
+def test_budget_alloc_properties():
+    rng = np.random.default_rng(4)
+    D, L, H = 128, 32, 8
+    for rho in (0.5, 0.7, 0.9):
+        sc = rng.lognormal(0, 1, (L, H, D // 2)) * np.linspace(0.6, 1.6, L)[:, None, None]
+        m, nv = O.budget_alloc(sc, rho, D)
+        sigma = sc.reshape(L, -1).mean(axis=1)
+        assert m.sum() == round(rho * 64 * L)                      # mean retain ratio = rho (Algorithm 2)
+        assert m.min() >= 1 and m.max() <= 64 and np.array_equal(nv, 2 * m)   # whole pairs; V keeps 2 m_l
+        order = np.argsort(sigma)
+        assert np.all(np.diff(m[order]) >= 0)                     # more sensitive layers never get less
+        if m.max() < 64 and m.min() > 1:                          # no clipping: proportional up to rounding
+            t = rho * 64 * L * sigma / sigma.sum()
+            assert np.abs(m - t).max() < 1.0
+    # equal layer scores: the uniform budget (rho * D/2 whole pairs everywhere when that is an integer;
+    # otherwise the layers differ by at most one pair and the mean is kept)
+    m, _ = O.budget_alloc(np.ones((8, 2, 64)), 0.75, 128)
+    assert np.array_equal(m, np.full(8, 48))
+    m, _ = O.budget_alloc(np.ones((8, 2, 64)), 0.7, 128)
+    assert m.sum() == 358 and set(m.tolist()) == {44, 45}
+    # one dominant layer is capped at all pairs and the rest share what is left
+    sc = np.ones((4, 1, 32)); sc[0] *= 100
+    m, _ = O.budget_alloc(sc, 0.5, 64)
+    assert m[0] == 32 and m.sum() == 64 and np.all(m[1:] >= 10)
