@@ -82,6 +82,16 @@ const char* rap_last_cuda_error(const rap_ctx* ctx);
  * RAP_EINVAL unless 0 < rho <= 1 and D even. */
 rap_status rap_retained_counts(double rho, int32_t head_dim, int32_t* n_pairs, int32_t* n_vch);
 
+/* Budget-Alloc (Algorithm 2): layer-adaptive pair budgets m_l proportional to the layer score
+ * sigma_l = mean over heads and pairs of h_k_pair_scores [L][H_kv][D/2] (HOST fp64, non-negative), with
+ * mean retain ratio rho; head-uniform inside a layer; V keeps 2 m_l channels (Balanced K/V).  The paper
+ * does not fix the rounding: the integer total is round(rho * D/2 * L), layers whose proportional share
+ * leaves [1, D/2] are pinned to the bound and the rest re-shared, shares are floored and the missing
+ * units go to the largest fractional parts (ties: lower layer).  Host-only, no GPU work.  The results
+ * feed rap_build_tables. */
+rap_status rap_budget_alloc(int32_t n_layers, int32_t n_kv_heads, int32_t head_dim, const double* h_k_pair_scores,
+                            double rho, int32_t* h_n_pairs, int32_t* h_n_vch);
+
 /* Element offset of (b, h, pos, c) in a cache of row width W: ((b*H_kv + h)*S_cap + pos)*W + c. */
 size_t rap_cache_elem_offset(int32_t n_kv_heads, int32_t S_cap, int32_t W, int32_t b, int32_t h,
                              int32_t pos, int32_t c);

@@ -25,7 +25,7 @@ EXPORTS = [
     "rap_decode_attn", "rap_decode_step", "rap_decode_step_host", "rap_lowrank_decode_attn",
     "rap_get_last_device_status", "rap_kernel_launch_count", "rap_set_attn_variant",
     "rap_decode_attn_noalloc", "rap_profile_attn", "rap_profile_attn_read",
-    "rap_pack_wo", "rap_out_proj",
+    "rap_pack_wo", "rap_out_proj", "rap_budget_alloc",
 ]
 
 
@@ -77,6 +77,7 @@ def _lib():
     lib.rap_kernel_launch_count.argtypes = [P]
     lib.rap_kernel_launch_count.restype = c_int64
     lib.rap_set_attn_variant.argtypes = [P, c_int32]
+    lib.rap_budget_alloc.argtypes = [c_int32, c_int32, c_int32, P, c_double, P, P]
     lib.rap_pack_wo.argtypes = [P, c_int32, P, P, P, P]
     lib.rap_out_proj.argtypes = [P, c_int32, c_int32, P, P, P, P]
     lib.rap_profile_attn.argtypes = [P, c_int32]
@@ -119,6 +120,17 @@ def rap_retained_counts(rho, head_dim):
     if s:
         raise RapError(s, "rap_retained_counts")
     return P.value, dv.value
+
+
+def rap_budget_alloc(k_pair_scores, rho, head_dim):
+    """(n_pairs [L], n_vch [L]) int32 arrays of Algorithm 2 for host scores [L][H_kv][D/2]."""
+    ks = np.ascontiguousarray(k_pair_scores, dtype=np.float64)
+    L, H = ks.shape[0], ks.shape[1]
+    n_pairs, n_vch = np.zeros(L, dtype=np.int32), np.zeros(L, dtype=np.int32)
+    s = _lib().rap_budget_alloc(L, H, head_dim, _ptr(ks), float(rho), _ptr(n_pairs), _ptr(n_vch))
+    if s:
+        raise RapError(s, "rap_budget_alloc")
+    return n_pairs, n_vch
 
 
 def rap_cache_elem_offset(n_kv_heads, S_cap, W, b, h, pos, c):

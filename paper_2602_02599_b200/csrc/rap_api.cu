@@ -79,6 +79,72 @@ size_t rap_cache_elem_offset(int32_t n_kv_heads, int32_t S_cap, int32_t W, int32
   return (((size_t)b * (size_t)n_kv_heads + (size_t)h) * (size_t)S_cap + (size_t)pos) * (size_t)W + (size_t)c;
 }
 
+rap_status rap_budget_alloc(int32_t n_layers, int32_t n_kv_heads, int32_t head_dim, const double* k_pair_scores,
+                            double rho, int32_t* n_pairs, int32_t* n_vch) {
+  if (!k_pair_scores || !n_pairs || !n_vch || n_layers < 1 || n_kv_heads < 1 || head_dim < 2 || (head_dim & 1) ||
+      !(rho > 0.0) || rho > 1.0)
+    return RAP_EINVAL;
+  const int L = n_layers, P = head_dim / 2;
+  const size_t per_layer = (size_t)n_kv_heads * P;
+  std::vector<double> sigma(L);
+  for (int l = 0; l < L; ++l) {
+    double s = 0.0;
+    for (size_t i = 0; i < per_layer; ++i) {
+      const double v = k_pair_scores[(size_t)l * per_layer + i];
+      if (std::isnan(v) || v < 0.0) return RAP_EINVAL;
+      s += v;
+    }
+    sigma[l] = s / (double)per_layer;
+  }
+  long total = (long)std::floor(rho * (double)P * (double)L + 0.5);
+  total = std::min<long>(std::max<long>(total, L), (long)P * L);
+  // water-filling: layers whose proportional share leaves [1, P] are pinned to the bound, the rest re-share
+  std::vector<int> pinned(L, 0);
+  std::vector<double> target(L, 0.0);
+  for (;;) {
+    long rest = total;
+    double ssum = 0.0;
+    int n_free = 0;
+    for (int l = 0; l < L; ++l) {
+      if (pinned[l]) rest -= pinned[l];
+      else { ssum += sigma[l]; ++n_free; }
+    }
+    if (n_free == 0) break;
+    bool over = false, under = false;
+    for (int l = 0; l < L; ++l) {
+      if (pinned[l]) continue;
+      target[l] = ssum > 0.0 ? (double)rest * sigma[l] / ssum : (double)rest / (double)n_free;
+      over |= target[l] > (double)P;
+      under |= target[l] < 1.0;
+    }
+    if (over) {
+      for (int l = 0; l < L; ++l) if (!pinned[l] && target[l] > (double)P) pinned[l] = P;
+    } else if (under) {
+      for (int l = 0; l < L; ++l) if (!pinned[l] && target[l] < 1.0) pinned[l] = 1;
+    } else {
+      break;
+    }
+  }
+  std::vector<int> free_layers;
+  long have = 0;
+  for (int l = 0; l < L; ++l) {
+    if (pinned[l]) n_pairs[l] = pinned[l];
+    else { n_pairs[l] = (int32_t)std::floor(target[l]); free_layers.push_back(l); }
+    have += n_pairs[l];
+  }
+  // the units lost to flooring go to the largest fractional parts (ties: lower layer)
+  std::stable_sort(free_layers.begin(), free_layers.end(), [&](int a, int b) {
+    return (target[a] - std::floor(target[a])) > (target[b] - std::floor(target[b]));
+  });
+  long missing = total - have;
+  for (size_t i = 0, spins = 0; missing > 0 && !free_layers.empty() && spins < 4 * free_layers.size() + (size_t)total; ++i, ++spins) {
+    const int l = free_layers[i % free_layers.size()];
+    if (n_pairs[l] < P) { ++n_pairs[l]; --missing; }
+  }
+  for (int l = 0; l < L; ++l) n_vch[l] = 2 * n_pairs[l];
+  return RAP_OK;
+}
+
 rap_status rap_create(const rap_model_desc* desc, rap_ctx** out) {
   if (!desc || !out) return RAP_EINVAL;
   *out = nullptr;

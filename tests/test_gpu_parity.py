@@ -53,11 +53,12 @@ def test_pack_weights_bit_exact():
     st.close()
 
 
-def _end_to_end(w, lens_before, n_split=0, with_bias=False, chunk=None):
+def _end_to_end(w, lens_before, n_split=0, with_bias=False, chunk=None, n_pairs=None, n_vch=None):
     """Prefill lens_before[b] tokens per sequence, then one decode step; compare every stage."""
     ks, vs = synth.draw_scores(w)
     T_pre = int(np.sum(lens_before))
-    st, tabs, w_host = util.build_small_stack(w, ks, vs, full_weights=True, max_rows=max(chunk or T_pre, w.batch))
+    st, tabs, w_host = util.build_small_stack(w, ks, vs, full_weights=True, max_rows=max(chunk or T_pre, w.batch),
+                                              n_pairs=n_pairs, n_vch=n_vch)
     B, Hq, Hkv, D = w.batch, w.n_q_heads, w.n_kv_heads, w.head_dim
     bias_host = None
     if with_bias:
@@ -354,3 +355,14 @@ def test_out_proj_matches_oracle(name, hidden, T):
         util.check_projection(util.to_np64(d_y), O.round_storage(want, w.dtype), w.dtype, f"{name} out_proj layer {l}")
     assert st.ctx.rap_get_last_device_status() == (0, 0)
     st.close()
+
+
+def test_layer_adaptive_budgets_end_to_end():
+    """Budgets from rap_budget_alloc (Algorithm 2: per-layer P_l, d_v' = 2 P_l) through tables, projection,
+    append and attention: every layer has its own row widths."""
+    w = synth.scaled_down(synth.LLAMA_8B, n_layers=4, batch=2, seq=300, hidden=256)
+    ks, _ = synth.draw_scores(w)
+    ks = ks * np.array([0.5, 1.0, 1.6, 0.9])[:, None, None]
+    n_pairs, n_vch = binding.rap_budget_alloc(ks, 0.7, w.head_dim)
+    assert len(set(n_pairs.tolist())) > 1 and n_pairs.sum() == round(0.7 * 64 * 4)
+    _end_to_end(w, [300, 211], chunk=256, n_pairs=n_pairs.tolist(), n_vch=n_vch.tolist())

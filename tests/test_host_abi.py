@@ -83,3 +83,20 @@ def test_missing_library_fails_loudly(monkeypatch):
     monkeypatch.setattr(binding, "LIB_PATH", "/nonexistent/librap_b200.so")
     with pytest.raises(RuntimeError, match="no fallback"):
         binding._lib()
+
+
+def test_budget_alloc_matches_the_oracle(lib):
+    """rap_budget_alloc (host C++) against the oracle's Algorithm 2 on seeded scores, with clipping cases."""
+    import numpy as np
+    from oracle import rap_oracle as O
+    rng = np.random.default_rng(9)
+    for L, H, D, rho, spread in [(32, 8, 128, 0.7, 1.0), (28, 8, 128, 0.9, 3.0), (48, 8, 128, 0.5, 0.3), (4, 1, 64, 0.5, 50.0),
+                                 (6, 2, 16, 0.2, 8.0)]:
+        sc = rng.lognormal(0, 1, (L, H, D // 2)) * np.exp(rng.normal(0, np.log1p(spread), L))[:, None, None]
+        got_p, got_v = binding.rap_budget_alloc(sc, rho, D)
+        want_p, want_v = O.budget_alloc(sc, rho, D)
+        assert np.array_equal(got_p, want_p) and np.array_equal(got_v, want_v), (L, rho)
+    n = np.zeros(2, dtype=np.int32)
+    bad = np.ones((2, 1, 8))
+    assert lib.rap_budget_alloc(2, 1, 16, binding._ptr(bad), 0.0, binding._ptr(n), binding._ptr(n)) == binding.RAP_EINVAL
+    assert lib.rap_budget_alloc(2, 1, 15, binding._ptr(bad), 0.5, binding._ptr(n), binding._ptr(n)) == binding.RAP_EINVAL
