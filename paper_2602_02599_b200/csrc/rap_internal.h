@@ -77,6 +77,29 @@ static inline bool rap_aligned16(const void* p) { return (reinterpret_cast<uintp
     }                                                                   \
   } while (0)
 
+// Parameters and lookup entry of the shape-specialised split-KV scan (rap_attn_scan_kernel.cuh).
+struct rap_scan_params {
+  const uint32_t* q;          // [B][Hq][WK] bf16 pairs
+  const unsigned char* k;     // [B][Hkv][S_cap][WK * 4 bytes]
+  const unsigned char* v;     // [B][Hkv][S_cap][DV * 2 bytes]
+  const int32_t* seq_len;
+  float* ws;
+  int32_t* status;
+  int len_add, Hq, Hkv, S_cap, n_split;
+  float qscale;
+  int32_t* unit_cnt;   // balanced mode: arrivals per (sequence, KV head) unit, zero between calls
+  float* out;          // balanced mode: [B][Hq][DV], written by the CTA that completes a unit
+  int B;               // sequences (used by the balanced mode)
+  int balanced;        // 0: grid (n_split, H_kv, B), equal tile ranges per split; 1: grid (CTAs), see SkPlan
+};
+struct rap_scan_entry {
+  int G, WK, DV;       // query heads per KV head, K words per row (= P), V channels (= d_v')
+  int smem, tile;      // dynamic shared memory, positions per tile
+  const void* fn;      // the kernel, launched with cudaLaunchKernel
+};
+// the instantiation built for this head shape, or nullptr (generated at build time)
+const rap_scan_entry* rap_scan_find(int G, int WK, int DV);
+
 // Launchers implemented in the kernel files.  All return RAP_OK or RAP_ECUDA.
 struct rap_attn_args {
   const void* q; const void* k; const void* v;

@@ -366,3 +366,13 @@ def test_layer_adaptive_budgets_end_to_end():
     n_pairs, n_vch = binding.rap_budget_alloc(ks, 0.7, w.head_dim)
     assert len(set(n_pairs.tolist())) > 1 and n_pairs.sum() == round(0.7 * 64 * 4)
     _end_to_end(w, [300, 211], chunk=256, n_pairs=n_pairs.tolist(), n_vch=n_vch.tolist())
+
+
+@pytest.mark.parametrize("P,dv", [(24, 48), (40, 80), (41, 82), (56, 112), (16, 32), (63, 126)])
+def test_layer_adaptive_head_shapes_attention(P, dv):
+    """Head shapes that layer-adaptive budgets produce (d_v' = 2P): K rows that are multiples of 32 bytes
+    take the rotated logits mapping with a partly filled last unit group, the others the chunked one."""
+    from dataclasses import replace
+    w = replace(synth.scaled_down(synth.LLAMA_8B, n_layers=1, batch=3, seq=3000), n_pairs=P, n_vch=dv)
+    _random_attn_case(w, [3000, 1777, 1], 0, seed=P)
+    _random_attn_case(w, [3000, 1777, 1], 3, seed=P)
