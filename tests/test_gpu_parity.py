@@ -376,3 +376,44 @@ def test_layer_adaptive_head_shapes_attention(P, dv):
     w = replace(synth.scaled_down(synth.LLAMA_8B, n_layers=1, batch=3, seq=3000), n_pairs=P, n_vch=dv)
     _random_attn_case(w, [3000, 1777, 1], 0, seed=P)
     _random_attn_case(w, [3000, 1777, 1], 3, seed=P)
+
+
+def test_decode_step_replays_from_a_cuda_graph():
+    """rap_decode_step reads the sequence lengths on the device and its balanced scan has a fixed grid, so a
+    step captured once can be replayed as the lengths advance: two replays equal two eager steps bit for bit."""
+    w = synth.scaled_down(synth.LLAMA_8B, n_layers=2, batch=2, seq=300, hidden=256)
+    ks, vs = synth.draw_scores(w)
+    st, tabs, w_host = util.build_small_stack(w, ks, vs, full_weights=False)
+    g = torch.Generator(device=st.device).manual_seed(5)
+    for l in range(w.n_layers):
+        st.k_cache[l].normal_(0, 1.0, generator=g)
+        st.v_cache[l].normal_(0, 1.0, generator=g)
+    k0 = [c.clone() for c in st.k_cache]
+    v0 = [c.clone() for c in st.v_cache]
+    x = torch.empty((w.n_layers, w.batch, w.hidden), dtype=st.dt, device=st.device).normal_(0, 1, generator=g)
+
+    def reset():
+        for l in range(w.n_layers):
+            st.k_cache[l].copy_(k0[l])
+            st.v_cache[l].copy_(v0[l])
+        st.seq_len.copy_(torch.tensor([300, 123], dtype=torch.int32))
+
+    reset()
+    eager = []
+    for i in range(2):
+        st.decode_step(x, 300 + i, advance=1)
+        eager.append(st.out.clone())
+    torch.cuda.synchronize()
+    reset()
+    graph = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    with torch.cuda.graph(graph, stream=side):
+        st.decode_step(x, 301, advance=1)      # the host bound covers both replays
+    reset()                                    # capture does not run the work, but keep the state explicit
+    for i in range(2):
+        graph.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(st.out, eager[i])
+    assert st.seq_len.cpu().tolist() == [302, 125]
+    assert st.ctx.rap_get_last_device_status() == (0, 0)
+    st.close()
