@@ -82,8 +82,10 @@ template <typename T> __device__ __forceinline__ float from_storage(T v);
 template <> __device__ __forceinline__ float from_storage<float>(float v) { return v; }
 template <> __device__ __forceinline__ float from_storage<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
 
-// One thread per (row t, item): items are the (H_q + H_kv) * P rotation pairs followed by the
-// H_kv * d_v' value channels.  y holds `ksplit` partial results, each [T][n_out].
+// One thread per (row t, item): items are the H_kv * P retained pairs (c-th pair of KV head h) followed by
+// the H_kv * d_v' value channels.  A pair item evaluates the angle pos * inv_freq[h][c] once (fp64) and
+// rotates the k pair of head h and the q pairs of its G query heads with it.  y holds `ksplit` partial
+// results, each [T][n_out].
 template <typename T>
 __global__ void rope_append_kernel(const float* __restrict__ y, int ksplit, const T* __restrict__ bias,
                                    const int32_t* __restrict__ seq_id, const int32_t* __restrict__ pos,
@@ -92,7 +94,7 @@ __global__ void rope_append_kernel(const float* __restrict__ y, int ksplit, cons
                                    int Hq, int Hkv, int P2, int dv, int half_dim, int B_cache, int S_cap,
                                    int32_t* __restrict__ status) {
   const int P = P2 >> 1;
-  const int n_pair_items = (Hq + Hkv) * P;
+  const int n_pair_items = Hkv * P;
   const int n_items = n_pair_items + Hkv * dv;
   const int n_out = (Hq + Hkv) * P2 + Hkv * dv;
   const long long gid = (long long)blockIdx.x * blockDim.x + threadIdx.x;
@@ -110,29 +112,31 @@ __global__ void rope_append_kernel(const float* __restrict__ y, int ksplit, cons
   const size_t split_stride = (size_t)Trows * n_out;
   const float* yr = y + (size_t)t * n_out;
   if (item < n_pair_items) {
-    const int head = item / P, c = item - head * P;     // head < Hq: query head, else KV head
-    const int col = head * P2 + 2 * c;
-    float a = 0.f, b = 0.f;
-    for (int s = 0; s < ksplit; ++s) {
-      a += yr[s * split_stride + col];
-      b += yr[s * split_stride + col + 1];
-    }
-    if (bias) { a += from_storage<T>(bias[col]); b += from_storage<T>(bias[col + 1]); }
+    const int h = item / P, c = item - h * P;
     const int G = Hq / Hkv;
-    const int h = head < Hq ? head / G : head - Hq;
     double sn, cs;
     sincos((double)p * inv_freq[h * half_dim + c], &sn, &cs);
     const float cf = (float)cs, sf = (float)sn;
-    const float ra = a * cf - b * sf;
-    const float rb = a * sf + b * cf;
-    if (head < Hq) {
-      T* dst = q_out + ((size_t)t * Hq + head) * P2 + 2 * c;
-      dst[0] = to_storage<T>(ra);
-      dst[1] = to_storage<T>(rb);
-    } else if (row_ok) {
-      T* dst = k_cache + (((size_t)sq * Hkv + h) * S_cap + sl) * P2 + 2 * c;
-      dst[0] = to_storage<T>(ra);
-      dst[1] = to_storage<T>(rb);
+    for (int j = 0; j <= G; ++j) {          // j < G: query head h*G + j; j == G: the key head itself
+      const int head = j < G ? h * G + j : Hq + h;
+      const int col = head * P2 + 2 * c;
+      float a = 0.f, b = 0.f;
+      for (int s = 0; s < ksplit; ++s) {
+        a += yr[s * split_stride + col];          // (rows of y are only 4-byte aligned when n_out is odd)
+        b += yr[s * split_stride + col + 1];
+      }
+      if (bias) { a += from_storage<T>(bias[col]); b += from_storage<T>(bias[col + 1]); }
+      const float ra = a * cf - b * sf;
+      const float rb = a * sf + b * cf;
+      if (j < G) {
+        T* dst = q_out + ((size_t)t * Hq + head) * P2 + 2 * c;
+        dst[0] = to_storage<T>(ra);
+        dst[1] = to_storage<T>(rb);
+      } else if (row_ok) {
+        T* dst = k_cache + (((size_t)sq * Hkv + h) * S_cap + sl) * P2 + 2 * c;
+        dst[0] = to_storage<T>(ra);
+        dst[1] = to_storage<T>(rb);
+      }
     }
   } else if (row_ok) {
     const int vi = item - n_pair_items;
@@ -233,7 +237,7 @@ rap_status run_generic(rap_ctx* ctx, const rap_proj_args& a, int n_out, cudaStre
 template <typename T>
 rap_status run_epilogue(rap_ctx* ctx, const rap_proj_args& a, int ksplit, cudaStream_t st) {
   const int P = a.P2 / 2;
-  const long long total = (long long)a.T * ((a.Hq + a.Hkv) * P + a.Hkv * a.dv);
+  const long long total = (long long)a.T * (a.Hkv * P + a.Hkv * a.dv);
   const int threads = 256;
   const unsigned blocks = (unsigned)((total + threads - 1) / threads);
   rope_append_kernel<T><<<blocks, threads, 0, st>>>(ctx->d_proj_ws, ksplit, (const T*)a.bias, a.seq_id, a.pos, a.slot,

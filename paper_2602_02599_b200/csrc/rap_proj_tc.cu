@@ -4,7 +4,7 @@
 //   Y[ks][t][n] = sum_{k in split ks} X[t][k] * W~[n][k]
 //
 // computed "swap-AB": the weight rows sit on the MMA's M side (128 rows per CTA, the full
-// tensor-memory lane range) and the tokens on its N side (32 / 64 / 128 per CTA), so that a
+// tensor-memory lane range) and the tokens on its N side (32 / 64 / 128 / 256 per CTA), so that a
 // decode-sized call (T <= 32) still issues full-height instructions and is bounded by streaming
 // the weights from HBM, while a prefill-shaped call (T in the thousands) is a dense contraction.
 // Both operands are K-major, staged by TMA (cp.async.bulk.tensor.2d, 128-byte swizzle, no
@@ -286,7 +286,7 @@ rap_status launch_tc(rap_ctx* ctx, const CUtensorMap& mw, const CUtensorMap& mx,
 rap_status rap_launch_gemm_tc(rap_ctx* ctx, const void* x, const void* w, int T, int K, int N, int* ksplit_out,
                               cudaStream_t st) {
   if (T < 1 || (K % 8) != 0) return RAP_EUNSUPPORTED;     // tensor-map rows must be multiples of 16 bytes
-  const int tn = T <= 32 ? 32 : T <= 64 ? 64 : 128;
+  const int tn = T <= 32 ? 32 : T <= 64 ? 64 : T <= 128 ? 128 : 256;
   CUtensorMap mw, mx;
   if (!make_map(ctx, &mw, w, (uint64_t)N, (uint64_t)K, TC_BM)) return RAP_EUNSUPPORTED;
   if (!make_map(ctx, &mx, x, (uint64_t)T, (uint64_t)K, (uint32_t)tn)) return RAP_EUNSUPPORTED;
@@ -308,7 +308,8 @@ rap_status rap_launch_gemm_tc(rap_ctx* ctx, const void* x, const void* w, int T,
   switch (tn) {
     case 32: return launch_tc<32>(ctx, mw, mx, p, grid, st);
     case 64: return launch_tc<64>(ctx, mw, mx, p, grid, st);
-    default: return launch_tc<128>(ctx, mw, mx, p, grid, st);
+    case 128: return launch_tc<128>(ctx, mw, mx, p, grid, st);
+    default: return launch_tc<256>(ctx, mw, mx, p, grid, st);
   }
 }
 
