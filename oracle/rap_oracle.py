@@ -270,6 +270,36 @@ def decode_attn(q, k_cache, v_cache, seq_len, head_dim):
     return out
 
 
+def prefill_attn(q, k_cache, v_cache, start, head_dim):
+    """Causal attention of T new tokens per sequence over the reduced dims (Eq. 2 for every t of
+    the block: token i of sequence b sits at cache row start[b] + i and attends rows 0 .. start[b] + i).
+
+    q [B][T][H_q][2P]; caches as in decode_attn, already holding the T new rows; output
+    [B][T][H_q][d_v'].  Written in the masked-matrix form softmax(Q K^T / sqrt(D) + mask) V, on purpose
+    unlike decode_attn's per-query loop: the two are pinned against each other.
+    """
+    q = np.asarray(q, dtype=np.float64)
+    B, T, Hq, _ = q.shape
+    Hkv = k_cache.shape[1]
+    G = Hq // Hkv
+    dv = v_cache.shape[3]
+    out = np.zeros((B, T, Hq, dv), dtype=np.float64)
+    for b in range(B):
+        n = int(start[b]) + T
+        rows = np.arange(n)[None, :]
+        allowed = rows <= (int(start[b]) + np.arange(T))[:, None]           # [T][n] causal mask
+        for g in range(Hq):
+            h = g // G
+            K = np.asarray(k_cache[b, h, :n], dtype=np.float64)
+            V = np.asarray(v_cache[b, h, :n], dtype=np.float64)
+            S = (q[b, :, g, :] @ K.T) / math.sqrt(float(head_dim))
+            S = np.where(allowed, S, -np.inf)
+            Pm = np.exp(S - S.max(axis=1, keepdims=True))
+            Pm = Pm / Pm.sum(axis=1, keepdims=True)
+            out[b, :, g, :] = Pm @ V
+    return out
+
+
 def attn_partial(q_g, K, V, head_dim):
     """(m, l, acc) of one split: m = max logit, l = sum exp(s-m), acc = sum exp(s-m) V."""
     if K.shape[0] == 0:

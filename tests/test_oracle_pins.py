@@ -393,3 +393,26 @@ def test_budget_alloc_properties():
     sc = np.ones((4, 1, 32)); sc[0] *= 100
     m, _ = O.budget_alloc(sc, 0.5, 64)
     assert m[0] == 32 and m.sum() == 64 and np.all(m[1:] >= 10)
+
+
+# ---- prefill (causal block) attention on the reduced dims --------------------------------------
+def test_prefill_attn_equals_per_token_decode_attention():
+    """The masked-matrix form equals running the decode definition token by token with the prefix length
+    of each token (Eq. 2 holds for every t), and the first token of an empty cache returns V_0."""
+    rng = np.random.default_rng(17)
+    B, T, Hq, Hkv, P2, dv, D, cap = 2, 5, 4, 2, 6, 5, 8, 16
+    K = rng.normal(0, 1, (B, Hkv, cap, P2))
+    V = rng.normal(0, 1, (B, Hkv, cap, dv))
+    q = rng.normal(0, 1, (B, T, Hq, P2))
+    start = [3, 0]
+    got = O.prefill_attn(q, K, V, start, D)
+    for i in range(T):
+        want = O.decode_attn(q[:, i], K, V, [start[0] + i + 1, start[1] + i + 1], D)
+        assert np.allclose(got[:, i], want, rtol=0, atol=1e-13)
+    assert np.allclose(got[1, 0], np.repeat(V[1, :, 0, :], Hq // Hkv, axis=0), rtol=0, atol=1e-15)
+    # a future row must not leak: changing rows after a token's position leaves its output unchanged
+    K2, V2 = K.copy(), V.copy()
+    K2[:, :, 6:, :] += 5.0
+    V2[:, :, 6:, :] -= 3.0
+    got2 = O.prefill_attn(q, K2, V2, start, D)
+    assert np.array_equal(got2[0, :3], got[0, :3]) and not np.allclose(got2[0, 3:], got[0, 3:])
