@@ -182,6 +182,16 @@ rap_status rap_decode_attn_noalloc(int32_t dtype, int32_t B, int32_t n_q_heads, 
                                    const int32_t* d_seq_len, int32_t h_seq_len_max, int32_t n_split,
                                    float* d_out, void* stream);
 
+/* ---- causal attention of a block of new tokens on the reduced dims (Eq. 2 for every t of the block) --
+ * Prefill-side counterpart of rap_decode_attn: each of the B sequences has T new tokens whose q~ rows are
+ * d_q [B][T][H_q][2P] and whose K / V rows are already in the caches (written by rap_qkv_rope_append) at
+ * rows d_start[b] .. d_start[b] + T - 1; token i attends rows 0 .. d_start[b] + i.
+ * d_out [B][T][H_q][d_v'] fp32.  h_start_max: caller's bound on d_start (RAP_ECAPACITY if
+ * h_start_max + T > S_cap).  Tensor-core kernel, bf16 storage only (RAP_EUNSUPPORTED for fp32 stacks). */
+rap_status rap_prefill_attn(rap_ctx* ctx, int32_t layer, int32_t B, int32_t T, const void* d_q, const void* d_k_cache,
+                            const void* d_v_cache, int32_t S_cap, const int32_t* d_start, int32_t h_start_max,
+                            float* d_out, void* stream);
+
 /* ---- output projection on the retained V channels (Algorithm 1: W~_o = E_v W_o) ------------
  * rap_pack_wo: offline column gather.  d_wo [hidden][H_q*D] is the dense W_o of `layer` (stored
  * [out][in]); d_wo_tilde [hidden][H_q*d_v'] receives, for query head g and retained channel c, the

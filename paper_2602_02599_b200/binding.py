@@ -25,7 +25,7 @@ EXPORTS = [
     "rap_decode_attn", "rap_decode_step", "rap_decode_step_host", "rap_lowrank_decode_attn",
     "rap_get_last_device_status", "rap_kernel_launch_count", "rap_set_attn_variant",
     "rap_decode_attn_noalloc", "rap_profile_attn", "rap_profile_attn_read",
-    "rap_pack_wo", "rap_out_proj", "rap_budget_alloc",
+    "rap_pack_wo", "rap_out_proj", "rap_budget_alloc", "rap_prefill_attn",
 ]
 
 
@@ -78,6 +78,7 @@ def _lib():
     lib.rap_kernel_launch_count.restype = c_int64
     lib.rap_set_attn_variant.argtypes = [P, c_int32]
     lib.rap_budget_alloc.argtypes = [c_int32, c_int32, c_int32, P, c_double, P, P]
+    lib.rap_prefill_attn.argtypes = [P, c_int32, c_int32, c_int32, P, P, P, c_int32, P, c_int32, P, P]
     lib.rap_pack_wo.argtypes = [P, c_int32, P, P, P, P]
     lib.rap_out_proj.argtypes = [P, c_int32, c_int32, P, P, P, P]
     lib.rap_profile_attn.argtypes = [P, c_int32]
@@ -244,6 +245,10 @@ class RapContext:
 
     def rap_kernel_launch_count(self):
         return int(_lib().rap_kernel_launch_count(self._ctx))
+
+    def rap_prefill_attn(self, layer, B, T, d_q, d_k_cache, d_v_cache, S_cap, d_start, h_start_max, d_out):
+        self._check(_lib().rap_prefill_attn(self._ctx, layer, B, T, _ptr(d_q), _ptr(d_k_cache), _ptr(d_v_cache), S_cap,
+                                            _ptr(d_start), h_start_max, _ptr(d_out), _stream()), "rap_prefill_attn")
 
     def rap_pack_wo(self, layer, d_wo, d_v_idx, d_wo_tilde):
         self._check(_lib().rap_pack_wo(self._ctx, layer, _ptr(d_wo), _ptr(d_v_idx), _ptr(d_wo_tilde), _stream()),

@@ -362,6 +362,24 @@ rap_status rap_decode_attn(rap_ctx* ctx, int32_t layer, int32_t B, const void* d
   return rap_launch_attn(ctx, a, (cudaStream_t)stream);
 }
 
+rap_status rap_prefill_attn(rap_ctx* ctx, int32_t layer, int32_t B, int32_t T, const void* d_q, const void* d_k_cache,
+                            const void* d_v_cache, int32_t S_cap, const int32_t* d_start, int32_t h_start_max,
+                            float* d_out, void* stream) {
+  if (!ctx || !d_q || !d_k_cache || !d_v_cache || !d_start || !d_out) return RAP_EINVAL;
+  if (!ctx->tables_built) return RAP_ESTATE;
+  const rap_model_desc& d = ctx->desc;
+  if (layer < 0 || layer >= d.n_layers || B < 0 || T < 0 || S_cap < 1 || h_start_max < 0) return RAP_EINVAL;
+  if (B > d.max_batch) return RAP_ESHAPE;
+  if (S_cap % 8) return RAP_EALIGN;
+  if ((long long)h_start_max + T > S_cap) return RAP_ECAPACITY;
+  if (!rap_aligned16(d_q) || !rap_aligned16(d_k_cache) || !rap_aligned16(d_v_cache) || !rap_aligned16(d_out) ||
+      !rap_aligned16(d_start))
+    return RAP_EALIGN;
+  if (B == 0 || T == 0) return RAP_OK;
+  return rap_launch_prefill_attn(ctx, B, T, d_q, d_k_cache, d_v_cache, 2 * ctx->n_pairs[layer], ctx->n_vch[layer], S_cap,
+                                 d_start, d_out, (cudaStream_t)stream);
+}
+
 rap_status rap_decode_step(rap_ctx* ctx, int32_t B, const void* d_x, const void* const* h_w_qkv,
                            const void* const* h_bias, const double* d_inv_freq, void* const* h_k_cache,
                            void* const* h_v_cache, int32_t S_cap, int32_t* d_seq_len, int32_t h_seq_len_max,

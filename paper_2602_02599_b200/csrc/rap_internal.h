@@ -130,6 +130,8 @@ rap_status rap_launch_pack(rap_ctx* ctx, int32_t layer, const void* wq, const vo
                            const int32_t* k_dim_idx, const int32_t* v_idx, void* w_qkv,
                            const void* bq, const void* bk, const void* bv, void* bias, cudaStream_t st);
 rap_status rap_launch_advance(rap_ctx* ctx, int32_t* seq_len, int32_t B, cudaStream_t st);
+rap_status rap_launch_prefill_attn(rap_ctx* ctx, int B, int T, const void* q, const void* k, const void* v, int P2,
+                                   int dv, int S_cap, const int32_t* start, float* out, cudaStream_t st);
 rap_status rap_launch_pack_wo(rap_ctx* ctx, int32_t layer, const void* wo, const int32_t* v_idx, void* dst, cudaStream_t st);
 rap_status rap_launch_out_proj(rap_ctx* ctx, int32_t layer, int32_t T, const float* attn_out, const void* wo_tilde,
                                void* y, cudaStream_t st);

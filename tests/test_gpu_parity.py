@@ -417,3 +417,27 @@ def test_decode_step_replays_from_a_cuda_graph():
     assert st.seq_len.cpu().tolist() == [302, 125]
     assert st.ctx.rap_get_last_device_status() == (0, 0)
     st.close()
+
+
+@pytest.mark.parametrize("name,T,starts", [("8b", 150, [0, 37]), ("3b", 100, [5, 0]), ("14b", 70, [64, 1]),
+                                           ("sweep1.0", 130, [0, 200]), ("sweep0.8", 65, [63, 0]), ("sweep0.5", 128, [0, 128])])
+def test_prefill_attn_matches_oracle(name, T, starts):
+    """rap_prefill_attn (tensor-core causal block attention on the reduced dims) against the oracle's masked
+    matrix form on the same bf16 caches and q~: several query blocks, ragged starts, tile-boundary lengths."""
+    w = synth.scaled_down(synth.CONFIGS[name], n_layers=1, batch=len(starts), seq=max(starts) + T)
+    st = DecodeStack(w, s_cap=((max(starts) + T + 8 + 7) // 8) * 8)
+    st.build_tables(*synth.draw_scores(w))
+    g = torch.Generator(device=st.device).manual_seed(T)
+    sig = float(np.sqrt(w.hidden) * 0.02)
+    st.k_cache[0].normal_(0, sig, generator=g)
+    st.v_cache[0].normal_(0, sig, generator=g)
+    B, Hq, P2, dv = w.batch, w.n_q_heads, 2 * w.n_pairs, w.n_vch
+    q = torch.empty((B, T, Hq, P2), dtype=st.dt, device=st.device).normal_(0, sig, generator=g)
+    ds = torch.tensor(starts, dtype=torch.int32, device=st.device)
+    out = torch.full((B, T, Hq, dv), float("nan"), dtype=torch.float32, device=st.device)
+    st.ctx.rap_prefill_attn(0, B, T, q, st.k_cache[0], st.v_cache[0], st.s_cap, ds, max(starts), out)
+    torch.cuda.synchronize()
+    want = O.prefill_attn(util.to_np64(q), util.to_np64(st.k_cache[0]), util.to_np64(st.v_cache[0]), starts, w.head_dim)
+    util.check_attn(util.to_np64(out).reshape(B * T, Hq, dv), want.reshape(B * T, Hq, dv), w.dtype)
+    assert st.ctx.rap_get_last_device_status() == (0, 0)
+    st.close()
