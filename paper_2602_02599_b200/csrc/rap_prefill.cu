@@ -39,6 +39,11 @@ __device__ __forceinline__ void mma16816(float (&c)[4], const uint32_t (&a)[4], 
       : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
       : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
+__device__ __forceinline__ float pf_ex2(float x) {      // 2^x, one instruction; 2^(-inf) = 0
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
 __device__ __forceinline__ uint32_t pf_pack(float lo, float hi) {
   const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
   return *reinterpret_cast<const uint32_t*>(&v);
@@ -86,21 +91,20 @@ __global__ void __launch_bounds__(PF_THREADS) prefill_attn_kernel(const PfParams
     const int j0 = tile * PF_BN;
     __nv_bfloat16* kd = ks + buf * K_TILE;
     __nv_bfloat16* vd = vs + buf * V_TILE;
-    for (int i = tid; i < PF_BN * kw; i += PF_THREADS) {
-      const int r = i / kw, w = i - r * kw;
+    // one row per warp and pass, lanes over the row's 4-byte words: no index divisions in the copy loop
+    for (int r = warp; r < PF_BN; r += PF_THREADS / 32) {
       const bool ok = j0 + r < n_valid;
-      cp_async4(pf_smem(kd + r * KSTR + 2 * w), kg + (size_t)(ok ? j0 + r : 0) * p.P2 + 2 * w, ok ? 4 : 0);
-    }
-    if (!v_odd) {
-      for (int i = tid; i < PF_BN * vw; i += PF_THREADS) {
-        const int r = i / vw, w = i - r * vw;
-        const bool ok = j0 + r < n_valid;
-        cp_async4(pf_smem(vd + r * VSTR + 2 * w), vg + (size_t)(ok ? j0 + r : 0) * p.dv + 2 * w, ok ? 4 : 0);
-      }
-    } else {   // rows are only 2-byte aligned: element-wise staging
-      for (int i = tid; i < PF_BN * p.dv; i += PF_THREADS) {
-        const int r = i / p.dv, c = i - r * p.dv;
-        vd[r * VSTR + c] = j0 + r < n_valid ? vg[(size_t)(j0 + r) * p.dv + c] : __float2bfloat16(0.f);
+      const int bytes = ok ? 4 : 0;
+      const __nv_bfloat16* ksrc = kg + (size_t)(ok ? j0 + r : 0) * p.P2;
+      const uint32_t kdst = pf_smem(kd + r * KSTR);
+      for (int w = lane; w < kw; w += 32) cp_async4(kdst + 4 * w, ksrc + 2 * w, bytes);
+      if (!v_odd) {
+        const __nv_bfloat16* vsrc = vg + (size_t)(ok ? j0 + r : 0) * p.dv;
+        const uint32_t vdst = pf_smem(vd + r * VSTR);
+        for (int w = lane; w < vw; w += 32) cp_async4(vdst + 4 * w, vsrc + 2 * w, bytes);
+      } else {   // rows are only 2-byte aligned: element-wise staging
+        const __nv_bfloat16* vsrc = vg + (size_t)(j0 + r) * p.dv;
+        for (int c = lane; c < p.dv; c += 32) vd[r * VSTR + c] = ok ? vsrc[c] : __float2bfloat16(0.f);
       }
     }
     cp_commit();
@@ -163,15 +167,27 @@ __global__ void __launch_bounds__(PF_THREADS) prefill_attn_kernel(const PfParams
     // ---- scale, causal mask, online softmax (rows gid and gid + 8 of the warp's 16) -------------------
     const int j0 = tile * PF_BN;
     float mx0 = -INFINITY, mx1 = -INFINITY;
+    const bool diagonal = j0 + PF_BN - 1 > start + q0 + 16 * warp;   // some key of the tile lies past this warp's first query
+    if (diagonal) {
 #pragma unroll
-    for (int n = 0; n < 8; ++n) {
+      for (int n = 0; n < 8; ++n) {
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const int key = j0 + 8 * n + 2 * tq + (e & 1);
-        const int pos = (e < 2) ? pos0 : pos1;
-        const float v = key <= pos ? s[n][e] * p.qscale : -INFINITY;
-        s[n][e] = v;
-        if (e < 2) mx0 = fmaxf(mx0, v); else mx1 = fmaxf(mx1, v);
+        for (int e = 0; e < 4; ++e) {
+          const int key = j0 + 8 * n + 2 * tq + (e & 1);
+          const int pos = (e < 2) ? pos0 : pos1;
+          const float v = key <= pos ? s[n][e] * p.qscale : -INFINITY;
+          s[n][e] = v;
+          if (e < 2) mx0 = fmaxf(mx0, v); else mx1 = fmaxf(mx1, v);
+        }
+      }
+    } else {
+#pragma unroll
+      for (int n = 0; n < 8; ++n) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          s[n][e] *= p.qscale;
+          if (e < 2) mx0 = fmaxf(mx0, s[n][e]); else mx1 = fmaxf(mx1, s[n][e]);
+        }
       }
     }
     mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
@@ -181,14 +197,14 @@ __global__ void __launch_bounds__(PF_THREADS) prefill_attn_kernel(const PfParams
     const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);
     // a row that has seen no allowed key yet keeps m = -inf: use 0 as its reference so that 2^(-inf - 0) = 0
     const float r0 = mn0 == -INFINITY ? 0.f : mn0, r1 = mn1 == -INFINITY ? 0.f : mn1;
-    const float a0 = exp2f(m0 - r0), a1 = exp2f(m1 - r1);
+    const float a0 = pf_ex2(m0 - r0), a1 = pf_ex2(m1 - r1);
     m0 = mn0; m1 = mn1;
     float sum0 = 0.f, sum1 = 0.f;
     uint32_t pa[4][4];                         // P as A fragments: k-step kk covers keys 16kk .. 16kk+15
 #pragma unroll
     for (int n = 0; n < 8; ++n) {
-      const float p00 = exp2f(s[n][0] - r0), p01 = exp2f(s[n][1] - r0);
-      const float p10 = exp2f(s[n][2] - r1), p11 = exp2f(s[n][3] - r1);
+      const float p00 = pf_ex2(s[n][0] - r0), p01 = pf_ex2(s[n][1] - r0);
+      const float p10 = pf_ex2(s[n][2] - r1), p11 = pf_ex2(s[n][3] - r1);
       sum0 += p00 + p01;
       sum1 += p10 + p11;
       pa[n >> 1][(n & 1) * 2 + 0] = pf_pack(p00, p01);
