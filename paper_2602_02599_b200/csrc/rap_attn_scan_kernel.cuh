@@ -72,6 +72,11 @@ struct ScanCfg {
   static constexpr bool VODD = (DV & 1) != 0;
   static constexpr int WVP = (DV + 1) / 2;                     // channel pairs per V row
   static constexpr int NG = (STHREADS / WVP) > ST ? ST : (STHREADS / WVP);   // PV row groups
+  // Odd d_v': rows are 2-byte aligned, but with an even number of row groups every thread only meets rows
+  // of one parity, and the aligned 32-bit word w of such a row holds channels (2w, 2w+1) for even rows and
+  // (2w-1, 2w) for odd rows -- same word loads as for even d_v', the channel shift is applied once, when
+  // the row groups are reduced.  (The half word that belongs to a neighbouring row is finite and dropped.)
+  static constexpr bool VWORD = !VODD || (NG % 2) == 0;
   static constexpr int RPG = (ST + NG - 1) / NG;               // rows per group (largest)
   static constexpr int LASTN = ST - (RPG - 1) * NG;            // groups that own a row in the last slot
   static constexpr int IP = (RPG + 1) / 2;                     // row pairs per group
@@ -476,11 +481,11 @@ __global__ void __launch_bounds__(STHREADS, 2) attn_scan_kernel(const ScanParams
         const bool okA = (iA < C::RPG - 1) || (iA == C::RPG - 1 && last_slot_ok);
         const bool okB = (iB < C::RPG - 1) || (iB == C::RPG - 1 && last_slot_ok);
         uint64_t lo, hi;
-        if constexpr (!C::VODD) {
-          constexpr int WV = DV / 2;
-          const uint32_t* pa = reinterpret_cast<const uint32_t*>(vt) + grp * WV + wch;
-          const uint32_t xa = okA ? pa[iA * C::NG * WV] : 0u;
-          const uint32_t xb = okB ? pa[iB * C::NG * WV] : 0u;
+        if constexpr (C::VWORD) {
+          constexpr int SLOT_WORDS = C::NG * DV / 2;      // words between a group's consecutive rows (NG * DV is even)
+          const uint32_t* pa = reinterpret_cast<const uint32_t*>(vt) + ((grp * DV) >> 1) + wch;
+          const uint32_t xa = okA ? pa[iA * SLOT_WORDS] : 0u;
+          const uint32_t xb = okB ? pa[iB * SLOT_WORDS] : 0u;
           lo = pack2u(xa << 16, xb << 16);
           hi = pack2u(xa & 0xffff0000u, xb & 0xffff0000u);
         } else {
@@ -530,11 +535,12 @@ __global__ void __launch_bounds__(STHREADS, 2) attn_scan_kernel(const ScanParams
   if (pv_active) {
 #pragma unroll
     for (int g = 0; g < G; ++g) {
+      const int ch = 2 * wch - ((C::VODD && C::VWORD) ? (grp & 1) : 0);   // odd rows of an odd d_v': shifted pairs
       float a, c;
       unpack2(accLo[g], a, c);
-      red[(grp * G + g) * DVP + 2 * wch] = a + c;
+      if (ch >= 0) red[(grp * G + g) * DVP + ch] = a + c;
       unpack2(accHi[g], a, c);
-      red[(grp * G + g) * DVP + 2 * wch + 1] = a + c;
+      red[(grp * G + g) * DVP + ch + 1] = a + c;
     }
   }
   __syncthreads();
