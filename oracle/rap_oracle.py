@@ -76,6 +76,30 @@ def bf16_bits(x):
     return (a.view(np.uint32) >> np.uint32(16)).astype(np.uint16)
 
 
+def build_tables_hybrid(k_pair_scores, k_chan_scores, v_chan_scores, rope_layer, n_pairs, n_vch, head_dim,
+                        rope_theta, pairing):
+    """Tables of a model whose layers are not all rotary (Section 4, "Hybrid compression": RAP where
+    RoPE is used, plain channel pruning of K elsewhere).
+
+    rope_layer[l] != 0: as build_tables.  rope_layer[l] == 0 (no positional rotation in that layer):
+    K keeps the 2 * n_pairs[l] channels with the largest k_chan_scores [L][H_kv][D], ascending, no pair
+    structure (k_pair_idx stays -1), and the frequency row is zero, i.e. the rotation of the shared
+    online path is the identity for that layer."""
+    tabs = build_tables(k_pair_scores, v_chan_scores, n_pairs, n_vch, head_dim, rope_theta, pairing)
+    kc = np.asarray(k_chan_scores, dtype=np.float64)
+    L, H, D = kc.shape
+    for l in range(L):
+        if rope_layer[l]:
+            continue
+        n = 2 * int(n_pairs[l])
+        for h in range(H):
+            tabs["k_pair_idx"][l, h, :] = -1
+            tabs["k_dim_idx"][l, h, :] = -1
+            tabs["k_dim_idx"][l, h, :n] = top_k_ascending(kc[l, h], n)
+            tabs["inv_freq"][l, h, :] = 0.0
+    return tabs
+
+
 # --------------------------------------------------------------------------------------
 # O1  tables  (Algorithm 2 selection lines; Eq. 6 RAPIndex; Eq. 3 frequencies)
 # --------------------------------------------------------------------------------------

@@ -29,7 +29,7 @@ def _small(pairing=O.PAIR_HALF, rho=0.75, D=16, Hq=4, Hkv=2, hidden=24, n=7, see
     Wv = rng.normal(0, 0.3, (Hkv * D, hidden))
     X = rng.normal(0, 1, (n, hidden))
     return dict(P=P, dv=dv, tabs=tabs, Wq=Wq, Wk=Wk, Wv=Wv, X=X, D=D, Hq=Hq, Hkv=Hkv,
-                pairing=pairing, theta=10000.0)
+                pairing=pairing, theta=10000.0, ks=ks, vs=vs)
 
 
 def _reduced(m, layer=0, **kw):
@@ -416,3 +416,40 @@ def test_prefill_attn_equals_per_token_decode_attention():
     V2[:, :, 6:, :] -= 3.0
     got2 = O.prefill_attn(q, K2, V2, start, D)
     assert np.array_equal(got2[0, :3], got[0, :3]) and not np.allclose(got2[0, 3:], got[0, 3:])
+
+
+# ---- hybrid models: layers without RoPE are channel-pruned -------------------------------------------
+def test_nope_layer_tables_give_plain_channel_pruned_attention():
+    """In a layer without positional rotation the reduced path (zero frequencies, per-channel K selection)
+    equals full-width dot-product attention with the dropped K channels zeroed -- written out with loops."""
+    m = _small(rho=0.5, D=16, Hq=4, Hkv=2, n=6, seed=41)
+    D, Hq, Hkv, P, dv = m["D"], m["Hq"], m["Hkv"], m["P"], m["dv"]
+    rng = np.random.default_rng(3)
+    kc = rng.lognormal(0, 1, (1, Hkv, D))
+    tabs = O.build_tables_hybrid(m["ks"], kc, m["vs"], [0], [P], [dv], D, m["theta"], m["pairing"])
+    assert np.all(tabs["inv_freq"] == 0.0) and np.all(tabs["k_pair_idx"] == -1)
+    for h in range(Hkv):
+        want = np.sort(np.argsort(-kc[0, h], kind="stable")[: 2 * P])
+        assert np.array_equal(tabs["k_dim_idx"][0, h, : 2 * P], want)
+    w = O.gather_weights(m["Wq"], m["Wk"], m["Wv"], tabs, 0, P, dv, D)
+    got, _, _, _ = O.reduced_attention_from_hidden(m["X"], w, tabs["inv_freq"][0], Hq, Hkv, P, dv, D)
+    # full-width reference without any rotation
+    X, n, G = m["X"], m["X"].shape[0], Hq // Hkv
+    want = np.zeros((Hq, dv))
+    for g in range(Hq):
+        h = g // G
+        keep = set(int(i) for i in tabs["k_dim_idx"][0, h, : 2 * P])
+        q = m["Wq"][g * D:(g + 1) * D] @ X[-1]
+        s = np.empty(n)
+        for j in range(n):
+            k = m["Wk"][h * D:(h + 1) * D] @ X[j]
+            s[j] = sum(q[d] * k[d] for d in range(D) if d in keep) / math.sqrt(D)
+        pr = np.exp(s - s.max()); pr /= pr.sum()
+        for c in range(dv):
+            u = tabs["v_idx"][0, h, c]
+            want[g, c] = sum(pr[j] * float(m["Wv"][h * D + u] @ X[j]) for j in range(n))
+    assert np.allclose(got, want, rtol=0, atol=1e-12)
+    # a rotary layer of the same call is unchanged
+    t2 = O.build_tables_hybrid(np.concatenate([m["ks"], m["ks"]]), np.concatenate([kc, kc]), np.concatenate([m["vs"], m["vs"]]),
+                               [1, 0], [P, P], [dv, dv], D, m["theta"], m["pairing"])
+    assert np.array_equal(t2["k_dim_idx"][0], m["tabs"]["k_dim_idx"][0]) and np.array_equal(t2["inv_freq"][0], m["tabs"]["inv_freq"][0])
