@@ -114,6 +114,16 @@ rap_status rap_build_tables(rap_ctx* ctx, const double* h_k_pair_scores, const d
                             int32_t* d_k_pair_idx, int32_t* d_k_dim_idx, int32_t* d_v_idx,
                             double* d_inv_freq, void* stream);
 
+/* Tables of a hybrid model (Section 4, "Hybrid compression"): RAP on the layers that use RoPE, plain
+ * channel pruning of K on the layers that do not (h_rope_layer[l] == 0).  For such a layer K keeps the
+ * 2 * h_n_pairs[l] channels with the largest h_k_chan_scores [L][H_kv][D] (ascending, no pair structure:
+ * its d_k_pair_idx row stays -1) and its frequency row is zero, so the shared online path rotates by the
+ * identity there.  Everything else as rap_build_tables. */
+rap_status rap_build_tables_hybrid(rap_ctx* ctx, const double* h_k_pair_scores, const double* h_k_chan_scores,
+                                   const double* h_v_chan_scores, const int32_t* h_rope_layer,
+                                   const int32_t* h_n_pairs, const int32_t* h_n_vch, int32_t* d_k_pair_idx,
+                                   int32_t* d_k_dim_idx, int32_t* d_v_idx, double* d_inv_freq, void* stream);
+
 /* ---- a0. offline weight gather (Algorithm 1: W~_k, W~_q = W_q E_k^T, W~_v) ----------------
  * Index selection, no arithmetic.  d_wq [H_q*D][hidden], d_wk / d_wv [H_kv*D][hidden] are the
  * dense weights of `layer`; d_w_qkv [N_out][hidden] receives the rows

@@ -203,9 +203,11 @@ rap_status rap_destroy(rap_ctx* ctx) {
   return RAP_OK;
 }
 
-rap_status rap_build_tables(rap_ctx* ctx, const double* ks, const double* vs, const int32_t* n_pairs,
-                            const int32_t* n_vch, int32_t* d_k_pair_idx, int32_t* d_k_dim_idx,
-                            int32_t* d_v_idx, double* d_inv_freq, void* stream) {
+// kc / rope_layer are NULL for an all-rotary model
+static rap_status build_tables_impl(rap_ctx* ctx, const double* ks, const double* kc, const double* vs,
+                                    const int32_t* rope_layer, const int32_t* n_pairs, const int32_t* n_vch,
+                                    int32_t* d_k_pair_idx, int32_t* d_k_dim_idx, int32_t* d_v_idx, double* d_inv_freq,
+                                    void* stream) {
   if (!ctx || !ks || !vs || !n_pairs || !n_vch || !d_k_pair_idx || !d_k_dim_idx || !d_v_idx || !d_inv_freq)
     return RAP_EINVAL;
   if (!rap_aligned16(d_k_pair_idx) || !rap_aligned16(d_k_dim_idx) || !rap_aligned16(d_v_idx) ||
@@ -219,6 +221,7 @@ rap_status rap_build_tables(rap_ctx* ctx, const double* ks, const double* vs, co
   const size_t units = (size_t)L * H;
   for (size_t i = 0; i < units * half; ++i) if (std::isnan(ks[i])) return RAP_EINVAL;
   for (size_t i = 0; i < units * D; ++i) if (std::isnan(vs[i])) return RAP_EINVAL;
+  if (kc) for (size_t i = 0; i < units * D; ++i) if (std::isnan(kc[i])) return RAP_EINVAL;
   cudaStream_t st = (cudaStream_t)stream;
   if (ctx->tables_inflight) {
     RAP_CUDA_TRY(ctx, cudaStreamSynchronize((cudaStream_t)ctx->tables_stream));
@@ -246,6 +249,12 @@ rap_status rap_build_tables(rap_ctx* ctx, const double* ks, const double* vs, co
     const int P = n_pairs[l], dv = n_vch[l];
     for (int h = 0; h < H; ++h) {
       const size_t u = (size_t)l * H + h;
+      if (rope_layer && !rope_layer[l]) {
+        // no positional rotation in this layer: plain channel pruning of K, zero frequencies (identity rotation)
+        top_k(kc + u * D, D, 2 * P, h_dim + u * D);
+        top_k(vs + u * D, D, dv, h_v + u * D);
+        continue;
+      }
       int32_t* pr = h_pair + u * half;
       top_k(ks + u * half, half, P, pr);
       for (int c = 0; c < P; ++c) {
@@ -274,6 +283,22 @@ rap_status rap_build_tables(rap_ctx* ctx, const double* ks, const double* vs, co
   }
   ctx->tables_built = true;
   return RAP_OK;
+}
+
+rap_status rap_build_tables(rap_ctx* ctx, const double* ks, const double* vs, const int32_t* n_pairs,
+                            const int32_t* n_vch, int32_t* d_k_pair_idx, int32_t* d_k_dim_idx,
+                            int32_t* d_v_idx, double* d_inv_freq, void* stream) {
+  return build_tables_impl(ctx, ks, nullptr, vs, nullptr, n_pairs, n_vch, d_k_pair_idx, d_k_dim_idx, d_v_idx, d_inv_freq,
+                           stream);
+}
+
+rap_status rap_build_tables_hybrid(rap_ctx* ctx, const double* ks, const double* kc, const double* vs,
+                                   const int32_t* rope_layer, const int32_t* n_pairs, const int32_t* n_vch,
+                                   int32_t* d_k_pair_idx, int32_t* d_k_dim_idx, int32_t* d_v_idx, double* d_inv_freq,
+                                   void* stream) {
+  if (!kc || !rope_layer) return RAP_EINVAL;
+  return build_tables_impl(ctx, ks, kc, vs, rope_layer, n_pairs, n_vch, d_k_pair_idx, d_k_dim_idx, d_v_idx, d_inv_freq,
+                           stream);
 }
 
 rap_status rap_pack_weights(rap_ctx* ctx, int32_t layer, const void* d_wq, const void* d_wk, const void* d_wv,

@@ -441,3 +441,42 @@ def test_prefill_attn_matches_oracle(name, T, starts):
     util.check_attn(util.to_np64(out).reshape(B * T, Hq, dv), want.reshape(B * T, Hq, dv), w.dtype)
     assert st.ctx.rap_get_last_device_status() == (0, 0)
     st.close()
+
+
+def test_hybrid_tables_and_nope_layer_end_to_end():
+    """rap_build_tables_hybrid: layer 0 rotary, layer 1 without RoPE (channel-pruned K, zero frequencies).
+    Tables bit-exact against the oracle, then one decode step through the unchanged online path."""
+    w = synth.scaled_down(synth.LLAMA_8B, n_layers=2, batch=2, seq=200, hidden=256)
+    ks, vs = synth.draw_scores(w)
+    kc = np.random.default_rng(6).lognormal(0, 1, (2, w.n_kv_heads, w.head_dim))
+    rope_layer = [1, 0]
+    st = DecodeStack(w, max_rows=256)
+    st.ctx.rap_build_tables_hybrid(ks, kc, vs, rope_layer, st.n_pairs, st.n_vch, st.k_pair_idx, st.k_dim_idx, st.v_idx,
+                                   st.inv_freq)
+    tabs = O.build_tables_hybrid(ks, kc, vs, rope_layer, st.n_pairs, st.n_vch, w.head_dim, w.rope_theta, w.pairing)
+    _tables_equal(st, tabs)
+    P, dv, Hq, Hkv, B = w.n_pairs, w.n_vch, w.n_q_heads, w.n_kv_heads, w.batch
+    w_host = []
+    for l in range(2):
+        Wq, Wk, Wv = synth.draw_full_weights(w, l)
+        st.pack_from_full(l, Wq, Wk, Wv)
+        wr = [O.round_storage(a, w.dtype) for a in (Wq, Wk, Wv)]
+        w_host.append(O.gather_weights(wr[0], wr[1], wr[2], tabs, l, P, dv, w.head_dim))
+        assert np.array_equal(util.to_np64(st.w_qkv[l]), w_host[l])
+    lens = [200, 77]
+    caches = util.prefill_both(st, tabs, w_host, w, lens, chunk=256)
+    st.seq_len.copy_(torch.tensor(lens, dtype=torch.int32))
+    X = np.stack([synth.draw_hidden(w, l, 1, B) for l in range(2)])
+    dx = torch.from_numpy(X).to(st.device).to(st.dt).contiguous()
+    st.decode_step(dx, max(lens), advance=0)
+    torch.cuda.synchronize()
+    for l in range(2):
+        q, k, v = O.qkv_rope(O.round_storage(X[l], w.dtype), w_host[l], None, np.array(lens), tabs["inv_freq"][l], Hq, Hkv, P, dv)
+        Kd, Vd = util.to_np64(st.k_cache[l]), util.to_np64(st.v_cache[l])
+        k_dev = np.stack([Kd[b, :, lens[b], :] for b in range(B)])
+        util.check_projection(k_dev, O.round_storage(k, w.dtype), w.dtype, f"k layer {l}")
+        want = O.decode_attn(O.round_storage(q, w.dtype), Kd, Vd, np.array(lens) + 1, w.head_dim)
+        got = util.to_np64(st.out[l][: B * Hq * dv]).reshape(B, Hq, dv)
+        util.check_attn(got, want, w.dtype)
+    assert st.ctx.rap_get_last_device_status() == (0, 0)
+    st.close()
