@@ -10,7 +10,9 @@
 // Both operands are K-major, staged by TMA (cp.async.bulk.tensor.2d, 128-byte swizzle, no
 // multicast, OOB rows / columns read as zeros) into a ring of shared-memory stages.
 //
-// Roles inside one CTA of 192 threads:
+// The kernel is persistent (one CTA per SM walks a list of work items = row tile x token tile x reduction
+// split); the accumulator is double buffered in tensor memory so the epilogue of one item overlaps the
+// MMAs of the next.  Roles inside one CTA of 192 threads:
 //   warp 0   producer: one lane waits for a free stage, arms its mbarrier with the byte count
 //            and issues the two tensor copies (W tile 128 x 64, X tile TN x 64);
 //   warp 1   allocates TN tensor-memory columns; one lane waits for a full stage and issues four
@@ -44,8 +46,8 @@ struct TcCfg {
   static constexpr int STAGE = TC_A_BYTES + B_BYTES;            // multiples of 1024: descriptors need no base offset
   static constexpr int NS_RAW = TC_SMEM_TILES / STAGE;
   static constexpr int NS = NS_RAW > 8 ? 8 : NS_RAW;
-  static constexpr int OFF_BARS = NS * STAGE;                   // full[NS], empty[NS], accum, tmem slot
-  static constexpr int SMEM = OFF_BARS + (2 * NS + 2) * 8 + 1024;   // + slack to align the ring to 1024 bytes
+  static constexpr int OFF_BARS = NS * STAGE;                   // full[NS], empty[NS], acc_full[2], acc_empty[2], tmem slot
+  static constexpr int SMEM = OFF_BARS + (2 * NS + 5) * 8 + 1024;   // + slack to align the ring to 1024 bytes
   // instruction descriptor: fp32 accumulate, bf16 x bf16, both K-major, N = TN, M = 128
   static constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(TN >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
 };
@@ -116,8 +118,16 @@ struct TcParams {
   float* y;            // [ksplit][T][n_out]
   int32_t* status;
   int T, n_out, nkb_total, nkb_per_split;
+  int row_tiles, tok_tiles, n_work;     // work items = row tiles x token tiles x reduction splits
 };
 
+__device__ __forceinline__ void tc_mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+
+// Persistent: CTA c takes work items c, c + gridDim.x, ...  The stage ring runs on across items, and the
+// accumulator is double buffered in tensor memory (2 x TN columns) so that the epilogue of one item
+// overlaps the MMAs of the next.
 template <int TN>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 proj_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x, const TcParams p) {
@@ -126,24 +136,26 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
   // the swizzled tiles and their descriptors want a 1024-byte aligned ring
   unsigned char* smem = tc_smem_raw + ((1024u - (tc_smem_u32(tc_smem_raw) & 1023u)) & 1023u);
   const uint32_t ring = tc_smem_u32(smem);
-  const uint32_t full0 = ring + C::OFF_BARS, empty0 = full0 + 8 * C::NS, accum_bar = empty0 + 8 * C::NS;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + C::OFF_BARS + (2 * C::NS + 1) * 8);
+  const uint32_t full0 = ring + C::OFF_BARS, empty0 = full0 + 8 * C::NS;
+  const uint32_t acc_full0 = empty0 + 8 * C::NS, acc_empty0 = acc_full0 + 16;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + C::OFF_BARS + (2 * C::NS + 4) * 8);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int n0 = blockIdx.x * TC_BM, t0 = blockIdx.y * TN, ks = blockIdx.z;
-  const int kb0 = ks * p.nkb_per_split;
-  const int nkb = max(0, min(p.nkb_per_split, p.nkb_total - kb0));
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < C::NS; ++s) {
       tc_mbar_init(full0 + 8 * s, 1);
       tc_mbar_init(empty0 + 8 * s, 1);
     }
-    tc_mbar_init(accum_bar, 1);
+    for (int s = 0; s < 2; ++s) {
+      tc_mbar_init(acc_full0 + 8 * s, 1);
+      tc_mbar_init(acc_empty0 + 8 * s, 4);      // one arrival per epilogue warp
+    }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 1) {   // tensor-memory columns for the accumulator (power of two >= 32)
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tc_smem_u32(tmem_slot)), "r"(TN)
+  if (warp == 1) {   // tensor-memory columns for two accumulators (power of two >= 32)
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tc_smem_u32(tmem_slot)),
+                 "r"(2 * TN)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -153,61 +165,102 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
   const uint32_t tmem_d = *tmem_slot;
   bool timed_out = false;
 
+  // work item w -> (token tile, row tile, split); token tiles vary fastest so that the CTAs working at the
+  // same time share a weight tile through L2
+  auto decode = [&](int w, int& n0, int& t0, int& ks, int& kb0, int& nkb) {
+    const int tt = w % p.tok_tiles, rest = w / p.tok_tiles;
+    const int rt = rest % p.row_tiles;
+    ks = rest / p.row_tiles;
+    n0 = rt * TC_BM;
+    t0 = tt * TN;
+    kb0 = ks * p.nkb_per_split;
+    nkb = max(0, min(p.nkb_per_split, p.nkb_total - kb0));
+  };
+
   if (warp == 0) {
     if (lane == 0) {
-      for (int kb = 0; kb < nkb; ++kb) {
-        const int s = kb % C::NS;
-        const uint32_t ph = (uint32_t)(kb / C::NS) & 1u;
-        if (!tc_mbar_wait(empty0 + 8 * s, ph ^ 1u)) { timed_out = true; break; }   // first lap passes at once
-        const uint32_t a = ring + s * C::STAGE, b = a + TC_A_BYTES;
-        tc_mbar_expect_tx(full0 + 8 * s, C::STAGE);
-        tc_tma_load_2d(a, &map_w, (kb0 + kb) * TC_BK, n0, full0 + 8 * s);
-        tc_tma_load_2d(b, &map_x, (kb0 + kb) * TC_BK, t0, full0 + 8 * s);
+      uint32_t kbg = 0;      // k-blocks issued so far: position in the ring
+      for (int w = blockIdx.x; w < p.n_work && !timed_out; w += gridDim.x) {
+        int n0, t0, ks, kb0, nkb;
+        decode(w, n0, t0, ks, kb0, nkb);
+        for (int kb = 0; kb < nkb; ++kb, ++kbg) {
+          const uint32_t s = kbg % C::NS, ph = (kbg / C::NS) & 1u;
+          if (!tc_mbar_wait(empty0 + 8 * s, ph ^ 1u)) { timed_out = true; break; }   // first lap passes at once
+          const uint32_t a = ring + s * C::STAGE, b = a + TC_A_BYTES;
+          tc_mbar_expect_tx(full0 + 8 * s, C::STAGE);
+          tc_tma_load_2d(a, &map_w, (kb0 + kb) * TC_BK, n0, full0 + 8 * s);
+          tc_tma_load_2d(b, &map_x, (kb0 + kb) * TC_BK, t0, full0 + 8 * s);
+        }
       }
     }
   } else if (warp == 1) {
     if (lane == 0) {
-      for (int kb = 0; kb < nkb; ++kb) {
-        const int s = kb % C::NS;
-        const uint32_t ph = (uint32_t)(kb / C::NS) & 1u;
-        if (!tc_mbar_wait(full0 + 8 * s, ph)) { timed_out = true; break; }
+      uint32_t kbg = 0, it = 0;    // it: items with work so far -> accumulator buffer and its phase
+      for (int w = blockIdx.x; w < p.n_work && !timed_out; w += gridDim.x) {
+        int n0, t0, ks, kb0, nkb;
+        decode(w, n0, t0, ks, kb0, nkb);
+        if (nkb == 0) continue;
+        const uint32_t buf = it & 1u, use = it >> 1;
+        if (!tc_mbar_wait(acc_empty0 + 8 * buf, (use & 1u) ^ 1u)) { timed_out = true; break; }   // epilogue done with it
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const uint64_t adesc = tc_smem_desc(ring + s * C::STAGE);
-        const uint64_t bdesc = tc_smem_desc(ring + s * C::STAGE + TC_A_BYTES);
+        for (int kb = 0; kb < nkb; ++kb, ++kbg) {
+          const uint32_t s = kbg % C::NS, ph = (kbg / C::NS) & 1u;
+          if (!tc_mbar_wait(full0 + 8 * s, ph)) { timed_out = true; break; }
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          const uint64_t adesc = tc_smem_desc(ring + s * C::STAGE);
+          const uint64_t bdesc = tc_smem_desc(ring + s * C::STAGE + TC_A_BYTES);
 #pragma unroll
-        for (int kk = 0; kk < TC_BK / 16; ++kk)   // 16 bf16 = 32 bytes = 2 descriptor address units per step
-          tc_mma(tmem_d, adesc + 2 * kk, bdesc + 2 * kk, C::IDESC, (kb | kk) != 0 ? 1u : 0u);
-        tc_commit(empty0 + 8 * s);     // arrives when the MMAs above have read the stage
+          for (int kk = 0; kk < TC_BK / 16; ++kk)   // 16 bf16 = 32 bytes = 2 descriptor address units per step
+            tc_mma(tmem_d + buf * TN, adesc + 2 * kk, bdesc + 2 * kk, C::IDESC, (kb | kk) != 0 ? 1u : 0u);
+          tc_commit(empty0 + 8 * s);     // arrives when the MMAs above have read the stage
+        }
+        if (timed_out) break;
+        tc_commit(acc_full0 + 8 * buf);
+        ++it;
       }
-      if (!timed_out) tc_commit(accum_bar);
     }
   } else {
     // epilogue: this warp reads tensor-memory lanes 32 * (warp % 4) .. + 31 = weight rows of the tile
     const int quarter = warp & 3;
-    const int n = n0 + quarter * 32 + lane;
-    bool ready = true;
-    if (nkb > 0) {
-      ready = __all_sync(0xffffffffu, tc_mbar_wait(accum_bar, 0));
-      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    }
-    if (!ready) timed_out = true;
-    float* ybase = p.y + (size_t)ks * p.T * p.n_out;
-#pragma unroll 1
-    for (int c0 = 0; c0 < TN; c0 += 32) {
-      uint32_t r[32];
-      if (nkb > 0 && ready) {
-        tc_ld32(tmem_d + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c0, r);
-        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-      } else {
-#pragma unroll
-        for (int j = 0; j < 32; ++j) r[j] = 0u;
+    uint32_t it = 0;
+    for (int w = blockIdx.x; w < p.n_work; w += gridDim.x) {
+      int n0, t0, ks, kb0, nkb;
+      decode(w, n0, t0, ks, kb0, nkb);
+      const int n = n0 + quarter * 32 + lane;
+      const uint32_t buf = it & 1u, use = it >> 1;
+      bool ready = true;
+      if (nkb > 0) {
+        ready = __all_sync(0xffffffffu, !timed_out && tc_mbar_wait(acc_full0 + 8 * buf, use & 1u));
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        if (!ready) timed_out = true;
       }
-      if (n < p.n_out) {
+      float* ybase = p.y + (size_t)ks * p.T * p.n_out;
+#pragma unroll 1
+      for (int c0 = 0; c0 < TN; c0 += 32) {
+        if (t0 + c0 >= p.T) break;             // columns past the last token hold zero-filled rows
+        uint32_t r[32];
+        if (nkb > 0 && ready) {
+          tc_ld32(tmem_d + buf * TN + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c0, r);
+          asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        } else {
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
-          const int t = t0 + c0 + j;
-          if (t < p.T) ybase[(size_t)t * p.n_out + n] = __uint_as_float(r[j]);
+          for (int j = 0; j < 32; ++j) r[j] = 0u;
         }
+        if (n < p.n_out) {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            const int t = t0 + c0 + j;
+            if (t < p.T) ybase[(size_t)t * p.n_out + n] = __uint_as_float(r[j]);
+          }
+        }
+      }
+      if (nkb > 0) {
+        if (ready) {
+          asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+          __syncwarp();
+          if (lane == 0) tc_mbar_arrive(acc_empty0 + 8 * buf);    // this warp has drained the accumulator
+        }
+        ++it;
       }
     }
   }
@@ -219,7 +272,7 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
   __syncthreads();
   if (warp == 1) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"(TN) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"(2 * TN) : "memory");
   }
 }
 
@@ -303,7 +356,8 @@ rap_status rap_launch_gemm_tc(rap_ctx* ctx, const void* x, const void* w, int T,
   if ((size_t)ksplit * T * N * sizeof(float) > ctx->proj_ws_bytes) return RAP_EUNSUPPORTED;
   TcParams p;
   p.y = ctx->d_proj_ws; p.status = ctx->d_status; p.T = T; p.n_out = N; p.nkb_total = nkb; p.nkb_per_split = per;
-  dim3 grid(row_tiles, tok_tiles, ksplit);
+  p.row_tiles = row_tiles; p.tok_tiles = tok_tiles; p.n_work = row_tiles * tok_tiles * ksplit;
+  dim3 grid(p.n_work < ctx->sm_count ? p.n_work : ctx->sm_count, 1, 1);
   *ksplit_out = ksplit;
   switch (tn) {
     case 32: return launch_tc<32>(ctx, mw, mx, p, grid, st);
