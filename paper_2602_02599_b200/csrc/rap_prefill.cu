@@ -263,8 +263,15 @@ rap_status launch_prefill(rap_ctx* ctx, const PfParams& p, int B, cudaStream_t s
 
 }  // namespace
 
+rap_status rap_launch_prefill_attn_tc(rap_ctx* ctx, int B, int T, const void* q, const void* k, const void* v, int P2,
+                                      int dv, int S_cap, const int32_t* start, float* out, cudaStream_t st);
+
 rap_status rap_launch_prefill_attn(rap_ctx* ctx, int B, int T, const void* q, const void* k, const void* v, int P2,
                                    int dv, int S_cap, const int32_t* start, float* out, cudaStream_t st) {
+  if (ctx->attn_variant == 0) {   // tcgen05 kernel first; this file's mma.sync kernel is the fallback / cross-check
+    const rap_status s = rap_launch_prefill_attn_tc(ctx, B, T, q, k, v, P2, dv, S_cap, start, out, st);
+    if (s != RAP_EUNSUPPORTED) return s;
+  }
   const rap_model_desc& d = ctx->desc;
   if (d.dtype != RAP_BF16 || P2 > 128 || dv > 128) return RAP_EUNSUPPORTED;
   PfParams p;

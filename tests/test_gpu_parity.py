@@ -434,11 +434,13 @@ def test_prefill_attn_matches_oracle(name, T, starts):
     B, Hq, P2, dv = w.batch, w.n_q_heads, 2 * w.n_pairs, w.n_vch
     q = torch.empty((B, T, Hq, P2), dtype=st.dt, device=st.device).normal_(0, sig, generator=g)
     ds = torch.tensor(starts, dtype=torch.int32, device=st.device)
-    out = torch.full((B, T, Hq, dv), float("nan"), dtype=torch.float32, device=st.device)
-    st.ctx.rap_prefill_attn(0, B, T, q, st.k_cache[0], st.v_cache[0], st.s_cap, ds, max(starts), out)
-    torch.cuda.synchronize()
     want = O.prefill_attn(util.to_np64(q), util.to_np64(st.k_cache[0]), util.to_np64(st.v_cache[0]), starts, w.head_dim)
-    util.check_attn(util.to_np64(out).reshape(B * T, Hq, dv), want.reshape(B * T, Hq, dv), w.dtype)
+    for variant in (0, 1):       # 0: tcgen05 kernel, 1: warp-level mma.sync kernel
+        st.ctx.rap_set_attn_variant(variant)
+        out = torch.full((B, T, Hq, dv), float("nan"), dtype=torch.float32, device=st.device)
+        st.ctx.rap_prefill_attn(0, B, T, q, st.k_cache[0], st.v_cache[0], st.s_cap, ds, max(starts), out)
+        torch.cuda.synchronize()
+        util.check_attn(util.to_np64(out).reshape(B * T, Hq, dv), want.reshape(B * T, Hq, dv), w.dtype)
     assert st.ctx.rap_get_last_device_status() == (0, 0)
     st.close()
 
