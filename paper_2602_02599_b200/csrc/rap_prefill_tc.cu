@@ -94,15 +94,16 @@ struct PtParams {
 
 // DK = k-steps of Q K^T (ceil(2P / 16)); NVP = d_v' rounded up to a multiple of 32 (N of the second MMA)
 template <int DK, int NVP>
-__global__ void __launch_bounds__(PT_THREADS, 1) prefill_tc_kernel(const PtParams p) {
+__global__ void __launch_bounds__(PT_THREADS, 2) prefill_tc_kernel(const PtParams p) {
   extern __shared__ unsigned char pt_raw[];
   unsigned char* smem = pt_raw + ((1024u - (pt_smem(pt_raw) & 1023u)) & 1023u);
   unsigned char* q_s = smem;                         // [128 queries][<=128 dims]
   unsigned char* k_s = q_s + PT_TILE_BYTES;          // [128 keys][<=128 dims]
   unsigned char* v_s = k_s + PT_TILE_BYTES;          // [NVP channels][128 keys]   (V transposed)
-  unsigned char* p_s = v_s + PT_TILE_BYTES;          // [128 queries][128 keys]
-  const uint32_t bar_s = pt_smem(p_s + PT_TILE_BYTES), bar_o = bar_s + 8;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(p_s + PT_TILE_BYTES + 16);
+  unsigned char* p_s = k_s;                          // [128 queries][128 keys]: reuses the K tile, which the
+                                                     // first MMA has finished reading when P is written
+  const uint32_t bar_s = pt_smem(v_s + PT_TILE_BYTES), bar_o = bar_s + 8;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(v_s + PT_TILE_BYTES + 16);
 
   const int qb = blockIdx.x, g = blockIdx.y, b = blockIdx.z;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -126,7 +127,7 @@ __global__ void __launch_bounds__(PT_THREADS, 1) prefill_tc_kernel(const PtParam
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   // zero all four tiles once (pad columns and pad channel rows are never written again), then stage Q
-  for (int i = tid; i < 4 * PT_TILE_BYTES / 16; i += PT_THREADS) reinterpret_cast<uint4*>(smem)[i] = make_uint4(0, 0, 0, 0);
+  for (int i = tid; i < 3 * PT_TILE_BYTES / 16; i += PT_THREADS) reinterpret_cast<uint4*>(smem)[i] = make_uint4(0, 0, 0, 0);
   __syncthreads();
   const int kw = p.P2 >> 1;                          // 4-byte words per q / K row
   for (int r = warp; r < PT_BM; r += PT_THREADS / 32) {
@@ -155,15 +156,28 @@ __global__ void __launch_bounds__(PT_THREADS, 1) prefill_tc_kernel(const PtParam
   for (int tile = 0; tile < n_tiles; ++tile) {
     const int j0 = tile * PT_BN;
     // ---- stage K (as stored) and V (transposed); rows past the end become zeros ------------------------
+    // K: 4-byte cp.async straight to the swizzled position (zero fill past the end), all in flight at once;
+    // V: eight rows per pass so that eight independent loads are in flight before the transposed stores
     for (int r = warp; r < PT_BN; r += PT_THREADS / 32) {
       const bool ok = j0 + r < n_valid;
-      const uint32_t* ksrc = reinterpret_cast<const uint32_t*>(kg + (size_t)(ok ? j0 + r : 0) * p.P2);
+      const __nv_bfloat16* ksrc = kg + (size_t)(ok ? j0 + r : 0) * p.P2;
       for (int w = lane; w < kw; w += 32)
-        *reinterpret_cast<uint32_t*>(k_s + pt_off(r, 2 * w, PT_BN)) = ok ? ksrc[w] : 0u;
-      const __nv_bfloat16* vsrc = vg + (size_t)(ok ? j0 + r : 0) * p.dv;
-      for (int c = lane; c < p.dv; c += 32)
-        *reinterpret_cast<__nv_bfloat16*>(v_s + pt_off(c, r, NVP)) = ok ? vsrc[c] : __float2bfloat16(0.f);
+        asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(pt_smem(k_s + pt_off(r, 2 * w, PT_BN))),
+                     "l"(ksrc + 2 * w), "r"(ok ? 4 : 0)
+                     : "memory");
     }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+    for (int r0 = 8 * warp; r0 < PT_BN; r0 += 8 * (PT_THREADS / 32)) {
+      for (int c = lane; c < p.dv; c += 32) {
+        __nv_bfloat16 vals[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i)
+          vals[i] = j0 + r0 + i < n_valid ? vg[(size_t)(j0 + r0 + i) * p.dv + c] : __float2bfloat16(0.f);
+        // rows r0 .. r0+7 of channel c are one 16-byte chunk of the transposed tile
+        *reinterpret_cast<uint4*>(v_s + pt_off(c, r0, NVP)) = *reinterpret_cast<const uint4*>(vals);
+      }
+    }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> tensor-core (async proxy) reads
     __syncthreads();
     // ---- S = Q K^T ----------------------------------------------------------------------------------------
@@ -273,7 +287,7 @@ __global__ void __launch_bounds__(PT_THREADS, 1) prefill_tc_kernel(const PtParam
 
 template <int DK, int NVP>
 rap_status launch_pt(rap_ctx* ctx, const PtParams& p, int B, cudaStream_t st) {
-  const int smem = 4 * PT_TILE_BYTES + 64 + 1024;
+  const int smem = 3 * PT_TILE_BYTES + 64 + 1024;
   RAP_CUDA_TRY(ctx, rap_raise_smem(ctx, prefill_tc_kernel<DK, NVP>, smem));
   dim3 grid((p.T + PT_BM - 1) / PT_BM, p.Hq, B);
   prefill_tc_kernel<DK, NVP><<<grid, PT_THREADS, smem, st>>>(p);
