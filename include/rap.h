@@ -96,7 +96,7 @@ rap_status rap_budget_alloc(int32_t n_layers, int32_t n_kv_heads, int32_t head_d
 size_t rap_cache_elem_offset(int32_t n_kv_heads, int32_t S_cap, int32_t W, int32_t b, int32_t h,
                              int32_t pos, int32_t c);
 
-/* ---- a1. tables (Algorithm 2, selection lines; Eq. 6 RAPIndex; Eq. 3 frequencies) --------
+/* ---- a1. tables (Algorithm 2, selection step; Eq. 6 RAPIndex; Eq. 3 frequencies) --------
  * For every (layer l, KV head h): keep the n_pairs[l] RoPE pairs with the largest score and
  * the n_vch[l] V channels with the largest score (ties: lower index), each list ascending.
  *   h_k_pair_scores [L][H_kv][D/2], h_v_chan_scores [L][H_kv][D]  HOST fp64

@@ -101,7 +101,7 @@ def build_tables_hybrid(k_pair_scores, k_chan_scores, v_chan_scores, rope_layer,
 
 
 # --------------------------------------------------------------------------------------
-# O1  tables  (Algorithm 2 selection lines; Eq. 6 RAPIndex; Eq. 3 frequencies)
+# O1  tables  (Algorithm 2, selection step; Eq. 6 RAPIndex; Eq. 3 frequencies)
 # --------------------------------------------------------------------------------------
 def retained_counts(rho, head_dim):
     """Per-head budget at retain ratio rho: P whole pairs for K, d_v' channels for V.
@@ -178,7 +178,7 @@ def selection_matrix(index, width):
 
 
 # --------------------------------------------------------------------------------------
-# O2  weight gather  (Algorithm 1 construction lines: W~_k, W~_q = W_q E_k^T, W~_v)
+# O2  weight gather  (Algorithm 1, construction step: W~_k, W~_q = W_q E_k^T, W~_v)
 # --------------------------------------------------------------------------------------
 def gather_weights(Wq, Wk, Wv, tables, layer, n_pairs_l, n_vch_l, head_dim):
     """Build W~_qkv [N_out][hidden] for one layer from full [out][in] weights.

@@ -1,5 +1,5 @@
 // Host side of the C ABI: context life cycle, argument validation, table construction
-// (Algorithm 2 selection lines, Eq. 6, Eq. 3) and the per-layer decode loop.
+// (Algorithm 2, selection step, Eq. 6, Eq. 3) and the per-layer decode loop.
 #include <algorithm>
 #include <cmath>
 #include <cstring>

@@ -107,7 +107,7 @@ def _end_to_end(w, lens_before, n_split=0, with_bias=False, chunk=None, n_pairs=
         v_dev = np.stack([Vd[b, :, lens_before[b], :] for b in range(B)])
         util.check_projection(k_dev, O.round_storage(k, w.dtype), w.dtype, f"k layer {l}")
         util.check_projection(v_dev, O.round_storage(v, w.dtype), w.dtype, f"v layer {l}")
-        # attention judged on the device's own rounded q~ and cache rows (a2-a4 judged above)
+        # attention judged on the device's own rounded q~ and cache rows (projection, RoPE and append are checked above)
         # -> recompute q~ on the device into a separate buffer
         dq = torch.empty((B, Hq, 2 * P), dtype=st.dt, device=st.device)
         tmp_k, tmp_v = st.k_cache[l].clone(), st.v_cache[l].clone()
