@@ -96,7 +96,7 @@ rap_status rap_budget_alloc(int32_t n_layers, int32_t n_kv_heads, int32_t head_d
 size_t rap_cache_elem_offset(int32_t n_kv_heads, int32_t S_cap, int32_t W, int32_t b, int32_t h,
                              int32_t pos, int32_t c);
 
-/* ---- a1. tables (Algorithm 2, selection step; Eq. 6 RAPIndex; Eq. 3 frequencies) --------
+/* ---- tables (Algorithm 2, selection step; Eq. 6 RAPIndex; Eq. 3 frequencies) --------
  * For every (layer l, KV head h): keep the n_pairs[l] RoPE pairs with the largest score and
  * the n_vch[l] V channels with the largest score (ties: lower index), each list ascending.
  *   h_k_pair_scores [L][H_kv][D/2], h_v_chan_scores [L][H_kv][D]  HOST fp64
@@ -124,7 +124,7 @@ rap_status rap_build_tables_hybrid(rap_ctx* ctx, const double* h_k_pair_scores, 
                                    const int32_t* h_n_pairs, const int32_t* h_n_vch, int32_t* d_k_pair_idx,
                                    int32_t* d_k_dim_idx, int32_t* d_v_idx, double* d_inv_freq, void* stream);
 
-/* ---- a0. offline weight gather (Algorithm 1: W~_k, W~_q = W_q E_k^T, W~_v) ----------------
+/* ---- offline weight gather (Algorithm 1: W~_k, W~_q = W_q E_k^T, W~_v) ----------------
  * Index selection, no arithmetic.  d_wq [H_q*D][hidden], d_wk / d_wv [H_kv*D][hidden] are the
  * dense weights of `layer`; d_w_qkv [N_out][hidden] receives the rows
  *   q head g: RAPIndex of KV head g/G (2P rows) | k head h: RAPIndex of h | v head h: v_idx of h,
@@ -135,7 +135,7 @@ rap_status rap_pack_weights(rap_ctx* ctx, int32_t layer, const void* d_wq, const
                             void* d_w_qkv, const void* d_bq, const void* d_bk, const void* d_bv,
                             void* d_bias, void* stream);
 
-/* ---- a2-a4. pruned QKV projection + index-aware RoPE + append (Eq. 1, Eq. 3, Section 4) ---
+/* ---- pruned QKV projection + index-aware RoPE + append (Eq. 1, Eq. 3, Section 4) ---
  * T rows of hidden states.  Row r belongs to sequence d_seq_id[r] (0..B-1), sits at position
  * d_pos[r] and is written to cache row d_slot[r].  For every row:
  *   y = W~_qkv x (+ bias), fp32 accumulate;
@@ -152,7 +152,7 @@ rap_status rap_qkv_rope_append(rap_ctx* ctx, int32_t layer, int32_t T, const voi
                                const double* d_inv_freq, void* d_q_out, void* d_k_cache,
                                void* d_v_cache, int32_t B_cache, int32_t S_cap, void* stream);
 
-/* ---- a5. split-KV decode attention on the reduced dims (Eq. 2, Eq. 7, scale 1/sqrt(D)) ----
+/* ---- split-KV decode attention on the reduced dims (Eq. 2, Eq. 7, scale 1/sqrt(D)) ----
  * For each sequence b and query head g (KV head h = g/G):
  *   s_j = q~_g . K[b,h,j] / sqrt(D),  j in [0, d_seq_len[b]);  p = softmax(s);
  *   out[b,g,:] = sum_j p_j V[b,h,j,:].
@@ -215,7 +215,7 @@ rap_status rap_pack_wo(rap_ctx* ctx, int32_t layer, const void* d_wo, const int3
 rap_status rap_out_proj(rap_ctx* ctx, int32_t layer, int32_t T, const float* d_attn_out, const void* d_wo_tilde,
                         void* d_y, void* stream);
 
-/* ---- one decode step over all layers (a2-a5 per layer) -------------------------------------
+/* ---- one decode step over all layers (projection + RoPE + append, then attention, per layer) -------------------------------------
  * Layer l consumes d_x + l*B*hidden (one hidden-state row per sequence) and produces
  * d_out + l*out_layer_stride ([B][H_q][d_v'_l] fp32).  d_seq_len[b] = rows cached BEFORE the
  * step: the new token takes position = slot = d_seq_len[b] and attends over d_seq_len[b]+1

@@ -101,7 +101,7 @@ def build_tables_hybrid(k_pair_scores, k_chan_scores, v_chan_scores, rope_layer,
 
 
 # --------------------------------------------------------------------------------------
-# O1  tables  (Algorithm 2, selection step; Eq. 6 RAPIndex; Eq. 3 frequencies)
+# Tables  (Algorithm 2, selection step; Eq. 6 RAPIndex; Eq. 3 frequencies)
 # --------------------------------------------------------------------------------------
 def retained_counts(rho, head_dim):
     """Per-head budget at retain ratio rho: P whole pairs for K, d_v' channels for V.
@@ -178,7 +178,7 @@ def selection_matrix(index, width):
 
 
 # --------------------------------------------------------------------------------------
-# O2  weight gather  (Algorithm 1, construction step: W~_k, W~_q = W_q E_k^T, W~_v)
+# Weight gather  (Algorithm 1, construction step: W~_k, W~_q = W_q E_k^T, W~_v)
 # --------------------------------------------------------------------------------------
 def gather_weights(Wq, Wk, Wv, tables, layer, n_pairs_l, n_vch_l, head_dim):
     """Build W~_qkv [N_out][hidden] for one layer from full [out][in] weights.
@@ -204,7 +204,7 @@ def gather_weights(Wq, Wk, Wv, tables, layer, n_pairs_l, n_vch_l, head_dim):
 
 
 # --------------------------------------------------------------------------------------
-# O3  projection (Eq. 1 on the reduced widths)   O4  index-aware RoPE (Eq. 3)
+# Projection (Eq. 1 on the reduced widths), then index-aware RoPE (Eq. 3)
 # --------------------------------------------------------------------------------------
 def project(x, w_qkv, bias=None):
     """y[t] = W~_qkv x[t] (+ bias): x [T][hidden], w_qkv [N_out][hidden] -> [T][N_out], fp64."""
@@ -231,7 +231,7 @@ def rope_reduced(vec, pos, inv_freq):
 
 
 def qkv_rope(x, w_qkv, bias, pos, inv_freq_l, Hq, Hkv, P, dv):
-    """O3 + O4 for T rows: returns unrounded fp64 (q [T][Hq][2P], k [T][Hkv][2P], v [T][Hkv][dv]).
+    """Projection and index-aware RoPE for T rows: returns unrounded fp64 (q [T][Hq][2P], k [T][Hkv][2P], v [T][Hkv][dv]).
 
     inv_freq_l: [H_kv][>=P] table of this layer; q head g uses KV head g // G's entries.
     """
@@ -255,7 +255,7 @@ def qkv_rope(x, w_qkv, bias, pos, inv_freq_l, Hq, Hkv, P, dv):
 
 
 # --------------------------------------------------------------------------------------
-# O5  append   O6  attention (Eq. 2 on the reduced dims, Eq. 7, scale 1/sqrt(D))
+# Append, then attention (Eq. 2 on the reduced dims, Eq. 7, scale 1/sqrt(D))
 # --------------------------------------------------------------------------------------
 def append(k_cache, v_cache, k_new, v_new, seq_id, slot, dtype):
     """Write rounded k/v rows into caches [B][H_kv][S_cap][W]; returns nothing.
@@ -413,7 +413,7 @@ def reduced_attention_from_hidden(X_hist, w_qkv, inv_freq_l, Hq, Hkv, P, dv, hea
                                   dtype=None, bias=None):
     """(R) end to end for one sequence: tokens X_hist at positions 0..n-1, query = last.
 
-    Builds the cache the real way (O3-O5 for every token) and runs O6.  dtype=None keeps
+    Builds the cache the real way (projection, RoPE and append for every token) and runs the attention.  dtype=None keeps
     everything in fp64 (used by the identity pins); 'bf16'/'f32' rounds q, k, v once.
     Returns (out [H_q][d_v'], q [H_q][2P], K [H_kv][n][2P], V [H_kv][n][d_v']).
     """

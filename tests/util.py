@@ -70,7 +70,7 @@ def build_small_stack(w, ks, vs, full_weights=True, s_cap=None, max_rows=None, n
 
 def prefill_both(st, tabs, w_host, w, lens, step_tag=0, chunk=None):
     """Fill the caches the real way on both sides: every sequence b gets lens[b] tokens at positions
-    0..lens[b]-1 through rap_qkv_rope_append (device) and O3-O5 (oracle).  Returns oracle caches
+    0..lens[b]-1 through rap_qkv_rope_append (device) and the projection, RoPE and append steps of the oracle.  Returns oracle caches
     (list per layer of (K, V) fp64 arrays [B][H_kv][S_cap][W])."""
     B = st.B
     rows = [(b, p) for b in range(B) for p in range(int(lens[b]))]
