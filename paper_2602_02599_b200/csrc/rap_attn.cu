@@ -16,6 +16,7 @@
 
 rap_status rap_launch_attn_fast(rap_ctx* ctx, const rap_attn_args& a, int n_split, cudaStream_t st);
 rap_status rap_launch_attn_scan(rap_ctx* ctx, const rap_attn_args& a, int n_split, cudaStream_t st);
+rap_status rap_launch_attn_mma(rap_ctx* ctx, const rap_attn_args& a, int n_split, cudaStream_t st);
 
 namespace {
 
@@ -175,8 +176,13 @@ static int choose_split(const rap_ctx* ctx, const rap_attn_args& a, int tile, in
 rap_status rap_launch_attn(rap_ctx* ctx, const rap_attn_args& a, cudaStream_t st) {
   const int G = a.Hq / a.Hkv;
   if (a.dtype == RAP_BF16 && ctx->attn_variant != 1) {
-    // shape-specialised scan, then the shape-generic bf16 scan, then the fully generic kernel
+    // shape-specialised scans (mma.sync, then FP32 pipes), then the shape-generic bf16 scan, then the fully
+    // generic kernel
     if (ctx->attn_variant == 0) {
+      const rap_status s = rap_launch_attn_mma(ctx, a, a.n_split, st);
+      if (s != RAP_EUNSUPPORTED) return s;
+    }
+    if (ctx->attn_variant == 0 || ctx->attn_variant == 3) {
       const rap_status s = rap_launch_attn_scan(ctx, a, a.n_split, st);
       if (s != RAP_EUNSUPPORTED) return s;
     }

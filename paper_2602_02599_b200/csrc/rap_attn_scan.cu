@@ -1,8 +1,9 @@
-// Launch side of the shape-specialised split-KV scan: kernel lookup by head shape, the balanced /
-// equal-split launch and the combine kernel of the equal-split mode.  The scan kernel template lives in
-// rap_attn_scan_kernel.cuh; its instantiations (one per supported (G, P, d_v')) are generated into
-// several translation units at build time (build.py) and found through rap_scan_find.
-#include "rap_attn_scan_kernel.cuh"
+// Launch side of the shape-specialised split-KV scans: kernel lookup by head shape, the balanced /
+// equal-split launch and the combine kernel of the equal-split mode.  The kernel templates live in
+// rap_attn_scan_kernel.cuh (FP32 pipes) and rap_attn_mma_kernel.cuh (mma.sync); their instantiations (one
+// per supported (G, P, d_v')) are generated into several translation units at build time (build.py) and
+// found through rap_scan_find / rap_mma_find.
+#include "rap_attn_common.cuh"
 
 namespace {
 
@@ -59,11 +60,8 @@ __global__ void __launch_bounds__(128) attn_scan_combine_kernel(const float* __r
 
 }  // namespace
 
-rap_status rap_launch_attn_scan(rap_ctx* ctx, const rap_attn_args& a, int n_split_req, cudaStream_t st) {
-  if (a.dtype != RAP_BF16 || (a.P2 & 1)) return RAP_EUNSUPPORTED;
-  const int G = a.Hq / a.Hkv, WK = a.P2 / 2;
-  const rap_scan_entry* e = rap_scan_find(G, WK, a.dv);
-  if (!e) return RAP_EUNSUPPORTED;
+static rap_status launch_split_kv(rap_ctx* ctx, const rap_attn_args& a, int n_split_req, cudaStream_t st,
+                                  const rap_scan_entry* e) {
   // n_split = 0: balanced mode, one CTA per resident slot; an explicit n_split keeps equal ranges per split
   const bool balanced = n_split_req <= 0 && (long long)a.B * a.Hkv * ((a.S_cap + 63) / 64) < (1LL << 31);
   int n_split = balanced ? RAP_MAX_SPLIT : n_split_req;
@@ -83,7 +81,7 @@ rap_status rap_launch_attn_scan(rap_ctx* ctx, const rap_attn_args& a, int n_spli
   dim3 grid(n_split, a.Hkv, a.B);
   if (balanced) grid = dim3(scan_grid, 1, 1);
   void* args[] = {&p};
-  RAP_CUDA_TRY(ctx, cudaLaunchKernel(e->fn, grid, dim3(STHREADS), args, (size_t)e->smem, st));
+  RAP_CUDA_TRY(ctx, cudaLaunchKernel(e->fn, grid, dim3(e->threads), args, (size_t)e->smem, st));
   ctx->launches++;
   RAP_CUDA_TRY(ctx, cudaGetLastError());
   if (balanced) {
@@ -94,4 +92,16 @@ rap_status rap_launch_attn_scan(rap_ctx* ctx, const rap_attn_args& a, int n_spli
   ctx->launches++;
   RAP_CUDA_TRY(ctx, cudaGetLastError());
   return RAP_OK;
+}
+
+rap_status rap_launch_attn_scan(rap_ctx* ctx, const rap_attn_args& a, int n_split_req, cudaStream_t st) {
+  if (a.dtype != RAP_BF16 || (a.P2 & 1)) return RAP_EUNSUPPORTED;
+  const rap_scan_entry* e = rap_scan_find(a.Hq / a.Hkv, a.P2 / 2, a.dv);
+  return e ? launch_split_kv(ctx, a, n_split_req, st, e) : RAP_EUNSUPPORTED;
+}
+
+rap_status rap_launch_attn_mma(rap_ctx* ctx, const rap_attn_args& a, int n_split_req, cudaStream_t st) {
+  if (a.dtype != RAP_BF16 || (a.P2 & 1)) return RAP_EUNSUPPORTED;
+  const rap_scan_entry* e = rap_mma_find(a.Hq / a.Hkv, a.P2 / 2, a.dv);
+  return e ? launch_split_kv(ctx, a, n_split_req, st, e) : RAP_EUNSUPPORTED;
 }

@@ -24,19 +24,13 @@
 //   * partials (acc[d_v'], m, l) of the split go to the workspace; a combine kernel merges.
 // Every mbarrier wait is bounded: on timeout the CTA records RAP_ETIMEOUT and leaves.
 #pragma once
-#include <math.h>
-
-#include "rap_internal.h"
+#include "rap_attn_common.cuh"
 
 namespace {
 
 constexpr int STHREADS = 256;
 constexpr int SCHUNKS = 8;       // dim chunks of the logits phase (= warps)
-constexpr uint32_t WAIT_LIMIT = 1u << 21;
-constexpr int SMEM_BUDGET = 115712;   // two CTAs per SM
 constexpr float LAZY_MAX_SLACK = 8.f;
-
-constexpr int cround(int x, int m) { return (x + m - 1) / m * m; }
 
 // positions per tile: the largest multiple of 32 (up to 192) whose two-stage ring fits beside the
 // partial-logit and p buffers of a CTA (two CTAs per SM).  Large tiles spread the per-tile costs
@@ -95,45 +89,6 @@ struct ScanCfg {
   static_assert(NG * 2 * WVP * G <= SCHUNKS * SPS, "row-group reduction reuses the partial-logit buffer");
 };
 
-using ScanParams = rap_scan_params;
-
-// Balanced mode.  All tiles of all (sequence, KV head) units form one sequence, unit-major, of T
-// tiles; CTA c of NC scans the tiles [c T / NC, (c + 1) T / NC), whatever units they belong to, so
-// every CTA does the same amount of work for any batch, length mix and SM count.  A unit touched by
-// several CTAs gets one partial per CTA ("segment"); segment index = CTA - first CTA of the unit.
-// NC is capped so that no unit has more than RAP_MAX_SPLIT segments.  The scan and the combine
-// kernel derive the same plan from seq_len with the helpers below.
-struct SkPlan {
-  int T;           // total tiles (the host side keeps B * H_kv * S_cap / 64 below 2^31)
-  int nc;          // CTAs that take part (<= gridDim.x)
-};
-__device__ __forceinline__ int sk_tiles_of(const int32_t* seq_len, int b, int len_add, int S_cap, int tile_rows) {
-  const int len = min(max(seq_len[b] + len_add, 0), S_cap);
-  return (len + tile_rows - 1) / tile_rows;
-}
-__device__ __forceinline__ SkPlan sk_plan(const int32_t* seq_len, int B, int Hkv, int len_add, int S_cap, int tile_rows,
-                                          int grid) {
-  long long T = 0;
-  int n_max = 0;
-  for (int b = 0; b < B; ++b) {
-    const int n = sk_tiles_of(seq_len, b, len_add, S_cap, tile_rows);
-    T += (long long)n * Hkv;
-    n_max = max(n_max, n);
-  }
-  SkPlan pl;
-  pl.T = (int)T;
-  pl.nc = 0;
-  if (T > 0) {
-    const long long cap = (long long)(RAP_MAX_SPLIT - 2) * T / n_max;     // segments per unit <= n_max NC / T + 2
-    pl.nc = (int)max(1LL, min(min((long long)grid, cap), T));             // and every CTA owns at least one tile
-  }
-  return pl;
-}
-// first CTA whose range holds global tile s:  max c with floor(c T / NC) <= s
-__device__ __forceinline__ int sk_cta_of(int s, const SkPlan& pl) { return (int)((((long long)s + 1) * pl.nc - 1) / pl.T); }
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
 __device__ __forceinline__ uint64_t pack2(float lo, float hi) {
   uint64_t r;
   asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
@@ -157,40 +112,6 @@ __device__ __forceinline__ uint64_t fmul2(uint64_t a, uint64_t b) {
   uint64_t d;
   asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
   return d;
-}
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity) {
-  for (uint32_t i = 0; i < WAIT_LIMIT; ++i)
-    if (mbar_try_wait(bar, parity)) return true;
-  return false;
-}
-// the copy is normally ahead of the math: one probe, and the bounded polling loop out of line
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity) {
-  if (mbar_try_wait(bar, parity)) return true;
-  return mbar_wait_slow(bar, parity);
-}
-// global -> this CTA's shared memory, completion counted in bytes on the mbarrier (no multicast)
-__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
-               "l"(src), "r"(bytes), "r"(bar)
-               : "memory");
 }
 
 template <int KV>

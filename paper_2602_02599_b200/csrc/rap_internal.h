@@ -95,10 +95,13 @@ struct rap_scan_params {
 struct rap_scan_entry {
   int G, WK, DV;       // query heads per KV head, K words per row (= P), V channels (= d_v')
   int smem, tile;      // dynamic shared memory, positions per tile
+  int threads;         // CTA size
   const void* fn;      // the kernel, launched with cudaLaunchKernel
 };
-// the instantiation built for this head shape, or nullptr (generated at build time)
+// the instantiation built for this head shape, or nullptr (generated at build time):
+// the FP32-pipe scan (rap_attn_scan_kernel.cuh) and the mma.sync scan (rap_attn_mma_kernel.cuh)
 const rap_scan_entry* rap_scan_find(int G, int WK, int DV);
+const rap_scan_entry* rap_mma_find(int G, int WK, int DV);
 
 // Launchers implemented in the kernel files.  All return RAP_OK or RAP_ECUDA.
 struct rap_attn_args {
