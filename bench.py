@@ -39,7 +39,7 @@ def load_peaks():
 
 def load_traffic(workload):
     """DRAM bytes per attention-scan launch from the committed ncu summary, if it lists this workload."""
-    path = os.path.join(ROOT, "profiles", "attn_scan_traffic.txt")
+    path = os.path.join(ROOT, "profiles", "attn_decode_traffic.txt")
     if os.path.exists(path):
         for line in open(path):
             f = line.split()

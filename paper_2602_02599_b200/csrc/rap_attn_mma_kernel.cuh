@@ -24,12 +24,19 @@
 //     the same channel of two rows, so two 32-bit loads (two rows, channels c, c+1) and two byte permutes
 //     give the B registers of an even-channel and an odd-channel n-tile.  Odd d_v' (rows only 2-byte
 //     aligned): the odd rows of a block take the neighbouring aligned words instead.
+//   * Rows of exactly 128 or 256 bytes (P = 32, 64 with d_v' = 64, 128: the unpruned cache and rho = 0.5) would
+//     put every row on the same banks.  For them the blocks come in through tensor maps instead
+//     (cp.async.bulk.tensor.2d, boxes of 32 rows x 128 bytes, 128-byte swizzle, no multicast): the 16-byte
+//     chunk c of row r lands at chunk c ^ (r % 8), which spreads the fragment loads over all banks at no
+//     extra instruction (the swizzled offsets are per-thread constants).
 //   * At the end of a unit the warps merge (maximum, scaled sums) through shared memory and the CTA writes
 //     one partial; the CTA that delivers a unit's last partial merges the unit (as in the FP32 scan).
 // P enters the second contraction as two bf16 operands, the rounded value and the rounding remainder (two
 // MMAs per tile on the same V fragments), so the weights carry about 17 bits; the row sum uses the fp32 values.
 // Every mbarrier wait is bounded: on timeout the CTA records RAP_ETIMEOUT and leaves.
 #pragma once
+#include <cuda.h>
+
 #include "rap_attn_common.cuh"
 
 namespace {
@@ -59,23 +66,27 @@ struct MmaCfg {
   // row step between the 8 columns of an n-tile: K-word stride * step = 4 * odd puts them on distinct banks
   static constexpr int RS_K = (WK % 2) ? 4 : (WK % 4) ? 2 : 1;
   static constexpr int RS = (VODD && RS_K == 1) ? 2 : RS_K;   // odd d_v' wants row pairs of one parity
+  // tensor-map staging with the 128-byte swizzle: panels of 32 rows x 128 bytes
+  static constexpr bool TMA = (WK % 32) == 0 && (DV % 64) == 0;
+  static constexpr int NKP = WK / 32, NVP = DV / 64;          // panels per K / V block (TMA only)
   static constexpr int K_BYTES = MMA_BR * WK * 4, V_BYTES = MMA_BR * DV * 2;
-  static constexpr int STAGE_BYTES = cround(K_BYTES + V_BYTES + 16, 128);
+  static constexpr int STAGE_BYTES = TMA ? K_BYTES + V_BYTES : cround(K_BYTES + V_BYTES + 16, 128);
+  static constexpr int STAGE_ALIGN = TMA ? 1024 : 128;
   static constexpr int NSTG = RAP_MMA_NSTG;
   static constexpr int RED_BYTES_1 = G * CW * 4;              // per warp
   static constexpr int MERGE_BYTES = (G * RAP_MAX_SPLIT + 8) * 4;
   static constexpr int OFF_RED = 512;
   static constexpr int fits(int nw) {
     const int red = nw * RED_BYTES_1 > MERGE_BYTES ? nw * RED_BYTES_1 : MERGE_BYTES;
-    return cround(OFF_RED + red, 128) + nw * NSTG * STAGE_BYTES;
+    return cround(OFF_RED + red, STAGE_ALIGN) + nw * NSTG * STAGE_BYTES + (TMA ? 1024 : 0);
   }
   static constexpr int NW = fits(RAP_MMA_NW) <= SMEM_BUDGET ? RAP_MMA_NW
                             : fits(3) <= SMEM_BUDGET        ? 3
                             : fits(2) <= SMEM_BUDGET        ? 2
                                                             : 1;
   static constexpr int RED_BYTES = NW * RED_BYTES_1 > MERGE_BYTES ? NW * RED_BYTES_1 : MERGE_BYTES;
-  static constexpr int OFF_STAGE = cround(OFF_RED + RED_BYTES, 128);
-  static constexpr int SMEM = OFF_STAGE + NW * NSTG * STAGE_BYTES;
+  static constexpr int OFF_STAGE = cround(OFF_RED + RED_BYTES, STAGE_ALIGN);
+  static constexpr int SMEM = OFF_STAGE + NW * NSTG * STAGE_BYTES + (TMA ? 1024 : 0);   // slack to align the base
   static constexpr int THREADS = NW * 32;
   static constexpr int ST = NW * MMA_BR;                      // positions per CTA tile
   static_assert(SMEM <= SMEM_BUDGET, "ring does not fit");
@@ -101,6 +112,13 @@ __device__ __forceinline__ uint32_t mma_pack_bf16(float lo, float hi) {
   asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
   return r;
 }
+// one box of a 2-D tensor map (x = element column, y = row) into this CTA's shared memory; no multicast
+__device__ __forceinline__ void mma_tma_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+      "l"(map), "r"(x), "r"(y), "r"(bar)
+      : "memory");
+}
 __device__ __forceinline__ uint32_t mma_prmt(uint32_t a, uint32_t b, uint32_t sel) {
   uint32_t r;
   asm("prmt.b32 %0, %1, %2, %3;" : "=r"(r) : "r"(a), "r"(b), "r"(sel));
@@ -108,11 +126,15 @@ __device__ __forceinline__ uint32_t mma_prmt(uint32_t a, uint32_t b, uint32_t se
 }
 
 template <int G, int WK, int DV>
-__global__ void __launch_bounds__(MmaCfg<G, WK, DV>::THREADS, 2) attn_mma_kernel(const ScanParams p) {
+__global__ void __launch_bounds__(MmaCfg<G, WK, DV>::THREADS, 2) attn_mma_kernel(const ScanParams p,
+                                                                                 const __grid_constant__ CUtensorMap map_k,
+                                                                                 const __grid_constant__ CUtensorMap map_v) {
   using C = MmaCfg<G, WK, DV>;
   constexpr int ST = C::ST, NW = C::NW, NSTG = C::NSTG, NKS = C::NKS, NCB = C::NCB, CW = C::CW;
   constexpr int THREADS = C::THREADS;
-  extern __shared__ __align__(128) unsigned char smem[];
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  // swizzled panels want a 1024-byte aligned base
+  unsigned char* smem = C::TMA ? smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u) : smem_raw;
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem);                        // [NW][NSTG]
   float* m_s = reinterpret_cast<float*>(smem + NW * NSTG * 8);               // [NW][8] reference maxima of the warps
   float* l_s = m_s + NW * 8;                                                 // [NW][8] scaled row sums
@@ -166,6 +188,17 @@ __global__ void __launch_bounds__(MmaCfg<G, WK, DV>::THREADS, 2) attn_mma_kernel
   int koff[4];
 #pragma unroll
   for (int t = 0; t < 4; ++t) koff[t] = C::row(t, gid) * WK + tq;
+  // swizzled panels (rows gid + 8 t, chunk c of the row at chunk c ^ gid): word offsets by chunk, the panel and
+  // the n-tile are immediates
+  int kx[8];
+#pragma unroll
+  for (int c = 0; c < 8; ++c) kx[c] = gid * 32 + ((c ^ gid) << 2) + tq;
+  // V, swizzled: rows 2 tq + e + 8 t, word 8 (cb % 4) + gid of the panel row
+  int vx[4][2];
+#pragma unroll
+  for (int cm = 0; cm < 4; ++cm)
+#pragma unroll
+    for (int e = 0; e < 2; ++e) vx[cm][e] = (2 * tq + e) * 32 + (((2 * cm + (gid >> 2)) ^ (2 * tq + e)) << 2) + (gid & 3);
   // V words of this thread's rows: row(t, 2 tq) of n-tile t, channel word gid (floor for odd rows of an odd d_v')
   int vofs[4];
 #pragma unroll
@@ -218,9 +251,19 @@ __global__ void __launch_bounds__(MmaCfg<G, WK, DV>::THREADS, 2) attn_mma_kernel
       const uint32_t kb = (uint32_t)rows * WK * 4, vb = (uint32_t)rows * DV * 2;
       if (lane == 0) {
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // earlier generic writes (zero fill) come first
-        mbar_expect_tx(bar, kb + vb);
-        bulk_g2s(dst, kg + (size_t)j0 * (WK * 4), kb, bar);
-        bulk_g2s(dst + C::K_BYTES, vg + (size_t)j0 * (DV * 2), vb, bar);
+        if constexpr (C::TMA) {
+          // whole boxes: rows past the end of the tensor are zero-filled, rows of a neighbouring unit are masked
+          const int y = (int)unit * p.S_cap + j0;
+          mbar_expect_tx(bar, C::STAGE_BYTES);
+#pragma unroll
+          for (int pn = 0; pn < C::NKP; ++pn) mma_tma_2d(dst + pn * 4096, &map_k, 64 * pn, y, bar);
+#pragma unroll
+          for (int pn = 0; pn < C::NVP; ++pn) mma_tma_2d(dst + C::K_BYTES + pn * 4096, &map_v, 64 * pn, y, bar);
+        } else {
+          mbar_expect_tx(bar, kb + vb);
+          bulk_g2s(dst, kg + (size_t)j0 * (WK * 4), kb, bar);
+          bulk_g2s(dst + C::K_BYTES, vg + (size_t)j0 * (DV * 2), vb, bar);
+        }
       }
     };
     {
@@ -265,8 +308,14 @@ __global__ void __launch_bounds__(MmaCfg<G, WK, DV>::THREADS, 2) attn_mma_kernel
       if (nrows < MMA_BR) {
         // last block of the sequence: rows >= nrows were not written by this sequence; zero their V so that
         // the second contraction meets 0 * 0 there
-        uint16_t* vz = reinterpret_cast<uint16_t*>(wstage + st * C::STAGE_BYTES + C::K_BYTES);
-        for (int x = nrows * DV + lane; x < MMA_BR * DV; x += 32) vz[x] = 0;
+        if constexpr (C::TMA) {   // a row is 128 contiguous bytes of each panel, whatever the swizzle
+          uint32_t* vz = reinterpret_cast<uint32_t*>(wstage + st * C::STAGE_BYTES + C::K_BYTES);
+          for (int pn = 0; pn < C::NVP; ++pn)
+            for (int x = nrows * 32 + lane; x < MMA_BR * 32; x += 32) vz[pn * 1024 + x] = 0u;
+        } else {
+          uint16_t* vz = reinterpret_cast<uint16_t*>(wstage + st * C::STAGE_BYTES + C::K_BYTES);
+          for (int x = nrows * DV + lane; x < MMA_BR * DV; x += 32) vz[x] = 0;
+        }
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // before a later bulk copy into this stage
         __syncwarp();
       }
@@ -280,7 +329,14 @@ __global__ void __launch_bounds__(MmaCfg<G, WK, DV>::THREADS, 2) attn_mma_kernel
         const int wb = ks < NKS - 1 ? 8 * ks : WK - 8;
 #pragma unroll
         for (int t = 0; t < 4; ++t) {
-          const uint32_t b0 = kw[koff[t] + wb], b1 = kw[koff[t] + wb + 4];
+          uint32_t b0, b1;
+          if constexpr (C::TMA) {
+            b0 = kw[kx[(2 * ks) % 8] + (ks / 4) * 1024 + 256 * t];
+            b1 = kw[kx[(2 * ks + 1) % 8] + (ks / 4) * 1024 + 256 * t];
+          } else {
+            b0 = kw[koff[t] + wb];
+            b1 = kw[koff[t] + wb + 4];
+          }
           mma_bf16(s[t], qa[ks][0], qa[ks][1], b0, b1);
         }
       }
@@ -343,10 +399,22 @@ __global__ void __launch_bounds__(MmaCfg<G, WK, DV>::THREADS, 2) attn_mma_kernel
 #pragma unroll
         for (int cb = 0; cb < NCB; ++cb) {
           const int cw = (cb < NCB - 1 ? 16 * cb : C::CB_LAST) / 2;
-          const uint32_t xa0 = v0[cw], xb0 = v0[cw + VPAIR];
+          uint32_t xa0, xb0;
+          if constexpr (C::TMA) {
+            xa0 = vw[vx[cb % 4][0] + (cb / 4) * 1024 + 256 * (2 * kb)];
+            xb0 = vw[vx[cb % 4][1] + (cb / 4) * 1024 + 256 * (2 * kb)];
+          } else {
+            xa0 = v0[cw];
+            xb0 = v0[cw + VPAIR];
+          }
           const uint32_t be0 = mma_prmt(xa0, xb0, 0x5410u), bo0 = mma_prmt(xa0, xb0, 0x7632u);
           uint32_t be1, bo1;
-          if constexpr (!C::VODD) {
+          if constexpr (C::TMA) {
+            const uint32_t xa1 = vw[vx[cb % 4][0] + (cb / 4) * 1024 + 256 * (2 * kb + 1)];
+            const uint32_t xb1 = vw[vx[cb % 4][1] + (cb / 4) * 1024 + 256 * (2 * kb + 1)];
+            be1 = mma_prmt(xa1, xb1, 0x5410u);
+            bo1 = mma_prmt(xa1, xb1, 0x7632u);
+          } else if constexpr (!C::VODD) {
             const uint32_t xa1 = v1[cw], xb1 = v1[cw + VPAIR];
             be1 = mma_prmt(xa1, xb1, 0x5410u);
             bo1 = mma_prmt(xa1, xb1, 0x7632u);

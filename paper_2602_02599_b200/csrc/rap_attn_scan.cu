@@ -80,7 +80,14 @@ static rap_status launch_split_kv(rap_ctx* ctx, const rap_attn_args& a, int n_sp
   const int scan_grid = 2 * ctx->sm_count;
   dim3 grid(n_split, a.Hkv, a.B);
   if (balanced) grid = dim3(scan_grid, 1, 1);
-  void* args[] = {&p};
+  alignas(64) unsigned char map_k[128] = {0}, map_v[128] = {0};   // CUtensorMap images (kernels without maps ignore them)
+  if (e->tma) {
+    const uint64_t rows = (uint64_t)a.B * a.Hkv * a.S_cap;
+    if (!rap_tensor_map_bf16(ctx, map_k, a.k, rows, (uint64_t)a.P2, 32) ||
+        !rap_tensor_map_bf16(ctx, map_v, a.v, rows, (uint64_t)a.dv, 32))
+      return RAP_EUNSUPPORTED;
+  }
+  void* args[] = {&p, map_k, map_v};
   RAP_CUDA_TRY(ctx, cudaLaunchKernel(e->fn, grid, dim3(e->threads), args, (size_t)e->smem, st));
   ctx->launches++;
   RAP_CUDA_TRY(ctx, cudaGetLastError());

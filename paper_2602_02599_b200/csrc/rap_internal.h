@@ -96,12 +96,16 @@ struct rap_scan_entry {
   int G, WK, DV;       // query heads per KV head, K words per row (= P), V channels (= d_v')
   int smem, tile;      // dynamic shared memory, positions per tile
   int threads;         // CTA size
+  int tma;             // 1: the kernel takes tensor maps of the K and V caches (boxes of 32 rows x 64 elements)
   const void* fn;      // the kernel, launched with cudaLaunchKernel
 };
 // the instantiation built for this head shape, or nullptr (generated at build time):
 // the FP32-pipe scan (rap_attn_scan_kernel.cuh) and the mma.sync scan (rap_attn_mma_kernel.cuh)
 const rap_scan_entry* rap_scan_find(int G, int WK, int DV);
 const rap_scan_entry* rap_mma_find(int G, int WK, int DV);
+// Tensor map over a row-major [rows][cols] bf16 matrix, boxes of box_rows x 64 elements, 128-byte swizzle,
+// zero fill outside; cached in the context by (pointer, shape, box).  map128 receives the 128-byte CUtensorMap.
+bool rap_tensor_map_bf16(rap_ctx* ctx, void* map128, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows);
 
 // Launchers implemented in the kernel files.  All return RAP_OK or RAP_ECUDA.
 struct rap_attn_args {

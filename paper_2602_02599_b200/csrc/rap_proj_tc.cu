@@ -335,6 +335,10 @@ rap_status launch_tc(rap_ctx* ctx, const CUtensorMap& mw, const CUtensorMap& mx,
 
 }  // namespace
 
+bool rap_tensor_map_bf16(rap_ctx* ctx, void* map128, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows) {
+  return make_map(ctx, reinterpret_cast<CUtensorMap*>(map128), base, rows, cols, box_rows);
+}
+
 // Y[ks][T][N] (fp32, context workspace) = X[T][K] * W[N][K]^T, bf16 operands, K split over grid.z.
 rap_status rap_launch_gemm_tc(rap_ctx* ctx, const void* x, const void* w, int T, int K, int N, int* ksplit_out,
                               cudaStream_t st) {
