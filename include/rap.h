@@ -269,7 +269,8 @@ rap_status rap_profile_attn_read(rap_ctx* ctx, float* ms_sum, int32_t* n_calls);
 /* Forces a kernel variant for rap_decode_attn: 0 = automatic (the shape-specialised scans when the
  * head shape has one, the tensor-core form first; the low-rank comparator's fast path), 1 = fully generic
  * kernels only, 2 = skip the shape-specialised scans, 3 = skip only the tensor-core form of the
- * shape-specialised scan.  Meant for tests and profiling. */
+ * shape-specialised scan, 4 = the tensor-core form or nothing (bf16 calls return RAP_EUNSUPPORTED when the
+ * head shape has no instantiation of it).  Meant for tests and profiling. */
 rap_status rap_set_attn_variant(rap_ctx* ctx, int32_t variant);
 
 #ifdef __cplusplus

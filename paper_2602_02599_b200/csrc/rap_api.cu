@@ -62,7 +62,7 @@ const char* rap_last_cuda_error(const rap_ctx* ctx) { return ctx ? ctx->cuda_err
 int64_t rap_kernel_launch_count(const rap_ctx* ctx) { return ctx ? ctx->launches : 0; }
 
 rap_status rap_set_attn_variant(rap_ctx* ctx, int32_t variant) {
-  if (!ctx || variant < 0 || variant > 3) return RAP_EINVAL;
+  if (!ctx || variant < 0 || variant > 4) return RAP_EINVAL;
   ctx->attn_variant = variant;
   return RAP_OK;
 }

@@ -178,6 +178,7 @@ rap_status rap_launch_attn(rap_ctx* ctx, const rap_attn_args& a, cudaStream_t st
   if (a.dtype == RAP_BF16 && ctx->attn_variant != 1) {
     // shape-specialised scans (mma.sync, then FP32 pipes), then the shape-generic bf16 scan, then the fully
     // generic kernel
+    if (ctx->attn_variant == 4) return rap_launch_attn_mma(ctx, a, a.n_split, st);
     if (ctx->attn_variant == 0) {
       const rap_status s = rap_launch_attn_mma(ctx, a, a.n_split, st);
       if (s != RAP_EUNSUPPORTED) return s;

@@ -164,9 +164,10 @@ def test_adjacent_pairing_end_to_end():
     _end_to_end(w, [40])
 
 
-def _random_attn_case(w, lens, n_split, seed=0):
+def _random_attn_case(w, lens, n_split, seed=0, variant=0):
     """rap_decode_attn alone on random caches (no projection), every unit checked."""
     st = DecodeStack(w, s_cap=((max(lens) + 8 + 7) // 8) * 8)
+    st.ctx.rap_set_attn_variant(variant)
     ks, vs = synth.draw_scores(w)
     st.build_tables(ks, vs)
     g = torch.Generator(device=st.device).manual_seed(seed)
@@ -196,6 +197,28 @@ def _random_attn_case(w, lens, n_split, seed=0):
 def test_attention_only_longer_sequences(name, n_split):
     w = synth.scaled_down(synth.CONFIGS[name], n_layers=1, batch=3, seq=4096)
     _random_attn_case(w, [4096, 2500, 1], n_split)
+
+
+@pytest.mark.parametrize("name", ["3b", "8b", "14b", "sweep1.0", "sweep0.5"])
+@pytest.mark.parametrize("n_split", [0, 5])
+def test_attention_fp32_pipe_scan(name, n_split):
+    """The shape-specialised scan on the FP32 pipes (the tier behind the tensor-core form) against the oracle."""
+    w = synth.scaled_down(synth.CONFIGS[name], n_layers=1, batch=3, seq=4096)
+    _random_attn_case(w, [4096, 2500, 1], n_split, variant=3)
+
+
+@pytest.mark.parametrize("G,P,dv", [(8, 45, 90), (1, 58, 115), (6, 51, 102), (2, 45, 90), (4, 22, 44), (4, 20, 40),
+                                    (5, 41, 82), (3, 63, 126), (4, 64, 64), (7, 32, 64), (8, 64, 128)])
+def test_attention_tensor_core_scan_head_shapes(G, P, dv):
+    """The tensor-core form of the scan, forced (variant 4 fails instead of falling back): group sizes 1..8,
+    odd and even d_v', the three row-spreading steps of the fragment loads (P odd, P = 2 mod 4, P = 0 mod 4)
+    and the shapes staged through swizzling tensor maps; ragged lengths, a block with one row, both split
+    modes."""
+    from dataclasses import replace
+    base = synth.scaled_down(synth.LLAMA_8B, n_layers=1, batch=4, seq=3000)
+    w = replace(base, n_pairs=P, n_vch=dv, n_q_heads=G * base.n_kv_heads)
+    _random_attn_case(w, [3000, 1777, 1, 33], 0, seed=P + G, variant=4)
+    _random_attn_case(w, [129, 0, 2999, 96], 3, seed=P, variant=4)
 
 
 def test_attention_generic_variant_matches():
