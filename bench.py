@@ -131,6 +131,8 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
     w = pick_workload(args)
     st = build_stack(w, torch, seed_offset=rank)
+    if args.attn_variant:
+        st.ctx.rap_set_attn_variant(args.attn_variant)
     L, B, K, W = w.n_layers, w.batch, args.steps, args.warmup
     n_steps = K + W
     assert w.seq + 2 * n_steps + 2 < st.s_cap, "cache capacity too small for this many steps"
@@ -217,10 +219,13 @@ def run_ours(args):
         "e2e": {"value": aggregate_throughput(B, world, e2e_ms), "unit": UNIT,
                 "h2d_bytes_per_step": int(hx[0].numel() * hx[0].element_size()),
                 "d2h_bytes_per_step": int(h_out.numel() * 4)},
-        "roofline": {"bound": "hbm", "kernel": "rap_decode_attn (split-KV scan with the merge of the splits fused in)", "achieved": achieved,
+        "roofline": {"bound": "hbm", "kernel": "rap_decode_attn (attn_mma_kernel: split-KV scan with the merge of the splits fused in)"
+                     if not args.attn_variant else "rap_decode_attn (forced tier %d)" % args.attn_variant,
+                     "achieved": achieved,
                      "peak": peak, "peak_source": peak_kind, "unit": "GB/s", "frac": achieved / peak,
                      "frac_of_nominal_8000": achieved / 8000.0, "bytes_per_launch": alg, "ms_per_launch": attn_ms,
-                     "traffic": load_traffic(args.workload)},
+                     "traffic": None if (args.attn_variant or args.layers or args.batch or args.seq)
+                     else load_traffic(args.workload)},
         "kernels": {"attn_ms_per_layer": attn_ms, "rest_ms_per_layer": proj_ms},
     }
     if args.cpu_baseline:
@@ -381,6 +386,8 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="cut the workload to this many layers (profiling)")
     ap.add_argument("--batch", type=int, default=0, help="cut the workload to this batch (profiling)")
     ap.add_argument("--seq", type=int, default=0, help="cut the workload to this context (profiling)")
+    ap.add_argument("--attn-variant", type=int, default=0,
+                    help="force a kernel tier of rap_decode_attn (profiling; 3 = the FP32-pipe scan)")
     ap.add_argument("--sweep", action="store_true", help="retain-ratio sweep with the dense and low-rank comparators")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
