@@ -100,6 +100,48 @@ def build_tables_hybrid(k_pair_scores, k_chan_scores, v_chan_scores, rope_layer,
     return tabs
 
 
+def build_tables_partial(k_pair_scores, k_chan_scores, v_chan_scores, rot_dims, n_rot_pairs, n_pairs, n_vch,
+                         head_dim, rope_theta, pairing):
+    """Tables of a model that rotates only the first rot_dims[l] dims of every head (Appendix "RoPE in Recent
+    Open LLMs": partial rotary; Section 4, "Hybrid compression": RAP on the rotated part, channel pruning
+    on the rest).
+
+    Layer l, KV head h.  Rotated part: pairs i = 0 .. R/2 - 1 with R = rot_dims[l], members (i, i + R/2)
+    (HALF pairing inside the rotated block) or (2i, 2i + 1) (ADJACENT), frequency theta ** (-2 i / R); the
+    n_rot_pairs[l] pairs with the largest k_pair_scores[l, h, :R/2] are kept, ascending.  Unrotated part:
+    channels R .. D - 1; the 2 * (n_pairs[l] - n_rot_pairs[l]) channels with the largest
+    k_chan_scores[l, h, R:] are kept, ascending.  The reduced K row is [kept pairs, members adjacent |
+    kept channels]; the frequency of a slot that holds unrotated channels is zero (identity rotation), so the
+    online path is the same as for a fully rotary layer.  V as in build_tables.
+    R = D reproduces build_tables, R = 0 a layer without positional rotation."""
+    kp = np.asarray(k_pair_scores, dtype=np.float64)
+    kc = np.asarray(k_chan_scores, dtype=np.float64)
+    vs = np.asarray(v_chan_scores, dtype=np.float64)
+    L, H, D = vs.shape
+    assert D == head_dim
+    tabs = {"k_pair_idx": np.full((L, H, D // 2), -1, dtype=np.int32),
+            "k_dim_idx": np.full((L, H, D), -1, dtype=np.int32),
+            "v_idx": np.full((L, H, D), -1, dtype=np.int32),
+            "inv_freq": np.zeros((L, H, D // 2), dtype=np.float64)}
+    for l in range(L):
+        R, Pr, P = int(rot_dims[l]), int(n_rot_pairs[l]), int(n_pairs[l])
+        C = 2 * (P - Pr)
+        assert R % 2 == 0 and 0 <= R <= D and 0 <= Pr <= R // 2 and 0 <= C <= D - R
+        for h in range(H):
+            pairs = top_k_ascending(kp[l, h, : R // 2], Pr) if Pr else np.zeros(0, dtype=np.int64)
+            for c, i in enumerate(pairs):
+                i = int(i)
+                tabs["k_pair_idx"][l, h, c] = i
+                a, b = (i, i + R // 2) if pairing == PAIR_HALF else (2 * i, 2 * i + 1)
+                tabs["k_dim_idx"][l, h, 2 * c] = a
+                tabs["k_dim_idx"][l, h, 2 * c + 1] = b
+                tabs["inv_freq"][l, h, c] = float(rope_theta) ** (-(2.0 * i) / R)
+            if C:
+                tabs["k_dim_idx"][l, h, 2 * Pr: 2 * P] = R + top_k_ascending(kc[l, h, R:], C)
+            tabs["v_idx"][l, h, : int(n_vch[l])] = top_k_ascending(vs[l, h], int(n_vch[l]))
+    return tabs
+
+
 # --------------------------------------------------------------------------------------
 # Tables  (Algorithm 2, selection step; Eq. 6 RAPIndex; Eq. 3 frequencies)
 # --------------------------------------------------------------------------------------

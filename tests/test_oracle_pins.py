@@ -453,3 +453,67 @@ def test_nope_layer_tables_give_plain_channel_pruned_attention():
     t2 = O.build_tables_hybrid(np.concatenate([m["ks"], m["ks"]]), np.concatenate([kc, kc]), np.concatenate([m["vs"], m["vs"]]),
                                [1, 0], [P, P], [dv, dv], D, m["theta"], m["pairing"])
     assert np.array_equal(t2["k_dim_idx"][0], m["tabs"]["k_dim_idx"][0]) and np.array_equal(t2["inv_freq"][0], m["tabs"]["inv_freq"][0])
+
+
+# ---- partial rotary: RAP on the rotated dims of a head, channel pruning on the rest -----------------
+def test_partial_rotary_tables_reduce_to_the_full_and_the_unrotated_case():
+    m = _small(rho=0.75, D=16, Hq=4, Hkv=2, n=5, seed=17)
+    D, Hkv, P, dv = m["D"], m["Hkv"], m["P"], m["dv"]
+    kc = np.random.default_rng(4).lognormal(0, 1, (1, Hkv, D))
+    full = O.build_tables_partial(m["ks"], kc, m["vs"], [D], [P], [P], [dv], D, m["theta"], m["pairing"])
+    for key in ("k_pair_idx", "k_dim_idx", "v_idx", "inv_freq"):
+        assert np.array_equal(full[key], m["tabs"][key]), key
+    none = O.build_tables_partial(m["ks"], kc, m["vs"], [0], [0], [P], [dv], D, m["theta"], m["pairing"])
+    want = O.build_tables_hybrid(m["ks"], kc, m["vs"], [0], [P], [dv], D, m["theta"], m["pairing"])
+    for key in ("k_pair_idx", "k_dim_idx", "v_idx", "inv_freq"):
+        assert np.array_equal(none[key], want[key]), key
+
+
+@pytest.mark.parametrize("pairing", [O.PAIR_HALF, O.PAIR_ADJACENT])
+def test_partial_rotary_reduced_path_equals_full_width_attention(pairing):
+    """Rotate only the first R dims of each head (the usual formulation, applied to that block with its own
+    table theta^(-2i/R)), zero the dropped K dims, keep the retained V channels: the reduced path built from
+    build_tables_partial gives the same output."""
+    m = _small(pairing=pairing, rho=0.75, D=16, Hq=4, Hkv=2, n=6, seed=29)
+    D, Hq, Hkv, dv, X = m["D"], m["Hq"], m["Hkv"], m["dv"], m["X"]
+    R, Pr, P = 8, 3, 5                          # 3 of 4 rotated pairs, 4 of 8 unrotated channels
+    kc = np.random.default_rng(8).lognormal(0, 1, (1, Hkv, D))
+    tabs = O.build_tables_partial(m["ks"], kc, m["vs"], [R], [Pr], [P], [dv], D, m["theta"], pairing)
+    # structure: pairs inside the rotated block, channels outside, zero frequency on the channel slots
+    for h in range(Hkv):
+        dims = tabs["k_dim_idx"][0, h, : 2 * P]
+        assert len(set(dims.tolist())) == 2 * P and np.all(dims[: 2 * Pr] < R) and np.all(dims[2 * Pr:] >= R)
+        assert np.all(np.diff(dims[2 * Pr:]) > 0) and np.all(tabs["inv_freq"][0, h, Pr:] == 0.0)
+        for c in range(Pr):
+            i = int(tabs["k_pair_idx"][0, h, c])
+            assert tabs["inv_freq"][0, h, c] == m["theta"] ** (-2.0 * i / R)
+        want_ch = R + np.sort(np.argsort(-kc[0, h, R:], kind="stable")[: 2 * (P - Pr)])
+        assert np.array_equal(dims[2 * Pr:], want_ch)
+    w = O.gather_weights(m["Wq"], m["Wk"], m["Wv"], tabs, 0, P, dv, D)
+    got, _, _, _ = O.reduced_attention_from_hidden(X, w, tabs["inv_freq"][0], Hq, Hkv, P, dv, D)
+    n, G = X.shape[0], Hq // Hkv
+
+    def rot(x, pos):
+        return np.concatenate([O.textbook_rope(x[:R], pos, R, m["theta"], pairing), x[R:]])
+
+    want = np.zeros((Hq, dv))
+    for g in range(Hq):
+        h = g // G
+        keep = [int(d) for d in tabs["k_dim_idx"][0, h, : 2 * P]]
+        q = rot(m["Wq"][g * D:(g + 1) * D] @ X[-1], n - 1)
+        s = np.empty(n)
+        for j in range(n):
+            k = rot(m["Wk"][h * D:(h + 1) * D] @ X[j], j)
+            s[j] = sum(q[d] * k[d] for d in keep) / math.sqrt(D)
+        pr = np.exp(s - s.max()); pr /= pr.sum()
+        for c in range(dv):
+            u = tabs["v_idx"][0, h, c]
+            want[g, c] = sum(pr[j] * float(m["Wv"][h * D + u] @ X[j]) for j in range(n))
+    assert np.allclose(got, want, rtol=0, atol=1e-12)
+    # the pin bites: a table that forgets the block-local frequency (theta^(-2i/D) instead of /R) fails it
+    bad = {k: v.copy() for k, v in tabs.items()}
+    for h in range(Hkv):
+        for c in range(Pr):
+            bad["inv_freq"][0, h, c] = m["theta"] ** (-2.0 * int(tabs["k_pair_idx"][0, h, c]) / D)
+    got_bad, _, _, _ = O.reduced_attention_from_hidden(X, w, bad["inv_freq"][0], Hq, Hkv, P, dv, D)
+    assert not np.allclose(got_bad, want, rtol=0, atol=1e-6)
