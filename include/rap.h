@@ -124,6 +124,22 @@ rap_status rap_build_tables_hybrid(rap_ctx* ctx, const double* h_k_pair_scores, 
                                    const int32_t* h_n_pairs, const int32_t* h_n_vch, int32_t* d_k_pair_idx,
                                    int32_t* d_k_dim_idx, int32_t* d_v_idx, double* d_inv_freq, void* stream);
 
+/* Tables of a model that rotates only the first h_rot_dims[l] dims of every head (appendix "RoPE in Recent Open
+ * LLMs", partial rotary; Section 4, "Hybrid compression": RAP on the rotated dims, channel pruning on the rest).
+ * Layer l with R = h_rot_dims[l] (even, 0..D): rotated pairs i = 0..R/2-1 have members (i, i + R/2) (or
+ * (2i, 2i+1) with adjacent pairing) and frequency theta^(-2i/R); the h_n_rot_pairs[l] (0..R/2) best of them by
+ * h_k_pair_scores[l][h][0..R/2) are kept.  Of the unrotated dims R..D-1 the 2 * (h_n_pairs[l] -
+ * h_n_rot_pairs[l]) (at most D - R) best by h_k_chan_scores[l][h][R..D) are kept.  The reduced K row is
+ * [kept pairs, members adjacent | kept channels ascending]; a slot that holds unrotated channels has
+ * d_k_pair_idx = -1 and frequency zero, so the shared online path rotates it by the identity.  R = D gives
+ * rap_build_tables, R = 0 a layer of rap_build_tables_hybrid without RoPE.  Everything else as rap_build_tables;
+ * RAP_EINVAL for counts outside those ranges. */
+rap_status rap_build_tables_partial(rap_ctx* ctx, const double* h_k_pair_scores, const double* h_k_chan_scores,
+                                    const double* h_v_chan_scores, const int32_t* h_rot_dims,
+                                    const int32_t* h_n_rot_pairs, const int32_t* h_n_pairs, const int32_t* h_n_vch,
+                                    int32_t* d_k_pair_idx, int32_t* d_k_dim_idx, int32_t* d_v_idx,
+                                    double* d_inv_freq, void* stream);
+
 /* ---- offline weight gather (Algorithm 1: W~_k, W~_q = W_q E_k^T, W~_v) ----------------
  * Index selection, no arithmetic.  d_wq [H_q*D][hidden], d_wk / d_wv [H_kv*D][hidden] are the
  * dense weights of `layer`; d_w_qkv [N_out][hidden] receives the rows

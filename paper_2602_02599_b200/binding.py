@@ -26,6 +26,7 @@ EXPORTS = [
     "rap_get_last_device_status", "rap_kernel_launch_count", "rap_set_attn_variant",
     "rap_decode_attn_noalloc", "rap_profile_attn", "rap_profile_attn_read",
     "rap_pack_wo", "rap_out_proj", "rap_budget_alloc", "rap_prefill_attn", "rap_build_tables_hybrid",
+    "rap_build_tables_partial",
 ]
 
 
@@ -68,6 +69,7 @@ def _lib():
     lib.rap_cache_elem_offset.restype = c_size_t
     lib.rap_build_tables.argtypes = [P] * 10
     lib.rap_build_tables_hybrid.argtypes = [P] * 12
+    lib.rap_build_tables_partial.argtypes = [P] * 13
     lib.rap_pack_weights.argtypes = [P, c_int32] + [P] * 11
     lib.rap_qkv_rope_append.argtypes = [P, c_int32, c_int32, P, P, P, P, P, P, c_int32, P, P, P, P, c_int32, c_int32, P]
     lib.rap_decode_attn.argtypes = [P, c_int32, c_int32, P, P, P, c_int32, P, c_int32, c_int32, P, P]
@@ -204,6 +206,15 @@ class RapContext:
         self._check(_lib().rap_build_tables_hybrid(self._ctx, _ptr(arrs[0]), _ptr(arrs[1]), _ptr(arrs[2]), _ptr(ints[0]),
                                                    _ptr(ints[1]), _ptr(ints[2]), _ptr(d_k_pair_idx), _ptr(d_k_dim_idx),
                                                    _ptr(d_v_idx), _ptr(d_inv_freq), _stream()), "rap_build_tables_hybrid")
+
+    def rap_build_tables_partial(self, k_pair_scores, k_chan_scores, v_chan_scores, rot_dims, n_rot_pairs, n_pairs, n_vch,
+                                 d_k_pair_idx, d_k_dim_idx, d_v_idx, d_inv_freq):
+        arrs = [np.ascontiguousarray(a, dtype=np.float64) for a in (k_pair_scores, k_chan_scores, v_chan_scores)]
+        ints = [np.ascontiguousarray(a, dtype=np.int32) for a in (rot_dims, n_rot_pairs, n_pairs, n_vch)]
+        self._check(_lib().rap_build_tables_partial(self._ctx, _ptr(arrs[0]), _ptr(arrs[1]), _ptr(arrs[2]), _ptr(ints[0]),
+                                                    _ptr(ints[1]), _ptr(ints[2]), _ptr(ints[3]), _ptr(d_k_pair_idx),
+                                                    _ptr(d_k_dim_idx), _ptr(d_v_idx), _ptr(d_inv_freq), _stream()),
+                    "rap_build_tables_partial")
 
     def rap_pack_weights(self, layer, d_wq, d_wk, d_wv, d_k_dim_idx, d_v_idx, d_w_qkv,
                          d_bq=None, d_bk=None, d_bv=None, d_bias=None):

@@ -204,8 +204,13 @@ rap_status rap_destroy(rap_ctx* ctx) {
 }
 
 // kc / rope_layer are NULL for an all-rotary model
+// Shared by the three table builders.  Per layer the first R dims of a head are rotary (pairs inside that block,
+// frequency theta^(-2i/R)) and Pr of the P kept pair slots hold rotated pairs; the other slots hold 2 (P - Pr)
+// channels of the unrotated dims R..D-1 with frequency zero.  rap_build_tables: R = D, Pr = P everywhere;
+// the hybrid form: R = 0, Pr = 0 on layers without RoPE; the partial form: R and Pr per layer from the caller.
 static rap_status build_tables_impl(rap_ctx* ctx, const double* ks, const double* kc, const double* vs,
-                                    const int32_t* rope_layer, const int32_t* n_pairs, const int32_t* n_vch,
+                                    const int32_t* rope_layer, const int32_t* rot_dims, const int32_t* n_rot_pairs,
+                                    const int32_t* n_pairs, const int32_t* n_vch,
                                     int32_t* d_k_pair_idx, int32_t* d_k_dim_idx, int32_t* d_v_idx, double* d_inv_freq,
                                     void* stream) {
   if (!ctx || !ks || !vs || !n_pairs || !n_vch || !d_k_pair_idx || !d_k_dim_idx || !d_v_idx || !d_inv_freq)
@@ -215,8 +220,15 @@ static rap_status build_tables_impl(rap_ctx* ctx, const double* ks, const double
     return RAP_EALIGN;
   const rap_model_desc& d = ctx->desc;
   const int L = d.n_layers, H = d.n_kv_heads, D = d.head_dim, half = D / 2;
+  std::vector<int> rot(L), prot(L);
   for (int l = 0; l < L; ++l) {
     if (n_pairs[l] < 1 || n_pairs[l] > half || n_vch[l] < 1 || n_vch[l] > D) return RAP_EINVAL;
+    rot[l] = rot_dims ? rot_dims[l] : (rope_layer && !rope_layer[l]) ? 0 : D;
+    prot[l] = rot_dims ? n_rot_pairs[l] : (rope_layer && !rope_layer[l]) ? 0 : n_pairs[l];
+    const int chans = 2 * (n_pairs[l] - prot[l]);
+    if (rot[l] < 0 || rot[l] > D || (rot[l] & 1) || prot[l] < 0 || prot[l] > rot[l] / 2 || chans < 0 ||
+        chans > D - rot[l] || (chans > 0 && !kc))
+      return RAP_EINVAL;
   }
   const size_t units = (size_t)L * H;
   for (size_t i = 0; i < units * half; ++i) if (std::isnan(ks[i])) return RAP_EINVAL;
@@ -249,24 +261,25 @@ static rap_status build_tables_impl(rap_ctx* ctx, const double* ks, const double
     const int P = n_pairs[l], dv = n_vch[l];
     for (int h = 0; h < H; ++h) {
       const size_t u = (size_t)l * H + h;
-      if (rope_layer && !rope_layer[l]) {
-        // no positional rotation in this layer: plain channel pruning of K, zero frequencies (identity rotation)
-        top_k(kc + u * D, D, 2 * P, h_dim + u * D);
-        top_k(vs + u * D, D, dv, h_v + u * D);
-        continue;
-      }
+      const int R = rot[l], Pr = prot[l];
       int32_t* pr = h_pair + u * half;
-      top_k(ks + u * half, half, P, pr);
-      for (int c = 0; c < P; ++c) {
+      if (Pr > 0) top_k(ks + u * half, R / 2, Pr, pr);
+      for (int c = 0; c < Pr; ++c) {
         const int i = pr[c];
         if (d.pairing == RAP_PAIR_HALF) {
           h_dim[u * D + 2 * c] = i;
-          h_dim[u * D + 2 * c + 1] = i + half;
+          h_dim[u * D + 2 * c + 1] = i + R / 2;
         } else {
           h_dim[u * D + 2 * c] = 2 * i;
           h_dim[u * D + 2 * c + 1] = 2 * i + 1;
         }
-        h_freq[u * half + c] = std::pow(d.rope_theta, -2.0 * (double)i / (double)D);
+        h_freq[u * half + c] = std::pow(d.rope_theta, -2.0 * (double)i / (double)R);
+      }
+      if (P > Pr) {
+        // unrotated dims: plain channel pruning; their slots keep frequency zero (identity rotation)
+        int32_t* ch = h_dim + u * D + 2 * Pr;
+        top_k(kc + u * D + R, D - R, 2 * (P - Pr), ch);
+        for (int c = 0; c < 2 * (P - Pr); ++c) ch[c] += R;
       }
       top_k(vs + u * D, D, dv, h_v + u * D);
     }
@@ -288,7 +301,7 @@ static rap_status build_tables_impl(rap_ctx* ctx, const double* ks, const double
 rap_status rap_build_tables(rap_ctx* ctx, const double* ks, const double* vs, const int32_t* n_pairs,
                             const int32_t* n_vch, int32_t* d_k_pair_idx, int32_t* d_k_dim_idx,
                             int32_t* d_v_idx, double* d_inv_freq, void* stream) {
-  return build_tables_impl(ctx, ks, nullptr, vs, nullptr, n_pairs, n_vch, d_k_pair_idx, d_k_dim_idx, d_v_idx, d_inv_freq,
+  return build_tables_impl(ctx, ks, nullptr, vs, nullptr, nullptr, nullptr, n_pairs, n_vch, d_k_pair_idx, d_k_dim_idx, d_v_idx, d_inv_freq,
                            stream);
 }
 
@@ -297,8 +310,17 @@ rap_status rap_build_tables_hybrid(rap_ctx* ctx, const double* ks, const double*
                                    int32_t* d_k_pair_idx, int32_t* d_k_dim_idx, int32_t* d_v_idx, double* d_inv_freq,
                                    void* stream) {
   if (!kc || !rope_layer) return RAP_EINVAL;
-  return build_tables_impl(ctx, ks, kc, vs, rope_layer, n_pairs, n_vch, d_k_pair_idx, d_k_dim_idx, d_v_idx, d_inv_freq,
-                           stream);
+  return build_tables_impl(ctx, ks, kc, vs, rope_layer, nullptr, nullptr, n_pairs, n_vch, d_k_pair_idx, d_k_dim_idx,
+                           d_v_idx, d_inv_freq, stream);
+}
+
+rap_status rap_build_tables_partial(rap_ctx* ctx, const double* ks, const double* kc, const double* vs,
+                                    const int32_t* rot_dims, const int32_t* n_rot_pairs, const int32_t* n_pairs,
+                                    const int32_t* n_vch, int32_t* d_k_pair_idx, int32_t* d_k_dim_idx,
+                                    int32_t* d_v_idx, double* d_inv_freq, void* stream) {
+  if (!kc || !rot_dims || !n_rot_pairs) return RAP_EINVAL;
+  return build_tables_impl(ctx, ks, kc, vs, nullptr, rot_dims, n_rot_pairs, n_pairs, n_vch, d_k_pair_idx, d_k_dim_idx,
+                           d_v_idx, d_inv_freq, stream);
 }
 
 rap_status rap_pack_weights(rap_ctx* ctx, int32_t layer, const void* d_wq, const void* d_wk, const void* d_wv,

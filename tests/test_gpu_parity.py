@@ -468,6 +468,35 @@ def test_prefill_attn_matches_oracle(name, T, starts):
     st.close()
 
 
+def _decode_step_with_tables(st, tabs, w, lens):
+    """Weights gathered with `tabs`, caches filled the real way, one decode step through the unchanged online
+    path; appended K rows and the attention output against the oracle."""
+    L = w.n_layers
+    P, dv, Hq, Hkv, B = w.n_pairs, w.n_vch, w.n_q_heads, w.n_kv_heads, w.batch
+    w_host = []
+    for l in range(L):
+        Wq, Wk, Wv = synth.draw_full_weights(w, l)
+        st.pack_from_full(l, Wq, Wk, Wv)
+        wr = [O.round_storage(a, w.dtype) for a in (Wq, Wk, Wv)]
+        w_host.append(O.gather_weights(wr[0], wr[1], wr[2], tabs, l, P, dv, w.head_dim))
+        assert np.array_equal(util.to_np64(st.w_qkv[l]), w_host[l])
+    util.prefill_both(st, tabs, w_host, w, lens, chunk=256)
+    st.seq_len.copy_(torch.tensor(lens, dtype=torch.int32))
+    X = np.stack([synth.draw_hidden(w, l, 1, B) for l in range(L)])
+    dx = torch.from_numpy(X).to(st.device).to(st.dt).contiguous()
+    st.decode_step(dx, max(lens), advance=0)
+    torch.cuda.synchronize()
+    for l in range(L):
+        q, k, v = O.qkv_rope(O.round_storage(X[l], w.dtype), w_host[l], None, np.array(lens), tabs["inv_freq"][l], Hq, Hkv, P, dv)
+        Kd, Vd = util.to_np64(st.k_cache[l]), util.to_np64(st.v_cache[l])
+        k_dev = np.stack([Kd[b, :, lens[b], :] for b in range(B)])
+        util.check_projection(k_dev, O.round_storage(k, w.dtype), w.dtype, f"k layer {l}")
+        want = O.decode_attn(O.round_storage(q, w.dtype), Kd, Vd, np.array(lens) + 1, w.head_dim)
+        got = util.to_np64(st.out[l][: B * Hq * dv]).reshape(B, Hq, dv)
+        util.check_attn(got, want, w.dtype)
+    assert st.ctx.rap_get_last_device_status() == (0, 0)
+
+
 def test_hybrid_tables_and_nope_layer_end_to_end():
     """rap_build_tables_hybrid: layer 0 rotary, layer 1 without RoPE (channel-pruned K, zero frequencies).
     Tables bit-exact against the oracle, then one decode step through the unchanged online path."""
@@ -480,28 +509,30 @@ def test_hybrid_tables_and_nope_layer_end_to_end():
                                    st.inv_freq)
     tabs = O.build_tables_hybrid(ks, kc, vs, rope_layer, st.n_pairs, st.n_vch, w.head_dim, w.rope_theta, w.pairing)
     _tables_equal(st, tabs)
-    P, dv, Hq, Hkv, B = w.n_pairs, w.n_vch, w.n_q_heads, w.n_kv_heads, w.batch
-    w_host = []
-    for l in range(2):
-        Wq, Wk, Wv = synth.draw_full_weights(w, l)
-        st.pack_from_full(l, Wq, Wk, Wv)
-        wr = [O.round_storage(a, w.dtype) for a in (Wq, Wk, Wv)]
-        w_host.append(O.gather_weights(wr[0], wr[1], wr[2], tabs, l, P, dv, w.head_dim))
-        assert np.array_equal(util.to_np64(st.w_qkv[l]), w_host[l])
-    lens = [200, 77]
-    caches = util.prefill_both(st, tabs, w_host, w, lens, chunk=256)
-    st.seq_len.copy_(torch.tensor(lens, dtype=torch.int32))
-    X = np.stack([synth.draw_hidden(w, l, 1, B) for l in range(2)])
-    dx = torch.from_numpy(X).to(st.device).to(st.dt).contiguous()
-    st.decode_step(dx, max(lens), advance=0)
-    torch.cuda.synchronize()
-    for l in range(2):
-        q, k, v = O.qkv_rope(O.round_storage(X[l], w.dtype), w_host[l], None, np.array(lens), tabs["inv_freq"][l], Hq, Hkv, P, dv)
-        Kd, Vd = util.to_np64(st.k_cache[l]), util.to_np64(st.v_cache[l])
-        k_dev = np.stack([Kd[b, :, lens[b], :] for b in range(B)])
-        util.check_projection(k_dev, O.round_storage(k, w.dtype), w.dtype, f"k layer {l}")
-        want = O.decode_attn(O.round_storage(q, w.dtype), Kd, Vd, np.array(lens) + 1, w.head_dim)
-        got = util.to_np64(st.out[l][: B * Hq * dv]).reshape(B, Hq, dv)
-        util.check_attn(got, want, w.dtype)
-    assert st.ctx.rap_get_last_device_status() == (0, 0)
+    _decode_step_with_tables(st, tabs, w, [200, 77])
+    st.close()
+
+
+def test_partial_rotary_tables_end_to_end():
+    """rap_build_tables_partial: a fully rotary layer, a layer that rotates 64 of 128 dims (22 of its 45 pair
+    slots hold rotated pairs, the rest unrotated channels), one that rotates 32 dims and one without RoPE.
+    Tables bit-exact against the oracle, then one decode step through the unchanged online path; out-of-range
+    counts are refused."""
+    w = synth.scaled_down(synth.LLAMA_8B, n_layers=4, batch=2, seq=150, hidden=256)
+    ks, vs = synth.draw_scores(w)
+    kc = np.random.default_rng(9).lognormal(0, 1, (4, w.n_kv_heads, w.head_dim))
+    D, P = w.head_dim, w.n_pairs
+    rot_dims = [D, 64, 32, 0]
+    n_rot = [P, 22, 16, 0]          # layer 1: 22 of 32 pairs + 46 of 64 channels; layer 2: all 16 pairs + 58 of 96
+    st = DecodeStack(w, max_rows=256)
+    args = (st.n_pairs, st.n_vch, st.k_pair_idx, st.k_dim_idx, st.v_idx, st.inv_freq)
+    st.ctx.rap_build_tables_partial(ks, kc, vs, rot_dims, n_rot, *args)
+    tabs = O.build_tables_partial(ks, kc, vs, rot_dims, n_rot, st.n_pairs, st.n_vch, D, w.rope_theta, w.pairing)
+    _tables_equal(st, tabs)
+    _decode_step_with_tables(st, tabs, w, [150, 61])
+    for bad_rot, bad_n in (([D, 63, 32, 0], n_rot), ([D, 64, 32, 0], [P, 33, 16, 0]), ([D, 64, 32, 0], [P, 22, 16, 1]),
+                           ([D, 64, 32, 0], [P, 10, 16, 0])):      # odd R; pairs > R/2; pairs without rotary dims; channels > D - R
+        with pytest.raises(binding.RapError) as e:
+            st.ctx.rap_build_tables_partial(ks, kc, vs, bad_rot, bad_n, *args)
+        assert e.value.status == 1
     st.close()
