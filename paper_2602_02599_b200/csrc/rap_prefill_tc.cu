@@ -1,23 +1,27 @@
 // tcgen05 version of rap_prefill_attn: causal attention of a block of T new tokens per sequence over the
 // reduced dims (Eq. 2 for every t of the block; 2P retained K dims, d_v' retained V channels, scale
-// 1/sqrt(D)).  One CTA handles 128 queries of one query head and walks 128-key tiles up to the causal limit:
-//   S      = Q K^T      tcgen05.mma (M = 128 queries, N = 128 keys, K = 2P in steps of 16), accumulator in TMEM
+// 1/sqrt(D)).  One CTA (one per SM) handles 128 queries of one query head and walks 128-key tiles up to the
+// causal limit:
+//   S      = Q K^T      tcgen05.mma (M = 128 queries, N = 128 keys, K = 2P in steps of 16), accumulator in TMEM,
+//                       double buffered: S of tile t + 1 is issued before the softmax of tile t has finished
 //   P      = 2^(S - m)  one thread per query row reads its S row from TMEM (tcgen05.ld), applies the causal
 //                       mask and a lazy running maximum, and writes P as bf16 into shared memory
 //   O_tile = P V        tcgen05.mma (N = d_v' rounded up to 32, K = 128 keys), fresh accumulator per tile;
 //                       the row's thread then folds O_tile into its register accumulator with the rescale
 //                       factor, so tensor memory never has to be rewritten.
-// Cache rows are not multiples of 16 bytes, so TMA tensor maps cannot describe them: all threads stage the
-// tiles by hand into the K-major, 128-byte-swizzled layout the MMA descriptors expect (Q and K as stored, V
-// transposed to [channel][key]); rows past the sequence end and pad columns are zeros.  Stages of one tile
-// run one after the other (no double buffering yet).  Every mbarrier wait is bounded.
+// Cache rows are not multiples of 16 bytes, so TMA tensor maps cannot describe them: four producer warps stage
+// the tiles by hand (4-byte cp.async), one tile ahead in a two-stage ring, into the 128-byte-swizzled layouts
+// the MMA descriptors expect (K as stored = K-major; V as stored = the N-major form of the B operand, so nothing
+// is transposed); rows past the sequence end and pad columns are zeros.  The roles (4 softmax warps, 1 MMA-issuing lane, 4 producer warps) meet only on mbarriers; every
+// wait is bounded and gives up early once another role has given up.
 #include <math.h>
 
 #include "rap_internal.h"
 
 namespace {
 
-constexpr int PT_BM = 128, PT_BN = 128, PT_THREADS = 160;       // warps 0-3: rows / softmax, warp 4: MMA issue
+constexpr int PT_BM = 128, PT_BN = 128;
+constexpr int PT_THREADS = 288, PT_PRODUCERS = 128;   // warps 0-3: rows / softmax, warp 4: MMA issue, warps 5-8: staging
 constexpr int PT_TILE_BYTES = 2 * 128 * 128;                     // two 64-element atom columns of 128 rows
 constexpr uint32_t PT_WAIT_LIMIT = 1u << 21;
 
@@ -33,11 +37,6 @@ __device__ __forceinline__ bool pt_try_wait(uint32_t bar, uint32_t parity) {
       "selp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
-}
-__device__ __forceinline__ bool pt_wait(uint32_t bar, uint32_t parity) {
-  for (uint32_t i = 0; i < PT_WAIT_LIMIT; ++i)
-    if (pt_try_wait(bar, parity)) return true;
-  return false;
 }
 // K-major operand tile, 128-byte swizzle: 8-row groups 1024 bytes apart (see rap_proj_tc.cu)
 __device__ __forceinline__ uint64_t pt_desc(uint32_t addr) {
@@ -69,6 +68,9 @@ __device__ __forceinline__ void pt_ld32(uint32_t taddr, uint32_t (&r)[32]) {
       : "memory");
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
+__device__ __forceinline__ void pt_cp4(uint32_t dst, const void* src, uint32_t src_bytes) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
 __device__ __forceinline__ float pt_ex2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -79,6 +81,20 @@ __device__ __forceinline__ float pt_ex2(float x) {
 __device__ __forceinline__ uint32_t pt_off(int row, int col, int rows) {
   const int ac = col >> 6, c = col & 63;
   return (uint32_t)(ac * rows * 128 + (row >> 3) * 1024 + (row & 7) * 128 + ((((c >> 3) ^ (row & 7))) << 4) + ((c & 7) << 1));
+}
+
+// N-major operand tile (B = V as stored, [key][channel]), 128-byte swizzle: an atom is 8 keys x 64 channels
+// (key rows of 128 bytes, 16-byte chunks XORed with key % 8); atoms of consecutive 8-key groups are 1024 bytes
+// apart (stride offset), the two 64-channel atom columns 16 KB apart (leading offset).
+__device__ __forceinline__ uint64_t pt_desc_n(uint32_t addr) {
+  const uint32_t lo = ((addr & 0x3FFFFu) >> 4) | ((16384u >> 4) << 16);
+  const uint32_t hi = (1024u >> 4) | (1u << 14) | (2u << 29);
+  return ((uint64_t)hi << 32) | lo;
+}
+// byte offset of (key, channel) in that tile
+__device__ __forceinline__ uint32_t pt_off_n(int key, int ch) {
+  const int c = ch & 63;
+  return (uint32_t)((ch >> 6) * 16384 + (key >> 3) * 1024 + (key & 7) * 128 + ((((c >> 3) ^ (key & 7))) << 4) + ((c & 7) << 1));
 }
 
 struct PtParams {
@@ -94,16 +110,20 @@ struct PtParams {
 
 // DK = k-steps of Q K^T (ceil(2P / 16)); NVP = d_v' rounded up to a multiple of 32 (N of the second MMA)
 template <int DK, int NVP>
-__global__ void __launch_bounds__(PT_THREADS, 2) prefill_tc_kernel(const PtParams p) {
+__global__ void __launch_bounds__(PT_THREADS, 1) prefill_tc_kernel(const PtParams p) {
   extern __shared__ unsigned char pt_raw[];
   unsigned char* smem = pt_raw + ((1024u - (pt_smem(pt_raw) & 1023u)) & 1023u);
-  unsigned char* q_s = smem;                         // [128 queries][<=128 dims]
-  unsigned char* k_s = q_s + PT_TILE_BYTES;          // [128 keys][<=128 dims]
-  unsigned char* v_s = k_s + PT_TILE_BYTES;          // [NVP channels][128 keys]   (V transposed)
-  unsigned char* p_s = k_s;                          // [128 queries][128 keys]: reuses the K tile, which the
-                                                     // first MMA has finished reading when P is written
-  const uint32_t bar_s = pt_smem(v_s + PT_TILE_BYTES), bar_o = bar_s + 8;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(v_s + PT_TILE_BYTES + 16);
+  unsigned char* q_s = smem;                                   // [128 queries][<=128 dims]
+  unsigned char* p_s = q_s + PT_TILE_BYTES;                    // [128 queries][128 keys]
+  unsigned char* k_s = p_s + PT_TILE_BYTES;                    // two stages of [128 keys][<=128 dims]
+  unsigned char* v_s = k_s + 2 * PT_TILE_BYTES;                // two stages of [128 keys][<=128 channels] (N-major)
+  unsigned char* tail = v_s + 2 * PT_TILE_BYTES;
+  // mbarriers: K/V stage filled (producers -> MMA), stage free (second MMA done -> producers), S ready (first
+  // MMA done -> softmax), P written (softmax -> MMA), O_tile ready (second MMA done -> softmax), drain
+  const uint32_t bar_full = pt_smem(tail), bar_empty = bar_full + 16, bar_s = bar_full + 32, bar_p = bar_full + 48,
+                 bar_o = bar_full + 56, bar_end = bar_full + 64;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 80);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 96);
 
   const int qb = blockIdx.x, g = blockIdx.y, b = blockIdx.z;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -117,17 +137,24 @@ __global__ void __launch_bounds__(PT_THREADS, 2) prefill_tc_kernel(const PtParam
   const __nv_bfloat16* vg = p.v + ((size_t)b * p.Hkv + h) * (size_t)p.S_cap * p.dv;
 
   if (tid == 0) {
-    pt_mbar_init(bar_s, 1);
+    for (int i = 0; i < 2; ++i) {
+      pt_mbar_init(bar_full + 8 * i, PT_PRODUCERS);
+      pt_mbar_init(bar_empty + 8 * i, 1);
+      pt_mbar_init(bar_s + 8 * i, 1);
+    }
+    pt_mbar_init(bar_p, 128);
     pt_mbar_init(bar_o, 1);
+    pt_mbar_init(bar_end, 1);
+    *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 4) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(pt_smem(tmem_slot)), "r"(256)
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(pt_smem(tmem_slot)), "r"(512)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-  // zero all four tiles once (pad columns and pad channel rows are never written again), then stage Q
-  for (int i = tid; i < 3 * PT_TILE_BYTES / 16; i += PT_THREADS) reinterpret_cast<uint4*>(smem)[i] = make_uint4(0, 0, 0, 0);
+  // zero all six tiles once (pad columns and pad channel rows are never written again), then stage Q
+  for (int i = tid; i < 6 * PT_TILE_BYTES / 16; i += PT_THREADS) reinterpret_cast<uint4*>(smem)[i] = make_uint4(0, 0, 0, 0);
   __syncthreads();
   const int kw = p.P2 >> 1;                          // 4-byte words per q / K row
   for (int r = warp; r < PT_BM; r += PT_THREADS / 32) {
@@ -137,80 +164,172 @@ __global__ void __launch_bounds__(PT_THREADS, 2) prefill_tc_kernel(const PtParam
       for (int w = lane; w < kw; w += 32) *reinterpret_cast<uint32_t*>(q_s + pt_off(r, 2 * w, PT_BM)) = src[w];
     }
   }
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-  const uint32_t tmem_s = *tmem_slot, tmem_o = tmem_s + 128;
+  const uint32_t tmem_base = *tmem_slot;             // S of tile t in columns [128 (t & 1), +128), O_tile in [256, 256 + NVP)
+  const uint32_t tmem_o = tmem_base + 256;
   constexpr uint32_t IDESC_S = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(PT_BN >> 3) << 17) | ((uint32_t)(PT_BM >> 4) << 24);
-  constexpr uint32_t IDESC_O = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(NVP >> 3) << 17) | ((uint32_t)(PT_BM >> 4) << 24);
+  // second MMA: B = V is N-major (bit 16)
+  constexpr uint32_t IDESC_O = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(NVP >> 3) << 17) |
+                               ((uint32_t)(PT_BM >> 4) << 24);
+  // a wait that gives up when its limit runs out or another role has given up; the loser raises the flag
+  auto wait = [&](uint32_t bar, uint32_t parity) -> bool {
+    for (uint32_t i = 0; i < PT_WAIT_LIMIT; ++i) {
+      if (pt_try_wait(bar, parity)) return true;
+      if (i >= 4) __nanosleep(64);                   // a long wait leaves the issue slots to the working warps
+      if ((i & 255u) == 255u && *abort_flag) return false;
+    }
+    *abort_flag = 1;
+    return false;
+  };
 
-  const int row = tid;                               // warps 0-3: query row = TMEM lane
-  const int pos = start + q0 + row;                  // cache row of this thread's query
+  if (warp >= 5) {
+    // ================= producers: stage K (as stored) and V (transposed) one tile ahead =================
+    const int pw = warp - 5;
+    const int vw = p.dv >> 1;
+    const bool v_even = (p.dv & 1) == 0;
+    uint32_t swz[2][2];                              // [row parity class][word slot]: in-row byte offset
+#pragma unroll
+    for (int c = 0; c < 2; ++c)
+#pragma unroll
+      for (int sl = 0; sl < 2; ++sl) {
+        const int w = lane + 32 * sl, r7 = (pw + 4 * c) & 7;
+        swz[c][sl] = (uint32_t)((w >> 5) * 16384 + ((((w & 31) >> 2) ^ r7) << 4) + (w & 3) * 4);
+      }
+    for (int tile = 0; tile < n_tiles; ++tile) {
+      const int stg = tile & 1, j0 = tile * PT_BN;
+      if (tile >= 2 && !wait(bar_empty + 8 * stg, ((tile >> 1) - 1) & 1)) break;
+      unsigned char* kd = k_s + stg * PT_TILE_BYTES;
+      unsigned char* vd = v_s + stg * PT_TILE_BYTES;
+      // K and V share one tile layout: word w of row r sits at (w / 32) 16 KB + r 128 + swizzled chunk.  A lane
+      // keeps its words (lane, lane + 32) and walks the rows pw, pw + 4, ...: r % 8 takes two values, so the
+      // swizzled in-row offsets are four constants per lane and a copy costs a few instructions.
+      const uint32_t kdu = pt_smem(kd), vdu = pt_smem(vd);
+      const int rows_ok = min(PT_BN, n_valid - j0);              // rows of this tile that exist (>= 1)
+#pragma unroll 2
+      for (int i = 0; i < PT_BN / 4; ++i) {
+        const int r = pw + 4 * i;
+        const uint32_t sz = r < rows_ok ? 4u : 0u;               // zero fill past the end
+        const size_t grow = (size_t)(j0 + (r < rows_ok ? r : 0));
+        const uint32_t* ksrc = reinterpret_cast<const uint32_t*>(kg + grow * p.P2);
+        const uint32_t rb = (uint32_t)r * 128u;
+        const uint32_t* sw = swz[i & 1];
+        if (lane < kw) pt_cp4(kdu + rb + sw[0], ksrc + lane, sz);
+        if (lane + 32 < kw) pt_cp4(kdu + rb + sw[1], ksrc + lane + 32, sz);
+        if (v_even) {
+          const uint32_t* vsrc = reinterpret_cast<const uint32_t*>(vg + grow * p.dv);
+          if (lane < vw) pt_cp4(vdu + rb + sw[0], vsrc + lane, sz);
+          if (lane + 32 < vw) pt_cp4(vdu + rb + sw[1], vsrc + lane + 32, sz);
+        }
+      }
+      if (!v_even) {   // rows of an odd d_v' are only 2-byte aligned: element by element
+        for (int r = pw; r < PT_BN; r += PT_PRODUCERS / 32) {
+          const bool ok = r < rows_ok;
+          const __nv_bfloat16* vsrc = vg + (size_t)(j0 + (ok ? r : 0)) * p.dv;
+          for (int c = lane; c < p.dv; c += 32)
+            *reinterpret_cast<__nv_bfloat16*>(vd + pt_off_n(r, c)) = ok ? vsrc[c] : __float2bfloat16(0.f);
+        }
+      }
+      asm volatile("cp.async.commit_group;" ::: "memory");
+      asm volatile("cp.async.wait_group 0;" ::: "memory");
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> tensor-core (async proxy) reads
+      asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar_full + 8 * stg) : "memory");
+    }
+  } else if (warp == 4) {
+    // ================= MMA issue: S(t + 1) = Q K^T is issued before P(t) is waited for =================
+    if (lane == 0) {
+      auto issue_s = [&](int tile) {
+        const uint32_t kb = pt_smem(k_s + (tile & 1) * PT_TILE_BYTES), td = tmem_base + 128u * (uint32_t)(tile & 1);
+#pragma unroll
+        for (int ks = 0; ks < DK; ++ks) {
+          const uint32_t o2 = (uint32_t)((ks >> 2) * PT_BM * 128 + (ks & 3) * 32);
+          pt_mma(td, pt_desc(pt_smem(q_s) + o2), pt_desc(kb + o2), IDESC_S, ks > 0 ? 1u : 0u);
+        }
+        pt_commit(bar_s + 8 * (tile & 1));
+      };
+      bool ok = wait(bar_full, 0);
+      if (ok) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        issue_s(0);
+      }
+      for (int tile = 0; ok && tile < n_tiles; ++tile) {
+        if (tile + 1 < n_tiles) {
+          if (!wait(bar_full + 8 * ((tile + 1) & 1), ((tile + 1) >> 1) & 1)) { ok = false; break; }
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          issue_s(tile + 1);
+        }
+        if (!wait(bar_p, tile & 1)) { ok = false; break; }
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint32_t vb = pt_smem(v_s + (tile & 1) * PT_TILE_BYTES);
+#pragma unroll
+        for (int ks = 0; ks < PT_BN / 16; ++ks) {
+          const uint32_t oa = (uint32_t)((ks >> 2) * PT_BM * 128 + (ks & 3) * 32);
+          // 16 keys = two 8-key groups of the N-major V tile
+          pt_mma(tmem_o, pt_desc(pt_smem(p_s) + oa), pt_desc_n(vb + (uint32_t)ks * 2048u), IDESC_O, ks > 0 ? 1u : 0u);
+        }
+        pt_commit(bar_o);
+        pt_commit(bar_empty + 8 * (tile & 1));
+      }
+      // every MMA issued above has completed before tensor memory is released
+      pt_commit(bar_end);
+      wait(bar_end, 0);
+    }
+    __syncwarp();
+  }
   float o[NVP];
+  float l_run = 0.f;
+  const int row = tid;                               // warps 0-3: query row = TMEM lane
+  if (warp < 4) {
+    // ================= softmax and output rows: one thread per query =================
+    const int pos = start + q0 + row;                // cache row of this thread's query
 #pragma unroll
-  for (int c = 0; c < NVP; ++c) o[c] = 0.f;
-  float m_ref = -1.0e30f, l_run = 0.f;
-  bool timed_out = false;
-  uint32_t phase = 0;
-
-  for (int tile = 0; tile < n_tiles; ++tile) {
-    const int j0 = tile * PT_BN;
-    // ---- stage K (as stored) and V (transposed); rows past the end become zeros ------------------------
-    // K: 4-byte cp.async straight to the swizzled position (zero fill past the end), all in flight at once;
-    // V: eight rows per pass so that eight independent loads are in flight before the transposed stores
-    for (int r = warp; r < PT_BN; r += PT_THREADS / 32) {
-      const bool ok = j0 + r < n_valid;
-      const __nv_bfloat16* ksrc = kg + (size_t)(ok ? j0 + r : 0) * p.P2;
-      for (int w = lane; w < kw; w += 32)
-        asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(pt_smem(k_s + pt_off(r, 2 * w, PT_BN))),
-                     "l"(ksrc + 2 * w), "r"(ok ? 4 : 0)
-                     : "memory");
-    }
-    asm volatile("cp.async.commit_group;" ::: "memory");
-    for (int r0 = 8 * warp; r0 < PT_BN; r0 += 8 * (PT_THREADS / 32)) {
-      for (int c = lane; c < p.dv; c += 32) {
-        __nv_bfloat16 vals[8];
-#pragma unroll
-        for (int i = 0; i < 8; ++i)
-          vals[i] = j0 + r0 + i < n_valid ? vg[(size_t)(j0 + r0 + i) * p.dv + c] : __float2bfloat16(0.f);
-        // rows r0 .. r0+7 of channel c are one 16-byte chunk of the transposed tile
-        *reinterpret_cast<uint4*>(v_s + pt_off(c, r0, NVP)) = *reinterpret_cast<const uint4*>(vals);
-      }
-    }
-    asm volatile("cp.async.wait_group 0;" ::: "memory");
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> tensor-core (async proxy) reads
-    __syncthreads();
-    // ---- S = Q K^T ----------------------------------------------------------------------------------------
-    if (warp == 4 && lane == 0) {
-      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-#pragma unroll
-      for (int ks = 0; ks < DK; ++ks) {
-        const uint32_t o2 = (uint32_t)((ks >> 2) * PT_BM * 128 + (ks & 3) * 32);
-        pt_mma(tmem_s, pt_desc(pt_smem(q_s) + o2), pt_desc(pt_smem(k_s) + o2), IDESC_S, ks > 0 ? 1u : 0u);
-      }
-      pt_commit(bar_s);
-    }
-    float alpha = 1.f;
-    if (warp < 4) {
-      if (!pt_wait(bar_s, phase)) timed_out = true;
-      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      const uint32_t trow = tmem_s + ((uint32_t)(warp * 32) << 16);
-      // pass 1: the row's maximum over the allowed keys of the tile
+    for (int c = 0; c < NVP; ++c) o[c] = 0.f;
+    float m_ref = -1.0e30f;
+    const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
+    // pass 1 of a tile: the row's maximum over the allowed keys; lazy reference maximum (p stays <= 2^8).
+    // Only the tiles that reach past the block's first query need the causal mask.
+    auto pass1 = [&](int tile) -> float {
+      const uint32_t trow = tmem_base + 128u * (uint32_t)(tile & 1) + lane_off;
+      const int j0 = tile * PT_BN;
+      const bool interior = j0 + PT_BN - 1 <= start + q0;
       float mx = -INFINITY;
 #pragma unroll 1
       for (int c0 = 0; c0 < PT_BN; c0 += 32) {
         uint32_t r[32];
         pt_ld32(trow + c0, r);
+        if (interior) {
 #pragma unroll
-        for (int j = 0; j < 32; ++j)
-          if (j0 + c0 + j <= pos) mx = fmaxf(mx, __uint_as_float(r[j]) * p.qscale);
+          for (int j = 0; j < 32; ++j) mx = fmaxf(mx, __uint_as_float(r[j]));
+        } else {
+#pragma unroll
+          for (int j = 0; j < 32; ++j)
+            if (j0 + c0 + j <= pos) mx = fmaxf(mx, __uint_as_float(r[j]));
+        }
       }
-      if (mx > m_ref + 8.f) {          // lazy reference maximum: p stays <= 2^8
+      mx *= p.qscale;                  // the scale is positive: the maximum commutes with it
+      float alpha = 1.f;
+      if (mx > m_ref + 8.f) {
         alpha = pt_ex2(m_ref - mx);    // first time: 2^(-1e30 - mx) = 0
         m_ref = mx;
         l_run *= alpha;
       }
-      // pass 2: p = 2^(s - m_ref), bf16, into the A-operand layout (this thread's row, 16 chunks of 8 keys)
+      return alpha;
+    };
+    bool ok = wait(bar_s, 0);
+    float alpha_t = 1.f;
+    if (ok) {
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      alpha_t = pass1(0);
+    }
+    for (int tile = 0; ok && tile < n_tiles; ++tile) {
+      const int j0 = tile * PT_BN;
+      const uint32_t trow = tmem_base + 128u * (uint32_t)(tile & 1) + lane_off;
+      // pass 2: p = 2^(s - m_ref), bf16, into the A-operand layout (this thread's row, 16 chunks of 8 keys);
+      // the second MMA of the previous tile, which read P, has completed (its O_tile was waited for below)
+      const bool interior = j0 + PT_BN - 1 <= start + q0;
+      const float nm = -m_ref;
 #pragma unroll 1
       for (int c0 = 0; c0 < PT_BN; c0 += 32) {
         uint32_t r[32];
@@ -218,11 +337,14 @@ __global__ void __launch_bounds__(PT_THREADS, 2) prefill_tc_kernel(const PtParam
         uint32_t pk[16];
 #pragma unroll
         for (int j = 0; j < 32; j += 2) {
-          const float p0 = j0 + c0 + j <= pos ? pt_ex2(__uint_as_float(r[j]) * p.qscale - m_ref) : 0.f;
-          const float p1 = j0 + c0 + j + 1 <= pos ? pt_ex2(__uint_as_float(r[j + 1]) * p.qscale - m_ref) : 0.f;
+          float p0 = pt_ex2(fmaf(__uint_as_float(r[j]), p.qscale, nm));
+          float p1 = pt_ex2(fmaf(__uint_as_float(r[j + 1]), p.qscale, nm));
+          if (!interior) {
+            if (j0 + c0 + j > pos) p0 = 0.f;
+            if (j0 + c0 + j + 1 > pos) p1 = 0.f;
+          }
+          l_run += p0 + p1;
           const __nv_bfloat162 v2 = __floats2bfloat162_rn(p0, p1);
-          // the row sum uses the rounded values the second MMA will see
-          l_run += __bfloat162float(v2.x) + __bfloat162float(v2.y);
           pk[j >> 1] = *reinterpret_cast<const uint32_t*>(&v2);
         }
 #pragma unroll
@@ -232,37 +354,31 @@ __global__ void __launch_bounds__(PT_THREADS, 2) prefill_tc_kernel(const PtParam
       }
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-    }
-    if (__syncthreads_or(timed_out)) { timed_out = true; break; }
-    // ---- O_tile = P V -----------------------------------------------------------------------------------------
-    if (warp == 4 && lane == 0) {
-      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-#pragma unroll
-      for (int ks = 0; ks < PT_BN / 16; ++ks) {
-        const uint32_t oa = (uint32_t)((ks >> 2) * PT_BM * 128 + (ks & 3) * 32);
-        const uint32_t ob = (uint32_t)((ks >> 2) * NVP * 128 + (ks & 3) * 32);
-        pt_mma(tmem_o, pt_desc(pt_smem(p_s) + oa), pt_desc(pt_smem(v_s) + ob), IDESC_O, ks > 0 ? 1u : 0u);
+      asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar_p) : "memory");
+      // while the second MMA runs: the maximum of the next tile, whose S is already in tensor memory
+      float alpha_next = 1.f;
+      if (tile + 1 < n_tiles) {
+        if (!wait(bar_s + 8 * ((tile + 1) & 1), ((tile + 1) >> 1) & 1)) { ok = false; break; }
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        alpha_next = pass1(tile + 1);
       }
-      pt_commit(bar_o);
-    }
-    // everybody waits for the second MMA: the next tile's staging overwrites what it reads
-    if (!pt_wait(bar_o, phase)) timed_out = true;
-    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    if (warp < 4) {
-      const uint32_t trow = tmem_o + ((uint32_t)(warp * 32) << 16);
+      if (!wait(bar_o, tile & 1)) { ok = false; break; }
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const uint32_t orow = tmem_o + lane_off;
 #pragma unroll
       for (int c0 = 0; c0 < NVP; c0 += 32) {
         uint32_t r[32];
-        pt_ld32(trow + c0, r);
+        pt_ld32(orow + c0, r);
 #pragma unroll
-        for (int j = 0; j < 32; ++j) o[c0 + j] = o[c0 + j] * alpha + __uint_as_float(r[j]);
+        for (int j = 0; j < 32; ++j) o[c0 + j] = o[c0 + j] * alpha_t + __uint_as_float(r[j]);
       }
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      alpha_t = alpha_next;
     }
-    phase ^= 1u;
-    if (__syncthreads_or(timed_out)) { timed_out = true; break; }
   }
-
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  const bool timed_out = *abort_flag != 0;
   if (timed_out && tid == 0) {
     atomicCAS(&p.status[0], 0, (int)RAP_ETIMEOUT);
     p.status[1] = 0x60000000 | (blockIdx.x & 0xffffff);
@@ -277,17 +393,15 @@ __global__ void __launch_bounds__(PT_THREADS, 2) prefill_tc_kernel(const PtParam
         if (c < p.dv) dst[c] = o[c] * inv;
     }
   }
-  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-  __syncthreads();
   if (warp == 4) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_s), "r"(256) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
   }
 }
 
 template <int DK, int NVP>
 rap_status launch_pt(rap_ctx* ctx, const PtParams& p, int B, cudaStream_t st) {
-  const int smem = 3 * PT_TILE_BYTES + 64 + 1024;
+  const int smem = 6 * PT_TILE_BYTES + 128 + 1024;
   RAP_CUDA_TRY(ctx, rap_raise_smem(ctx, prefill_tc_kernel<DK, NVP>, smem));
   dim3 grid((p.T + PT_BM - 1) / PT_BM, p.Hq, B);
   prefill_tc_kernel<DK, NVP><<<grid, PT_THREADS, smem, st>>>(p);
