@@ -10,7 +10,8 @@
 //                       the row's thread then folds O_tile into its register accumulator with the rescale
 //                       factor, so tensor memory never has to be rewritten.
 // Cache rows are not multiples of 16 bytes, so TMA tensor maps cannot describe them: four producer warps stage
-// the tiles by hand (4-byte cp.async), one tile ahead in a two-stage ring, into the 128-byte-swizzled layouts
+// the tiles by hand (4-byte cp.async), two tiles ahead (K in a ring of three buffers, V of two), into the
+// 128-byte-swizzled layouts
 // the MMA descriptors expect (K as stored = K-major; V as stored = the N-major form of the B operand, so nothing
 // is transposed); rows past the sequence end and pad columns are zeros.  The roles (4 softmax warps, 1 MMA-issuing lane, 4 producer warps) meet only on mbarriers; every
 // wait is bounded and gives up early once another role has given up.
@@ -21,7 +22,8 @@
 namespace {
 
 constexpr int PT_BM = 128, PT_BN = 128;
-constexpr int PT_THREADS = 288, PT_PRODUCERS = 128;   // warps 0-3: rows / softmax, warp 4: MMA issue, warps 5-8: staging
+constexpr int PT_THREADS = 288;   // warps 0-3: rows / softmax, warp 4: MMA issue, warps 5-6: K staging, warps 7-8: V staging
+constexpr int PT_KSTAGES = 3, PT_VSTAGES = 2;
 constexpr int PT_TILE_BYTES = 2 * 128 * 128;                     // two 64-element atom columns of 128 rows
 constexpr uint32_t PT_WAIT_LIMIT = 1u << 21;
 
@@ -68,7 +70,31 @@ __device__ __forceinline__ void pt_ld32(uint32_t taddr, uint32_t (&r)[32]) {
       : "memory");
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
-__device__ __forceinline__ void pt_cp4(uint32_t dst, const void* src, uint32_t src_bytes) {
+__device__ __forceinline__ void pt_ld32_nowait(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void pt_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+      "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+      "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};" ::"r"(taddr),
+      "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]),
+      "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]), "r"(r[18]),
+      "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]),
+      "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+      : "memory");
+}
+// 4-byte cp.async; the first src_bytes come from memory, the rest of the copy is zero-filled
+__device__ __forceinline__ void pt_cp4(uint32_t dst, const void* src, int src_bytes) {
   asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
 }
 __device__ __forceinline__ float pt_ex2(float x) {
@@ -91,10 +117,31 @@ __device__ __forceinline__ uint64_t pt_desc_n(uint32_t addr) {
   const uint32_t hi = (1024u >> 4) | (1u << 14) | (2u << 29);
   return ((uint64_t)hi << 32) | lo;
 }
-// byte offset of (key, channel) in that tile
-__device__ __forceinline__ uint32_t pt_off_n(int key, int ch) {
-  const int c = ch & 63;
-  return (uint32_t)((ch >> 6) * 16384 + (key >> 3) * 1024 + (key & 7) * 128 + ((((c >> 3) ^ (key & 7))) << 4) + ((c & 7) << 1));
+// Byte offset inside a tile row of its byte e: 64-element (128-byte) atom columns 16 KB apart, 16-byte chunks
+// XORed with row % 8 (the layout is the same for the K-major K tile and the N-major V tile).
+__device__ __forceinline__ uint32_t pt_swz(int e, int r7) {
+  const int w = e >> 2;
+  return (uint32_t)(((w >> 5) << 14) + ((((w & 31) >> 2) ^ r7) << 4) + ((w & 3) << 2));
+}
+// The odd rows (1, 3, ..., 127) of a tile with an odd row length start 2 bytes off a word.  Channel pair (2w, 2w+1) is
+// the high half of one aligned word and the low half of the next; the last word holds one channel.
+__device__ __forceinline__ void pt_stage_odd_rows(uint32_t du, const unsigned char* tile_src, int rowlen, int rows_ok,
+                                                  int lane) {
+  const int wl = (rowlen - 1) >> 1;
+#pragma unroll 2
+  for (int r = 1; r < 128; r += 2) {
+    const bool ok = r < rows_ok;
+    const uint32_t* g = reinterpret_cast<const uint32_t*>(tile_src + (size_t)r * rowlen * 2 - 2);
+    const uint32_t dst = du + (uint32_t)r * 128u;
+    for (int w = lane; w <= wl; w += 32) {
+      uint32_t val = 0u;                               // rows past the end: zeros, and nothing is read
+      if (ok) {
+        const uint32_t a = g[w], b2 = w < wl ? g[w + 1] : 0u;
+        asm("prmt.b32 %0, %1, %2, 0x5432;" : "=r"(val) : "r"(a), "r"(b2));
+      }
+      asm volatile("st.shared.u32 [%0], %1;" ::"r"(dst + pt_swz(4 * w, r & 7)), "r"(val) : "memory");
+    }
+  }
 }
 
 struct PtParams {
@@ -115,15 +162,15 @@ __global__ void __launch_bounds__(PT_THREADS, 1) prefill_tc_kernel(const PtParam
   unsigned char* smem = pt_raw + ((1024u - (pt_smem(pt_raw) & 1023u)) & 1023u);
   unsigned char* q_s = smem;                                   // [128 queries][<=128 dims]
   unsigned char* p_s = q_s + PT_TILE_BYTES;                    // [128 queries][128 keys]
-  unsigned char* k_s = p_s + PT_TILE_BYTES;                    // two stages of [128 keys][<=128 dims]
-  unsigned char* v_s = k_s + 2 * PT_TILE_BYTES;                // two stages of [128 keys][<=128 channels] (N-major)
-  unsigned char* tail = v_s + 2 * PT_TILE_BYTES;
-  // mbarriers: K/V stage filled (producers -> MMA), stage free (second MMA done -> producers), S ready (first
-  // MMA done -> softmax), P written (softmax -> MMA), O_tile ready (second MMA done -> softmax), drain
-  const uint32_t bar_full = pt_smem(tail), bar_empty = bar_full + 16, bar_s = bar_full + 32, bar_p = bar_full + 48,
-                 bar_o = bar_full + 56, bar_end = bar_full + 64;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 80);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 96);
+  unsigned char* k_s = p_s + PT_TILE_BYTES;                    // ring of [128 keys][<=128 dims]
+  unsigned char* v_s = k_s + PT_KSTAGES * PT_TILE_BYTES;       // ring of [128 keys][<=128 channels] (N-major)
+  unsigned char* tail = v_s + PT_VSTAGES * PT_TILE_BYTES;
+  // mbarriers: K / V buffer filled (producers -> MMA), buffer free (the MMA that read it is done -> producers),
+  // S ready (first MMA done -> softmax), P written (softmax -> MMA), O updated (second MMA done -> softmax), drain
+  const uint32_t bar_fk = pt_smem(tail), bar_ek = bar_fk + 24, bar_fv = bar_fk + 48, bar_ev = bar_fk + 64,
+                 bar_s = bar_fk + 80, bar_p = bar_fk + 96, bar_o = bar_fk + 104, bar_end = bar_fk + 112;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 120);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 124);
 
   const int qb = blockIdx.x, g = blockIdx.y, b = blockIdx.z;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -137,11 +184,15 @@ __global__ void __launch_bounds__(PT_THREADS, 1) prefill_tc_kernel(const PtParam
   const __nv_bfloat16* vg = p.v + ((size_t)b * p.Hkv + h) * (size_t)p.S_cap * p.dv;
 
   if (tid == 0) {
-    for (int i = 0; i < 2; ++i) {
-      pt_mbar_init(bar_full + 8 * i, PT_PRODUCERS);
-      pt_mbar_init(bar_empty + 8 * i, 1);
-      pt_mbar_init(bar_s + 8 * i, 1);
+    for (int i = 0; i < PT_KSTAGES; ++i) {
+      pt_mbar_init(bar_fk + 8 * i, 64);
+      pt_mbar_init(bar_ek + 8 * i, 1);
     }
+    for (int i = 0; i < PT_VSTAGES; ++i) {
+      pt_mbar_init(bar_fv + 8 * i, 64);
+      pt_mbar_init(bar_ev + 8 * i, 1);
+    }
+    for (int i = 0; i < 2; ++i) pt_mbar_init(bar_s + 8 * i, 1);
     pt_mbar_init(bar_p, 128);
     pt_mbar_init(bar_o, 1);
     pt_mbar_init(bar_end, 1);
@@ -154,7 +205,7 @@ __global__ void __launch_bounds__(PT_THREADS, 1) prefill_tc_kernel(const PtParam
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   // zero all six tiles once (pad columns and pad channel rows are never written again), then stage Q
-  for (int i = tid; i < 6 * PT_TILE_BYTES / 16; i += PT_THREADS) reinterpret_cast<uint4*>(smem)[i] = make_uint4(0, 0, 0, 0);
+  for (int i = tid; i < (2 + PT_KSTAGES + PT_VSTAGES) * PT_TILE_BYTES / 16; i += PT_THREADS) reinterpret_cast<uint4*>(smem)[i] = make_uint4(0, 0, 0, 0);
   __syncthreads();
   const int kw = p.P2 >> 1;                          // 4-byte words per q / K row
   for (int r = warp; r < PT_BM; r += PT_THREADS / 32) {
@@ -186,91 +237,90 @@ __global__ void __launch_bounds__(PT_THREADS, 1) prefill_tc_kernel(const PtParam
   };
 
   if (warp >= 5) {
-    // ================= producers: stage K (as stored) and V (transposed) one tile ahead =================
-    const int pw = warp - 5;
-    const int vw = p.dv >> 1;
-    const bool v_even = (p.dv & 1) == 0;
-    uint32_t swz[2][2];                              // [row parity class][word slot]: in-row byte offset
+    // ================= producers: warps 5-6 stage K (three buffers), warps 7-8 stage V (two buffers) =================
+    // A warp takes every second row in order (neighbouring rows share cache lines and are fetched together by the
+    // two warps); a lane keeps its words (lane, lane + 32) of every row.  r % 8 takes four values per warp, so the
+    // swizzled in-row offsets are eight constants per lane and a copy costs a few instructions.
+    const bool is_v = warp >= 7;
+    const int pw = (warp - 5) & 1;
+    const int rowlen = is_v ? p.dv : p.P2;             // elements per row
+    const unsigned char* src0 = reinterpret_cast<const unsigned char*>(is_v ? vg : kg);
+    const int nst = is_v ? PT_VSTAGES : PT_KSTAGES;
+    unsigned char* ring = is_v ? v_s : k_s;
+    const uint32_t bar_f = is_v ? bar_fv : bar_fk, bar_e = is_v ? bar_ev : bar_ek;
+    const bool odd_rows = (rowlen & 1) && pw == 1;     // odd rows of an odd d_v' are only 2-byte aligned
+    uint32_t swz[4][2];                                // [row class][word slot]: in-row byte offset
+    int nb[2];                                         // bytes this lane copies per slot (0: none; 2: the half-filled word)
 #pragma unroll
-    for (int c = 0; c < 2; ++c)
+    for (int sl = 0; sl < 2; ++sl) {
+      const int w = lane + 32 * sl;
+      nb[sl] = min(4, max(0, 2 * rowlen - 4 * w));
 #pragma unroll
-      for (int sl = 0; sl < 2; ++sl) {
-        const int w = lane + 32 * sl, r7 = (pw + 4 * c) & 7;
-        swz[c][sl] = (uint32_t)((w >> 5) * 16384 + ((((w & 31) >> 2) ^ r7) << 4) + (w & 3) * 4);
-      }
+      for (int c = 0; c < 4; ++c) swz[c][sl] = pt_swz(4 * w, (pw + 2 * c) & 7);
+    }
+    int stg = 0, use = 0;                              // buffer of this tile and how often it has been used before
     for (int tile = 0; tile < n_tiles; ++tile) {
-      const int stg = tile & 1, j0 = tile * PT_BN;
-      if (tile >= 2 && !wait(bar_empty + 8 * stg, ((tile >> 1) - 1) & 1)) break;
-      unsigned char* kd = k_s + stg * PT_TILE_BYTES;
-      unsigned char* vd = v_s + stg * PT_TILE_BYTES;
-      // K and V share one tile layout: word w of row r sits at (w / 32) 16 KB + r 128 + swizzled chunk.  A lane
-      // keeps its words (lane, lane + 32) and walks the rows pw, pw + 4, ...: r % 8 takes two values, so the
-      // swizzled in-row offsets are four constants per lane and a copy costs a few instructions.
-      const uint32_t kdu = pt_smem(kd), vdu = pt_smem(vd);
-      const int rows_ok = min(PT_BN, n_valid - j0);              // rows of this tile that exist (>= 1)
-#pragma unroll 2
-      for (int i = 0; i < PT_BN / 4; ++i) {
-        const int r = pw + 4 * i;
-        const uint32_t sz = r < rows_ok ? 4u : 0u;               // zero fill past the end
-        const size_t grow = (size_t)(j0 + (r < rows_ok ? r : 0));
-        const uint32_t* ksrc = reinterpret_cast<const uint32_t*>(kg + grow * p.P2);
-        const uint32_t rb = (uint32_t)r * 128u;
-        const uint32_t* sw = swz[i & 1];
-        if (lane < kw) pt_cp4(kdu + rb + sw[0], ksrc + lane, sz);
-        if (lane + 32 < kw) pt_cp4(kdu + rb + sw[1], ksrc + lane + 32, sz);
-        if (v_even) {
-          const uint32_t* vsrc = reinterpret_cast<const uint32_t*>(vg + grow * p.dv);
-          if (lane < vw) pt_cp4(vdu + rb + sw[0], vsrc + lane, sz);
-          if (lane + 32 < vw) pt_cp4(vdu + rb + sw[1], vsrc + lane + 32, sz);
-        }
-      }
-      if (!v_even) {   // rows of an odd d_v' are only 2-byte aligned: element by element
-        for (int r = pw; r < PT_BN; r += PT_PRODUCERS / 32) {
-          const bool ok = r < rows_ok;
-          const __nv_bfloat16* vsrc = vg + (size_t)(j0 + (ok ? r : 0)) * p.dv;
-          for (int c = lane; c < p.dv; c += 32)
-            *reinterpret_cast<__nv_bfloat16*>(vd + pt_off_n(r, c)) = ok ? vsrc[c] : __float2bfloat16(0.f);
+      const int j0 = tile * PT_BN;
+      if (use > 0 && !wait(bar_e + 8 * stg, (use - 1) & 1)) break;
+      const uint32_t du = pt_smem(ring + stg * PT_TILE_BYTES);
+      const int rows_ok = min(PT_BN, n_valid - j0);    // rows of this tile that exist (>= 1)
+      const unsigned char* tsrc = src0 + (size_t)j0 * (size_t)(2 * rowlen);
+      if (odd_rows) {
+        pt_stage_odd_rows(du, tsrc, rowlen, rows_ok, lane);
+      } else {
+#pragma unroll 4
+        for (int i = 0; i < PT_BN / 2; ++i) {
+          const int r = pw + 2 * i;
+          const bool ok = r < rows_ok;                 // rows past the end: zero fill, nothing is read
+          const uint32_t* src = reinterpret_cast<const uint32_t*>(tsrc + (size_t)(ok ? r : 0) * (size_t)(2 * rowlen));
+          const uint32_t rb = du + (uint32_t)r * 128u;
+          if (nb[0] > 0) pt_cp4(rb + swz[i & 3][0], src + lane, ok ? nb[0] : 0);
+          if (nb[1] > 0) pt_cp4(rb + swz[i & 3][1], src + lane + 32, ok ? nb[1] : 0);
         }
       }
       asm volatile("cp.async.commit_group;" ::: "memory");
       asm volatile("cp.async.wait_group 0;" ::: "memory");
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> tensor-core (async proxy) reads
-      asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar_full + 8 * stg) : "memory");
+      asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar_f + 8 * stg) : "memory");
+      if (++stg == nst) { stg = 0; ++use; }
     }
   } else if (warp == 4) {
     // ================= MMA issue: S(t + 1) = Q K^T is issued before P(t) is waited for =================
     if (lane == 0) {
       auto issue_s = [&](int tile) {
-        const uint32_t kb = pt_smem(k_s + (tile & 1) * PT_TILE_BYTES), td = tmem_base + 128u * (uint32_t)(tile & 1);
+        const int kbuf = tile % PT_KSTAGES;
+        const uint32_t kb = pt_smem(k_s + kbuf * PT_TILE_BYTES), td = tmem_base + 128u * (uint32_t)(tile & 1);
 #pragma unroll
         for (int ks = 0; ks < DK; ++ks) {
           const uint32_t o2 = (uint32_t)((ks >> 2) * PT_BM * 128 + (ks & 3) * 32);
           pt_mma(td, pt_desc(pt_smem(q_s) + o2), pt_desc(kb + o2), IDESC_S, ks > 0 ? 1u : 0u);
         }
         pt_commit(bar_s + 8 * (tile & 1));
+        pt_commit(bar_ek + 8 * kbuf);
       };
-      bool ok = wait(bar_full, 0);
+      bool ok = wait(bar_fk, 0);
       if (ok) {
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         issue_s(0);
       }
       for (int tile = 0; ok && tile < n_tiles; ++tile) {
         if (tile + 1 < n_tiles) {
-          if (!wait(bar_full + 8 * ((tile + 1) & 1), ((tile + 1) >> 1) & 1)) { ok = false; break; }
+          if (!wait(bar_fk + 8 * ((tile + 1) % PT_KSTAGES), ((tile + 1) / PT_KSTAGES) & 1)) { ok = false; break; }
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
           issue_s(tile + 1);
         }
+        if (!wait(bar_fv + 8 * (tile % PT_VSTAGES), (tile / PT_VSTAGES) & 1)) { ok = false; break; }
         if (!wait(bar_p, tile & 1)) { ok = false; break; }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const uint32_t vb = pt_smem(v_s + (tile & 1) * PT_TILE_BYTES);
+        const uint32_t vb = pt_smem(v_s + (tile % PT_VSTAGES) * PT_TILE_BYTES);
 #pragma unroll
         for (int ks = 0; ks < PT_BN / 16; ++ks) {
           const uint32_t oa = (uint32_t)((ks >> 2) * PT_BM * 128 + (ks & 3) * 32);
           // 16 keys = two 8-key groups of the N-major V tile
-          pt_mma(tmem_o, pt_desc(pt_smem(p_s) + oa), pt_desc_n(vb + (uint32_t)ks * 2048u), IDESC_O, ks > 0 ? 1u : 0u);
+          pt_mma(tmem_o, pt_desc(pt_smem(p_s) + oa), pt_desc_n(vb + (uint32_t)ks * 2048u), IDESC_O, (tile > 0 || ks > 0) ? 1u : 0u);
         }
         pt_commit(bar_o);
-        pt_commit(bar_empty + 8 * (tile & 1));
+        pt_commit(bar_ev + 8 * (tile % PT_VSTAGES));
       }
       // every MMA issued above has completed before tensor memory is released
       pt_commit(bar_end);
@@ -278,103 +328,85 @@ __global__ void __launch_bounds__(PT_THREADS, 1) prefill_tc_kernel(const PtParam
     }
     __syncwarp();
   }
-  float o[NVP];
   float l_run = 0.f;
   const int row = tid;                               // warps 0-3: query row = TMEM lane
+  const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
+  bool rows_ok = true;
   if (warp < 4) {
-    // ================= softmax and output rows: one thread per query =================
+    // ================= softmax: one thread per query row =================
     const int pos = start + q0 + row;                // cache row of this thread's query
-#pragma unroll
-    for (int c = 0; c < NVP; ++c) o[c] = 0.f;
     float m_ref = -1.0e30f;
-    const uint32_t lane_off = (uint32_t)(warp * 32) << 16;
-    // pass 1 of a tile: the row's maximum over the allowed keys; lazy reference maximum (p stays <= 2^8).
-    // Only the tiles that reach past the block's first query need the causal mask.
-    auto pass1 = [&](int tile) -> float {
-      const uint32_t trow = tmem_base + 128u * (uint32_t)(tile & 1) + lane_off;
+    for (int tile = 0; tile < n_tiles; ++tile) {
       const int j0 = tile * PT_BN;
+      const uint32_t trow = tmem_base + 128u * (uint32_t)(tile & 1) + lane_off;
+      if (!__all_sync(0xffffffffu, wait(bar_s + 8 * (tile & 1), (tile >> 1) & 1))) { rows_ok = false; break; }
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      // the whole S row in registers: four loads in flight, one wait
+      uint32_t r[128];
+      pt_ld32_nowait(trow, *reinterpret_cast<uint32_t(*)[32]>(r));
+      pt_ld32_nowait(trow + 32, *reinterpret_cast<uint32_t(*)[32]>(r + 32));
+      pt_ld32_nowait(trow + 64, *reinterpret_cast<uint32_t(*)[32]>(r + 64));
+      pt_ld32_nowait(trow + 96, *reinterpret_cast<uint32_t(*)[32]>(r + 96));
+      asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+      // only the tiles that reach past the block's first query need the causal mask
       const bool interior = j0 + PT_BN - 1 <= start + q0;
       float mx = -INFINITY;
-#pragma unroll 1
-      for (int c0 = 0; c0 < PT_BN; c0 += 32) {
-        uint32_t r[32];
-        pt_ld32(trow + c0, r);
-        if (interior) {
+      if (interior) {
 #pragma unroll
-          for (int j = 0; j < 32; ++j) mx = fmaxf(mx, __uint_as_float(r[j]));
-        } else {
+        for (int j = 0; j < 128; ++j) mx = fmaxf(mx, __uint_as_float(r[j]));
+      } else {
 #pragma unroll
-          for (int j = 0; j < 32; ++j)
-            if (j0 + c0 + j <= pos) mx = fmaxf(mx, __uint_as_float(r[j]));
-        }
+        for (int j = 0; j < 128; ++j)
+          if (j0 + j <= pos) mx = fmaxf(mx, __uint_as_float(r[j]));
       }
       mx *= p.qscale;                  // the scale is positive: the maximum commutes with it
       float alpha = 1.f;
-      if (mx > m_ref + 8.f) {
+      if (mx > m_ref + 8.f) {          // lazy reference maximum: p stays <= 2^8
         alpha = pt_ex2(m_ref - mx);    // first time: 2^(-1e30 - mx) = 0
         m_ref = mx;
         l_run *= alpha;
       }
-      return alpha;
-    };
-    bool ok = wait(bar_s, 0);
-    float alpha_t = 1.f;
-    if (ok) {
-      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      alpha_t = pass1(0);
-    }
-    for (int tile = 0; ok && tile < n_tiles; ++tile) {
-      const int j0 = tile * PT_BN;
-      const uint32_t trow = tmem_base + 128u * (uint32_t)(tile & 1) + lane_off;
-      // pass 2: p = 2^(s - m_ref), bf16, into the A-operand layout (this thread's row, 16 chunks of 8 keys);
-      // the second MMA of the previous tile, which read P, has completed (its O_tile was waited for below)
-      const bool interior = j0 + PT_BN - 1 <= start + q0;
+      // p = 2^(s - m_ref) as packed bf16 pairs (in place)
       const float nm = -m_ref;
-#pragma unroll 1
-      for (int c0 = 0; c0 < PT_BN; c0 += 32) {
-        uint32_t r[32];
-        pt_ld32(trow + c0, r);
-        uint32_t pk[16];
 #pragma unroll
-        for (int j = 0; j < 32; j += 2) {
-          float p0 = pt_ex2(fmaf(__uint_as_float(r[j]), p.qscale, nm));
-          float p1 = pt_ex2(fmaf(__uint_as_float(r[j + 1]), p.qscale, nm));
-          if (!interior) {
-            if (j0 + c0 + j > pos) p0 = 0.f;
-            if (j0 + c0 + j + 1 > pos) p1 = 0.f;
-          }
-          l_run += p0 + p1;
-          const __nv_bfloat162 v2 = __floats2bfloat162_rn(p0, p1);
-          pk[j >> 1] = *reinterpret_cast<const uint32_t*>(&v2);
+      for (int j = 0; j < 128; j += 2) {
+        float p0 = pt_ex2(fmaf(__uint_as_float(r[j]), p.qscale, nm));
+        float p1 = pt_ex2(fmaf(__uint_as_float(r[j + 1]), p.qscale, nm));
+        if (!interior) {
+          if (j0 + j > pos) p0 = 0.f;
+          if (j0 + j + 1 > pos) p1 = 0.f;
         }
-#pragma unroll
-        for (int ch = 0; ch < 4; ++ch)
-          *reinterpret_cast<uint4*>(p_s + pt_off(row, c0 + 8 * ch, PT_BM)) =
-              make_uint4(pk[4 * ch], pk[4 * ch + 1], pk[4 * ch + 2], pk[4 * ch + 3]);
+        l_run += p0 + p1;
+        const __nv_bfloat162 v2 = __floats2bfloat162_rn(p0, p1);
+        r[j >> 1] = *reinterpret_cast<const uint32_t*>(&v2);
       }
+      // the second MMA of the previous tile has read P and has added into O: wait for it before touching either
+      if (tile > 0) {
+        if (!__all_sync(0xffffffffu, wait(bar_o, (tile - 1) & 1))) { rows_ok = false; break; }
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        // rescale this warp's 32 accumulator rows in tensor memory (rare: the maximum is lazy)
+        if (__any_sync(0xffffffffu, alpha != 1.f)) {
+#pragma unroll 1
+          for (int c0 = 0; c0 < NVP; c0 += 32) {
+            uint32_t oc[32];
+            pt_ld32(tmem_o + lane_off + c0, oc);
+#pragma unroll
+            for (int j = 0; j < 32; ++j) oc[j] = __float_as_uint(__uint_as_float(oc[j]) * alpha);
+            pt_st32(tmem_o + lane_off + c0, oc);
+          }
+          asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+        }
+      }
+      // P into the A-operand layout (this thread's row, 16 chunks of 8 keys)
+#pragma unroll
+      for (int ch = 0; ch < 16; ++ch)
+        *reinterpret_cast<uint4*>(p_s + pt_off(row, 8 * ch, PT_BM)) = make_uint4(r[4 * ch], r[4 * ch + 1], r[4 * ch + 2], r[4 * ch + 3]);
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar_p) : "memory");
-      // while the second MMA runs: the maximum of the next tile, whose S is already in tensor memory
-      float alpha_next = 1.f;
-      if (tile + 1 < n_tiles) {
-        if (!wait(bar_s + 8 * ((tile + 1) & 1), ((tile + 1) >> 1) & 1)) { ok = false; break; }
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        alpha_next = pass1(tile + 1);
-      }
-      if (!wait(bar_o, tile & 1)) { ok = false; break; }
-      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      const uint32_t orow = tmem_o + lane_off;
-#pragma unroll
-      for (int c0 = 0; c0 < NVP; c0 += 32) {
-        uint32_t r[32];
-        pt_ld32(orow + c0, r);
-#pragma unroll
-        for (int j = 0; j < 32; ++j) o[c0 + j] = o[c0 + j] * alpha_t + __uint_as_float(r[j]);
-      }
-      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-      alpha_t = alpha_next;
     }
+    if (rows_ok && !__all_sync(0xffffffffu, wait(bar_o, (n_tiles - 1) & 1))) rows_ok = false;
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
@@ -384,15 +416,23 @@ __global__ void __launch_bounds__(PT_THREADS, 1) prefill_tc_kernel(const PtParam
     p.status[1] = 0x60000000 | (blockIdx.x & 0xffffff);
   }
   if (warp < 4 && !timed_out) {
+    // every row's thread reads its accumulator row (all lanes of the warp take part in the load)
     const int t = q0 + row;
-    if (t < p.T) {
-      const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
-      float* dst = p.out + (((size_t)b * p.T + t) * p.Hq + g) * p.dv;
+    const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
+    float* dst = p.out + (((size_t)b * p.T + min(t, p.T - 1)) * p.Hq + g) * p.dv;
+#pragma unroll 1
+    for (int c0 = 0; c0 < NVP; c0 += 32) {
+      uint32_t oc[32];
+      pt_ld32(tmem_o + lane_off + c0, oc);
+      if (t < p.T) {
 #pragma unroll
-      for (int c = 0; c < NVP; ++c)
-        if (c < p.dv) dst[c] = o[c] * inv;
+        for (int j = 0; j < 32; ++j)
+          if (c0 + j < p.dv) dst[c0 + j] = __uint_as_float(oc[j]) * inv;
+      }
     }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   }
+  __syncthreads();
   if (warp == 4) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
@@ -401,7 +441,7 @@ __global__ void __launch_bounds__(PT_THREADS, 1) prefill_tc_kernel(const PtParam
 
 template <int DK, int NVP>
 rap_status launch_pt(rap_ctx* ctx, const PtParams& p, int B, cudaStream_t st) {
-  const int smem = 6 * PT_TILE_BYTES + 128 + 1024;
+  const int smem = (2 + PT_KSTAGES + PT_VSTAGES) * PT_TILE_BYTES + 128 + 1024;
   RAP_CUDA_TRY(ctx, rap_raise_smem(ctx, prefill_tc_kernel<DK, NVP>, smem));
   dim3 grid((p.T + PT_BM - 1) / PT_BM, p.Hq, B);
   prefill_tc_kernel<DK, NVP><<<grid, PT_THREADS, smem, st>>>(p);
