@@ -123,23 +123,49 @@ __device__ __forceinline__ uint32_t pt_swz(int e, int r7) {
   const int w = e >> 2;
   return (uint32_t)(((w >> 5) << 14) + ((((w & 31) >> 2) ^ r7) << 4) + ((w & 3) << 2));
 }
-// The odd rows (1, 3, ..., 127) of a tile with an odd row length start 2 bytes off a word.  Channel pair (2w, 2w+1) is
-// the high half of one aligned word and the low half of the next; the last word holds one channel.
-__device__ __forceinline__ void pt_stage_odd_rows(uint32_t du, const unsigned char* tile_src, int rowlen, int rows_ok,
-                                                  int lane) {
-  const int wl = (rowlen - 1) >> 1;
-#pragma unroll 2
-  for (int r = 1; r < 128; r += 2) {
-    const bool ok = r < rows_ok;
-    const uint32_t* g = reinterpret_cast<const uint32_t*>(tile_src + (size_t)r * rowlen * 2 - 2);
-    const uint32_t dst = du + (uint32_t)r * 128u;
-    for (int w = lane; w <= wl; w += 32) {
-      uint32_t val = 0u;                               // rows past the end: zeros, and nothing is read
-      if (ok) {
-        const uint32_t a = g[w], b2 = w < wl ? g[w + 1] : 0u;
-        asm("prmt.b32 %0, %1, %2, 0x5432;" : "=r"(val) : "r"(a), "r"(b2));
+// Rows of an odd length (odd d_v'), for the warp that takes the row pairs (4k + 2 pw, 4k + 2 pw + 1).  The even row of
+// a pair starts on a word: 4-byte copies, the last word half filled.  The odd row starts 2 bytes off a word: channel
+// pair (2w, 2w+1) is the high half of one aligned word and the low half of the next (two loads, a byte permute, a
+// store); eight rows are loaded before the first store so that the loads overlap.
+__device__ __forceinline__ void pt_stage_odd_len(uint32_t du, const unsigned char* tile_src, int rowlen, int rows_ok,
+                                                 int pw, int lane) {
+  const int wl = (rowlen - 1) >> 1;                    // last word of a row: one channel
+  const int RB = 2 * rowlen;
+  for (int k0 = 0; k0 < 32; k0 += 8) {
+    uint32_t va[8][2], vb[8][2];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      const int r = 4 * (k0 + k) + 2 * pw + 1;         // odd row
+      const bool ok = r < rows_ok;
+      const uint32_t* g = reinterpret_cast<const uint32_t*>(tile_src + (size_t)r * RB - 2);
+#pragma unroll
+      for (int sl = 0; sl < 2; ++sl) {
+        const int w = lane + 32 * sl;
+        va[k][sl] = (ok && w <= wl) ? g[w] : 0u;
+        vb[k][sl] = (ok && w < wl) ? g[w + 1] : 0u;
       }
-      asm volatile("st.shared.u32 [%0], %1;" ::"r"(dst + pt_swz(4 * w, r & 7)), "r"(val) : "memory");
+    }
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      const int re = 4 * (k0 + k) + 2 * pw, r = re + 1;
+      // even row: asynchronous copies
+      const bool oke = re < rows_ok;
+      const unsigned char* se = tile_src + (size_t)(oke ? re : 0) * RB;
+#pragma unroll
+      for (int sl = 0; sl < 2; ++sl) {
+        const int w = lane + 32 * sl;
+        if (w <= wl) pt_cp4(du + (uint32_t)re * 128u + pt_swz(4 * w, re & 7), se + 4 * w, oke ? (w == wl ? 2 : 4) : 0);
+      }
+      // odd row: from the registers
+#pragma unroll
+      for (int sl = 0; sl < 2; ++sl) {
+        const int w = lane + 32 * sl;
+        if (w <= wl) {
+          uint32_t val;
+          asm("prmt.b32 %0, %1, %2, 0x5432;" : "=r"(val) : "r"(va[k][sl]), "r"(vb[k][sl]));
+          asm volatile("st.shared.u32 [%0], %1;" ::"r"(du + (uint32_t)r * 128u + pt_swz(4 * w, r & 7)), "r"(val) : "memory");
+        }
+      }
     }
   }
 }
@@ -248,7 +274,7 @@ __global__ void __launch_bounds__(PT_THREADS, 1) prefill_tc_kernel(const PtParam
     const int nst = is_v ? PT_VSTAGES : PT_KSTAGES;
     unsigned char* ring = is_v ? v_s : k_s;
     const uint32_t bar_f = is_v ? bar_fv : bar_fk, bar_e = is_v ? bar_ev : bar_ek;
-    const bool odd_rows = (rowlen & 1) && pw == 1;     // odd rows of an odd d_v' are only 2-byte aligned
+    const bool odd_len = (rowlen & 1) != 0;            // odd d_v': every second row is only 2-byte aligned
     uint32_t swz[4][2];                                // [row class][word slot]: in-row byte offset
     int nb[2];                                         // bytes this lane copies per slot (0: none; 2: the half-filled word)
 #pragma unroll
@@ -265,8 +291,8 @@ __global__ void __launch_bounds__(PT_THREADS, 1) prefill_tc_kernel(const PtParam
       const uint32_t du = pt_smem(ring + stg * PT_TILE_BYTES);
       const int rows_ok = min(PT_BN, n_valid - j0);    // rows of this tile that exist (>= 1)
       const unsigned char* tsrc = src0 + (size_t)j0 * (size_t)(2 * rowlen);
-      if (odd_rows) {
-        pt_stage_odd_rows(du, tsrc, rowlen, rows_ok, lane);
+      if (odd_len) {
+        pt_stage_odd_len(du, tsrc, rowlen, rows_ok, pw, lane);
       } else {
 #pragma unroll 4
         for (int i = 0; i < PT_BN / 2; ++i) {
