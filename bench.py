@@ -375,6 +375,65 @@ def run_sweep(args):
                       "sweep": rows}), flush=True)
 
 
+def run_prefill(args):
+    """rap_prefill_attn (causal block attention on the reduced dims) on the 8B head shapes of the retain-ratio
+    sweep: time per call, TFLOP/s on the causal flops B H_q T (T + 1) (2P + d_v'), and the fraction of the measured
+    dense bf16 peak.  --prefill-case B:T picks the size (default 2:4096 and 1:16384); --attn-variant 1 times the
+    warp-level mma.sync kernel instead of the tcgen05 one."""
+    import torch
+    from dataclasses import replace
+    from paper_2602_02599_b200.stack import DecodeStack
+    torch.cuda.set_device(0)
+    peak = None
+    pp = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(pp):
+        peak = json.load(open(pp)).get("bf16_tflops")
+    cases = [tuple(int(v) for v in c.split(":")) for c in (args.prefill_case.split(",") if args.prefill_case else ["2:4096", "1:16384"])]
+    rows = []
+    for B, T in cases:
+        dense_ms = None
+        for rho in sorted(synth.SWEEP_COUNTS, reverse=True):
+            w = replace(synth.sweep_workload(rho), n_layers=1, batch=B, seq=T)
+            st = DecodeStack(w, s_cap=T + 8)
+            st.build_tables(*synth.draw_scores(w))
+            if args.attn_variant:
+                st.ctx.rap_set_attn_variant(args.attn_variant)
+            g = torch.Generator(device=st.device).manual_seed(w.seed)
+            sigma = float(np.sqrt(w.hidden) * 0.02)
+            st.k_cache[0].normal_(0.0, sigma, generator=g)
+            st.v_cache[0].normal_(0.0, sigma, generator=g)
+            q = torch.empty((B, T, w.n_q_heads, 2 * w.n_pairs), dtype=st.dt, device=st.device).normal_(0, sigma, generator=g)
+            ds = torch.zeros(B, dtype=torch.int32, device=st.device)
+            out = torch.empty((B, T, w.n_q_heads, w.n_vch), dtype=torch.float32, device=st.device)
+            call = lambda: st.ctx.rap_prefill_attn(0, B, T, q, st.k_cache[0], st.v_cache[0], st.s_cap, ds, 0, out)
+            for _ in range(args.warmup):
+                call()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(args.steps):
+                call()
+            e1.record()
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1) / args.steps
+            code, detail = st.ctx.rap_get_last_device_status()
+            assert code == 0, (code, detail)
+            if rho == 1.0:
+                dense_ms = ms
+            flops = B * w.n_q_heads * T * (T + 1) * (2 * w.n_pairs + w.n_vch)
+            tf = flops / ms / 1e9
+            rows.append({"rho": rho, "P": w.n_pairs, "dv": w.n_vch, "B": B, "T": T, "ms": ms, "TFLOPs": tf,
+                         "frac_of_measured_bf16_peak": tf / peak if peak else None, "time_vs_dense": ms / dense_ms})
+            st.close()
+            del st, q, out
+            torch.cuda.empty_cache()
+    print(json.dumps({"metric": "prefill_attention_tflops", "unit": "TFLOP/s", "n_gpus": 1, "steps": args.steps,
+                      "warmup": args.warmup, "dtype": "bf16", "data": "synthetic", "higher_is_better": True,
+                      "config": {"workload": "rap_prefill_attn on the 8B head shapes (32q/8kv heads, D=128), start = 0"},
+                      "roofline": {"bound": "tensor", "peak": peak, "peak_source": "measured" if peak else None, "unit": "TFLOP/s"},
+                      "prefill": rows}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -388,6 +447,8 @@ def main():
     ap.add_argument("--seq", type=int, default=0, help="cut the workload to this context (profiling)")
     ap.add_argument("--attn-variant", type=int, default=0,
                     help="force a kernel tier of rap_decode_attn (profiling; 3 = the FP32-pipe scan)")
+    ap.add_argument("--prefill", action="store_true", help="time rap_prefill_attn on the sweep's head shapes")
+    ap.add_argument("--prefill-case", default="", help="B:T[,B:T...] for --prefill")
     ap.add_argument("--sweep", action="store_true", help="retain-ratio sweep with the dense and low-rank comparators")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":
@@ -398,6 +459,8 @@ def main():
         run_reference(args)
     elif args.sweep:
         run_sweep(args)
+    elif args.prefill:
+        run_prefill(args)
     else:
         run_ours(args)
 

@@ -304,10 +304,14 @@ __global__ void __launch_bounds__(PT_THREADS, 1) prefill_tc_kernel(const PtParam
           if (nb[1] > 0) pt_cp4(rb + swz[i & 3][1], src + lane + 32, ok ? nb[1] : 0);
         }
       }
-      asm volatile("cp.async.commit_group;" ::: "memory");
-      asm volatile("cp.async.wait_group 0;" ::: "memory");
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic writes -> tensor-core (async proxy) reads
-      asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar_f + 8 * stg) : "memory");
+      if (odd_len) {   // plain stores took part: wait, order them before the tensor-core (async proxy) reads, arrive
+        asm volatile("cp.async.commit_group;" ::: "memory");
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar_f + 8 * stg) : "memory");
+      } else {         // the arrival is triggered by the completion of this thread's copies: go on to the next tile
+        asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar_f + 8 * stg) : "memory");
+      }
       if (++stg == nst) { stg = 0; ++use; }
     }
   } else if (warp == 4) {
@@ -326,17 +330,20 @@ __global__ void __launch_bounds__(PT_THREADS, 1) prefill_tc_kernel(const PtParam
       };
       bool ok = wait(bar_fk, 0);
       if (ok) {
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         issue_s(0);
       }
       for (int tile = 0; ok && tile < n_tiles; ++tile) {
         if (tile + 1 < n_tiles) {
           if (!wait(bar_fk + 8 * ((tile + 1) % PT_KSTAGES), ((tile + 1) / PT_KSTAGES) & 1)) { ok = false; break; }
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the copies' writes before the MMA's reads
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
           issue_s(tile + 1);
         }
         if (!wait(bar_fv + 8 * (tile % PT_VSTAGES), (tile / PT_VSTAGES) & 1)) { ok = false; break; }
         if (!wait(bar_p, tile & 1)) { ok = false; break; }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t vb = pt_smem(v_s + (tile % PT_VSTAGES) * PT_TILE_BYTES);
 #pragma unroll
