@@ -25,19 +25,21 @@ constexpr int PT_BM = 128, PT_BN = 128;
 constexpr int PT_THREADS = 288;   // warps 0-3: rows / softmax, warp 4: MMA issue, warps 5-6: K staging, warps 7-8: V staging
 constexpr int PT_KSTAGES = 3, PT_VSTAGES = 2;
 constexpr int PT_TILE_BYTES = 2 * 128 * 128;                     // two 64-element atom columns of 128 rows
-constexpr uint32_t PT_WAIT_LIMIT = 1u << 21;
+constexpr uint32_t PT_WAIT_HINT_NS = 20000;      // a parked probe returns at the phase change or after this long
+constexpr uint32_t PT_WAIT_LIMIT = 1u << 15;    // probes before a wait gives up (well under a second)
 
 __device__ __forceinline__ uint32_t pt_smem(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void pt_mbar_init(uint32_t bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
 }
+// one probe of the barrier's phase; the hardware may park the thread for up to PT_WAIT_HINT_NS before it answers
 __device__ __forceinline__ bool pt_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+      : "=r"(ok) : "r"(bar), "r"(parity), "r"(PT_WAIT_HINT_NS) : "memory");
   return ok != 0;
 }
 // K-major operand tile, 128-byte swizzle: 8-row groups 1024 bytes apart (see rap_proj_tc.cu)
@@ -254,9 +256,8 @@ __global__ void __launch_bounds__(PT_THREADS, 1) prefill_tc_kernel(const PtParam
   // a wait that gives up when its limit runs out or another role has given up; the loser raises the flag
   auto wait = [&](uint32_t bar, uint32_t parity) -> bool {
     for (uint32_t i = 0; i < PT_WAIT_LIMIT; ++i) {
-      if (pt_try_wait(bar, parity)) return true;
-      if (i >= 4) __nanosleep(64);                   // a long wait leaves the issue slots to the working warps
-      if ((i & 255u) == 255u && *abort_flag) return false;
+      if (pt_try_wait(bar, parity)) return true;     // parks in hardware: no issue slots burnt while waiting
+      if ((i & 15u) == 15u && *abort_flag) return false;
     }
     *abort_flag = 1;
     return false;
@@ -294,14 +295,38 @@ __global__ void __launch_bounds__(PT_THREADS, 1) prefill_tc_kernel(const PtParam
       if (odd_len) {
         pt_stage_odd_len(du, tsrc, rowlen, rows_ok, pw, lane);
       } else {
+        if (rows_ok == PT_BN) {
+          // a full tile (all but the last one of a sequence): no predicates, running pointers
+          const unsigned char* sp = tsrc + (size_t)pw * (size_t)(2 * rowlen) + 4 * lane;
+          uint32_t db = du + (uint32_t)pw * 128u;
+          const bool two = nb[1] > 0;
+          if (nb[0] == 4 && (!two || nb[1] == 4)) {
 #pragma unroll 4
-        for (int i = 0; i < PT_BN / 2; ++i) {
-          const int r = pw + 2 * i;
-          const bool ok = r < rows_ok;                 // rows past the end: zero fill, nothing is read
-          const uint32_t* src = reinterpret_cast<const uint32_t*>(tsrc + (size_t)(ok ? r : 0) * (size_t)(2 * rowlen));
-          const uint32_t rb = du + (uint32_t)r * 128u;
-          if (nb[0] > 0) pt_cp4(rb + swz[i & 3][0], src + lane, ok ? nb[0] : 0);
-          if (nb[1] > 0) pt_cp4(rb + swz[i & 3][1], src + lane + 32, ok ? nb[1] : 0);
+            for (int i = 0; i < PT_BN / 2; ++i) {
+              pt_cp4(db + swz[i & 3][0], sp, 4);
+              if (two) pt_cp4(db + swz[i & 3][1], sp + 128, 4);
+              sp += 4 * rowlen;                        // two rows on
+              db += 256;
+            }
+          } else {
+#pragma unroll 4
+            for (int i = 0; i < PT_BN / 2; ++i) {
+              if (nb[0] > 0) pt_cp4(db + swz[i & 3][0], sp, nb[0]);
+              if (two) pt_cp4(db + swz[i & 3][1], sp + 128, nb[1]);
+              sp += 4 * rowlen;
+              db += 256;
+            }
+          }
+        } else {
+#pragma unroll 4
+          for (int i = 0; i < PT_BN / 2; ++i) {
+            const int r = pw + 2 * i;
+            const bool ok = r < rows_ok;               // rows past the end: zero fill, nothing is read
+            const uint32_t* src = reinterpret_cast<const uint32_t*>(tsrc + (size_t)(ok ? r : 0) * (size_t)(2 * rowlen));
+            const uint32_t rb = du + (uint32_t)r * 128u;
+            if (nb[0] > 0) pt_cp4(rb + swz[i & 3][0], src + lane, ok ? nb[0] : 0);
+            if (nb[1] > 0) pt_cp4(rb + swz[i & 3][1], src + lane + 32, ok ? nb[1] : 0);
+          }
         }
       }
       if (odd_len) {   // plain stores took part: wait, order them before the tensor-core (async proxy) reads, arrive
