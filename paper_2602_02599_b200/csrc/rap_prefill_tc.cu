@@ -408,16 +408,17 @@ __global__ void __launch_bounds__(PT_THREADS, 1) prefill_tc_kernel(const PtParam
       asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
       // only the tiles that reach past the block's first query need the causal mask
       const bool interior = j0 + PT_BN - 1 <= start + q0;
-      float mx = -INFINITY;
+      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // four chains instead of one of 128 steps
       if (interior) {
 #pragma unroll
-        for (int j = 0; j < 128; ++j) mx = fmaxf(mx, __uint_as_float(r[j]));
+        for (int j = 0; j < 128; ++j) mx4[j & 3] = fmaxf(mx4[j & 3], __uint_as_float(r[j]));
       } else {
 #pragma unroll
         for (int j = 0; j < 128; ++j)
-          if (j0 + j <= pos) mx = fmaxf(mx, __uint_as_float(r[j]));
+          if (j0 + j <= pos) mx4[j & 3] = fmaxf(mx4[j & 3], __uint_as_float(r[j]));
       }
-      mx *= p.qscale;                  // the scale is positive: the maximum commutes with it
+      // the scale is positive: the maximum commutes with it
+      const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.qscale;
       float alpha = 1.f;
       if (mx > m_ref + 8.f) {          // lazy reference maximum: p stays <= 2^8
         alpha = pt_ex2(m_ref - mx);    // first time: 2^(-1e30 - mx) = 0
@@ -426,6 +427,7 @@ __global__ void __launch_bounds__(PT_THREADS, 1) prefill_tc_kernel(const PtParam
       }
       // p = 2^(s - m_ref) as packed bf16 pairs (in place)
       const float nm = -m_ref;
+      float ls[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
       for (int j = 0; j < 128; j += 2) {
         float p0 = pt_ex2(fmaf(__uint_as_float(r[j]), p.qscale, nm));
@@ -434,10 +436,11 @@ __global__ void __launch_bounds__(PT_THREADS, 1) prefill_tc_kernel(const PtParam
           if (j0 + j > pos) p0 = 0.f;
           if (j0 + j + 1 > pos) p1 = 0.f;
         }
-        l_run += p0 + p1;
+        ls[(j >> 1) & 3] += p0 + p1;
         const __nv_bfloat162 v2 = __floats2bfloat162_rn(p0, p1);
         r[j >> 1] = *reinterpret_cast<const uint32_t*>(&v2);
       }
+      l_run += (ls[0] + ls[1]) + (ls[2] + ls[3]);
       // the second MMA of the previous tile has read P and has added into O: wait for it before touching either
       if (tile > 0) {
         if (!__all_sync(0xffffffffu, wait(bar_o, (tile - 1) & 1))) { rows_ok = false; break; }
