@@ -114,9 +114,13 @@ __global__ void rope_append_kernel(const float* __restrict__ y, int ksplit, cons
   if (item < n_pair_items) {
     const int h = item / P, c = item - h * P;
     const int G = Hq / Hkv;
-    double sn, cs;
-    sincos((double)p * inv_freq[h * half_dim + c], &sn, &cs);
-    const float cf = (float)cs, sf = (float)sn;
+    // angle and its reduction to [-pi, pi] in fp64 (positions reach 1e5: an fp32 angle would be off by 1e-2 rad),
+    // sine and cosine of the reduced angle in fp32 (about 2e-7 absolute)
+    const double ang = (double)p * inv_freq[h * half_dim + c];
+    const double turns = rint(ang * 0.15915494309189535);                        // 1 / (2 pi)
+    const double red = fma(-turns, 2.4492935982947064e-16, fma(-turns, 6.283185307179586, ang));   // 2 pi = hi + lo
+    float sf, cf;
+    sincosf((float)red, &sf, &cf);
     for (int j = 0; j <= G; ++j) {          // j < G: query head h*G + j; j == G: the key head itself
       const int head = j < G ? h * G + j : Hq + h;
       const int col = head * P2 + 2 * c;
