@@ -1,30 +1,35 @@
 // tcgen05 version of rap_prefill_attn: causal attention of a block of T new tokens per sequence over the
 // reduced dims (Eq. 2 for every t of the block; 2P retained K dims, d_v' retained V channels, scale
-// 1/sqrt(D)).  One CTA (one per SM) handles 128 queries of one query head and walks 128-key tiles up to the
-// causal limit:
-//   S      = Q K^T      tcgen05.mma (M = 128 queries, N = 128 keys, K = 2P in steps of 16), accumulator in TMEM,
-//                       double buffered: S of tile t + 1 is issued before the softmax of tile t has finished
-//   P      = 2^(S - m)  one thread per query row reads its S row from TMEM (tcgen05.ld), applies the causal
-//                       mask and a lazy running maximum, and writes P as bf16 into shared memory
-//   O_tile = P V        tcgen05.mma (N = d_v' rounded up to 32, K = 128 keys), fresh accumulator per tile;
-//                       the row's thread then folds O_tile into its register accumulator with the rescale
-//                       factor, so tensor memory never has to be rewritten.
-// Cache rows are not multiples of 16 bytes, so TMA tensor maps cannot describe them: four producer warps stage
-// the tiles by hand (4-byte cp.async), two tiles ahead (K in a ring of three buffers, V of two), into the
-// 128-byte-swizzled layouts
-// the MMA descriptors expect (K as stored = K-major; V as stored = the N-major form of the B operand, so nothing
-// is transposed); rows past the sequence end and pad columns are zeros.  The roles (4 softmax warps, 1 MMA-issuing lane, 4 producer warps) meet only on mbarriers; every
-// wait is bounded and gives up early once another role has given up.
+// 1/sqrt(D)).  One CTA (one per SM, 416 threads) handles 256 consecutive queries of one query head as two query
+// tiles A and B of 128, and walks 64-key tiles up to each tile's causal limit:
+//   S_X    = Q_X K^T    tcgen05.mma (M = 128 queries, N = 64 keys, K = 2P in steps of 16), accumulator in TMEM,
+//                       double buffered per query tile: S of key tile t + 1 is issued before P of t is waited for
+//   P_X    = 2^(S - m)  softmax warp group X (warps 0-3: A, 4-7: B), one thread per query row: the S row in
+//                       registers with one TMEM round trip, causal mask only on the tiles that reach the diagonal,
+//                       lazy running maximum, P as bf16 into shared memory
+//   O_X   += P_X V      tcgen05.mma (N = d_v' rounded up to 32, K = 64 keys) accumulating in TMEM across the key
+//                       tiles; a warp rescales its 32 accumulator rows (tcgen05.ld / st) only in the rare tile
+//                       where the lazy maximum moved.
+// While one group runs its softmax the tensor core works for the other, and a staged K / V tile serves 256 queries.
+// Cache rows are not multiples of 16 bytes, so TMA tensor maps cannot describe them: four producer warps (9-10: K,
+// 11-12: V) stage the tiles by hand (4-byte cp.async) into rings of four buffers each, in the 128-byte-swizzled
+// layouts the MMA descriptors expect (K as stored = K-major; V as stored = the N-major form of the B operand, so
+// nothing is transposed); rows past the sequence end and pad columns are zeros.  The copies' completion arrives on
+// the buffer's mbarrier by itself; the consumer issues the proxy fence.  The roles meet only on mbarriers; every wait
+// is bounded and gives up early once another role has given up.  One lane of warp 8 issues all MMAs.
 #include <math.h>
 
 #include "rap_internal.h"
 
 namespace {
 
-constexpr int PT_BM = 128, PT_BN = 128;
-constexpr int PT_THREADS = 288;   // warps 0-3: rows / softmax, warp 4: MMA issue, warps 5-6: K staging, warps 7-8: V staging
-constexpr int PT_KSTAGES = 3, PT_VSTAGES = 2;
-constexpr int PT_TILE_BYTES = 2 * 128 * 128;                     // two 64-element atom columns of 128 rows
+constexpr int P2_KT = 64;                              // keys per tile
+constexpr int P2_THREADS = 416;
+constexpr int P2_STAGES = 4;                           // K buffers and V buffers
+constexpr int P2_Q_BYTES = 2 * 128 * 128;              // [128 queries][<=128 dims]: two 64-element atom columns
+constexpr int P2_P_BYTES = 128 * 128;                  // [128 queries][64 keys]
+constexpr int P2_KV_BYTES = 2 * P2_KT * 128;           // [64 keys][<=128 dims or channels]
+constexpr int P2_SMEM = 2 * P2_Q_BYTES + 2 * P2_P_BYTES + 2 * P2_STAGES * P2_KV_BYTES + 256;
 constexpr uint32_t PT_WAIT_HINT_NS = 20000;      // a parked probe returns at the phase change or after this long
 constexpr uint32_t PT_WAIT_LIMIT = 1u << 15;    // probes before a wait gives up (well under a second)
 
@@ -113,27 +118,27 @@ __device__ __forceinline__ uint32_t pt_off(int row, int col, int rows) {
 
 // N-major operand tile (B = V as stored, [key][channel]), 128-byte swizzle: an atom is 8 keys x 64 channels
 // (key rows of 128 bytes, 16-byte chunks XORed with key % 8); atoms of consecutive 8-key groups are 1024 bytes
-// apart (stride offset), the two 64-channel atom columns 16 KB apart (leading offset).
-__device__ __forceinline__ uint64_t pt_desc_n(uint32_t addr) {
-  const uint32_t lo = ((addr & 0x3FFFFu) >> 4) | ((16384u >> 4) << 16);
+// apart (stride offset), the two 64-channel atom columns of a 64-key tile 8 KB apart (leading offset).
+__device__ __forceinline__ uint64_t pt_desc_n2(uint32_t addr) {
+  const uint32_t lo = ((addr & 0x3FFFFu) >> 4) | ((8192u >> 4) << 16);
   const uint32_t hi = (1024u >> 4) | (1u << 14) | (2u << 29);
   return ((uint64_t)hi << 32) | lo;
 }
-// Byte offset inside a tile row of its byte e: 64-element (128-byte) atom columns 16 KB apart, 16-byte chunks
+// Byte offset inside a 64-row tile row of its byte e: 64-element (128-byte) atom columns 8 KB apart, 16-byte chunks
 // XORed with row % 8 (the layout is the same for the K-major K tile and the N-major V tile).
-__device__ __forceinline__ uint32_t pt_swz(int e, int r7) {
+__device__ __forceinline__ uint32_t pt_swz2(int e, int r7) {
   const int w = e >> 2;
-  return (uint32_t)(((w >> 5) << 14) + ((((w & 31) >> 2) ^ r7) << 4) + ((w & 3) << 2));
+  return (uint32_t)(((w >> 5) << 13) + ((((w & 31) >> 2) ^ r7) << 4) + ((w & 3) << 2));
 }
-// Rows of an odd length (odd d_v'), for the warp that takes the row pairs (4k + 2 pw, 4k + 2 pw + 1).  The even row of
-// a pair starts on a word: 4-byte copies, the last word half filled.  The odd row starts 2 bytes off a word: channel
-// pair (2w, 2w+1) is the high half of one aligned word and the low half of the next (two loads, a byte permute, a
-// store); eight rows are loaded before the first store so that the loads overlap.
+// Rows of an odd length (odd d_v'), for the warp that takes the row pairs (4k + 2 pw, 4k + 2 pw + 1) of a 64-row tile.
+// The even row of a pair starts on a word: 4-byte copies, the last word half filled.  The odd row starts 2 bytes off
+// a word: channel pair (2w, 2w+1) is the high half of one aligned word and the low half of the next (two loads, a
+// byte permute, a store); eight rows are loaded before the first store so that the loads overlap.
 __device__ __forceinline__ void pt_stage_odd_len(uint32_t du, const unsigned char* tile_src, int rowlen, int rows_ok,
                                                  int pw, int lane) {
   const int wl = (rowlen - 1) >> 1;                    // last word of a row: one channel
   const int RB = 2 * rowlen;
-  for (int k0 = 0; k0 < 32; k0 += 8) {
+  for (int k0 = 0; k0 < P2_KT / 4; k0 += 8) {
     uint32_t va[8][2], vb[8][2];
 #pragma unroll
     for (int k = 0; k < 8; ++k) {
@@ -150,22 +155,16 @@ __device__ __forceinline__ void pt_stage_odd_len(uint32_t du, const unsigned cha
 #pragma unroll
     for (int k = 0; k < 8; ++k) {
       const int re = 4 * (k0 + k) + 2 * pw, r = re + 1;
-      // even row: asynchronous copies
       const bool oke = re < rows_ok;
       const unsigned char* se = tile_src + (size_t)(oke ? re : 0) * RB;
 #pragma unroll
       for (int sl = 0; sl < 2; ++sl) {
         const int w = lane + 32 * sl;
-        if (w <= wl) pt_cp4(du + (uint32_t)re * 128u + pt_swz(4 * w, re & 7), se + 4 * w, oke ? (w == wl ? 2 : 4) : 0);
-      }
-      // odd row: from the registers
-#pragma unroll
-      for (int sl = 0; sl < 2; ++sl) {
-        const int w = lane + 32 * sl;
         if (w <= wl) {
+          pt_cp4(du + (uint32_t)re * 128u + pt_swz2(4 * w, re & 7), se + 4 * w, oke ? (w == wl ? 2 : 4) : 0);
           uint32_t val;
           asm("prmt.b32 %0, %1, %2, 0x5432;" : "=r"(val) : "r"(va[k][sl]), "r"(vb[k][sl]));
-          asm volatile("st.shared.u32 [%0], %1;" ::"r"(du + (uint32_t)r * 128u + pt_swz(4 * w, r & 7)), "r"(val) : "memory");
+          asm volatile("st.shared.u32 [%0], %1;" ::"r"(du + (uint32_t)r * 128u + pt_swz2(4 * w, r & 7)), "r"(val) : "memory");
         }
       }
     }
@@ -185,268 +184,256 @@ struct PtParams {
 
 // DK = k-steps of Q K^T (ceil(2P / 16)); NVP = d_v' rounded up to a multiple of 32 (N of the second MMA)
 template <int DK, int NVP>
-__global__ void __launch_bounds__(PT_THREADS, 1) prefill_tc_kernel(const PtParams p) {
+__global__ void __launch_bounds__(P2_THREADS, 1) prefill_tc2_kernel(const PtParams p) {
   extern __shared__ unsigned char pt_raw[];
   unsigned char* smem = pt_raw + ((1024u - (pt_smem(pt_raw) & 1023u)) & 1023u);
-  unsigned char* q_s = smem;                                   // [128 queries][<=128 dims]
-  unsigned char* p_s = q_s + PT_TILE_BYTES;                    // [128 queries][128 keys]
-  unsigned char* k_s = p_s + PT_TILE_BYTES;                    // ring of [128 keys][<=128 dims]
-  unsigned char* v_s = k_s + PT_KSTAGES * PT_TILE_BYTES;       // ring of [128 keys][<=128 channels] (N-major)
-  unsigned char* tail = v_s + PT_VSTAGES * PT_TILE_BYTES;
-  // mbarriers: K / V buffer filled (producers -> MMA), buffer free (the MMA that read it is done -> producers),
-  // S ready (first MMA done -> softmax), P written (softmax -> MMA), O updated (second MMA done -> softmax), drain
-  const uint32_t bar_fk = pt_smem(tail), bar_ek = bar_fk + 24, bar_fv = bar_fk + 48, bar_ev = bar_fk + 64,
-                 bar_s = bar_fk + 80, bar_p = bar_fk + 96, bar_o = bar_fk + 104, bar_end = bar_fk + 112;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 120);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 124);
+  unsigned char* q_s = smem;                                   // Q_A, Q_B
+  unsigned char* p_s = q_s + 2 * P2_Q_BYTES;                   // P_A, P_B
+  unsigned char* k_s = p_s + 2 * P2_P_BYTES;                   // ring of K tiles
+  unsigned char* v_s = k_s + P2_STAGES * P2_KV_BYTES;          // ring of V tiles (N-major)
+  unsigned char* tail = v_s + P2_STAGES * P2_KV_BYTES;
+  const uint32_t bar_fk = pt_smem(tail), bar_ek = bar_fk + 32, bar_fv = bar_fk + 64, bar_ev = bar_fk + 96,
+                 bar_s = bar_fk + 128 /* [X][2] */, bar_p = bar_fk + 160 /* [X] */, bar_o = bar_fk + 176 /* [X] */,
+                 bar_end = bar_fk + 192;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 200);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 204);
 
   const int qb = blockIdx.x, g = blockIdx.y, b = blockIdx.z;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int h = g / (p.Hq / p.Hkv);
   const int start = min(max(p.start[b], 0), p.S_cap - p.T);
   const int n_valid = start + p.T;
-  const int q0 = qb * PT_BM;
-  const int last_pos = start + min(p.T, q0 + PT_BM) - 1;
-  const int n_tiles = last_pos / PT_BN + 1;
+  const int q0 = qb * 256;
+  // key tiles each query tile needs (tile B may lie wholly past the block)
+  int nt[2];
+#pragma unroll
+  for (int X = 0; X < 2; ++X) {
+    const int q0x = q0 + 128 * X;
+    nt[X] = q0x < p.T ? (start + min(p.T, q0x + 128) - 1) / P2_KT + 1 : 0;
+  }
+  const int n_max = max(nt[0], nt[1]);
   const __nv_bfloat16* kg = p.k + ((size_t)b * p.Hkv + h) * (size_t)p.S_cap * p.P2;
   const __nv_bfloat16* vg = p.v + ((size_t)b * p.Hkv + h) * (size_t)p.S_cap * p.dv;
 
   if (tid == 0) {
-    for (int i = 0; i < PT_KSTAGES; ++i) {
+    for (int i = 0; i < P2_STAGES; ++i) {
       pt_mbar_init(bar_fk + 8 * i, 64);
       pt_mbar_init(bar_ek + 8 * i, 1);
-    }
-    for (int i = 0; i < PT_VSTAGES; ++i) {
       pt_mbar_init(bar_fv + 8 * i, 64);
       pt_mbar_init(bar_ev + 8 * i, 1);
     }
-    for (int i = 0; i < 2; ++i) pt_mbar_init(bar_s + 8 * i, 1);
-    pt_mbar_init(bar_p, 128);
-    pt_mbar_init(bar_o, 1);
+    for (int i = 0; i < 4; ++i) pt_mbar_init(bar_s + 8 * i, 1);
+    for (int X = 0; X < 2; ++X) {
+      pt_mbar_init(bar_p + 8 * X, 128);
+      pt_mbar_init(bar_o + 8 * X, 1);
+    }
     pt_mbar_init(bar_end, 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 4) {
+  if (warp == 8) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(pt_smem(tmem_slot)), "r"(512)
                  : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
-  // zero all six tiles once (pad columns and pad channel rows are never written again), then stage Q
-  for (int i = tid; i < (2 + PT_KSTAGES + PT_VSTAGES) * PT_TILE_BYTES / 16; i += PT_THREADS) reinterpret_cast<uint4*>(smem)[i] = make_uint4(0, 0, 0, 0);
+  // zero every tile once (pad columns and pad channel rows are never written again), then stage Q_A and Q_B
+  for (int i = tid; i < (P2_SMEM - 256) / 16; i += P2_THREADS) reinterpret_cast<uint4*>(smem)[i] = make_uint4(0, 0, 0, 0);
   __syncthreads();
   const int kw = p.P2 >> 1;                          // 4-byte words per q / K row
-  for (int r = warp; r < PT_BM; r += PT_THREADS / 32) {
+  for (int r = warp; r < 256; r += P2_THREADS / 32) {
     const int t = q0 + r;
     if (t < p.T) {
       const uint32_t* src = reinterpret_cast<const uint32_t*>(p.q + (((size_t)b * p.T + t) * p.Hq + g) * p.P2);
-      for (int w = lane; w < kw; w += 32) *reinterpret_cast<uint32_t*>(q_s + pt_off(r, 2 * w, PT_BM)) = src[w];
+      unsigned char* qd = q_s + (r >> 7) * P2_Q_BYTES;
+      for (int w = lane; w < kw; w += 32) *reinterpret_cast<uint32_t*>(qd + pt_off(r & 127, 2 * w, 128)) = src[w];
     }
   }
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-  const uint32_t tmem_base = *tmem_slot;             // S of tile t in columns [128 (t & 1), +128), O_tile in [256, 256 + NVP)
-  const uint32_t tmem_o = tmem_base + 256;
-  constexpr uint32_t IDESC_S = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(PT_BN >> 3) << 17) | ((uint32_t)(PT_BM >> 4) << 24);
-  // second MMA: B = V is N-major (bit 16)
+  const uint32_t tmem_base = *tmem_slot;             // S_X(t): columns 128 X + 64 (t & 1); O_X: columns 256 + 128 X
+  constexpr uint32_t IDESC_S = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(P2_KT >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
   constexpr uint32_t IDESC_O = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(NVP >> 3) << 17) |
-                               ((uint32_t)(PT_BM >> 4) << 24);
-  // a wait that gives up when its limit runs out or another role has given up; the loser raises the flag
+                               ((uint32_t)(128 >> 4) << 24);
   auto wait = [&](uint32_t bar, uint32_t parity) -> bool {
     for (uint32_t i = 0; i < PT_WAIT_LIMIT; ++i) {
-      if (pt_try_wait(bar, parity)) return true;     // parks in hardware: no issue slots burnt while waiting
+      if (pt_try_wait(bar, parity)) return true;
       if ((i & 15u) == 15u && *abort_flag) return false;
     }
     *abort_flag = 1;
     return false;
   };
 
-  if (warp >= 5) {
-    // ================= producers: warps 5-6 stage K (three buffers), warps 7-8 stage V (two buffers) =================
-    // A warp takes every second row in order (neighbouring rows share cache lines and are fetched together by the
-    // two warps); a lane keeps its words (lane, lane + 32) of every row.  r % 8 takes four values per warp, so the
-    // swizzled in-row offsets are eight constants per lane and a copy costs a few instructions.
-    const bool is_v = warp >= 7;
-    const int pw = (warp - 5) & 1;
-    const int rowlen = is_v ? p.dv : p.P2;             // elements per row
+  float l_run = 0.f;
+  const int X = (warp >> 2) & 1;                     // softmax group = query tile
+  const int row = (warp & 3) * 32 + lane;
+  const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
+  const uint32_t tmem_o = tmem_base + 256 + 128 * X;
+  if (warp >= 9) {
+    // ================= producers: warps 9-10 stage K, warps 11-12 stage V, in order, tiles of 64 rows =================
+    const bool is_v = warp >= 11;
+    const int pw = (warp - 9) & 1;
+    const int rowlen = is_v ? p.dv : p.P2;
     const unsigned char* src0 = reinterpret_cast<const unsigned char*>(is_v ? vg : kg);
-    const int nst = is_v ? PT_VSTAGES : PT_KSTAGES;
     unsigned char* ring = is_v ? v_s : k_s;
     const uint32_t bar_f = is_v ? bar_fv : bar_fk, bar_e = is_v ? bar_ev : bar_ek;
-    const bool odd_len = (rowlen & 1) != 0;            // odd d_v': every second row is only 2-byte aligned
-    uint32_t swz[4][2];                                // [row class][word slot]: in-row byte offset
-    int nb[2];                                         // bytes this lane copies per slot (0: none; 2: the half-filled word)
+    const bool odd_len = (rowlen & 1) != 0;
+    uint32_t swz[4][2];
+    int nb[2];
 #pragma unroll
     for (int sl = 0; sl < 2; ++sl) {
       const int w = lane + 32 * sl;
       nb[sl] = min(4, max(0, 2 * rowlen - 4 * w));
 #pragma unroll
-      for (int c = 0; c < 4; ++c) swz[c][sl] = pt_swz(4 * w, (pw + 2 * c) & 7);
+      for (int c = 0; c < 4; ++c) swz[c][sl] = pt_swz2(4 * w, (pw + 2 * c) & 7);
     }
-    int stg = 0, use = 0;                              // buffer of this tile and how often it has been used before
-    for (int tile = 0; tile < n_tiles; ++tile) {
-      const int j0 = tile * PT_BN;
+    int stg = 0, use = 0;
+    for (int tile = 0; tile < n_max; ++tile) {
+      const int j0 = tile * P2_KT;
       if (use > 0 && !wait(bar_e + 8 * stg, (use - 1) & 1)) break;
-      const uint32_t du = pt_smem(ring + stg * PT_TILE_BYTES);
-      const int rows_ok = min(PT_BN, n_valid - j0);    // rows of this tile that exist (>= 1)
+      const uint32_t du = pt_smem(ring + stg * P2_KV_BYTES);
+      const int rows_ok = min(P2_KT, n_valid - j0);
       const unsigned char* tsrc = src0 + (size_t)j0 * (size_t)(2 * rowlen);
       if (odd_len) {
         pt_stage_odd_len(du, tsrc, rowlen, rows_ok, pw, lane);
+        asm volatile("cp.async.commit_group;" ::: "memory");
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar_f + 8 * stg) : "memory");
       } else {
-        if (rows_ok == PT_BN) {
-          // a full tile (all but the last one of a sequence): no predicates, running pointers
+        if (rows_ok == P2_KT && nb[0] == 4 && (nb[1] == 4 || nb[1] == 0)) {
           const unsigned char* sp = tsrc + (size_t)pw * (size_t)(2 * rowlen) + 4 * lane;
           uint32_t db = du + (uint32_t)pw * 128u;
           const bool two = nb[1] > 0;
-          if (nb[0] == 4 && (!two || nb[1] == 4)) {
 #pragma unroll 4
-            for (int i = 0; i < PT_BN / 2; ++i) {
-              pt_cp4(db + swz[i & 3][0], sp, 4);
-              if (two) pt_cp4(db + swz[i & 3][1], sp + 128, 4);
-              sp += 4 * rowlen;                        // two rows on
-              db += 256;
-            }
-          } else {
-#pragma unroll 4
-            for (int i = 0; i < PT_BN / 2; ++i) {
-              if (nb[0] > 0) pt_cp4(db + swz[i & 3][0], sp, nb[0]);
-              if (two) pt_cp4(db + swz[i & 3][1], sp + 128, nb[1]);
-              sp += 4 * rowlen;
-              db += 256;
-            }
+          for (int i = 0; i < P2_KT / 2; ++i) {
+            pt_cp4(db + swz[i & 3][0], sp, 4);
+            if (two) pt_cp4(db + swz[i & 3][1], sp + 128, 4);
+            sp += 4 * rowlen;
+            db += 256;
           }
         } else {
 #pragma unroll 4
-          for (int i = 0; i < PT_BN / 2; ++i) {
+          for (int i = 0; i < P2_KT / 2; ++i) {
             const int r = pw + 2 * i;
-            const bool ok = r < rows_ok;               // rows past the end: zero fill, nothing is read
+            const bool ok = r < rows_ok;
             const uint32_t* src = reinterpret_cast<const uint32_t*>(tsrc + (size_t)(ok ? r : 0) * (size_t)(2 * rowlen));
             const uint32_t rb = du + (uint32_t)r * 128u;
             if (nb[0] > 0) pt_cp4(rb + swz[i & 3][0], src + lane, ok ? nb[0] : 0);
             if (nb[1] > 0) pt_cp4(rb + swz[i & 3][1], src + lane + 32, ok ? nb[1] : 0);
           }
         }
-      }
-      if (odd_len) {   // plain stores took part: wait, order them before the tensor-core (async proxy) reads, arrive
-        asm volatile("cp.async.commit_group;" ::: "memory");
-        asm volatile("cp.async.wait_group 0;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar_f + 8 * stg) : "memory");
-      } else {         // the arrival is triggered by the completion of this thread's copies: go on to the next tile
         asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar_f + 8 * stg) : "memory");
       }
-      if (++stg == nst) { stg = 0; ++use; }
+      if (++stg == P2_STAGES) { stg = 0; ++use; }
     }
-  } else if (warp == 4) {
-    // ================= MMA issue: S(t + 1) = Q K^T is issued before P(t) is waited for =================
+  } else if (warp == 8) {
+    // ================= MMA issue =================
     if (lane == 0) {
-      auto issue_s = [&](int tile) {
-        const int kbuf = tile % PT_KSTAGES;
-        const uint32_t kb = pt_smem(k_s + kbuf * PT_TILE_BYTES), td = tmem_base + 128u * (uint32_t)(tile & 1);
+      auto issue_s = [&](int Y, int tile) {
+        const uint32_t kb = pt_smem(k_s + (tile % P2_STAGES) * P2_KV_BYTES), qx = pt_smem(q_s + Y * P2_Q_BYTES);
+        const uint32_t td = tmem_base + 128u * (uint32_t)Y + 64u * (uint32_t)(tile & 1);
 #pragma unroll
-        for (int ks = 0; ks < DK; ++ks) {
-          const uint32_t o2 = (uint32_t)((ks >> 2) * PT_BM * 128 + (ks & 3) * 32);
-          pt_mma(td, pt_desc(pt_smem(q_s) + o2), pt_desc(kb + o2), IDESC_S, ks > 0 ? 1u : 0u);
-        }
-        pt_commit(bar_s + 8 * (tile & 1));
-        pt_commit(bar_ek + 8 * kbuf);
+        for (int ks = 0; ks < DK; ++ks)
+          pt_mma(td, pt_desc(qx + (uint32_t)((ks >> 2) * 16384 + (ks & 3) * 32)),
+                 pt_desc(kb + (uint32_t)((ks >> 2) * 8192 + (ks & 3) * 32)), IDESC_S, ks > 0 ? 1u : 0u);
+        pt_commit(bar_s + 8 * (2 * Y + (tile & 1)));
       };
-      bool ok = wait(bar_fk, 0);
+      bool ok = n_max > 0 && wait(bar_fk, 0);
       if (ok) {
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        issue_s(0);
+        for (int Y = 0; Y < 2; ++Y)
+          if (nt[Y] > 0) issue_s(Y, 0);
+        pt_commit(bar_ek);
       }
-      for (int tile = 0; ok && tile < n_tiles; ++tile) {
-        if (tile + 1 < n_tiles) {
-          if (!wait(bar_fk + 8 * ((tile + 1) % PT_KSTAGES), ((tile + 1) / PT_KSTAGES) & 1)) { ok = false; break; }
-          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the copies' writes before the MMA's reads
+      for (int tile = 0; ok && tile < n_max; ++tile) {
+        if (tile + 1 < n_max) {
+          const int kbuf = (tile + 1) % P2_STAGES;
+          if (!wait(bar_fk + 8 * kbuf, ((tile + 1) / P2_STAGES) & 1)) { ok = false; break; }
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-          issue_s(tile + 1);
+          for (int Y = 0; Y < 2; ++Y)
+            if (tile + 1 < nt[Y]) issue_s(Y, tile + 1);
+          pt_commit(bar_ek + 8 * kbuf);
         }
-        if (!wait(bar_fv + 8 * (tile % PT_VSTAGES), (tile / PT_VSTAGES) & 1)) { ok = false; break; }
-        if (!wait(bar_p, tile & 1)) { ok = false; break; }
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const uint32_t vb = pt_smem(v_s + (tile % PT_VSTAGES) * PT_TILE_BYTES);
+        const int vbuf = tile % P2_STAGES;
+        if (!wait(bar_fv + 8 * vbuf, (tile / P2_STAGES) & 1)) { ok = false; break; }
+        const uint32_t vb = pt_smem(v_s + vbuf * P2_KV_BYTES);
+        for (int Y = 0; Y < 2 && ok; ++Y) {
+          if (tile >= nt[Y]) continue;
+          if (!wait(bar_p + 8 * Y, tile & 1)) { ok = false; break; }
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          const uint32_t pa = pt_smem(p_s + Y * P2_P_BYTES);
 #pragma unroll
-        for (int ks = 0; ks < PT_BN / 16; ++ks) {
-          const uint32_t oa = (uint32_t)((ks >> 2) * PT_BM * 128 + (ks & 3) * 32);
-          // 16 keys = two 8-key groups of the N-major V tile
-          pt_mma(tmem_o, pt_desc(pt_smem(p_s) + oa), pt_desc_n(vb + (uint32_t)ks * 2048u), IDESC_O, (tile > 0 || ks > 0) ? 1u : 0u);
+          for (int ks = 0; ks < P2_KT / 16; ++ks)
+            pt_mma(tmem_base + 256u + 128u * (uint32_t)Y, pt_desc(pa + (uint32_t)ks * 32u), pt_desc_n2(vb + (uint32_t)ks * 2048u),
+                   IDESC_O, (tile > 0 || ks > 0) ? 1u : 0u);
+          pt_commit(bar_o + 8 * Y);
         }
-        pt_commit(bar_o);
-        pt_commit(bar_ev + 8 * (tile % PT_VSTAGES));
+        if (!ok) break;
+        pt_commit(bar_ev + 8 * vbuf);
       }
-      // every MMA issued above has completed before tensor memory is released
       pt_commit(bar_end);
       wait(bar_end, 0);
     }
     __syncwarp();
-  }
-  float l_run = 0.f;
-  const int row = tid;                               // warps 0-3: query row = TMEM lane
-  const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
-  bool rows_ok = true;
-  if (warp < 4) {
-    // ================= softmax: one thread per query row =================
-    const int pos = start + q0 + row;                // cache row of this thread's query
+  } else {
+    // ================= softmax group X: one thread per query row of tile X =================
+    const int q0x = q0 + 128 * X;
+    const int pos = start + q0x + row;
+    const int n_my = nt[X];
     float m_ref = -1.0e30f;
-    for (int tile = 0; tile < n_tiles; ++tile) {
-      const int j0 = tile * PT_BN;
-      const uint32_t trow = tmem_base + 128u * (uint32_t)(tile & 1) + lane_off;
-      if (!__all_sync(0xffffffffu, wait(bar_s + 8 * (tile & 1), (tile >> 1) & 1))) { rows_ok = false; break; }
+    bool rows_ok = true;
+    for (int tile = 0; tile < n_my; ++tile) {
+      const int j0 = tile * P2_KT;
+      const uint32_t trow = tmem_base + 128u * (uint32_t)X + 64u * (uint32_t)(tile & 1) + lane_off;
+      if (!__all_sync(0xffffffffu, wait(bar_s + 8 * (2 * X + (tile & 1)), (tile >> 1) & 1))) { rows_ok = false; break; }
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      // the whole S row in registers: four loads in flight, one wait
-      uint32_t r[128];
+      uint32_t r[64];
       pt_ld32_nowait(trow, *reinterpret_cast<uint32_t(*)[32]>(r));
       pt_ld32_nowait(trow + 32, *reinterpret_cast<uint32_t(*)[32]>(r + 32));
-      pt_ld32_nowait(trow + 64, *reinterpret_cast<uint32_t(*)[32]>(r + 64));
-      pt_ld32_nowait(trow + 96, *reinterpret_cast<uint32_t(*)[32]>(r + 96));
       asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-      // only the tiles that reach past the block's first query need the causal mask
-      const bool interior = j0 + PT_BN - 1 <= start + q0;
-      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};   // four chains instead of one of 128 steps
+      const bool interior = j0 + P2_KT - 1 <= start + q0x;   // no key of the tile is masked for any row of the tile
+      float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
       if (interior) {
 #pragma unroll
-        for (int j = 0; j < 128; ++j) mx4[j & 3] = fmaxf(mx4[j & 3], __uint_as_float(r[j]));
+        for (int j = 0; j < 64; ++j) mx4[j & 3] = fmaxf(mx4[j & 3], __uint_as_float(r[j]));
       } else {
 #pragma unroll
-        for (int j = 0; j < 128; ++j)
+        for (int j = 0; j < 64; ++j)
           if (j0 + j <= pos) mx4[j & 3] = fmaxf(mx4[j & 3], __uint_as_float(r[j]));
       }
-      // the scale is positive: the maximum commutes with it
       const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.qscale;
       float alpha = 1.f;
       if (mx > m_ref + 8.f) {          // lazy reference maximum: p stays <= 2^8
-        alpha = pt_ex2(m_ref - mx);    // first time: 2^(-1e30 - mx) = 0
+        alpha = pt_ex2(m_ref - mx);
         m_ref = mx;
         l_run *= alpha;
       }
-      // p = 2^(s - m_ref) as packed bf16 pairs (in place)
       const float nm = -m_ref;
       float ls[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-      for (int j = 0; j < 128; j += 2) {
+      for (int j = 0; j < 64; j += 2) {
         float p0 = pt_ex2(fmaf(__uint_as_float(r[j]), p.qscale, nm));
         float p1 = pt_ex2(fmaf(__uint_as_float(r[j + 1]), p.qscale, nm));
         if (!interior) {
           if (j0 + j > pos) p0 = 0.f;
           if (j0 + j + 1 > pos) p1 = 0.f;
         }
-        ls[(j >> 1) & 3] += p0 + p1;
         const __nv_bfloat162 v2 = __floats2bfloat162_rn(p0, p1);
-        r[j >> 1] = *reinterpret_cast<const uint32_t*>(&v2);
+        const uint32_t pk = *reinterpret_cast<const uint32_t*>(&v2);
+        // the row sum takes the rounded values the second MMA will see: a row with one key comes out exact
+        ls[(j >> 1) & 3] += __uint_as_float(pk << 16) + __uint_as_float(pk & 0xffff0000u);
+        r[j >> 1] = pk;
       }
       l_run += (ls[0] + ls[1]) + (ls[2] + ls[3]);
-      // the second MMA of the previous tile has read P and has added into O: wait for it before touching either
       if (tile > 0) {
-        if (!__all_sync(0xffffffffu, wait(bar_o, (tile - 1) & 1))) { rows_ok = false; break; }
+        if (!__all_sync(0xffffffffu, wait(bar_o + 8 * X, (tile - 1) & 1))) { rows_ok = false; break; }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        // rescale this warp's 32 accumulator rows in tensor memory (rare: the maximum is lazy)
-        if (__any_sync(0xffffffffu, alpha != 1.f)) {
+        if (__any_sync(0xffffffffu, alpha != 1.f)) {   // rare: rescale this warp's accumulator rows in tensor memory
 #pragma unroll 1
           for (int c0 = 0; c0 < NVP; c0 += 32) {
             uint32_t oc[32];
@@ -458,15 +445,15 @@ __global__ void __launch_bounds__(PT_THREADS, 1) prefill_tc_kernel(const PtParam
           asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
         }
       }
-      // P into the A-operand layout (this thread's row, 16 chunks of 8 keys)
+      unsigned char* pd = p_s + X * P2_P_BYTES;
 #pragma unroll
-      for (int ch = 0; ch < 16; ++ch)
-        *reinterpret_cast<uint4*>(p_s + pt_off(row, 8 * ch, PT_BM)) = make_uint4(r[4 * ch], r[4 * ch + 1], r[4 * ch + 2], r[4 * ch + 3]);
+      for (int ch = 0; ch < 8; ++ch)
+        *reinterpret_cast<uint4*>(pd + pt_off(row, 8 * ch, 128)) = make_uint4(r[4 * ch], r[4 * ch + 1], r[4 * ch + 2], r[4 * ch + 3]);
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-      asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar_p) : "memory");
+      asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar_p + 8 * X) : "memory");
     }
-    if (rows_ok && !__all_sync(0xffffffffu, wait(bar_o, (n_tiles - 1) & 1))) rows_ok = false;
+    if (rows_ok && n_my > 0) __all_sync(0xffffffffu, wait(bar_o + 8 * X, (n_my - 1) & 1));
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -476,9 +463,8 @@ __global__ void __launch_bounds__(PT_THREADS, 1) prefill_tc_kernel(const PtParam
     atomicCAS(&p.status[0], 0, (int)RAP_ETIMEOUT);
     p.status[1] = 0x60000000 | (blockIdx.x & 0xffffff);
   }
-  if (warp < 4 && !timed_out) {
-    // every row's thread reads its accumulator row (all lanes of the warp take part in the load)
-    const int t = q0 + row;
+  if (warp < 8 && !timed_out && nt[X] > 0) {
+    const int t = q0 + 128 * X + row;
     const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
     float* dst = p.out + (((size_t)b * p.T + min(t, p.T - 1)) * p.Hq + g) * p.dv;
 #pragma unroll 1
@@ -494,18 +480,18 @@ __global__ void __launch_bounds__(PT_THREADS, 1) prefill_tc_kernel(const PtParam
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   }
   __syncthreads();
-  if (warp == 4) {
+  if (warp == 8) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
   }
 }
 
 template <int DK, int NVP>
-rap_status launch_pt(rap_ctx* ctx, const PtParams& p, int B, cudaStream_t st) {
-  const int smem = (2 + PT_KSTAGES + PT_VSTAGES) * PT_TILE_BYTES + 128 + 1024;
-  RAP_CUDA_TRY(ctx, rap_raise_smem(ctx, prefill_tc_kernel<DK, NVP>, smem));
-  dim3 grid((p.T + PT_BM - 1) / PT_BM, p.Hq, B);
-  prefill_tc_kernel<DK, NVP><<<grid, PT_THREADS, smem, st>>>(p);
+rap_status launch_pt2(rap_ctx* ctx, const PtParams& p, int B, cudaStream_t st) {
+  const int smem = P2_SMEM + 1024;
+  RAP_CUDA_TRY(ctx, rap_raise_smem(ctx, prefill_tc2_kernel<DK, NVP>, smem));
+  dim3 grid((p.T + 255) / 256, p.Hq, B);
+  prefill_tc2_kernel<DK, NVP><<<grid, P2_THREADS, smem, st>>>(p);
   ctx->launches++;
   RAP_CUDA_TRY(ctx, cudaGetLastError());
   return RAP_OK;
@@ -524,7 +510,7 @@ rap_status rap_launch_prefill_attn_tc(rap_ctx* ctx, int B, int T, const void* q,
   p.T = T; p.Hq = d.n_q_heads; p.Hkv = d.n_kv_heads; p.P2 = P2; p.dv = dv; p.S_cap = S_cap;
   p.qscale = (float)(1.4426950408889634 / sqrt((double)d.head_dim));
   const int dk = (P2 + 15) / 16, nvp = (dv + 31) / 32 * 32;
-  if (dk <= 4 && nvp <= 64) return launch_pt<4, 64>(ctx, p, B, st);
-  if (dk <= 6 && nvp <= 96) return launch_pt<6, 96>(ctx, p, B, st);
-  return launch_pt<8, 128>(ctx, p, B, st);
+  if (dk <= 4 && nvp <= 64) return launch_pt2<4, 64>(ctx, p, B, st);
+  if (dk <= 6 && nvp <= 96) return launch_pt2<6, 96>(ctx, p, B, st);
+  return launch_pt2<8, 128>(ctx, p, B, st);
 }
