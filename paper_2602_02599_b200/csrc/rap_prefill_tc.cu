@@ -184,7 +184,7 @@ struct PtParams {
 
 // DK = k-steps of Q K^T (ceil(2P / 16)); NVP = d_v' rounded up to a multiple of 32 (N of the second MMA)
 template <int DK, int NVP>
-__global__ void __launch_bounds__(P2_THREADS, 1) prefill_tc2_kernel(const PtParams p) {
+__global__ void __launch_bounds__(P2_THREADS, 1) prefill_tc_kernel(const PtParams p) {
   extern __shared__ unsigned char pt_raw[];
   unsigned char* smem = pt_raw + ((1024u - (pt_smem(pt_raw) & 1023u)) & 1023u);
   unsigned char* q_s = smem;                                   // Q_A, Q_B
@@ -487,11 +487,11 @@ __global__ void __launch_bounds__(P2_THREADS, 1) prefill_tc2_kernel(const PtPara
 }
 
 template <int DK, int NVP>
-rap_status launch_pt2(rap_ctx* ctx, const PtParams& p, int B, cudaStream_t st) {
+rap_status launch_pt(rap_ctx* ctx, const PtParams& p, int B, cudaStream_t st) {
   const int smem = P2_SMEM + 1024;
-  RAP_CUDA_TRY(ctx, rap_raise_smem(ctx, prefill_tc2_kernel<DK, NVP>, smem));
+  RAP_CUDA_TRY(ctx, rap_raise_smem(ctx, prefill_tc_kernel<DK, NVP>, smem));
   dim3 grid((p.T + 255) / 256, p.Hq, B);
-  prefill_tc2_kernel<DK, NVP><<<grid, P2_THREADS, smem, st>>>(p);
+  prefill_tc_kernel<DK, NVP><<<grid, P2_THREADS, smem, st>>>(p);
   ctx->launches++;
   RAP_CUDA_TRY(ctx, cudaGetLastError());
   return RAP_OK;
@@ -510,7 +510,7 @@ rap_status rap_launch_prefill_attn_tc(rap_ctx* ctx, int B, int T, const void* q,
   p.T = T; p.Hq = d.n_q_heads; p.Hkv = d.n_kv_heads; p.P2 = P2; p.dv = dv; p.S_cap = S_cap;
   p.qscale = (float)(1.4426950408889634 / sqrt((double)d.head_dim));
   const int dk = (P2 + 15) / 16, nvp = (dv + 31) / 32 * 32;
-  if (dk <= 4 && nvp <= 64) return launch_pt2<4, 64>(ctx, p, B, st);
-  if (dk <= 6 && nvp <= 96) return launch_pt2<6, 96>(ctx, p, B, st);
-  return launch_pt2<8, 128>(ctx, p, B, st);
+  if (dk <= 4 && nvp <= 64) return launch_pt<4, 64>(ctx, p, B, st);
+  if (dk <= 6 && nvp <= 96) return launch_pt<6, 96>(ctx, p, B, st);
+  return launch_pt<8, 128>(ctx, p, B, st);
 }
