@@ -208,12 +208,13 @@ def test_attention_fp32_pipe_scan(name, n_split):
 
 
 @pytest.mark.parametrize("G,P,dv", [(8, 45, 90), (1, 58, 115), (6, 51, 102), (2, 45, 90), (4, 22, 44), (4, 20, 40),
-                                    (5, 41, 82), (3, 63, 126), (4, 64, 64), (7, 32, 64), (8, 64, 128)])
+                                    (5, 41, 82), (3, 63, 126), (4, 64, 64), (7, 32, 64), (8, 64, 128),
+                                    (4, 24, 48), (5, 16, 32), (3, 48, 96), (4, 56, 112)])
 def test_attention_tensor_core_scan_head_shapes(G, P, dv):
     """The tensor-core form of the scan, forced (variant 4 fails instead of falling back): group sizes 1..8,
-    odd and even d_v', the three row-spreading steps of the fragment loads (P odd, P = 2 mod 4, P = 0 mod 4)
-    and the shapes staged through swizzling tensor maps; ragged lengths, a block with one row, both split
-    modes."""
+    odd and even d_v', the three row-spreading steps of the fragment loads (P odd, P = 2 mod 4, P = 0 mod 4),
+    the shapes staged through swizzling tensor maps and other multiples of 8 (which keep some bank conflicts);
+    ragged lengths, a block with one row, both split modes."""
     from dataclasses import replace
     base = synth.scaled_down(synth.LLAMA_8B, n_layers=1, batch=4, seq=3000)
     w = replace(base, n_pairs=P, n_vch=dv, n_q_heads=G * base.n_kv_heads)
@@ -393,8 +394,7 @@ def test_layer_adaptive_budgets_end_to_end():
 
 @pytest.mark.parametrize("P,dv", [(24, 48), (40, 80), (41, 82), (56, 112), (16, 32), (63, 126)])
 def test_layer_adaptive_head_shapes_attention(P, dv):
-    """Head shapes that layer-adaptive budgets produce (d_v' = 2P): K rows that are multiples of 32 bytes
-    take the rotated logits mapping with a partly filled last unit group, the others the chunked one."""
+    """Head shapes that layer-adaptive budgets produce (d_v' = 2P), through the default tier."""
     from dataclasses import replace
     w = replace(synth.scaled_down(synth.LLAMA_8B, n_layers=1, batch=3, seq=3000), n_pairs=P, n_vch=dv)
     _random_attn_case(w, [3000, 1777, 1], 0, seed=P)
