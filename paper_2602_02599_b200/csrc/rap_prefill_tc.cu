@@ -1,6 +1,6 @@
 // tcgen05 version of rap_prefill_attn: causal attention of a block of T new tokens per sequence over the
 // reduced dims (Eq. 2 for every t of the block; 2P retained K dims, d_v' retained V channels, scale
-// 1/sqrt(D)).  One CTA (one per SM, 416 threads) handles 256 consecutive queries of one query head as two query
+// 1/sqrt(D)).  One CTA (one per SM, 448 threads) handles 256 consecutive queries of one query head as two query
 // tiles A and B of 128, and walks 64-key tiles up to each tile's causal limit:
 //   S_X    = Q_X K^T    tcgen05.mma (M = 128 queries, N = 64 keys, K = 2P in steps of 16), accumulator in TMEM,
 //                       double buffered per query tile: S of key tile t + 1 is issued before P of t is waited for
@@ -11,12 +11,13 @@
 //                       tiles; a warp rescales its 32 accumulator rows (tcgen05.ld / st) only in the rare tile
 //                       where the lazy maximum moved.
 // While one group runs its softmax the tensor core works for the other, and a staged K / V tile serves 256 queries.
-// Cache rows are not multiples of 16 bytes, so TMA tensor maps cannot describe them: four producer warps (9-10: K,
-// 11-12: V) stage the tiles by hand (4-byte cp.async) into rings of four buffers each, in the 128-byte-swizzled
+// Cache rows are not multiples of 16 bytes, so TMA tensor maps cannot describe them: four producer warps (10-11: K,
+// 12-13: V) stage the tiles by hand (4-byte cp.async) into rings of four buffers each, in the 128-byte-swizzled
 // layouts the MMA descriptors expect (K as stored = K-major; V as stored = the N-major form of the B operand, so
 // nothing is transposed); rows past the sequence end and pad columns are zeros.  The copies' completion arrives on
 // the buffer's mbarrier by itself; the consumer issues the proxy fence.  The roles meet only on mbarriers; every wait
-// is bounded and gives up early once another role has given up.  One lane of warp 8 issues all MMAs.
+// is bounded and gives up early once another role has given up.  Lane 0 of warp 8 issues the MMAs of query tile A,
+// lane 0 of warp 9 those of B.
 #include <math.h>
 
 #include "rap_internal.h"
@@ -24,7 +25,7 @@
 namespace {
 
 constexpr int P2_KT = 64;                              // keys per tile
-constexpr int P2_THREADS = 416;
+constexpr int P2_THREADS = 448;
 constexpr int P2_STAGES = 4;                           // K buffers and V buffers
 constexpr int P2_Q_BYTES = 2 * 128 * 128;              // [128 queries][<=128 dims]: two 64-element atom columns
 constexpr int P2_P_BYTES = 128 * 128;                  // [128 queries][64 keys]
@@ -195,8 +196,8 @@ __global__ void __launch_bounds__(P2_THREADS, 1) prefill_tc_kernel(const PtParam
   const uint32_t bar_fk = pt_smem(tail), bar_ek = bar_fk + 32, bar_fv = bar_fk + 64, bar_ev = bar_fk + 96,
                  bar_s = bar_fk + 128 /* [X][2] */, bar_p = bar_fk + 160 /* [X] */, bar_o = bar_fk + 176 /* [X] */,
                  bar_end = bar_fk + 192;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 200);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 204);
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 208);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 212);
 
   const int qb = blockIdx.x, g = blockIdx.y, b = blockIdx.z;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -218,9 +219,9 @@ __global__ void __launch_bounds__(P2_THREADS, 1) prefill_tc_kernel(const PtParam
   if (tid == 0) {
     for (int i = 0; i < P2_STAGES; ++i) {
       pt_mbar_init(bar_fk + 8 * i, 64);
-      pt_mbar_init(bar_ek + 8 * i, 1);
+      pt_mbar_init(bar_ek + 8 * i, 2);               // both MMA-issuing lanes release a buffer
       pt_mbar_init(bar_fv + 8 * i, 64);
-      pt_mbar_init(bar_ev + 8 * i, 1);
+      pt_mbar_init(bar_ev + 8 * i, 2);
     }
     for (int i = 0; i < 4; ++i) pt_mbar_init(bar_s + 8 * i, 1);
     for (int X = 0; X < 2; ++X) {
@@ -228,6 +229,7 @@ __global__ void __launch_bounds__(P2_THREADS, 1) prefill_tc_kernel(const PtParam
       pt_mbar_init(bar_o + 8 * X, 1);
     }
     pt_mbar_init(bar_end, 1);
+    pt_mbar_init(bar_end + 8, 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -270,10 +272,10 @@ __global__ void __launch_bounds__(P2_THREADS, 1) prefill_tc_kernel(const PtParam
   const int row = (warp & 3) * 32 + lane;
   const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
   const uint32_t tmem_o = tmem_base + 256 + 128 * X;
-  if (warp >= 9) {
-    // ================= producers: warps 9-10 stage K, warps 11-12 stage V, in order, tiles of 64 rows =================
-    const bool is_v = warp >= 11;
-    const int pw = (warp - 9) & 1;
+  if (warp >= 10) {
+    // ================= producers: warps 10-11 stage K, warps 12-13 stage V, in order, tiles of 64 rows =================
+    const bool is_v = warp >= 12;
+    const int pw = (warp - 10) & 1;
     const int rowlen = is_v ? p.dv : p.P2;
     const unsigned char* src0 = reinterpret_cast<const unsigned char*>(is_v ? vg : kg);
     unsigned char* ring = is_v ? v_s : k_s;
@@ -328,25 +330,34 @@ __global__ void __launch_bounds__(P2_THREADS, 1) prefill_tc_kernel(const PtParam
       }
       if (++stg == P2_STAGES) { stg = 0; ++use; }
     }
-  } else if (warp == 8) {
-    // ================= MMA issue =================
+  } else if (warp >= 8) {
+    // ================= MMA issue: lane 0 of warp 8 for query tile A, of warp 9 for query tile B =================
+    // Two issuing lanes halve the serial chain of waits, fences, descriptors and commits per key tile.  A buffer of
+    // the K / V rings is free when both lanes have committed past it; a lane whose tile needs no more keys keeps
+    // arriving in step (after the buffer was filled), so the phases stay aligned.
     if (lane == 0) {
-      auto issue_s = [&](int Y, int tile) {
-        const uint32_t kb = pt_smem(k_s + (tile % P2_STAGES) * P2_KV_BYTES), qx = pt_smem(q_s + Y * P2_Q_BYTES);
-        const uint32_t td = tmem_base + 128u * (uint32_t)Y + 64u * (uint32_t)(tile & 1);
+      const int Y = warp - 8, n_y = nt[Y];
+      const uint32_t qx = pt_smem(q_s + Y * P2_Q_BYTES), pa = pt_smem(p_s + Y * P2_P_BYTES);
+      const uint32_t tmem_sy = tmem_base + 128u * (uint32_t)Y, tmem_oy = tmem_base + 256u + 128u * (uint32_t)Y;
+      auto issue_s = [&](int tile) {
+        const uint32_t kb = pt_smem(k_s + (tile % P2_STAGES) * P2_KV_BYTES);
+        const uint32_t td = tmem_sy + 64u * (uint32_t)(tile & 1);
 #pragma unroll
         for (int ks = 0; ks < DK; ++ks)
           pt_mma(td, pt_desc(qx + (uint32_t)((ks >> 2) * 16384 + (ks & 3) * 32)),
                  pt_desc(kb + (uint32_t)((ks >> 2) * 8192 + (ks & 3) * 32)), IDESC_S, ks > 0 ? 1u : 0u);
         pt_commit(bar_s + 8 * (2 * Y + (tile & 1)));
       };
-      bool ok = n_max > 0 && wait(bar_fk, 0);
+      auto release = [&](uint32_t bar, bool issued) {   // after MMAs: when they complete; otherwise at once
+        if (issued) pt_commit(bar);
+        else asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+      };
+      bool ok = wait(bar_fk, 0);
       if (ok) {
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        for (int Y = 0; Y < 2; ++Y)
-          if (nt[Y] > 0) issue_s(Y, 0);
-        pt_commit(bar_ek);
+        if (n_y > 0) issue_s(0);
+        release(bar_ek, n_y > 0);
       }
       for (int tile = 0; ok && tile < n_max; ++tile) {
         if (tile + 1 < n_max) {
@@ -354,30 +365,27 @@ __global__ void __launch_bounds__(P2_THREADS, 1) prefill_tc_kernel(const PtParam
           if (!wait(bar_fk + 8 * kbuf, ((tile + 1) / P2_STAGES) & 1)) { ok = false; break; }
           asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-          for (int Y = 0; Y < 2; ++Y)
-            if (tile + 1 < nt[Y]) issue_s(Y, tile + 1);
-          pt_commit(bar_ek + 8 * kbuf);
+          if (tile + 1 < n_y) issue_s(tile + 1);
+          release(bar_ek + 8 * kbuf, tile + 1 < n_y);
         }
         const int vbuf = tile % P2_STAGES;
         if (!wait(bar_fv + 8 * vbuf, (tile / P2_STAGES) & 1)) { ok = false; break; }
-        const uint32_t vb = pt_smem(v_s + vbuf * P2_KV_BYTES);
-        for (int Y = 0; Y < 2 && ok; ++Y) {
-          if (tile >= nt[Y]) continue;
+        if (tile < n_y) {
           if (!wait(bar_p + 8 * Y, tile & 1)) { ok = false; break; }
           asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-          const uint32_t pa = pt_smem(p_s + Y * P2_P_BYTES);
+          const uint32_t vb = pt_smem(v_s + vbuf * P2_KV_BYTES);
 #pragma unroll
           for (int ks = 0; ks < P2_KT / 16; ++ks)
-            pt_mma(tmem_base + 256u + 128u * (uint32_t)Y, pt_desc(pa + (uint32_t)ks * 32u), pt_desc_n2(vb + (uint32_t)ks * 2048u),
-                   IDESC_O, (tile > 0 || ks > 0) ? 1u : 0u);
+            pt_mma(tmem_oy, pt_desc(pa + (uint32_t)ks * 32u), pt_desc_n2(vb + (uint32_t)ks * 2048u), IDESC_O,
+                   (tile > 0 || ks > 0) ? 1u : 0u);
           pt_commit(bar_o + 8 * Y);
         }
-        if (!ok) break;
-        pt_commit(bar_ev + 8 * vbuf);
+        release(bar_ev + 8 * vbuf, tile < n_y);
       }
-      pt_commit(bar_end);
-      wait(bar_end, 0);
+      // every MMA issued above has completed before tensor memory is released
+      pt_commit(bar_end + 8 * Y);
+      wait(bar_end + 8 * Y, 0);
     }
     __syncwarp();
   } else {
