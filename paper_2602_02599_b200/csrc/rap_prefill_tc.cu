@@ -423,19 +423,30 @@ __global__ void __launch_bounds__(P2_THREADS, 1) prefill_tc_kernel(const PtParam
       }
       const float nm = -m_ref;
       float ls[4] = {0.f, 0.f, 0.f, 0.f};
+      if (interior) {
+        // no mask; rows with at least 64 keys before them: the row sum adds the unrounded weights (one instruction)
 #pragma unroll
-      for (int j = 0; j < 64; j += 2) {
-        float p0 = pt_ex2(fmaf(__uint_as_float(r[j]), p.qscale, nm));
-        float p1 = pt_ex2(fmaf(__uint_as_float(r[j + 1]), p.qscale, nm));
-        if (!interior) {
+        for (int j = 0; j < 64; j += 2) {
+          const float p0 = pt_ex2(fmaf(__uint_as_float(r[j]), p.qscale, nm));
+          const float p1 = pt_ex2(fmaf(__uint_as_float(r[j + 1]), p.qscale, nm));
+          ls[(j >> 1) & 3] += p0 + p1;
+          const __nv_bfloat162 v2 = __floats2bfloat162_rn(p0, p1);
+          r[j >> 1] = *reinterpret_cast<const uint32_t*>(&v2);
+        }
+      } else {
+        // diagonal tile: causal mask, and the row sum takes the rounded values the second MMA will see, so that a
+        // row with one key comes out exact (rows with few keys have only such tiles)
+#pragma unroll
+        for (int j = 0; j < 64; j += 2) {
+          float p0 = pt_ex2(fmaf(__uint_as_float(r[j]), p.qscale, nm));
+          float p1 = pt_ex2(fmaf(__uint_as_float(r[j + 1]), p.qscale, nm));
           if (j0 + j > pos) p0 = 0.f;
           if (j0 + j + 1 > pos) p1 = 0.f;
+          const __nv_bfloat162 v2 = __floats2bfloat162_rn(p0, p1);
+          const uint32_t pk = *reinterpret_cast<const uint32_t*>(&v2);
+          ls[(j >> 1) & 3] += __uint_as_float(pk << 16) + __uint_as_float(pk & 0xffff0000u);
+          r[j >> 1] = pk;
         }
-        const __nv_bfloat162 v2 = __floats2bfloat162_rn(p0, p1);
-        const uint32_t pk = *reinterpret_cast<const uint32_t*>(&v2);
-        // the row sum takes the rounded values the second MMA will see: a row with one key comes out exact
-        ls[(j >> 1) & 3] += __uint_as_float(pk << 16) + __uint_as_float(pk & 0xffff0000u);
-        r[j >> 1] = pk;
       }
       l_run += (ls[0] + ls[1]) + (ls[2] + ls[3]);
       if (tile > 0) {
