@@ -425,13 +425,28 @@ __global__ void __launch_bounds__(P2_THREADS, 1) prefill_tc_kernel(const PtParam
       float ls[4] = {0.f, 0.f, 0.f, 0.f};
       if (interior) {
         // no mask; rows with at least 64 keys before them: the row sum adds the unrounded weights (one instruction)
+        // two logits per packed FMA, two weights per packed add
+        uint64_t qs2, nm2, l2[4] = {0ull, 0ull, 0ull, 0ull};
+        asm("mov.b64 %0, {%1, %1};" : "=l"(qs2) : "f"(p.qscale));
+        asm("mov.b64 %0, {%1, %1};" : "=l"(nm2) : "f"(nm));
 #pragma unroll
         for (int j = 0; j < 64; j += 2) {
-          const float p0 = pt_ex2(fmaf(__uint_as_float(r[j]), p.qscale, nm));
-          const float p1 = pt_ex2(fmaf(__uint_as_float(r[j + 1]), p.qscale, nm));
-          ls[(j >> 1) & 3] += p0 + p1;
+          uint64_t s2, x2, p2;
+          asm("mov.b64 %0, {%1, %2};" : "=l"(s2) : "r"(r[j]), "r"(r[j + 1]));
+          asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(x2) : "l"(s2), "l"(qs2), "l"(nm2));
+          float x0, x1;
+          asm("mov.b64 {%0, %1}, %2;" : "=f"(x0), "=f"(x1) : "l"(x2));
+          const float p0 = pt_ex2(x0), p1 = pt_ex2(x1);
+          asm("mov.b64 %0, {%1, %2};" : "=l"(p2) : "f"(p0), "f"(p1));
+          asm("add.rn.f32x2 %0, %1, %2;" : "=l"(l2[(j >> 1) & 3]) : "l"(l2[(j >> 1) & 3]), "l"(p2));
           const __nv_bfloat162 v2 = __floats2bfloat162_rn(p0, p1);
           r[j >> 1] = *reinterpret_cast<const uint32_t*>(&v2);
+        }
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          float a0, a1;
+          asm("mov.b64 {%0, %1}, %2;" : "=f"(a0), "=f"(a1) : "l"(l2[k]));
+          ls[k] += a0 + a1;
         }
       } else {
         // diagonal tile: causal mask, and the row sum takes the rounded values the second MMA will see, so that a
