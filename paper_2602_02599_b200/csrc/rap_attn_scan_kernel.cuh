@@ -1,5 +1,6 @@
-// Shape-specialised bf16 split-KV scan for rap_decode_attn (Eq. 2 on the retained dims, Eq. 7,
-// scale 1/sqrt(D)): the kernel the 3B / 8B / 14B-shaped workloads run.
+// Shape-specialised bf16 split-KV scan for rap_decode_attn on the plain FP32 pipes (Eq. 2 on the retained dims,
+// Eq. 7, scale 1/sqrt(D)): the tier behind the tensor-core form of the scan (rap_attn_mma_kernel.cuh), kept for
+// cross-checks and for the low-rank comparator's full-width K.
 //
 // The scan reads every cache byte once and does G flops per byte, so HBM bandwidth bounds it;
 // what decides whether it gets there is the number of issue slots spent per cache word on the
@@ -21,7 +22,8 @@
 //     a logit exceeds it by more than 8, so p = 2^(s - m_ref) <= 256 and most tiles need neither
 //     shuffles nor a rescale; the row sum stays per lane until the end of the scan.
 //   * PV: thread (row group, channel pair) accumulates its rows two at a time per packed FMA.
-//   * partials (acc[d_v'], m, l) of the split go to the workspace; a combine kernel merges.
+//   * partials (acc[d_v'], m, l) of the split go to the workspace; in balanced mode the CTA that delivers a unit's
+//     last partial merges them, with an explicit n_split a combine kernel does.
 // Every mbarrier wait is bounded: on timeout the CTA records RAP_ETIMEOUT and leaves.
 #pragma once
 #include "rap_attn_common.cuh"
