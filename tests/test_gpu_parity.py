@@ -164,8 +164,9 @@ def test_adjacent_pairing_end_to_end():
     _end_to_end(w, [40])
 
 
-def _random_attn_case(w, lens, n_split, seed=0, variant=0):
-    """rap_decode_attn alone on random caches (no projection), every unit checked."""
+def _random_attn_case(w, lens, n_split, seed=0, variant=0, q_gain=1.0, ramp=0.0):
+    """rap_decode_attn alone on random caches (no projection), every unit checked.  q_gain scales q (peaked
+    softmax); ramp > 0 makes the K rows grow with the position (the running maximum keeps moving)."""
     st = DecodeStack(w, s_cap=((max(lens) + 8 + 7) // 8) * 8)
     st.ctx.rap_set_attn_variant(variant)
     ks, vs = synth.draw_scores(w)
@@ -176,7 +177,11 @@ def _random_attn_case(w, lens, n_split, seed=0, variant=0):
     for l in range(w.n_layers):
         st.k_cache[l].normal_(0, sig, generator=g)
         st.v_cache[l].normal_(0, sig, generator=g)
-    q = torch.empty((w.batch, w.n_q_heads, P2), dtype=st.dt, device=st.device).normal_(0, sig, generator=g)
+    q = torch.empty((w.batch, w.n_q_heads, P2), dtype=st.dt, device=st.device).normal_(0, sig * q_gain, generator=g)
+    if ramp > 0:
+        pos = torch.arange(st.s_cap, device=st.device, dtype=torch.float32).view(1, 1, -1, 1)
+        for l in range(w.n_layers):
+            st.k_cache[l].copy_((st.k_cache[l].float() * (1.0 + ramp * pos)).to(st.dt))
     dl = torch.tensor(lens, dtype=torch.int32, device=st.device)
     for l in range(w.n_layers):
         out = st.decode_attn(l, q, dl, int(max(lens)), n_split=n_split)
@@ -220,6 +225,17 @@ def test_attention_tensor_core_scan_head_shapes(G, P, dv):
     w = replace(base, n_pairs=P, n_vch=dv, n_q_heads=G * base.n_kv_heads)
     _random_attn_case(w, [3000, 1777, 1, 33], 0, seed=P + G, variant=4)
     _random_attn_case(w, [129, 0, 2999, 96], 3, seed=P, variant=4)
+
+
+@pytest.mark.parametrize("variant", [4, 3])
+@pytest.mark.parametrize("q_gain,ramp", [(12.0, 0.0), (3.0, 0.002), (0.05, 0.0)])
+def test_attention_peaked_moving_and_flat_softmax(variant, q_gain, ramp):
+    """Logit regimes that exercise the lazy reference maximum of both shape-specialised scans: nearly one-hot
+    weights (large q), a maximum that keeps rising along the sequence (K grows with the position, so every
+    few blocks rescale the accumulators) and nearly uniform weights."""
+    w = synth.scaled_down(synth.LLAMA_8B, n_layers=1, batch=3, seq=2500)
+    _random_attn_case(w, [2500, 1333, 40], 0, seed=7, variant=variant, q_gain=q_gain, ramp=ramp)
+    _random_attn_case(w, [2500, 1333, 40], 4, seed=8, variant=variant, q_gain=q_gain, ramp=ramp)
 
 
 def test_attention_generic_variant_matches():
