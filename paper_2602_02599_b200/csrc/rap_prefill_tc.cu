@@ -424,7 +424,7 @@ __global__ void __launch_bounds__(P2_THREADS, 1) prefill_tc_kernel(const PtParam
       const float nm = -m_ref;
       float ls[4] = {0.f, 0.f, 0.f, 0.f};
       if (interior) {
-        // no mask; rows with at least 64 keys before them: the row sum adds the unrounded weights (one instruction)
+        // no mask
         // two logits per packed FMA, two weights per packed add
         uint64_t qs2, nm2, l2[4] = {0ull, 0ull, 0ull, 0ull};
         asm("mov.b64 %0, {%1, %1};" : "=l"(qs2) : "f"(p.qscale));
@@ -437,10 +437,12 @@ __global__ void __launch_bounds__(P2_THREADS, 1) prefill_tc_kernel(const PtParam
           float x0, x1;
           asm("mov.b64 {%0, %1}, %2;" : "=f"(x0), "=f"(x1) : "l"(x2));
           const float p0 = pt_ex2(x0), p1 = pt_ex2(x1);
-          asm("mov.b64 %0, {%1, %2};" : "=l"(p2) : "f"(p0), "f"(p1));
-          asm("add.rn.f32x2 %0, %1, %2;" : "=l"(l2[(j >> 1) & 3]) : "l"(l2[(j >> 1) & 3]), "l"(p2));
           const __nv_bfloat162 v2 = __floats2bfloat162_rn(p0, p1);
-          r[j >> 1] = *reinterpret_cast<const uint32_t*>(&v2);
+          const uint32_t pk = *reinterpret_cast<const uint32_t*>(&v2);
+          // the row sum takes the rounded weights the second MMA will see (a one-hot row comes out exact)
+          asm("mov.b64 %0, {%1, %2};" : "=l"(p2) : "r"(pk << 16), "r"(pk & 0xffff0000u));
+          asm("add.rn.f32x2 %0, %1, %2;" : "=l"(l2[(j >> 1) & 3]) : "l"(l2[(j >> 1) & 3]), "l"(p2));
+          r[j >> 1] = pk;
         }
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
@@ -449,8 +451,7 @@ __global__ void __launch_bounds__(P2_THREADS, 1) prefill_tc_kernel(const PtParam
           ls[k] += a0 + a1;
         }
       } else {
-        // diagonal tile: causal mask, and the row sum takes the rounded values the second MMA will see, so that a
-        // row with one key comes out exact (rows with few keys have only such tiles)
+        // diagonal tile: causal mask
 #pragma unroll
         for (int j = 0; j < 64; j += 2) {
           float p0 = pt_ex2(fmaf(__uint_as_float(r[j]), p.qscale, nm));

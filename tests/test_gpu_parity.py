@@ -461,6 +461,10 @@ def test_decode_step_replays_from_a_cuda_graph():
 @pytest.mark.parametrize("name,T,starts", [("8b", 150, [0, 37]), ("3b", 100, [5, 0]), ("14b", 70, [64, 1]),
                                            ("sweep1.0", 130, [0, 200]), ("sweep0.8", 65, [63, 0]), ("sweep0.5", 128, [0, 128])])
 def test_prefill_attn_matches_oracle(name, T, starts):
+    _prefill_case(name, T, starts)
+
+
+def _prefill_case(name, T, starts, q_gain=1.0, ramp=0.0):
     """rap_prefill_attn (tensor-core causal block attention on the reduced dims) against the oracle's masked
     matrix form on the same bf16 caches and q~: several query blocks, ragged starts, tile-boundary lengths."""
     w = synth.scaled_down(synth.CONFIGS[name], n_layers=1, batch=len(starts), seq=max(starts) + T)
@@ -471,7 +475,10 @@ def test_prefill_attn_matches_oracle(name, T, starts):
     st.k_cache[0].normal_(0, sig, generator=g)
     st.v_cache[0].normal_(0, sig, generator=g)
     B, Hq, P2, dv = w.batch, w.n_q_heads, 2 * w.n_pairs, w.n_vch
-    q = torch.empty((B, T, Hq, P2), dtype=st.dt, device=st.device).normal_(0, sig, generator=g)
+    q = torch.empty((B, T, Hq, P2), dtype=st.dt, device=st.device).normal_(0, sig * q_gain, generator=g)
+    if ramp > 0:      # K grows with the position: the running maximum keeps moving, the accumulators get rescaled
+        pos = torch.arange(st.s_cap, device=st.device, dtype=torch.float32).view(1, 1, -1, 1)
+        st.k_cache[0].copy_((st.k_cache[0].float() * (1.0 + ramp * pos)).to(st.dt))
     ds = torch.tensor(starts, dtype=torch.int32, device=st.device)
     want = O.prefill_attn(util.to_np64(q), util.to_np64(st.k_cache[0]), util.to_np64(st.v_cache[0]), starts, w.head_dim)
     for variant in (0, 1):       # 0: tcgen05 kernel, 1: warp-level mma.sync kernel
@@ -482,6 +489,13 @@ def test_prefill_attn_matches_oracle(name, T, starts):
         util.check_attn(util.to_np64(out).reshape(B * T, Hq, dv), want.reshape(B * T, Hq, dv), w.dtype)
     assert st.ctx.rap_get_last_device_status() == (0, 0)
     st.close()
+
+
+@pytest.mark.parametrize("q_gain,ramp", [(10.0, 0.0), (3.0, 0.004)])
+def test_prefill_attn_peaked_and_moving_maximum(q_gain, ramp):
+    """Nearly one-hot weights, and a maximum that rises along the keys so that the kernels keep rescaling their
+    accumulators (in tensor memory for the tcgen05 kernel)."""
+    _prefill_case("8b", 300, [0, 500], q_gain=q_gain, ramp=ramp)
 
 
 def _decode_step_with_tables(st, tabs, w, lens):
