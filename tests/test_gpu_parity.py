@@ -225,6 +225,9 @@ def test_attention_tensor_core_scan_head_shapes(G, P, dv):
     w = replace(base, n_pairs=P, n_vch=dv, n_q_heads=G * base.n_kv_heads)
     _random_attn_case(w, [3000, 1777, 1, 33], 0, seed=P + G, variant=4)
     _random_attn_case(w, [129, 0, 2999, 96], 3, seed=P, variant=4)
+    # a cache capacity that is not a multiple of the 32-row block: the last block of every unit reaches into the
+    # next unit's rows, and the last unit's past the end of the cache (where tensor-map boxes are zero-filled)
+    _random_attn_case(w, [3010, 3010, 3010, 3010], 0, seed=G, variant=4)
 
 
 @pytest.mark.parametrize("variant", [4, 3])
