@@ -141,6 +141,33 @@ def test_config1_split_counts(n_split):
     _end_to_end(synth.TINY, [synth.TINY.seq], n_split=n_split)
 
 
+def test_rope_at_large_positions_fp32():
+    """Index-aware RoPE far out (positions up to 10^6 with the cache slot kept small): the device reduces the fp64
+    angle before it takes the fp32 sine and cosine, so q~ and the appended K row stay within the fp32 tolerance."""
+    w = synth.TINY
+    ks, vs = synth.draw_scores(w)
+    st, tabs, w_host = util.build_small_stack(w, ks, vs, full_weights=True, max_rows=8)
+    pos = np.array([0, 1, 4097, 32768, 99999, 1000003], dtype=np.int32)
+    T = len(pos)
+    X = synth.draw_hidden(w, 0, 7, T)
+    dx = torch.from_numpy(X).to(st.device).to(st.dt).contiguous()
+    dq = torch.empty((T, w.n_q_heads, 2 * w.n_pairs), dtype=st.dt, device=st.device)
+    sid = torch.zeros(T, dtype=torch.int32, device=st.device)
+    slot = torch.arange(T, dtype=torch.int32, device=st.device)
+    st.qkv_rope_append(0, dx, sid, torch.from_numpy(pos).to(st.device), slot, T - 1, q_out=dq)
+    torch.cuda.synchronize()
+    q, k, v = O.qkv_rope(O.round_storage(X, w.dtype), w_host[0], None, pos, tabs["inv_freq"][0], w.n_q_heads,
+                         w.n_kv_heads, w.n_pairs, w.n_vch)
+    util.check_projection(util.to_np64(dq), q, w.dtype, "q at large positions")
+    Kd = util.to_np64(st.k_cache[0])
+    k_dev = np.stack([Kd[0, :, t, :] for t in range(T)])
+    util.check_projection(k_dev, k, w.dtype, "k at large positions")
+    # the rotation is not the identity out there: an unrotated row would miss by far more than the tolerance
+    assert np.abs(k_dev[-1] - O.qkv_rope(O.round_storage(X, w.dtype), w_host[0], None, np.zeros(T, np.int32),
+                                         tabs["inv_freq"][0], w.n_q_heads, w.n_kv_heads, w.n_pairs, w.n_vch)[1][-1]).max() > 1e-2
+    st.close()
+
+
 def test_tiny_with_bias():
     _end_to_end(synth.TINY, [0], with_bias=True)
 
