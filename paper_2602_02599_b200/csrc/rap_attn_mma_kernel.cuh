@@ -501,38 +501,67 @@ __global__ void __launch_bounds__(MmaCfg<G, WK, DV>::THREADS, 2) attn_mma_kernel
       __syncthreads();
       if (*s_last) {
         __threadfence();
-        float* wgt = red;        // [G][RAP_MAX_SPLIT] segment weights, then G reciprocals of the denominators
         const float* ub = p.ws + ((size_t)b * p.Hq + (size_t)h * G) * RAP_MAX_SPLIT * (size_t)(DV + 2);
-        for (int g = warp; g < G; g += NW) {
-          const float* gb = ub + (size_t)g * ws_head;
-          float mv[2], lv[2];
+        if (nseg <= 4) {
+          // few partials (the usual case): every output thread loads the maxima, the sums and its own channel of all
+          // partials at once -- one round trip through the memory system instead of two -- and weighs them itself
+          for (int i = tid; i < G * DV; i += THREADS) {
+            const int g = i / DV, c = i - g * DV;
+            const float* gb = ub + (size_t)g * ws_head;
+            float mv[4], lv[4], av[4];
 #pragma unroll
-          for (int k = 0; k < 2; ++k) {
-            const int sg = lane + 32 * k;
-            lv[k] = sg < nseg ? __ldcg(gb + (size_t)sg * (DV + 2) + DV + 1) : 0.f;
-            mv[k] = (sg < nseg && lv[k] > 0.f) ? __ldcg(gb + (size_t)sg * (DV + 2) + DV) : -INFINITY;
+            for (int sg = 0; sg < 4; ++sg) {
+              const bool on = sg < nseg;
+              lv[sg] = on ? __ldcg(gb + (size_t)sg * (DV + 2) + DV + 1) : 0.f;
+              mv[sg] = on ? __ldcg(gb + (size_t)sg * (DV + 2) + DV) : -INFINITY;
+              av[sg] = on ? __ldcg(gb + (size_t)sg * (DV + 2) + c) : 0.f;
+            }
+            float M = -INFINITY;
+#pragma unroll
+            for (int sg = 0; sg < 4; ++sg)
+              if (lv[sg] > 0.f) M = fmaxf(M, mv[sg]);
+            float den = 0.f, num = 0.f;
+#pragma unroll
+            for (int sg = 0; sg < 4; ++sg) {
+              const float wk = lv[sg] > 0.f ? exp2f(mv[sg] - M) : 0.f;
+              den += wk * lv[sg];
+              num += wk * av[sg];
+            }
+            p.out[((size_t)b * p.Hq + (size_t)h * G + g) * DV + c] = den > 0.f ? num / den : 0.f;
           }
-          float M = fmaxf(mv[0], mv[1]);
-#pragma unroll
-          for (int o2 = 16; o2 > 0; o2 >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o2));
-          float den = 0.f;
-#pragma unroll
-          for (int k = 0; k < 2; ++k) {
-            const float wk = lv[k] > 0.f ? exp2f(mv[k] - M) : 0.f;
-            wgt[g * RAP_MAX_SPLIT + lane + 32 * k] = wk;
-            den += wk * lv[k];
+        } else {
+          float* wgt = red;        // [G][RAP_MAX_SPLIT] segment weights, then G reciprocals of the denominators
+          for (int g = warp; g < G; g += NW) {
+            const float* gb = ub + (size_t)g * ws_head;
+            float mv[2], lv[2];
+  #pragma unroll
+            for (int k = 0; k < 2; ++k) {
+              const int sg = lane + 32 * k;
+              lv[k] = sg < nseg ? __ldcg(gb + (size_t)sg * (DV + 2) + DV + 1) : 0.f;
+              mv[k] = (sg < nseg && lv[k] > 0.f) ? __ldcg(gb + (size_t)sg * (DV + 2) + DV) : -INFINITY;
+            }
+            float M = fmaxf(mv[0], mv[1]);
+  #pragma unroll
+            for (int o2 = 16; o2 > 0; o2 >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o2));
+            float den = 0.f;
+  #pragma unroll
+            for (int k = 0; k < 2; ++k) {
+              const float wk = lv[k] > 0.f ? exp2f(mv[k] - M) : 0.f;
+              wgt[g * RAP_MAX_SPLIT + lane + 32 * k] = wk;
+              den += wk * lv[k];
+            }
+  #pragma unroll
+            for (int o2 = 16; o2 > 0; o2 >>= 1) den += __shfl_xor_sync(0xffffffffu, den, o2);
+            if (lane == 0) wgt[G * RAP_MAX_SPLIT + g] = den > 0.f ? 1.f / den : 0.f;
           }
-#pragma unroll
-          for (int o2 = 16; o2 > 0; o2 >>= 1) den += __shfl_xor_sync(0xffffffffu, den, o2);
-          if (lane == 0) wgt[G * RAP_MAX_SPLIT + g] = den > 0.f ? 1.f / den : 0.f;
-        }
-        __syncthreads();
-        for (int i = tid; i < G * DV; i += THREADS) {
-          const int g = i / DV, c = i - g * DV;
-          const float* gb = ub + (size_t)g * ws_head + c;
-          float num = 0.f;
-          for (int sg = 0; sg < nseg; ++sg) num += wgt[g * RAP_MAX_SPLIT + sg] * __ldcg(gb + (size_t)sg * (DV + 2));
-          p.out[((size_t)b * p.Hq + (size_t)h * G + g) * DV + c] = num * wgt[G * RAP_MAX_SPLIT + g];
+          __syncthreads();
+          for (int i = tid; i < G * DV; i += THREADS) {
+            const int g = i / DV, c = i - g * DV;
+            const float* gb = ub + (size_t)g * ws_head + c;
+            float num = 0.f;
+            for (int sg = 0; sg < nseg; ++sg) num += wgt[g * RAP_MAX_SPLIT + sg] * __ldcg(gb + (size_t)sg * (DV + 2));
+            p.out[((size_t)b * p.Hq + (size_t)h * G + g) * DV + c] = num * wgt[G * RAP_MAX_SPLIT + g];
+          }
         }
         if (tid == 0) p.unit_cnt[u] = 0;   // ready for the next call on this context
       }
