@@ -100,3 +100,20 @@ def test_budget_alloc_matches_the_oracle(lib):
     bad = np.ones((2, 1, 8))
     assert lib.rap_budget_alloc(2, 1, 16, binding._ptr(bad), 0.0, binding._ptr(n), binding._ptr(n)) == binding.RAP_EINVAL
     assert lib.rap_budget_alloc(2, 1, 15, binding._ptr(bad), 0.5, binding._ptr(n), binding._ptr(n)) == binding.RAP_EINVAL
+
+
+def test_every_named_workload_has_both_shape_specialised_scans():
+    """The build instantiates the tensor-core scan (and the FP32-pipe scan behind it) for the head shape of every
+    bf16 workload the benchmark and the sweep name, so none of them can end up on a slower generic tier."""
+    from paper_2602_02599_b200 import build, synth
+    mma, fp32 = set(build.mma_shapes()), set(build.scan_shapes())
+    for name, w in synth.CONFIGS.items():
+        if w.dtype != "bf16":
+            continue
+        shape = (w.n_q_heads // w.n_kv_heads, w.n_pairs, w.n_vch)
+        assert shape in mma, (name, shape)
+        assert shape in fp32, (name, shape)
+    # layer-adaptive budgets (d_v' = 2P) of the shaped models all have the tensor-core form
+    for G in (3, 4, 5):
+        for P in range(16, 65):
+            assert (G, P, 2 * P) in mma
