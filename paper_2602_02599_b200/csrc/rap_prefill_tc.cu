@@ -26,11 +26,11 @@ namespace {
 
 constexpr int P2_KT = 64;                              // keys per tile
 constexpr int P2_THREADS = 448;
-constexpr int P2_STAGES = 4;                           // K buffers and V buffers
+constexpr int P2_STAGES = 5;                           // K buffers and V buffers
 constexpr int P2_Q_BYTES = 2 * 128 * 128;              // [128 queries][<=128 dims]: two 64-element atom columns
-constexpr int P2_P_BYTES = 128 * 128;                  // [128 queries][64 keys]
 constexpr int P2_KV_BYTES = 2 * P2_KT * 128;           // [64 keys][<=128 dims or channels]
-constexpr int P2_SMEM = 2 * P2_Q_BYTES + 2 * P2_P_BYTES + 2 * P2_STAGES * P2_KV_BYTES + 256;
+constexpr int P2_TAIL = 320;                           // mbarriers, TMEM address, give-up flag
+constexpr int P2_SMEM = 2 * P2_Q_BYTES + 2 * P2_STAGES * P2_KV_BYTES + P2_TAIL;
 constexpr uint32_t PT_WAIT_HINT_NS = 20000;      // a parked probe returns at the phase change or after this long
 constexpr uint32_t PT_WAIT_LIMIT = 1u << 15;    // probes before a wait gives up (well under a second)
 
@@ -60,6 +60,15 @@ __device__ __forceinline__ void pt_mma(uint32_t tmem_d, uint64_t adesc, uint64_t
       "setp.ne.b32 p, %4, 0;\n\t"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(tmem_d),
       "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc)
+      : "memory");
+}
+// the same with the A operand in tensor memory (row = lane, two bf16 K elements per 32-bit column)
+__device__ __forceinline__ void pt_mma_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}" ::"r"(tmem_d),
+      "r"(tmem_a), "l"(bdesc), "r"(idesc), "r"(acc)
       : "memory");
 }
 __device__ __forceinline__ void pt_commit(uint32_t bar) {
@@ -189,15 +198,15 @@ __global__ void __launch_bounds__(P2_THREADS, 1) prefill_tc_kernel(const PtParam
   extern __shared__ unsigned char pt_raw[];
   unsigned char* smem = pt_raw + ((1024u - (pt_smem(pt_raw) & 1023u)) & 1023u);
   unsigned char* q_s = smem;                                   // Q_A, Q_B
-  unsigned char* p_s = q_s + 2 * P2_Q_BYTES;                   // P_A, P_B
-  unsigned char* k_s = p_s + 2 * P2_P_BYTES;                   // ring of K tiles
+  unsigned char* k_s = q_s + 2 * P2_Q_BYTES;                   // ring of K tiles
   unsigned char* v_s = k_s + P2_STAGES * P2_KV_BYTES;          // ring of V tiles (N-major)
   unsigned char* tail = v_s + P2_STAGES * P2_KV_BYTES;
-  const uint32_t bar_fk = pt_smem(tail), bar_ek = bar_fk + 32, bar_fv = bar_fk + 64, bar_ev = bar_fk + 96,
-                 bar_s = bar_fk + 128 /* [X][2] */, bar_p = bar_fk + 160 /* [X] */, bar_o = bar_fk + 176 /* [X] */,
-                 bar_end = bar_fk + 192;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 208);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 212);
+  const uint32_t bar_fk = pt_smem(tail), bar_ek = bar_fk + 8 * P2_STAGES, bar_fv = bar_ek + 8 * P2_STAGES,
+                 bar_ev = bar_fv + 8 * P2_STAGES, bar_s = bar_ev + 8 * P2_STAGES /* [X][2] */, bar_p = bar_s + 32 /* [X][2] */,
+                 bar_o = bar_p + 32 /* [X] */, bar_end = bar_o + 16 /* [X] */;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 32 * P2_STAGES + 96);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 32 * P2_STAGES + 100);
+  static_assert(32 * P2_STAGES + 104 <= P2_TAIL, "barriers and flags fit the tail");
 
   const int qb = blockIdx.x, g = blockIdx.y, b = blockIdx.z;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -223,11 +232,13 @@ __global__ void __launch_bounds__(P2_THREADS, 1) prefill_tc_kernel(const PtParam
       pt_mbar_init(bar_fv + 8 * i, 64);
       pt_mbar_init(bar_ev + 8 * i, 2);
     }
-    for (int i = 0; i < 4; ++i) pt_mbar_init(bar_s + 8 * i, 1);
-    for (int X = 0; X < 2; ++X) {
-      pt_mbar_init(bar_p + 8 * X, 128);
-      pt_mbar_init(bar_o + 8 * X, 1);
+    for (int i = 0; i < 4; ++i) {
+      pt_mbar_init(bar_s + 8 * i, 1);
+      // "P written" has one barrier per S buffer: the softmax may be a tile ahead of the lane that waits for it, and
+      // with a single barrier two completed phases would look like none
+      pt_mbar_init(bar_p + 8 * i, 128);
     }
+    for (int X = 0; X < 2; ++X) pt_mbar_init(bar_o + 8 * X, 1);
     pt_mbar_init(bar_end, 1);
     pt_mbar_init(bar_end + 8, 1);
     *abort_flag = 0;
@@ -239,7 +250,7 @@ __global__ void __launch_bounds__(P2_THREADS, 1) prefill_tc_kernel(const PtParam
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   // zero every tile once (pad columns and pad channel rows are never written again), then stage Q_A and Q_B
-  for (int i = tid; i < (P2_SMEM - 256) / 16; i += P2_THREADS) reinterpret_cast<uint4*>(smem)[i] = make_uint4(0, 0, 0, 0);
+  for (int i = tid; i < (P2_SMEM - P2_TAIL) / 16; i += P2_THREADS) reinterpret_cast<uint4*>(smem)[i] = make_uint4(0, 0, 0, 0);
   __syncthreads();
   const int kw = p.P2 >> 1;                          // 4-byte words per q / K row
   for (int r = warp; r < 256; r += P2_THREADS / 32) {
@@ -337,7 +348,7 @@ __global__ void __launch_bounds__(P2_THREADS, 1) prefill_tc_kernel(const PtParam
     // arriving in step (after the buffer was filled), so the phases stay aligned.
     if (lane == 0) {
       const int Y = warp - 8, n_y = nt[Y];
-      const uint32_t qx = pt_smem(q_s + Y * P2_Q_BYTES), pa = pt_smem(p_s + Y * P2_P_BYTES);
+      const uint32_t qx = pt_smem(q_s + Y * P2_Q_BYTES);
       const uint32_t tmem_sy = tmem_base + 128u * (uint32_t)Y, tmem_oy = tmem_base + 256u + 128u * (uint32_t)Y;
       auto issue_s = [&](int tile) {
         const uint32_t kb = pt_smem(k_s + (tile % P2_STAGES) * P2_KV_BYTES);
@@ -371,14 +382,14 @@ __global__ void __launch_bounds__(P2_THREADS, 1) prefill_tc_kernel(const PtParam
         const int vbuf = tile % P2_STAGES;
         if (!wait(bar_fv + 8 * vbuf, (tile / P2_STAGES) & 1)) { ok = false; break; }
         if (tile < n_y) {
-          if (!wait(bar_p + 8 * Y, tile & 1)) { ok = false; break; }
+          if (!wait(bar_p + 8 * (2 * Y + (tile & 1)), (tile >> 1) & 1)) { ok = false; break; }
           asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
           const uint32_t vb = pt_smem(v_s + vbuf * P2_KV_BYTES);
 #pragma unroll
-          for (int ks = 0; ks < P2_KT / 16; ++ks)
-            pt_mma(tmem_oy, pt_desc(pa + (uint32_t)ks * 32u), pt_desc_n2(vb + (uint32_t)ks * 2048u), IDESC_O,
-                   (tile > 0 || ks > 0) ? 1u : 0u);
+          for (int ks = 0; ks < P2_KT / 16; ++ks)   // A = P in tensor memory, over the S columns it was computed from
+            pt_mma_ts(tmem_oy, tmem_sy + 64u * (uint32_t)(tile & 1) + 8u * (uint32_t)ks, pt_desc_n2(vb + (uint32_t)ks * 2048u),
+                      IDESC_O, (tile > 0 || ks > 0) ? 1u : 0u);
           pt_commit(bar_o + 8 * Y);
         }
         release(bar_ev + 8 * vbuf, tile < n_y);
@@ -465,10 +476,11 @@ __global__ void __launch_bounds__(P2_THREADS, 1) prefill_tc_kernel(const PtParam
         }
       }
       l_run += (ls[0] + ls[1]) + (ls[2] + ls[3]);
-      if (tile > 0) {
+      if (tile > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
+        // rare: rescale this warp's accumulator rows in tensor memory, once the previous tile's update is in
         if (!__all_sync(0xffffffffu, wait(bar_o + 8 * X, (tile - 1) & 1))) { rows_ok = false; break; }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        if (__any_sync(0xffffffffu, alpha != 1.f)) {   // rare: rescale this warp's accumulator rows in tensor memory
+        {
 #pragma unroll 1
           for (int c0 = 0; c0 < NVP; c0 += 32) {
             uint32_t oc[32];
@@ -480,13 +492,12 @@ __global__ void __launch_bounds__(P2_THREADS, 1) prefill_tc_kernel(const PtParam
           asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
         }
       }
-      unsigned char* pd = p_s + X * P2_P_BYTES;
-#pragma unroll
-      for (int ch = 0; ch < 8; ++ch)
-        *reinterpret_cast<uint4*>(pd + pt_off(row, 8 * ch, 128)) = make_uint4(r[4 * ch], r[4 * ch + 1], r[4 * ch + 2], r[4 * ch + 3]);
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      // P (64 bf16 = 32 packed columns) goes back into tensor memory over the first half of the S columns it came
+      // from: it is the A operand of the second MMA, and the next S into this buffer is issued after that MMA
+      pt_st32(trow, *reinterpret_cast<uint32_t(*)[32]>(r));
+      asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-      asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar_p + 8 * X) : "memory");
+      asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar_p + 8 * (2 * X + (tile & 1))) : "memory");
     }
     if (rows_ok && n_my > 0) __all_sync(0xffffffffu, wait(bar_o + 8 * X, (n_my - 1) & 1));
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");

@@ -521,6 +521,13 @@ def _prefill_case(name, T, starts, q_gain=1.0, ramp=0.0):
     st.close()
 
 
+def test_prefill_attn_many_key_tiles_odd_value_width():
+    """A block long enough for the key-tile pipeline to reach its steady state (18 key tiles per query tile), on the
+    shape whose V rows have an odd width: their staging is the slowest producer, so the softmax groups run ahead
+    of the MMA-issuing lanes as far as the barriers let them."""
+    _prefill_case("3b", 1100, [0])
+
+
 @pytest.mark.parametrize("q_gain,ramp", [(10.0, 0.0), (3.0, 0.004)])
 def test_prefill_attn_peaked_and_moving_maximum(q_gain, ramp):
     """Nearly one-hot weights, and a maximum that rises along the keys so that the kernels keep rescaling their
