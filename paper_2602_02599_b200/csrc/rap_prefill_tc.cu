@@ -6,13 +6,14 @@
 //                       double buffered per query tile: S of key tile t + 1 is issued before P of t is waited for
 //   P_X    = 2^(S - m)  softmax warp group X (warps 0-3: A, 4-7: B), one thread per query row: the S row in
 //                       registers with one TMEM round trip, causal mask only on the tiles that reach the diagonal,
-//                       lazy running maximum, P as bf16 into shared memory
-//   O_X   += P_X V      tcgen05.mma (N = d_v' rounded up to 32, K = 64 keys) accumulating in TMEM across the key
-//                       tiles; a warp rescales its 32 accumulator rows (tcgen05.ld / st) only in the rare tile
-//                       where the lazy maximum moved.
+//                       lazy running maximum, P as packed bf16 back into tensor memory over the S columns it
+//                       came from
+//   O_X   += P_X V      tcgen05.mma with A = P in tensor memory (N = d_v' rounded up to 32, K = 64 keys),
+//                       accumulating in TMEM across the key tiles; a warp rescales its 32 accumulator rows
+//                       (tcgen05.ld / st) only in the rare tile where the lazy maximum moved.
 // While one group runs its softmax the tensor core works for the other, and a staged K / V tile serves 256 queries.
 // Cache rows are not multiples of 16 bytes, so TMA tensor maps cannot describe them: four producer warps (10-11: K,
-// 12-13: V) stage the tiles by hand (4-byte cp.async) into rings of four buffers each, in the 128-byte-swizzled
+// 12-13: V) stage the tiles by hand (4-byte cp.async) into rings of five buffers each, in the 128-byte-swizzled
 // layouts the MMA descriptors expect (K as stored = K-major; V as stored = the N-major form of the B operand, so
 // nothing is transposed); rows past the sequence end and pad columns are zeros.  The copies' completion arrives on
 // the buffer's mbarrier by itself; the consumer issues the proxy fence.  The roles meet only on mbarriers; every wait
