@@ -209,7 +209,8 @@ __global__ void __launch_bounds__(P2_THREADS, 1) prefill_tc_kernel(const PtParam
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 32 * P2_STAGES + 100);
   static_assert(32 * P2_STAGES + 104 <= P2_TAIL, "barriers and flags fit the tail");
 
-  const int qb = blockIdx.x, g = blockIdx.y, b = blockIdx.z;
+  // the blocks with the most key tiles (the last queries) are dispatched first, the short ones fill the tail
+  const int qb = (int)gridDim.z - 1 - (int)blockIdx.z, g = blockIdx.x, b = blockIdx.y;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int h = g / (p.Hq / p.Hkv);
   const int start = min(max(p.start[b], 0), p.S_cap - p.T);
@@ -508,7 +509,7 @@ __global__ void __launch_bounds__(P2_THREADS, 1) prefill_tc_kernel(const PtParam
   const bool timed_out = *abort_flag != 0;
   if (timed_out && tid == 0) {
     atomicCAS(&p.status[0], 0, (int)RAP_ETIMEOUT);
-    p.status[1] = 0x60000000 | (blockIdx.x & 0xffffff);
+    p.status[1] = 0x60000000 | (qb & 0xffffff);
   }
   if (warp < 8 && !timed_out && nt[X] > 0) {
     const int t = q0 + 128 * X + row;
@@ -537,7 +538,7 @@ template <int DK, int NVP>
 rap_status launch_pt(rap_ctx* ctx, const PtParams& p, int B, cudaStream_t st) {
   const int smem = P2_SMEM + 1024;
   RAP_CUDA_TRY(ctx, rap_raise_smem(ctx, prefill_tc_kernel<DK, NVP>, smem));
-  dim3 grid((p.T + 255) / 256, p.Hq, B);
+  dim3 grid(p.Hq, B, (p.T + 255) / 256);
   prefill_tc_kernel<DK, NVP><<<grid, P2_THREADS, smem, st>>>(p);
   ctx->launches++;
   RAP_CUDA_TRY(ctx, cudaGetLastError());
