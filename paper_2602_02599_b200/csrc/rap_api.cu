@@ -32,6 +32,7 @@ void free_all(rap_ctx* c) {
   if (c->d_stage_out) cudaFree(c->d_stage_out);
   if (c->d_stage_q) cudaFree(c->d_stage_q);
   if (c->d_oproj_x) cudaFree(c->d_oproj_x);
+  if (c->d_pf_v) cudaFree(c->d_pf_v);
   if (c->d_lr_k) cudaFree(c->d_lr_k);
   if (c->d_lr_cs) cudaFree(c->d_lr_cs);
   if (c->h_tables) cudaFreeHost(c->h_tables);

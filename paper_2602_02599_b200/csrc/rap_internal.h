@@ -33,6 +33,8 @@ struct rap_ctx {
   float* d_stage_out = nullptr;
   void* d_stage_q = nullptr;
   void* d_oproj_x = nullptr;      // rap_out_proj: attention output rounded to the storage dtype
+  void* d_pf_v = nullptr;         // prefill attention, odd d_v': V rows copied to an even row length (grown on demand)
+  size_t pf_v_bytes = 0;
   void* d_lr_k = nullptr;         // low-rank comparator: rebuilt, rotated full-width K (grown on demand)
   size_t lr_k_bytes = 0;
   void* d_lr_cs = nullptr;        // low-rank comparator: (cos, sin) table [positions][D/2]

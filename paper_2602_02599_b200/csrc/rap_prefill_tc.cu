@@ -141,47 +141,6 @@ __device__ __forceinline__ uint32_t pt_swz2(int e, int r7) {
   const int w = e >> 2;
   return (uint32_t)(((w >> 5) << 13) + ((((w & 31) >> 2) ^ r7) << 4) + ((w & 3) << 2));
 }
-// Rows of an odd length (odd d_v'), for the warp that takes the row pairs (4k + 2 pw, 4k + 2 pw + 1) of a 64-row tile.
-// The even row of a pair starts on a word: 4-byte copies, the last word half filled.  The odd row starts 2 bytes off
-// a word: channel pair (2w, 2w+1) is the high half of one aligned word and the low half of the next (two loads, a
-// byte permute, a store); eight rows are loaded before the first store so that the loads overlap.
-__device__ __forceinline__ void pt_stage_odd_len(uint32_t du, const unsigned char* tile_src, int rowlen, int rows_ok,
-                                                 int pw, int lane) {
-  const int wl = (rowlen - 1) >> 1;                    // last word of a row: one channel
-  const int RB = 2 * rowlen;
-  for (int k0 = 0; k0 < P2_KT / 4; k0 += 8) {
-    uint32_t va[8][2], vb[8][2];
-#pragma unroll
-    for (int k = 0; k < 8; ++k) {
-      const int r = 4 * (k0 + k) + 2 * pw + 1;         // odd row
-      const bool ok = r < rows_ok;
-      const uint32_t* g = reinterpret_cast<const uint32_t*>(tile_src + (size_t)r * RB - 2);
-#pragma unroll
-      for (int sl = 0; sl < 2; ++sl) {
-        const int w = lane + 32 * sl;
-        va[k][sl] = (ok && w <= wl) ? g[w] : 0u;
-        vb[k][sl] = (ok && w < wl) ? g[w + 1] : 0u;
-      }
-    }
-#pragma unroll
-    for (int k = 0; k < 8; ++k) {
-      const int re = 4 * (k0 + k) + 2 * pw, r = re + 1;
-      const bool oke = re < rows_ok;
-      const unsigned char* se = tile_src + (size_t)(oke ? re : 0) * RB;
-#pragma unroll
-      for (int sl = 0; sl < 2; ++sl) {
-        const int w = lane + 32 * sl;
-        if (w <= wl) {
-          pt_cp4(du + (uint32_t)re * 128u + pt_swz2(4 * w, re & 7), se + 4 * w, oke ? (w == wl ? 2 : 4) : 0);
-          uint32_t val;
-          asm("prmt.b32 %0, %1, %2, 0x5432;" : "=r"(val) : "r"(va[k][sl]), "r"(vb[k][sl]));
-          asm volatile("st.shared.u32 [%0], %1;" ::"r"(du + (uint32_t)r * 128u + pt_swz2(4 * w, r & 7)), "r"(val) : "memory");
-        }
-      }
-    }
-  }
-}
-
 struct PtParams {
   const __nv_bfloat16* q;     // [B][T][Hq][P2]
   const __nv_bfloat16* k;     // [B][Hkv][S_cap][P2]
@@ -190,8 +149,25 @@ struct PtParams {
   float* out;                 // [B][T][Hq][dv]
   int32_t* status;
   int T, Hq, Hkv, P2, dv, S_cap;
+  int vs;                     // elements between V rows: d_v', or d_v' + 1 when the rows were copied to an even length
   float qscale;               // log2(e) / sqrt(D)
 };
+
+// Odd d_v': V rows are only 2-byte aligned, which rules out the 4-byte asynchronous copies of the staging.  The rows
+// the block can see (start + T per sequence) are first copied to rows of d_v' + 1 elements (the last one zero): a
+// few MB against the GB the attention itself moves through the SMs.
+__global__ void __launch_bounds__(256) prefill_repack_v_kernel(const __nv_bfloat16* __restrict__ v, __nv_bfloat16* __restrict__ dst,
+                                                               const int32_t* __restrict__ start, int T, int Hkv, int dv,
+                                                               int S_cap) {
+  const int unit = blockIdx.y, b = unit / Hkv;
+  const int n = min(max(start[b], 0), S_cap - T) + T;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  for (int row = blockIdx.x * 8 + warp; row < n; row += gridDim.x * 8) {
+    const __nv_bfloat16* src = v + ((size_t)unit * S_cap + row) * dv;
+    __nv_bfloat16* d = dst + ((size_t)unit * S_cap + row) * (dv + 1);
+    for (int c = lane; c <= dv; c += 32) d[c] = c < dv ? src[c] : __float2bfloat16(0.f);
+  }
+}
 
 // DK = k-steps of Q K^T (ceil(2P / 16)); NVP = d_v' rounded up to a multiple of 32 (N of the second MMA)
 template <int DK, int NVP>
@@ -225,7 +201,7 @@ __global__ void __launch_bounds__(P2_THREADS, 1) prefill_tc_kernel(const PtParam
   }
   const int n_max = max(nt[0], nt[1]);
   const __nv_bfloat16* kg = p.k + ((size_t)b * p.Hkv + h) * (size_t)p.S_cap * p.P2;
-  const __nv_bfloat16* vg = p.v + ((size_t)b * p.Hkv + h) * (size_t)p.S_cap * p.dv;
+  const __nv_bfloat16* vg = p.v + ((size_t)b * p.Hkv + h) * (size_t)p.S_cap * p.vs;
 
   if (tid == 0) {
     for (int i = 0; i < P2_STAGES; ++i) {
@@ -289,17 +265,16 @@ __global__ void __launch_bounds__(P2_THREADS, 1) prefill_tc_kernel(const PtParam
     // ================= producers: warps 10-11 stage K, warps 12-13 stage V, in order, tiles of 64 rows =================
     const bool is_v = warp >= 12;
     const int pw = (warp - 10) & 1;
-    const int rowlen = is_v ? p.dv : p.P2;
+    const int rowlen = is_v ? p.vs : p.P2;            // even in both cases
     const unsigned char* src0 = reinterpret_cast<const unsigned char*>(is_v ? vg : kg);
     unsigned char* ring = is_v ? v_s : k_s;
     const uint32_t bar_f = is_v ? bar_fv : bar_fk, bar_e = is_v ? bar_ev : bar_ek;
-    const bool odd_len = (rowlen & 1) != 0;
     uint32_t swz[4][2];
-    int nb[2];
+    int nb[2];                                        // this lane's words of a row: 4 bytes each, or none
 #pragma unroll
     for (int sl = 0; sl < 2; ++sl) {
       const int w = lane + 32 * sl;
-      nb[sl] = min(4, max(0, 2 * rowlen - 4 * w));
+      nb[sl] = 2 * rowlen - 4 * w >= 4 ? 4 : 0;
 #pragma unroll
       for (int c = 0; c < 4; ++c) swz[c][sl] = pt_swz2(4 * w, (pw + 2 * c) & 7);
     }
@@ -310,37 +285,31 @@ __global__ void __launch_bounds__(P2_THREADS, 1) prefill_tc_kernel(const PtParam
       const uint32_t du = pt_smem(ring + stg * P2_KV_BYTES);
       const int rows_ok = min(P2_KT, n_valid - j0);
       const unsigned char* tsrc = src0 + (size_t)j0 * (size_t)(2 * rowlen);
-      if (odd_len) {
-        pt_stage_odd_len(du, tsrc, rowlen, rows_ok, pw, lane);
-        asm volatile("cp.async.commit_group;" ::: "memory");
-        asm volatile("cp.async.wait_group 0;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar_f + 8 * stg) : "memory");
-      } else {
-        if (rows_ok == P2_KT && nb[0] == 4 && (nb[1] == 4 || nb[1] == 0)) {
-          const unsigned char* sp = tsrc + (size_t)pw * (size_t)(2 * rowlen) + 4 * lane;
-          uint32_t db = du + (uint32_t)pw * 128u;
-          const bool two = nb[1] > 0;
+      if (rows_ok == P2_KT) {
+        // a full tile (all but the last one of a sequence): no predicates, running pointers
+        const unsigned char* sp = tsrc + (size_t)pw * (size_t)(2 * rowlen) + 4 * lane;
+        uint32_t db = du + (uint32_t)pw * 128u;
+        const bool one = nb[0] > 0, two = nb[1] > 0;
 #pragma unroll 4
-          for (int i = 0; i < P2_KT / 2; ++i) {
-            pt_cp4(db + swz[i & 3][0], sp, 4);
-            if (two) pt_cp4(db + swz[i & 3][1], sp + 128, 4);
-            sp += 4 * rowlen;
-            db += 256;
-          }
-        } else {
-#pragma unroll 4
-          for (int i = 0; i < P2_KT / 2; ++i) {
-            const int r = pw + 2 * i;
-            const bool ok = r < rows_ok;
-            const uint32_t* src = reinterpret_cast<const uint32_t*>(tsrc + (size_t)(ok ? r : 0) * (size_t)(2 * rowlen));
-            const uint32_t rb = du + (uint32_t)r * 128u;
-            if (nb[0] > 0) pt_cp4(rb + swz[i & 3][0], src + lane, ok ? nb[0] : 0);
-            if (nb[1] > 0) pt_cp4(rb + swz[i & 3][1], src + lane + 32, ok ? nb[1] : 0);
-          }
+        for (int i = 0; i < P2_KT / 2; ++i) {
+          if (one) pt_cp4(db + swz[i & 3][0], sp, 4);
+          if (two) pt_cp4(db + swz[i & 3][1], sp + 128, 4);
+          sp += 4 * rowlen;                            // two rows on
+          db += 256;
         }
-        asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar_f + 8 * stg) : "memory");
+      } else {
+#pragma unroll 4
+        for (int i = 0; i < P2_KT / 2; ++i) {
+          const int r = pw + 2 * i;
+          const bool ok = r < rows_ok;                 // rows past the end: zero fill, nothing is read
+          const uint32_t* src = reinterpret_cast<const uint32_t*>(tsrc + (size_t)(ok ? r : 0) * (size_t)(2 * rowlen));
+          const uint32_t rb = du + (uint32_t)r * 128u;
+          if (nb[0] > 0) pt_cp4(rb + swz[i & 3][0], src + lane, ok ? 4 : 0);
+          if (nb[1] > 0) pt_cp4(rb + swz[i & 3][1], src + lane + 32, ok ? 4 : 0);
+        }
       }
+      // the arrival is triggered by the completion of this thread's copies: go on to the next tile
+      asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar_f + 8 * stg) : "memory");
       if (++stg == P2_STAGES) { stg = 0; ++use; }
     }
   } else if (warp >= 8) {
@@ -555,8 +524,26 @@ rap_status rap_launch_prefill_attn_tc(rap_ctx* ctx, int B, int T, const void* q,
   PtParams p;
   p.q = (const __nv_bfloat16*)q; p.k = (const __nv_bfloat16*)k; p.v = (const __nv_bfloat16*)v; p.start = start; p.out = out;
   p.status = ctx->d_status;
-  p.T = T; p.Hq = d.n_q_heads; p.Hkv = d.n_kv_heads; p.P2 = P2; p.dv = dv; p.S_cap = S_cap;
+  p.T = T; p.Hq = d.n_q_heads; p.Hkv = d.n_kv_heads; p.P2 = P2; p.dv = dv; p.S_cap = S_cap; p.vs = dv;
   p.qscale = (float)(1.4426950408889634 / sqrt((double)d.head_dim));
+  if (dv & 1) {
+    // rows of an odd length: copy what the block can see to rows of d_v' + 1 elements (workspace grown on demand;
+    // the growth allocates, so the first call at a new size is not for a stream capture)
+    const size_t need = (size_t)B * d.n_kv_heads * (size_t)S_cap * (size_t)(dv + 1) * sizeof(__nv_bfloat16);
+    if (need > ctx->pf_v_bytes) {
+      RAP_CUDA_TRY(ctx, cudaStreamSynchronize(st));
+      if (ctx->d_pf_v) cudaFree(ctx->d_pf_v);
+      ctx->d_pf_v = nullptr; ctx->pf_v_bytes = 0;
+      RAP_CUDA_TRY(ctx, cudaMalloc(&ctx->d_pf_v, need));
+      ctx->pf_v_bytes = need;
+    }
+    dim3 grid(64, B * d.n_kv_heads);
+    prefill_repack_v_kernel<<<grid, 256, 0, st>>>(p.v, (__nv_bfloat16*)ctx->d_pf_v, start, T, d.n_kv_heads, dv, S_cap);
+    ctx->launches++;
+    RAP_CUDA_TRY(ctx, cudaGetLastError());
+    p.v = (const __nv_bfloat16*)ctx->d_pf_v;
+    p.vs = dv + 1;
+  }
   const int dk = (P2 + 15) / 16, nvp = (dv + 31) / 32 * 32;
   if (dk <= 4 && nvp <= 64) return launch_pt<4, 64>(ctx, p, B, st);
   if (dk <= 6 && nvp <= 96) return launch_pt<6, 96>(ctx, p, B, st);
