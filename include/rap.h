@@ -213,7 +213,10 @@ rap_status rap_decode_attn_noalloc(int32_t dtype, int32_t B, int32_t n_q_heads, 
  * d_q [B][T][H_q][2P] and whose K / V rows are already in the caches (written by rap_qkv_rope_append) at
  * rows d_start[b] .. d_start[b] + T - 1; token i attends rows 0 .. d_start[b] + i.
  * d_out [B][T][H_q][d_v'] fp32.  h_start_max: caller's bound on d_start (RAP_ECAPACITY if
- * h_start_max + T > S_cap).  Tensor-core kernel, bf16 storage only (RAP_EUNSUPPORTED for fp32 stacks). */
+ * h_start_max + T > S_cap).  Tensor-core kernel, bf16 storage only (RAP_EUNSUPPORTED for fp32 stacks).
+ * For a layer with an odd d_v' the call first copies the visible V rows to an even row length in a
+ * context-owned workspace of B * H_kv * S_cap * (d_v' + 1) elements; the workspace is allocated (and the
+ * stream synchronized) the first time a call needs that much, so make that call outside a stream capture. */
 rap_status rap_prefill_attn(rap_ctx* ctx, int32_t layer, int32_t B, int32_t T, const void* d_q, const void* d_k_cache,
                             const void* d_v_cache, int32_t S_cap, const int32_t* d_start, int32_t h_start_max,
                             float* d_out, void* stream);
