@@ -521,6 +521,13 @@ def _prefill_case(name, T, starts, q_gain=1.0, ramp=0.0):
     st.close()
 
 
+@pytest.mark.parametrize("T,starts", [(1, [0, 300]), (257, [63, 0]), (129, [1, 64])])
+def test_prefill_attn_block_edges(T, starts):
+    """Blocks of one token, of one token more than two query tiles, and of one more than a tile; starts on and
+    next to key-tile boundaries."""
+    _prefill_case("8b", T, starts)
+
+
 def test_prefill_attn_many_key_tiles_odd_value_width():
     """A block long enough for the key-tile pipeline to reach its steady state (18 key tiles per query tile), on the
     shape whose V rows have an odd width: their staging is the slowest producer, so the softmax groups run ahead
