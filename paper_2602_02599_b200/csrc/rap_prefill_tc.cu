@@ -547,5 +547,6 @@ rap_status rap_launch_prefill_attn_tc(rap_ctx* ctx, int B, int T, const void* q,
   const int dk = (P2 + 15) / 16, nvp = (dv + 31) / 32 * 32;
   if (dk <= 4 && nvp <= 64) return launch_pt<4, 64>(ctx, p, B, st);
   if (dk <= 6 && nvp <= 96) return launch_pt<6, 96>(ctx, p, B, st);
+  if (dk <= 7) return launch_pt<7, 128>(ctx, p, B, st);
   return launch_pt<8, 128>(ctx, p, B, st);
 }
