@@ -83,7 +83,7 @@ const char* rap_last_cuda_error(const rap_ctx* ctx);
 rap_status rap_retained_counts(double rho, int32_t head_dim, int32_t* n_pairs, int32_t* n_vch);
 
 /* Budget-Alloc (Algorithm 2): layer-adaptive pair budgets m_l proportional to the layer score
- * sigma_l = mean over heads and pairs of h_k_pair_scores [L][H_kv][D/2] (HOST fp64, non-negative), with
+ * sigma_l = mean over heads and pairs of h_k_pair_scores [L][H_kv][D/2] (HOST fp64, finite, non-negative), with
  * mean retain ratio rho; head-uniform inside a layer; V keeps 2 m_l channels (Balanced K/V).  The paper
  * does not fix the rounding: the integer total is round(rho * D/2 * L), layers whose proportional share
  * leaves [1, D/2] are pinned to the bound and the rest re-shared, shares are floored and the missing
@@ -113,6 +113,18 @@ rap_status rap_build_tables(rap_ctx* ctx, const double* h_k_pair_scores, const d
                             const int32_t* h_n_pairs, const int32_t* h_n_vch,
                             int32_t* d_k_pair_idx, int32_t* d_k_dim_idx, int32_t* d_v_idx,
                             double* d_inv_freq, void* stream);
+
+/* Tables of a model whose RoPE does not use theta^(-2i/D): frequency-scaled variants (Section 4, "Practical
+ * Considerations", "RoPE variants": they change the frequencies or their scaling but keep the 2x2 rotation
+ * blocks, so the pair selection applies unchanged).  h_pair_freq [L][D/2] HOST fp64 (finite) is the model's own
+ * frequency, in radians per position, of ORIGINAL pair i of layer l; retained pair c of (l, h) gets
+ * d_inv_freq[l][h][c] = h_pair_freq[l][i_c] -- index-aware, as in rap_build_tables -- and the online path is the
+ * same.  A variant that also rescales the rotated vectors by a constant (an attention temperature) folds that
+ * constant into the rows of W~_q offline; it needs no table.  Everything else as rap_build_tables. */
+rap_status rap_build_tables_freq(rap_ctx* ctx, const double* h_k_pair_scores, const double* h_v_chan_scores,
+                                 const double* h_pair_freq, const int32_t* h_n_pairs, const int32_t* h_n_vch,
+                                 int32_t* d_k_pair_idx, int32_t* d_k_dim_idx, int32_t* d_v_idx, double* d_inv_freq,
+                                 void* stream);
 
 /* Tables of a hybrid model (Section 4, "Hybrid compression"): RAP on the layers that use RoPE, plain
  * channel pruning of K on the layers that do not (h_rope_layer[l] == 0).  For such a layer K keeps the
@@ -192,16 +204,18 @@ rap_status rap_decode_attn(rap_ctx* ctx, int32_t layer, int32_t B, const void* d
  *   d_q [B][H_q][2P], d_k_cache [B][H_kv][S_cap][2P], d_v_cache [B][H_kv][S_cap][d_v'],
  *   d_seq_len[b] valid rows (as in rap_decode_attn), d_out [B][H_q][d_v'] fp32.
  * Scratch: the split-KV partials go to a 4 MiB array that is part of the library image
- * (RAP_NOALLOC_WS_FLOATS = 2^20 floats); every GPU that loads the library holds those 4 MiB
+ * (RAP_NOALLOC_WS_FLOATS floats, defined below); every GPU that loads the library holds those 4 MiB
  * until the process exits.  A call needs B * H_q * n_split * (d_v' + 2) floats: with
  * n_split = 0 the library picks a split count that fits; RAP_ESHAPE if the requested n_split
- * does not fit, or if even one split does not (B * H_q * (d_v' + 2) > 2^20).
+ * does not fit, if even one split does not (B * H_q * (d_v' + 2) > RAP_NOALLOC_WS_FLOATS), or if B or H_kv
+ * exceeds 65535 (they index the launch grid).
  * The first call on each device looks up the array's device address (with that device
  * current); make that first call outside any stream capture.
  * All calls on a device share the one array and it keeps the previous call's contents.  The
  * kernels write every partial they later read, so nothing needs clearing, but two calls whose
  * kernels overlap on the GPU (different streams, or a graph with parallel branches) race on
  * it: serialize them.  Always uses the shape-generic kernel (any 2P, d_v' <= 256, G <= 8). */
+#define RAP_NOALLOC_WS_FLOATS (1u << 20)
 rap_status rap_decode_attn_noalloc(int32_t dtype, int32_t B, int32_t n_q_heads, int32_t n_kv_heads,
                                    int32_t head_dim, int32_t n_pairs, int32_t n_vch, const void* d_q,
                                    const void* d_k_cache, const void* d_v_cache, int32_t S_cap,
@@ -216,7 +230,9 @@ rap_status rap_decode_attn_noalloc(int32_t dtype, int32_t B, int32_t n_q_heads, 
  * h_start_max + T > S_cap).  Tensor-core kernel, bf16 storage only (RAP_EUNSUPPORTED for fp32 stacks).
  * For a layer with an odd d_v' the call first copies the visible V rows to an even row length in a
  * context-owned workspace of B * H_kv * S_cap * (d_v' + 1) elements; the workspace is allocated (and the
- * stream synchronized) the first time a call needs that much, so make that call outside a stream capture. */
+ * stream synchronized) the first time a call needs that much, so make that call outside a stream capture.
+ * Calls on one context must not overlap on the GPU (the workspace is shared, and growing it frees the old one
+ * after synchronizing only the calling stream). */
 rap_status rap_prefill_attn(rap_ctx* ctx, int32_t layer, int32_t B, int32_t T, const void* d_q, const void* d_k_cache,
                             const void* d_v_cache, int32_t S_cap, const int32_t* d_start, int32_t h_start_max,
                             float* d_out, void* stream);
@@ -273,24 +289,6 @@ rap_status rap_lowrank_decode_attn(rap_ctx* ctx, int32_t B, int32_t r, int32_t d
  * rap_status (RAP_OK, RAP_ECAPACITY for a skipped out-of-range row, RAP_ETIMEOUT for a bounded
  * wait that gave up); detail identifies the row / stage. */
 rap_status rap_get_last_device_status(rap_ctx* ctx, int32_t* code, int32_t* detail, void* stream);
-
-/* Number of kernels this context has launched since creation (for launch accounting). */
-int64_t rap_kernel_launch_count(const rap_ctx* ctx);
-
-/* Timing of the attention launches inside rap_decode_step / rap_decode_step_host, for roofline
- * reports: after rap_profile_attn(ctx, capacity) the next `capacity` attention launches (one per layer
- * and step) are bracketed by CUDA events on the caller's stream; rap_profile_attn_read waits for them,
- * returns the summed device time in milliseconds and the number of launches covered, and rearms the
- * same events.  capacity = 0 switches the timing off.  Event creation happens in rap_profile_attn. */
-rap_status rap_profile_attn(rap_ctx* ctx, int32_t capacity);
-rap_status rap_profile_attn_read(rap_ctx* ctx, float* ms_sum, int32_t* n_calls);
-
-/* Forces a kernel variant for rap_decode_attn: 0 = automatic (the shape-specialised scans when the
- * head shape has one, the tensor-core form first; the low-rank comparator's fast path), 1 = fully generic
- * kernels only, 2 = skip the shape-specialised scans, 3 = skip only the tensor-core form of the
- * shape-specialised scan, 4 = the tensor-core form or nothing (bf16 calls return RAP_EUNSUPPORTED when the
- * head shape has no instantiation of it).  Meant for tests and profiling. */
-rap_status rap_set_attn_variant(rap_ctx* ctx, int32_t variant);
 
 #ifdef __cplusplus
 }

@@ -1,0 +1,38 @@
+/*
+ * rap_debug.h -- test, accounting and profiling hooks of the RAP decode library.
+ *
+ * These entry points are exported by the same shared library as rap.h but are not part of the
+ * product interface: they count launches, time the attention launches of a decode step and force
+ * a kernel tier so that tests and profiles can reach every one of them.  Same conventions as rap.h.
+ */
+#ifndef RAP_DEBUG_H_
+#define RAP_DEBUG_H_
+
+#include "rap.h"
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Number of kernels this context has launched since creation (for launch accounting). */
+int64_t rap_kernel_launch_count(const rap_ctx* ctx);
+
+/* Timing of the attention launches inside rap_decode_step / rap_decode_step_host, for roofline
+ * reports: after rap_profile_attn(ctx, capacity) the next `capacity` attention launches (one per layer
+ * and step) are bracketed by CUDA events on the caller's stream; rap_profile_attn_read waits for them,
+ * returns the summed device time in milliseconds and the number of launches covered, and rearms the
+ * same events.  capacity = 0 switches the timing off.  Event creation happens in rap_profile_attn. */
+rap_status rap_profile_attn(rap_ctx* ctx, int32_t capacity);
+rap_status rap_profile_attn_read(rap_ctx* ctx, float* ms_sum, int32_t* n_calls);
+
+/* Forces a kernel variant for rap_decode_attn: 0 = automatic (the shape-specialised scans when the
+ * head shape has one, the tensor-core form first; the low-rank comparator's fast path), 1 = fully generic
+ * kernels only, 2 = skip the shape-specialised scans, 3 = skip only the tensor-core form of the
+ * shape-specialised scan, 4 = the tensor-core form or nothing (bf16 calls return RAP_EUNSUPPORTED when the
+ * head shape has no instantiation of it).  Meant for tests and profiling. */
+rap_status rap_set_attn_variant(rap_ctx* ctx, int32_t variant);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RAP_DEBUG_H_ */

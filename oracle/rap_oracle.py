@@ -22,7 +22,7 @@ loop-written column gather.
 Pins (in tests/test_oracle_pins.py): rho=1 equals an independent textbook RoPE GQA
 attention; (R)==(F) for rho<1 in both pairings; the per-pair relative-rotation
 identity R_m^T R_n = R_(n-m); position-shift invariance; E_k E_k^T = I and
-E_k R_t = R_(t,S) E_k; the retained-fraction column of Table 13; the bytes/token row
+E_k R_t = R_(t,S) E_k (also for a frequency table that is not theta^(-2i/D)); the retained-fraction column of Table 13; the bytes/token row
 of Table 15; brute-force loops on tiny inputs; closed-form softmax cases.
 
 Parity unpinned: the paper prints no worked numeric example of an attention output, so
@@ -209,6 +209,27 @@ def build_tables(k_pair_scores, v_chan_scores, n_pairs, n_vch, head_dim, rope_th
             for c in range(P):
                 inv_freq[l, h, c] = float(rope_theta) ** (-2.0 * float(pairs[c]) / float(D))
     return dict(k_pair_idx=k_pair_idx, k_dim_idx=k_dim_idx, v_idx=v_idx, inv_freq=inv_freq)
+
+
+def build_tables_freq(k_pair_scores, v_chan_scores, pair_freq, n_pairs, n_vch, head_dim, pairing):
+    """Tables of a model whose RoPE has its own per-pair frequencies (Section 4, "Practical Considerations":
+    frequency-scaled variants keep the 2x2 rotation blocks, so the pair selection applies unchanged).
+
+    pair_freq [L][D/2] is the frequency (radians per position) of ORIGINAL pair i in layer l.  Reading: the
+    selection is build_tables's; the retained pair c of (l, h) rotates at the frequency of its original pair,
+    inv_freq[l, h, c] = pair_freq[l, i_c]  (index-aware, exactly as for the standard table).  A constant
+    rescaling of the rotated vectors, which some variants add, is linear and belongs to W~_q; it is not part
+    of the tables."""
+    pf = np.asarray(pair_freq, dtype=np.float64)
+    tabs = build_tables(k_pair_scores, v_chan_scores, n_pairs, n_vch, head_dim, 2.0, pairing)
+    L, H, half = tabs["k_pair_idx"].shape
+    assert pf.shape == (L, half)
+    tabs["inv_freq"][:] = 0.0
+    for l in range(L):
+        for h in range(H):
+            for c in range(int(n_pairs[l])):
+                tabs["inv_freq"][l, h, c] = pf[l, int(tabs["k_pair_idx"][l, h, c])]
+    return tabs
 
 
 def selection_matrix(index, width):

@@ -26,7 +26,7 @@ EXPORTS = [
     "rap_get_last_device_status", "rap_kernel_launch_count", "rap_set_attn_variant",
     "rap_decode_attn_noalloc", "rap_profile_attn", "rap_profile_attn_read",
     "rap_pack_wo", "rap_out_proj", "rap_budget_alloc", "rap_prefill_attn", "rap_build_tables_hybrid",
-    "rap_build_tables_partial",
+    "rap_build_tables_partial", "rap_build_tables_freq",
 ]
 
 
@@ -68,6 +68,7 @@ def _lib():
     lib.rap_cache_elem_offset.argtypes = [c_int32] * 7
     lib.rap_cache_elem_offset.restype = c_size_t
     lib.rap_build_tables.argtypes = [P] * 10
+    lib.rap_build_tables_freq.argtypes = [P] * 11
     lib.rap_build_tables_hybrid.argtypes = [P] * 12
     lib.rap_build_tables_partial.argtypes = [P] * 13
     lib.rap_pack_weights.argtypes = [P, c_int32] + [P] * 11
@@ -141,7 +142,17 @@ def rap_cache_elem_offset(n_kv_heads, S_cap, W, b, h, pos, c):
     return _lib().rap_cache_elem_offset(n_kv_heads, S_cap, W, b, h, pos, c)
 
 
-NOALLOC_WS_FLOATS = 1 << 20
+def _noalloc_ws_floats():
+    """RAP_NOALLOC_WS_FLOATS as include/rap.h defines it (the one place the limit is written down)."""
+    import re
+    text = open(os.path.join(os.path.dirname(_HERE), "include", "rap.h")).read()
+    m = re.search(r"#define\s+RAP_NOALLOC_WS_FLOATS\s+\(1u\s*<<\s*(\d+)\)", text)
+    if not m:
+        raise RuntimeError("include/rap.h does not define RAP_NOALLOC_WS_FLOATS as (1u << n)")
+    return 1 << int(m.group(1))
+
+
+NOALLOC_WS_FLOATS = _noalloc_ws_floats()
 
 
 def rap_decode_attn_noalloc(dtype, B, n_q_heads, n_kv_heads, head_dim, n_pairs, n_vch, d_q, d_k_cache, d_v_cache,
@@ -198,6 +209,14 @@ class RapContext:
         self._check(_lib().rap_build_tables(self._ctx, _ptr(ks), _ptr(vs), _ptr(npairs), _ptr(nvch),
                                             _ptr(d_k_pair_idx), _ptr(d_k_dim_idx), _ptr(d_v_idx),
                                             _ptr(d_inv_freq), _stream()), "rap_build_tables")
+
+    def rap_build_tables_freq(self, k_pair_scores, v_chan_scores, pair_freq, n_pairs, n_vch, d_k_pair_idx, d_k_dim_idx,
+                              d_v_idx, d_inv_freq):
+        arrs = [np.ascontiguousarray(a, dtype=np.float64) for a in (k_pair_scores, v_chan_scores, pair_freq)]
+        ints = [np.ascontiguousarray(a, dtype=np.int32) for a in (n_pairs, n_vch)]
+        self._check(_lib().rap_build_tables_freq(self._ctx, _ptr(arrs[0]), _ptr(arrs[1]), _ptr(arrs[2]), _ptr(ints[0]),
+                                                 _ptr(ints[1]), _ptr(d_k_pair_idx), _ptr(d_k_dim_idx), _ptr(d_v_idx),
+                                                 _ptr(d_inv_freq), _stream()), "rap_build_tables_freq")
 
     def rap_build_tables_hybrid(self, k_pair_scores, k_chan_scores, v_chan_scores, rope_layer, n_pairs, n_vch,
                                 d_k_pair_idx, d_k_dim_idx, d_v_idx, d_inv_freq):

@@ -92,7 +92,7 @@ rap_status rap_budget_alloc(int32_t n_layers, int32_t n_kv_heads, int32_t head_d
     double s = 0.0;
     for (size_t i = 0; i < per_layer; ++i) {
       const double v = k_pair_scores[(size_t)l * per_layer + i];
-      if (std::isnan(v) || v < 0.0) return RAP_EINVAL;
+      if (!std::isfinite(v) || v < 0.0) return RAP_EINVAL;
       s += v;
     }
     sigma[l] = s / (double)per_layer;
@@ -209,8 +209,9 @@ rap_status rap_destroy(rap_ctx* ctx) {
 // frequency theta^(-2i/R)) and Pr of the P kept pair slots hold rotated pairs; the other slots hold 2 (P - Pr)
 // channels of the unrotated dims R..D-1 with frequency zero.  rap_build_tables: R = D, Pr = P everywhere;
 // the hybrid form: R = 0, Pr = 0 on layers without RoPE; the partial form: R and Pr per layer from the caller.
+// pair_freq (NULL, or [L][D/2]): the model's own frequency of every original pair, used instead of theta^(-2i/D).
 static rap_status build_tables_impl(rap_ctx* ctx, const double* ks, const double* kc, const double* vs,
-                                    const int32_t* rope_layer, const int32_t* rot_dims, const int32_t* n_rot_pairs,
+                                    const double* pair_freq, const int32_t* rope_layer, const int32_t* rot_dims, const int32_t* n_rot_pairs,
                                     const int32_t* n_pairs, const int32_t* n_vch,
                                     int32_t* d_k_pair_idx, int32_t* d_k_dim_idx, int32_t* d_v_idx, double* d_inv_freq,
                                     void* stream) {
@@ -235,6 +236,7 @@ static rap_status build_tables_impl(rap_ctx* ctx, const double* ks, const double
   for (size_t i = 0; i < units * half; ++i) if (std::isnan(ks[i])) return RAP_EINVAL;
   for (size_t i = 0; i < units * D; ++i) if (std::isnan(vs[i])) return RAP_EINVAL;
   if (kc) for (size_t i = 0; i < units * D; ++i) if (std::isnan(kc[i])) return RAP_EINVAL;
+  if (pair_freq) for (size_t i = 0; i < (size_t)L * half; ++i) if (!std::isfinite(pair_freq[i])) return RAP_EINVAL;
   cudaStream_t st = (cudaStream_t)stream;
   if (ctx->tables_inflight) {
     RAP_CUDA_TRY(ctx, cudaStreamSynchronize((cudaStream_t)ctx->tables_stream));
@@ -274,7 +276,7 @@ static rap_status build_tables_impl(rap_ctx* ctx, const double* ks, const double
           h_dim[u * D + 2 * c] = 2 * i;
           h_dim[u * D + 2 * c + 1] = 2 * i + 1;
         }
-        h_freq[u * half + c] = std::pow(d.rope_theta, -2.0 * (double)i / (double)R);
+        h_freq[u * half + c] = pair_freq ? pair_freq[(size_t)l * half + i] : std::pow(d.rope_theta, -2.0 * (double)i / (double)R);
       }
       if (P > Pr) {
         // unrotated dims: plain channel pruning; their slots keep frequency zero (identity rotation)
@@ -302,8 +304,16 @@ static rap_status build_tables_impl(rap_ctx* ctx, const double* ks, const double
 rap_status rap_build_tables(rap_ctx* ctx, const double* ks, const double* vs, const int32_t* n_pairs,
                             const int32_t* n_vch, int32_t* d_k_pair_idx, int32_t* d_k_dim_idx,
                             int32_t* d_v_idx, double* d_inv_freq, void* stream) {
-  return build_tables_impl(ctx, ks, nullptr, vs, nullptr, nullptr, nullptr, n_pairs, n_vch, d_k_pair_idx, d_k_dim_idx, d_v_idx, d_inv_freq,
-                           stream);
+  return build_tables_impl(ctx, ks, nullptr, vs, nullptr, nullptr, nullptr, nullptr, n_pairs, n_vch, d_k_pair_idx, d_k_dim_idx, d_v_idx,
+                           d_inv_freq, stream);
+}
+
+rap_status rap_build_tables_freq(rap_ctx* ctx, const double* ks, const double* vs, const double* pair_freq,
+                                 const int32_t* n_pairs, const int32_t* n_vch, int32_t* d_k_pair_idx,
+                                 int32_t* d_k_dim_idx, int32_t* d_v_idx, double* d_inv_freq, void* stream) {
+  if (!pair_freq) return RAP_EINVAL;
+  return build_tables_impl(ctx, ks, nullptr, vs, pair_freq, nullptr, nullptr, nullptr, n_pairs, n_vch, d_k_pair_idx, d_k_dim_idx,
+                           d_v_idx, d_inv_freq, stream);
 }
 
 rap_status rap_build_tables_hybrid(rap_ctx* ctx, const double* ks, const double* kc, const double* vs,
@@ -311,7 +321,7 @@ rap_status rap_build_tables_hybrid(rap_ctx* ctx, const double* ks, const double*
                                    int32_t* d_k_pair_idx, int32_t* d_k_dim_idx, int32_t* d_v_idx, double* d_inv_freq,
                                    void* stream) {
   if (!kc || !rope_layer) return RAP_EINVAL;
-  return build_tables_impl(ctx, ks, kc, vs, rope_layer, nullptr, nullptr, n_pairs, n_vch, d_k_pair_idx, d_k_dim_idx,
+  return build_tables_impl(ctx, ks, kc, vs, nullptr, rope_layer, nullptr, nullptr, n_pairs, n_vch, d_k_pair_idx, d_k_dim_idx,
                            d_v_idx, d_inv_freq, stream);
 }
 
@@ -320,7 +330,7 @@ rap_status rap_build_tables_partial(rap_ctx* ctx, const double* ks, const double
                                     const int32_t* n_vch, int32_t* d_k_pair_idx, int32_t* d_k_dim_idx,
                                     int32_t* d_v_idx, double* d_inv_freq, void* stream) {
   if (!kc || !rot_dims || !n_rot_pairs) return RAP_EINVAL;
-  return build_tables_impl(ctx, ks, kc, vs, nullptr, rot_dims, n_rot_pairs, n_pairs, n_vch, d_k_pair_idx, d_k_dim_idx,
+  return build_tables_impl(ctx, ks, kc, vs, nullptr, nullptr, rot_dims, n_rot_pairs, n_pairs, n_vch, d_k_pair_idx, d_k_dim_idx,
                            d_v_idx, d_inv_freq, stream);
 }
 

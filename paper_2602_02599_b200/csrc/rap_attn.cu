@@ -190,6 +190,7 @@ rap_status rap_launch_attn(rap_ctx* ctx, const rap_attn_args& a, cudaStream_t st
     const rap_status s = rap_launch_attn_fast(ctx, a, a.n_split, st);
     if (s != RAP_EUNSUPPORTED) return s;
   }
+  if (a.B > 65535 || a.Hkv > 65535) return RAP_ESHAPE;   // grid.z / grid.y of the generic scan
   const int n_split = a.n_split > 0 ? a.n_split : choose_split(ctx, a, GEN_TILE, 4, 4);
   const float qscale = (float)(1.4426950408889634 / sqrt((double)a.head_dim));
   const size_t smem = (size_t)(G * a.P2 + G * GEN_TILE + G) * sizeof(float);
@@ -212,8 +213,8 @@ rap_status rap_launch_attn(rap_ctx* ctx, const rap_attn_args& a, cudaStream_t st
 
 // ---- allocation-free variant ---------------------------------------------------------------
 // Split-KV partials of rap_decode_attn_noalloc live in this file-scope array instead of a
-// context workspace.  Every GPU that loads the library reserves it until the process exits.
-#define RAP_NOALLOC_WS_FLOATS (1u << 20)   // 4 MiB
+// context workspace (RAP_NOALLOC_WS_FLOATS floats = 4 MiB, the limit rap.h documents).  Every GPU that loads
+// the library reserves it until the process exits.
 static __device__ __align__(256) float g_noalloc_ws[RAP_NOALLOC_WS_FLOATS];
 
 namespace {
@@ -253,6 +254,7 @@ extern "C" rap_status rap_decode_attn_noalloc(int32_t dtype, int32_t B, int32_t 
     return RAP_EINVAL;
   const int G = n_q_heads / n_kv_heads;
   if (G > RAP_MAX_GROUP || n_split > RAP_MAX_SPLIT) return RAP_ESHAPE;
+  if (B > 65535 || n_kv_heads > 65535) return RAP_ESHAPE;   // grid.z / grid.y of the scan
   if (S_cap % 8) return RAP_EALIGN;
   if (h_seq_len_max > S_cap) return RAP_ECAPACITY;
   if (!rap_aligned16(d_q) || !rap_aligned16(d_k_cache) || !rap_aligned16(d_v_cache) || !rap_aligned16(d_out) ||

@@ -10,6 +10,7 @@
 #include <vector>
 
 #include "rap.h"
+#include "rap_debug.h"
 
 #define RAP_MAX_SPLIT 64     // upper bound on sequence splits of the attention scan
 #define RAP_MAX_GROUP 8      // largest G = H_q / H_kv

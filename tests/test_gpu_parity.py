@@ -257,7 +257,34 @@ def test_attention_tensor_core_scan_head_shapes(G, P, dv):
     _random_attn_case(w, [3010, 3010, 3010, 3010], 0, seed=G, variant=4)
 
 
-@pytest.mark.parametrize("variant", [4, 3])
+@pytest.mark.parametrize("G,P,dv", [(2, 37, 70), (4, 45, 90), (3, 58, 115), (5, 64, 128), (1, 8, 16), (4, 30, 61),
+                                    (5, 32, 64)])
+@pytest.mark.parametrize("n_split", [0, 5])
+def test_attention_run_time_shape_scan(G, P, dv, n_split):
+    """The bf16 scan that takes the head shape at run time -- the tier a shape without any instantiation falls to
+    (G = 2, P = 37, d_v' = 70 has none), forced here for instantiated shapes too (variant 2 skips both
+    shape-specialised scans): odd, 2 mod 4 and 0 mod 4 pair counts, rows that are multiples of 32 bytes (padded
+    in shared memory), odd and even d_v', ragged lengths, a one-row sequence and an empty one."""
+    from dataclasses import replace
+    base = synth.scaled_down(synth.LLAMA_8B, n_layers=1, batch=4, seq=3000)
+    w = replace(base, n_pairs=P, n_vch=dv, n_q_heads=G * base.n_kv_heads)
+    _random_attn_case(w, [3000, 1777, 1, 33], n_split, seed=P + G, variant=2)
+    _random_attn_case(w, [129, 0, 2999, 96], n_split, seed=P, variant=2)
+
+
+def test_attention_shape_without_instantiation_takes_the_default_path():
+    """No forced tier: a head shape nobody instantiated still goes through rap_decode_attn and meets the oracle,
+    and the tensor-core-or-nothing variant refuses it."""
+    from dataclasses import replace
+    base = synth.scaled_down(synth.LLAMA_8B, n_layers=1, batch=3, seq=2000)
+    w = replace(base, n_pairs=37, n_vch=70, n_q_heads=2 * base.n_kv_heads)
+    _random_attn_case(w, [2000, 1, 777], 0, seed=3)
+    with pytest.raises(binding.RapError) as e:
+        _random_attn_case(w, [2000, 1, 777], 0, seed=3, variant=4)
+    assert e.value.status == binding.RAP_EUNSUPPORTED
+
+
+@pytest.mark.parametrize("variant", [4, 3, 2])
 @pytest.mark.parametrize("q_gain,ramp", [(12.0, 0.0), (3.0, 0.002), (0.05, 0.0)])
 def test_attention_peaked_moving_and_flat_softmax(variant, q_gain, ramp):
     """Logit regimes that exercise the lazy reference maximum of both shape-specialised scans: nearly one-hot
@@ -609,4 +636,57 @@ def test_partial_rotary_tables_end_to_end():
         with pytest.raises(binding.RapError) as e:
             st.ctx.rap_build_tables_partial(ks, kc, vs, bad_rot, bad_n, *args)
         assert e.value.status == 1
+    st.close()
+
+
+def test_frequency_scaled_tables_end_to_end():
+    """rap_build_tables_freq: the model's own per-pair frequency table (every pair of the standard table slowed
+    down by its own factor, different per layer) instead of theta^(-2i/D).  Index tables and the gathered
+    frequencies equal the oracle's exactly; one decode step through the unchanged online path (appended K rows and
+    the attention output against the oracle); then a block of new tokens through rap_prefill_attn on the caches that
+    the scaled rotation wrote.  The frequencies are far from the standard ones, so a path that ignored the table
+    would miss the appended rows by much more than the tolerance."""
+    w = synth.scaled_down(synth.LLAMA_8B, n_layers=2, batch=2, seq=200, hidden=256)
+    ks, vs = synth.draw_scores(w)
+    D, half, L = w.head_dim, w.head_dim // 2, w.n_layers
+    base = w.rope_theta ** (-2.0 * np.arange(half) / D)
+    rng = np.random.default_rng(31)
+    freq = np.stack([base / np.linspace(1.0, 16.0, half), base * rng.uniform(0.2, 1.0, half)])
+    st = DecodeStack(w, max_rows=256)
+    st.ctx.rap_build_tables_freq(ks, vs, freq, st.n_pairs, st.n_vch, st.k_pair_idx, st.k_dim_idx, st.v_idx, st.inv_freq)
+    tabs = O.build_tables_freq(ks, vs, freq, st.n_pairs, st.n_vch, D, w.pairing)
+    torch.cuda.synchronize()
+    for key, dev in (("k_pair_idx", st.k_pair_idx), ("k_dim_idx", st.k_dim_idx), ("v_idx", st.v_idx), ("inv_freq", st.inv_freq)):
+        assert np.array_equal(dev.cpu().numpy(), tabs[key]), key
+    std = util.oracle_tables(w, ks, vs)
+    assert np.abs(tabs["inv_freq"] - std["inv_freq"]).max() > 0.1
+    lens = [200, 77]
+    _decode_step_with_tables(st, tabs, w, lens)
+    # the standard table would have put the new K rows somewhere else entirely
+    l, P, dv = 1, w.n_pairs, w.n_vch
+    X = O.round_storage(synth.draw_hidden(w, l, 1, w.batch), w.dtype)
+    w_host = util.to_np64(st.w_qkv[l])
+    _, k_std, _ = O.qkv_rope(X, w_host, None, np.array(lens), std["inv_freq"][l], w.n_q_heads, w.n_kv_heads, P, dv)
+    Kd = util.to_np64(st.k_cache[l])
+    k_dev = np.stack([Kd[b, :, lens[b], :] for b in range(w.batch)])
+    assert np.abs(k_dev - k_std).max() > 0.1
+    # prefill-side attention over the same caches: 60 new tokens per sequence written through the scaled rotation
+    T = 60
+    rows = [(b, lens[b] + 1 + i) for b in range(w.batch) for i in range(T)]
+    sid = torch.tensor([r[0] for r in rows], dtype=torch.int32, device=st.device)
+    pos = torch.tensor([r[1] for r in rows], dtype=torch.int32, device=st.device)
+    xb = torch.from_numpy(synth.draw_hidden(w, l, 2, len(rows))).to(st.device).to(st.dt).contiguous()
+    q = torch.empty((len(rows), w.n_q_heads, 2 * P), dtype=st.dt, device=st.device)
+    st.qkv_rope_append(l, xb, sid, pos, pos, int(pos.max()), q_out=q)
+    start = torch.tensor([n + 1 for n in lens], dtype=torch.int32, device=st.device)
+    out = torch.full((w.batch, T, w.n_q_heads, dv), float("nan"), dtype=torch.float32, device=st.device)
+    st.ctx.rap_prefill_attn(l, w.batch, T, q, st.k_cache[l], st.v_cache[l], st.s_cap, start, max(lens) + 1, out)
+    torch.cuda.synchronize()
+    qo, ko, _ = O.qkv_rope(O.round_storage(util.to_np64(xb), w.dtype), w_host, None, pos.cpu().numpy(), tabs["inv_freq"][l],
+                           w.n_q_heads, w.n_kv_heads, P, dv)
+    util.check_projection(util.to_np64(q), O.round_storage(qo, w.dtype), w.dtype, "q of the block")
+    want = O.prefill_attn(util.to_np64(q).reshape(w.batch, T, w.n_q_heads, 2 * P), util.to_np64(st.k_cache[l]),
+                          util.to_np64(st.v_cache[l]), [n + 1 for n in lens], D)
+    util.check_attn(util.to_np64(out).reshape(w.batch * T, w.n_q_heads, dv), want.reshape(w.batch * T, w.n_q_heads, dv), w.dtype)
+    assert st.ctx.rap_get_last_device_status() == (0, 0)
     st.close()

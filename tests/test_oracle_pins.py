@@ -389,6 +389,20 @@ def test_budget_alloc_properties():
     assert np.array_equal(m, np.full(8, 48))
     m, _ = O.budget_alloc(np.ones((8, 2, 64)), 0.7, 128)
     assert m.sum() == 358 and set(m.tolist()) == {44, 45}
+    # the tie rule, worked by hand: total = round(0.7 * 64 * 8) = 358, every share is 358 / 8 = 44.75, the floors
+    # give 8 * 44 = 352, and the six missing pairs go to equal fractional parts in layer order: layers 0..5
+    assert m.tolist() == [45, 45, 45, 45, 45, 45, 44, 44]
+    # two layers with a larger fraction come first, then the tie among the others is broken by layer index:
+    # scores (1, 1, 1.1, 1, 1.1, 1), rho = 0.5, D = 16: total 24, shares 3.871 (x4) and 4.258 (x2), floors 3 / 4
+    # sum to 20, the four missing pairs go to fraction 0.871 in layer order -> layers 0, 1, 3, 5
+    sc = np.ones((6, 1, 8)) * np.array([1, 1, 1.1, 1, 1.1, 1])[:, None, None]
+    m, nv = O.budget_alloc(sc, 0.5, 16)
+    assert m.tolist() == [4, 4, 4, 4, 4, 4] and nv.tolist() == [8] * 6
+    sc = np.ones((6, 1, 8)) * np.array([1, 1, 1.3, 1, 1.3, 1])[:, None, None]
+    # shares 24 / 6.6 = 3.636 (x4) and 4.727 (x2): floors 3, 3, 4, 3, 4, 3 = 20; fractions 0.727 (layers 2, 4) beat
+    # 0.636, so they take two of the four missing pairs and the tie among the rest gives the other two to layers 0, 1
+    m, _ = O.budget_alloc(sc, 0.5, 16)
+    assert m.tolist() == [4, 4, 5, 3, 5, 3]
     # one dominant layer is capped at all pairs and the rest share what is left
     sc = np.ones((4, 1, 32)); sc[0] *= 100
     m, _ = O.budget_alloc(sc, 0.5, 64)
@@ -517,3 +531,68 @@ def test_partial_rotary_reduced_path_equals_full_width_attention(pairing):
             bad["inv_freq"][0, h, c] = m["theta"] ** (-2.0 * int(tabs["k_pair_idx"][0, h, c]) / D)
     got_bad, _, _, _ = O.reduced_attention_from_hidden(X, w, bad["inv_freq"][0], Hq, Hkv, P, dv, D)
     assert not np.allclose(got_bad, want, rtol=0, atol=1e-6)
+
+
+# ---- frequency-scaled RoPE variants (Section 4, "Practical Considerations") -----------------------
+def _full_width_rope_with_table(x, pos, freq, pairing):
+    """Full-width RoPE of one head vector with an arbitrary per-pair frequency table, written as D/2 explicit
+    2x2 rotations (no RAP object, no oracle call)."""
+    D = len(x)
+    y = np.array(x, dtype=np.float64)
+    for i in range(D // 2):
+        a, b = (i, i + D // 2) if pairing == O.PAIR_HALF else (2 * i, 2 * i + 1)
+        c, s = math.cos(pos * freq[i]), math.sin(pos * freq[i])
+        y[a], y[b] = x[a] * c - x[b] * s, x[a] * s + x[b] * c
+    return y
+
+
+@pytest.mark.parametrize("pairing", [O.PAIR_HALF, O.PAIR_ADJACENT])
+def test_scaled_frequency_tables_keep_the_pair_identities(pairing):
+    """A model table that is not theta^(-2i/D) (every pair slowed down by its own factor, as a context-extension
+    variant does): the selection is unchanged, E_k R_t = R_(t,S) E_k holds with the scaled full table, the reduced
+    attention equals full-width attention under that table with the removed pairs zeroed, and taking the table
+    by reduced position c instead of original pair i_c breaks it."""
+    m = _small(pairing=pairing, D=16, rho=0.6, n=9, seed=21, L=2)
+    D, P, dv, Hq, Hkv = m["D"], m["P"], m["dv"], m["Hq"], m["Hkv"]
+    rng = np.random.default_rng(8)
+    base = np.array([m["theta"] ** (-2.0 * i / D) for i in range(D // 2)])
+    freq = np.stack([base * rng.uniform(0.1, 1.0, D // 2), base / np.linspace(1.0, 8.0, D // 2)])   # [L][D/2]
+    tabs = O.build_tables_freq(m["ks"], m["vs"], freq, [P] * 2, [dv] * 2, D, pairing)
+    for key in ("k_pair_idx", "k_dim_idx", "v_idx"):
+        assert np.array_equal(tabs[key], m["tabs"][key])
+    # the standard table through the same call reproduces build_tables
+    std = O.build_tables_freq(m["ks"], m["vs"], np.stack([base, base]), [P] * 2, [dv] * 2, D, pairing)
+    assert np.allclose(std["inv_freq"], m["tabs"]["inv_freq"], rtol=1e-15, atol=0)
+    G = Hq // Hkv
+    for l in range(2):
+        for h in range(Hkv):
+            pairs = tabs["k_pair_idx"][l, h, :P]
+            assert np.array_equal(tabs["inv_freq"][l, h, :P], freq[l][pairs])
+            assert np.all(tabs["inv_freq"][l, h, P:] == 0.0)
+            E = O.selection_matrix(tabs["k_dim_idx"][l, h, :2 * P], D)
+            x = np.random.default_rng(10 * l + h).normal(size=D)
+            for t in (0, 3, 250, 4097):
+                lhs = E @ _full_width_rope_with_table(x, t, freq[l], pairing)
+                assert np.allclose(lhs, O.rope_reduced(E @ x, t, tabs["inv_freq"][l, h]), rtol=0, atol=1e-12)
+        # attention: reduced path with the gathered table == full width with the scaled table, removed pairs zeroed
+        w = O.gather_weights(m["Wq"], m["Wk"], m["Wv"], tabs, l, P, dv, D)
+        out, _, _, _ = O.reduced_attention_from_hidden(m["X"], w, tabs["inv_freq"][l], Hq, Hkv, P, dv, D)
+        n = m["X"].shape[0]
+        qf = (m["Wq"] @ m["X"][-1]).reshape(Hq, D)
+        kf = (m["X"] @ m["Wk"].T).reshape(n, Hkv, D)
+        vf = (m["X"] @ m["Wv"].T).reshape(n, Hkv, D)
+        ref = np.zeros((Hq, dv))
+        for g in range(Hq):
+            h = g // G
+            keep = np.zeros(D)
+            keep[tabs["k_dim_idx"][l, h, :2 * P]] = 1.0
+            qr = _full_width_rope_with_table(qf[g], n - 1, freq[l], pairing)
+            s = np.array([qr @ (_full_width_rope_with_table(kf[j, h], j, freq[l], pairing) * keep) for j in range(n)])
+            p = np.exp(s / math.sqrt(D) - (s / math.sqrt(D)).max())
+            ref[g] = (p / p.sum()) @ vf[:, h, :][:, tabs["v_idx"][l, h, :dv]]
+        assert np.allclose(out, ref, rtol=0, atol=1e-12)
+        # negative control: frequencies taken by reduced position instead of by original pair
+        wrong = np.zeros_like(tabs["inv_freq"][l])
+        wrong[:, :P] = freq[l][:P]
+        bad, _, _, _ = O.reduced_attention_from_hidden(m["X"], w, wrong, Hq, Hkv, P, dv, D)
+        assert np.abs(bad - ref).max() > 1e-4
