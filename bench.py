@@ -38,14 +38,19 @@ def load_peaks():
 
 
 def load_traffic(workload):
-    """DRAM bytes per attention-scan launch from the committed ncu summary, if it lists this workload."""
+    """(DRAM bytes per attention-scan launch, where the figure comes from) from the committed ncu summary, if it
+    lists this workload.  The counters are not taken in this run: the file holds one capture on a cut-down launch,
+    scaled to the full launch by the number of (sequence, KV head) units."""
     path = os.path.join(ROOT, "profiles", "attn_decode_traffic.txt")
     if os.path.exists(path):
+        source = "ncu capture on a cut-down launch, scaled by units (profiles/attn_decode_traffic.txt)"
         for line in open(path):
+            if line.startswith("# source:"):
+                source = line[len("# source:"):].strip()
             f = line.split()
             if len(f) == 2 and f[0] == workload:
-                return float(f[1])
-    return None
+                return float(f[1]), source
+    return None, None
 
 
 class ClockSampler(threading.Thread):
@@ -81,10 +86,11 @@ class ClockSampler(threading.Thread):
                 "reasons": reasons, "samples": len(sm)}
 
 
-def build_stack(w, torch, seed_offset=0):
-    """Allocate the stack, build tables, upload weights and fill the caches (synthetic, seeded)."""
+def build_stack(w, torch, seed_offset=0, new_rows=64):
+    """Allocate the stack (cache capacity: the workload's context plus room for new_rows decode steps), build
+    tables, upload weights and fill the caches (synthetic, seeded)."""
     from paper_2602_02599_b200.stack import DecodeStack
-    st = DecodeStack(w, max_rows=max(w.batch, 2048))
+    st = DecodeStack(w, max_rows=max(w.batch, 2048), s_cap=((w.seq + max(64, new_rows) + 7) // 8) * 8)
     ks, vs = synth.draw_scores(w)
     st.build_tables(ks, vs)
     st.fill_synthetic(w.seed + seed_offset, tail=T_PREFILL_TAIL)
@@ -120,6 +126,53 @@ def attn_bytes(w, length):
     return w.batch * w.n_kv_heads * length * (2 * w.n_pairs + w.n_vch) * w.elem_bytes
 
 
+def workload_string(w):
+    return (f"{w.name}: L={w.n_layers} hidden={w.hidden} Hq/Hkv={w.n_q_heads}/{w.n_kv_heads} D={w.head_dim} "
+            f"rho={w.rho} P={w.n_pairs} dv={w.n_vch} B={w.batch} S={w.seq}")
+
+
+def time_decode_steps(st, w, torch, K, W, first_len, x_all, barrier=None):
+    """W warm-up steps, then K timed steps of rap_decode_step (CUDA events on the launching stream, a
+    synchronize on both sides), with CUDA events around every rap_decode_attn launch of the timed steps.
+    Returns ms per step, ms per attention launch, ms per layer for the rest, and the launches counted."""
+    L = w.n_layers
+    barrier = barrier or torch.cuda.synchronize
+    st.seq_len.fill_(first_len)
+    for i in range(W):
+        st.decode_step(x_all[i % len(x_all)], first_len + i, advance=1)
+    barrier()
+    launches0 = st.ctx.rap_kernel_launch_count()
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    st.ctx.rap_profile_attn(K * L)
+    t0.record()
+    for i in range(K):
+        st.decode_step(x_all[(W + i) % len(x_all)], first_len + W + i, advance=1)
+    t1.record()
+    barrier()
+    launches = st.ctx.rap_kernel_launch_count() - launches0
+    ms_total = t0.elapsed_time(t1)
+    attn_sum, attn_calls = st.ctx.rap_profile_attn_read()
+    st.ctx.rap_profile_attn(0)
+    assert attn_calls == K * L, (attn_calls, K * L)
+    code, detail = st.ctx.rap_get_last_device_status()
+    assert code == 0, f"device status {code} detail {detail}"
+    mean_len = first_len + W + (K + 1) / 2.0
+    return {"ms_total": ms_total, "ms_step": ms_total / K, "attn_ms": attn_sum / attn_calls,
+            "rest_ms": (ms_total - attn_sum) / attn_calls, "launches": int(launches), "mean_len": mean_len}
+
+
+def summarize(w, r, peak):
+    """One workload's numbers in the shape the extra keys of the bench line use."""
+    alg = attn_bytes(w, r["mean_len"])
+    gbps = alg / (r["attn_ms"] * 1e-3) / 1e9
+    step_bytes = w.n_layers * (alg + w.hidden * w.n_out * w.elem_bytes)
+    return {"workload": workload_string(w), "tokens_per_s": w.batch / (r["ms_step"] * 1e-3), "ms_per_step": r["ms_step"],
+            "attn_ms_per_layer": r["attn_ms"], "rest_ms_per_layer": r["rest_ms"], "attn_gbps": gbps,
+            "frac": gbps / peak, "frac_of_nominal_8000": gbps / 8000.0,
+            "step_gbps": step_bytes / (r["ms_step"] * 1e-3) / 1e9,
+            "tokens_per_s_at_70pct_of_nominal": w.batch / (step_bytes / 5600e9)}
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -130,68 +183,49 @@ def run_ours(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
     w = pick_workload(args)
-    st = build_stack(w, torch, seed_offset=rank)
-    if args.attn_variant:
-        st.ctx.rap_set_attn_variant(args.attn_variant)
     L, B, K, W = w.n_layers, w.batch, args.steps, args.warmup
     n_steps = K + W
-    assert w.seq + 2 * n_steps + 2 < st.s_cap, "cache capacity too small for this many steps"
+    st = build_stack(w, torch, seed_offset=rank, new_rows=2 * n_steps + 16)
+    if args.attn_variant:
+        st.ctx.rap_set_attn_variant(args.attn_variant)
+    cut = bool(args.attn_variant or args.layers or args.batch or args.seq)
+    extras = args.extras and world == 1 and not cut and args.workload == "8b"
+    assert w.seq + 2 * n_steps + 8 < st.s_cap, "cache capacity too small for this many steps"
     dev = st.device
     # per-step inputs, resident in HBM before the timed region
     xg = torch.Generator(device=dev).manual_seed(w.seed + 17 + rank)
     x_all = torch.empty((n_steps, L, B, w.hidden), dtype=st.dt, device=dev).normal_(0.0, 1.0, generator=xg)
-    ev = lambda: torch.cuda.Event(enable_timing=True)
-    st.seq_len.fill_(w.seq)
-
-    def step(i):
-        # one C call per step: every layer's projection + RoPE + append, then the attention; the
-        # library advances seq_len on the device
-        st.decode_step(x_all[i], w.seq + i, advance=1)
 
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
-    for i in range(W):
-        step(i)
-    barrier()
     sampler = ClockSampler(local)
     sampler.start()
     time.sleep(0.3)
-    launches0 = st.ctx.rap_kernel_launch_count()
-    t0, t1 = ev(), ev()
-    barrier()
-    st.ctx.rap_profile_attn(K * L)      # CUDA events around every rap_decode_attn launch of the timed steps
-    t0.record()
-    for i in range(K):
-        step(W + i)
-    t1.record()
-    barrier()
-    launches = st.ctx.rap_kernel_launch_count() - launches0
+    # one C call per step: every layer's projection + RoPE + append, then the attention; the library
+    # advances seq_len on the device
+    r = time_decode_steps(st, w, torch, K, W, w.seq, x_all, barrier)
     clocks = sampler.stop()
-    ms_total = t0.elapsed_time(t1)
-    attn_sum, attn_calls = st.ctx.rap_profile_attn_read()
-    st.ctx.rap_profile_attn(0)
-    assert attn_calls == K * L, (attn_calls, K * L)
-    attn_ms = attn_sum / attn_calls
-    proj_ms = (ms_total - attn_sum) / attn_calls      # projection + RoPE + append + launch gaps, per layer
-    code, detail = st.ctx.rap_get_last_device_status()
-    assert code == 0, f"device status {code} detail {detail}"
+    ms_total, attn_ms, proj_ms, launches = r["ms_total"], r["attn_ms"], r["rest_ms"], r["launches"]
 
     # ---- end to end through the host-buffer entry point ------------------------------------
+    ev = lambda: torch.cuda.Event(enable_timing=True)
     hx = [torch.empty((L, B, w.hidden), dtype=st.dt).pin_memory() for _ in range(2)]
     for h in hx:
         h.copy_(x_all[0].cpu())
     h_out = torch.empty((L, st.out_stride), dtype=torch.float32).pin_memory()
-    e2e_steps = max(2, min(K, 5))
-    st.decode_step_host(hx[0], h_out, w.seq + n_steps, advance=1)       # warm-up
+    e2e_steps = K
+    e2e_warm = 3
+    for i in range(e2e_warm):
+        st.decode_step_host(hx[i & 1], h_out, w.seq + n_steps + i, advance=1)
     barrier()
     e0 = time.perf_counter()
     d0, d1 = ev(), ev()
     d0.record()
     for i in range(e2e_steps):
-        st.decode_step_host(hx[i & 1], h_out, w.seq + n_steps + 1 + i, advance=1)
+        st.decode_step_host(hx[i & 1], h_out, w.seq + n_steps + e2e_warm + i, advance=1)
     d1.record()
     barrier()
     e2e_ms = max(d0.elapsed_time(d1), (time.perf_counter() - e0) * 1e3) / e2e_steps
@@ -203,48 +237,97 @@ def run_ours(args):
         return
     ms_step = ms_total / K
     peak, peak_kind = load_peaks()
-    mean_len = w.seq + W + (K + 1) / 2.0
-    alg = attn_bytes(w, mean_len)
+    alg = attn_bytes(w, r["mean_len"])
     achieved = alg / (attn_ms * 1e-3) / 1e9
+    traffic, traffic_source = (None, None) if cut else load_traffic(args.workload)
     line = {
         "metric": METRIC, "value": aggregate_throughput(B, world, ms_step), "unit": UNIT, "n_gpus": world, "steps": K,
         "warmup": W, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16" if w.dtype == "bf16" else "f32", "data": "synthetic",
-        "config": {"workload": f"{w.name}: L={L} hidden={w.hidden} Hq/Hkv={w.n_q_heads}/{w.n_kv_heads} D={w.head_dim} "
-                               f"rho={w.rho} P={w.n_pairs} dv={w.n_vch} B={B} S={w.seq}",
+        "config": {"workload": workload_string(w),
                    "per_gpu_batch": B, "global_batch": world * B, "context": w.seq,
                    "l2": "inputs larger than L2 (%.1f GB of KV cache per step)" % (L * alg / 1e9),
                    "parallelism": "replicas" if world > 1 else "single"},
         "clocks": clocks, "gpu_launches": int(launches),
-        "e2e": {"value": aggregate_throughput(B, world, e2e_ms), "unit": UNIT,
+        "e2e": {"value": aggregate_throughput(B, world, e2e_ms), "unit": UNIT, "steps": e2e_steps, "warmup": e2e_warm,
                 "h2d_bytes_per_step": int(hx[0].numel() * hx[0].element_size()),
                 "d2h_bytes_per_step": int(h_out.numel() * 4)},
         "roofline": {"bound": "hbm", "kernel": "rap_decode_attn (attn_mma_kernel: split-KV scan with the merge of the splits fused in)"
                      if not args.attn_variant else "rap_decode_attn (forced tier %d)" % args.attn_variant,
                      "achieved": achieved,
-                     "peak": peak, "peak_source": peak_kind, "unit": "GB/s", "frac": achieved / peak,
+                     "peak": peak, "peak_source": peak_kind + " copy bandwidth (read + write); a read-only stream can exceed it",
+                     "unit": "GB/s", "frac": achieved / peak,
                      "frac_of_nominal_8000": achieved / 8000.0, "bytes_per_launch": alg, "ms_per_launch": attn_ms,
-                     "traffic": None if (args.attn_variant or args.layers or args.batch or args.seq)
-                     else load_traffic(args.workload)},
+                     "traffic": traffic, "traffic_source": traffic_source},
         "kernels": {"attn_ms_per_layer": attn_ms, "rest_ms_per_layer": proj_ms},
     }
+    if achieved > peak:
+        line["roofline"]["note"] = ("achieved exceeds the measured copy figure: that figure is a read+write copy, this kernel only "
+                                    "reads; judge it by frac_of_nominal_8000")
+    if extras:
+        # the scan on the plain FP32 pipes (no tensor-core instruction), same workload and protocol
+        st.ctx.rap_set_attn_variant(3)
+        k2 = min(K, 5)
+        r3 = time_decode_steps(st, w, torch, k2, 3, w.seq, x_all)      # rewrites the rows the first pass appended
+        st.ctx.rap_set_attn_variant(0)
+        line["fp32_pipe_scan"] = dict(summarize(w, r3, peak), steps=k2, warmup=3, kernel="attn_scan_kernel (forced tier 3)")
     if args.cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(w, st, torch)
+    if extras:
+        st.close()
+        del st, x_all
+        torch.cuda.empty_cache()
+        line["other_workloads"] = other_workloads(torch, min(K, 10), peak)
+        line["sweep"] = sweep_rows(torch, min(K, 10), 3, peak)
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
+
+
+def other_workloads(torch, K, peak):
+    """The 3B- and 14B-shaped workloads through the same protocol as the headline (whole decode steps)."""
+    rows = []
+    for name in ("3b", "14b"):
+        w = synth.CONFIGS[name]
+        st = build_stack(w, torch, new_rows=K + 8)
+        xg = torch.Generator(device=st.device).manual_seed(w.seed + 17)
+        x_all = torch.empty((K + 3, w.n_layers, w.batch, w.hidden), dtype=st.dt, device=st.device).normal_(0.0, 1.0, generator=xg)
+        r = time_decode_steps(st, w, torch, K, 3, w.seq, x_all)
+        rows.append(dict(summarize(w, r, peak), steps=K, warmup=3))
+        st.close()
+        del st, x_all
+        torch.cuda.empty_cache()
+    return rows
+
+
+class CoreMeter:
+    """Cores that actually worked inside the `with` blocks: process CPU time over wall time."""
+
+    def __init__(self):
+        self.cpu, self.wall = 0.0, 0.0
+
+    def __enter__(self):
+        t = os.times()
+        self._c, self._w = t.user + t.system, time.perf_counter()
+
+    def __exit__(self, *exc):
+        t = os.times()
+        self.cpu += t.user + t.system - self._c
+        self.wall += time.perf_counter() - self._w
+
+    def cores(self):
+        return max(1, int(round(self.cpu / self.wall))) if self.wall > 0 else 1
 
 
 def cpu_baseline(w, st, torch, budget_s=15.0):
     """The oracle, as it stands, on the host cores: full-length scans of sampled (layer, b, kv-head)
     units plus one layer's projection, extrapolated linearly to a whole step."""
     from oracle import rap_oracle as O
-    from threadpoolctl import threadpool_info
-    cores = max([i.get("num_threads", 1) for i in threadpool_info()] + [1])
     rng = np.random.default_rng(123)
     L, B, Hkv, Hq, G = w.n_layers, w.batch, w.n_kv_heads, w.n_q_heads, w.group
     n = w.seq + 1
     torch.cuda.synchronize()
+    busy = CoreMeter()
     times, t_start = [], time.perf_counter()
     while time.perf_counter() - t_start < budget_s and len(times) < 256:
         l, b, h = int(rng.integers(L)), int(rng.integers(B)), int(rng.integers(Hkv))
@@ -252,18 +335,21 @@ def cpu_baseline(w, st, torch, budget_s=15.0):
         V = st.v_cache[l][b, h, :n].to(torch.float64).cpu().numpy()[None, None]
         q = rng.standard_normal((1, G, K.shape[-1]))
         t = time.perf_counter()
-        O.decode_attn(q, K, V, [n], w.head_dim)
+        with busy:
+            O.decode_attn(q, K, V, [n], w.head_dim)
         times.append(time.perf_counter() - t)
     x = O.round_storage(synth.draw_hidden(w, 0, 0, B), w.dtype)
     wq = st.w_qkv[0].to(torch.float64).cpu().numpy()
     inv = st.inv_freq[0].cpu().numpy()
     t = time.perf_counter()
-    O.qkv_rope(x, wq, None, np.full(B, w.seq), inv, Hq, Hkv, w.n_pairs, w.n_vch)
+    with busy:
+        O.qkv_rope(x, wq, None, np.full(B, w.seq), inv, Hq, Hkv, w.n_pairs, w.n_vch)
     t_proj = time.perf_counter() - t
     t_step = float(np.mean(times)) * L * B * Hkv + L * t_proj
-    return {"value": B / t_step, "unit": UNIT, "cores": int(cores), "kind": "oracle",
+    return {"value": B / t_step, "unit": UNIT, "cores": busy.cores(), "cores_available": os.cpu_count(), "kind": "oracle",
             "sample": f"{len(times)} of {L * B * Hkv} (layer, sequence, kv-head) full-length scans + 1 of {L} layer "
-                      f"projections, extrapolated linearly to one step"}
+                      f"projections, one after the other (the NumPy routines decide how many threads work: `cores` is "
+                      f"process CPU time / wall time over the timed calls), extrapolated linearly to one step"}
 
 
 def run_reference(args):
@@ -272,12 +358,11 @@ def run_reference(args):
     if rank != 0:
         return
     from oracle import rap_oracle as O
-    from threadpoolctl import threadpool_info
     w = pick_workload(args)
-    cores = max([i.get("num_threads", 1) for i in threadpool_info()] + [1])
+    busy = CoreMeter()
     L, B, Hkv, Hq, G = w.n_layers, w.batch, w.n_kv_heads, w.n_q_heads, w.group
     n = w.seq + 1
-    units_per_step = 4
+    units_per_step = 8
     rng = np.random.default_rng(w.seed)
     sigma = float(np.sqrt(w.hidden) * 0.02)
     wq = O.round_storage(synth.draw_packed_weights(w, 0), w.dtype)
@@ -291,11 +376,13 @@ def run_reference(args):
             V = O.round_storage(synth.draw_cache_rows(w, 0, i, u, n, w.n_vch, 1), w.dtype)[None, None]
             q = O.round_storage(rng.standard_normal((1, G, 2 * w.n_pairs)) * sigma, w.dtype)
             t = time.perf_counter()
-            O.decode_attn(q, K, V, [n], w.head_dim)
+            with busy:
+                O.decode_attn(q, K, V, [n], w.head_dim)
             t_units += time.perf_counter() - t
         x = O.round_storage(synth.draw_hidden(w, 0, i, B), w.dtype)
         t = time.perf_counter()
-        O.qkv_rope(x, wq, None, np.full(B, w.seq), tabs["inv_freq"][0], Hq, Hkv, w.n_pairs, w.n_vch)
+        with busy:
+            O.qkv_rope(x, wq, None, np.full(B, w.seq), tabs["inv_freq"][0], Hq, Hkv, w.n_pairs, w.n_vch)
         t_proj = time.perf_counter() - t
         return t_units / units_per_step * L * B * Hkv + L * t_proj
 
@@ -305,26 +392,28 @@ def run_reference(args):
     t_step = float(np.mean(est))
     val = B / t_step
     sample = (f"per step: {units_per_step} of {L * B * Hkv} (layer, sequence, kv-head) full-length scans + 1 of {L} "
-              f"layer projections on synthetic rows, extrapolated linearly to the whole step")
+              f"layer projections on synthetic rows, one after the other (`cores` is process CPU time / wall time over "
+              f"the timed calls), extrapolated linearly to the whole step")
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": t_step * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": f"{w.name}: L={L} hidden={w.hidden} Hq/Hkv={Hq}/{Hkv} D={w.head_dim} rho={w.rho} "
                                f"P={w.n_pairs} dv={w.n_vch} B={B} S={w.seq}"},
-        "cpu_baseline": {"value": val, "unit": UNIT, "cores": int(cores), "kind": "oracle", "sample": sample},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": busy.cores(), "cores_available": os.cpu_count(), "kind": "oracle",
+                         "sample": sample},
         "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }), flush=True)
 
 
-def run_sweep(args):
+def sweep_rows(torch, steps, warmup, peak):
     """Retain-ratio sweep on the 8B shape (batch 16, 16384-token cache, two layers resident): time of
     rap_decode_attn per layer at each rho against the same kernel at rho = 1 (dense), and against the
-    low-rank comparator at equal cached dims (latent K of width 2P rebuilt and rotated every call)."""
-    import torch
+    low-rank comparator at equal cached dims (latent K of width 2P rebuilt and rotated every call).  Beside the
+    comparator's time stands its own bound: reading the latents and V and writing and re-reading the rebuilt
+    full-width K at the measured copy bandwidth."""
     from dataclasses import replace
     from paper_2602_02599_b200.stack import DecodeStack
-    torch.cuda.set_device(0)
     rows, dense_ms = [], None
     for rho in sorted(synth.SWEEP_COUNTS, reverse=True):
         w = replace(synth.sweep_workload(rho), n_layers=2)
@@ -343,16 +432,16 @@ def run_sweep(args):
         out = torch.empty((w.batch, w.n_q_heads, w.n_vch), dtype=torch.float32, device=st.device)
 
         def timed(fn):
-            for i in range(args.warmup):
+            for i in range(warmup):
                 fn(i & 1)
             torch.cuda.synchronize()
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record()
-            for i in range(args.steps):
+            for i in range(steps):
                 fn(i & 1)          # alternate the two layers: 2 x ~1 GB of cache, larger than L2
             e1.record()
             torch.cuda.synchronize()
-            return e0.elapsed_time(e1) / args.steps
+            return e0.elapsed_time(e1) / steps
 
         rap_ms = timed(lambda l: st.decode_attn(l, q, dl, n))
         low_ms = timed(lambda l: st.ctx.rap_lowrank_decode_attn(w.batch, 2 * w.n_pairs, w.n_vch, qf, st.k_cache[l], bk,
@@ -362,13 +451,26 @@ def run_sweep(args):
         if rho == 1.0:
             dense_ms = rap_ms
         by = attn_bytes(w, n)
+        units = w.batch * w.n_kv_heads * n * w.elem_bytes
+        low_bytes = units * (2 * w.n_pairs + 2 * w.head_dim + w.n_vch)
+        low_bound_ms = low_bytes / (peak * 1e9) * 1e3
         rows.append({"rho": rho, "P": w.n_pairs, "dv": w.n_vch, "kv_bytes_per_layer": by, "rap_attn_ms": rap_ms,
-                     "rap_GBps": by / rap_ms / 1e6, "rap_vs_dense": rap_ms / dense_ms,
+                     "rap_GBps": by / rap_ms / 1e6, "rap_frac": by / rap_ms / 1e6 / peak,
+                     "rap_frac_of_nominal_8000": by / rap_ms / 1e6 / 8000.0, "rap_vs_dense": rap_ms / dense_ms,
                      "bytes_vs_dense": (2 * w.n_pairs + w.n_vch) / 256.0, "lowrank_attn_ms": low_ms,
-                     "lowrank_vs_dense": low_ms / dense_ms})
+                     "lowrank_vs_dense": low_ms / dense_ms, "lowrank_bound_ms": low_bound_ms,
+                     "lowrank_bound_vs_dense": low_bound_ms / dense_ms, "lowrank_frac_of_its_bound": low_bound_ms / low_ms})
         st.close()
         del st, q, qf, bk, out
         torch.cuda.empty_cache()
+    return rows
+
+
+def run_sweep(args):
+    import torch
+    torch.cuda.set_device(0)
+    peak, _ = load_peaks()
+    rows = sweep_rows(torch, args.steps, args.warmup, peak)
     print(json.dumps({"metric": "attention_cost_ratio_vs_dense", "unit": "ratio", "n_gpus": 1, "steps": args.steps,
                       "warmup": args.warmup, "dtype": "bf16", "data": "synthetic", "higher_is_better": False,
                       "config": {"workload": "sweep on the 8B shape: 32q/8kv heads, D=128, B=16, S=16384, 2 layers resident"},
@@ -434,6 +536,17 @@ def run_prefill(args):
                       "prefill": rows}), flush=True)
 
 
+def replica_launch_command(n, argv):
+    """`bench.py --gpus N` started without a launcher: the command that starts N replica processes of this
+    script, one per GPU, on this node (rendezvous on 127.0.0.1 at a free port)."""
+    import socket
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    return [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+            "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + list(argv)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -450,7 +563,11 @@ def main():
     ap.add_argument("--prefill", action="store_true", help="time rap_prefill_attn on the sweep's head shapes")
     ap.add_argument("--prefill-case", default="", help="B:T[,B:T...] for --prefill")
     ap.add_argument("--sweep", action="store_true", help="retain-ratio sweep with the dense and low-rank comparators")
+    ap.add_argument("--no-extras", dest="extras", action="store_false",
+                    help="headline measurement only (skip the other workloads, the sweep and the FP32-pipe scan)")
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        sys.exit(subprocess.call(replica_launch_command(args.gpus, sys.argv[1:])))
     if args.warmup < 3 and args.impl == "ours":
         args.warmup = 3
     if int(os.environ.get("WORLD_SIZE", "1")) > 1:

@@ -43,3 +43,16 @@ def test_max_over_ranks_and_aggregate_on_two_gloo_ranks():
     # two replicas of batch 32 at 20 ms per step: 3200 tokens/s for the whole job
     assert abs(bench.aggregate_throughput(32, 2, 20.0) - 3200.0) < 1e-9
     assert bench.max_over_ranks([3.0], torch.device("cpu"), 1) == [3.0]
+
+
+def test_gpus_flag_without_a_launcher_starts_that_many_replicas():
+    """`bench.py --gpus N` run directly (no WORLD_SIZE in the environment) re-launches itself as N replica
+    processes on this node with a loopback rendezvous; the command is checked here, not run."""
+    sys.path.insert(0, ROOT)
+    import bench
+    cmd = bench.replica_launch_command(4, ["--gpus", "4", "--steps", "5"])
+    assert cmd[1:3] == ["-m", "torch.distributed.run"]
+    assert "--nproc-per-node=4" in cmd and "--nnodes=1" in cmd
+    assert cmd[cmd.index("--master-addr") + 1] == "127.0.0.1"
+    assert 0 < int(cmd[cmd.index("--master-port") + 1]) < 65536
+    assert cmd[-5] == os.path.join(ROOT, "bench.py") and cmd[-4:] == ["--gpus", "4", "--steps", "5"]
