@@ -32,6 +32,11 @@ rap_status rap_profile_attn_read(rap_ctx* ctx, float* ms_sum, int32_t* n_calls);
  * head shape has no instantiation of it).  Meant for tests and profiling. */
 rap_status rap_set_attn_variant(rap_ctx* ctx, int32_t variant);
 
+/* Forces the form of rap_qkv_rope_append: 0 = automatic (decode-sized bf16 calls, T <= 32, run as one kernel with
+ * the RoPE / append epilogue fused into the tcgen05 GEMM), 1 = always two stages (GEMM into the fp32 workspace, then
+ * the epilogue kernel).  Meant for tests, which check the two forms against each other and against the oracle. */
+rap_status rap_set_proj_variant(rap_ctx* ctx, int32_t variant);
+
 #ifdef __cplusplus
 }
 #endif

@@ -28,6 +28,7 @@ void free_all(rap_ctx* c) {
   if (c->d_attn_ws) cudaFree(c->d_attn_ws);
   if (c->d_unit_cnt) cudaFree(c->d_unit_cnt);
   if (c->d_proj_ws) cudaFree(c->d_proj_ws);
+  if (c->d_proj_cnt) cudaFree(c->d_proj_cnt);
   if (c->d_stage_x) cudaFree(c->d_stage_x);
   if (c->d_stage_out) cudaFree(c->d_stage_out);
   if (c->d_stage_q) cudaFree(c->d_stage_q);
@@ -65,6 +66,12 @@ int64_t rap_kernel_launch_count(const rap_ctx* ctx) { return ctx ? ctx->launches
 rap_status rap_set_attn_variant(rap_ctx* ctx, int32_t variant) {
   if (!ctx || variant < 0 || variant > 4) return RAP_EINVAL;
   ctx->attn_variant = variant;
+  return RAP_OK;
+}
+
+rap_status rap_set_proj_variant(rap_ctx* ctx, int32_t variant) {
+  if (!ctx || variant < 0 || variant > 1) return RAP_EINVAL;
+  ctx->proj_variant = variant;
   return RAP_OK;
 }
 
@@ -182,9 +189,12 @@ rap_status rap_create(const rap_model_desc* desc, rap_ctx** out) {
   RAP_CUDA_TRY(c, cudaMalloc(&c->d_status, 2 * sizeof(int32_t)));
   RAP_CUDA_TRY(c, cudaMemset(c->d_status, 0, 2 * sizeof(int32_t)));
   RAP_CUDA_TRY(c, cudaMalloc(&c->d_attn_ws, c->attn_ws_bytes));
-  RAP_CUDA_TRY(c, cudaMalloc(&c->d_unit_cnt, (size_t)d.max_batch * d.n_kv_heads * sizeof(int32_t)));
-  RAP_CUDA_TRY(c, cudaMemset(c->d_unit_cnt, 0, (size_t)d.max_batch * d.n_kv_heads * sizeof(int32_t)));
+  RAP_CUDA_TRY(c, cudaMalloc(&c->d_unit_cnt, 2 * (size_t)d.max_batch * d.n_kv_heads * sizeof(int32_t)));
+  RAP_CUDA_TRY(c, cudaMemset(c->d_unit_cnt, 0, 2 * (size_t)d.max_batch * d.n_kv_heads * sizeof(int32_t)));
   RAP_CUDA_TRY(c, cudaMalloc(&c->d_proj_ws, c->proj_ws_bytes));
+  c->proj_cnt_n = 4 * (int)((n_out_max + 127) / 128);
+  RAP_CUDA_TRY(c, cudaMalloc(&c->d_proj_cnt, 2 * (size_t)c->proj_cnt_n * sizeof(int32_t)));
+  RAP_CUDA_TRY(c, cudaMemset(c->d_proj_cnt, 0, 2 * (size_t)c->proj_cnt_n * sizeof(int32_t)));
   RAP_CUDA_TRY(c, cudaMalloc(&c->d_stage_x, c->stage_x_bytes));
   RAP_CUDA_TRY(c, cudaMalloc(&c->d_stage_out, c->stage_out_bytes));
   RAP_CUDA_TRY(c, cudaMalloc(&c->d_stage_q, (size_t)d.max_batch * d.n_q_heads * d.head_dim * e));
@@ -465,6 +475,7 @@ rap_status rap_decode_step(rap_ctx* ctx, int32_t B, const void* d_x, const void*
   cudaStream_t st = (cudaStream_t)stream;
   const size_t e = rap_elem_bytes(d.dtype);
   for (int l = 0; l < d.n_layers; ++l) {
+    const bool timed = 2 * (ctx->prof_pairs + 1) <= (int)ctx->prof_ev.size();   // events around this layer's attention
     rap_proj_args p;
     p.x = (const char*)d_x + (size_t)l * B * d.hidden * e;
     p.w = h_w_qkv[l]; p.bias = h_bias ? h_bias[l] : nullptr;
@@ -474,6 +485,10 @@ rap_status rap_decode_step(rap_ctx* ctx, int32_t B, const void* d_x, const void*
     p.T = B; p.hidden = d.hidden; p.Hq = d.n_q_heads; p.Hkv = d.n_kv_heads;
     p.P2 = 2 * ctx->n_pairs[l]; p.dv = ctx->n_vch[l]; p.half_dim = d.head_dim / 2;
     p.B_cache = B; p.S_cap = S_cap; p.dtype = d.dtype;
+    // Inside a step the library knows what precedes each launch: from the second layer on the projection follows
+    // an attention launch that does not touch what the projection reads, so it may start streaming its weights
+    // while that launch drains (the first projection follows caller work, e.g. the length update, and waits).
+    p.pdl = (l > 0 && !timed) ? 1 : 0;
     rap_status s = rap_launch_qkv_rope_append(ctx, p, st);
     if (s != RAP_OK) return s;
     rap_attn_args a;
@@ -481,7 +496,7 @@ rap_status rap_decode_step(rap_ctx* ctx, int32_t B, const void* d_x, const void*
     a.B = B; a.Hq = d.n_q_heads; a.Hkv = d.n_kv_heads; a.P2 = p.P2; a.dv = p.dv; a.S_cap = S_cap;
     a.head_dim = d.head_dim; a.dtype = d.dtype; a.n_split = n_split; a.h_len_max = h_seq_len_max + 1;
     a.out = d_out + (size_t)l * out_layer_stride;
-    const bool timed = 2 * (ctx->prof_pairs + 1) <= (int)ctx->prof_ev.size();
+    a.pdl = timed ? 0 : 1;
     if (timed) RAP_CUDA_TRY(ctx, cudaEventRecord(ctx->prof_ev[2 * ctx->prof_pairs], st));
     s = rap_launch_attn(ctx, a, st);
     if (s != RAP_OK) return s;
@@ -577,9 +592,10 @@ rap_status rap_get_last_device_status(rap_ctx* ctx, int32_t* code, int32_t* deta
   RAP_CUDA_TRY(ctx, cudaMemcpyAsync(h, ctx->d_status, sizeof(h), cudaMemcpyDeviceToHost, st));
   RAP_CUDA_TRY(ctx, cudaMemsetAsync(ctx->d_status, 0, sizeof(h), st));
   RAP_CUDA_TRY(ctx, cudaStreamSynchronize(st));
-  if (h[0] != 0) {   // a kernel that gave up may have left unit arrival counters behind
+  if (h[0] != 0) {   // a kernel that gave up may have left arrival counters behind (the next launches clear them too)
     const rap_model_desc& d = ctx->desc;
-    RAP_CUDA_TRY(ctx, cudaMemsetAsync(ctx->d_unit_cnt, 0, (size_t)d.max_batch * d.n_kv_heads * sizeof(int32_t), st));
+    RAP_CUDA_TRY(ctx, cudaMemsetAsync(ctx->d_unit_cnt, 0, 2 * (size_t)d.max_batch * d.n_kv_heads * sizeof(int32_t), st));
+    RAP_CUDA_TRY(ctx, cudaMemsetAsync(ctx->d_proj_cnt, 0, 2 * (size_t)ctx->proj_cnt_n * sizeof(int32_t), st));
     RAP_CUDA_TRY(ctx, cudaStreamSynchronize(st));
   }
   *code = h[0];

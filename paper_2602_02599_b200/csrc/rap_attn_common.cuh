@@ -78,6 +78,11 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
   if (mbar_try_wait(bar, parity)) return true;
   return mbar_wait_slow(bar, parity);
 }
+// Programmatic dependent launch (no-ops in a kernel launched without the attribute): wait until the previous kernel
+// in the stream has completed and its writes are visible; let the next kernel in the stream start its prologue.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // global -> this CTA's shared memory, completion counted in bytes on the mbarrier (no multicast)
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
   asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),

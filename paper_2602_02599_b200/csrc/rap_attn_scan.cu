@@ -75,7 +75,13 @@ static rap_status launch_split_kv(rap_ctx* ctx, const rap_attn_args& a, int n_sp
   p.len_add = a.len_add; p.Hq = a.Hq; p.Hkv = a.Hkv; p.S_cap = a.S_cap; p.n_split = n_split;
   p.qscale = (float)(1.4426950408889634 / sqrt((double)a.head_dim));
   p.B = a.B; p.balanced = balanced ? 1 : 0;
-  p.unit_cnt = ctx->d_unit_cnt; p.out = a.out;
+  {   // two counter sets take turns; each launch clears the one its predecessor used
+    const size_t n_units = (size_t)ctx->desc.max_batch * ctx->desc.n_kv_heads;
+    const uint32_t set = balanced ? (ctx->scan_epoch++ & 1u) : 0u;
+    p.unit_cnt = ctx->d_unit_cnt + set * n_units;
+    p.unit_cnt_other = ctx->d_unit_cnt + (set ^ 1u) * n_units;
+  }
+  p.out = a.out;
   RAP_CUDA_TRY(ctx, rap_raise_smem(ctx, e->fn, e->smem));
   const int scan_grid = 2 * ctx->sm_count;
   dim3 grid(n_split, a.Hkv, a.B);
@@ -88,7 +94,17 @@ static rap_status launch_split_kv(rap_ctx* ctx, const rap_attn_args& a, int n_sp
       return RAP_EUNSUPPORTED;
   }
   void* args[] = {&p, map_k, map_v};
-  RAP_CUDA_TRY(ctx, cudaLaunchKernel(e->fn, grid, dim3(e->threads), args, (size_t)e->smem, st));
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = dim3(e->threads);
+  cfg.dynamicSmemBytes = (size_t)e->smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = a.pdl ? 1 : 0;      // the kernel waits for its predecessor before it reads q~ or a cache row
+  RAP_CUDA_TRY(ctx, cudaLaunchKernelExC(&cfg, e->fn, args));
   ctx->launches++;
   RAP_CUDA_TRY(ctx, cudaGetLastError());
   if (balanced) {

@@ -153,8 +153,14 @@ __global__ void __launch_bounds__(STHREADS, 2) attn_scan_kernel(const ScanParams
   plan.T = 0; plan.nc = 0;
   int cur = 0, hi = 0, unit_start = 0;
   if (p.balanced) {
-    plan = sk_plan(p.seq_len, p.B, p.Hkv, p.len_add, p.S_cap, ST, (int)gridDim.x);
+    plan = sk_plan(p.seq_len, p.B, p.Hkv, p.len_add, p.S_cap, ST, (int)gridDim.x);   // reads the lengths only
+    // Everything below reads q~ and the cache rows the previous kernel in the stream wrote, and writes what the next
+    // one may depend on: wait for the predecessor first, and only then let the successor start (it may begin to
+    // stream its weights while this scan runs, and waits for this kernel before it writes anything this one reads).
+    pdl_wait();
+    pdl_launch_dependents();
     if (blockIdx.x == 0) {   // sequences without any row are scanned by nobody: their output is zero
+      for (int i = tid; i < p.B * p.Hkv; i += STHREADS) p.unit_cnt_other[i] = 0;   // counters a launch that gave up left behind
       for (int bb = 0; bb < p.B; ++bb)
         if (sk_tiles_of(p.seq_len, bb, p.len_add, p.S_cap, ST) == 0)
           for (int i = tid; i < p.Hq * DV; i += STHREADS) p.out[(size_t)bb * p.Hq * DV + i] = 0.f;
@@ -174,6 +180,8 @@ __global__ void __launch_bounds__(STHREADS, 2) attn_scan_kernel(const ScanParams
     h = (cur - pb) / ntb;
     unit_start = pb + h * ntb;
   } else {
+    pdl_wait();
+    pdl_launch_dependents();
     b = blockIdx.z;
     h = blockIdx.y;
   }

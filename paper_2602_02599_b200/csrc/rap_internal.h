@@ -27,9 +27,13 @@ struct rap_ctx {
   int32_t* d_status = nullptr;    // [2] = {code, detail}
   float* d_attn_ws = nullptr;     // split-KV partials
   size_t attn_ws_bytes = 0;
-  int32_t* d_unit_cnt = nullptr;  // [max_batch][H_kv] partial-arrival counters of the balanced scan (zero between calls)
+  int32_t* d_unit_cnt = nullptr;  // [2][max_batch][H_kv] partial-arrival counters of the balanced scan (zero between calls)
+  uint32_t scan_epoch = 0;        // balanced scans launched so far: picks the counter set
   float* d_proj_ws = nullptr;     // fp32 projection results / split-K partials
   size_t proj_ws_bytes = 0;
+  int32_t* d_proj_cnt = nullptr;  // fused projection: two sets of [row tiles][4] split-arrival counters (zero between calls)
+  int proj_cnt_n = 0;             // counters per set
+  uint32_t proj_epoch = 0;        // launches of the fused projection so far: picks the set
   void* d_stage_x = nullptr;      // staging for rap_decode_step_host
   float* d_stage_out = nullptr;
   void* d_stage_q = nullptr;
@@ -55,6 +59,7 @@ struct rap_ctx {
   std::vector<MapSlot> tmaps;         // encoded tensor maps, reused while (pointer, shape, box) repeat
   size_t tmap_next = 0;
   int32_t attn_variant = 0;
+  int32_t proj_variant = 0;       // 1: rap_qkv_rope_append always takes the two-stage path (GEMM, then the epilogue kernel)
   int64_t launches = 0;
   std::string cuda_error;
   // lazily created tensor maps / per-device attributes live in the .cu files
@@ -91,6 +96,7 @@ struct rap_scan_params {
   int len_add, Hq, Hkv, S_cap, n_split;
   float qscale;
   int32_t* unit_cnt;   // balanced mode: arrivals per (sequence, KV head) unit, zero between calls
+  int32_t* unit_cnt_other;   // the set the previous launch used; cleared by this launch (two sets take turns)
   float* out;          // balanced mode: [B][Hq][DV], written by the CTA that completes a unit
   int B;               // sequences (used by the balanced mode)
   int balanced;        // 0: grid (n_split, H_kv, B), equal tile ranges per split; 1: grid (CTAs), see SkPlan
@@ -117,6 +123,7 @@ struct rap_attn_args {
   int32_t B, Hq, Hkv, P2, dv, S_cap, head_dim, dtype;
   int32_t n_split, h_len_max;
   float* out;
+  int32_t pdl = 0;          // launch the scan with programmatic stream serialization (inside rap_decode_step)
 };
 rap_status rap_launch_attn(rap_ctx* ctx, const rap_attn_args& a, cudaStream_t st);
 
@@ -126,6 +133,7 @@ struct rap_proj_args {
   const double* inv_freq;   // this layer's [H_kv][D/2]
   void* q_out; void* k_cache; void* v_cache;
   int32_t T, hidden, Hq, Hkv, P2, dv, half_dim, B_cache, S_cap, dtype;
+  int32_t pdl = 0;          // launch with programmatic stream serialization (inside rap_decode_step, after an attention launch)
 };
 rap_status rap_launch_qkv_rope_append(rap_ctx* ctx, const rap_proj_args& a, cudaStream_t st);
 

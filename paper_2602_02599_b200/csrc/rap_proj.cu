@@ -1,7 +1,8 @@
 // Pruned QKV projection (Eq. 1 on the reduced widths), index-aware RoPE on the retained
 // pairs (Eq. 3 with each pair's original frequency) and append into the compact cache.
 //
-// Two stages on the caller's stream:
+// Decode-sized bf16 calls (T <= 32) run as ONE kernel: the tcgen05 GEMM of rap_proj_tc.cu with this epilogue
+// fused in.  Every other call takes two stages on the caller's stream:
 //   1. a GEMM  Y[ks][t][n] = sum_{k in split ks} X[t][k] * W~[n][k]   (fp32 results in the
 //      context workspace; ks = reduction split so that weight streaming can use every SM),
 //   2. an epilogue that sums the splits, adds the bias, rotates q~/k~ pairs, rounds once to the
@@ -12,6 +13,7 @@
 #include "rap_internal.h"
 
 rap_status rap_launch_proj_tc(rap_ctx* ctx, const rap_proj_args& a, int* ksplit_out, cudaStream_t st);
+rap_status rap_launch_proj_fused(rap_ctx* ctx, const rap_proj_args& a, cudaStream_t st);
 rap_status rap_launch_gemm_tc(rap_ctx* ctx, const void* x, const void* w, int T, int K, int N, int* ksplit_out,
                               cudaStream_t st);
 
@@ -258,6 +260,10 @@ rap_status rap_launch_qkv_rope_append(rap_ctx* ctx, const rap_proj_args& a, cuda
   const int n_out = (a.Hq + a.Hkv) * a.P2 + a.Hkv * a.dv;
   int ksplit = 1;
   rap_status s = RAP_EUNSUPPORTED;
+  if (a.dtype == RAP_BF16 && ctx->proj_variant != 1) {      // decode-sized calls: one launch, epilogue fused in
+    s = rap_launch_proj_fused(ctx, a, st);
+    if (s != RAP_EUNSUPPORTED) return s;
+  }
   if (a.dtype == RAP_BF16) s = rap_launch_proj_tc(ctx, a, &ksplit, st);
   if (s == RAP_EUNSUPPORTED) {
     ksplit = 1;

@@ -20,9 +20,17 @@
 //            stage; a last commit signals the accumulator;
 //   warps 2-5 epilogue: tcgen05.ld of the warp's 32 lanes x 32 columns, coalesced fp32 stores to
 //            the workspace (consecutive lanes = consecutive output features n).
-// A reduction split (grid.z) lets a decode-sized call use every SM; the RoPE / append epilogue
-// kernel sums the splits.  Every mbarrier wait is bounded; a wait that gives up records
-// RAP_ETIMEOUT in the device status word and the CTA winds down.
+// A reduction split lets a decode-sized call use every SM.  For calls of more than 32 rows the RoPE / append
+// epilogue kernel (rap_proj.cu) sums the splits.  For decode-sized calls (T <= 32) the epilogue is fused in
+// (FUSED = true): every epilogue warp owns 32 weight rows of its CTA's row tile; it stores its partial, and the warp
+// that delivers the last split of those 32 rows (an arrival counter per row tile and warp quarter) sums the
+// splits from L2, adds the bias, rotates the retained pairs (the partner of a row is the adjacent row, i.e. the
+// adjacent lane), rounds once and scatters q~ / K row / V row -- no second launch, no second pass.  The sine and
+// cosine of a lane's rows are computed while the warp would otherwise wait for the accumulator.  The fused kernel
+// also takes part in programmatic dependent launch: it lets its successor start early and waits for its
+// predecessor only before it writes q~ and the cache rows (its weight streaming overlaps the predecessor's tail).
+// Every mbarrier wait is bounded; a wait that gives up records RAP_ETIMEOUT in the device status word and the
+// CTA winds down.
 #include <cuda.h>
 
 #include <string.h>
@@ -48,6 +56,10 @@ struct TcCfg {
   static constexpr int NS = NS_RAW > 8 ? 8 : NS_RAW;
   static constexpr int OFF_BARS = NS * STAGE;                   // full[NS], empty[NS], acc_full[2], acc_empty[2], tmem slot
   static constexpr int SMEM = OFF_BARS + (2 * NS + 5) * 8 + 1024;   // + slack to align the ring to 1024 bytes
+  // fused epilogue: per epilogue warp [16][32] (cos, sin) pairs and [32][32] summed results
+  static constexpr int OFF_FUSED = (OFF_BARS + (2 * NS + 5) * 8 + 15) & ~15;
+  static constexpr int FUSED_WARP_BYTES = 16 * 32 * 8 + 32 * 32 * 4;
+  static constexpr int SMEM_FUSED = OFF_FUSED + 4 * FUSED_WARP_BYTES + 1024;
   // instruction descriptor: fp32 accumulate, bf16 x bf16, both K-major, N = TN, M = 128
   static constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(TN >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
 };
@@ -121,6 +133,25 @@ struct TcParams {
   int row_tiles, tok_tiles, n_work;     // work items = row tiles x token tiles x reduction splits
 };
 
+// What the fused RoPE / append epilogue needs beyond the GEMM (decode-sized calls, one token tile).
+struct TcFused {
+  const __nv_bfloat16* bias;                 // [n_out] or nullptr
+  const int32_t* seq_id;                     // nullptr: row t belongs to sequence t
+  const int32_t* pos;
+  const int32_t* slot;                       // nullptr: slot = pos
+  const double* inv_freq;                    // this layer's [H_kv][half_dim]
+  __nv_bfloat16* q_out;
+  __nv_bfloat16* k_cache;
+  __nv_bfloat16* v_cache;
+  int32_t* cnt;                              // [row_tiles][4] split arrivals of this launch (zero on entry, zero on exit)
+  int32_t* cnt_other;                        // the set the previous launch used: cleared here in case that launch gave up
+  int n_cnt;
+  int ksplit, Hq, Hkv, P2, dv, half_dim, B_cache, S_cap;
+};
+
+__device__ __forceinline__ void tc_pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void tc_pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 __device__ __forceinline__ void tc_mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
@@ -128,10 +159,12 @@ __device__ __forceinline__ void tc_mbar_arrive(uint32_t bar) {
 // Persistent: CTA c takes work items c, c + gridDim.x, ...  The stage ring runs on across items, and the
 // accumulator is double buffered in tensor memory (2 x TN columns) so that the epilogue of one item
 // overlaps the MMAs of the next.
-template <int TN>
+template <int TN, bool FUSED>
 __global__ void __launch_bounds__(TC_THREADS, 1)
-proj_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x, const TcParams p) {
+proj_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_x, const TcParams p,
+               const TcFused f) {
   using C = TcCfg<TN>;
+  static_assert(!FUSED || TN == 32, "the fused epilogue holds one 32-token chunk per lane");
   extern __shared__ unsigned char tc_smem_raw[];
   // the swizzled tiles and their descriptors want a 1024-byte aligned ring
   unsigned char* smem = tc_smem_raw + ((1024u - (tc_smem_u32(tc_smem_raw) & 1023u)) & 1023u);
@@ -164,6 +197,11 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_d = *tmem_slot;
   bool timed_out = false;
+  if constexpr (FUSED) {
+    tc_pdl_launch_dependents();      // the next kernel in the stream may start its own prologue
+    if (blockIdx.x == 0)             // counters a predecessor that gave up may have left behind
+      for (int i = threadIdx.x; i < f.n_cnt; i += TC_THREADS) f.cnt_other[i] = 0;
+  }
 
   // work item w -> (token tile, row tile, split); token tiles vary fastest so that the CTAs working at the
   // same time share a weight tile through L2
@@ -228,6 +266,46 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
       decode(w, n0, t0, ks, kb0, nkb);
       const int n = n0 + quarter * 32 + lane;
       const uint32_t buf = it & 1u, use = it >> 1;
+
+      // fused epilogue, part 1 (while the MMAs of this item run): what this lane's weight row is, where its results
+      // go, and the sine and cosine of its pair -- each lane of a pair evaluates half of the tokens (the even lane
+      // 0..15, the odd lane 16..31) into shared memory.  The loops of the fused epilogue are kept rolled: a warp runs
+      // this code once, so its cost is the instruction fetch as much as the arithmetic.
+      int kind = 2;                            // 0: q row, 1: k row, 2: v row (or past the end)
+      __nv_bfloat16* dst = nullptr;            // q~: element of token 0; K / V: element of cache row 0 of this lane's head
+      int row_w = 0;                           // K / V: row width in elements
+      float2* cs_w = nullptr;                  // [16][32] (cos, sin): entry [j][l] belongs to token j + 16 (l & 1) of lane l's pair
+      float* vs_w = nullptr;                   // [32][32] summed results, token-major
+      if constexpr (FUSED) {
+        unsigned char* fw = smem + C::OFF_FUSED + quarter * C::FUSED_WARP_BYTES;
+        cs_w = reinterpret_cast<float2*>(fw);
+        vs_w = reinterpret_cast<float*>(fw + 16 * 32 * 8);
+        const int nq = f.Hq * f.P2, nk = f.Hkv * f.P2;
+        int head = 0, r = 0;
+        if (n < nq) { kind = 0; head = n / f.P2; r = n - head * f.P2; }
+        else if (n < nq + nk) { kind = 1; head = (n - nq) / f.P2; r = n - nq - head * f.P2; }
+        else if (n < p.n_out) { head = (n - nq - nk) / f.dv; r = n - nq - nk - head * f.dv; }
+        const int hkv = kind == 0 ? head / (f.Hq / f.Hkv) : head;
+        const double freq = kind < 2 ? f.inv_freq[hkv * f.half_dim + (r >> 1)] : 0.0;
+        if (kind == 0) dst = f.q_out + (size_t)head * f.P2 + r;
+        else if (kind == 1) { dst = f.k_cache + (size_t)head * f.S_cap * f.P2 + r; row_w = f.P2; }
+        else { dst = f.v_cache + (size_t)head * f.S_cap * f.dv + r; row_w = f.dv; }
+#pragma unroll 1
+        for (int j = 0; j < 16; ++j) {
+          const int t = j + 16 * (lane & 1);
+          float c = 1.f, sn = 0.f;
+          if (t < p.T && freq != 0.0) {
+            // fp64 angle and reduction to [-pi, pi] (positions reach 1e5 and more), fp32 sine and cosine of the rest
+            const double ang = (double)f.pos[t] * freq;
+            const double turns = rint(ang * 0.15915494309189535);
+            const double red = fma(-turns, 2.4492935982947064e-16, fma(-turns, 6.283185307179586, ang));
+            sincosf((float)red, &sn, &c);
+          }
+          cs_w[j * 32 + lane] = make_float2(c, sn);
+        }
+        __syncwarp();
+      }
+
       bool ready = true;
       if (nkb > 0) {
         ready = __all_sync(0xffffffffu, !timed_out && tc_mbar_wait(acc_full0 + 8 * buf, use & 1u));
@@ -238,19 +316,19 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
 #pragma unroll 1
       for (int c0 = 0; c0 < TN; c0 += 32) {
         if (t0 + c0 >= p.T) break;             // columns past the last token hold zero-filled rows
-        uint32_t r[32];
+        uint32_t r32[32];
         if (nkb > 0 && ready) {
-          tc_ld32(tmem_d + buf * TN + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c0, r);
+          tc_ld32(tmem_d + buf * TN + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c0, r32);
           asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
         } else {
 #pragma unroll
-          for (int j = 0; j < 32; ++j) r[j] = 0u;
+          for (int j = 0; j < 32; ++j) r32[j] = 0u;
         }
         if (n < p.n_out) {
 #pragma unroll
           for (int j = 0; j < 32; ++j) {
             const int t = t0 + c0 + j;
-            if (t < p.T) ybase[(size_t)t * p.n_out + n] = __uint_as_float(r[j]);
+            if (t < p.T) ybase[(size_t)t * p.n_out + n] = __uint_as_float(r32[j]);
           }
         }
       }
@@ -261,6 +339,73 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
           if (lane == 0) tc_mbar_arrive(acc_empty0 + 8 * buf);    // this warp has drained the accumulator
         }
         ++it;
+      }
+
+      if constexpr (FUSED) {
+        // fused epilogue, part 2: count this warp's partial in; the warp that brings the last one finishes the rows.
+        // A warp that timed out does not count itself in, so the rows are never finished from a missing partial.
+        int last = 0;
+        if (ready) {
+          __threadfence();                       // the partial is visible before the arrival is
+          __syncwarp();
+          const int slot_c = (n0 / TC_BM) * 4 + quarter;
+          if (lane == 0) last = atomicAdd(&f.cnt[slot_c], 1) == f.ksplit - 1;
+          last = __shfl_sync(0xffffffffu, last, 0);
+          if (last) {
+            __threadfence();
+            tc_pdl_wait();                       // the previous kernel in the stream may still read q~
+            const size_t split_stride = (size_t)p.T * p.n_out;
+            const bool in_range = n < p.n_out;
+            // sum the splits: a split at a time, its (up to) 32 loads independent of one another
+            {
+              float v[32];
+              const float bias = (in_range && f.bias) ? __bfloat162float(f.bias[n]) : 0.f;
+#pragma unroll
+              for (int t = 0; t < 32; ++t) v[t] = bias;
+#pragma unroll 1
+              for (int s2 = 0; s2 < f.ksplit; ++s2) {
+                const float* src = p.y + s2 * split_stride + n;
+                float part[32];
+#pragma unroll
+                for (int t = 0; t < 32; ++t) part[t] = (t < p.T && in_range) ? __ldcg(src + (size_t)t * p.n_out) : 0.f;
+#pragma unroll
+                for (int t = 0; t < 32; ++t) v[t] += part[t];
+              }
+#pragma unroll
+              for (int t = 0; t < 32; ++t) vs_w[t * 32 + lane] = v[t];
+            }
+            // where the row of token `lane` goes: its cache row index over all sequences and heads of head 0, or -1
+            int my_row = -1;
+            if (lane < p.T) {
+              const int ps = f.pos[lane];
+              const int sq = f.seq_id ? f.seq_id[lane] : lane;
+              const int sl = f.slot ? f.slot[lane] : ps;
+              if (sq >= 0 && sq < f.B_cache && sl >= 0 && sl < f.S_cap) {
+                my_row = sq * f.Hkv * f.S_cap + sl;      // the host checked that B_cache * H_kv * S_cap fits
+              } else if (n0 == 0 && quarter == 0) {      // reported once per launch: by the warp that owns weight row 0
+                atomicCAS(&p.status[0], 0, (int)RAP_ECAPACITY);
+                p.status[1] = lane;
+              }
+            }
+            __syncwarp();
+            const size_t q_stride = (size_t)f.Hq * f.P2;
+            const int cs_lane = (lane & ~1);
+#pragma unroll 4
+            for (int t = 0; t < p.T; ++t) {
+              const float mine = vs_w[t * 32 + lane], other = vs_w[t * 32 + (lane ^ 1)];
+              const float2 cs = cs_w[(t & 15) * 32 + (cs_lane | (t >> 4))];
+              const int row = __shfl_sync(0xffffffffu, my_row, t);
+              // pair (a, b) on lanes (even, odd):  a' = a cos - b sin,  b' = a sin + b cos
+              const float rot = (lane & 1) ? fmaf(other, cs.y, mine * cs.x) : fmaf(-other, cs.y, mine * cs.x);
+              const __nv_bfloat16 o = __float2bfloat16_rn(kind == 2 ? mine : rot);
+              if (in_range) {
+                if (kind == 0) dst[t * q_stride] = o;
+                else if (row >= 0) dst[(size_t)row * row_w] = o;   // a row whose sequence or slot is out of range is skipped
+              }
+            }
+            if (lane == 0) f.cnt[slot_c] = 0;      // ready for the next launch that uses this set
+          }
+        }
       }
     }
   }
@@ -326,11 +471,32 @@ bool make_map(rap_ctx* ctx, CUtensorMap* map, const void* base, uint64_t rows, u
 template <int TN>
 rap_status launch_tc(rap_ctx* ctx, const CUtensorMap& mw, const CUtensorMap& mx, const TcParams& p, dim3 grid,
                      cudaStream_t st) {
-  RAP_CUDA_TRY(ctx, rap_raise_smem(ctx, proj_tc_kernel<TN>, TcCfg<TN>::SMEM));
-  proj_tc_kernel<TN><<<grid, TC_THREADS, TcCfg<TN>::SMEM, st>>>(mw, mx, p);
+  RAP_CUDA_TRY(ctx, rap_raise_smem(ctx, proj_tc_kernel<TN, false>, TcCfg<TN>::SMEM));
+  proj_tc_kernel<TN, false><<<grid, TC_THREADS, TcCfg<TN>::SMEM, st>>>(mw, mx, p, TcFused{});
   ctx->launches++;
   RAP_CUDA_TRY(ctx, cudaGetLastError());
   return RAP_OK;
+}
+
+// Work split of one GEMM call: token tile width, reduction splits (enough CTAs for every SM on decode-sized
+// calls, within the workspace, no empty split) and the work-item counts.
+bool plan_gemm(const rap_ctx* ctx, int T, int K, int N, int* tn_out, int* ksplit_out, TcParams* p) {
+  const int tn = T <= 32 ? 32 : T <= 64 ? 64 : T <= 128 ? 128 : 256;
+  const int row_tiles = (N + TC_BM - 1) / TC_BM, tok_tiles = (T + tn - 1) / tn;
+  const int nkb = (K + TC_BK - 1) / TC_BK;
+  int ksplit = ctx->sm_count / (row_tiles * tok_tiles);
+  if (ksplit > RAP_MAX_KSPLIT) ksplit = RAP_MAX_KSPLIT;
+  if (ksplit > nkb / 4) ksplit = nkb / 4;
+  while (ksplit > 1 && (size_t)ksplit * T * N * sizeof(float) > ctx->proj_ws_bytes) --ksplit;
+  if (ksplit < 1) ksplit = 1;
+  const int per = (nkb + ksplit - 1) / ksplit;
+  ksplit = (nkb + per - 1) / per;          // no empty split
+  if ((size_t)ksplit * T * N * sizeof(float) > ctx->proj_ws_bytes) return false;
+  p->y = ctx->d_proj_ws; p->status = ctx->d_status; p->T = T; p->n_out = N; p->nkb_total = nkb; p->nkb_per_split = per;
+  p->row_tiles = row_tiles; p->tok_tiles = tok_tiles; p->n_work = row_tiles * tok_tiles * ksplit;
+  *tn_out = tn;
+  *ksplit_out = ksplit;
+  return true;
 }
 
 }  // namespace
@@ -339,28 +505,16 @@ bool rap_tensor_map_bf16(rap_ctx* ctx, void* map128, const void* base, uint64_t 
   return make_map(ctx, reinterpret_cast<CUtensorMap*>(map128), base, rows, cols, box_rows);
 }
 
-// Y[ks][T][N] (fp32, context workspace) = X[T][K] * W[N][K]^T, bf16 operands, K split over grid.z.
+// Y[ks][T][N] (fp32, context workspace) = X[T][K] * W[N][K]^T, bf16 operands, K split over work items.
 rap_status rap_launch_gemm_tc(rap_ctx* ctx, const void* x, const void* w, int T, int K, int N, int* ksplit_out,
                               cudaStream_t st) {
   if (T < 1 || (K % 8) != 0) return RAP_EUNSUPPORTED;     // tensor-map rows must be multiples of 16 bytes
-  const int tn = T <= 32 ? 32 : T <= 64 ? 64 : T <= 128 ? 128 : 256;
+  TcParams p;
+  int tn = 0, ksplit = 1;
+  if (!plan_gemm(ctx, T, K, N, &tn, &ksplit, &p)) return RAP_EUNSUPPORTED;
   CUtensorMap mw, mx;
   if (!make_map(ctx, &mw, w, (uint64_t)N, (uint64_t)K, TC_BM)) return RAP_EUNSUPPORTED;
   if (!make_map(ctx, &mx, x, (uint64_t)T, (uint64_t)K, (uint32_t)tn)) return RAP_EUNSUPPORTED;
-  const int row_tiles = (N + TC_BM - 1) / TC_BM, tok_tiles = (T + tn - 1) / tn;
-  const int nkb = (K + TC_BK - 1) / TC_BK;
-  // reduction split: enough CTAs for every SM on decode-sized calls, within the workspace
-  int ksplit = ctx->sm_count / (row_tiles * tok_tiles);
-  if (ksplit > RAP_MAX_KSPLIT) ksplit = RAP_MAX_KSPLIT;
-  if (ksplit > nkb / 4) ksplit = nkb / 4;
-  while (ksplit > 1 && (size_t)ksplit * T * N * sizeof(float) > ctx->proj_ws_bytes) --ksplit;
-  if (ksplit < 1) ksplit = 1;
-  int per = (nkb + ksplit - 1) / ksplit;
-  ksplit = (nkb + per - 1) / per;          // no empty split
-  if ((size_t)ksplit * T * N * sizeof(float) > ctx->proj_ws_bytes) return RAP_EUNSUPPORTED;
-  TcParams p;
-  p.y = ctx->d_proj_ws; p.status = ctx->d_status; p.T = T; p.n_out = N; p.nkb_total = nkb; p.nkb_per_split = per;
-  p.row_tiles = row_tiles; p.tok_tiles = tok_tiles; p.n_work = row_tiles * tok_tiles * ksplit;
   dim3 grid(p.n_work < ctx->sm_count ? p.n_work : ctx->sm_count, 1, 1);
   *ksplit_out = ksplit;
   switch (tn) {
@@ -375,4 +529,44 @@ rap_status rap_launch_proj_tc(rap_ctx* ctx, const rap_proj_args& a, int* ksplit_
   if (a.dtype != RAP_BF16) return RAP_EUNSUPPORTED;
   const int n_out = (a.Hq + a.Hkv) * a.P2 + a.Hkv * a.dv;
   return rap_launch_gemm_tc(ctx, a.x, a.w, a.T, a.hidden, n_out, ksplit_out, st);
+}
+
+// Decode-sized rap_qkv_rope_append in ONE launch: the tcgen05 GEMM with the RoPE / append epilogue fused in.
+// RAP_EUNSUPPORTED when the call is not decode-sized (T > 32) or not bf16; the caller then takes the two-stage path.
+// a.pdl != 0 launches the kernel with programmatic stream serialization (its weight streaming may overlap the tail
+// of the previous kernel in the stream; it waits for that kernel before it writes q~ or the cache rows).
+rap_status rap_launch_proj_fused(rap_ctx* ctx, const rap_proj_args& a, cudaStream_t st) {
+  if (a.dtype != RAP_BF16 || a.T < 1 || a.T > 32 || (a.hidden % 8) != 0 || (a.P2 & 1)) return RAP_EUNSUPPORTED;
+  const int n_out = (a.Hq + a.Hkv) * a.P2 + a.Hkv * a.dv;
+  TcParams p;
+  int tn = 0, ksplit = 1;
+  if (!plan_gemm(ctx, a.T, a.hidden, n_out, &tn, &ksplit, &p) || tn != 32 || p.tok_tiles != 1) return RAP_EUNSUPPORTED;
+  if (4 * p.row_tiles > ctx->proj_cnt_n) return RAP_EUNSUPPORTED;
+  if ((long long)a.B_cache * a.Hkv * a.S_cap >= (1LL << 31)) return RAP_EUNSUPPORTED;   // cache row indices are 32-bit in the epilogue
+  CUtensorMap mw, mx;
+  if (!make_map(ctx, &mw, a.w, (uint64_t)n_out, (uint64_t)a.hidden, TC_BM)) return RAP_EUNSUPPORTED;
+  if (!make_map(ctx, &mx, a.x, (uint64_t)a.T, (uint64_t)a.hidden, 32u)) return RAP_EUNSUPPORTED;
+  TcFused f;
+  f.bias = (const __nv_bfloat16*)a.bias; f.seq_id = a.seq_id; f.pos = a.pos; f.slot = a.slot; f.inv_freq = a.inv_freq;
+  f.q_out = (__nv_bfloat16*)a.q_out; f.k_cache = (__nv_bfloat16*)a.k_cache; f.v_cache = (__nv_bfloat16*)a.v_cache;
+  const int set = (int)(ctx->proj_epoch++ & 1u);       // two counter sets take turns; each launch clears the other one
+  f.cnt = ctx->d_proj_cnt + set * ctx->proj_cnt_n;
+  f.cnt_other = ctx->d_proj_cnt + (set ^ 1) * ctx->proj_cnt_n;
+  f.n_cnt = ctx->proj_cnt_n;
+  f.ksplit = ksplit; f.Hq = a.Hq; f.Hkv = a.Hkv; f.P2 = a.P2; f.dv = a.dv; f.half_dim = a.half_dim;
+  f.B_cache = a.B_cache; f.S_cap = a.S_cap;
+  RAP_CUDA_TRY(ctx, rap_raise_smem(ctx, proj_tc_kernel<32, true>, TcCfg<32>::SMEM_FUSED));
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(p.n_work < ctx->sm_count ? p.n_work : ctx->sm_count, 1, 1);
+  cfg.blockDim = dim3(TC_THREADS, 1, 1);
+  cfg.dynamicSmemBytes = TcCfg<32>::SMEM_FUSED;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = a.pdl ? 1 : 0;
+  RAP_CUDA_TRY(ctx, cudaLaunchKernelEx(&cfg, proj_tc_kernel<32, true>, mw, mx, p, f));
+  ctx->launches++;
+  return RAP_OK;
 }

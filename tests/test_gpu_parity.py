@@ -690,3 +690,83 @@ def test_frequency_scaled_tables_end_to_end():
     util.check_attn(util.to_np64(out).reshape(w.batch * T, w.n_q_heads, dv), want.reshape(w.batch * T, w.n_q_heads, dv), w.dtype)
     assert st.ctx.rap_get_last_device_status() == (0, 0)
     st.close()
+
+
+@pytest.mark.parametrize("name,T,with_bias", [("8b", 32, False), ("3b", 16, True), ("14b", 4, False), ("sweep1.0", 1, True),
+                                              ("sweep0.5", 7, False), ("8b", 31, True)])
+def test_fused_projection_against_the_oracle_and_the_two_stage_form(name, T, with_bias):
+    """Decode-sized rap_qkv_rope_append runs as one kernel (RoPE, rounding and append fused into the tcgen05 GEMM's
+    epilogue, finished by whichever warp delivers a row block's last reduction split).  Rows of several sequences at
+    scattered slots and far-apart positions, with and without a bias, on head shapes whose q / k / v sections start in
+    the middle of a 32-row block (odd d_v' included): q~, the K rows and the V rows against the oracle, against the
+    two-stage form of the same call, canaries around every written row, and twice in a row (the arrival counters
+    must come back to zero)."""
+    w = synth.scaled_down(synth.CONFIGS[name], n_layers=2, batch=3, seq=64, hidden=1024)
+    ks, vs = synth.draw_scores(w)
+    st, tabs, w_host = util.build_small_stack(w, ks, vs, full_weights=False, s_cap=4096, max_rows=32)
+    Hq, Hkv, P, dv = w.n_q_heads, w.n_kv_heads, w.n_pairs, w.n_vch
+    rng = np.random.default_rng(T)
+    sid = rng.integers(0, w.batch, T).astype(np.int32)
+    slot = rng.choice(4096, size=T, replace=False).astype(np.int32)        # distinct rows, so the result is unique
+    pos = np.where(rng.random(T) < 0.5, slot, rng.integers(0, 120000, T)).astype(np.int32)
+    d_sid, d_slot, d_pos = (torch.from_numpy(a).to(st.device) for a in (sid, slot, pos))
+    bias_host = None
+    if with_bias:
+        st.bias, bias_host = [], []
+        for l in range(w.n_layers):
+            b = synth.draw_bias(w, l, st.n_out(l))
+            st.bias.append(torch.from_numpy(b).to(st.device).to(st.dt))
+            bias_host.append(O.round_storage(b, w.dtype))
+    for l in range(w.n_layers):
+        X = synth.draw_hidden(w, l, 5, T)
+        dx = torch.from_numpy(X).to(st.device).to(st.dt).contiguous()
+        q, k, v = O.qkv_rope(O.round_storage(X, w.dtype), w_host[l], None if bias_host is None else bias_host[l], pos,
+                             tabs["inv_freq"][l], Hq, Hkv, P, dv)
+        results = []
+        for variant, rounds in ((0, 2), (1, 1)):        # fused (twice), then the two-stage form
+            st.ctx.rap_set_proj_variant(variant)
+            for _ in range(rounds):
+                st.k_cache[l].fill_(-77.0)
+                st.v_cache[l].fill_(-77.0)
+                dq = torch.full((T, Hq, 2 * P), float("nan"), dtype=st.dt, device=st.device)
+                n0 = st.ctx.rap_kernel_launch_count()
+                st.qkv_rope_append(l, dx, d_sid, d_pos, d_slot, int(slot.max()), q_out=dq)
+                torch.cuda.synchronize()
+                assert st.ctx.rap_kernel_launch_count() - n0 == (1 if variant == 0 else 2)
+                assert st.ctx.rap_get_last_device_status() == (0, 0)
+                Kd, Vd = util.to_np64(st.k_cache[l]), util.to_np64(st.v_cache[l])
+                written = np.zeros(Kd.shape[:3], dtype=bool)
+                written[sid, :, slot] = True
+                assert np.all(Kd[~written] == -77.0) and np.all(Vd[~written] == -77.0)
+                k_dev, v_dev = Kd[sid, :, slot, :], Vd[sid, :, slot, :]
+                util.check_projection(util.to_np64(dq), O.round_storage(q, w.dtype), w.dtype, f"q layer {l}")
+                util.check_projection(k_dev, O.round_storage(k, w.dtype), w.dtype, f"k layer {l}")
+                util.check_projection(v_dev, O.round_storage(v, w.dtype), w.dtype, f"v layer {l}")
+                results.append((util.to_np64(dq), k_dev, v_dev))
+        for a, b in zip(results[0], results[1]):
+            assert np.array_equal(a, b)                  # the same call twice: bit-identical
+        for a, b in zip(results[0], results[2]):         # the two forms differ by the rounding order of one product
+            assert np.abs(a - b).max() <= 2.0 ** -7 * max(1e-30, np.abs(b).max())
+        assert np.array_equal(results[0][2], results[2][2])          # V rows take no rotation: identical
+    st.ctx.rap_set_proj_variant(0)
+    st.close()
+
+
+def test_fused_projection_skips_and_reports_an_out_of_range_row():
+    w = synth.scaled_down(synth.LLAMA_8B, n_layers=1, batch=2, seq=64, hidden=256)
+    st, tabs, w_host = util.build_small_stack(w, *synth.draw_scores(w), full_weights=False, s_cap=72, max_rows=8)
+    x = torch.ones((3, w.hidden), dtype=st.dt, device=st.device)
+    sid = torch.tensor([0, 1, 5], dtype=torch.int32, device=st.device)      # the third row names a sequence that is not there
+    pos = torch.tensor([3, 4, 5], dtype=torch.int32, device=st.device)
+    st.k_cache[0].fill_(5.0)
+    st.v_cache[0].fill_(5.0)
+    n0 = st.ctx.rap_kernel_launch_count()
+    st.qkv_rope_append(0, x, sid, pos, pos, 5)
+    torch.cuda.synchronize()
+    assert st.ctx.rap_kernel_launch_count() - n0 == 1
+    assert st.ctx.rap_get_last_device_status() == (binding.RAP_ECAPACITY, 2)
+    changed = (st.k_cache[0] != 5.0).any(dim=-1).cpu().numpy()
+    expect = np.zeros_like(changed)
+    expect[0, :, 3] = expect[1, :, 4] = True
+    assert np.array_equal(changed, expect)
+    st.close()
