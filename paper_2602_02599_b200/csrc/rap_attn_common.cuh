@@ -46,6 +46,56 @@ __device__ __forceinline__ SkPlan sk_plan(const int32_t* seq_len, int B, int Hkv
   }
   return pl;
 }
+// The same plan, computed once per CTA by its first warp instead of by every thread: the inclusive prefix of the
+// tiles of sequences 0..b (all KV heads) goes to `pref` (shared memory, room for `cap` ints, B <= cap - 2 or the
+// function returns false and leaves everything to sk_plan), the total and the longest sequence to its last two
+// slots.  Every thread of the CTA must call it; pref[0..B) stays valid until the caller reuses the memory.
+__device__ __forceinline__ bool sk_plan_shared(const int32_t* seq_len, int B, int Hkv, int len_add, int S_cap, int tile_rows,
+                                               int grid, int* pref, int cap, SkPlan* out) {
+  if (B > cap - 2) return false;
+  const int tid = threadIdx.x, lane = tid & 31;
+  if (tid < 32) {
+    int carry = 0, n_max = 0;
+    for (int base = 0; base < B; base += 32) {
+      const int bb = base + lane;
+      const int n = bb < B ? sk_tiles_of(seq_len, bb, len_add, S_cap, tile_rows) : 0;
+      n_max = max(n_max, n);
+      int x = n * Hkv;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int y = __shfl_up_sync(0xffffffffu, x, o);
+        if (lane >= o) x += y;
+      }
+      if (bb < B) pref[bb] = carry + x;
+      carry += __shfl_sync(0xffffffffu, x, 31);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) n_max = max(n_max, __shfl_xor_sync(0xffffffffu, n_max, o));
+    if (lane == 0) {
+      pref[cap - 2] = carry;
+      pref[cap - 1] = n_max;
+    }
+  }
+  __syncthreads();
+  const long long T = pref[cap - 2];
+  const int n_max = pref[cap - 1];
+  out->T = (int)T;
+  out->nc = 0;
+  if (T > 0) {
+    const long long lim = (long long)(RAP_MAX_SPLIT - 2) * T / n_max;
+    out->nc = (int)max(1LL, min(min((long long)grid, lim), T));
+  }
+  return true;
+}
+// sequence that holds global tile `cur` (< total), given the inclusive prefix: smallest b with pref[b] > cur
+__device__ __forceinline__ int sk_seq_of(const int* pref, int B, int cur) {
+  int lo = 0, hi = B - 1;
+  while (lo < hi) {
+    const int mid = (lo + hi) >> 1;
+    if (pref[mid] > cur) hi = mid; else lo = mid + 1;
+  }
+  return lo;
+}
 // first CTA whose range holds global tile s:  max c with floor(c T / NC) <= s
 __device__ __forceinline__ int sk_cta_of(int s, const SkPlan& pl) { return (int)((((long long)s + 1) * pl.nc - 1) / pl.T); }
 

@@ -151,7 +151,12 @@ __global__ void __launch_bounds__(MmaCfg<G, WK, DV>::THREADS, 2) attn_mma_kernel
   plan.T = 0; plan.nc = 0;
   int cur = 0, hi = 0, unit_start = 0;
   if (p.balanced) {
-    plan = sk_plan(p.seq_len, p.B, p.Hkv, p.len_add, p.S_cap, ST, (int)gridDim.x);   // reads the lengths only
+    // the plan (reads the lengths only): computed by the first warp into the reduction buffer, which is free until
+    // the first merge; batches too large for that buffer are planned by every thread on its own
+    int* pref = reinterpret_cast<int*>(red);
+    const bool shared_plan = sk_plan_shared(p.seq_len, p.B, p.Hkv, p.len_add, p.S_cap, ST, (int)gridDim.x, pref,
+                                            C::RED_BYTES / 4, &plan);
+    if (!shared_plan) plan = sk_plan(p.seq_len, p.B, p.Hkv, p.len_add, p.S_cap, ST, (int)gridDim.x);
     // Everything below reads q~ and the cache rows the previous kernel in the stream wrote, and writes what the next
     // one may depend on: wait for the predecessor first, and only then let the successor start (it may begin to
     // stream its weights while this scan runs, and waits for this kernel before it writes anything this one reads).
@@ -159,19 +164,27 @@ __global__ void __launch_bounds__(MmaCfg<G, WK, DV>::THREADS, 2) attn_mma_kernel
     pdl_launch_dependents();
     if (blockIdx.x == 0) {   // sequences without any row are scanned by nobody: their output is zero
       for (int i = tid; i < p.B * p.Hkv; i += THREADS) p.unit_cnt_other[i] = 0;   // counters a launch that gave up left behind
-      for (int bb = 0; bb < p.B; ++bb)
-        if (sk_tiles_of(p.seq_len, bb, p.len_add, p.S_cap, ST) == 0)
+      for (int bb = 0; bb < p.B; ++bb) {
+        const bool empty = shared_plan ? pref[bb] == (bb > 0 ? pref[bb - 1] : 0)
+                                       : sk_tiles_of(p.seq_len, bb, p.len_add, p.S_cap, ST) == 0;
+        if (empty)
           for (int i = tid; i < p.Hq * DV; i += THREADS) p.out[(size_t)bb * p.Hq * DV + i] = 0.f;
+      }
     }
     if ((int)blockIdx.x >= plan.nc) return;
     cur = (int)((long long)blockIdx.x * plan.T / plan.nc);
     hi = (int)((long long)(blockIdx.x + 1) * plan.T / plan.nc);
     if (cur >= hi) return;
     int pb = 0;
-    for (b = 0; b < p.B; ++b) {   // the unit that holds tile `cur`
-      const int nb = sk_tiles_of(p.seq_len, b, p.len_add, p.S_cap, ST) * p.Hkv;
-      if (cur < pb + nb) break;
-      pb += nb;
+    if (shared_plan) {       // the unit that holds tile `cur`
+      b = sk_seq_of(pref, p.B, cur);
+      pb = b > 0 ? pref[b - 1] : 0;
+    } else {
+      for (b = 0; b < p.B; ++b) {
+        const int nb = sk_tiles_of(p.seq_len, b, p.len_add, p.S_cap, ST) * p.Hkv;
+        if (cur < pb + nb) break;
+        pb += nb;
+      }
     }
     const int ntb = sk_tiles_of(p.seq_len, b, p.len_add, p.S_cap, ST);
     h = (cur - pb) / ntb;

@@ -276,7 +276,17 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
       int row_w = 0;                           // K / V: row width in elements
       float2* cs_w = nullptr;                  // [16][32] (cos, sin): entry [j][l] belongs to token j + 16 (l & 1) of lane l's pair
       float* vs_w = nullptr;                   // [32][32] summed results, token-major
+      float bias = 0.f;
+      int my_row = -1;                         // lane t: cache row of token t over all sequences, for head 0; -1 = skip the row
+      bool bad_row = false;                    // lane t: token t names a sequence or a slot that is not there
       if constexpr (FUSED) {
+        if (n < p.n_out && f.bias) bias = __bfloat162float(f.bias[n]);
+        if (lane < p.T) {
+          const int sq = f.seq_id ? f.seq_id[lane] : lane;
+          const int sl = f.slot ? f.slot[lane] : f.pos[lane];
+          if (sq >= 0 && sq < f.B_cache && sl >= 0 && sl < f.S_cap) my_row = sq * f.Hkv * f.S_cap + sl;   // fits: checked on the host
+          else bad_row = true;
+        }
         unsigned char* fw = smem + C::OFF_FUSED + quarter * C::FUSED_WARP_BYTES;
         cs_w = reinterpret_cast<float2*>(fw);
         vs_w = reinterpret_cast<float*>(fw + 16 * 32 * 8);
@@ -356,36 +366,34 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             tc_pdl_wait();                       // the previous kernel in the stream may still read q~
             const size_t split_stride = (size_t)p.T * p.n_out;
             const bool in_range = n < p.n_out;
-            // sum the splits: a split at a time, its (up to) 32 loads independent of one another
+            // sum the splits.  Every batch of loads is one round trip through a memory system that other CTAs are
+            // still saturating (microseconds, not hundreds of nanoseconds), so a batch covers all tokens and four
+            // splits: 128 independent loads for the usual split counts
             {
               float v[32];
-              const float bias = (in_range && f.bias) ? __bfloat162float(f.bias[n]) : 0.f;
 #pragma unroll
-              for (int t = 0; t < 32; ++t) v[t] = bias;
+              for (int t = 0; t < 32; ++t) v[t] = 0.f;
 #pragma unroll 1
-              for (int s2 = 0; s2 < f.ksplit; ++s2) {
-                const float* src = p.y + s2 * split_stride + n;
-                float part[32];
+              for (int s0 = 0; s0 < f.ksplit; s0 += 4) {
+                float part[4][32];
 #pragma unroll
-                for (int t = 0; t < 32; ++t) part[t] = (t < p.T && in_range) ? __ldcg(src + (size_t)t * p.n_out) : 0.f;
+                for (int u = 0; u < 4; ++u) {
+                  const float* src = p.y + (size_t)(s0 + u) * split_stride + n;
+                  const bool on = s0 + u < f.ksplit && in_range;
 #pragma unroll
-                for (int t = 0; t < 32; ++t) v[t] += part[t];
+                  for (int t = 0; t < 32; ++t) part[u][t] = (on && t < p.T) ? __ldcg(src + (size_t)t * p.n_out) : 0.f;
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+#pragma unroll
+                  for (int t = 0; t < 32; ++t) v[t] += part[u][t];
               }
 #pragma unroll
-              for (int t = 0; t < 32; ++t) vs_w[t * 32 + lane] = v[t];
+              for (int t = 0; t < 32; ++t) vs_w[t * 32 + lane] = v[t] + bias;     // splits in order, then the bias
             }
-            // where the row of token `lane` goes: its cache row index over all sequences and heads of head 0, or -1
-            int my_row = -1;
-            if (lane < p.T) {
-              const int ps = f.pos[lane];
-              const int sq = f.seq_id ? f.seq_id[lane] : lane;
-              const int sl = f.slot ? f.slot[lane] : ps;
-              if (sq >= 0 && sq < f.B_cache && sl >= 0 && sl < f.S_cap) {
-                my_row = sq * f.Hkv * f.S_cap + sl;      // the host checked that B_cache * H_kv * S_cap fits
-              } else if (n0 == 0 && quarter == 0) {      // reported once per launch: by the warp that owns weight row 0
-                atomicCAS(&p.status[0], 0, (int)RAP_ECAPACITY);
-                p.status[1] = lane;
-              }
+            if (bad_row && n0 == 0 && quarter == 0) {    // reported once per launch: by the warp that owns weight row 0
+              atomicCAS(&p.status[0], 0, (int)RAP_ECAPACITY);
+              p.status[1] = lane;
             }
             __syncwarp();
             const size_t q_stride = (size_t)f.Hq * f.P2;
