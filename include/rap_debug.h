@@ -37,6 +37,15 @@ rap_status rap_set_attn_variant(rap_ctx* ctx, int32_t variant);
  * the epilogue kernel).  Meant for tests, which check the two forms against each other and against the oracle. */
 rap_status rap_set_proj_variant(rap_ctx* ctx, int32_t variant);
 
+/* Makes one bounded device-side wait run out, without faulting or hanging anything: the next launch of the
+ * tensor-core scan of rap_decode_attn (head shapes staged by plain bulk copies) has the first warp of its first CTA
+ * arm one stage barrier without issuing the copy for it, and polls stage barriers a few thousand times instead of
+ * millions.  That warp gives up, its CTA records RAP_ETIMEOUT in the device status word, waits (bounded) for its
+ * other copies and returns; every other CTA finishes normally.  The units that CTA touched stay unfinished (their
+ * outputs are not written).  Later launches run normally: each launch clears the arrival counters its predecessor
+ * used, so nothing has to be reset by hand.  The hook disarms itself when it is used. */
+rap_status rap_debug_arm_wait_timeout(rap_ctx* ctx);
+
 #ifdef __cplusplus
 }
 #endif

@@ -26,7 +26,7 @@ EXPORTS = [
     "rap_get_last_device_status", "rap_kernel_launch_count", "rap_set_attn_variant",
     "rap_decode_attn_noalloc", "rap_profile_attn", "rap_profile_attn_read",
     "rap_pack_wo", "rap_out_proj", "rap_budget_alloc", "rap_prefill_attn", "rap_build_tables_hybrid",
-    "rap_build_tables_partial", "rap_build_tables_freq", "rap_set_proj_variant",
+    "rap_build_tables_partial", "rap_build_tables_freq", "rap_set_proj_variant", "rap_debug_arm_wait_timeout",
 ]
 
 
@@ -82,6 +82,7 @@ def _lib():
     lib.rap_kernel_launch_count.restype = c_int64
     lib.rap_set_attn_variant.argtypes = [P, c_int32]
     lib.rap_set_proj_variant.argtypes = [P, c_int32]
+    lib.rap_debug_arm_wait_timeout.argtypes = [P]
     lib.rap_budget_alloc.argtypes = [c_int32, c_int32, c_int32, P, c_double, P, P]
     lib.rap_prefill_attn.argtypes = [P, c_int32, c_int32, c_int32, P, P, P, c_int32, P, c_int32, P, P]
     lib.rap_pack_wo.argtypes = [P, c_int32, P, P, P, P]
@@ -305,6 +306,9 @@ class RapContext:
         ms, n = ctypes.c_float(), c_int32()
         self._check(_lib().rap_profile_attn_read(self._ctx, byref(ms), byref(n)), "rap_profile_attn_read")
         return ms.value, n.value
+
+    def rap_debug_arm_wait_timeout(self):
+        self._check(_lib().rap_debug_arm_wait_timeout(self._ctx), "rap_debug_arm_wait_timeout")
 
     def rap_set_proj_variant(self, variant):
         self._check(_lib().rap_set_proj_variant(self._ctx, variant), "rap_set_proj_variant")

@@ -69,6 +69,12 @@ rap_status rap_set_attn_variant(rap_ctx* ctx, int32_t variant) {
   return RAP_OK;
 }
 
+rap_status rap_debug_arm_wait_timeout(rap_ctx* ctx) {
+  if (!ctx) return RAP_EINVAL;
+  ctx->dbg_arm_timeout = 1;
+  return RAP_OK;
+}
+
 rap_status rap_set_proj_variant(rap_ctx* ctx, int32_t variant) {
   if (!ctx || variant < 0 || variant > 1) return RAP_EINVAL;
   ctx->proj_variant = variant;

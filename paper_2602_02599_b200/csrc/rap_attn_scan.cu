@@ -61,7 +61,7 @@ __global__ void __launch_bounds__(128) attn_scan_combine_kernel(const float* __r
 }  // namespace
 
 static rap_status launch_split_kv(rap_ctx* ctx, const rap_attn_args& a, int n_split_req, cudaStream_t st,
-                                  const rap_scan_entry* e) {
+                                  const rap_scan_entry* e, bool is_mma) {
   // n_split = 0: balanced mode, one CTA per resident slot; an explicit n_split keeps equal ranges per split
   const bool balanced = n_split_req <= 0 && (long long)a.B * a.Hkv * ((a.S_cap + 63) / 64) < (1LL << 31);
   int n_split = balanced ? RAP_MAX_SPLIT : n_split_req;
@@ -82,6 +82,15 @@ static rap_status launch_split_kv(rap_ctx* ctx, const rap_attn_args& a, int n_sp
     p.unit_cnt_other = ctx->d_unit_cnt + (set ^ 1u) * n_units;
   }
   p.out = a.out;
+  p.wait_limit = WAIT_LIMIT;
+  p.dbg_skip_copy = 0;
+  if (ctx->dbg_arm_timeout && !e->tma && is_mma) {
+    // test hook (rap_debug_arm_wait_timeout): one stage of this launch is armed without a copy and polled a few
+    // thousand times only, so the launch reports RAP_ETIMEOUT and leaves its units unfinished
+    p.wait_limit = 4096;
+    p.dbg_skip_copy = 1;
+    ctx->dbg_arm_timeout = 0;
+  }
   RAP_CUDA_TRY(ctx, rap_raise_smem(ctx, e->fn, e->smem));
   const int scan_grid = 2 * ctx->sm_count;
   dim3 grid(n_split, a.Hkv, a.B);
@@ -120,11 +129,11 @@ static rap_status launch_split_kv(rap_ctx* ctx, const rap_attn_args& a, int n_sp
 rap_status rap_launch_attn_scan(rap_ctx* ctx, const rap_attn_args& a, int n_split_req, cudaStream_t st) {
   if (a.dtype != RAP_BF16 || (a.P2 & 1)) return RAP_EUNSUPPORTED;
   const rap_scan_entry* e = rap_scan_find(a.Hq / a.Hkv, a.P2 / 2, a.dv);
-  return e ? launch_split_kv(ctx, a, n_split_req, st, e) : RAP_EUNSUPPORTED;
+  return e ? launch_split_kv(ctx, a, n_split_req, st, e, false) : RAP_EUNSUPPORTED;
 }
 
 rap_status rap_launch_attn_mma(rap_ctx* ctx, const rap_attn_args& a, int n_split_req, cudaStream_t st) {
   if (a.dtype != RAP_BF16 || (a.P2 & 1)) return RAP_EUNSUPPORTED;
   const rap_scan_entry* e = rap_mma_find(a.Hq / a.Hkv, a.P2 / 2, a.dv);
-  return e ? launch_split_kv(ctx, a, n_split_req, st, e) : RAP_EUNSUPPORTED;
+  return e ? launch_split_kv(ctx, a, n_split_req, st, e, true) : RAP_EUNSUPPORTED;
 }

@@ -59,6 +59,7 @@ struct rap_ctx {
   std::vector<MapSlot> tmaps;         // encoded tensor maps, reused while (pointer, shape, box) repeat
   size_t tmap_next = 0;
   int32_t attn_variant = 0;
+  int32_t dbg_arm_timeout = 0;    // the next tensor-core scan launch runs into a bounded wait on purpose (rap_debug.h)
   int32_t proj_variant = 0;       // 1: rap_qkv_rope_append always takes the two-stage path (GEMM, then the epilogue kernel)
   int64_t launches = 0;
   std::string cuda_error;
@@ -98,6 +99,8 @@ struct rap_scan_params {
   int32_t* unit_cnt;   // balanced mode: arrivals per (sequence, KV head) unit, zero between calls
   int32_t* unit_cnt_other;   // the set the previous launch used; cleared by this launch (two sets take turns)
   float* out;          // balanced mode: [B][Hq][DV], written by the CTA that completes a unit
+  uint32_t wait_limit; // probes of a stage barrier before a warp gives up (RAP_ETIMEOUT)
+  int dbg_skip_copy;   // test hook: the first warp of the first CTA arms its first stage and issues no copy for it
   int B;               // sequences (used by the balanced mode)
   int balanced;        // 0: grid (n_split, H_kv, B), equal tile ranges per split; 1: grid (CTAs), see SkPlan
 };

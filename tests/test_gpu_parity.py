@@ -770,3 +770,46 @@ def test_fused_projection_skips_and_reports_an_out_of_range_row():
     expect[0, :, 3] = expect[1, :, 4] = True
     assert np.array_equal(changed, expect)
     st.close()
+
+
+def test_bounded_wait_gives_up_reports_and_the_next_launches_recover():
+    """A device-side wait that cannot complete (a stage barrier armed by the test hook without a copy behind it, polled
+    a few thousand times): the launch ends by itself, the status word says RAP_ETIMEOUT, the context stays usable,
+    and the launches after it are right again without any reset from the host -- each launch clears the arrival
+    counters its predecessor used, so the units the timed-out CTA left half counted do not poison later merges."""
+    w = synth.scaled_down(synth.LLAMA_8B, n_layers=1, batch=3, seq=3000)
+    lens = [3000, 1777, 640]
+    st = DecodeStack(w, s_cap=3008)
+    st.build_tables(*synth.draw_scores(w))
+    g = torch.Generator(device=st.device).manual_seed(4)
+    sig = float(np.sqrt(w.hidden) * 0.02)
+    st.k_cache[0].normal_(0, sig, generator=g)
+    st.v_cache[0].normal_(0, sig, generator=g)
+    q = torch.empty((w.batch, w.n_q_heads, 2 * w.n_pairs), dtype=st.dt, device=st.device).normal_(0, sig, generator=g)
+    dl = torch.tensor(lens, dtype=torch.int32, device=st.device)
+    want = O.decode_attn(util.to_np64(q), util.to_np64(st.k_cache[0]), util.to_np64(st.v_cache[0]), lens, w.head_dim)
+    shape = (w.batch, w.n_q_heads, w.n_vch)
+
+    def run():
+        out = st.decode_attn(0, q, dl, max(lens))
+        torch.cuda.synchronize()
+        return util.to_np64(out[: int(np.prod(shape))]).reshape(shape)
+
+    util.check_attn(run(), want, w.dtype)
+    assert st.ctx.rap_get_last_device_status() == (0, 0)
+    st.out.fill_(float("nan"))
+    st.ctx.rap_debug_arm_wait_timeout()
+    got = run()                                   # returns: the wait is bounded
+    assert np.isnan(got[0, : w.group]).all()      # the first unit (sequence 0, KV head 0) was never finished ...
+    finished = ~np.isnan(got).any(axis=-1)
+    assert finished.sum() >= finished.size - 2 * w.group          # ... the CTA touched two units at most
+    util.check_attn(got[finished], want[finished], w.dtype)
+    # no status read, no reset: two more launches (one per counter set) are complete and right
+    for _ in range(2):
+        st.out.fill_(float("nan"))
+        util.check_attn(run(), want, w.dtype)
+    code, detail = st.ctx.rap_get_last_device_status()
+    assert code == binding.RAP_ETIMEOUT
+    assert st.ctx.rap_get_last_device_status() == (0, 0)
+    util.check_attn(run(), want, w.dtype)
+    st.close()
