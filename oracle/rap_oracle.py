@@ -25,6 +25,10 @@ identity R_m^T R_n = R_(n-m); position-shift invariance; E_k E_k^T = I and
 E_k R_t = R_(t,S) E_k (also for a frequency table that is not theta^(-2i/D)); the retained-fraction column of Table 13; the bytes/token row
 of Table 15; brute-force loops on tiny inputs; closed-form softmax cases.
 
+Cache quantisation (quantize_rows and the functions on top of it): a reading of a composition the paper only
+names; pinned by exact rational arithmetic on hand-made rows, the half-step round-trip bound, exact
+power-of-two scale equivariance and closed forms.
+
 Parity unpinned: the paper prints no worked numeric example of an attention output, so
 absolute outputs are pinned only through the identities and closed forms above.
 The low-rank comparator (lowrank_decode_attn) is pinned only against the textbook
@@ -597,6 +601,61 @@ def out_proj(attn_out, wo_tilde):
     """y[t] = W~_o o[t]: attn_out [T][H_q][d_v'] (reduced V coordinates) -> [T][hidden], fp64."""
     o = np.asarray(attn_out, dtype=np.float64)
     return o.reshape(o.shape[0], -1) @ np.asarray(wo_tilde, dtype=np.float64).T
+
+
+# --------------------------------------------------------------------------------------
+# composition with KV-cache quantisation (Introduction and Related Work: pruning the cache width and lowering
+# the bit-width of what is cached are orthogonal; the paper's own composition study uses a plain symmetric
+# round-to-nearest quantiser)
+# --------------------------------------------------------------------------------------
+def quantize_rows(x):
+    """8-bit symmetric round-to-nearest quantisation of cache rows, one scale per row.
+
+    Reading (the paper names the quantiser family, not a cache format): every compact cache row x [W] keeps
+    codes c_i in [-127, 127] and one scale s with x_i ~ c_i * s:
+        s  = bf16( max_i |x_i| / 127 )          the scale is stored in the cache's 16-bit float type
+        c_i = clip( rint( x_i / s ), -127, 127 )  round half to even; an all-zero row has s = 0 and c = 0.
+    The decision is taken in fp32 (x as fp32, both divisions in fp32), the precision the kernels take it in.
+    x [..., W] -> (codes int8 [..., W], scales fp64 [...], holding bf16 values)."""
+    x32 = np.asarray(x, dtype=np.float32)
+    amax = np.max(np.abs(x32), axis=-1)
+    s32 = (amax / np.float32(127.0)).astype(np.float32)
+    s = round_bf16(s32).astype(np.float32)
+    safe = np.where(s > 0, s, np.float32(1.0)).astype(np.float32)
+    c = np.rint((x32 / safe[..., None]).astype(np.float32))
+    c = np.clip(c, -127.0, 127.0)
+    c = np.where((s > 0)[..., None], c, 0.0)
+    return c.astype(np.int8), s.astype(np.float64)
+
+
+def dequantize_rows(codes, scales):
+    """x_i = c_i * s, fp64."""
+    return np.asarray(codes, dtype=np.float64) * np.asarray(scales, dtype=np.float64)[..., None]
+
+
+def append_q8(k_codes, k_scales, v_codes, v_scales, k_new, v_new, seq_id, slot):
+    """Quantised append: rows k_new [T][H_kv][2P], v_new [T][H_kv][d_v'] (after RoPE, before any rounding)
+    are quantised row by row and written to codes [B][H_kv][S_cap][W] / scales [B][H_kv][S_cap]."""
+    for r in range(k_new.shape[0]):
+        c, s = quantize_rows(k_new[r])
+        k_codes[seq_id[r], :, slot[r], :] = c
+        k_scales[seq_id[r], :, slot[r]] = s
+        c, s = quantize_rows(v_new[r])
+        v_codes[seq_id[r], :, slot[r], :] = c
+        v_scales[seq_id[r], :, slot[r]] = s
+
+
+def decode_attn_q8(q, k_codes, k_scales, v_codes, v_scales, seq_len, head_dim):
+    """Eq. 2 on the reduced dims over a quantised cache: the attention of decode_attn on the dequantised rows
+    K_j = c^K_j s^K_j, V_j = c^V_j s^V_j (q is not quantised)."""
+    return decode_attn(q, dequantize_rows(k_codes, k_scales), dequantize_rows(v_codes, v_scales), seq_len, head_dim)
+
+
+def kv_bytes_per_token_q8(n_layers, n_kv_heads, k_width, v_width):
+    """Resident bytes per token of the quantised cache as the library lays it out: per row the codes, then a
+    16-bit scale in the last two bytes of a row padded to a multiple of four bytes."""
+    row = lambda w: (w + 2 + 3) // 4 * 4
+    return n_layers * n_kv_heads * (row(k_width) + row(v_width))
 
 
 # --------------------------------------------------------------------------------------

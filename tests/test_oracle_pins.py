@@ -596,3 +596,113 @@ def test_scaled_frequency_tables_keep_the_pair_identities(pairing):
         wrong[:, :P] = freq[l][:P]
         bad, _, _, _ = O.reduced_attention_from_hidden(m["X"], w, wrong, Hq, Hkv, P, dv, D)
         assert np.abs(bad - ref).max() > 1e-4
+
+
+# ---- composition with KV-cache quantisation -----------------------------------------------------------
+def _bf16_exact(fr):
+    """Nearest bf16 (8 significant bits, ties to even) of a positive Fraction, as a Fraction -- exact arithmetic."""
+    from fractions import Fraction
+    e = 0
+    while fr >= 2 ** (e + 1):
+        e += 1
+    while fr < 2 ** e:
+        e -= 1
+    ulp = Fraction(2) ** (e - 7)
+    n = fr / ulp
+    lo = n.numerator // n.denominator
+    rem = n - lo
+    if rem > Fraction(1, 2) or (rem == Fraction(1, 2) and lo % 2 == 1):
+        lo += 1
+    return lo * ulp
+
+
+def test_quantize_rows_against_exact_rational_arithmetic():
+    """Codes and scale of hand-made rows recomputed with Fractions (no floating point): s = bf16(fp32(amax / 127)),
+    c = round-half-even(x / s) clipped to +-127.  The rows are fp32 numbers, so the Fractions are their exact values;
+    the fp32 divisions of the oracle are checked to land on the same codes, ties and clipping included."""
+    from fractions import Fraction
+    rng = np.random.default_rng(2)
+    rows = [np.array([1.27, -0.635, 0.01, 0.0], dtype=np.float32),
+            np.array([3.0, -3.0, 1.5, 0.75, 0.011811024], dtype=np.float32),
+            np.array([1e-3, -2e-3, 5e-4], dtype=np.float32),
+            rng.normal(0, 1.3, 90).astype(np.float32), rng.normal(0, 40.0, 115).astype(np.float32),
+            np.zeros(7, dtype=np.float32)]
+    for x in rows:
+        codes, s = O.quantize_rows(x)
+        amax = max(abs(Fraction(float(v))) for v in x)
+        if amax == 0:
+            assert s == 0.0 and not codes.any()
+            continue
+        s32 = Fraction(float(np.float32(float(amax)) / np.float32(127.0)))      # one fp32 division: the stated precision
+        s_exact = _bf16_exact(s32)
+        assert Fraction(float(s)) == s_exact
+        for v, c in zip(x, codes):
+            ratio = Fraction(float(v)) / s_exact
+            # the fp32 quotient is the rounding of this exact ratio; away from .5 boundaries the code is fixed by it
+            lo = ratio.numerator // ratio.denominator
+            frac = ratio - lo
+            want = lo + (1 if frac > Fraction(1, 2) else 0)
+            if abs(frac - Fraction(1, 2)) < Fraction(1, 2 ** 12):
+                assert int(c) in (max(-127, min(127, lo)), max(-127, min(127, lo + 1)))
+            else:
+                assert int(c) == max(-127, min(127, want)), (float(v), float(s), int(c), want)
+    # the worked row: amax 1.27 -> s = bf16(0.01) = 0.010009765625 -> 126.88, -63.44, 0.999, 0
+    codes, s = O.quantize_rows(np.array([1.27, -0.635, 0.01, 0.0], dtype=np.float32))
+    assert s == 0.010009765625 and codes.tolist() == [127, -63, 1, 0]
+
+
+def test_quantize_rows_round_trip_scale_equivariance_and_layout():
+    rng = np.random.default_rng(5)
+    x = (rng.normal(0, 1, (4, 3, 50, 90)) * rng.lognormal(0, 2, (4, 3, 50, 1))).astype(np.float32)
+    codes, s = O.quantize_rows(x)
+    assert codes.dtype == np.int8 and codes.shape == x.shape and s.shape == x.shape[:-1]
+    assert np.abs(codes.astype(int)).max() <= 127
+    back = O.dequantize_rows(codes, s)
+    # round to nearest: half a step per element (the largest element may also lose what clipping to 127 takes:
+    # the bf16 scale can sit up to 2^-9 below amax / 127)
+    step = s[..., None]
+    assert np.all(np.abs(back - x) <= 0.5 * step + np.abs(x) * 2.0 ** -8 + 1e-30)
+    assert np.all(np.abs(back - x)[np.abs(codes) < 127] <= (0.5 * step * np.ones_like(x))[np.abs(codes) < 127] * (1 + 1e-6))
+    # every row uses its range: the largest element maps to +-127 or +-126
+    assert np.all(np.abs(codes).max(axis=-1) >= 126)
+    # scaling a row by a power of two scales s by it and leaves the codes alone (all operations are exact then)
+    c2, s2 = O.quantize_rows(x * np.float32(8.0))
+    assert np.array_equal(c2, codes) and np.array_equal(s2, 8.0 * s)
+    # rows are independent: a per-tensor scale would wipe out the small rows
+    small = np.abs(x).max(axis=-1) < 0.05 * np.abs(x).max()
+    assert small.any() and np.all(np.abs(codes[small]).max(axis=-1) >= 126)
+    # the scale is a bf16 number
+    assert np.array_equal(O.round_bf16(s), s)
+    # all elements equal: one code value, +-127 or +-126, and the row comes back within half a step
+    c, sc = O.quantize_rows(np.full((1, 16), -0.3, dtype=np.float32))
+    assert len(set(c.ravel().tolist())) == 1 and c[0, 0] in (-127, -126) and abs(c[0, 0] * sc[0] + 0.3) <= 0.5 * sc[0]
+
+
+def test_quantised_append_and_attention_closed_forms():
+    """append_q8 writes exactly the named rows; decode_attn_q8 is Eq. 2 on c * s: a single cached row returns that
+    row's dequantised V, equal K rows average the dequantised V rows, and the output moves by no more than the
+    quantisation step of V when the cache is quantised (a bound, not a tolerance)."""
+    rng = np.random.default_rng(9)
+    B, Hkv, G, cap, P2, dv, D = 2, 2, 2, 8, 6, 5, 8
+    k8 = np.zeros((B, Hkv, cap, P2), np.int8); ks = np.zeros((B, Hkv, cap))
+    v8 = np.zeros((B, Hkv, cap, dv), np.int8); vs = np.zeros((B, Hkv, cap))
+    k_new = rng.normal(0, 1, (3, Hkv, P2)); v_new = rng.normal(0, 2, (3, Hkv, dv))
+    O.append_q8(k8, ks, v8, vs, k_new, v_new, [0, 1, 0], [0, 0, 1])
+    touched = np.zeros((B, Hkv, cap), bool); touched[0, :, 0] = touched[1, :, 0] = touched[0, :, 1] = True
+    assert not k8[~touched].any() and not vs[~touched].any() and np.all(ks[touched] > 0)
+    assert np.array_equal(k8[0, :, 1], O.quantize_rows(k_new[2])[0]) and np.array_equal(vs[1, :, 0], O.quantize_rows(v_new[1])[1])
+    q = rng.normal(0, 1, (B, Hkv * G, P2))
+    out = O.decode_attn_q8(q, k8, ks, v8, vs, [2, 1], D)
+    Vd = O.dequantize_rows(v8, vs)
+    assert np.allclose(out[1], np.repeat(Vd[1, :, 0], G, axis=0), rtol=0, atol=1e-15)          # one row: its V
+    k8[0, :, 1] = k8[0, :, 0]; ks[0, :, 1] = ks[0, :, 0]                                       # equal K rows: the mean
+    out = O.decode_attn_q8(q, k8, ks, v8, vs, [2, 1], D)
+    assert np.allclose(out[0], np.repeat(0.5 * (Vd[0, :, 0] + Vd[0, :, 1]), G, axis=0), rtol=0, atol=1e-15)
+    # against the unquantised cache with the same K: a convex combination of V rows moves by at most half a V step
+    Kd = O.dequantize_rows(k8, ks)
+    Vfull = np.zeros((B, Hkv, cap, dv)); Vfull[0, :, 0] = v_new[0]; Vfull[0, :, 1] = v_new[2]; Vfull[1, :, 0] = v_new[1]
+    ref = O.decode_attn(q, Kd, Vfull.astype(np.float32), [2, 1], D)
+    assert np.abs(out - ref).max() <= 0.5 * vs.max() * (1 + 2.0 ** -7)
+    # bytes per token of the layout: codes + 16-bit scale, rows padded to four bytes (8B shape, rho = 0.7: 184 B / head)
+    assert O.kv_bytes_per_token_q8(32, 8, 90, 90) == 32 * 8 * (92 + 92)
+    assert O.kv_bytes_per_token_q8(1, 1, 116, 115) == 120 + 120 and O.kv_bytes_per_token_q8(1, 1, 128, 128) == 264
