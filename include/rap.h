@@ -194,6 +194,31 @@ rap_status rap_decode_attn(rap_ctx* ctx, int32_t layer, int32_t B, const void* d
                            const int32_t* d_seq_len, int32_t h_seq_len_max, int32_t n_split,
                            float* d_out, void* stream);
 
+/* ---- composition with 8-bit cache quantisation (Introduction and Related Work: pruning the width of the cache and
+ * lowering the bit-width of what is cached are orthogonal; the appendix on composing RAP with quantisation uses a
+ * plain symmetric round-to-nearest quantiser).  The paper fixes no cache format; the reading taken here: every
+ * compact cache row x of width W (W = 2P for K, d_v' for V) keeps int8 codes c_i in [-127, 127] and one scale
+ *     s = bf16(max_i |x_i| / 127),   c_i = clip(rint(x_i / s), -127, 127),   x_i ~ c_i s
+ * (an all-zero row has s = 0), decided in fp32 with round-half-even.  A quantised row occupies
+ * rap_q8_row_bytes(W) = (W + 2) rounded up to a multiple of 4 bytes: the codes, zero padding, and the bf16 scale
+ * in the last two bytes.  Quantised caches are [B][H_kv][S_cap][row bytes], dense; q~ is not quantised.
+ *   rap_quantize_rows       d_rows [n_rows][W] (dtype_in = RAP_F32 or RAP_BF16) -> d_q8 [n_rows][row bytes]; also the
+ *                           way to convert an existing cache of a layer (n_rows = B * H_kv * S_cap).
+ *   rap_qkv_rope_append_q8  rap_qkv_rope_append with the new K and V rows quantised straight from their fp32 values
+ *                           (no rounding to the storage dtype in between); q~ as in rap_qkv_rope_append.
+ *   rap_decode_attn_q8      rap_decode_attn over quantised caches: Eq. 2 on K_j = c^K_j s^K_j, V_j = c^V_j s^V_j.
+ * Arguments, errors and stream behaviour as for the unquantised calls; head_dim <= 256. */
+size_t rap_q8_row_bytes(int32_t W);
+rap_status rap_quantize_rows(rap_ctx* ctx, int32_t dtype_in, int64_t n_rows, int32_t W, const void* d_rows, void* d_q8,
+                             void* stream);
+rap_status rap_qkv_rope_append_q8(rap_ctx* ctx, int32_t layer, int32_t T, const void* d_x, const void* d_w_qkv,
+                                  const void* d_bias, const int32_t* d_seq_id, const int32_t* d_pos,
+                                  const int32_t* d_slot, int32_t h_slot_max, const double* d_inv_freq, void* d_q_out,
+                                  void* d_k8, void* d_v8, int32_t B_cache, int32_t S_cap, void* stream);
+rap_status rap_decode_attn_q8(rap_ctx* ctx, int32_t layer, int32_t B, const void* d_q, const void* d_k8, const void* d_v8,
+                              int32_t S_cap, const int32_t* d_seq_len, int32_t h_seq_len_max, int32_t n_split,
+                              float* d_out, void* stream);
+
 /* ---- decode attention without any allocation (the paper has no counterpart) --------------
  * Same result as rap_decode_attn, for callers that cannot allocate device memory: code running
  * inside someone else's memory budget (a serving engine that hands out every byte of HBM up

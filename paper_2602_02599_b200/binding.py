@@ -27,6 +27,7 @@ EXPORTS = [
     "rap_decode_attn_noalloc", "rap_profile_attn", "rap_profile_attn_read",
     "rap_pack_wo", "rap_out_proj", "rap_budget_alloc", "rap_prefill_attn", "rap_build_tables_hybrid",
     "rap_build_tables_partial", "rap_build_tables_freq", "rap_set_proj_variant", "rap_debug_arm_wait_timeout",
+    "rap_q8_row_bytes", "rap_quantize_rows", "rap_qkv_rope_append_q8", "rap_decode_attn_q8",
 ]
 
 
@@ -83,6 +84,11 @@ def _lib():
     lib.rap_set_attn_variant.argtypes = [P, c_int32]
     lib.rap_set_proj_variant.argtypes = [P, c_int32]
     lib.rap_debug_arm_wait_timeout.argtypes = [P]
+    lib.rap_q8_row_bytes.argtypes = [c_int32]
+    lib.rap_q8_row_bytes.restype = c_size_t
+    lib.rap_quantize_rows.argtypes = [P, c_int32, c_int64, c_int32, P, P, P]
+    lib.rap_qkv_rope_append_q8.argtypes = lib.rap_qkv_rope_append.argtypes
+    lib.rap_decode_attn_q8.argtypes = lib.rap_decode_attn.argtypes
     lib.rap_budget_alloc.argtypes = [c_int32, c_int32, c_int32, P, c_double, P, P]
     lib.rap_prefill_attn.argtypes = [P, c_int32, c_int32, c_int32, P, P, P, c_int32, P, c_int32, P, P]
     lib.rap_pack_wo.argtypes = [P, c_int32, P, P, P, P]
@@ -138,6 +144,10 @@ def rap_budget_alloc(k_pair_scores, rho, head_dim):
     if s:
         raise RapError(s, "rap_budget_alloc")
     return n_pairs, n_vch
+
+
+def rap_q8_row_bytes(W):
+    return int(_lib().rap_q8_row_bytes(W))
 
 
 def rap_cache_elem_offset(n_kv_heads, S_cap, W, b, h, pos, c):
@@ -254,6 +264,22 @@ class RapContext:
         self._check(_lib().rap_decode_attn(self._ctx, layer, B, _ptr(d_q), _ptr(d_k_cache), _ptr(d_v_cache), S_cap,
                                            _ptr(d_seq_len), h_seq_len_max, n_split, _ptr(d_out), _stream()),
                     "rap_decode_attn")
+
+    def rap_quantize_rows(self, dtype_in, n_rows, W, d_rows, d_q8):
+        self._check(_lib().rap_quantize_rows(self._ctx, dtype_in, n_rows, W, _ptr(d_rows), _ptr(d_q8), _stream()),
+                    "rap_quantize_rows")
+
+    def rap_qkv_rope_append_q8(self, layer, T, d_x, d_w_qkv, d_bias, d_seq_id, d_pos, d_slot, h_slot_max, d_inv_freq,
+                               d_q_out, d_k8, d_v8, B_cache, S_cap):
+        self._check(_lib().rap_qkv_rope_append_q8(self._ctx, layer, T, _ptr(d_x), _ptr(d_w_qkv), _ptr(d_bias),
+                                                  _ptr(d_seq_id), _ptr(d_pos), _ptr(d_slot), h_slot_max,
+                                                  _ptr(d_inv_freq), _ptr(d_q_out), _ptr(d_k8), _ptr(d_v8), B_cache,
+                                                  S_cap, _stream()), "rap_qkv_rope_append_q8")
+
+    def rap_decode_attn_q8(self, layer, B, d_q, d_k8, d_v8, S_cap, d_seq_len, h_seq_len_max, n_split, d_out):
+        self._check(_lib().rap_decode_attn_q8(self._ctx, layer, B, _ptr(d_q), _ptr(d_k8), _ptr(d_v8), S_cap,
+                                              _ptr(d_seq_len), h_seq_len_max, n_split, _ptr(d_out), _stream()),
+                    "rap_decode_attn_q8")
 
     def rap_decode_step(self, B, d_x, w_qkv, bias, d_inv_freq, k_cache, v_cache, S_cap, d_seq_len,
                         h_seq_len_max, n_split, d_q_scratch, d_out, out_layer_stride, advance):

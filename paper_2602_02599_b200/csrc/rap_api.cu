@@ -436,6 +436,68 @@ rap_status rap_decode_attn(rap_ctx* ctx, int32_t layer, int32_t B, const void* d
   return rap_launch_attn(ctx, a, (cudaStream_t)stream);
 }
 
+size_t rap_q8_row_bytes(int32_t W) { return W < 1 ? 0 : ((size_t)W + 2 + 3) / 4 * 4; }
+
+rap_status rap_quantize_rows(rap_ctx* ctx, int32_t dtype_in, int64_t n_rows, int32_t W, const void* d_rows, void* d_q8,
+                             void* stream) {
+  if (!ctx || !d_rows || !d_q8) return RAP_EINVAL;
+  if ((dtype_in != RAP_F32 && dtype_in != RAP_BF16) || n_rows < 0 || W < 1 || W > 65535) return RAP_EINVAL;
+  if (!rap_aligned16(d_rows) || !rap_aligned16(d_q8)) return RAP_EALIGN;
+  if (n_rows == 0) return RAP_OK;
+  if ((n_rows + 7) / 8 > 0x7fffffffLL) return RAP_ESHAPE;
+  return rap_launch_quantize_rows(ctx, dtype_in, n_rows, W, d_rows, d_q8, (cudaStream_t)stream);
+}
+
+rap_status rap_qkv_rope_append_q8(rap_ctx* ctx, int32_t layer, int32_t T, const void* d_x, const void* d_w_qkv,
+                                  const void* d_bias, const int32_t* d_seq_id, const int32_t* d_pos, const int32_t* d_slot,
+                                  int32_t h_slot_max, const double* d_inv_freq, void* d_q_out, void* d_k8, void* d_v8,
+                                  int32_t B_cache, int32_t S_cap, void* stream) {
+  if (!ctx || !d_x || !d_w_qkv || !d_seq_id || !d_pos || !d_slot || !d_inv_freq || !d_q_out || !d_k8 || !d_v8)
+    return RAP_EINVAL;
+  if (!ctx->tables_built) return RAP_ESTATE;
+  const rap_model_desc& d = ctx->desc;
+  if (layer < 0 || layer >= d.n_layers || T < 0 || B_cache < 1 || S_cap < 1) return RAP_EINVAL;
+  if (T > d.max_rows) return RAP_ESHAPE;
+  if (S_cap % 8) return RAP_EALIGN;
+  if (h_slot_max < 0) return RAP_EINVAL;
+  if (h_slot_max >= S_cap) return RAP_ECAPACITY;
+  if (d.head_dim > 256) return RAP_EUNSUPPORTED;
+  if (!rap_aligned16(d_x) || !rap_aligned16(d_w_qkv) || !rap_aligned16(d_q_out) || !rap_aligned16(d_k8) ||
+      !rap_aligned16(d_v8) || !rap_aligned16(d_inv_freq) || (d_bias && !rap_aligned16(d_bias)))
+    return RAP_EALIGN;
+  if (T == 0) return RAP_OK;
+  rap_proj_args a;
+  a.x = d_x; a.w = d_w_qkv; a.bias = d_bias;
+  a.seq_id = d_seq_id; a.pos = d_pos; a.slot = d_slot;
+  a.inv_freq = d_inv_freq + (size_t)layer * d.n_kv_heads * (d.head_dim / 2);
+  a.q_out = d_q_out; a.k_cache = d_k8; a.v_cache = d_v8;
+  a.T = T; a.hidden = d.hidden; a.Hq = d.n_q_heads; a.Hkv = d.n_kv_heads;
+  a.P2 = 2 * ctx->n_pairs[layer]; a.dv = ctx->n_vch[layer]; a.half_dim = d.head_dim / 2;
+  a.B_cache = B_cache; a.S_cap = S_cap; a.dtype = d.dtype;
+  return rap_launch_qkv_rope_append_q8(ctx, a, (cudaStream_t)stream);
+}
+
+rap_status rap_decode_attn_q8(rap_ctx* ctx, int32_t layer, int32_t B, const void* d_q, const void* d_k8, const void* d_v8,
+                              int32_t S_cap, const int32_t* d_seq_len, int32_t h_seq_len_max, int32_t n_split, float* d_out,
+                              void* stream) {
+  if (!ctx || !d_q || !d_k8 || !d_v8 || !d_seq_len || !d_out) return RAP_EINVAL;
+  if (!ctx->tables_built) return RAP_ESTATE;
+  const rap_model_desc& d = ctx->desc;
+  if (layer < 0 || layer >= d.n_layers || B < 0 || S_cap < 1 || n_split < 0 || h_seq_len_max < 0) return RAP_EINVAL;
+  if (B > d.max_batch || n_split > RAP_MAX_SPLIT) return RAP_ESHAPE;
+  if (S_cap % 8) return RAP_EALIGN;
+  if (h_seq_len_max > S_cap) return RAP_ECAPACITY;
+  if (!rap_aligned16(d_q) || !rap_aligned16(d_k8) || !rap_aligned16(d_v8) || !rap_aligned16(d_out) || !rap_aligned16(d_seq_len))
+    return RAP_EALIGN;
+  if (B == 0) return RAP_OK;
+  rap_attn_args a;
+  a.q = d_q; a.k = d_k8; a.v = d_v8; a.seq_len = d_seq_len; a.len_add = 0;
+  a.B = B; a.Hq = d.n_q_heads; a.Hkv = d.n_kv_heads; a.P2 = 2 * ctx->n_pairs[layer]; a.dv = ctx->n_vch[layer];
+  a.S_cap = S_cap; a.head_dim = d.head_dim; a.dtype = d.dtype; a.n_split = n_split; a.h_len_max = h_seq_len_max;
+  a.out = d_out;
+  return rap_launch_attn_q8(ctx, a, (cudaStream_t)stream);
+}
+
 rap_status rap_prefill_attn(rap_ctx* ctx, int32_t layer, int32_t B, int32_t T, const void* d_q, const void* d_k_cache,
                             const void* d_v_cache, int32_t S_cap, const int32_t* d_start, int32_t h_start_max,
                             float* d_out, void* stream) {

@@ -156,3 +156,9 @@ rap_status rap_launch_prefill_attn(rap_ctx* ctx, int B, int T, const void* q, co
 rap_status rap_launch_pack_wo(rap_ctx* ctx, int32_t layer, const void* wo, const int32_t* v_idx, void* dst, cudaStream_t st);
 rap_status rap_launch_out_proj(rap_ctx* ctx, int32_t layer, int32_t T, const float* attn_out, const void* wo_tilde,
                                void* y, cudaStream_t st);
+
+// 8-bit cache quantisation (rap_q8.cu, rap_attn_q8.cu)
+rap_status rap_launch_quantize_rows(rap_ctx* ctx, int32_t dtype_in, long long n_rows, int W, const void* src, void* dst,
+                                    cudaStream_t st);
+rap_status rap_launch_qkv_rope_append_q8(rap_ctx* ctx, const rap_proj_args& a, cudaStream_t st);
+rap_status rap_launch_attn_q8(rap_ctx* ctx, const rap_attn_args& a, cudaStream_t st);

@@ -273,6 +273,12 @@ rap_status rap_launch_qkv_rope_append(rap_ctx* ctx, const rap_proj_args& a, cuda
   return a.dtype == RAP_F32 ? run_epilogue<float>(ctx, a, ksplit, st) : run_epilogue<__nv_bfloat16>(ctx, a, ksplit, st);
 }
 
+// Y[T][n_out] (fp32, context workspace, one split) with the CUDA-core GEMM: any dtype and shape.
+rap_status rap_launch_proj_generic(rap_ctx* ctx, const rap_proj_args& a, cudaStream_t st) {
+  const int n_out = (a.Hq + a.Hkv) * a.P2 + a.Hkv * a.dv;
+  return a.dtype == RAP_F32 ? run_generic<float>(ctx, a, n_out, st) : run_generic<__nv_bfloat16>(ctx, a, n_out, st);
+}
+
 rap_status rap_launch_pack(rap_ctx* ctx, int32_t layer, const void* wq, const void* wk, const void* wv,
                            const int32_t* k_dim_idx, const int32_t* v_idx, void* w_qkv, const void* bq,
                            const void* bk, const void* bv, void* bias, cudaStream_t st) {
