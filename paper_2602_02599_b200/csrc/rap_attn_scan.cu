@@ -137,3 +137,10 @@ rap_status rap_launch_attn_mma(rap_ctx* ctx, const rap_attn_args& a, int n_split
   const rap_scan_entry* e = rap_mma_find(a.Hq / a.Hkv, a.P2 / 2, a.dv);
   return e ? launch_split_kv(ctx, a, n_split_req, st, e, true) : RAP_EUNSUPPORTED;
 }
+
+// a.k / a.v are quantised caches (rap_q8.cu); same plan, workspace and merge as the other two scans
+rap_status rap_launch_attn_q8_mma(rap_ctx* ctx, const rap_attn_args& a, int n_split_req, cudaStream_t st) {
+  if (a.dtype != RAP_BF16 || (a.P2 & 1)) return RAP_EUNSUPPORTED;
+  const rap_scan_entry* e = rap_q8_find(a.Hq / a.Hkv, a.P2 / 2, a.dv);
+  return e ? launch_split_kv(ctx, a, n_split_req, st, e, false) : RAP_EUNSUPPORTED;
+}

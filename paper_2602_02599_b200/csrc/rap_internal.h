@@ -115,6 +115,7 @@ struct rap_scan_entry {
 // the FP32-pipe scan (rap_attn_scan_kernel.cuh) and the mma.sync scan (rap_attn_mma_kernel.cuh)
 const rap_scan_entry* rap_scan_find(int G, int WK, int DV);
 const rap_scan_entry* rap_mma_find(int G, int WK, int DV);
+const rap_scan_entry* rap_q8_find(int G, int WK, int DV);      // the scan over an 8-bit quantised cache (rap_attn_q8_kernel.cuh)
 // Tensor map over a row-major [rows][cols] bf16 matrix, boxes of box_rows x 64 elements, 128-byte swizzle,
 // zero fill outside; cached in the context by (pointer, shape, box).  map128 receives the 128-byte CUtensorMap.
 bool rap_tensor_map_bf16(rap_ctx* ctx, void* map128, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows);
