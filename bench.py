@@ -307,6 +307,7 @@ def run_ours(args):
         torch.cuda.empty_cache()
         line["other_workloads"] = other_workloads(torch, min(K, 10), peak)
         line["sweep"] = sweep_rows(torch, min(K, 10), 3, peak)
+        line["quantised_cache"] = q8_rows(torch, min(K, 10), 3, peak)
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
@@ -490,6 +491,65 @@ def sweep_rows(torch, steps, warmup, peak):
                      "lowrank_bound_vs_dense": low_bound_ms / dense_ms, "lowrank_frac_of_its_bound": low_bound_ms / low_ms})
         st.close()
         del st, q, qf, bk, out
+        torch.cuda.empty_cache()
+    return rows
+
+
+def q8_rows(torch, steps, warmup, peak):
+    """Composition with 8-bit cache quantisation: rap_decode_attn_q8 against rap_decode_attn on the shaped workloads
+    (full batch and context, two layers resident and alternated so that the caches are larger than L2).  The
+    quantised caches are made from the same synthetic bf16 rows by rap_quantize_rows.  Algorithmic bytes of the
+    quantised scan: B * H_kv * len * (row bytes of K + row bytes of V), scales and padding included."""
+    from dataclasses import replace
+    from paper_2602_02599_b200 import binding
+    from paper_2602_02599_b200.stack import DecodeStack
+    rows = []
+    for name in ("3b", "8b", "14b"):
+        w = replace(synth.CONFIGS[name], n_layers=2)
+        st = DecodeStack(w)
+        st.build_tables(*synth.draw_scores(w))
+        g = torch.Generator(device=st.device).manual_seed(w.seed)
+        sigma = float(np.sqrt(w.hidden) * 0.02)
+        kb, vb = binding.rap_q8_row_bytes(2 * w.n_pairs), binding.rap_q8_row_bytes(w.n_vch)
+        n_rows = w.batch * w.n_kv_heads * st.s_cap
+        k8, v8 = [], []
+        for l in range(2):
+            st.k_cache[l].normal_(0.0, sigma, generator=g)
+            st.v_cache[l].normal_(0.0, sigma, generator=g)
+            k8.append(torch.empty((n_rows, kb), dtype=torch.uint8, device=st.device))
+            v8.append(torch.empty((n_rows, vb), dtype=torch.uint8, device=st.device))
+            st.ctx.rap_quantize_rows(binding.RAP_BF16, n_rows, 2 * w.n_pairs, st.k_cache[l], k8[l])
+            st.ctx.rap_quantize_rows(binding.RAP_BF16, n_rows, w.n_vch, st.v_cache[l], v8[l])
+        n = w.seq + 1
+        q = torch.empty((w.batch, w.n_q_heads, 2 * w.n_pairs), dtype=st.dt, device=st.device).normal_(0, sigma, generator=g)
+        dl = torch.full((w.batch,), n, dtype=torch.int32, device=st.device)
+        out = torch.empty((w.batch, w.n_q_heads, w.n_vch), dtype=torch.float32, device=st.device)
+
+        def timed(fn):
+            for i in range(warmup):
+                fn(i & 1)
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for i in range(steps):
+                fn(i & 1)
+            e1.record()
+            torch.cuda.synchronize()
+            return e0.elapsed_time(e1) / steps
+
+        ms16 = timed(lambda l: st.decode_attn(l, q, dl, n))
+        ms8 = timed(lambda l: st.ctx.rap_decode_attn_q8(l, w.batch, q, k8[l], v8[l], st.s_cap, dl, n, 0, out))
+        code, detail = st.ctx.rap_get_last_device_status()
+        assert code == 0, (code, detail)
+        by16 = attn_bytes(w, n)
+        by8 = w.batch * w.n_kv_heads * n * (kb + vb)
+        dense = w.batch * w.n_kv_heads * n * 2 * w.head_dim * w.elem_bytes
+        rows.append({"workload": workload_string(w), "bf16_attn_ms": ms16, "q8_attn_ms": ms8, "q8_speedup": ms16 / ms8,
+                     "q8_bytes_per_layer": by8, "q8_bytes_vs_bf16": by8 / by16, "q8_bytes_vs_unpruned_bf16": by8 / dense,
+                     "q8_GBps": by8 / ms8 / 1e6, "q8_frac": by8 / ms8 / 1e6 / peak, "q8_frac_of_nominal_8000": by8 / ms8 / 1e6 / 8000.0,
+                     "steps": steps, "warmup": warmup})
+        st.close()
+        del st, k8, v8, q, out
         torch.cuda.empty_cache()
     return rows
 

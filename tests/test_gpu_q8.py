@@ -184,3 +184,47 @@ def test_q8_attention_head_shape_without_specialised_scan_and_fp32():
     w = replace(synth.TINY, batch=2, seq=200)
     _random_q8_case(w, [200, 77], 0, seed=2)
     _random_q8_case(w, [200, 77], 3, seed=3)
+
+
+@pytest.mark.parametrize("name", ["8b", "3b", "14b"])
+def test_q8_full_size_sampled_units(name):
+    """rap_decode_attn_q8 at the workloads' full batch and context, in the launch configuration the benchmark times
+    (balanced split, one layer resident): sampled (sequence, KV head) units recomputed by the oracle from that unit's
+    codes and scales, ragged lengths included."""
+    w = replace(synth.CONFIGS[name], n_layers=1)
+    st = DecodeStack(w)
+    st.build_tables(*synth.draw_scores(w))
+    g = torch.Generator(device=st.device).manual_seed(w.seed)
+    sig = float(np.sqrt(w.hidden) * 0.02)
+    st.k_cache[0].normal_(0, sig, generator=g)
+    st.v_cache[0].normal_(0, sig, generator=g)
+    B, Hq, Hkv, G, P2, dv = w.batch, w.n_q_heads, w.n_kv_heads, w.group, 2 * w.n_pairs, w.n_vch
+    kb, vb = binding.rap_q8_row_bytes(P2), binding.rap_q8_row_bytes(dv)
+    n_rows = B * Hkv * st.s_cap
+    k8 = torch.empty((B, Hkv, st.s_cap, kb), dtype=torch.uint8, device=st.device)
+    v8 = torch.empty((B, Hkv, st.s_cap, vb), dtype=torch.uint8, device=st.device)
+    st.ctx.rap_quantize_rows(binding.RAP_BF16, n_rows, P2, st.k_cache[0], k8)
+    st.ctx.rap_quantize_rows(binding.RAP_BF16, n_rows, dv, st.v_cache[0], v8)
+    st.k_cache[0] = st.v_cache[0] = None          # the bf16 rows are no longer needed
+    torch.cuda.empty_cache()
+    q = torch.empty((B, Hq, P2), dtype=st.dt, device=st.device).normal_(0, sig, generator=g)
+    out = torch.empty((B, Hq, dv), dtype=torch.float32, device=st.device)
+    rng = np.random.default_rng(3)
+    for lens in (np.full(B, w.seq + 1, dtype=np.int32), synth.ragged_lengths(w) + 1):
+        dl = torch.from_numpy(lens.astype(np.int32)).to(st.device)
+        out.fill_(float("nan"))
+        st.ctx.rap_decode_attn_q8(0, B, q, k8, v8, st.s_cap, dl, int(lens.max()), 0, out)
+        torch.cuda.synchronize()
+        assert st.ctx.rap_get_last_device_status() == (0, 0)
+        assert not torch.isnan(out).any()
+        units = {(0, 0), (B - 1, Hkv - 1), (0, Hkv - 1), (B - 1, 0)}
+        while len(units) < 8:
+            units.add((int(rng.integers(B)), int(rng.integers(Hkv))))
+        for b, h in sorted(units):
+            n = int(lens[b])
+            kc, ks = util.unpack_q8(k8[b, h, :n], P2)
+            vc, vs = util.unpack_q8(v8[b, h, :n], dv)
+            want = O.decode_attn_q8(util.to_np64(q[b, h * G:(h + 1) * G])[None], kc[None, None], ks[None, None], vc[None, None],
+                                    vs[None, None], [n], w.head_dim)[0]
+            util.check_attn(util.to_np64(out[b, h * G:(h + 1) * G]), want, w.dtype)
+    st.close()
