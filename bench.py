@@ -495,7 +495,7 @@ def sweep_rows(torch, steps, warmup, peak):
     return rows
 
 
-def q8_rows(torch, steps, warmup, peak):
+def q8_rows(torch, steps, warmup, peak, names=("3b", "8b", "14b"), batch=0):
     """Composition with 8-bit cache quantisation: rap_decode_attn_q8 against rap_decode_attn on the shaped workloads
     (full batch and context, two layers resident and alternated so that the caches are larger than L2).  The
     quantised caches are made from the same synthetic bf16 rows by rap_quantize_rows.  Algorithmic bytes of the
@@ -504,8 +504,10 @@ def q8_rows(torch, steps, warmup, peak):
     from paper_2602_02599_b200 import binding
     from paper_2602_02599_b200.stack import DecodeStack
     rows = []
-    for name in ("3b", "8b", "14b"):
+    for name in names:
         w = replace(synth.CONFIGS[name], n_layers=2)
+        if batch:
+            w = replace(w, batch=batch, name=w.name + "-cut")
         st = DecodeStack(w)
         st.build_tables(*synth.draw_scores(w))
         g = torch.Generator(device=st.device).manual_seed(w.seed)
@@ -552,6 +554,18 @@ def q8_rows(torch, steps, warmup, peak):
         del st, k8, v8, q, out
         torch.cuda.empty_cache()
     return rows
+
+
+def run_q8(args):
+    """--q8: the quantised-cache rows alone (optionally one workload, optionally a cut batch for profiler runs)."""
+    import torch
+    torch.cuda.set_device(0)
+    peak, _ = load_peaks()
+    names = (args.workload,) if args.workload in ("3b", "14b") or args.batch else ("3b", "8b", "14b")
+    rows = q8_rows(torch, args.steps, args.warmup, peak, names=names, batch=args.batch)
+    print(json.dumps({"metric": "quantised_cache_attention", "unit": "ms", "n_gpus": 1, "steps": args.steps,
+                      "warmup": args.warmup, "dtype": "int8 codes, fp16 MMA, fp32 accumulate", "data": "synthetic",
+                      "higher_is_better": False, "quantised_cache": rows}), flush=True)
 
 
 def run_sweep(args):
@@ -651,6 +665,7 @@ def main():
     ap.add_argument("--prefill", action="store_true", help="time rap_prefill_attn on the sweep's head shapes")
     ap.add_argument("--prefill-case", default="", help="B:T[,B:T...] for --prefill")
     ap.add_argument("--sweep", action="store_true", help="retain-ratio sweep with the dense and low-rank comparators")
+    ap.add_argument("--q8", action="store_true", help="rap_decode_attn_q8 against rap_decode_attn on the shaped workloads")
     ap.add_argument("--no-extras", dest="extras", action="store_false",
                     help="headline measurement only (skip the other workloads, the sweep and the FP32-pipe scan)")
     args = ap.parse_args()
@@ -662,6 +677,8 @@ def main():
         args.cpu_baseline = False
     if args.impl == "reference":
         run_reference(args)
+    elif args.q8:
+        run_q8(args)
     elif args.sweep:
         run_sweep(args)
     elif args.prefill:

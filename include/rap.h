@@ -200,8 +200,9 @@ rap_status rap_decode_attn(rap_ctx* ctx, int32_t layer, int32_t B, const void* d
  * compact cache row x of width W (W = 2P for K, d_v' for V) keeps int8 codes c_i in [-127, 127] and one scale
  *     s = bf16(max_i |x_i| / 127),   c_i = clip(rint(x_i / s), -127, 127),   x_i ~ c_i s
  * (an all-zero row has s = 0), decided in fp32 with round-half-even.  A quantised row occupies
- * rap_q8_row_bytes(W) = (W + 2) rounded up to a multiple of 4 bytes: the codes, zero padding, and the bf16 scale
- * in the last two bytes.  Quantised caches are [B][H_kv][S_cap][row bytes], dense; q~ is not quantised.
+ * rap_q8_row_bytes(W) = (W + 2) rounded up to a multiple of 4 bytes: the codes, each stored as the unsigned byte
+ * c_i + 128, then zero padding, and the bf16 scale in the last two bytes.  Quantised caches are
+ * [B][H_kv][S_cap][row bytes], dense; q~ is not quantised.
  *   rap_quantize_rows       d_rows [n_rows][W] (dtype_in = RAP_F32 or RAP_BF16) -> d_q8 [n_rows][row bytes]; also the
  *                           way to convert an existing cache of a layer (n_rows = B * H_kv * S_cap).
  *   rap_qkv_rope_append_q8  rap_qkv_rope_append with the new K and V rows quantised straight from their fp32 values

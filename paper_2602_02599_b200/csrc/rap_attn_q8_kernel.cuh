@@ -3,10 +3,13 @@
 // in the last two bytes of a row of rap_q8_row_bytes(W) bytes).  Same work plan, per-warp copy pipelines, lazy online
 // softmax and fused merge; what changes is how the operands reach the MMAs (mma.sync m16n8k16, fp16 in, fp32
 // accumulate):
-//   * a code byte c (two's complement) becomes the fp16 number 1152 + c with one byte permute and one XOR: flipping
-//     the sign bit gives u = c + 128 in [1, 255], and the bit pattern 0x6400 | u is the fp16 number 1024 + u (fp16
-//     has a step of one between 1024 and 2048), so a 32-bit word of four codes turns into two operand registers
-//     without any integer-to-float conversion.
+//   * a code c is stored as the byte u = c + 128 in [1, 255], and the bit pattern 0x6400 | u is the fp16 number
+//     1024 + u = 1152 + c (fp16 has a step of one between 1024 and 2048): one byte permute turns two stored codes
+//     into one operand register, a 32-bit word of four codes into two, without any integer-to-float conversion.
+//   * which cache rows form an n-tile and which dims of a k-step sit on which MMA k-slot is free as long as both
+//     operands agree: a thread's four k-slots of a step are the four bytes of ONE stored K word (one load per
+//     n-tile and step), and column n of n-tile t is block row 4 n + t, which puts the 32 loads of a warp on 32
+//     banks for rows of an odd number of words (and spreads the V loads of the four row pairs likewise).
 //   * S^T = q K^T: q enters as fp16 (its bf16 values converted once per unit: exact but for values below the fp16
 //     normal range), the K operand as 1152 + c.  The products are exact in fp32; the constant is taken out again on
 //     the accumulators (1152 times the sum of the head's q, known per unit), and the row's K scale is applied to the
@@ -57,8 +60,14 @@ struct Q8Cfg {
   static_assert(SMEM <= SMEM_BUDGET, "ring does not fit");
   static_assert(NW * NSTG * 8 + NW * 64 <= OFF_RED - 16, "barriers and merge scalars sit below the reduction buffer");
   static_assert((K_BYTES % 16) == 0 && (V_BYTES % 16) == 0, "blocks are whole 16-byte units");
-  // row of column n of n-tile t inside the warp's block
-  static __device__ __forceinline__ constexpr int row(int t, int n) { return 8 * t + n; }
+  // row of column n of n-tile t inside the warp's block: 4 n + t (rows 0, 4, .., 28 of a row of an odd number of
+  // words start on banks 0, 28, 24, .., 4)
+  static __device__ __forceinline__ constexpr int row(int t, int n) { return 4 * n + t; }
+  // dims where the last k-step starts when 2P is not a multiple of 16: moved back so that it ends at (or, for a row
+  // of 4 m + 2 code bytes, two bytes past) the end of the codes and starts on a word; what it covers twice, and the
+  // two bytes past the codes, meet zeroed q
+  static constexpr int LAST_BASE = ((2 * WK) % 4 == 2) ? 2 * WK - 14 : 2 * WK - 16;
+  static constexpr bool LAST_SHIFTED = (2 * WK) % 16 != 0;
 };
 
 __device__ __forceinline__ void q8_mma_f16(float (&c)[4], uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1) {
@@ -90,7 +99,6 @@ __device__ __forceinline__ uint32_t q8_hsub2(uint32_t a, uint32_t b) {
 }
 __device__ __forceinline__ float q8_bf16_bits(uint32_t h) { return __uint_as_float(h << 16); }
 constexpr uint32_t Q8_EXP = 0x64646464u;        // high byte of the fp16 numbers 1024 .. 1279
-constexpr uint32_t Q8_SIGN = 0x80808080u;       // code byte -> code + 128
 constexpr uint32_t Q8_1152 = 0x64806480u;       // fp16 pair (1152, 1152)
 
 template <int G, int WK, int DV>
@@ -172,17 +180,12 @@ __global__ void __launch_bounds__(Q8Cfg<G, WK, DV>::THREADS, 2) attn_q8_kernel(c
   }
   __syncthreads();
 
-  // fragment addressing inside a block.  K: this thread supplies column gid of every n-tile, i.e. block row
-  // 8 t + gid, and of a k-step the dims base + 2 tq, + 1 and base + 8 + 2 tq, + 1: two bytes of one stored word each.
-  // base = 16 ks, or 2P - 16 for the last step of a row that is not a multiple of 16 dims (shifted back; its overlap
-  // meets zeroed q), so the in-word offset of the byte pair is a per-thread constant for either kind of step.
-  constexpr int LAST_BASE = 2 * WK - 16;                    // dims where the last k-step starts
-  const int kbyte_reg = 2 * tq, kbyte_last = LAST_BASE + 2 * tq;
-  const uint32_t ksel_reg = (kbyte_reg & 2) ? 0x4342u : 0x4140u;     // bytes (2, 3) or (0, 1) of the word, each under 0x64
-  const uint32_t ksel_last = (kbyte_last & 2) ? 0x4342u : 0x4140u;
-  const int krow = gid * KSW;                               // + 8 t KSW for n-tile t
-  // V: this thread's rows of a 16-row step are 2 tq, 2 tq + 1 (+ 8), its word of a 32-channel group is gid
-  const int vrow = 2 * tq * VSW + gid;
+  // fragment addressing inside a block.  K: this thread supplies column gid of every n-tile (block row 4 gid + t)
+  // and, of a k-step that starts at byte `base` of the row, the word base / 4 + tq: its bytes 0, 1 are the k-slots
+  // 2 tq, 2 tq + 1, its bytes 2, 3 the k-slots 2 tq + 8, 2 tq + 9.
+  const int krow = 4 * gid * KSW + tq;                      // + t KSW for n-tile t, + base / 4 for the step
+  // V: the k-slots 2 tq, 2 tq + 1 of n-tile t are block rows 8 tq + t and 8 tq + 4 + t; word gid of a 32-channel group
+  const int vrow = 8 * tq * VSW + gid;
   int st = 0;                  // ring position and phase of this warp, running on across units
   uint32_t parity = 0;
   bool timed_out = false;
@@ -239,20 +242,22 @@ __global__ void __launch_bounds__(Q8Cfg<G, WK, DV>::THREADS, 2) attn_q8_kernel(c
       for (int i = 0; i < pre; ++i) issue_block(i, (st + i) % NSTG);
     }
 
-    // ---- q as the A operand (fp16): head gid, dims base + 2 tq, + 1 and base + 8 + 2 tq, + 1 of every k-step; zero
-    // for the padding heads and for the dims an earlier step covered.  off_q = 1152 * (sum of the head's q): what
-    // the constant in the K operand adds to every raw logit of this head.
+    // ---- q as the A operand (fp16): head gid; of the step that starts at dim `base` the dims base + 4 tq, + 1 (k-slots
+    // 2 tq, 2 tq + 1) and base + 4 tq + 2, + 3 (k-slots 2 tq + 8, 2 tq + 9); zero for the padding heads, for dims an
+    // earlier step covered and for dims past the row.  off_q = 1152 * (sum of the head's q): what the constant in
+    // the K operand adds to every raw logit of this head.
     uint32_t qa[NKS][2];
     float off_q = 0.f;
     {
       const uint32_t* qrow = p.q + ((size_t)b * p.Hq + (size_t)h * G + (gid < G ? gid : 0)) * WK;
 #pragma unroll
       for (int ks = 0; ks < NKS; ++ks) {
-        const int wb = ks < NKS - 1 ? 8 * ks : WK - 8;        // first bf16 pair (word) of the step
+        const bool shifted = C::LAST_SHIFTED && ks == NKS - 1;
+        const int wb = (shifted ? C::LAST_BASE : 16 * ks) / 2;     // first bf16 pair (word of q) of the step
 #pragma unroll
         for (int hlf = 0; hlf < 2; ++hlf) {
-          const int w = wb + 4 * hlf + tq;
-          const bool fresh = w >= 8 * ks;                      // not covered by an earlier step
+          const int w = wb + 2 * tq + hlf;
+          const bool fresh = w >= 8 * ks && w < WK;             // not covered by an earlier step, inside the row
           const uint32_t bits = (gid < G && fresh) ? qrow[w] : 0u;
           qa[ks][hlf] = q8_pack_f16(__uint_as_float(bits << 16), __uint_as_float(bits & 0xffff0000u));
           const __half2 hq = *reinterpret_cast<const __half2*>(&qa[ks][hlf]);
@@ -289,25 +294,21 @@ __global__ void __launch_bounds__(Q8Cfg<G, WK, DV>::THREADS, 2) attn_q8_kernel(c
       for (int t = 0; t < 4; ++t) s[t][0] = s[t][1] = s[t][2] = s[t][3] = 0.f;
 #pragma unroll
       for (int ks = 0; ks < NKS; ++ks) {
-        const bool last = (ks == NKS - 1) && (LAST_BASE != 16 * (NKS - 1));
-        const int kbyte = last ? kbyte_last : 16 * ks + kbyte_reg;
-        const uint32_t sel = last ? ksel_last : ksel_reg;
-        const int w0 = kbyte >> 2;                   // word of dims base + 2 tq, + 1; the dims 8 further on are 2 words on
+        const int w0 = ((C::LAST_SHIFTED && ks == NKS - 1) ? C::LAST_BASE : 16 * ks) / 4;
 #pragma unroll
         for (int t = 0; t < 4; ++t) {
-          const uint32_t x0 = kw[krow + 8 * t * KSW + w0] ^ Q8_SIGN;
-          const uint32_t x1 = kw[krow + 8 * t * KSW + w0 + 2] ^ Q8_SIGN;
-          q8_mma_f16(s[t], qa[ks][0], qa[ks][1], q8_prmt(x0, Q8_EXP, sel), q8_prmt(x1, Q8_EXP, sel));
+          const uint32_t x = kw[krow + t * KSW + w0];
+          q8_mma_f16(s[t], qa[ks][0], qa[ks][1], q8_prmt(x, Q8_EXP, 0x4140u), q8_prmt(x, Q8_EXP, 0x4342u));
         }
       }
 
-      // ---- scales of this thread's rows 8 t + 2 tq + e (bf16 in the last two bytes of a row) ----
+      // ---- scales of this thread's rows 4 (2 tq + e) + t (bf16 in the last two bytes of a row) ----
       float ksc[4][2], vsc[4][2];
 #pragma unroll
       for (int t = 0; t < 4; ++t)
 #pragma unroll
         for (int e = 0; e < 2; ++e) {
-          const int r = 8 * t + 2 * tq + e;
+          const int r = C::row(t, 2 * tq + e);
           const bool valid = r < nrows;
           const uint32_t kb16 = *reinterpret_cast<const uint16_t*>(stage + r * C::KS + C::KS - 2);
           const uint32_t vb16 = *reinterpret_cast<const uint16_t*>(stage + C::K_BYTES + r * C::VS + C::VS - 2);
@@ -324,7 +325,7 @@ __global__ void __launch_bounds__(Q8Cfg<G, WK, DV>::THREADS, 2) attn_q8_kernel(c
         for (int e = 0; e < 2; ++e) {
           s[t][e] = (s[t][e] - off_q) * ksc[t][e];                     // the logit in base-2 units
           x[t][e] = s[t][e] - m_ref;
-          if (nrows < MMA_BR && 8 * t + 2 * tq + e >= nrows) x[t][e] = -INFINITY;
+          if (nrows < MMA_BR && C::row(t, 2 * tq + e) >= nrows) x[t][e] = -INFINITY;
           raise |= x[t][e] > Q8_LAZY_SLACK;
         }
       if (__any_sync(0xffffffffu, raise)) {
@@ -333,7 +334,7 @@ __global__ void __launch_bounds__(Q8Cfg<G, WK, DV>::THREADS, 2) attn_q8_kernel(c
         for (int t = 0; t < 4; ++t)
 #pragma unroll
           for (int e = 0; e < 2; ++e) {
-            const bool masked = nrows < MMA_BR && 8 * t + 2 * tq + e >= nrows;
+            const bool masked = nrows < MMA_BR && C::row(t, 2 * tq + e) >= nrows;
             x[t][e] = masked ? -INFINITY : s[t][e];
             mx = fmaxf(mx, x[t][e]);
           }
@@ -366,12 +367,13 @@ __global__ void __launch_bounds__(Q8Cfg<G, WK, DV>::THREADS, 2) attn_q8_kernel(c
       // ---- O += P V: two steps of 16 rows (n-tiles 2 kb, 2 kb + 1), NCG groups of 32 channels ----
 #pragma unroll
       for (int kb = 0; kb < 2; ++kb) {
-        const uint32_t* v0 = vw + vrow + 16 * kb * VSW;          // row 16 kb + 2 tq; + VSW: the next row; + 8 VSW: 8 rows on
+        // rows of this thread's k-slots: n-tile 2 kb -> 8 tq + 2 kb and 8 tq + 4 + 2 kb, n-tile 2 kb + 1 -> one row further
+        const uint32_t* v0 = vw + vrow + 2 * kb * VSW;
 #pragma unroll
         for (int cg = 0; cg < NCG; ++cg) {
-          const uint32_t xa = v0[8 * cg] ^ Q8_SIGN, xb = v0[8 * cg + VSW] ^ Q8_SIGN;
-          const uint32_t xc = v0[8 * cg + 8 * VSW] ^ Q8_SIGN, xd = v0[8 * cg + 9 * VSW] ^ Q8_SIGN;
-          // channel pairs (0, 1) and (2, 3) of the word, each as (row, next row)
+          const uint32_t xa = v0[8 * cg], xb = v0[8 * cg + 4 * VSW];
+          const uint32_t xc = v0[8 * cg + VSW], xd = v0[8 * cg + 5 * VSW];
+          // channel pairs (0, 1) and (2, 3) of the word, each as (first row, second row) of the k-slot pair
           const uint32_t g01 = q8_prmt(xa, xb, 0x5140u), g23 = q8_prmt(xa, xb, 0x7362u);
           const uint32_t h01 = q8_prmt(xc, xd, 0x5140u), h23 = q8_prmt(xc, xd, 0x7362u);
 #pragma unroll

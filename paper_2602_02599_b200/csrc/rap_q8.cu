@@ -4,7 +4,9 @@
 //     s = bf16(max|x| / 127),   c_i = clip(rint(x_i / s), -127, 127),   x_i ~ c_i s,
 // decided in fp32.  A quantised row of width W occupies rap_q8_row_bytes(W) = (W + 2) rounded up to 4 bytes: the
 // codes, padding, and the bf16 scale in the last two bytes, so a block of rows is one contiguous byte range that
-// carries its scales along.
+// carries its scales along.  A code is stored as the unsigned byte c + 128 (1 .. 255): that byte under the high byte
+// 0x64 is the fp16 number 1152 + c, which is how the tensor-core scan turns codes into MMA operands without a
+// conversion instruction.
 //
 // This file holds the quantiser (rap_quantize_rows), the RoPE / append epilogue that quantises the new K and V rows
 // straight from their fp32 values (rap_qkv_rope_append_q8; the projection GEMM is the one of rap_qkv_rope_append),
@@ -32,11 +34,13 @@ __device__ __forceinline__ float warp_max(float v) {
 }
 // the scale of a row with largest magnitude amax, as stored (a bf16 number) -- fp32 division, one rounding to bf16
 __device__ __forceinline__ float q8_scale(float amax) { return __bfloat162float(__float2bfloat16_rn(__fdiv_rn(amax, 127.0f))); }
-__device__ __forceinline__ signed char q8_code(float x, float s) {
-  if (!(s > 0.f)) return 0;
+// the stored byte of x under scale s: code + 128
+__device__ __forceinline__ unsigned char q8_code(float x, float s) {
+  if (!(s > 0.f)) return 128;
   const float c = rintf(__fdiv_rn(x, s));
-  return (signed char)fminf(fmaxf(c, -127.f), 127.f);
+  return (unsigned char)(128 + (int)fminf(fmaxf(c, -127.f), 127.f));
 }
+__device__ __forceinline__ float q8_value(unsigned char byte) { return (float)((int)byte - 128); }
 // codes are written by the lanes that own them; lane 0 adds the padding and the scale
 __device__ __forceinline__ void q8_finish_row(unsigned char* row, int W, int row_bytes, float s, int lane) {
   if (lane == 0) {
@@ -57,7 +61,7 @@ __global__ void __launch_bounds__(256) quantize_rows_kernel(const T* __restrict_
   for (int i = lane; i < W; i += 32) amax = fmaxf(amax, fabsf(q8_ld(x + i)));
   const float s = q8_scale(warp_max(amax));
   unsigned char* d = dst + row * row_bytes;
-  for (int i = lane; i < W; i += 32) d[i] = (unsigned char)q8_code(q8_ld(x + i), s);
+  for (int i = lane; i < W; i += 32) d[i] = q8_code(q8_ld(x + i), s);
   q8_finish_row(d, W, row_bytes, s, lane);
 }
 
@@ -135,8 +139,8 @@ rope_append_q8_kernel(const float* __restrict__ y, int ksplit, const T* __restri
       for (int k = 0; k < 4; ++k) {
         const int c = lane + 32 * k;
         if (c < P) {
-          d[2 * c] = (unsigned char)q8_code(ra[k], s);
-          d[2 * c + 1] = (unsigned char)q8_code(rb[k], s);
+          d[2 * c] = q8_code(ra[k], s);
+          d[2 * c + 1] = q8_code(rb[k], s);
         }
       }
       q8_finish_row(d, P2, k_row_bytes, s, lane);
@@ -157,7 +161,7 @@ rope_append_q8_kernel(const float* __restrict__ y, int ksplit, const T* __restri
 #pragma unroll
     for (int k = 0; k < 8; ++k) {
       const int c = lane + 32 * k;
-      if (c < dv) d[c] = (unsigned char)q8_code(v[k], s);
+      if (c < dv) d[c] = q8_code(v[k], s);
     }
     q8_finish_row(d, dv, v_row_bytes, s, lane);
   }
@@ -206,7 +210,7 @@ attn_q8_generic_kernel(const T* __restrict__ q, const unsigned char* __restrict_
 #pragma unroll
       for (int g = 0; g < RAP_MAX_GROUP; ++g) part[g] = 0.f;
       for (int d = lane; d < P2; d += 32) {
-        const float kv = (float)(signed char)kr[d];
+        const float kv = q8_value(kr[d]);
 #pragma unroll
         for (int g = 0; g < RAP_MAX_GROUP; ++g)
           if (g < G) part[g] = fmaf(kv, q_s[g * P2 + d], part[g]);
@@ -249,7 +253,7 @@ attn_q8_generic_kernel(const T* __restrict__ q, const unsigned char* __restrict_
       for (int g = 0; g < RAP_MAX_GROUP; ++g)
         if (g < G) acc[g] *= alpha_s[g];
       for (int j = 0; j < nj; ++j) {
-        const float vv = (float)(signed char)vb[(size_t)(j0 + j) * v_row_bytes + tid] * vs_s[j];
+        const float vv = q8_value(vb[(size_t)(j0 + j) * v_row_bytes + tid]) * vs_s[j];
 #pragma unroll
         for (int g = 0; g < RAP_MAX_GROUP; ++g)
           if (g < G) acc[g] = fmaf(s_s[g * Q8G_TILE + j], vv, acc[g]);

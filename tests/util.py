@@ -103,9 +103,9 @@ def prefill_both(st, tabs, w_host, w, lens, step_tag=0, chunk=None):
 
 def unpack_q8(t, W):
     """A quantised cache tensor (uint8 [..., row bytes]) -> (codes int8 [..., W], scales fp64 [...]): the codes come
-    first, the bf16 scale sits in the last two bytes of the row."""
+    first, each stored as code + 128; the bf16 scale sits in the last two bytes of the row."""
     a = t.detach().cpu().numpy()
-    codes = a[..., :W].view(np.int8)
+    codes = (a[..., :W].astype(np.int16) - 128).astype(np.int8)
     bits = a[..., -2].astype(np.uint32) | (a[..., -1].astype(np.uint32) << 8)
     scales = (bits << 16).astype(np.uint32).view(np.float32).astype(np.float64)
     return codes, scales
@@ -115,7 +115,7 @@ def pack_q8(codes, scales, row_bytes):
     """Oracle-side codes and (bf16-valued) scales -> the byte layout of a quantised cache, as a uint8 array."""
     codes = np.asarray(codes, dtype=np.int8)
     out = np.zeros(codes.shape[:-1] + (row_bytes,), dtype=np.uint8)
-    out[..., : codes.shape[-1]] = codes.view(np.uint8)
+    out[..., : codes.shape[-1]] = (codes.astype(np.int16) + 128).astype(np.uint8)
     bits = (np.asarray(scales, dtype=np.float32).view(np.uint32) >> 16).astype(np.uint16)
     out[..., -2] = (bits & 0xFF).astype(np.uint8)
     out[..., -1] = (bits >> 8).astype(np.uint8)
