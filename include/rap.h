@@ -48,7 +48,9 @@ typedef enum {
   RAP_EUNSUPPORTED = 5, /* valid request this build does not implement                  */
   RAP_ECUDA = 6,        /* a CUDA runtime call failed (see rap_last_cuda_error)          */
   RAP_ETIMEOUT = 7,     /* a bounded device-side wait gave up (device status word)      */
-  RAP_ESTATE = 8        /* call order: tables not built yet for this context            */
+  RAP_ESTATE = 8,       /* call order: tables not built yet for this context            */
+  RAP_EBOUNDS = 9       /* only from a library built with RAP_DEBUG_BOUNDS: a kernel's index check failed
+                           (device status word; detail = which check); the access was skipped  */
 } rap_status;
 
 typedef enum { RAP_F32 = 0, RAP_BF16 = 1 } rap_dtype;

@@ -46,6 +46,13 @@ rap_status rap_set_proj_variant(rap_ctx* ctx, int32_t variant);
  * used, so nothing has to be reset by hand.  The hook disarms itself when it is used. */
 rap_status rap_debug_arm_wait_timeout(rap_ctx* ctx);
 
+/* Shows that the index checks of the bounds-checking build (librap_b200_dbg.so, compiled with -DRAP_DEBUG_BOUNDS) are
+ * live, without any access leaving a buffer: the next shape-specialised scan launch is told that the split-KV
+ * workspace holds only n_floats floats (it is as large as ever).  In the bounds-checking build the writes of partials
+ * beyond that claim are skipped and the device status word reports RAP_EBOUNDS; in the normal build, which has no
+ * checks, the call changes nothing.  The hook disarms itself when it is used; 0 switches it off. */
+rap_status rap_debug_claim_scan_workspace(rap_ctx* ctx, int64_t n_floats);
+
 #ifdef __cplusplus
 }
 #endif

@@ -13,9 +13,10 @@ from ctypes import POINTER, byref, c_char_p, c_double, c_int32, c_int64, c_size_
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "librap_b200.so")
+# RAP_LIBRARY selects another build of the same library (the bounds-checking one, librap_b200_dbg.so, in tests)
+LIB_PATH = os.environ.get("RAP_LIBRARY") or os.path.join(_HERE, "librap_b200.so")
 
-RAP_OK, RAP_EINVAL, RAP_ESHAPE, RAP_ECAPACITY, RAP_EALIGN, RAP_EUNSUPPORTED, RAP_ECUDA, RAP_ETIMEOUT, RAP_ESTATE = range(9)
+RAP_OK, RAP_EINVAL, RAP_ESHAPE, RAP_ECAPACITY, RAP_EALIGN, RAP_EUNSUPPORTED, RAP_ECUDA, RAP_ETIMEOUT, RAP_ESTATE, RAP_EBOUNDS = range(10)
 RAP_F32, RAP_BF16 = 0, 1
 RAP_PAIR_HALF, RAP_PAIR_ADJACENT = 0, 1
 
@@ -26,7 +27,7 @@ EXPORTS = [
     "rap_get_last_device_status", "rap_kernel_launch_count", "rap_set_attn_variant",
     "rap_decode_attn_noalloc", "rap_profile_attn", "rap_profile_attn_read",
     "rap_pack_wo", "rap_out_proj", "rap_budget_alloc", "rap_prefill_attn", "rap_build_tables_hybrid",
-    "rap_build_tables_partial", "rap_build_tables_freq", "rap_set_proj_variant", "rap_debug_arm_wait_timeout",
+    "rap_build_tables_partial", "rap_build_tables_freq", "rap_set_proj_variant", "rap_debug_arm_wait_timeout", "rap_debug_claim_scan_workspace",
     "rap_q8_row_bytes", "rap_quantize_rows", "rap_qkv_rope_append_q8", "rap_decode_attn_q8",
 ]
 
@@ -84,6 +85,7 @@ def _lib():
     lib.rap_set_attn_variant.argtypes = [P, c_int32]
     lib.rap_set_proj_variant.argtypes = [P, c_int32]
     lib.rap_debug_arm_wait_timeout.argtypes = [P]
+    lib.rap_debug_claim_scan_workspace.argtypes = [P, c_int64]
     lib.rap_q8_row_bytes.argtypes = [c_int32]
     lib.rap_q8_row_bytes.restype = c_size_t
     lib.rap_quantize_rows.argtypes = [P, c_int32, c_int64, c_int32, P, P, P]
@@ -332,6 +334,9 @@ class RapContext:
         ms, n = ctypes.c_float(), c_int32()
         self._check(_lib().rap_profile_attn_read(self._ctx, byref(ms), byref(n)), "rap_profile_attn_read")
         return ms.value, n.value
+
+    def rap_debug_claim_scan_workspace(self, n_floats):
+        self._check(_lib().rap_debug_claim_scan_workspace(self._ctx, n_floats), "rap_debug_claim_scan_workspace")
 
     def rap_debug_arm_wait_timeout(self):
         self._check(_lib().rap_debug_arm_wait_timeout(self._ctx), "rap_debug_arm_wait_timeout")

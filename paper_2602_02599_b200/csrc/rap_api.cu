@@ -55,6 +55,7 @@ const char* rap_status_string(rap_status s) {
     case RAP_ECUDA: return "RAP_ECUDA: CUDA runtime error";
     case RAP_ETIMEOUT: return "RAP_ETIMEOUT: bounded device wait gave up";
     case RAP_ESTATE: return "RAP_ESTATE: rap_build_tables has not run on this context";
+    case RAP_EBOUNDS: return "RAP_EBOUNDS: an index check of the bounds-checking build failed";
   }
   return "unknown rap_status";
 }
@@ -66,6 +67,12 @@ int64_t rap_kernel_launch_count(const rap_ctx* ctx) { return ctx ? ctx->launches
 rap_status rap_set_attn_variant(rap_ctx* ctx, int32_t variant) {
   if (!ctx || variant < 0 || variant > 4) return RAP_EINVAL;
   ctx->attn_variant = variant;
+  return RAP_OK;
+}
+
+rap_status rap_debug_claim_scan_workspace(rap_ctx* ctx, int64_t n_floats) {
+  if (!ctx || n_floats < 0) return RAP_EINVAL;
+  ctx->dbg_ws_floats = n_floats;
   return RAP_OK;
 }
 

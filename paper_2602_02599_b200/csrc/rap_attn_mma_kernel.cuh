@@ -271,7 +271,8 @@ __global__ void __launch_bounds__(MmaCfg<G, WK, DV>::THREADS, 2) attn_mma_kernel
       const int rows = min(MMA_BR, len8 - j0);
       const uint32_t bar = bar0 + 8 * stg, dst = wstage_u + stg * C::STAGE_BYTES;
       const uint32_t kb = (uint32_t)rows * WK * 4, vb = (uint32_t)rows * DV * 2;
-      if (lane == 0) {
+      if (lane == 0 && RAP_BOUNDS(j0 + rows - 1, p.S_cap, p.status, 0x102) && RAP_BOUNDS(stg, NSTG, p.status, 0x103) &&
+          RAP_BOUNDS(rows - 1, MMA_BR, p.status, 0x104)) {
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // earlier generic writes (zero fill) come first
         if constexpr (C::TMA) {
           // whole boxes: rows past the end of the tensor are zero-filled, rows of a neighbouring unit are masked
@@ -309,7 +310,7 @@ __global__ void __launch_bounds__(MmaCfg<G, WK, DV>::THREADS, 2) attn_mma_kernel
         for (int hlf = 0; hlf < 2; ++hlf) {
           const int w = wb + 4 * hlf + tq;
           const bool fresh = w >= 8 * ks;                      // not covered by an earlier step
-          qa[ks][hlf] = (gid < G && fresh) ? qrow[w] : 0u;
+          qa[ks][hlf] = (gid < G && fresh && RAP_BOUNDS(w, WK, p.status, 0x101)) ? qrow[w] : 0u;
         }
       }
     }
@@ -358,11 +359,12 @@ __global__ void __launch_bounds__(MmaCfg<G, WK, DV>::THREADS, 2) attn_mma_kernel
         for (int t = 0; t < 4; ++t) {
           uint32_t b0, b1;
           if constexpr (C::TMA) {
-            b0 = kw[kx[(2 * ks) % 8] + (ks / 4) * 1024 + 256 * t];
-            b1 = kw[kx[(2 * ks + 1) % 8] + (ks / 4) * 1024 + 256 * t];
+            const int i0 = kx[(2 * ks) % 8] + (ks / 4) * 1024 + 256 * t, i1 = kx[(2 * ks + 1) % 8] + (ks / 4) * 1024 + 256 * t;
+            b0 = RAP_BOUNDS(i0, C::K_BYTES / 4, p.status, 0x105) ? kw[i0] : 0u;
+            b1 = RAP_BOUNDS(i1, C::K_BYTES / 4, p.status, 0x105) ? kw[i1] : 0u;
           } else {
-            b0 = kw[koff[t] + wb];
-            b1 = kw[koff[t] + wb + 4];
+            b0 = RAP_BOUNDS(koff[t] + wb, C::K_BYTES / 4, p.status, 0x106) ? kw[koff[t] + wb] : 0u;
+            b1 = RAP_BOUNDS(koff[t] + wb + 4, C::K_BYTES / 4, p.status, 0x106) ? kw[koff[t] + wb + 4] : 0u;
           }
           mma_bf16(s[t], qa[ks][0], qa[ks][1], b0, b1);
         }
@@ -419,8 +421,18 @@ __global__ void __launch_bounds__(MmaCfg<G, WK, DV>::THREADS, 2) attn_mma_kernel
       }
 
       // ---- O += P V: two k-blocks of 16 rows (n-tiles 2 kb and 2 kb + 1), NCB blocks of 16 channels ----
+      // (bounds-checking build: the fragment offsets do not depend on the data, so their largest value is checked
+      // once per block against the words this stage holds behind the K block)
+      bool v_ok = true;
+      {
+        constexpr int V_WORDS = (C::STAGE_BYTES - C::K_BYTES) / 4;
+        const int cw_last = C::CB_LAST / 2;
+        const int far = C::TMA ? vx[3][1] + ((NCB - 1) / 4) * 1024 + 256 * 3
+                               : max(vofs[1], vofs[3]) + cw_last + VPAIR + (C::VODD ? 1 : 0);
+        v_ok = RAP_BOUNDS(far, V_WORDS, p.status, 0x107);
+      }
 #pragma unroll
-      for (int kb = 0; kb < 2; ++kb) {
+      for (int kb = 0; kb < 2 && v_ok; ++kb) {
         const uint32_t* v0 = vw + vofs[2 * kb];
         const uint32_t* v1 = vw + vofs[2 * kb + 1];
 #pragma unroll
@@ -488,7 +500,7 @@ __global__ void __launch_bounds__(MmaCfg<G, WK, DV>::THREADS, 2) attn_mma_kernel
     for (int w = 0; w < NW; ++w) m_all = fmaxf(m_all, m_s[w * 8 + gid]);
     const float f = m_ref == -INFINITY ? 0.f : mma_ex2(m_ref - m_all);   // a warp without a block contributes nothing
     if (tq == 0) l_s[warp * 8 + gid] = l_thr * f;
-    if (gid < G) {
+    if (gid < G && RAP_BOUNDS(((size_t)warp * G + gid) * CW + CW - 1, C::RED_BYTES / 4, p.status, 0x108)) {
       float* rr = red + ((size_t)warp * G + gid) * CW;
 #pragma unroll
       for (int cb = 0; cb < NCB; ++cb) {
@@ -500,14 +512,15 @@ __global__ void __launch_bounds__(MmaCfg<G, WK, DV>::THREADS, 2) attn_mma_kernel
       }
     }
     __syncthreads();
-    for (int i = tid; i < G * DV; i += THREADS) {
+    const bool ws_ok = RAP_BOUNDS((ws_base - p.ws) + (long long)(G - 1) * ws_head + DV + 1, p.ws_floats, p.status, 0x109);
+    for (int i = tid; i < G * DV && ws_ok; i += THREADS) {
       const int g = i / DV, c = i - g * DV;
       float sum = 0.f;
 #pragma unroll
       for (int w = 0; w < NW; ++w) sum += red[((size_t)w * G + g) * CW + c];
       ws_base[g * ws_head + c] = sum;
     }
-    if (tid < G) {
+    if (tid < G && ws_ok) {
       float l = 0.f, mm = -INFINITY;
 #pragma unroll
       for (int w = 0; w < NW; ++w) {
@@ -524,12 +537,17 @@ __global__ void __launch_bounds__(MmaCfg<G, WK, DV>::THREADS, 2) attn_mma_kernel
       const int first = sk_cta_of(unit_start, plan);
       const int nseg = sk_cta_of(unit_start + seg_tiles - 1, plan) - first + 1;
       const int u = b * p.Hkv + h;
-      if (tid == 0) *s_last = atomicAdd(&p.unit_cnt[u], 1) == nseg - 1;
+      if (tid == 0) *s_last = RAP_BOUNDS(u, p.B * p.Hkv, p.status, 0x10a) && atomicAdd(&p.unit_cnt[u], 1) == nseg - 1;
       __syncthreads();
       if (*s_last) {
         __threadfence();
         const float* ub = p.ws + ((size_t)b * p.Hq + (size_t)h * G) * RAP_MAX_SPLIT * (size_t)(DV + 2);
-        if (nseg <= 4) {
+        const bool m_ok = RAP_BOUNDS((ub - p.ws) + (long long)(G - 1) * ws_head + (long long)(nseg - 1) * (DV + 2) + DV + 1,
+                                     p.ws_floats, p.status, 0x10b) &&
+                          RAP_BOUNDS(((size_t)b * p.Hq + (size_t)h * G + G - 1) * DV + DV - 1, (size_t)p.B * p.Hq * DV, p.status, 0x10c);
+        if (!m_ok) {
+          // (bounds-checking build only) the unit's merge would leave its buffers: skipped and reported
+        } else if (nseg <= 4) {
           // few partials (the usual case): every output thread loads the maxima, the sums and its own channel of all
           // partials at once -- one round trip through the memory system instead of two -- and weighs them itself
           for (int i = tid; i < G * DV; i += THREADS) {

@@ -231,7 +231,8 @@ __global__ void __launch_bounds__(Q8Cfg<G, WK, DV>::THREADS, 2) attn_q8_kernel(c
       const int rows = min(MMA_BR, len8 - j0);
       const uint32_t bar = bar0 + 8 * stg, dst = wstage_u + stg * C::STAGE_BYTES;
       const uint32_t kb = (uint32_t)rows * C::KS, vb = (uint32_t)rows * C::VS;     // multiples of 16: rows is a multiple of 8
-      if (lane == 0) {
+      if (lane == 0 && RAP_BOUNDS(j0 + rows - 1, p.S_cap, p.status, 0x202) && RAP_BOUNDS(stg, NSTG, p.status, 0x203) &&
+          RAP_BOUNDS(rows - 1, MMA_BR, p.status, 0x204)) {
         mbar_expect_tx(bar, kb + vb);
         bulk_g2s(dst, kg + (size_t)j0 * C::KS, kb, bar);
         bulk_g2s(dst + C::K_BYTES, vg + (size_t)j0 * C::VS, vb, bar);
@@ -258,7 +259,7 @@ __global__ void __launch_bounds__(Q8Cfg<G, WK, DV>::THREADS, 2) attn_q8_kernel(c
         for (int hlf = 0; hlf < 2; ++hlf) {
           const int w = wb + 2 * tq + hlf;
           const bool fresh = w >= 8 * ks && w < WK;             // not covered by an earlier step, inside the row
-          const uint32_t bits = (gid < G && fresh) ? qrow[w] : 0u;
+          const uint32_t bits = (gid < G && fresh && RAP_BOUNDS(w, WK, p.status, 0x201)) ? qrow[w] : 0u;
           qa[ks][hlf] = q8_pack_f16(__uint_as_float(bits << 16), __uint_as_float(bits & 0xffff0000u));
           const __half2 hq = *reinterpret_cast<const __half2*>(&qa[ks][hlf]);
           off_q += __low2float(hq) + __high2float(hq);
@@ -297,7 +298,7 @@ __global__ void __launch_bounds__(Q8Cfg<G, WK, DV>::THREADS, 2) attn_q8_kernel(c
         const int w0 = ((C::LAST_SHIFTED && ks == NKS - 1) ? C::LAST_BASE : 16 * ks) / 4;
 #pragma unroll
         for (int t = 0; t < 4; ++t) {
-          const uint32_t x = kw[krow + t * KSW + w0];
+          const uint32_t x = RAP_BOUNDS(krow + t * KSW + w0, C::K_BYTES / 4, p.status, 0x205) ? kw[krow + t * KSW + w0] : 0u;
           q8_mma_f16(s[t], qa[ks][0], qa[ks][1], q8_prmt(x, Q8_EXP, 0x4140u), q8_prmt(x, Q8_EXP, 0x4342u));
         }
       }
@@ -310,8 +311,9 @@ __global__ void __launch_bounds__(Q8Cfg<G, WK, DV>::THREADS, 2) attn_q8_kernel(c
         for (int e = 0; e < 2; ++e) {
           const int r = C::row(t, 2 * tq + e);
           const bool valid = r < nrows;
-          const uint32_t kb16 = *reinterpret_cast<const uint16_t*>(stage + r * C::KS + C::KS - 2);
-          const uint32_t vb16 = *reinterpret_cast<const uint16_t*>(stage + C::K_BYTES + r * C::VS + C::VS - 2);
+          const bool sc_ok = RAP_BOUNDS(r, MMA_BR, p.status, 0x206);
+          const uint32_t kb16 = sc_ok ? *reinterpret_cast<const uint16_t*>(stage + r * C::KS + C::KS - 2) : 0u;
+          const uint32_t vb16 = sc_ok ? *reinterpret_cast<const uint16_t*>(stage + C::K_BYTES + r * C::VS + C::VS - 2) : 0u;
           ksc[t][e] = valid ? q8_bf16_bits(kb16) * cs : 0.f;
           vsc[t][e] = valid ? q8_bf16_bits(vb16) : 0.f;
         }
@@ -365,8 +367,11 @@ __global__ void __launch_bounds__(Q8Cfg<G, WK, DV>::THREADS, 2) attn_q8_kernel(c
       }
 
       // ---- O += P V: two steps of 16 rows (n-tiles 2 kb, 2 kb + 1), NCG groups of 32 channels ----
+      // (bounds-checking build: the word offsets do not depend on the data; the largest one is checked once per block
+      // against the words this stage holds behind the K block)
+      const bool v_ok = RAP_BOUNDS(vrow + (2 + 5) * VSW + 8 * (NCG - 1), (C::STAGE_BYTES - C::K_BYTES) / 4, p.status, 0x207);
 #pragma unroll
-      for (int kb = 0; kb < 2; ++kb) {
+      for (int kb = 0; kb < 2 && v_ok; ++kb) {
         // rows of this thread's k-slots: n-tile 2 kb -> 8 tq + 2 kb and 8 tq + 4 + 2 kb, n-tile 2 kb + 1 -> one row further
         const uint32_t* v0 = vw + vrow + 2 * kb * VSW;
 #pragma unroll
@@ -415,7 +420,7 @@ __global__ void __launch_bounds__(Q8Cfg<G, WK, DV>::THREADS, 2) attn_q8_kernel(c
     for (int w = 0; w < NW; ++w) m_all = fmaxf(m_all, m_s[w * 8 + gid]);
     const float f = m_ref == -INFINITY ? 0.f : q8_ex2(m_ref - m_all);   // a warp without a block contributes nothing
     if (tq == 0) l_s[warp * 8 + gid] = l_thr * f;
-    if (gid < G) {
+    if (gid < G && RAP_BOUNDS(((size_t)warp * G + gid) * CW + CW - 1, C::RED_BYTES / 4, p.status, 0x208)) {
       float* rr = red + ((size_t)warp * G + gid) * CW;
 #pragma unroll
       for (int cg = 0; cg < NCG; ++cg)
@@ -427,14 +432,15 @@ __global__ void __launch_bounds__(Q8Cfg<G, WK, DV>::THREADS, 2) attn_q8_kernel(c
         }
     }
     __syncthreads();
-    for (int i = tid; i < G * DV; i += THREADS) {
+    const bool ws_ok = RAP_BOUNDS((ws_base - p.ws) + (long long)(G - 1) * ws_head + DV + 1, p.ws_floats, p.status, 0x209);
+    for (int i = tid; i < G * DV && ws_ok; i += THREADS) {
       const int g = i / DV, c = i - g * DV;
       float sum = 0.f;
 #pragma unroll
       for (int w = 0; w < NW; ++w) sum += red[((size_t)w * G + g) * CW + c];
       ws_base[g * ws_head + c] = sum;
     }
-    if (tid < G) {
+    if (tid < G && ws_ok) {
       float l = 0.f, mm = -INFINITY;
 #pragma unroll
       for (int w = 0; w < NW; ++w) {
@@ -451,12 +457,17 @@ __global__ void __launch_bounds__(Q8Cfg<G, WK, DV>::THREADS, 2) attn_q8_kernel(c
       const int first = sk_cta_of(unit_start, plan);
       const int nseg = sk_cta_of(unit_start + seg_tiles - 1, plan) - first + 1;
       const int u = b * p.Hkv + h;
-      if (tid == 0) *s_last = atomicAdd(&p.unit_cnt[u], 1) == nseg - 1;
+      if (tid == 0) *s_last = RAP_BOUNDS(u, p.B * p.Hkv, p.status, 0x20a) && atomicAdd(&p.unit_cnt[u], 1) == nseg - 1;
       __syncthreads();
       if (*s_last) {
         __threadfence();
         const float* ub = p.ws + ((size_t)b * p.Hq + (size_t)h * G) * RAP_MAX_SPLIT * (size_t)(DV + 2);
-        if (nseg <= 4) {
+        const bool m_ok = RAP_BOUNDS((ub - p.ws) + (long long)(G - 1) * ws_head + (long long)(nseg - 1) * (DV + 2) + DV + 1,
+                                     p.ws_floats, p.status, 0x20b) &&
+                          RAP_BOUNDS(((size_t)b * p.Hq + (size_t)h * G + G - 1) * DV + DV - 1, (size_t)p.B * p.Hq * DV, p.status, 0x20c);
+        if (!m_ok) {
+          // (bounds-checking build only) the unit's merge would leave its buffers: skipped and reported
+        } else if (nseg <= 4) {
           // few partials (the usual case): every output thread loads the maxima, the sums and its own channel of all
           // partials at once -- one round trip through the memory system instead of two -- and weighs them itself
           for (int i = tid; i < G * DV; i += THREADS) {

@@ -72,6 +72,11 @@ static rap_status launch_split_kv(rap_ctx* ctx, const rap_attn_args& a, int n_sp
   ScanParams p;
   p.q = (const uint32_t*)a.q; p.k = (const unsigned char*)a.k; p.v = (const unsigned char*)a.v;
   p.seq_len = a.seq_len; p.ws = ctx->d_attn_ws; p.status = ctx->d_status;
+  p.ws_floats = (long long)(ctx->attn_ws_bytes / sizeof(float));
+  if (ctx->dbg_ws_floats > 0) {      // test hook: understate the workspace (it is as large as ever), see rap_debug.h
+    p.ws_floats = ctx->dbg_ws_floats;
+    ctx->dbg_ws_floats = 0;
+  }
   p.len_add = a.len_add; p.Hq = a.Hq; p.Hkv = a.Hkv; p.S_cap = a.S_cap; p.n_split = n_split;
   p.qscale = (float)(1.4426950408889634 / sqrt((double)a.head_dim));
   p.B = a.B; p.balanced = balanced ? 1 : 0;

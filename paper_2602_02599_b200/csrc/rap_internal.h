@@ -59,6 +59,7 @@ struct rap_ctx {
   std::vector<MapSlot> tmaps;         // encoded tensor maps, reused while (pointer, shape, box) repeat
   size_t tmap_next = 0;
   int32_t attn_variant = 0;
+  long long dbg_ws_floats = 0;    // > 0: the next scan launch is told its workspace holds only this many floats (rap_debug.h)
   int32_t dbg_arm_timeout = 0;    // the next tensor-core scan launch runs into a bounded wait on purpose (rap_debug.h)
   int32_t proj_variant = 0;       // 1: rap_qkv_rope_append always takes the two-stage path (GEMM, then the epilogue kernel)
   int64_t launches = 0;
@@ -73,6 +74,22 @@ static inline cudaError_t rap_raise_smem(rap_ctx* ctx, F fn, int bytes) {
   if (!ctx->attr_done.insert((const void*)fn).second) return cudaSuccess;
   return cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
 }
+
+// Index checks of the bounds-checking build (-DRAP_DEBUG_BOUNDS, a second library next to the normal one): RAP_BOUNDS(i,
+// n, status, tag) is true when 0 <= i < n; otherwise it records RAP_EBOUNDS with `tag` in the device status word (the
+// first failure wins) and the caller skips the access.  In the normal build it is the constant true and costs nothing.
+#ifdef RAP_DEBUG_BOUNDS
+#ifdef __CUDACC__
+__device__ __forceinline__ bool rap_in_bounds(long long i, long long n, int32_t* status, int tag) {
+  if (i >= 0 && i < n) return true;
+  if (atomicCAS(&status[0], 0, (int)RAP_EBOUNDS) == 0) status[1] = tag;
+  return false;
+}
+#endif
+#define RAP_BOUNDS(i, n, status, tag) rap_in_bounds((long long)(i), (long long)(n), (status), (tag))
+#else
+#define RAP_BOUNDS(i, n, status, tag) true
+#endif
 
 static inline int rap_elem_bytes(int32_t dtype) { return dtype == RAP_F32 ? 4 : 2; }
 static inline bool rap_aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -93,6 +110,7 @@ struct rap_scan_params {
   const unsigned char* v;     // [B][Hkv][S_cap][DV * 2 bytes]
   const int32_t* seq_len;
   float* ws;
+  long long ws_floats; // size of ws (used by the index checks of the bounds-checking build)
   int32_t* status;
   int len_add, Hq, Hkv, S_cap, n_split;
   float qscale;

@@ -379,7 +379,9 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
                   const float* src = p.y + (size_t)(s0 + u) * split_stride + n;
-                  const bool on = s0 + u < f.ksplit && in_range;
+                  const bool on = s0 + u < f.ksplit && in_range &&
+                                  RAP_BOUNDS((size_t)(s0 + u) * split_stride + (size_t)(p.T - 1) * p.n_out + n,
+                                             (size_t)f.ksplit * split_stride, p.status, 0x301);
 #pragma unroll
                   for (int t = 0; t < 32; ++t) part[u][t] = (on && t < p.T) ? __ldcg(src + (size_t)t * p.n_out) : 0.f;
                 }
@@ -400,6 +402,7 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
             const int cs_lane = (lane & ~1);
 #pragma unroll 4
             for (int t = 0; t < p.T; ++t) {
+              if (!RAP_BOUNDS(t, 32, p.status, 0x304)) break;     // (the staging buffers hold 32 tokens)
               const float mine = vs_w[t * 32 + lane], other = vs_w[t * 32 + (lane ^ 1)];
               const float2 cs = cs_w[(t & 15) * 32 + (cs_lane | (t >> 4))];
               const int row = __shfl_sync(0xffffffffu, my_row, t);
@@ -407,8 +410,14 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
               const float rot = (lane & 1) ? fmaf(other, cs.y, mine * cs.x) : fmaf(-other, cs.y, mine * cs.x);
               const __nv_bfloat16 o = __float2bfloat16_rn(kind == 2 ? mine : rot);
               if (in_range) {
-                if (kind == 0) dst[t * q_stride] = o;
-                else if (row >= 0) dst[(size_t)row * row_w] = o;   // a row whose sequence or slot is out of range is skipped
+                if (kind == 0) {
+                  if (RAP_BOUNDS((dst - f.q_out) + (long long)(t * q_stride), (long long)p.T * (long long)q_stride, p.status, 0x302))
+                    dst[t * q_stride] = o;
+                } else if (row >= 0) {                             // a row whose sequence or slot is out of range is skipped
+                  if (RAP_BOUNDS((dst - (kind == 1 ? f.k_cache : f.v_cache)) + (long long)row * row_w,
+                                 (long long)f.B_cache * f.Hkv * f.S_cap * row_w, p.status, 0x303))
+                    dst[(size_t)row * row_w] = o;
+                }
               }
             }
             if (lane == 0) f.cnt[slot_c] = 0;      // ready for the next launch that uses this set

@@ -221,6 +221,7 @@ def _random_attn_case(w, lens, n_split, seed=0, variant=0, q_gain=1.0, ramp=0.0)
                 want[b] = 0.0
         got = util.to_np64(out[: w.batch * w.n_q_heads * dv]).reshape(w.batch, w.n_q_heads, dv)
         util.check_attn(got, want, w.dtype)
+    assert st.ctx.rap_get_last_device_status() == (0, 0)
     st.close()
 
 

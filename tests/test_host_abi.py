@@ -53,7 +53,7 @@ def test_cache_offset_is_dense_row_major(lib):
 
 
 def test_status_strings_and_bad_descriptions(lib):
-    for s in range(9):
+    for s in range(10):
         assert lib.rap_status_string(s).decode().startswith("RAP_")
     good = dict(n_layers=1, hidden=256, n_q_heads=4, n_kv_heads=2, head_dim=64, rope_theta=10000.0, pairing=0,
                 dtype=0, max_batch=1, max_rows=1)
