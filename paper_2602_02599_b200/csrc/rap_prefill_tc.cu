@@ -11,6 +11,10 @@
 //   O_X   += P_X V      tcgen05.mma with A = P in tensor memory (N = d_v' rounded up to 32, K = 64 keys),
 //                       accumulating in TMEM across the key tiles; a warp rescales its 32 accumulator rows
 //                       (tcgen05.ld / st) only in the rare tile where the lazy maximum moved.
+// Where the N of the second MMA has a spare column (d_v' below its multiple of 32: every pruned shape), that column of
+// every staged V tile holds the constant one, so the tensor core accumulates the row sum of the weights next to O --
+// from the very bf16 weights it multiplies, rescaled with O when the maximum moves -- and the softmax threads keep no
+// sum at all (LSUM; a third of their instructions per weight otherwise).
 // While one group runs its softmax the tensor core works for the other, and a staged K / V tile serves 256 queries.
 // Cache rows are not multiples of 16 bytes, so TMA tensor maps cannot describe them: four producer warps (10-11: K,
 // 12-13: V) stage the tiles by hand (4-byte cp.async) into rings of five buffers each, in the 128-byte-swizzled
@@ -100,6 +104,12 @@ __device__ __forceinline__ void pt_ld32_nowait(uint32_t taddr, uint32_t (&r)[32]
       : "r"(taddr)
       : "memory");
 }
+__device__ __forceinline__ uint32_t pt_ld1(uint32_t taddr) {     // one column of this warp's 32 lanes
+  uint32_t r;
+  asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];" : "=r"(r) : "r"(taddr) : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+  return r;
+}
 __device__ __forceinline__ void pt_st32(uint32_t taddr, const uint32_t (&r)[32]) {
   asm volatile(
       "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
@@ -170,7 +180,8 @@ __global__ void __launch_bounds__(256) prefill_repack_v_kernel(const __nv_bfloat
 }
 
 // DK = k-steps of Q K^T (ceil(2P / 16)); NVP = d_v' rounded up to a multiple of 32 (N of the second MMA)
-template <int DK, int NVP>
+// LSUM: column p.vs (< NVP) of every V tile is the constant one and the row sums come out of the second MMA
+template <int DK, int NVP, bool LSUM>
 __global__ void __launch_bounds__(P2_THREADS, 1) prefill_tc_kernel(const PtParams p) {
   extern __shared__ unsigned char pt_raw[];
   unsigned char* smem = pt_raw + ((1024u - (pt_smem(pt_raw) & 1023u)) & 1023u);
@@ -230,6 +241,14 @@ __global__ void __launch_bounds__(P2_THREADS, 1) prefill_tc_kernel(const PtParam
   // zero every tile once (pad columns and pad channel rows are never written again), then stage Q_A and Q_B
   for (int i = tid; i < (P2_SMEM - P2_TAIL) / 16; i += P2_THREADS) reinterpret_cast<uint4*>(smem)[i] = make_uint4(0, 0, 0, 0);
   __syncthreads();
+  if constexpr (LSUM) {
+    // the ones column: channel p.vs of all 64 key rows of every V buffer (the producers never write that element)
+    for (int i = tid; i < P2_STAGES * P2_KT; i += P2_THREADS) {
+      const int buf = i / P2_KT, r = i - buf * P2_KT, c = p.vs;
+      unsigned char* e = v_s + buf * P2_KV_BYTES + r * 128 + pt_swz2(4 * (c >> 1), r & 7) + 2 * (c & 1);
+      *reinterpret_cast<__nv_bfloat16*>(e) = __float2bfloat16(1.0f);
+    }
+  }
   const int kw = p.P2 >> 1;                          // 4-byte words per q / K row
   for (int r = warp; r < 256; r += P2_THREADS / 32) {
     const int t = q0 + r;
@@ -421,9 +440,11 @@ __global__ void __launch_bounds__(P2_THREADS, 1) prefill_tc_kernel(const PtParam
           const float p0 = pt_ex2(x0), p1 = pt_ex2(x1);
           const __nv_bfloat162 v2 = __floats2bfloat162_rn(p0, p1);
           const uint32_t pk = *reinterpret_cast<const uint32_t*>(&v2);
-          // the row sum takes the rounded weights the second MMA will see (a one-hot row comes out exact)
-          asm("mov.b64 %0, {%1, %2};" : "=l"(p2) : "r"(pk << 16), "r"(pk & 0xffff0000u));
-          asm("add.rn.f32x2 %0, %1, %2;" : "=l"(l2[(j >> 1) & 3]) : "l"(l2[(j >> 1) & 3]), "l"(p2));
+          if constexpr (!LSUM) {
+            // the row sum takes the rounded weights the second MMA will see (a one-hot row comes out exact)
+            asm("mov.b64 %0, {%1, %2};" : "=l"(p2) : "r"(pk << 16), "r"(pk & 0xffff0000u));
+            asm("add.rn.f32x2 %0, %1, %2;" : "=l"(l2[(j >> 1) & 3]) : "l"(l2[(j >> 1) & 3]), "l"(p2));
+          }
           r[j >> 1] = pk;
         }
 #pragma unroll
@@ -442,7 +463,7 @@ __global__ void __launch_bounds__(P2_THREADS, 1) prefill_tc_kernel(const PtParam
           if (j0 + j + 1 > pos) p1 = 0.f;
           const __nv_bfloat162 v2 = __floats2bfloat162_rn(p0, p1);
           const uint32_t pk = *reinterpret_cast<const uint32_t*>(&v2);
-          ls[(j >> 1) & 3] += __uint_as_float(pk << 16) + __uint_as_float(pk & 0xffff0000u);
+          if constexpr (!LSUM) ls[(j >> 1) & 3] += __uint_as_float(pk << 16) + __uint_as_float(pk & 0xffff0000u);
           r[j >> 1] = pk;
         }
       }
@@ -482,6 +503,7 @@ __global__ void __launch_bounds__(P2_THREADS, 1) prefill_tc_kernel(const PtParam
   }
   if (warp < 8 && !timed_out && nt[X] > 0) {
     const int t = q0 + 128 * X + row;
+    if constexpr (LSUM) l_run = __uint_as_float(pt_ld1(tmem_o + lane_off + (uint32_t)p.vs));
     const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
     float* dst = p.out + (((size_t)b * p.T + min(t, p.T - 1)) * p.Hq + g) * p.dv;
 #pragma unroll 1
@@ -503,12 +525,12 @@ __global__ void __launch_bounds__(P2_THREADS, 1) prefill_tc_kernel(const PtParam
   }
 }
 
-template <int DK, int NVP>
+template <int DK, int NVP, bool LSUM>
 rap_status launch_pt(rap_ctx* ctx, const PtParams& p, int B, cudaStream_t st) {
   const int smem = P2_SMEM + 1024;
-  RAP_CUDA_TRY(ctx, rap_raise_smem(ctx, prefill_tc_kernel<DK, NVP>, smem));
+  RAP_CUDA_TRY(ctx, rap_raise_smem(ctx, prefill_tc_kernel<DK, NVP, LSUM>, smem));
   dim3 grid(p.Hq, B, (p.T + 255) / 256);
-  prefill_tc_kernel<DK, NVP><<<grid, P2_THREADS, smem, st>>>(p);
+  prefill_tc_kernel<DK, NVP, LSUM><<<grid, P2_THREADS, smem, st>>>(p);
   ctx->launches++;
   RAP_CUDA_TRY(ctx, cudaGetLastError());
   return RAP_OK;
@@ -544,9 +566,13 @@ rap_status rap_launch_prefill_attn_tc(rap_ctx* ctx, int B, int T, const void* q,
     p.v = (const __nv_bfloat16*)ctx->d_pf_v;
     p.vs = dv + 1;
   }
-  const int dk = (P2 + 15) / 16, nvp = (dv + 31) / 32 * 32;
-  if (dk <= 4 && nvp <= 64) return launch_pt<4, 64>(ctx, p, B, st);
-  if (dk <= 6 && nvp <= 96) return launch_pt<6, 96>(ctx, p, B, st);
-  if (dk <= 7) return launch_pt<7, 128>(ctx, p, B, st);
-  return launch_pt<8, 128>(ctx, p, B, st);
+  // p.vs + 1 channels when the row sums ride along as a ones column (every shape but the ones that fill their last
+  // 32-channel block: then the softmax threads keep the sums)
+  const int dk = (P2 + 15) / 16, nvp = (p.vs + 1 + 31) / 32 * 32;
+  if (dk <= 4 && nvp <= 64) return launch_pt<4, 64, true>(ctx, p, B, st);
+  if (dk <= 4 && nvp <= 96) return launch_pt<4, 96, true>(ctx, p, B, st);
+  if (dk <= 6 && nvp <= 96) return launch_pt<6, 96, true>(ctx, p, B, st);
+  if (dk <= 7 && nvp <= 128) return launch_pt<7, 128, true>(ctx, p, B, st);
+  if (nvp <= 128) return launch_pt<8, 128, true>(ctx, p, B, st);
+  return launch_pt<8, 128, false>(ctx, p, B, st);
 }
