@@ -308,6 +308,7 @@ def run_ours(args):
         line["other_workloads"] = other_workloads(torch, min(K, 10), peak)
         line["sweep"] = sweep_rows(torch, min(K, 10), 3, peak)
         line["quantised_cache"] = q8_rows(torch, min(K, 10), 3, peak)
+        line["quantised_cache_step"] = q8_step(torch, "8b", min(K, 10), 3)
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
@@ -495,6 +496,58 @@ def sweep_rows(torch, steps, warmup, peak):
     return rows
 
 
+def q8_step(torch, name, K, W):
+    """Whole decode steps over quantised caches (rap_decode_step_q8: per layer the projection, the quantising append
+    and the attention over the quantised cache) on a named workload at full size: tokens/s.  The caches are made
+    layer by layer from synthetic bf16 rows by rap_quantize_rows."""
+    from paper_2602_02599_b200 import binding
+    from paper_2602_02599_b200.stack import DecodeStack
+    w = synth.CONFIGS[name]
+    st = DecodeStack(w, max_rows=max(w.batch, 32), s_cap=((w.seq + 64 + 7) // 8) * 8, alloc_cache=False)
+    st.build_tables(*synth.draw_scores(w))
+    g = torch.Generator(device=st.device).manual_seed(w.seed)
+    sigma = float(np.sqrt(w.hidden) * 0.02)
+    kb, vb = binding.rap_q8_row_bytes(2 * w.n_pairs), binding.rap_q8_row_bytes(w.n_vch)
+    n_rows = w.batch * w.n_kv_heads * st.s_cap
+    k8, v8 = [], []
+    tk = torch.empty((n_rows, 2 * w.n_pairs), dtype=st.dt, device=st.device)
+    tv = torch.empty((n_rows, w.n_vch), dtype=st.dt, device=st.device)
+    for l in range(w.n_layers):
+        st.set_packed_weights(l, synth.draw_packed_weights(w, l))
+        tk.normal_(0.0, sigma, generator=g)
+        tv.normal_(0.0, sigma, generator=g)
+        k8.append(torch.empty((n_rows, kb), dtype=torch.uint8, device=st.device))
+        v8.append(torch.empty((n_rows, vb), dtype=torch.uint8, device=st.device))
+        st.ctx.rap_quantize_rows(binding.RAP_BF16, n_rows, 2 * w.n_pairs, tk, k8[l])
+        st.ctx.rap_quantize_rows(binding.RAP_BF16, n_rows, w.n_vch, tv, v8[l])
+    del tk, tv
+    x_all = torch.empty((K + W, w.n_layers, w.batch, w.hidden), dtype=st.dt, device=st.device).normal_(0.0, 1.0, generator=g)
+    wq, k8p, v8p = binding.ptr_array(st.w_qkv), binding.ptr_array(k8), binding.ptr_array(v8)
+    st.seq_len.fill_(w.seq)
+
+    def step(i):
+        st.ctx.rap_decode_step_q8(w.batch, x_all[i], wq, None, st.inv_freq, k8p, v8p, st.s_cap, st.seq_len, w.seq + i, 0,
+                                  st.q_scratch, st.out, st.out_stride, 1)
+
+    for i in range(W):
+        step(i)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(K):
+        step(W + i)
+    e1.record()
+    torch.cuda.synchronize()
+    code, detail = st.ctx.rap_get_last_device_status()
+    assert code == 0, (code, detail)
+    ms = e0.elapsed_time(e1) / K
+    st.close()
+    del st, k8, v8, x_all
+    torch.cuda.empty_cache()
+    return {"workload": workload_string(w), "tokens_per_s": w.batch / (ms * 1e-3), "ms_per_step": ms, "steps": K, "warmup": W,
+            "kv_bytes_per_step": w.n_layers * w.batch * w.n_kv_heads * (w.seq + W + (K + 1) / 2.0) * (kb + vb)}
+
+
 def q8_rows(torch, steps, warmup, peak, names=("3b", "8b", "14b"), batch=0):
     """Composition with 8-bit cache quantisation: rap_decode_attn_q8 against rap_decode_attn on the shaped workloads
     (full batch and context, two layers resident and alternated so that the caches are larger than L2).  The
@@ -563,9 +616,12 @@ def run_q8(args):
     peak, _ = load_peaks()
     names = (args.workload,) if args.workload in ("3b", "14b") or args.batch else ("3b", "8b", "14b")
     rows = q8_rows(torch, args.steps, args.warmup, peak, names=names, batch=args.batch)
-    print(json.dumps({"metric": "quantised_cache_attention", "unit": "ms", "n_gpus": 1, "steps": args.steps,
-                      "warmup": args.warmup, "dtype": "int8 codes, fp16 MMA, fp32 accumulate", "data": "synthetic",
-                      "higher_is_better": False, "quantised_cache": rows}), flush=True)
+    line = {"metric": "quantised_cache_attention", "unit": "ms", "n_gpus": 1, "steps": args.steps,
+            "warmup": args.warmup, "dtype": "int8 codes, fp16 MMA, fp32 accumulate", "data": "synthetic",
+            "higher_is_better": False, "quantised_cache": rows}
+    if not args.batch:
+        line["quantised_cache_step"] = q8_step(torch, args.workload if args.workload in ("3b", "8b", "14b") else "8b", args.steps, args.warmup)
+    print(json.dumps(line), flush=True)
 
 
 def run_sweep(args):

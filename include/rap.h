@@ -210,6 +210,8 @@ rap_status rap_decode_attn(rap_ctx* ctx, int32_t layer, int32_t B, const void* d
  *   rap_qkv_rope_append_q8  rap_qkv_rope_append with the new K and V rows quantised straight from their fp32 values
  *                           (no rounding to the storage dtype in between); q~ as in rap_qkv_rope_append.
  *   rap_decode_attn_q8      rap_decode_attn over quantised caches: Eq. 2 on K_j = c^K_j s^K_j, V_j = c^V_j s^V_j.
+ *   rap_decode_step_q8      rap_decode_step over quantised caches (h_k8 / h_v8: HOST arrays of L device pointers):
+ *                           per layer the quantising append, then the attention over the quantised cache.
  * Arguments, errors and stream behaviour as for the unquantised calls; head_dim <= 256. */
 size_t rap_q8_row_bytes(int32_t W);
 rap_status rap_quantize_rows(rap_ctx* ctx, int32_t dtype_in, int64_t n_rows, int32_t W, const void* d_rows, void* d_q8,
@@ -221,6 +223,12 @@ rap_status rap_qkv_rope_append_q8(rap_ctx* ctx, int32_t layer, int32_t T, const 
 rap_status rap_decode_attn_q8(rap_ctx* ctx, int32_t layer, int32_t B, const void* d_q, const void* d_k8, const void* d_v8,
                               int32_t S_cap, const int32_t* d_seq_len, int32_t h_seq_len_max, int32_t n_split,
                               float* d_out, void* stream);
+
+rap_status rap_decode_step_q8(rap_ctx* ctx, int32_t B, const void* d_x, const void* const* h_w_qkv,
+                              const void* const* h_bias, const double* d_inv_freq, void* const* h_k8,
+                              void* const* h_v8, int32_t S_cap, int32_t* d_seq_len, int32_t h_seq_len_max,
+                              int32_t n_split, void* d_q_scratch, float* d_out, size_t out_layer_stride,
+                              int32_t advance, void* stream);
 
 /* ---- decode attention without any allocation (the paper has no counterpart) --------------
  * Same result as rap_decode_attn, for callers that cannot allocate device memory: code running

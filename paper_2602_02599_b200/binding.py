@@ -28,7 +28,7 @@ EXPORTS = [
     "rap_decode_attn_noalloc", "rap_profile_attn", "rap_profile_attn_read",
     "rap_pack_wo", "rap_out_proj", "rap_budget_alloc", "rap_prefill_attn", "rap_build_tables_hybrid",
     "rap_build_tables_partial", "rap_build_tables_freq", "rap_set_proj_variant", "rap_debug_arm_wait_timeout", "rap_debug_claim_scan_workspace",
-    "rap_q8_row_bytes", "rap_quantize_rows", "rap_qkv_rope_append_q8", "rap_decode_attn_q8",
+    "rap_q8_row_bytes", "rap_quantize_rows", "rap_qkv_rope_append_q8", "rap_decode_attn_q8", "rap_decode_step_q8",
 ]
 
 
@@ -91,6 +91,7 @@ def _lib():
     lib.rap_quantize_rows.argtypes = [P, c_int32, c_int64, c_int32, P, P, P]
     lib.rap_qkv_rope_append_q8.argtypes = lib.rap_qkv_rope_append.argtypes
     lib.rap_decode_attn_q8.argtypes = lib.rap_decode_attn.argtypes
+    lib.rap_decode_step_q8.argtypes = lib.rap_decode_step.argtypes
     lib.rap_budget_alloc.argtypes = [c_int32, c_int32, c_int32, P, c_double, P, P]
     lib.rap_prefill_attn.argtypes = [P, c_int32, c_int32, c_int32, P, P, P, c_int32, P, c_int32, P, P]
     lib.rap_pack_wo.argtypes = [P, c_int32, P, P, P, P]
@@ -291,6 +292,13 @@ class RapContext:
                                            args[3], S_cap, _ptr(d_seq_len), h_seq_len_max, n_split,
                                            _ptr(d_q_scratch), _ptr(d_out), out_layer_stride, advance, _stream()),
                     "rap_decode_step")
+
+    def rap_decode_step_q8(self, B, d_x, w_qkv, bias, d_inv_freq, k8, v8, S_cap, d_seq_len, h_seq_len_max, n_split,
+                           d_q_scratch, d_out, out_layer_stride, advance):
+        args = [a if isinstance(a, ctypes.Array) or a is None else _ptr_array(a) for a in (w_qkv, bias, k8, v8)]
+        self._check(_lib().rap_decode_step_q8(self._ctx, B, _ptr(d_x), args[0], args[1], _ptr(d_inv_freq), args[2], args[3],
+                                              S_cap, _ptr(d_seq_len), h_seq_len_max, n_split, _ptr(d_q_scratch),
+                                              _ptr(d_out), out_layer_stride, advance, _stream()), "rap_decode_step_q8")
 
     def rap_decode_step_host(self, B, h_x, w_qkv, bias, d_inv_freq, k_cache, v_cache, S_cap, d_seq_len,
                              h_seq_len_max, n_split, h_out, out_layer_stride, advance):

@@ -505,6 +505,57 @@ rap_status rap_decode_attn_q8(rap_ctx* ctx, int32_t layer, int32_t B, const void
   return rap_launch_attn_q8(ctx, a, (cudaStream_t)stream);
 }
 
+rap_status rap_decode_step_q8(rap_ctx* ctx, int32_t B, const void* d_x, const void* const* h_w_qkv, const void* const* h_bias,
+                              const double* d_inv_freq, void* const* h_k8, void* const* h_v8, int32_t S_cap,
+                              int32_t* d_seq_len, int32_t h_seq_len_max, int32_t n_split, void* d_q_scratch, float* d_out,
+                              size_t out_layer_stride, int32_t advance, void* stream) {
+  if (!ctx || !d_x || !h_w_qkv || !d_inv_freq || !h_k8 || !h_v8 || !d_seq_len || !d_q_scratch || !d_out) return RAP_EINVAL;
+  if (!ctx->tables_built) return RAP_ESTATE;
+  const rap_model_desc& d = ctx->desc;
+  if (B < 0 || S_cap < 1 || n_split < 0 || h_seq_len_max < 0) return RAP_EINVAL;
+  if (B > d.max_batch || B > d.max_rows || n_split > RAP_MAX_SPLIT) return RAP_ESHAPE;
+  if (S_cap % 8) return RAP_EALIGN;
+  if (h_seq_len_max >= S_cap) return RAP_ECAPACITY;
+  if (d.head_dim > 256) return RAP_EUNSUPPORTED;
+  if (!rap_aligned16(d_x) || !rap_aligned16(d_inv_freq) || !rap_aligned16(d_seq_len) || !rap_aligned16(d_q_scratch) ||
+      !rap_aligned16(d_out) || (out_layer_stride % 4))
+    return RAP_EALIGN;
+  for (int l = 0; l < d.n_layers; ++l) {
+    if (!h_w_qkv[l] || !h_k8[l] || !h_v8[l]) return RAP_EINVAL;
+    if (out_layer_stride < (size_t)B * d.n_q_heads * ctx->n_vch[l]) return RAP_ESHAPE;
+    if (!rap_aligned16(h_w_qkv[l]) || !rap_aligned16(h_k8[l]) || !rap_aligned16(h_v8[l]) ||
+        (h_bias && h_bias[l] && !rap_aligned16(h_bias[l])))
+      return RAP_EALIGN;
+  }
+  if (B == 0) return RAP_OK;
+  cudaStream_t st = (cudaStream_t)stream;
+  const size_t e = rap_elem_bytes(d.dtype);
+  for (int l = 0; l < d.n_layers; ++l) {
+    rap_proj_args p;
+    p.x = (const char*)d_x + (size_t)l * B * d.hidden * e;
+    p.w = h_w_qkv[l]; p.bias = h_bias ? h_bias[l] : nullptr;
+    p.seq_id = nullptr; p.pos = d_seq_len; p.slot = nullptr;   // decode mode: row r = sequence r at pos = slot = len
+    p.inv_freq = d_inv_freq + (size_t)l * d.n_kv_heads * (d.head_dim / 2);
+    p.q_out = d_q_scratch; p.k_cache = h_k8[l]; p.v_cache = h_v8[l];
+    p.T = B; p.hidden = d.hidden; p.Hq = d.n_q_heads; p.Hkv = d.n_kv_heads;
+    p.P2 = 2 * ctx->n_pairs[l]; p.dv = ctx->n_vch[l]; p.half_dim = d.head_dim / 2;
+    p.B_cache = B; p.S_cap = S_cap; p.dtype = d.dtype;
+    p.pdl = l > 0 ? 1 : 0;     // the GEMM of layer l may stream its weights while the scan of layer l - 1 drains
+    rap_status s = rap_launch_qkv_rope_append_q8(ctx, p, st);
+    if (s != RAP_OK) return s;
+    rap_attn_args a;
+    a.q = d_q_scratch; a.k = h_k8[l]; a.v = h_v8[l]; a.seq_len = d_seq_len; a.len_add = 1;
+    a.B = B; a.Hq = d.n_q_heads; a.Hkv = d.n_kv_heads; a.P2 = p.P2; a.dv = p.dv; a.S_cap = S_cap;
+    a.head_dim = d.head_dim; a.dtype = d.dtype; a.n_split = n_split; a.h_len_max = h_seq_len_max + 1;
+    a.out = d_out + (size_t)l * out_layer_stride;
+    a.pdl = 1;
+    s = rap_launch_attn_q8(ctx, a, st);
+    if (s != RAP_OK) return s;
+  }
+  if (advance) return rap_launch_advance(ctx, d_seq_len, B, st);
+  return RAP_OK;
+}
+
 rap_status rap_prefill_attn(rap_ctx* ctx, int32_t layer, int32_t B, int32_t T, const void* d_q, const void* d_k_cache,
                             const void* d_v_cache, int32_t S_cap, const int32_t* d_start, int32_t h_start_max,
                             float* d_out, void* stream) {

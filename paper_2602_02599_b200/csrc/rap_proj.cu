@@ -15,7 +15,7 @@
 rap_status rap_launch_proj_tc(rap_ctx* ctx, const rap_proj_args& a, int* ksplit_out, cudaStream_t st);
 rap_status rap_launch_proj_fused(rap_ctx* ctx, const rap_proj_args& a, cudaStream_t st);
 rap_status rap_launch_gemm_tc(rap_ctx* ctx, const void* x, const void* w, int T, int K, int N, int* ksplit_out,
-                              cudaStream_t st);
+                              cudaStream_t st, int pdl);
 
 namespace {
 
@@ -341,7 +341,7 @@ rap_status rap_launch_out_proj(rap_ctx* ctx, int32_t layer, int32_t T, const flo
     cast_bf16_kernel<<<(unsigned)((nx + 255) / 256), 256, 0, st>>>(attn_out, (__nv_bfloat16*)ctx->d_oproj_x, nx);
     ctx->launches++;
     RAP_CUDA_TRY(ctx, cudaGetLastError());
-    rap_status s = rap_launch_gemm_tc(ctx, ctx->d_oproj_x, wo_tilde, T, K, N, &ksplit, st);
+    rap_status s = rap_launch_gemm_tc(ctx, ctx->d_oproj_x, wo_tilde, T, K, N, &ksplit, st, 0);
     if (s == RAP_EUNSUPPORTED) {
       if ((K * 2) % 16) return RAP_EUNSUPPORTED;
       ksplit = 1;

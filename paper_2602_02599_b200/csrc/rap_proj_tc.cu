@@ -197,8 +197,8 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_d = *tmem_slot;
   bool timed_out = false;
+  tc_pdl_launch_dependents();        // the next kernel in the stream may start its own prologue
   if constexpr (FUSED) {
-    tc_pdl_launch_dependents();      // the next kernel in the stream may start its own prologue
     if (blockIdx.x == 0)             // counters a predecessor that gave up may have left behind
       for (int i = threadIdx.x; i < f.n_cnt; i += TC_THREADS) f.cnt_other[i] = 0;
   }
@@ -436,6 +436,10 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"(2 * TN) : "memory");
   }
+  // The plain form writes nothing its predecessor in the stream reads, so it never had to wait for it; but a kernel
+  // launched behind this one with programmatic serialization only waits for THIS kernel: by not ending before the
+  // predecessor has, this kernel's completion stands for both.
+  if constexpr (!FUSED) tc_pdl_wait();
 }
 
 typedef CUresult (*encode_tiled_t)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -485,13 +489,25 @@ bool make_map(rap_ctx* ctx, CUtensorMap* map, const void* base, uint64_t rows, u
   return true;
 }
 
+// pdl: launch with programmatic stream serialization.  The plain GEMM reads X and W and writes only the projection
+// workspace, none of which the kernel before it in a decode step (an attention scan) touches, so it may run alongside
+// that kernel's tail without waiting for it; the epilogue kernel after it is launched normally and waits for both.
 template <int TN>
 rap_status launch_tc(rap_ctx* ctx, const CUtensorMap& mw, const CUtensorMap& mx, const TcParams& p, dim3 grid,
-                     cudaStream_t st) {
+                     cudaStream_t st, int pdl) {
   RAP_CUDA_TRY(ctx, rap_raise_smem(ctx, proj_tc_kernel<TN, false>, TcCfg<TN>::SMEM));
-  proj_tc_kernel<TN, false><<<grid, TC_THREADS, TcCfg<TN>::SMEM, st>>>(mw, mx, p, TcFused{});
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = dim3(TC_THREADS, 1, 1);
+  cfg.dynamicSmemBytes = TcCfg<TN>::SMEM;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl ? 1 : 0;
+  RAP_CUDA_TRY(ctx, cudaLaunchKernelEx(&cfg, proj_tc_kernel<TN, false>, mw, mx, p, TcFused{}));
   ctx->launches++;
-  RAP_CUDA_TRY(ctx, cudaGetLastError());
   return RAP_OK;
 }
 
@@ -524,7 +540,7 @@ bool rap_tensor_map_bf16(rap_ctx* ctx, void* map128, const void* base, uint64_t 
 
 // Y[ks][T][N] (fp32, context workspace) = X[T][K] * W[N][K]^T, bf16 operands, K split over work items.
 rap_status rap_launch_gemm_tc(rap_ctx* ctx, const void* x, const void* w, int T, int K, int N, int* ksplit_out,
-                              cudaStream_t st) {
+                              cudaStream_t st, int pdl) {
   if (T < 1 || (K % 8) != 0) return RAP_EUNSUPPORTED;     // tensor-map rows must be multiples of 16 bytes
   TcParams p;
   int tn = 0, ksplit = 1;
@@ -535,17 +551,17 @@ rap_status rap_launch_gemm_tc(rap_ctx* ctx, const void* x, const void* w, int T,
   dim3 grid(p.n_work < ctx->sm_count ? p.n_work : ctx->sm_count, 1, 1);
   *ksplit_out = ksplit;
   switch (tn) {
-    case 32: return launch_tc<32>(ctx, mw, mx, p, grid, st);
-    case 64: return launch_tc<64>(ctx, mw, mx, p, grid, st);
-    case 128: return launch_tc<128>(ctx, mw, mx, p, grid, st);
-    default: return launch_tc<256>(ctx, mw, mx, p, grid, st);
+    case 32: return launch_tc<32>(ctx, mw, mx, p, grid, st, pdl);
+    case 64: return launch_tc<64>(ctx, mw, mx, p, grid, st, pdl);
+    case 128: return launch_tc<128>(ctx, mw, mx, p, grid, st, pdl);
+    default: return launch_tc<256>(ctx, mw, mx, p, grid, st, pdl);
   }
 }
 
 rap_status rap_launch_proj_tc(rap_ctx* ctx, const rap_proj_args& a, int* ksplit_out, cudaStream_t st) {
   if (a.dtype != RAP_BF16) return RAP_EUNSUPPORTED;
   const int n_out = (a.Hq + a.Hkv) * a.P2 + a.Hkv * a.dv;
-  return rap_launch_gemm_tc(ctx, a.x, a.w, a.T, a.hidden, n_out, ksplit_out, st);
+  return rap_launch_gemm_tc(ctx, a.x, a.w, a.T, a.hidden, n_out, ksplit_out, st, a.pdl);
 }
 
 // Decode-sized rap_qkv_rope_append in ONE launch: the tcgen05 GEMM with the RoPE / append epilogue fused in.

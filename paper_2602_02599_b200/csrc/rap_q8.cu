@@ -76,6 +76,10 @@ rope_append_q8_kernel(const float* __restrict__ y, int ksplit, const T* __restri
                       T* __restrict__ q_out, unsigned char* __restrict__ k8, unsigned char* __restrict__ v8, int Trows, int Hq,
                       int Hkv, int P2, int dv, int half_dim, int B_cache, int S_cap, int k_row_bytes, int v_row_bytes,
                       int32_t* __restrict__ status) {
+  // launched behind the GEMM with programmatic serialization inside a decode step: nothing above this line touches
+  // memory; the GEMM's results (and, through the GEMM, the end of the scan before it) are awaited here
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const int items = Hq + 2 * Hkv;
   const long long wid = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
@@ -93,18 +97,23 @@ rope_append_q8_kernel(const float* __restrict__ y, int ksplit, const T* __restri
   }
   const size_t split_stride = (size_t)Trows * n_out;
   const float* yr = y + (size_t)t * n_out;
-  auto summed = [&](int col) {
-    float a = 0.f;
-    for (int s = 0; s < ksplit; ++s) a += yr[s * split_stride + col];
-    if (bias) a += q8_ld(bias + col);
-    return a;
-  };
   if (item < Hq + Hkv) {
     const bool is_q = item < Hq;
     const int h = is_q ? item / G : item - Hq;                 // KV head whose frequencies apply
     const int col0 = item * P2;                                // q heads, then k heads: item * 2P either way
     float ra[4], rb[4];
     float amax = 0.f;
+    // every partial of this lane's pairs first (independent loads), then the sums in split order and the bias
+    float pa[4][RAP_MAX_KSPLIT], pb[4][RAP_MAX_KSPLIT];
+#pragma unroll
+    for (int k = 0; k < 4; ++k)
+#pragma unroll
+      for (int s = 0; s < RAP_MAX_KSPLIT; ++s) {
+        const int c = lane + 32 * k;
+        const bool on = c < P && s < ksplit;
+        pa[k][s] = on ? yr[s * split_stride + col0 + 2 * c] : 0.f;
+        pb[k][s] = on ? yr[s * split_stride + col0 + 2 * c + 1] : 0.f;
+      }
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
       const int c = lane + 32 * k;
@@ -116,7 +125,11 @@ rope_append_q8_kernel(const float* __restrict__ y, int ksplit, const T* __restri
         const double red = fma(-turns, 2.4492935982947064e-16, fma(-turns, 6.283185307179586, ang));
         float sf, cf;
         sincosf((float)red, &sf, &cf);
-        const float a = summed(col0 + 2 * c), b = summed(col0 + 2 * c + 1);
+        float a = 0.f, b = 0.f;
+#pragma unroll
+        for (int s = 0; s < RAP_MAX_KSPLIT; ++s)
+          if (s < ksplit) { a += pa[k][s]; b += pb[k][s]; }
+        if (bias) { a += q8_ld(bias + col0 + 2 * c); b += q8_ld(bias + col0 + 2 * c + 1); }
         ra[k] = a * cf - b * sf;
         rb[k] = a * sf + b * cf;
         amax = fmaxf(amax, fmaxf(fabsf(ra[k]), fabsf(rb[k])));
@@ -150,10 +163,20 @@ rope_append_q8_kernel(const float* __restrict__ y, int ksplit, const T* __restri
     const int col0 = (Hq + Hkv) * P2 + h * dv;
     float v[8];
     float amax = 0.f;
+    float pv[8][RAP_MAX_KSPLIT];
+#pragma unroll
+    for (int k = 0; k < 8; ++k)
+#pragma unroll
+      for (int s = 0; s < RAP_MAX_KSPLIT; ++s) pv[k][s] = (lane + 32 * k < dv && s < ksplit) ? yr[s * split_stride + col0 + lane + 32 * k] : 0.f;
 #pragma unroll
     for (int k = 0; k < 8; ++k) {
       const int c = lane + 32 * k;
-      v[k] = c < dv ? summed(col0 + c) : 0.f;
+      float a = 0.f;
+#pragma unroll
+      for (int s = 0; s < RAP_MAX_KSPLIT; ++s)
+        if (s < ksplit) a += pv[k][s];
+      if (bias && c < dv) a += q8_ld(bias + col0 + c);
+      v[k] = c < dv ? a : 0.f;
       amax = fmaxf(amax, fabsf(v[k]));
     }
     const float s = q8_scale(warp_max(amax));
@@ -324,18 +347,30 @@ rap_status rap_launch_qkv_rope_append_q8(rap_ctx* ctx, const rap_proj_args& a, c
   const long long warps = (long long)a.T * (a.Hq + 2 * a.Hkv);
   const unsigned blocks = (unsigned)((warps + 7) / 8);
   const int krb = (int)rap_q8_row_bytes(a.P2), vrb = (int)rap_q8_row_bytes(a.dv);
+  // inside a decode step (a.pdl): launched behind the tcgen05 GEMM with programmatic serialization, so that its launch
+  // overlaps the GEMM's tail; the kernel waits for the GEMM before it touches memory (the CUDA-core GEMM of the other
+  // path never triggers early, which makes the attribute a no-op there)
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(blocks, 1, 1);
+  cfg.blockDim = dim3(256, 1, 1);
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = a.pdl ? 1 : 0;
+  const float* y = ctx->d_proj_ws;
+  unsigned char* k8 = (unsigned char*)a.k_cache;
+  unsigned char* v8 = (unsigned char*)a.v_cache;
   if (a.dtype == RAP_F32)
-    rope_append_q8_kernel<float><<<blocks, 256, 0, st>>>(ctx->d_proj_ws, ksplit, (const float*)a.bias, a.seq_id, a.pos, a.slot,
-                                                         a.inv_freq, (float*)a.q_out, (unsigned char*)a.k_cache,
-                                                         (unsigned char*)a.v_cache, a.T, a.Hq, a.Hkv, a.P2, a.dv, a.half_dim,
-                                                         a.B_cache, a.S_cap, krb, vrb, ctx->d_status);
+    RAP_CUDA_TRY(ctx, cudaLaunchKernelEx(&cfg, rope_append_q8_kernel<float>, y, ksplit, (const float*)a.bias, a.seq_id, a.pos,
+                                         a.slot, a.inv_freq, (float*)a.q_out, k8, v8, a.T, a.Hq, a.Hkv, a.P2, a.dv,
+                                         a.half_dim, a.B_cache, a.S_cap, krb, vrb, ctx->d_status));
   else
-    rope_append_q8_kernel<__nv_bfloat16><<<blocks, 256, 0, st>>>(
-        ctx->d_proj_ws, ksplit, (const __nv_bfloat16*)a.bias, a.seq_id, a.pos, a.slot, a.inv_freq, (__nv_bfloat16*)a.q_out,
-        (unsigned char*)a.k_cache, (unsigned char*)a.v_cache, a.T, a.Hq, a.Hkv, a.P2, a.dv, a.half_dim, a.B_cache, a.S_cap, krb,
-        vrb, ctx->d_status);
+    RAP_CUDA_TRY(ctx, cudaLaunchKernelEx(&cfg, rope_append_q8_kernel<__nv_bfloat16>, y, ksplit, (const __nv_bfloat16*)a.bias,
+                                         a.seq_id, a.pos, a.slot, a.inv_freq, (__nv_bfloat16*)a.q_out, k8, v8, a.T, a.Hq, a.Hkv,
+                                         a.P2, a.dv, a.half_dim, a.B_cache, a.S_cap, krb, vrb, ctx->d_status));
   ctx->launches++;
-  RAP_CUDA_TRY(ctx, cudaGetLastError());
   return RAP_OK;
 }
 

@@ -228,3 +228,58 @@ def test_q8_full_size_sampled_units(name):
                                     vs[None, None], [n], w.head_dim)[0]
             util.check_attn(util.to_np64(out[b, h * G:(h + 1) * G]), want, w.dtype)
     st.close()
+
+
+@pytest.mark.parametrize("name", ["8b", "3b"])
+def test_q8_decode_step_equals_the_separate_calls_and_the_oracle(name):
+    """rap_decode_step_q8 (all layers: quantising append, then attention over the quantised cache; consecutive launches
+    overlap) against the same step made of rap_qkv_rope_append_q8 + rap_decode_attn_q8 calls -- bit for bit, caches
+    and outputs -- and its attention against the oracle on the device's own codes; the lengths advance."""
+    w = synth.scaled_down(synth.CONFIGS[name], n_layers=3, batch=2, seq=300, hidden=512)
+    lens = np.array([300, 211], dtype=np.int32)
+    ks, vs = synth.draw_scores(w)
+    st, tabs, w_host = util.build_small_stack(w, ks, vs, full_weights=False, max_rows=256)
+    B, Hq, Hkv, D, L = w.batch, w.n_q_heads, w.n_kv_heads, w.head_dim, w.n_layers
+    g = torch.Generator(device=st.device).manual_seed(11)
+    sig = float(np.sqrt(w.hidden) * 0.02)
+    k8, v8 = [], []
+    n_rows = B * Hkv * st.s_cap
+    for l in range(L):
+        st.k_cache[l].normal_(0, sig, generator=g)
+        st.v_cache[l].normal_(0, sig, generator=g)
+        a, b = _q8_caches(st, l)
+        st.ctx.rap_quantize_rows(binding.RAP_BF16, n_rows, 2 * st.n_pairs[l], st.k_cache[l], a)
+        st.ctx.rap_quantize_rows(binding.RAP_BF16, n_rows, st.n_vch[l], st.v_cache[l], b)
+        k8.append(a)
+        v8.append(b)
+    x = torch.empty((L, B, w.hidden), dtype=st.dt, device=st.device).normal_(0, 1, generator=g)
+    # the step as separate calls, on copies
+    k8_ref, v8_ref = [t.clone() for t in k8], [t.clone() for t in v8]
+    dl = torch.from_numpy(lens).to(st.device)
+    sid = torch.arange(B, dtype=torch.int32, device=st.device)
+    out_ref, q_ref = [], []
+    for l in range(L):
+        q = torch.empty((B, Hq, 2 * st.n_pairs[l]), dtype=st.dt, device=st.device)
+        st.ctx.rap_qkv_rope_append_q8(l, B, x[l], st.w_qkv[l], None, sid, dl, dl, int(lens.max()), st.inv_freq, q, k8_ref[l],
+                                      v8_ref[l], B, st.s_cap)
+        o = torch.empty((B, Hq, st.n_vch[l]), dtype=torch.float32, device=st.device)
+        st.ctx.rap_decode_attn_q8(l, B, q, k8_ref[l], v8_ref[l], st.s_cap, dl + 1, int(lens.max()) + 1, 0, o)
+        out_ref.append(o)
+        q_ref.append(q)
+    st.seq_len.copy_(dl)
+    st.out.fill_(float("nan"))
+    st.ctx.rap_decode_step_q8(B, x, st.w_qkv, None, st.inv_freq, k8, v8, st.s_cap, st.seq_len, int(lens.max()), 0, st.q_scratch,
+                              st.out, st.out_stride, 1)
+    torch.cuda.synchronize()
+    assert st.ctx.rap_get_last_device_status() == (0, 0)
+    assert st.seq_len.cpu().tolist() == (lens + 1).tolist()
+    for l in range(L):
+        P2, dv = 2 * st.n_pairs[l], st.n_vch[l]
+        assert torch.equal(k8[l], k8_ref[l]) and torch.equal(v8[l], v8_ref[l])
+        got = st.out[l][: B * Hq * dv].reshape(B, Hq, dv)
+        assert torch.equal(got, out_ref[l])
+        kc, ksc = util.unpack_q8(k8[l], P2)
+        vc, vsc = util.unpack_q8(v8[l], dv)
+        want = O.decode_attn_q8(util.to_np64(q_ref[l]), kc, ksc, vc, vsc, lens + 1, D)
+        util.check_attn(util.to_np64(got), want, w.dtype)
+    st.close()
