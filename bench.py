@@ -428,8 +428,9 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": int(os.environ.get("WORLD_SIZE", "1")),
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": t_step * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-        "config": {"workload": f"{w.name}: L={L} hidden={w.hidden} Hq/Hkv={Hq}/{Hkv} D={w.head_dim} rho={w.rho} "
-                               f"P={w.n_pairs} dv={w.n_vch} B={B} S={w.seq}"},
+        "config": {"workload": workload_string(w), "per_gpu_batch": B, "global_batch": B, "context": w.seq,
+                   "l2": "inputs larger than L2 (%.1f GB of KV cache per step)" % (L * attn_bytes(w, w.seq + args.warmup + (args.steps + 1) / 2.0) / 1e9),
+                   "parallelism": "single"},
         "cpu_baseline": {"value": val, "unit": UNIT, "cores": busy.cores(), "cores_available": os.cpu_count(), "kind": "oracle",
                          "sample": sample},
         "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
