@@ -303,7 +303,10 @@ rap_status rap_decode_step(rap_ctx* ctx, int32_t B, const void* d_x, const void*
 
 /* Same step with HOST input and output: h_x [L][B][hidden] (storage dtype) is copied to the
  * device, the step runs, out is copied back to h_out [L][out_layer_stride] and the stream is
- * synchronized before returning.  Pinned host memory makes the copies asynchronous. */
+ * synchronized before returning.  With pinned host memory the copies are asynchronous and overlap the
+ * layers: the inputs of layers >= 1 arrive on a context-owned stream while layer 0 runs, and the outputs
+ * of all but the last layer leave on another while later layers run.  h_x must stay unchanged and h_out
+ * unread until the call returns. */
 rap_status rap_decode_step_host(rap_ctx* ctx, int32_t B, const void* h_x, const void* const* h_w_qkv,
                                 const void* const* h_bias, const double* d_inv_freq,
                                 void* const* h_k_cache, void* const* h_v_cache, int32_t S_cap,

@@ -37,6 +37,10 @@ void free_all(rap_ctx* c) {
   if (c->d_lr_k) cudaFree(c->d_lr_k);
   if (c->d_lr_cs) cudaFree(c->d_lr_cs);
   if (c->h_tables) cudaFreeHost(c->h_tables);
+  if (c->copy_in) cudaStreamDestroy((cudaStream_t)c->copy_in);
+  if (c->copy_out) cudaStreamDestroy((cudaStream_t)c->copy_out);
+  if (c->ev_in) cudaEventDestroy((cudaEvent_t)c->ev_in);
+  if (c->ev_mid) cudaEventDestroy((cudaEvent_t)c->ev_mid);
   for (cudaEvent_t e : c->prof_ev) cudaEventDestroy(e);
 }
 
@@ -216,6 +220,18 @@ rap_status rap_create(const rap_model_desc* desc, rap_ctx** out) {
   c->h_tables_bytes = units * ((size_t)(d.head_dim / 2 + 2 * d.head_dim) * sizeof(int32_t) +
                                (size_t)(d.head_dim / 2) * sizeof(double));
   RAP_CUDA_TRY(c, cudaMallocHost(&c->h_tables, c->h_tables_bytes));
+  {   // copy streams and events of rap_decode_step_host
+    cudaStream_t s1, s2;
+    cudaEvent_t e1, e2;
+    RAP_CUDA_TRY(c, cudaStreamCreateWithFlags(&s1, cudaStreamNonBlocking));
+    c->copy_in = s1;
+    RAP_CUDA_TRY(c, cudaStreamCreateWithFlags(&s2, cudaStreamNonBlocking));
+    c->copy_out = s2;
+    RAP_CUDA_TRY(c, cudaEventCreateWithFlags(&e1, cudaEventDisableTiming));
+    c->ev_in = e1;
+    RAP_CUDA_TRY(c, cudaEventCreateWithFlags(&e2, cudaEventDisableTiming));
+    c->ev_mid = e2;
+  }
   return RAP_OK;
 }
 
@@ -574,11 +590,11 @@ rap_status rap_prefill_attn(rap_ctx* ctx, int32_t layer, int32_t B, int32_t T, c
                                  d_start, d_out, (cudaStream_t)stream);
 }
 
-rap_status rap_decode_step(rap_ctx* ctx, int32_t B, const void* d_x, const void* const* h_w_qkv,
-                           const void* const* h_bias, const double* d_inv_freq, void* const* h_k_cache,
-                           void* const* h_v_cache, int32_t S_cap, int32_t* d_seq_len, int32_t h_seq_len_max,
-                           int32_t n_split, void* d_q_scratch, float* d_out, size_t out_layer_stride,
-                           int32_t advance, void* stream) {
+// argument checks of a decode step (everything but launching it)
+static rap_status decode_step_check(rap_ctx* ctx, int32_t B, const void* d_x, const void* const* h_w_qkv,
+                                    const void* const* h_bias, const double* d_inv_freq, void* const* h_k_cache,
+                                    void* const* h_v_cache, int32_t S_cap, int32_t* d_seq_len, int32_t h_seq_len_max,
+                                    int32_t n_split, void* d_q_scratch, float* d_out, size_t out_layer_stride) {
   if (!ctx || !d_x || !h_w_qkv || !d_inv_freq || !h_k_cache || !h_v_cache || !d_seq_len || !d_q_scratch || !d_out)
     return RAP_EINVAL;
   if (!ctx->tables_built) return RAP_ESTATE;
@@ -597,10 +613,17 @@ rap_status rap_decode_step(rap_ctx* ctx, int32_t B, const void* d_x, const void*
         (h_bias && h_bias[l] && !rap_aligned16(h_bias[l])))
       return RAP_EALIGN;
   }
-  if (B == 0) return RAP_OK;
-  cudaStream_t st = (cudaStream_t)stream;
+  return RAP_OK;
+}
+
+// layers [l0, l1) of a decode step whose arguments have been checked
+static rap_status decode_layers(rap_ctx* ctx, int l0, int l1, int32_t B, const void* d_x, const void* const* h_w_qkv,
+                                const void* const* h_bias, const double* d_inv_freq, void* const* h_k_cache,
+                                void* const* h_v_cache, int32_t S_cap, int32_t* d_seq_len, int32_t h_seq_len_max,
+                                int32_t n_split, void* d_q_scratch, float* d_out, size_t out_layer_stride, cudaStream_t st) {
+  const rap_model_desc& d = ctx->desc;
   const size_t e = rap_elem_bytes(d.dtype);
-  for (int l = 0; l < d.n_layers; ++l) {
+  for (int l = l0; l < l1; ++l) {
     const bool timed = 2 * (ctx->prof_pairs + 1) <= (int)ctx->prof_ev.size();   // events around this layer's attention
     rap_proj_args p;
     p.x = (const char*)d_x + (size_t)l * B * d.hidden * e;
@@ -611,10 +634,10 @@ rap_status rap_decode_step(rap_ctx* ctx, int32_t B, const void* d_x, const void*
     p.T = B; p.hidden = d.hidden; p.Hq = d.n_q_heads; p.Hkv = d.n_kv_heads;
     p.P2 = 2 * ctx->n_pairs[l]; p.dv = ctx->n_vch[l]; p.half_dim = d.head_dim / 2;
     p.B_cache = B; p.S_cap = S_cap; p.dtype = d.dtype;
-    // Inside a step the library knows what precedes each launch: from the second layer on the projection follows
-    // an attention launch that does not touch what the projection reads, so it may start streaming its weights
-    // while that launch drains (the first projection follows caller work, e.g. the length update, and waits).
-    p.pdl = (l > 0 && !timed) ? 1 : 0;
+    // Inside a run of layers the library knows what precedes each launch: from the run's second layer on the
+    // projection follows an attention launch that does not touch what the projection reads, so it may start
+    // streaming its weights while that launch drains (the first projection follows caller work or a copy, and waits).
+    p.pdl = (l > l0 && !timed) ? 1 : 0;
     rap_status s = rap_launch_qkv_rope_append(ctx, p, st);
     if (s != RAP_OK) return s;
     rap_attn_args a;
@@ -631,6 +654,21 @@ rap_status rap_decode_step(rap_ctx* ctx, int32_t B, const void* d_x, const void*
       ctx->prof_pairs++;
     }
   }
+  return RAP_OK;
+}
+
+rap_status rap_decode_step(rap_ctx* ctx, int32_t B, const void* d_x, const void* const* h_w_qkv,
+                           const void* const* h_bias, const double* d_inv_freq, void* const* h_k_cache,
+                           void* const* h_v_cache, int32_t S_cap, int32_t* d_seq_len, int32_t h_seq_len_max,
+                           int32_t n_split, void* d_q_scratch, float* d_out, size_t out_layer_stride,
+                           int32_t advance, void* stream) {
+  rap_status s = decode_step_check(ctx, B, d_x, h_w_qkv, h_bias, d_inv_freq, h_k_cache, h_v_cache, S_cap, d_seq_len,
+                                   h_seq_len_max, n_split, d_q_scratch, d_out, out_layer_stride);
+  if (s != RAP_OK || B == 0) return s;
+  cudaStream_t st = (cudaStream_t)stream;
+  s = decode_layers(ctx, 0, ctx->desc.n_layers, B, d_x, h_w_qkv, h_bias, d_inv_freq, h_k_cache, h_v_cache, S_cap, d_seq_len,
+                    h_seq_len_max, n_split, d_q_scratch, d_out, out_layer_stride, st);
+  if (s != RAP_OK) return s;
   if (advance) return rap_launch_advance(ctx, d_seq_len, B, st);
   return RAP_OK;
 }
@@ -649,13 +687,49 @@ rap_status rap_decode_step_host(rap_ctx* ctx, int32_t B, const void* h_x, const 
   const size_t xb = (size_t)d.n_layers * B * d.hidden * rap_elem_bytes(d.dtype);
   const size_t ob = (size_t)d.n_layers * out_layer_stride * sizeof(float);
   if (B == 0) return RAP_OK;
-  RAP_CUDA_TRY(ctx, cudaMemcpyAsync(ctx->d_stage_x, h_x, xb, cudaMemcpyHostToDevice, st));
-  rap_status s = rap_decode_step(ctx, B, ctx->d_stage_x, h_w_qkv, h_bias, d_inv_freq, h_k_cache, h_v_cache, S_cap,
-                                 d_seq_len, h_seq_len_max, n_split, ctx->d_stage_q, ctx->d_stage_out,
-                                 out_layer_stride, advance, stream);
+  rap_status s = decode_step_check(ctx, B, ctx->d_stage_x, h_w_qkv, h_bias, d_inv_freq, h_k_cache, h_v_cache, S_cap, d_seq_len,
+                                   h_seq_len_max, n_split, ctx->d_stage_q, ctx->d_stage_out, out_layer_stride);
   if (s != RAP_OK) return s;
-  RAP_CUDA_TRY(ctx, cudaMemcpyAsync(h_out, ctx->d_stage_out, ob, cudaMemcpyDeviceToHost, st));
+  const int L = d.n_layers;
+  const size_t x_layer = (size_t)B * d.hidden * rap_elem_bytes(d.dtype), o_layer = out_layer_stride * sizeof(float);
+  auto layers = [&](int l0, int l1) {
+    return decode_layers(ctx, l0, l1, B, ctx->d_stage_x, h_w_qkv, h_bias, d_inv_freq, h_k_cache, h_v_cache, S_cap, d_seq_len,
+                         h_seq_len_max, n_split, ctx->d_stage_q, ctx->d_stage_out, out_layer_stride, st);
+  };
+  if (L < 4) {       // short stacks: copy in, run, copy out
+    RAP_CUDA_TRY(ctx, cudaMemcpyAsync(ctx->d_stage_x, h_x, xb, cudaMemcpyHostToDevice, st));
+    if ((s = layers(0, L)) != RAP_OK) return s;
+    if (advance && (s = rap_launch_advance(ctx, d_seq_len, B, st)) != RAP_OK) return s;
+    RAP_CUDA_TRY(ctx, cudaMemcpyAsync(h_out, ctx->d_stage_out, ob, cudaMemcpyDeviceToHost, st));
+    RAP_CUDA_TRY(ctx, cudaStreamSynchronize(st));
+    return RAP_OK;
+  }
+  // The copies overlap the layers.  Only layer 0's inputs are copied ahead of it on the caller's stream; the rest
+  // arrive on a second stream while layer 0 runs (layer 0's copy is issued first: a copy engine serves copies in
+  // the order they were issued).  The outputs leave in three pieces: layers [0, L/2) on a third stream while the
+  // second half runs, [L/2, L-1) while the last layer runs, the last layer's on the caller's stream.  The staging
+  // buffers are free when a call starts: the previous call synchronized every stream that touched them.
+  cudaStream_t cin = (cudaStream_t)ctx->copy_in, cout = (cudaStream_t)ctx->copy_out;
+  const char* hx = (const char*)h_x;
+  RAP_CUDA_TRY(ctx, cudaMemcpyAsync(ctx->d_stage_x, hx, x_layer, cudaMemcpyHostToDevice, st));
+  RAP_CUDA_TRY(ctx, cudaMemcpyAsync((char*)ctx->d_stage_x + x_layer, hx + x_layer, xb - x_layer, cudaMemcpyHostToDevice, cin));
+  RAP_CUDA_TRY(ctx, cudaEventRecord((cudaEvent_t)ctx->ev_in, cin));
+  if ((s = layers(0, 1)) != RAP_OK) return s;
+  RAP_CUDA_TRY(ctx, cudaStreamWaitEvent(st, (cudaEvent_t)ctx->ev_in, 0));
+  const int cut[3] = {0, L / 2, L - 1};
+  for (int c = 0; c < 2; ++c) {
+    if ((s = layers(c == 0 ? 1 : cut[c], cut[c + 1])) != RAP_OK) return s;
+    RAP_CUDA_TRY(ctx, cudaEventRecord((cudaEvent_t)ctx->ev_mid, st));
+    RAP_CUDA_TRY(ctx, cudaStreamWaitEvent(cout, (cudaEvent_t)ctx->ev_mid, 0));
+    RAP_CUDA_TRY(ctx, cudaMemcpyAsync((char*)h_out + (size_t)cut[c] * o_layer, (const char*)ctx->d_stage_out + (size_t)cut[c] * o_layer,
+                                      (size_t)(cut[c + 1] - cut[c]) * o_layer, cudaMemcpyDeviceToHost, cout));
+  }
+  if ((s = layers(L - 1, L)) != RAP_OK) return s;
+  if (advance && (s = rap_launch_advance(ctx, d_seq_len, B, st)) != RAP_OK) return s;
+  RAP_CUDA_TRY(ctx, cudaMemcpyAsync((char*)h_out + (size_t)(L - 1) * o_layer, (const char*)ctx->d_stage_out + (size_t)(L - 1) * o_layer,
+                                    o_layer, cudaMemcpyDeviceToHost, st));
   RAP_CUDA_TRY(ctx, cudaStreamSynchronize(st));
+  RAP_CUDA_TRY(ctx, cudaStreamSynchronize(cout));
   return RAP_OK;
 }
 

@@ -46,6 +46,10 @@ struct rap_ctx {
   size_t lr_cs_bytes = 0;
   int lr_cs_len = 0;              // positions the table currently covers
   size_t stage_x_bytes = 0, stage_out_bytes = 0;
+  void* copy_in = nullptr;        // rap_decode_step_host: stream of the input copies behind layer 0's (cudaStream_t)
+  void* copy_out = nullptr;       // rap_decode_step_host: stream of the early output copies
+  void* ev_in = nullptr;          // the inputs of layers >= 1 have arrived (cudaEvent_t)
+  void* ev_mid = nullptr;         // the layers before a cut have run
   // pinned host staging for rap_build_tables
   void* h_tables = nullptr;
   size_t h_tables_bytes = 0;

@@ -313,8 +313,9 @@ def test_attention_generic_variant_matches():
     st.close()
 
 
-def test_decode_step_host_matches_device_step():
-    w = synth.scaled_down(synth.LLAMA_8B, n_layers=2, batch=2, seq=256, hidden=256)
+@pytest.mark.parametrize("n_layers", [2, 4, 7])      # below 4 layers the copies do not overlap the layers; 7: odd cut
+def test_decode_step_host_matches_device_step(n_layers):
+    w = synth.scaled_down(synth.LLAMA_8B, n_layers=n_layers, batch=2, seq=256, hidden=256)
     ks, vs = synth.draw_scores(w)
     st, tabs, w_host = util.build_small_stack(w, ks, vs, full_weights=False)
     g = torch.Generator(device=st.device).manual_seed(3)
@@ -331,6 +332,7 @@ def test_decode_step_host_matches_device_step():
         st.k_cache[l][:, :, 256, :] = 0
         st.v_cache[l][:, :, 256, :] = 0
     h_out = torch.empty((w.n_layers, st.out_stride), dtype=torch.float32).pin_memory()
+    h_out.fill_(float("nan"))
     st.decode_step_host(hx, h_out, 256, advance=1)
     assert torch.equal(h_out, ref.cpu())
     assert all(torch.equal(a, b) for a, b in zip(kref, st.k_cache))
