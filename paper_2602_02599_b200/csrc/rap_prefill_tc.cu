@@ -76,6 +76,27 @@ __device__ __forceinline__ void pt_mma_ts(uint32_t tmem_d, uint32_t tmem_a, uint
       "r"(tmem_a), "l"(bdesc), "r"(idesc), "r"(acc)
       : "memory");
 }
+// The same two with the descriptors given as (low word, high word): the low word carries the start address (in 16-byte
+// units, 14 bits), so walking a ring or the k-steps of a tile is one 32-bit add on it.
+__device__ __forceinline__ void pt_mma2(uint32_t tmem_d, uint32_t a_lo, uint32_t b_lo, uint32_t hi, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+      "mov.b64 da, {%1, %3};\n\t"
+      "mov.b64 db, {%2, %3};\n\t"
+      "setp.ne.b32 p, %5, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t}" ::"r"(tmem_d),
+      "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc), "r"(acc)
+      : "memory");
+}
+__device__ __forceinline__ void pt_mma_ts2(uint32_t tmem_d, uint32_t tmem_a, uint32_t b_lo, uint32_t hi, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .b64 db;\n\t"
+      "mov.b64 db, {%2, %3};\n\t"
+      "setp.ne.b32 p, %5, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n\t}" ::"r"(tmem_d),
+      "r"(tmem_a), "r"(b_lo), "r"(hi), "r"(idesc), "r"(acc)
+      : "memory");
+}
 __device__ __forceinline__ void pt_commit(uint32_t bar) {
   asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
@@ -250,12 +271,37 @@ __global__ void __launch_bounds__(P2_THREADS, 1) prefill_tc_kernel(const PtParam
     }
   }
   const int kw = p.P2 >> 1;                          // 4-byte words per q / K row
-  for (int r = warp; r < 256; r += P2_THREADS / 32) {
-    const int t = q0 + r;
-    if (t < p.T) {
-      const uint32_t* src = reinterpret_cast<const uint32_t*>(p.q + (((size_t)b * p.T + t) * p.Hq + g) * p.P2);
-      unsigned char* qd = q_s + (r >> 7) * P2_Q_BYTES;
-      for (int w = lane; w < kw; w += 32) *reinterpret_cast<uint32_t*>(qd + pt_off(r & 127, 2 * w, 128)) = src[w];
+  {
+    // a warp takes rows warp, warp + 14, ...; the loads of ten rows are in flight before the first store (one round
+    // trip to memory per batch instead of one per row)
+    constexpr int NWARP = P2_THREADS / 32, QB = 10;
+    const size_t q_row = (size_t)p.Hq * p.P2 / 2;    // words between consecutive queries of one head
+    const uint32_t* qsrc = reinterpret_cast<const uint32_t*>(p.q + (((size_t)b * p.T + q0) * p.Hq + g) * p.P2);
+#pragma unroll 1
+    for (int r0 = warp; r0 < 256; r0 += NWARP * QB) {
+      uint32_t qv[QB][2];
+#pragma unroll
+      for (int u = 0; u < QB; ++u) {
+        const int r = r0 + NWARP * u;
+        const bool ok = r < 256 && q0 + r < p.T;
+#pragma unroll
+        for (int sl = 0; sl < 2; ++sl) {
+          const int w = lane + 32 * sl;
+          qv[u][sl] = (ok && w < kw) ? __ldg(qsrc + (size_t)r * q_row + w) : 0u;
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < QB; ++u) {
+        const int r = r0 + NWARP * u;
+        if (r < 256 && q0 + r < p.T) {
+          unsigned char* qd = q_s + (r >> 7) * P2_Q_BYTES;
+#pragma unroll
+          for (int sl = 0; sl < 2; ++sl) {
+            const int w = lane + 32 * sl;
+            if (w < kw) *reinterpret_cast<uint32_t*>(qd + pt_off(r & 127, 2 * w, 128)) = qv[u][sl];
+          }
+        }
+      }
     }
   }
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -338,16 +384,24 @@ __global__ void __launch_bounds__(P2_THREADS, 1) prefill_tc_kernel(const PtParam
     // arriving in step (after the buffer was filled), so the phases stay aligned.
     if (lane == 0) {
       const int Y = warp - 8, n_y = nt[Y];
-      const uint32_t qx = pt_smem(q_s + Y * P2_Q_BYTES);
       const uint32_t tmem_sy = tmem_base + 128u * (uint32_t)Y, tmem_oy = tmem_base + 256u + 128u * (uint32_t)Y;
-      auto issue_s = [&](int tile) {
-        const uint32_t kb = pt_smem(k_s + (tile % P2_STAGES) * P2_KV_BYTES);
-        const uint32_t td = tmem_sy + 64u * (uint32_t)(tile & 1);
+      // This lane's instructions are the serial part of a key tile, so everything that does not change is worked out
+      // here: the descriptors' high word, the low words of Q's k-steps, of the first K and V buffers; ring positions
+      // and phases are counters, not divisions.
+      constexpr uint32_t DESC_HI = (1024u >> 4) | (1u << 14) | (2u << 29);
+      constexpr uint32_t BUF16 = (uint32_t)P2_KV_BYTES >> 4;
+      uint32_t q_lo[DK];
+#pragma unroll
+      for (int ks = 0; ks < DK; ++ks)
+        q_lo[ks] = (((pt_smem(q_s + Y * P2_Q_BYTES) + (uint32_t)((ks >> 2) * 16384 + (ks & 3) * 32)) & 0x3FFFFu) >> 4) | (1u << 16);
+      const uint32_t k_lo0 = ((pt_smem(k_s) & 0x3FFFFu) >> 4) | (1u << 16);
+      const uint32_t v_lo0 = ((pt_smem(v_s) & 0x3FFFFu) >> 4) | ((8192u >> 4) << 16);
+      auto issue_s = [&](uint32_t kbuf, uint32_t sbuf) {     // S into buffer sbuf from K buffer kbuf
+        const uint32_t kb = k_lo0 + kbuf * BUF16, td = tmem_sy + 64u * sbuf;
 #pragma unroll
         for (int ks = 0; ks < DK; ++ks)
-          pt_mma(td, pt_desc(qx + (uint32_t)((ks >> 2) * 16384 + (ks & 3) * 32)),
-                 pt_desc(kb + (uint32_t)((ks >> 2) * 8192 + (ks & 3) * 32)), IDESC_S, ks > 0 ? 1u : 0u);
-        pt_commit(bar_s + 8 * (2 * Y + (tile & 1)));
+          pt_mma2(td, q_lo[ks], kb + (uint32_t)(((ks >> 2) * 8192 + (ks & 3) * 32) >> 4), DESC_HI, IDESC_S, ks > 0 ? 1u : 0u);
+        pt_commit(bar_s + 8 * (2 * Y + sbuf));
       };
       auto release = [&](uint32_t bar, bool issued) {   // after MMAs: when they complete; otherwise at once
         if (issued) pt_commit(bar);
@@ -357,32 +411,35 @@ __global__ void __launch_bounds__(P2_THREADS, 1) prefill_tc_kernel(const PtParam
       if (ok) {
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        if (n_y > 0) issue_s(0);
+        if (n_y > 0) issue_s(0, 0);
         release(bar_ek, n_y > 0);
       }
+      uint32_t kbuf = 1, kpar = 0;       // ring position and phase of K tile + 1
+      uint32_t vbuf = 0, vpar = 0;       // of V tile
       for (int tile = 0; ok && tile < n_max; ++tile) {
+        const uint32_t sb = (uint32_t)tile & 1u;
         if (tile + 1 < n_max) {
-          const int kbuf = (tile + 1) % P2_STAGES;
-          if (!wait(bar_fk + 8 * kbuf, ((tile + 1) / P2_STAGES) & 1)) { ok = false; break; }
+          if (!wait(bar_fk + 8 * kbuf, kpar)) { ok = false; break; }
           asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-          if (tile + 1 < n_y) issue_s(tile + 1);
+          if (tile + 1 < n_y) issue_s(kbuf, sb ^ 1u);
           release(bar_ek + 8 * kbuf, tile + 1 < n_y);
+          if (++kbuf == P2_STAGES) { kbuf = 0; kpar ^= 1u; }
         }
-        const int vbuf = tile % P2_STAGES;
-        if (!wait(bar_fv + 8 * vbuf, (tile / P2_STAGES) & 1)) { ok = false; break; }
+        if (!wait(bar_fv + 8 * vbuf, vpar)) { ok = false; break; }
         if (tile < n_y) {
-          if (!wait(bar_p + 8 * (2 * Y + (tile & 1)), (tile >> 1) & 1)) { ok = false; break; }
+          if (!wait(bar_p + 8 * (2 * Y + sb), (uint32_t)(tile >> 1) & 1u)) { ok = false; break; }
           asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-          const uint32_t vb = pt_smem(v_s + vbuf * P2_KV_BYTES);
+          const uint32_t vb = v_lo0 + vbuf * BUF16, ta = tmem_sy + 64u * sb;
 #pragma unroll
           for (int ks = 0; ks < P2_KT / 16; ++ks)   // A = P in tensor memory, over the S columns it was computed from
-            pt_mma_ts(tmem_oy, tmem_sy + 64u * (uint32_t)(tile & 1) + 8u * (uint32_t)ks, pt_desc_n2(vb + (uint32_t)ks * 2048u),
-                      IDESC_O, (tile > 0 || ks > 0) ? 1u : 0u);
+            pt_mma_ts2(tmem_oy, ta + 8u * (uint32_t)ks, vb + (uint32_t)(ks * 2048 >> 4), DESC_HI, IDESC_O,
+                       (tile > 0 || ks > 0) ? 1u : 0u);
           pt_commit(bar_o + 8 * Y);
         }
         release(bar_ev + 8 * vbuf, tile < n_y);
+        if (++vbuf == P2_STAGES) { vbuf = 0; vpar ^= 1u; }
       }
       // every MMA issued above has completed before tensor memory is released
       pt_commit(bar_end + 8 * Y);
@@ -501,24 +558,36 @@ __global__ void __launch_bounds__(P2_THREADS, 1) prefill_tc_kernel(const PtParam
     atomicCAS(&p.status[0], 0, (int)RAP_ETIMEOUT);
     p.status[1] = 0x60000000 | (qb & 0xffffff);
   }
+  // The tiles are free now (every MMA has completed, every copy has landed).  A thread owns a query row in tensor
+  // memory, but a row of the output is contiguous in global memory: the normalised rows go through shared memory
+  // (rows of NVP + 1 floats: the row-per-thread stores hit 32 banks) and leave as whole rows, one warp per row.
+  float* o_s = reinterpret_cast<float*>(smem);
+  constexpr int OS = NVP + 1;
+  static_assert(256 * OS * 4 <= P2_SMEM - P2_TAIL, "the output tile fits the freed tiles");
   if (warp < 8 && !timed_out && nt[X] > 0) {
-    const int t = q0 + 128 * X + row;
     if constexpr (LSUM) l_run = __uint_as_float(pt_ld1(tmem_o + lane_off + (uint32_t)p.vs));
     const float inv = l_run > 0.f ? 1.f / l_run : 0.f;
-    float* dst = p.out + (((size_t)b * p.T + min(t, p.T - 1)) * p.Hq + g) * p.dv;
+    float* orow = o_s + (size_t)(128 * X + row) * OS;
 #pragma unroll 1
     for (int c0 = 0; c0 < NVP; c0 += 32) {
       uint32_t oc[32];
       pt_ld32(tmem_o + lane_off + c0, oc);
-      if (t < p.T) {
 #pragma unroll
-        for (int j = 0; j < 32; ++j)
-          if (c0 + j < p.dv) dst[c0 + j] = __uint_as_float(oc[j]) * inv;
-      }
+      for (int j = 0; j < 32; ++j) orow[c0 + j] = __uint_as_float(oc[j]) * inv;
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   }
   __syncthreads();
+  if (!timed_out) {
+    for (int r = warp; r < 256; r += P2_THREADS / 32) {
+      const int t = q0 + r;
+      if (t < p.T && nt[r >> 7] > 0) {
+        float* dst = p.out + (((size_t)b * p.T + t) * p.Hq + g) * p.dv;
+        const float* src = o_s + (size_t)r * OS;
+        for (int c = lane; c < p.dv; c += 32) dst[c] = src[c];
+      }
+    }
+  }
   if (warp == 8) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
