@@ -1,44 +1,41 @@
 // tcgen05 version of rap_prefill_attn: causal attention of a block of T new tokens per sequence over the
 // reduced dims (Eq. 2 for every t of the block; 2P retained K dims, d_v' retained V channels, scale
 // 1/sqrt(D)).  One CTA (one per SM, 448 threads) handles 256 consecutive queries of one query head as two query
-// tiles A and B of 128, and walks 128-key tiles up to each tile's causal limit:
-//   S_X    = Q_X K^T    tcgen05.mma (M = 128 queries, N = 128 keys, K = 2P in steps of 16), accumulator in TMEM
-//   P_X    = 2^(S - m)  softmax warp group X (warps 0-3: A, 4-7: B), one thread per query row, two passes over the S
-//                       row in tensor memory (maximum; then weights, 64 keys at a time), causal mask only on the
-//                       tiles that reach the diagonal, lazy running maximum, P as bf16 into shared memory in two
-//                       halves of 64 keys
-//   O_X   += P_X V      tcgen05.mma per half (A = P half, N = d_v' rounded up to 32, K = 64 keys), accumulating in TMEM
-//                       across the key tiles; a warp rescales its 32 accumulator rows (tcgen05.ld / st) only in the
-//                       rare tile where the lazy maximum moved.
-// The shapes follow what one tcgen05.mma costs on this part: about 71 cycles with both operands in shared memory for
-// any N up to 128 (N = 256: 124), about 125 with A in tensor memory.  So S takes 128 keys per instruction, and P goes
-// through shared memory rather than tensor memory.  The issuing lane of a query tile orders its work as
-// PV(first half of t), S(t + 1), PV(second half of t): S(t + 1) is issued as soon as the softmax threads have read
-// S(t) for the last time and runs while they finish the second half's weights.
+// tiles A and B of 128, and walks 64-key tiles up to each tile's causal limit:
+//   S_X    = Q_X K^T    tcgen05.mma (M = 128 queries, N = 64 keys, K = 2P in steps of 16), accumulator in TMEM,
+//                       double buffered per query tile: S of key tile t + 1 is issued before P of t is waited for
+//   P_X    = 2^(S - m)  softmax warp group X (warps 0-3: A, 4-7: B), one thread per query row: the S row in
+//                       registers with one TMEM round trip, causal mask only on the tiles that reach the diagonal,
+//                       lazy running maximum, P as packed bf16 back into tensor memory over the S columns it
+//                       came from
+//   O_X   += P_X V      tcgen05.mma with A = P in tensor memory (N = d_v' rounded up to 32, K = 64 keys),
+//                       accumulating in TMEM across the key tiles; a warp rescales its 32 accumulator rows
+//                       (tcgen05.ld / st) only in the rare tile where the lazy maximum moved.
 // Where the N of the second MMA has a spare column (d_v' below its multiple of 32: every pruned shape), that column of
 // every staged V tile holds the constant one, so the tensor core accumulates the row sum of the weights next to O --
 // from the very bf16 weights it multiplies, rescaled with O when the maximum moves -- and the softmax threads keep no
 // sum at all (LSUM; a third of their instructions per weight otherwise).
-// Cache rows are not multiples of 16 bytes, so TMA tensor maps cannot describe them: four producer warps (10-13)
-// stage the tiles by hand (4-byte cp.async), K(t + 1) and V(t) in turn, in the 128-byte-swizzled layouts the MMA
-// descriptors expect (K as stored = K-major; V as stored = the N-major form of the B operand, so nothing is
-// transposed); rows past the sequence end and pad columns are zeros.  The copies' completion arrives on the buffer's
-// mbarrier by itself; the consumer issues the proxy fence.  The roles meet only on mbarriers; every wait is bounded
-// and gives up early once another role has given up.  Lane 0 of warp 8 issues the MMAs of query tile A, lane 0 of
-// warp 9 those of B.
+// While one group runs its softmax the tensor core works for the other, and a staged K / V tile serves 256 queries.
+// Cache rows are not multiples of 16 bytes, so TMA tensor maps cannot describe them: four producer warps (10-11: K,
+// 12-13: V) stage the tiles by hand (4-byte cp.async) into rings of five buffers each, in the 128-byte-swizzled
+// layouts the MMA descriptors expect (K as stored = K-major; V as stored = the N-major form of the B operand, so
+// nothing is transposed); rows past the sequence end and pad columns are zeros.  The copies' completion arrives on
+// the buffer's mbarrier by itself; the consumer issues the proxy fence.  The roles meet only on mbarriers; every wait
+// is bounded and gives up early once another role has given up.  Lane 0 of warp 8 issues the MMAs of query tile A,
+// lane 0 of warp 9 those of B.
 #include <math.h>
 
 #include "rap_internal.h"
 
 namespace {
 
-constexpr int P2_KT = 128;                             // keys per tile
+constexpr int P2_KT = 64;                              // keys per tile
 constexpr int P2_THREADS = 448;
-constexpr int P2_NK = 1, P2_NV = 2;                    // K buffers, V buffers
-constexpr int P2_COL = 128 * 128;                      // one atom column: 128 rows of 64 elements (128 bytes)
-constexpr int P2_TILE = 2 * P2_COL;                    // [128 rows][<=128 elements]: Q_X, a K tile, a V tile
+constexpr int P2_STAGES = 5;                           // K buffers and V buffers
+constexpr int P2_Q_BYTES = 2 * 128 * 128;              // [128 queries][<=128 dims]: two 64-element atom columns
+constexpr int P2_KV_BYTES = 2 * P2_KT * 128;           // [64 keys][<=128 dims or channels]
 constexpr int P2_TAIL = 320;                           // mbarriers, TMEM address, give-up flag
-constexpr int P2_SMEM = (2 + 2 + P2_NK + P2_NV) * P2_TILE + P2_TAIL;   // Q_A Q_B, P_A P_B, K ring, V ring
+constexpr int P2_SMEM = 2 * P2_Q_BYTES + 2 * P2_STAGES * P2_KV_BYTES + P2_TAIL;
 constexpr uint32_t PT_WAIT_HINT_NS = 20000;      // a parked probe returns at the phase change or after this long
 constexpr uint32_t PT_WAIT_LIMIT = 1u << 15;    // probes before a wait gives up (well under a second)
 
@@ -56,10 +53,6 @@ __device__ __forceinline__ bool pt_try_wait(uint32_t bar, uint32_t parity) {
       : "=r"(ok) : "r"(bar), "r"(parity), "r"(PT_WAIT_HINT_NS) : "memory");
   return ok != 0;
 }
-// Shared-memory operand descriptors are passed as (low word, high word).  128-byte swizzle, 8-row groups 1024 bytes
-// apart: the high word is the same for every operand here; the low word carries the start address (in 16-byte units,
-// 14 bits) and the leading offset (bits 16-29), so walking a ring or the k-steps of a tile is one 32-bit add on it.
-constexpr uint32_t PT_DESC_HI = (1024u >> 4) | (1u << 14) | (2u << 29);
 // one probe that never parks the thread
 __device__ __forceinline__ bool pt_test_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
@@ -70,6 +63,31 @@ __device__ __forceinline__ bool pt_test_wait(uint32_t bar, uint32_t parity) {
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
+// K-major operand tile, 128-byte swizzle: 8-row groups 1024 bytes apart (see rap_proj_tc.cu)
+__device__ __forceinline__ uint64_t pt_desc(uint32_t addr) {
+  const uint32_t lo = ((addr & 0x3FFFFu) >> 4) | (1u << 16);
+  const uint32_t hi = (1024u >> 4) | (1u << 14) | (2u << 29);
+  return ((uint64_t)hi << 32) | lo;
+}
+__device__ __forceinline__ void pt_mma(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(tmem_d),
+      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc)
+      : "memory");
+}
+// the same with the A operand in tensor memory (row = lane, two bf16 K elements per 32-bit column)
+__device__ __forceinline__ void pt_mma_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}" ::"r"(tmem_d),
+      "r"(tmem_a), "l"(bdesc), "r"(idesc), "r"(acc)
+      : "memory");
+}
+// The same two with the descriptors given as (low word, high word): the low word carries the start address (in 16-byte
+// units, 14 bits), so walking a ring or the k-steps of a tile is one 32-bit add on it.
 __device__ __forceinline__ void pt_mma2(uint32_t tmem_d, uint32_t a_lo, uint32_t b_lo, uint32_t hi, uint32_t idesc, uint32_t acc) {
   asm volatile(
       "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
@@ -78,6 +96,15 @@ __device__ __forceinline__ void pt_mma2(uint32_t tmem_d, uint32_t a_lo, uint32_t
       "setp.ne.b32 p, %5, 0;\n\t"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t}" ::"r"(tmem_d),
       "r"(a_lo), "r"(b_lo), "r"(hi), "r"(idesc), "r"(acc)
+      : "memory");
+}
+__device__ __forceinline__ void pt_mma_ts2(uint32_t tmem_d, uint32_t tmem_a, uint32_t b_lo, uint32_t hi, uint32_t idesc, uint32_t acc) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t.reg .b64 db;\n\t"
+      "mov.b64 db, {%2, %3};\n\t"
+      "setp.ne.b32 p, %5, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n\t}" ::"r"(tmem_d),
+      "r"(tmem_a), "r"(b_lo), "r"(hi), "r"(idesc), "r"(acc)
       : "memory");
 }
 __device__ __forceinline__ void pt_commit(uint32_t bar) {
@@ -134,33 +161,26 @@ __device__ __forceinline__ float pt_ex2(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
-// The special-function unit delivers 16 exponentials per cycle and SM; a 128 x 128 block of weights would keep it busy
-// for longer than the two MMAs of the block take.  So a part of the weights gets its 2^x on the FMA pipe instead, two
-// at a time in packed fp32: n = round(x) through the 1.5 * 2^23 trick, f = x - n in [-0.5, 0.5], a cubic for 2^f
-// (fitted for the relative error: 7.5e-5, a thirtieth of the bf16 rounding that follows), n added to the exponent field;
-// anything below -126 comes out as if it were -126 (about 1e-38).
-constexpr uint32_t PT_POLY_PAIRS = 0x52u;          // of every 8 pairs of weights, pairs 1, 4 and 6 take this path
-__device__ __forceinline__ uint64_t pt_pack2(float a, float b) {
-  uint64_t r;
-  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b));
-  return r;
+// byte offset of element (row, col) of a K-major bf16 tile of `rows` rows: 64-column atom columns, rows of
+// 128 bytes whose 16-byte chunks are XORed with row % 8
+__device__ __forceinline__ uint32_t pt_off(int row, int col, int rows) {
+  const int ac = col >> 6, c = col & 63;
+  return (uint32_t)(ac * rows * 128 + (row >> 3) * 1024 + (row & 7) * 128 + ((((c >> 3) ^ (row & 7))) << 4) + ((c & 7) << 1));
 }
-__device__ __forceinline__ uint64_t pt_fma2(uint64_t a, uint64_t b, uint64_t c) {
-  uint64_t r;
-  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
-  return r;
+
+// N-major operand tile (B = V as stored, [key][channel]), 128-byte swizzle: an atom is 8 keys x 64 channels
+// (key rows of 128 bytes, 16-byte chunks XORed with key % 8); atoms of consecutive 8-key groups are 1024 bytes
+// apart (stride offset), the two 64-channel atom columns of a 64-key tile 8 KB apart (leading offset).
+__device__ __forceinline__ uint64_t pt_desc_n2(uint32_t addr) {
+  const uint32_t lo = ((addr & 0x3FFFFu) >> 4) | ((8192u >> 4) << 16);
+  const uint32_t hi = (1024u >> 4) | (1u << 14) | (2u << 29);
+  return ((uint64_t)hi << 32) | lo;
 }
-__device__ __forceinline__ uint64_t pt_add2(uint64_t a, uint64_t b) {
-  uint64_t r;
-  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
-  return r;
-}
-// Byte offset of 4-byte word w of row r in a tile of 128 rows: 64-element (128-byte) atom columns P2_COL apart, rows of
-// 128 bytes whose 16-byte chunks are XORed with r % 8.  The same arrangement serves the K-major tiles (Q, K, P: a row
-// is a query or a key, the columns are dims or keys) and the N-major V tile (a row is a key, the columns are channels;
-// 8-key atoms 1024 bytes apart, the two 64-channel atom columns P2_COL apart).
-__device__ __forceinline__ uint32_t pt_word(int r, int w) {
-  return (uint32_t)((w >> 5) * P2_COL + r * 128 + ((((w & 31) >> 2) ^ (r & 7)) << 4) + ((w & 3) << 2));
+// Byte offset inside a 64-row tile row of its byte e: 64-element (128-byte) atom columns 8 KB apart, 16-byte chunks
+// XORed with row % 8 (the layout is the same for the K-major K tile and the N-major V tile).
+__device__ __forceinline__ uint32_t pt_swz2(int e, int r7) {
+  const int w = e >> 2;
+  return (uint32_t)(((w >> 5) << 13) + ((((w & 31) >> 2) ^ r7) << 4) + ((w & 3) << 2));
 }
 struct PtParams {
   const __nv_bfloat16* q;     // [B][T][Hq][P2]
@@ -197,17 +217,15 @@ __global__ void __launch_bounds__(P2_THREADS, 1) prefill_tc_kernel(const PtParam
   extern __shared__ unsigned char pt_raw[];
   unsigned char* smem = pt_raw + ((1024u - (pt_smem(pt_raw) & 1023u)) & 1023u);
   unsigned char* q_s = smem;                                   // Q_A, Q_B
-  unsigned char* p_s = q_s + 2 * P2_TILE;                      // P_A, P_B: atom column h holds keys [64h, 64h + 64)
-  unsigned char* k_s = p_s + 2 * P2_TILE;                      // ring of K tiles
-  unsigned char* v_s = k_s + P2_NK * P2_TILE;                  // ring of V tiles (N-major)
-  unsigned char* tail = v_s + P2_NV * P2_TILE;
-  const uint32_t bar_fk = pt_smem(tail), bar_ek = bar_fk + 8 * P2_NK, bar_fv = bar_ek + 8 * P2_NK, bar_ev = bar_fv + 8 * P2_NV,
-                 bar_s = bar_ev + 8 * P2_NV /* [X] S complete */, bar_sf = bar_s + 16 /* [X] S read for the last time */,
-                 bar_p = bar_sf + 16 /* [X][half] P written */, bar_o = bar_p + 32 /* [X] O updated */, bar_end = bar_o + 16 /* [X] */;
-  constexpr int N_BAR = 2 * P2_NK + 2 * P2_NV + 12;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 8 * N_BAR);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 8 * N_BAR + 4);
-  static_assert(8 * N_BAR + 8 <= P2_TAIL, "barriers and flags fit the tail");
+  unsigned char* k_s = q_s + 2 * P2_Q_BYTES;                   // ring of K tiles
+  unsigned char* v_s = k_s + P2_STAGES * P2_KV_BYTES;          // ring of V tiles (N-major)
+  unsigned char* tail = v_s + P2_STAGES * P2_KV_BYTES;
+  const uint32_t bar_fk = pt_smem(tail), bar_ek = bar_fk + 8 * P2_STAGES, bar_fv = bar_ek + 8 * P2_STAGES,
+                 bar_ev = bar_fv + 8 * P2_STAGES, bar_s = bar_ev + 8 * P2_STAGES /* [X][2] */, bar_p = bar_s + 32 /* [X][2] */,
+                 bar_o = bar_p + 32 /* [X] */, bar_end = bar_o + 16 /* [X] */;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tail + 32 * P2_STAGES + 96);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tail + 32 * P2_STAGES + 100);
+  static_assert(32 * P2_STAGES + 104 <= P2_TAIL, "barriers and flags fit the tail");
 
   // the blocks with the most key tiles (the last queries) are dispatched first, the short ones fill the tail
   const int qb = (int)gridDim.z - 1 - (int)blockIdx.z, g = blockIdx.x, b = blockIdx.y;
@@ -228,22 +246,21 @@ __global__ void __launch_bounds__(P2_THREADS, 1) prefill_tc_kernel(const PtParam
   const __nv_bfloat16* vg = p.v + ((size_t)b * p.Hkv + h) * (size_t)p.S_cap * p.vs;
 
   if (tid == 0) {
-    for (int i = 0; i < P2_NK; ++i) {
-      pt_mbar_init(bar_fk + 8 * i, 128);             // the copies of the 128 producer threads
+    for (int i = 0; i < P2_STAGES; ++i) {
+      pt_mbar_init(bar_fk + 8 * i, 64);
       pt_mbar_init(bar_ek + 8 * i, 2);               // both MMA-issuing lanes release a buffer
-    }
-    for (int i = 0; i < P2_NV; ++i) {
-      pt_mbar_init(bar_fv + 8 * i, 128);
+      pt_mbar_init(bar_fv + 8 * i, 64);
       pt_mbar_init(bar_ev + 8 * i, 2);
     }
-    for (int X = 0; X < 2; ++X) {
-      pt_mbar_init(bar_s + 8 * X, 1);
-      pt_mbar_init(bar_sf + 8 * X, 128);
-      pt_mbar_init(bar_p + 16 * X, 128);
-      pt_mbar_init(bar_p + 16 * X + 8, 128);
-      pt_mbar_init(bar_o + 8 * X, 1);
-      pt_mbar_init(bar_end + 8 * X, 1);
+    for (int i = 0; i < 4; ++i) {
+      pt_mbar_init(bar_s + 8 * i, 1);
+      // "P written" has one barrier per S buffer: the softmax may be a tile ahead of the lane that waits for it, and
+      // with a single barrier two completed phases would look like none
+      pt_mbar_init(bar_p + 8 * i, 128);
     }
+    for (int X = 0; X < 2; ++X) pt_mbar_init(bar_o + 8 * X, 1);
+    pt_mbar_init(bar_end, 1);
+    pt_mbar_init(bar_end + 8, 1);
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
@@ -256,10 +273,10 @@ __global__ void __launch_bounds__(P2_THREADS, 1) prefill_tc_kernel(const PtParam
   for (int i = tid; i < (P2_SMEM - P2_TAIL) / 16; i += P2_THREADS) reinterpret_cast<uint4*>(smem)[i] = make_uint4(0, 0, 0, 0);
   __syncthreads();
   if constexpr (LSUM) {
-    // the ones column: channel p.vs of all key rows of every V buffer (the producers never write that element)
-    for (int i = tid; i < P2_NV * P2_KT; i += P2_THREADS) {
+    // the ones column: channel p.vs of all 64 key rows of every V buffer (the producers never write that element)
+    for (int i = tid; i < P2_STAGES * P2_KT; i += P2_THREADS) {
       const int buf = i / P2_KT, r = i - buf * P2_KT, c = p.vs;
-      unsigned char* e = v_s + buf * P2_TILE + pt_word(r, c >> 1) + 2 * (c & 1);
+      unsigned char* e = v_s + buf * P2_KV_BYTES + r * 128 + pt_swz2(4 * (c >> 1), r & 7) + 2 * (c & 1);
       *reinterpret_cast<__nv_bfloat16*>(e) = __float2bfloat16(1.0f);
     }
   }
@@ -287,11 +304,11 @@ __global__ void __launch_bounds__(P2_THREADS, 1) prefill_tc_kernel(const PtParam
       for (int u = 0; u < QB; ++u) {
         const int r = r0 + NWARP * u;
         if (r < 256 && q0 + r < p.T) {
-          unsigned char* qd = q_s + (r >> 7) * P2_TILE;
+          unsigned char* qd = q_s + (r >> 7) * P2_Q_BYTES;
 #pragma unroll
           for (int sl = 0; sl < 2; ++sl) {
             const int w = lane + 32 * sl;
-            if (w < kw) *reinterpret_cast<uint32_t*>(qd + pt_word(r & 127, w)) = qv[u][sl];
+            if (w < kw) *reinterpret_cast<uint32_t*>(qd + pt_off(r & 127, 2 * w, 128)) = qv[u][sl];
           }
         }
       }
@@ -301,12 +318,12 @@ __global__ void __launch_bounds__(P2_THREADS, 1) prefill_tc_kernel(const PtParam
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-  const uint32_t tmem_base = *tmem_slot;             // S_X: columns 128 X; O_X: columns 256 + 128 X
+  const uint32_t tmem_base = *tmem_slot;             // S_X(t): columns 128 X + 64 (t & 1); O_X: columns 256 + 128 X
   constexpr uint32_t IDESC_S = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(P2_KT >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
   constexpr uint32_t IDESC_O = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(NVP >> 3) << 17) |
                                ((uint32_t)(128 >> 4) << 24);
   auto wait = [&](uint32_t bar, uint32_t parity) -> bool {
-    if (pt_test_wait(bar, parity)) return true;        // the usual case: the phase is long over
+    if (pt_test_wait(bar, parity)) return true;        // the usual case: the phase is long over (a parking probe costs ~250 cycles even then)
     for (uint32_t i = 0; i < PT_WAIT_LIMIT; ++i) {
       if (pt_try_wait(bar, parity)) return true;
       if ((i & 15u) == 15u && *abort_flag) return false;
@@ -321,138 +338,119 @@ __global__ void __launch_bounds__(P2_THREADS, 1) prefill_tc_kernel(const PtParam
   const uint32_t lane_off = (uint32_t)((warp & 3) * 32) << 16;
   const uint32_t tmem_o = tmem_base + 256 + 128 * X;
   if (warp >= 10) {
-    // ================= producers: warps 10-13 stage K(0), then V(t) and K(t + 1) in turn, tiles of 128 rows =================
-    const int pw = warp - 10;                         // rows pw, pw + 4, ...
-    uint32_t swz[2][2];                               // [row % 8 = pw, pw + 4][word lane, lane + 32]: offset inside the row
+    // ================= producers: warps 10-11 stage K, warps 12-13 stage V, in order, tiles of 64 rows =================
+    const bool is_v = warp >= 12;
+    const int pw = (warp - 10) & 1;
+    const int rowlen = is_v ? p.vs : p.P2;            // even in both cases
+    const unsigned char* src0 = reinterpret_cast<const unsigned char*>(is_v ? vg : kg);
+    unsigned char* ring = is_v ? v_s : k_s;
+    const uint32_t bar_f = is_v ? bar_fv : bar_fk, bar_e = is_v ? bar_ev : bar_ek;
+    uint32_t swz[4][2];
+    int nb[2];                                        // this lane's words of a row: 4 bytes each, or none
 #pragma unroll
-    for (int a = 0; a < 2; ++a)
+    for (int sl = 0; sl < 2; ++sl) {
+      const int w = lane + 32 * sl;
+      nb[sl] = 2 * rowlen - 4 * w >= 4 ? 4 : 0;
 #pragma unroll
-      for (int sl = 0; sl < 2; ++sl) swz[a][sl] = pt_word(pw + 4 * a, lane + 32 * sl) - (uint32_t)(pw + 4 * a) * 128u;
-    auto fill = [&](const __nv_bfloat16* base, int rowlen, int tile, unsigned char* dst, uint32_t bar_f) {
-      const unsigned char* src0 = reinterpret_cast<const unsigned char*>(base);
-      const bool one = 2 * rowlen - 4 * lane >= 4, two = 2 * rowlen - 4 * (lane + 32) >= 4;   // this lane's words of a row
+      for (int c = 0; c < 4; ++c) swz[c][sl] = pt_swz2(4 * w, (pw + 2 * c) & 7);
+    }
+    int stg = 0, use = 0;
+    for (int tile = 0; tile < n_max; ++tile) {
       const int j0 = tile * P2_KT;
-      const uint32_t du = pt_smem(dst);
+      if (use > 0 && !wait(bar_e + 8 * stg, (use - 1) & 1)) break;
+      const uint32_t du = pt_smem(ring + stg * P2_KV_BYTES);
       const int rows_ok = min(P2_KT, n_valid - j0);
       const unsigned char* tsrc = src0 + (size_t)j0 * (size_t)(2 * rowlen);
       if (rows_ok == P2_KT) {
         // a full tile (all but the last one of a sequence): no predicates, running pointers
         const unsigned char* sp = tsrc + (size_t)pw * (size_t)(2 * rowlen) + 4 * lane;
         uint32_t db = du + (uint32_t)pw * 128u;
+        const bool one = nb[0] > 0, two = nb[1] > 0;
 #pragma unroll 4
-        for (int i = 0; i < P2_KT / 4; ++i) {
-          if (one) pt_cp4(db + swz[i & 1][0], sp, 4);
-          if (two) pt_cp4(db + swz[i & 1][1], sp + 128, 4);
-          sp += 8 * rowlen;                            // four rows on
-          db += 512;
+        for (int i = 0; i < P2_KT / 2; ++i) {
+          if (one) pt_cp4(db + swz[i & 3][0], sp, 4);
+          if (two) pt_cp4(db + swz[i & 3][1], sp + 128, 4);
+          sp += 4 * rowlen;                            // two rows on
+          db += 256;
         }
       } else {
 #pragma unroll 4
-        for (int i = 0; i < P2_KT / 4; ++i) {
-          const int r = pw + 4 * i;
+        for (int i = 0; i < P2_KT / 2; ++i) {
+          const int r = pw + 2 * i;
           const bool ok = r < rows_ok;                 // rows past the end: zero fill, nothing is read
           const uint32_t* src = reinterpret_cast<const uint32_t*>(tsrc + (size_t)(ok ? r : 0) * (size_t)(2 * rowlen));
           const uint32_t rb = du + (uint32_t)r * 128u;
-          if (one) pt_cp4(rb + swz[i & 1][0], src + lane, ok ? 4 : 0);
-          if (two) pt_cp4(rb + swz[i & 1][1], src + lane + 32, ok ? 4 : 0);
+          if (nb[0] > 0) pt_cp4(rb + swz[i & 3][0], src + lane, ok ? 4 : 0);
+          if (nb[1] > 0) pt_cp4(rb + swz[i & 3][1], src + lane + 32, ok ? 4 : 0);
         }
       }
       // the arrival is triggered by the completion of this thread's copies: go on to the next tile
-      asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar_f) : "memory");
-    };
-    int ks_ = 0, ku = 0, vs_ = 0, vu = 0;              // ring positions and how often each ring has wrapped
-    bool ok = true;
-    auto fill_k = [&](int tile) {
-      if (ku > 0 && !wait(bar_ek + 8 * ks_, (uint32_t)(ku - 1) & 1u)) { ok = false; return; }
-      fill(kg, p.P2, tile, k_s + ks_ * P2_TILE, bar_fk + 8 * ks_);
-      if (++ks_ == P2_NK) { ks_ = 0; ++ku; }
-    };
-    auto fill_v = [&](int tile) {
-      if (vu > 0 && !wait(bar_ev + 8 * vs_, (uint32_t)(vu - 1) & 1u)) { ok = false; return; }
-      fill(vg, p.vs, tile, v_s + vs_ * P2_TILE, bar_fv + 8 * vs_);
-      if (++vs_ == P2_NV) { vs_ = 0; ++vu; }
-    };
-    fill_k(0);
-    for (int tile = 0; ok && tile < n_max; ++tile) {
-      fill_v(tile);
-      if (ok && tile + 1 < n_max) fill_k(tile + 1);
+      asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar_f + 8 * stg) : "memory");
+      if (++stg == P2_STAGES) { stg = 0; ++use; }
     }
   } else if (warp >= 8) {
     // ================= MMA issue: lane 0 of warp 8 for query tile A, of warp 9 for query tile B =================
-    // Two issuing lanes halve the serial chain of waits, fences and commits per key tile.  A buffer of the K / V rings
-    // is free when both lanes have committed past it; a lane whose tile needs no more keys keeps arriving in step
-    // (after the buffer was filled), so the phases stay aligned.
+    // Two issuing lanes halve the serial chain of waits, fences, descriptors and commits per key tile.  A buffer of
+    // the K / V rings is free when both lanes have committed past it; a lane whose tile needs no more keys keeps
+    // arriving in step (after the buffer was filled), so the phases stay aligned.
     if (lane == 0) {
       const int Y = warp - 8, n_y = nt[Y];
       const uint32_t tmem_sy = tmem_base + 128u * (uint32_t)Y, tmem_oy = tmem_base + 256u + 128u * (uint32_t)Y;
       // This lane's instructions are the serial part of a key tile, so everything that does not change is worked out
-      // here: the low descriptor words of Q's k-steps, of P's halves, of the first K and V buffers; ring positions and
-      // phases are counters, not divisions.
-      constexpr uint32_t TILE16 = (uint32_t)P2_TILE >> 4, COL16 = (uint32_t)P2_COL >> 4;
+      // here: the descriptors' high word, the low words of Q's k-steps, of the first K and V buffers; ring positions
+      // and phases are counters, not divisions.
+      constexpr uint32_t DESC_HI = (1024u >> 4) | (1u << 14) | (2u << 29);
+      constexpr uint32_t BUF16 = (uint32_t)P2_KV_BYTES >> 4;
       uint32_t q_lo[DK];
 #pragma unroll
       for (int ks = 0; ks < DK; ++ks)
-        q_lo[ks] = (((pt_smem(q_s + Y * P2_TILE) + (uint32_t)((ks >> 2) * P2_COL + (ks & 3) * 32)) & 0x3FFFFu) >> 4) | (1u << 16);
+        q_lo[ks] = (((pt_smem(q_s + Y * P2_Q_BYTES) + (uint32_t)((ks >> 2) * 16384 + (ks & 3) * 32)) & 0x3FFFFu) >> 4) | (1u << 16);
       const uint32_t k_lo0 = ((pt_smem(k_s) & 0x3FFFFu) >> 4) | (1u << 16);
-      const uint32_t p_lo0 = ((pt_smem(p_s + Y * P2_TILE) & 0x3FFFFu) >> 4) | (1u << 16);
-      const uint32_t v_lo0 = ((pt_smem(v_s) & 0x3FFFFu) >> 4) | (COL16 << 16);   // leading offset: the next 64 channels
-      auto issue_s = [&](uint32_t kslot) {
-        const uint32_t kb = k_lo0 + kslot * TILE16;
+      const uint32_t v_lo0 = ((pt_smem(v_s) & 0x3FFFFu) >> 4) | ((8192u >> 4) << 16);
+      auto issue_s = [&](uint32_t kbuf, uint32_t sbuf) {     // S into buffer sbuf from K buffer kbuf
+        const uint32_t kb = k_lo0 + kbuf * BUF16, td = tmem_sy + 64u * sbuf;
 #pragma unroll
         for (int ks = 0; ks < DK; ++ks)
-          pt_mma2(tmem_sy, q_lo[ks], kb + (uint32_t)(((ks >> 2) * P2_COL + (ks & 3) * 32) >> 4), PT_DESC_HI, IDESC_S, ks > 0 ? 1u : 0u);
-        pt_commit(bar_s + 8 * Y);
-      };
-      auto issue_pv = [&](uint32_t vslot, uint32_t half, bool first) {   // O += P[half] V[keys 64 half ...]
-        const uint32_t pa = p_lo0 + half * COL16, vb = v_lo0 + vslot * TILE16 + half * (uint32_t)(64 * 128 >> 4);
-#pragma unroll
-        for (int ks = 0; ks < 4; ++ks)
-          pt_mma2(tmem_oy, pa + (uint32_t)(ks * 32 >> 4), vb + (uint32_t)(ks * 16 * 128 >> 4), PT_DESC_HI, IDESC_O,
-                  (first && ks == 0) ? 0u : 1u);
+          pt_mma2(td, q_lo[ks], kb + (uint32_t)(((ks >> 2) * 8192 + (ks & 3) * 32) >> 4), DESC_HI, IDESC_S, ks > 0 ? 1u : 0u);
+        pt_commit(bar_s + 8 * (2 * Y + sbuf));
       };
       auto release = [&](uint32_t bar, bool issued) {   // after MMAs: when they complete; otherwise at once
         if (issued) pt_commit(bar);
         else asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
       };
-      auto fences = [&]() {
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      };
       bool ok = wait(bar_fk, 0);
       if (ok) {
-        fences();
-        if (n_y > 0) issue_s(0);
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        if (n_y > 0) issue_s(0, 0);
         release(bar_ek, n_y > 0);
       }
-      uint32_t kslot = P2_NK > 1 ? 1u : 0u, kpar = P2_NK > 1 ? 0u : 1u;   // ring position and phase of K tile + 1
-      uint32_t vslot = 0, vpar = 0;                                       // of V tile
+      uint32_t kbuf = 1, kpar = 0;       // ring position and phase of K tile + 1
+      uint32_t vbuf = 0, vpar = 0;       // of V tile
       for (int tile = 0; ok && tile < n_max; ++tile) {
-        const uint32_t tp = (uint32_t)tile & 1u;
-        const bool mine = tile < n_y;
-        if (!wait(bar_fv + 8 * vslot, vpar)) { ok = false; break; }
-        if (mine) {
-          if (!wait(bar_p + 16 * Y, tp)) { ok = false; break; }
-          fences();
-          issue_pv(vslot, 0, tile == 0);
-        }
+        const uint32_t sb = (uint32_t)tile & 1u;
         if (tile + 1 < n_max) {
-          if (!wait(bar_fk + 8 * kslot, kpar)) { ok = false; break; }
-          if (tile + 1 < n_y) {
-            if (!wait(bar_sf + 8 * Y, tp)) { ok = false; break; }     // the softmax threads hold S(tile) in registers
-            fences();
-            issue_s(kslot);
-          }
-          release(bar_ek + 8 * kslot, tile + 1 < n_y);
-          if (++kslot == P2_NK) { kslot = 0; kpar ^= 1u; }
+          if (!wait(bar_fk + 8 * kbuf, kpar)) { ok = false; break; }
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          if (tile + 1 < n_y) issue_s(kbuf, sb ^ 1u);
+          release(bar_ek + 8 * kbuf, tile + 1 < n_y);
+          if (++kbuf == P2_STAGES) { kbuf = 0; kpar ^= 1u; }
         }
-        if (mine) {
-          if (!wait(bar_p + 16 * Y + 8, tp)) { ok = false; break; }
-          fences();
-          issue_pv(vslot, 1, false);
+        if (!wait(bar_fv + 8 * vbuf, vpar)) { ok = false; break; }
+        if (tile < n_y) {
+          if (!wait(bar_p + 8 * (2 * Y + sb), (uint32_t)(tile >> 1) & 1u)) { ok = false; break; }
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          const uint32_t vb = v_lo0 + vbuf * BUF16, ta = tmem_sy + 64u * sb;
+#pragma unroll
+          for (int ks = 0; ks < P2_KT / 16; ++ks)   // A = P in tensor memory, over the S columns it was computed from
+            pt_mma_ts2(tmem_oy, ta + 8u * (uint32_t)ks, vb + (uint32_t)(ks * 2048 >> 4), DESC_HI, IDESC_O,
+                       (tile > 0 || ks > 0) ? 1u : 0u);
           pt_commit(bar_o + 8 * Y);
         }
-        release(bar_ev + 8 * vslot, mine);
-        if (++vslot == P2_NV) { vslot = 0; vpar ^= 1u; }
+        release(bar_ev + 8 * vbuf, tile < n_y);
+        if (++vbuf == P2_STAGES) { vbuf = 0; vpar ^= 1u; }
       }
       // every MMA issued above has completed before tensor memory is released
       pt_commit(bar_end + 8 * Y);
@@ -466,30 +464,24 @@ __global__ void __launch_bounds__(P2_THREADS, 1) prefill_tc_kernel(const PtParam
     const int n_my = nt[X];
     float m_ref = -1.0e30f;
     bool rows_ok = true;
-    const uint32_t trow = tmem_base + 128u * (uint32_t)X + lane_off;
-    unsigned char* prow = p_s + X * P2_TILE + row * 128;       // this row's 128-byte line in either half of P_X
     for (int tile = 0; tile < n_my; ++tile) {
       const int j0 = tile * P2_KT;
-      const uint32_t tp = (uint32_t)tile & 1u;
-      if (!__all_sync(0xffffffffu, wait(bar_s + 8 * X, tp))) { rows_ok = false; break; }
+      const uint32_t trow = tmem_base + 128u * (uint32_t)X + 64u * (uint32_t)(tile & 1) + lane_off;
+      if (!__all_sync(0xffffffffu, wait(bar_s + 8 * (2 * X + (tile & 1)), (tile >> 1) & 1))) { rows_ok = false; break; }
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      const bool interior = j0 + P2_KT - 1 <= start + q0x;   // no key of the tile is masked for any row of the tile
       uint32_t r[64];
-      // ---- first pass over the S row: its maximum ----
+      pt_ld32_nowait(trow, *reinterpret_cast<uint32_t(*)[32]>(r));
+      pt_ld32_nowait(trow + 32, *reinterpret_cast<uint32_t(*)[32]>(r + 32));
+      asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+      const bool interior = j0 + P2_KT - 1 <= start + q0x;   // no key of the tile is masked for any row of the tile
       float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+      if (interior) {
 #pragma unroll
-      for (int hf = 0; hf < 2; ++hf) {
-        pt_ld32_nowait(trow + 64 * hf, *reinterpret_cast<uint32_t(*)[32]>(r));
-        pt_ld32_nowait(trow + 64 * hf + 32, *reinterpret_cast<uint32_t(*)[32]>(r + 32));
-        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-        if (interior) {
+        for (int j = 0; j < 64; ++j) mx4[j & 3] = fmaxf(mx4[j & 3], __uint_as_float(r[j]));
+      } else {
 #pragma unroll
-          for (int j = 0; j < 64; ++j) mx4[j & 3] = fmaxf(mx4[j & 3], __uint_as_float(r[j]));
-        } else {
-#pragma unroll
-          for (int j = 0; j < 64; ++j)
-            if (j0 + 64 * hf + j <= pos) mx4[j & 3] = fmaxf(mx4[j & 3], __uint_as_float(r[j]));
-        }
+        for (int j = 0; j < 64; ++j)
+          if (j0 + j <= pos) mx4[j & 3] = fmaxf(mx4[j & 3], __uint_as_float(r[j]));
       }
       const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * p.qscale;
       float alpha = 1.f;
@@ -499,146 +491,75 @@ __global__ void __launch_bounds__(P2_THREADS, 1) prefill_tc_kernel(const PtParam
         l_run *= alpha;
       }
       const float nm = -m_ref;
-      bool o_waited = false;
+      float ls[4] = {0.f, 0.f, 0.f, 0.f};
+      if (interior) {
+        // no mask
+        // two logits per packed FMA, two weights per packed add
+        uint64_t qs2, nm2, l2[4] = {0ull, 0ull, 0ull, 0ull};
+        asm("mov.b64 %0, {%1, %1};" : "=l"(qs2) : "f"(p.qscale));
+        asm("mov.b64 %0, {%1, %1};" : "=l"(nm2) : "f"(nm));
+#pragma unroll
+        for (int j = 0; j < 64; j += 2) {
+          uint64_t s2, x2, p2;
+          asm("mov.b64 %0, {%1, %2};" : "=l"(s2) : "r"(r[j]), "r"(r[j + 1]));
+          asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(x2) : "l"(s2), "l"(qs2), "l"(nm2));
+          float x0, x1;
+          asm("mov.b64 {%0, %1}, %2;" : "=f"(x0), "=f"(x1) : "l"(x2));
+          const float p0 = pt_ex2(x0), p1 = pt_ex2(x1);
+          const __nv_bfloat162 v2 = __floats2bfloat162_rn(p0, p1);
+          const uint32_t pk = *reinterpret_cast<const uint32_t*>(&v2);
+          if constexpr (!LSUM) {
+            // the row sum takes the rounded weights the second MMA will see (a one-hot row comes out exact)
+            asm("mov.b64 %0, {%1, %2};" : "=l"(p2) : "r"(pk << 16), "r"(pk & 0xffff0000u));
+            asm("add.rn.f32x2 %0, %1, %2;" : "=l"(l2[(j >> 1) & 3]) : "l"(l2[(j >> 1) & 3]), "l"(p2));
+          }
+          r[j >> 1] = pk;
+        }
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          float a0, a1;
+          asm("mov.b64 {%0, %1}, %2;" : "=f"(a0), "=f"(a1) : "l"(l2[k]));
+          ls[k] += a0 + a1;
+        }
+      } else {
+        // diagonal tile: causal mask
+#pragma unroll
+        for (int j = 0; j < 64; j += 2) {
+          float p0 = pt_ex2(fmaf(__uint_as_float(r[j]), p.qscale, nm));
+          float p1 = pt_ex2(fmaf(__uint_as_float(r[j + 1]), p.qscale, nm));
+          if (j0 + j > pos) p0 = 0.f;
+          if (j0 + j + 1 > pos) p1 = 0.f;
+          const __nv_bfloat162 v2 = __floats2bfloat162_rn(p0, p1);
+          const uint32_t pk = *reinterpret_cast<const uint32_t*>(&v2);
+          if constexpr (!LSUM) ls[(j >> 1) & 3] += __uint_as_float(pk << 16) + __uint_as_float(pk & 0xffff0000u);
+          r[j >> 1] = pk;
+        }
+      }
+      l_run += (ls[0] + ls[1]) + (ls[2] + ls[3]);
       if (tile > 0 && __any_sync(0xffffffffu, alpha != 1.f)) {
         // rare: rescale this warp's accumulator rows in tensor memory, once the previous tile's update is in
-        if (!__all_sync(0xffffffffu, wait(bar_o + 8 * X, tp ^ 1u))) { rows_ok = false; break; }
-        o_waited = true;
+        if (!__all_sync(0xffffffffu, wait(bar_o + 8 * X, (tile - 1) & 1))) { rows_ok = false; break; }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        {
 #pragma unroll 1
-        for (int c0 = 0; c0 < NVP; c0 += 32) {
-          uint32_t oc[32];
-          pt_ld32(tmem_o + lane_off + c0, oc);
+          for (int c0 = 0; c0 < NVP; c0 += 32) {
+            uint32_t oc[32];
+            pt_ld32(tmem_o + lane_off + c0, oc);
 #pragma unroll
-          for (int j = 0; j < 32; ++j) oc[j] = __float_as_uint(__uint_as_float(oc[j]) * alpha);
-          pt_st32(tmem_o + lane_off + c0, oc);
+            for (int j = 0; j < 32; ++j) oc[j] = __float_as_uint(__uint_as_float(oc[j]) * alpha);
+            pt_st32(tmem_o + lane_off + c0, oc);
+          }
+          asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
         }
-        asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
-        asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       }
-      // ---- second pass: the weights, 64 keys at a time ----
-      float ls[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-      for (int hf = 0; hf < 2; ++hf) {
-        pt_ld32_nowait(trow + 64 * hf, *reinterpret_cast<uint32_t(*)[32]>(r));
-        pt_ld32_nowait(trow + 64 * hf + 32, *reinterpret_cast<uint32_t(*)[32]>(r + 32));
-        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-        if (hf == 1) {
-          // S(tile) is in registers: the next S may overwrite it
-          asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-          asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar_sf + 8 * X) : "memory");
-        }
-        if (interior) {
-          // no mask; two logits per packed FMA, two weights per packed add
-          uint64_t qs2, nm2, l2[4] = {0ull, 0ull, 0ull, 0ull};
-          asm("mov.b64 %0, {%1, %1};" : "=l"(qs2) : "f"(p.qscale));
-          asm("mov.b64 %0, {%1, %1};" : "=l"(nm2) : "f"(nm));
-          // Blocks of eight pairs, written stage by stage so that the instruction stream already interleaves
-          // independent pairs (a thread has one other warp to hide its latencies behind): the scaled logits of the
-          // block, then the first steps of the FMA-pipe pairs, the special-function pairs, the rest of the cubic, the
-          // rounding to bf16.
-          const uint64_t MAGIC2 = pt_pack2(12582912.f, 12582912.f), NMAGIC2 = pt_pack2(-12582912.f, -12582912.f),
-                         MONE2 = pt_pack2(-1.f, -1.f), C3 = pt_pack2(5.517164618e-02f, 5.517164618e-02f),
-                         C2 = pt_pack2(2.426111251e-01f, 2.426111251e-01f), C1 = pt_pack2(6.932609677e-01f, 6.932609677e-01f),
-                         C0 = pt_pack2(9.999280572e-01f, 9.999280572e-01f);
-#pragma unroll
-          for (int jb = 0; jb < 32; jb += 8) {             // pair index of the block's first pair
-            uint64_t x2[8];
-#pragma unroll
-            for (int u = 0; u < 8; ++u) {
-              uint64_t s2;
-              asm("mov.b64 %0, {%1, %2};" : "=l"(s2) : "r"(r[2 * (jb + u)]), "r"(r[2 * (jb + u) + 1]));
-              x2[u] = pt_fma2(s2, qs2, nm2);
-            }
-            float pv[16];
-            uint64_t fi2[8], f2[8], q2[8];
-#pragma unroll
-            for (int u = 0; u < 8; ++u)
-              if ((PT_POLY_PAIRS >> u) & 1u) {
-                float x0, x1;
-                asm("mov.b64 {%0, %1}, %2;" : "=f"(x0), "=f"(x1) : "l"(x2[u]));
-                x2[u] = pt_pack2(fmaxf(x0, -126.f), fmaxf(x1, -126.f));
-                fi2[u] = pt_add2(x2[u], MAGIC2);           // the integer part sits in the low mantissa bits
-              }
-#pragma unroll
-            for (int u = 0; u < 8; ++u)
-              if ((PT_POLY_PAIRS >> u) & 1u) f2[u] = pt_fma2(pt_add2(fi2[u], NMAGIC2), MONE2, x2[u]);
-#pragma unroll
-            for (int u = 0; u < 8; ++u)
-              if (!((PT_POLY_PAIRS >> u) & 1u)) {
-                float x0, x1;
-                asm("mov.b64 {%0, %1}, %2;" : "=f"(x0), "=f"(x1) : "l"(x2[u]));
-                pv[2 * u] = pt_ex2(x0);
-                pv[2 * u + 1] = pt_ex2(x1);
-              }
-#pragma unroll
-            for (int u = 0; u < 8; ++u)
-              if ((PT_POLY_PAIRS >> u) & 1u) q2[u] = pt_fma2(C3, f2[u], C2);
-#pragma unroll
-            for (int u = 0; u < 8; ++u)
-              if ((PT_POLY_PAIRS >> u) & 1u) q2[u] = pt_fma2(q2[u], f2[u], C1);
-#pragma unroll
-            for (int u = 0; u < 8; ++u)
-              if ((PT_POLY_PAIRS >> u) & 1u) {
-                q2[u] = pt_fma2(q2[u], f2[u], C0);
-                uint32_t qa, qb, ia, ib;
-                asm("mov.b64 {%0, %1}, %2;" : "=r"(qa), "=r"(qb) : "l"(q2[u]));
-                asm("mov.b64 {%0, %1}, %2;" : "=r"(ia), "=r"(ib) : "l"(fi2[u]));
-                pv[2 * u] = __uint_as_float(ia * 0x800000u + qa);        // + n << 23
-                pv[2 * u + 1] = __uint_as_float(ib * 0x800000u + qb);
-              }
-#pragma unroll
-            for (int u = 0; u < 8; ++u) {
-              const __nv_bfloat162 v2 = __floats2bfloat162_rn(pv[2 * u], pv[2 * u + 1]);
-              const uint32_t pk = *reinterpret_cast<const uint32_t*>(&v2);
-              if constexpr (!LSUM) {
-                // the row sum takes the rounded weights the second MMA will see (a one-hot row comes out exact)
-                uint64_t p2;
-                asm("mov.b64 %0, {%1, %2};" : "=l"(p2) : "r"(pk << 16), "r"(pk & 0xffff0000u));
-                l2[u & 3] = pt_add2(l2[u & 3], p2);
-              }
-              r[jb + u] = pk;
-            }
-          }
-          if constexpr (!LSUM) {
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-              float a0, a1;
-              asm("mov.b64 {%0, %1}, %2;" : "=f"(a0), "=f"(a1) : "l"(l2[k]));
-              ls[k] += a0 + a1;
-            }
-          }
-        } else {
-          // diagonal tile: causal mask
-#pragma unroll
-          for (int j = 0; j < 64; j += 2) {
-            float p0 = pt_ex2(fmaf(__uint_as_float(r[j]), p.qscale, nm));
-            float p1 = pt_ex2(fmaf(__uint_as_float(r[j + 1]), p.qscale, nm));
-            if (j0 + 64 * hf + j > pos) p0 = 0.f;
-            if (j0 + 64 * hf + j + 1 > pos) p1 = 0.f;
-            const __nv_bfloat162 v2 = __floats2bfloat162_rn(p0, p1);
-            const uint32_t pk = *reinterpret_cast<const uint32_t*>(&v2);
-            if constexpr (!LSUM) ls[(j >> 1) & 3] += __uint_as_float(pk << 16) + __uint_as_float(pk & 0xffff0000u);
-            r[j >> 1] = pk;
-          }
-        }
-        if (hf == 1 && tile > 0 && !o_waited) {
-          // the second half of P_X is read by the previous tile's last MMAs (the first half is safe: S(tile), which
-          // this thread has waited for, was issued after the MMAs that read it)
-          if (!__all_sync(0xffffffffu, wait(bar_o + 8 * X, tp ^ 1u))) { rows_ok = false; break; }
-        }
-        // this row's 64 weights: eight 16-byte chunks, chunk c at c ^ (row % 8) of the row's 128-byte line
-        unsigned char* pl = prow + hf * P2_COL;
-#pragma unroll
-        for (int c = 0; c < 8; ++c)
-          *reinterpret_cast<uint4*>(pl + ((c ^ (row & 7)) << 4)) = make_uint4(r[4 * c], r[4 * c + 1], r[4 * c + 2], r[4 * c + 3]);
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar_p + 16 * X + 8 * hf) : "memory");
-      }
-      if (!rows_ok) break;
-      l_run += (ls[0] + ls[1]) + (ls[2] + ls[3]);
+      // P (64 bf16 = 32 packed columns) goes back into tensor memory over the first half of the S columns it came
+      // from: it is the A operand of the second MMA, and the next S into this buffer is issued after that MMA
+      pt_st32(trow, *reinterpret_cast<uint32_t(*)[32]>(r));
+      asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar_p + 8 * (2 * X + (tile & 1))) : "memory");
     }
-    if (rows_ok && n_my > 0) __all_sync(0xffffffffu, wait(bar_o + 8 * X, (uint32_t)(n_my - 1) & 1u));
+    if (rows_ok && n_my > 0) __all_sync(0xffffffffu, wait(bar_o + 8 * X, (n_my - 1) & 1));
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
