@@ -123,9 +123,21 @@ __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, uint3
     if (mbar_try_wait(bar, parity)) return true;
   return false;
 }
+// one probe that never parks the thread (try_wait may, and then costs a few hundred cycles even when the phase is over)
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
 // the copy is normally ahead of the math: one probe, and the bounded polling loop out of line
 __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, uint32_t limit = WAIT_LIMIT) {
-  if (mbar_try_wait(bar, parity)) return true;
+  if (mbar_test_wait(bar, parity)) return true;
   return mbar_wait_slow(bar, parity, limit);
 }
 // Programmatic dependent launch (no-ops in a kernel launched without the attribute): wait until the previous kernel

@@ -84,6 +84,17 @@ __device__ __forceinline__ bool tc_mbar_try_wait(uint32_t bar, uint32_t parity) 
   return ok != 0;
 }
 __device__ __forceinline__ bool tc_mbar_wait(uint32_t bar, uint32_t parity) {
+  {   // first a probe that never parks the thread: try_wait may, and then costs a few hundred cycles even when the phase is over
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    if (ok) return true;
+  }
   for (uint32_t i = 0; i < TC_WAIT_LIMIT; ++i)
     if (tc_mbar_try_wait(bar, parity)) return true;
   return false;
