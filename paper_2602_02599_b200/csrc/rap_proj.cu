@@ -132,8 +132,10 @@ __global__ void rope_append_kernel(const float* __restrict__ y, int ksplit, cons
         b += yr[s * split_stride + col + 1];
       }
       if (bias) { a += from_storage<T>(bias[col]); b += from_storage<T>(bias[col + 1]); }
-      const float ra = a * cf - b * sf;
-      const float rb = a * sf + b * cf;
+      // one rounded product and one fused multiply-add each, spelled out: every kernel that rotates (this one, the
+      // one-launch projection, the quantising epilogue) rounds the same way, whatever the compiler would contract
+      const float ra = fmaf(-b, sf, __fmul_rn(a, cf));
+      const float rb = fmaf(a, sf, __fmul_rn(b, cf));
       if (j < G) {
         T* dst = q_out + ((size_t)t * Hq + head) * P2 + 2 * c;
         dst[0] = to_storage<T>(ra);

@@ -418,7 +418,7 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
               const float2 cs = cs_w[(t & 15) * 32 + (cs_lane | (t >> 4))];
               const int row = __shfl_sync(0xffffffffu, my_row, t);
               // pair (a, b) on lanes (even, odd):  a' = a cos - b sin,  b' = a sin + b cos
-              const float rot = (lane & 1) ? fmaf(other, cs.y, mine * cs.x) : fmaf(-other, cs.y, mine * cs.x);
+              const float rot = (lane & 1) ? fmaf(other, cs.y, __fmul_rn(mine, cs.x)) : fmaf(-other, cs.y, __fmul_rn(mine, cs.x));
               const __nv_bfloat16 o = __float2bfloat16_rn(kind == 2 ? mine : rot);
               if (in_range) {
                 if (kind == 0) {

@@ -130,8 +130,8 @@ rope_append_q8_kernel(const float* __restrict__ y, int ksplit, const T* __restri
         for (int s = 0; s < RAP_MAX_KSPLIT; ++s)
           if (s < ksplit) { a += pa[k][s]; b += pb[k][s]; }
         if (bias) { a += q8_ld(bias + col0 + 2 * c); b += q8_ld(bias + col0 + 2 * c + 1); }
-        ra[k] = a * cf - b * sf;
-        rb[k] = a * sf + b * cf;
+        ra[k] = fmaf(-b, sf, __fmul_rn(a, cf));          // the same roundings as the unquantised kernels
+        rb[k] = fmaf(a, sf, __fmul_rn(b, cf));
         amax = fmaxf(amax, fmaxf(fabsf(ra[k]), fabsf(rb[k])));
       }
     }

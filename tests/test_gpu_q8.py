@@ -230,6 +230,54 @@ def test_q8_full_size_sampled_units(name):
     st.close()
 
 
+@pytest.mark.parametrize("name,T", [("8b", 32), ("8b", 5), ("3b", 17), ("sweep1.0", 1)])
+def test_q8_decode_sized_append(name, T):
+    """Decode-sized rap_qkv_rope_append_q8 calls (T <= 32: the token-tile width the step uses; scattered sequences and
+    slots).  q~ equals, bit for bit, what the unquantised entry point writes for the same rows (every rotating kernel
+    rounds the same way); against the oracle: codes within one step, scales within a bf16 step (fp32 against fp64
+    accumulation); nothing but the named rows is touched."""
+    w = synth.scaled_down(synth.CONFIGS[name], n_layers=2, batch=3, seq=64, hidden=512)
+    ks, vs = synth.draw_scores(w)
+    st, tabs, w_host = util.build_small_stack(w, ks, vs, full_weights=True, max_rows=64)
+    B, Hq, Hkv = w.batch, w.n_q_heads, w.n_kv_heads
+    rng = np.random.default_rng(5)
+    seq_id = rng.integers(0, B, size=T).astype(np.int32)
+    pos = np.zeros(T, np.int32)
+    for b in range(B):                                   # distinct slots per sequence
+        m = seq_id == b
+        pos[m] = rng.permutation(60)[: m.sum()]
+    sid, ps = torch.from_numpy(seq_id).to(st.device), torch.from_numpy(pos).to(st.device)
+    for l in range(w.n_layers):
+        P, dv = st.n_pairs[l], st.n_vch[l]
+        X = synth.draw_hidden(w, l, 3, T)
+        dx = torch.from_numpy(X).to(st.device).to(st.dt).contiguous()
+        k8, v8 = _q8_caches(st, l)
+        q_dev = torch.full((T, Hq, 2 * P), float("nan"), dtype=st.dt, device=st.device)
+        st.ctx.rap_qkv_rope_append_q8(l, T, dx, st.w_qkv[l], None, sid, ps, ps, int(pos.max()), st.inv_freq, q_dev, k8, v8, B,
+                                      st.s_cap)
+        q_plain = torch.full((T, Hq, 2 * P), float("nan"), dtype=st.dt, device=st.device)
+        st.qkv_rope_append(l, dx, sid, ps, ps, int(pos.max()), q_out=q_plain)
+        torch.cuda.synchronize()
+        assert st.ctx.rap_get_last_device_status() == (0, 0)
+        assert torch.equal(q_dev, q_plain)
+        q, k, v = O.qkv_rope(O.round_storage(X, w.dtype), w_host[l], None, pos, tabs["inv_freq"][l], Hq, Hkv, P, dv)
+        util.check_projection(util.to_np64(q_dev), O.round_storage(q, w.dtype), w.dtype, f"q layer {l}")
+        kc_o = np.zeros((B, Hkv, st.s_cap, 2 * P), np.int8); ks_o = np.zeros((B, Hkv, st.s_cap))
+        vc_o = np.zeros((B, Hkv, st.s_cap, dv), np.int8); vs_o = np.zeros((B, Hkv, st.s_cap))
+        O.append_q8(kc_o, ks_o, vc_o, vs_o, k, v, seq_id, pos)
+        for dev, W, c_o, s_o, what in ((k8, 2 * P, kc_o, ks_o, "K"), (v8, dv, vc_o, vs_o, "V")):
+            c_d, s_d = util.unpack_q8(dev, W)
+            written = np.zeros(c_d.shape[:3], bool)
+            written[seq_id, :, pos] = True
+            assert not dev.cpu().numpy()[~written].any()
+            diff = np.abs(c_d.astype(int) - c_o.astype(int))[written]
+            assert diff.max() <= 1, what
+            assert (diff != 0).mean() < 0.02, (what, (diff != 0).mean())
+            assert np.all(np.abs(s_d - s_o)[written] <= 2.0 ** -7 * s_o[written] + 1e-30), what
+            assert not dev.cpu().numpy()[..., W:-2].any()
+    st.close()
+
+
 @pytest.mark.parametrize("name", ["8b", "3b"])
 def test_q8_decode_step_equals_the_separate_calls_and_the_oracle(name):
     """rap_decode_step_q8 (all layers: quantising append, then attention over the quantised cache; consecutive launches
