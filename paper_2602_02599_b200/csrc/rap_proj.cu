@@ -213,6 +213,7 @@ __global__ void pack_wo_kernel(const T* __restrict__ wo, const int32_t* __restri
 }
 
 __global__ void cast_bf16_kernel(const float* __restrict__ src, __nv_bfloat16* __restrict__ dst, size_t n) {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");     // a GEMM launched behind this may start its prologue
   const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i < n) dst[i] = __float2bfloat16_rn(src[i]);
 }
@@ -220,6 +221,8 @@ __global__ void cast_bf16_kernel(const float* __restrict__ src, __nv_bfloat16* _
 // y[i] = storage( sum over the reduction splits of ws[ks][i] )
 template <typename T>
 __global__ void sum_splits_kernel(const float* __restrict__ ws, int ksplit, size_t n, T* __restrict__ y) {
+  // (launched behind the GEMM with programmatic serialization in rap_out_proj: the partial results are awaited here)
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n) return;
   float a = 0.f;
@@ -343,7 +346,9 @@ rap_status rap_launch_out_proj(rap_ctx* ctx, int32_t layer, int32_t T, const flo
     cast_bf16_kernel<<<(unsigned)((nx + 255) / 256), 256, 0, st>>>(attn_out, (__nv_bfloat16*)ctx->d_oproj_x, nx);
     ctx->launches++;
     RAP_CUDA_TRY(ctx, cudaGetLastError());
-    rap_status s = rap_launch_gemm_tc(ctx, ctx->d_oproj_x, wo_tilde, T, K, N, &ksplit, st, 0);
+    // the three launches are chained with programmatic serialization: the GEMM's prologue and first weight tiles
+    // overlap the cast, the split sum is resident and waiting when the GEMM ends
+    rap_status s = rap_launch_gemm_tc(ctx, ctx->d_oproj_x, wo_tilde, T, K, N, &ksplit, st, 2);
     if (s == RAP_EUNSUPPORTED) {
       if ((K * 2) % 16) return RAP_EUNSUPPORTED;
       ksplit = 1;
@@ -355,7 +360,19 @@ rap_status rap_launch_out_proj(rap_ctx* ctx, int32_t layer, int32_t T, const flo
     } else if (s != RAP_OK) {
       return s;
     }
-    sum_splits_kernel<__nv_bfloat16><<<(unsigned)((n + 255) / 256), 256, 0, st>>>(ctx->d_proj_ws, ksplit, n, (__nv_bfloat16*)y);
+    {
+      cudaLaunchConfig_t cfg = {};
+      cfg.gridDim = dim3((unsigned)((n + 255) / 256), 1, 1);
+      cfg.blockDim = dim3(256, 1, 1);
+      cfg.stream = st;
+      cudaLaunchAttribute attr[1];
+      attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+      attr[0].val.programmaticStreamSerializationAllowed = 1;
+      cfg.attrs = attr;
+      cfg.numAttrs = 1;
+      RAP_CUDA_TRY(ctx, cudaLaunchKernelEx(&cfg, sum_splits_kernel<__nv_bfloat16>, (const float*)ctx->d_proj_ws, ksplit, n,
+                                           (__nv_bfloat16*)y));
+    }
   } else {
     if ((K * 4) % 16) return RAP_EUNSUPPORTED;
     dim3 grid((N + PROJ_WARPS - 1) / PROJ_WARPS, (T + PROJ_TT - 1) / PROJ_TT);

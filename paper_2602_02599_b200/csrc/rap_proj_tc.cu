@@ -142,6 +142,7 @@ struct TcParams {
   int32_t* status;
   int T, n_out, nkb_total, nkb_per_split;
   int row_tiles, tok_tiles, n_work;     // work items = row tiles x token tiles x reduction splits
+  int wait_x;          // x is written by the previous kernel in the stream (programmatic launch): wait for it before x is read
 };
 
 // What the fused RoPE / append epilogue needs beyond the GEMM (decode-sized calls, one token tile).
@@ -229,10 +230,26 @@ proj_tc_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant_
   if (warp == 0) {
     if (lane == 0) {
       uint32_t kbg = 0;      // k-blocks issued so far: position in the ring
+      int pre = 0;           // k-blocks of the first item already issued
+      if (p.wait_x) {
+        // The weights do not depend on the previous kernel: the first ring-full of W tiles goes out before the wait,
+        // the x tiles of those stages after it (the stages are empty on the first lap).
+        int n0, t0, ks, kb0, nkb = 0;
+        if ((int)blockIdx.x < p.n_work) decode(blockIdx.x, n0, t0, ks, kb0, nkb);
+        pre = nkb < C::NS ? nkb : C::NS;
+        for (int kb = 0; kb < pre; ++kb) {
+          tc_mbar_expect_tx(full0 + 8 * kb, C::STAGE);
+          tc_tma_load_2d(ring + kb * C::STAGE, &map_w, (kb0 + kb) * TC_BK, n0, full0 + 8 * kb);
+        }
+        tc_pdl_wait();
+        for (int kb = 0; kb < pre; ++kb)
+          tc_tma_load_2d(ring + kb * C::STAGE + TC_A_BYTES, &map_x, (kb0 + kb) * TC_BK, t0, full0 + 8 * kb);
+        kbg = (uint32_t)pre;
+      }
       for (int w = blockIdx.x; w < p.n_work && !timed_out; w += gridDim.x) {
         int n0, t0, ks, kb0, nkb;
         decode(w, n0, t0, ks, kb0, nkb);
-        for (int kb = 0; kb < nkb; ++kb, ++kbg) {
+        for (int kb = (w == (int)blockIdx.x ? pre : 0); kb < nkb; ++kb, ++kbg) {
           const uint32_t s = kbg % C::NS, ph = (kbg / C::NS) & 1u;
           if (!tc_mbar_wait(empty0 + 8 * s, ph ^ 1u)) { timed_out = true; break; }   // first lap passes at once
           const uint32_t a = ring + s * C::STAGE, b = a + TC_A_BYTES;
@@ -538,6 +555,7 @@ bool plan_gemm(const rap_ctx* ctx, int T, int K, int N, int* tn_out, int* ksplit
   if ((size_t)ksplit * T * N * sizeof(float) > ctx->proj_ws_bytes) return false;
   p->y = ctx->d_proj_ws; p->status = ctx->d_status; p->T = T; p->n_out = N; p->nkb_total = nkb; p->nkb_per_split = per;
   p->row_tiles = row_tiles; p->tok_tiles = tok_tiles; p->n_work = row_tiles * tok_tiles * ksplit;
+  p->wait_x = 0;
   *tn_out = tn;
   *ksplit_out = ksplit;
   return true;
@@ -550,6 +568,8 @@ bool rap_tensor_map_bf16(rap_ctx* ctx, void* map128, const void* base, uint64_t 
 }
 
 // Y[ks][T][N] (fp32, context workspace) = X[T][K] * W[N][K]^T, bf16 operands, K split over work items.
+// pdl: 0 = ordinary launch; 1 = programmatic stream serialization, x does not depend on the previous kernel in the
+// stream; 2 = the same, and x is what that kernel writes (the first weight tiles still go out before the wait)
 rap_status rap_launch_gemm_tc(rap_ctx* ctx, const void* x, const void* w, int T, int K, int N, int* ksplit_out,
                               cudaStream_t st, int pdl) {
   if (T < 1 || (K % 8) != 0) return RAP_EUNSUPPORTED;     // tensor-map rows must be multiples of 16 bytes
@@ -561,6 +581,7 @@ rap_status rap_launch_gemm_tc(rap_ctx* ctx, const void* x, const void* w, int T,
   if (!make_map(ctx, &mx, x, (uint64_t)T, (uint64_t)K, (uint32_t)tn)) return RAP_EUNSUPPORTED;
   dim3 grid(p.n_work < ctx->sm_count ? p.n_work : ctx->sm_count, 1, 1);
   *ksplit_out = ksplit;
+  p.wait_x = pdl == 2 ? 1 : 0;
   switch (tn) {
     case 32: return launch_tc<32>(ctx, mw, mx, p, grid, st, pdl);
     case 64: return launch_tc<64>(ctx, mw, mx, p, grid, st, pdl);
