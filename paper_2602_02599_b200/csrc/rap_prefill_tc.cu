@@ -63,31 +63,11 @@ __device__ __forceinline__ bool pt_test_wait(uint32_t bar, uint32_t parity) {
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
-// K-major operand tile, 128-byte swizzle: 8-row groups 1024 bytes apart (see rap_proj_tc.cu)
-__device__ __forceinline__ uint64_t pt_desc(uint32_t addr) {
-  const uint32_t lo = ((addr & 0x3FFFFu) >> 4) | (1u << 16);
-  const uint32_t hi = (1024u >> 4) | (1u << 14) | (2u << 29);
-  return ((uint64_t)hi << 32) | lo;
-}
-__device__ __forceinline__ void pt_mma(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(tmem_d),
-      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(acc)
-      : "memory");
-}
-// the same with the A operand in tensor memory (row = lane, two bf16 K elements per 32-bit column)
-__device__ __forceinline__ void pt_mma_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t bdesc, uint32_t idesc, uint32_t acc) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}" ::"r"(tmem_d),
-      "r"(tmem_a), "l"(bdesc), "r"(idesc), "r"(acc)
-      : "memory");
-}
-// The same two with the descriptors given as (low word, high word): the low word carries the start address (in 16-byte
-// units, 14 bits), so walking a ring or the k-steps of a tile is one 32-bit add on it.
+// tcgen05.mma with shared-memory operand descriptors given as (low word, high word).  K-major operand tile, 128-byte
+// swizzle, 8-row groups 1024 bytes apart (see rap_proj_tc.cu): the high word is the same for every operand here; the
+// low word carries the start address (in 16-byte units, 14 bits) and the leading offset (bits 16-29), so walking a
+// ring or the k-steps of a tile is one 32-bit add on it.  pt_mma_ts2: A in tensor memory (row = lane, two bf16 K
+// elements per 32-bit column).
 __device__ __forceinline__ void pt_mma2(uint32_t tmem_d, uint32_t a_lo, uint32_t b_lo, uint32_t hi, uint32_t idesc, uint32_t acc) {
   asm volatile(
       "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
@@ -170,12 +150,8 @@ __device__ __forceinline__ uint32_t pt_off(int row, int col, int rows) {
 
 // N-major operand tile (B = V as stored, [key][channel]), 128-byte swizzle: an atom is 8 keys x 64 channels
 // (key rows of 128 bytes, 16-byte chunks XORed with key % 8); atoms of consecutive 8-key groups are 1024 bytes
-// apart (stride offset), the two 64-channel atom columns of a 64-key tile 8 KB apart (leading offset).
-__device__ __forceinline__ uint64_t pt_desc_n2(uint32_t addr) {
-  const uint32_t lo = ((addr & 0x3FFFFu) >> 4) | ((8192u >> 4) << 16);
-  const uint32_t hi = (1024u >> 4) | (1u << 14) | (2u << 29);
-  return ((uint64_t)hi << 32) | lo;
-}
+// apart (stride offset), the two 64-channel atom columns of a 64-key tile 8 KB apart (leading offset: bits 16-29 of
+// the descriptor's low word).
 // Byte offset inside a 64-row tile row of its byte e: 64-element (128-byte) atom columns 8 KB apart, 16-byte chunks
 // XORed with row % 8 (the layout is the same for the K-major K tile and the N-major V tile).
 __device__ __forceinline__ uint32_t pt_swz2(int e, int r7) {
