@@ -54,8 +54,9 @@ lr_rebuild_kernel(const __nv_bfloat16* __restrict__ latent, const __nv_bfloat16*
   constexpr int BS = RP + 8;                       // B_k^T row stride (bf16): keeps the fragment reads conflict-free
   extern __shared__ __align__(16) unsigned char rb_smem[];
   __nv_bfloat16* bkt = reinterpret_cast<__nv_bfloat16*>(rb_smem);          // [128][BS]: B_k^T, zero padded in k
-  __nv_bfloat16* lat = bkt + RB_D * BS;                                    // [64][r] latent tile as stored, + 16 zeros
-  __nv_bfloat16* kst = lat + RB_TILE * RB_D + 16;                          // [64][136] rotated tile before the coalesced store
+  __nv_bfloat16* lat0 = bkt + RB_D * BS;                                   // 2 x ([64][r] latent tile as stored, + 16 zeros)
+  constexpr int LAT = RB_TILE * RB_D + 16;
+  __nv_bfloat16* kst = lat0 + 2 * LAT;                                     // [64][136] rotated tile before the coalesced store
   const int h = blockIdx.y, b = blockIdx.z;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int len = min(max(seq_len[b], 0), S_cap);
@@ -68,17 +69,40 @@ lr_rebuild_kernel(const __nv_bfloat16* __restrict__ latent, const __nv_bfloat16*
   }
   // the fragment loads of the last k step run past the row (into the next row, or the pad after the
   // last one) where B_k^T holds zeros: those values only have to be finite
-  for (int i = tid; i < RB_TILE * RB_D + 16; i += 256) lat[i] = zero;
+  for (int i = tid; i < 2 * LAT; i += 256) lat0[i] = zero;
+  __syncthreads();
   const int g = lane >> 2, t = lane & 3;
-  for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
+  // the latent tiles are fetched one tile ahead (16-byte asynchronous copies into the other buffer)
+  auto fetch = [&](int tile, int buf) {
+    const int j0 = tile * RB_TILE;
+    const int nj = min(RB_TILE, len - j0);
+    const unsigned char* lsrc = reinterpret_cast<const unsigned char*>(latent + (((size_t)b * Hkv + h) * S_cap + j0) * r);
+    const int nvec = (nj * r * 2 + 15) / 16;          // the tile is one contiguous, 16-byte aligned range
+    const uint32_t dst = (uint32_t)__cvta_generic_to_shared(lat0 + buf * LAT);
+    for (int i = tid; i < nvec; i += 256)
+      asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst + 16u * (uint32_t)i), "l"(lsrc + 16 * (size_t)i) : "memory");
+  };
+  int buf = 0;
+  if ((int)blockIdx.x < n_tiles) fetch(blockIdx.x, 0);
+  asm volatile("cp.async.commit_group;" ::: "memory");
+  for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, buf ^= 1) {
   const int j0 = tile * RB_TILE;
   const int nj = min(RB_TILE, len - j0);
-  __syncthreads();                                  // the previous tile's fragments have been read
-  const uint4* lsrc = reinterpret_cast<const uint4*>(latent + (((size_t)b * Hkv + h) * S_cap + j0) * r);
-  const int nvec = (nj * r * 2 + 15) / 16;          // the tile is one contiguous, 16-byte aligned range
-  for (int i = tid; i < nvec; i += 256) reinterpret_cast<uint4*>(lat)[i] = lsrc[i];
-  __syncthreads();
+  const __nv_bfloat16* lat = lat0 + buf * LAT;
+  if (tile + (int)gridDim.x < n_tiles) fetch(tile + gridDim.x, buf ^ 1);   // its last readers passed the barrier below a tile ago
+  asm volatile("cp.async.commit_group;" ::: "memory");
   const int row0 = 16 * (warp >> 1), cset = warp & 1;
+  // this thread's (cos, sin) pairs, on their way while the tile lands and the MMAs run
+  float4 csv[2][4];
+#pragma unroll
+  for (int hr = 0; hr < 2; ++hr) {
+    const int row = min(row0 + g + 8 * hr, nj - 1);
+    const float4* csr = reinterpret_cast<const float4*>(cs + (size_t)(j0 + row) * (RB_D / 2));
+#pragma unroll
+    for (int nt = 0; nt < 4; ++nt) csv[hr][nt] = __ldg(csr + ((32 * cset + 8 * nt + 2 * t) >> 1));
+  }
+  asm volatile("cp.async.wait_group 1;" ::: "memory");
+  __syncthreads();                                  // this tile has landed for every thread; the previous tile's rows are stored
   float acc[8][4];
 #pragma unroll
   for (int nt = 0; nt < 8; ++nt)
@@ -105,11 +129,10 @@ lr_rebuild_kernel(const __nv_bfloat16* __restrict__ latent, const __nv_bfloat16*
   for (int hr = 0; hr < 2; ++hr) {
     const int row = row0 + g + 8 * hr;
     if (row < nj) {
-      const float4* csr = reinterpret_cast<const float4*>(cs + (size_t)(j0 + row) * (RB_D / 2));
 #pragma unroll
       for (int nt = 0; nt < 4; ++nt) {
         const int i = 32 * cset + 8 * nt + 2 * t;           // pair indices i, i + 1
-        const float4 c = csr[i >> 1];                       // (cos_i, sin_i, cos_i+1, sin_i+1)
+        const float4 c = csv[hr][nt];                       // (cos_i, sin_i, cos_i+1, sin_i+1)
         const float x0 = acc[nt][2 * hr], x1 = acc[nt][2 * hr + 1];
         const float y0 = acc[nt + 4][2 * hr], y1 = acc[nt + 4][2 * hr + 1];
         *reinterpret_cast<uint32_t*>(kst + row * KSS + i) = pack_bf16(x0 * c.x - y0 * c.y, x1 * c.z - y1 * c.w);
@@ -124,11 +147,12 @@ lr_rebuild_kernel(const __nv_bfloat16* __restrict__ latent, const __nv_bfloat16*
     kdst[i] = *reinterpret_cast<const uint4*>(kst + row * KSS + c8 * 8);
   }
   }   // tile loop
+  asm volatile("cp.async.wait_group 0;" ::: "memory");
 }
 
 template <int RP>
 rap_status launch_rebuild(rap_ctx* ctx, const rap_lowrank_args& a, cudaStream_t st) {
-  const size_t smem = (size_t)(RB_D * (RP + 8) + RB_TILE * RB_D + 16 + RB_TILE * (RB_D + 8)) * sizeof(__nv_bfloat16);
+  const size_t smem = (size_t)(RB_D * (RP + 8) + 2 * (RB_TILE * RB_D + 16) + RB_TILE * (RB_D + 8)) * sizeof(__nv_bfloat16);
   RAP_CUDA_TRY(ctx, rap_raise_smem(ctx, lr_rebuild_kernel<RP>, (int)smem));
   // a few CTAs per SM, each looping over tiles so that the B_k^T staging is paid once per CTA
   const int n_tiles = (a.h_len_max + RB_TILE - 1) / RB_TILE;
