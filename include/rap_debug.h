@@ -46,6 +46,14 @@ rap_status rap_set_proj_variant(rap_ctx* ctx, int32_t variant);
  * used, so nothing has to be reset by hand.  The hook disarms itself when it is used. */
 rap_status rap_debug_arm_wait_timeout(rap_ctx* ctx);
 
+/* The tensor-core scan of rap_decode_attn normally decides by the size of a launch whether its last tiles are handed
+ * out at run time (pieces of some tiles, claimed from a counter by the CTAs as they finish) or assigned up front like
+ * the rest.  This forces the choice for every later launch on the context, so that small test cases take the run-time
+ * path: piece_tiles > 0 tiles per piece and frac_x256 / 256 of all tiles handed out that way; piece_tiles = 0: nothing
+ * is handed out at run time; piece_tiles = -1: back to the automatic choice.  The result of a launch does not depend on
+ * which CTA ends up with which piece (a piece is a fixed range of tiles, and partials are merged in tile order). */
+rap_status rap_debug_set_scan_pieces(rap_ctx* ctx, int32_t piece_tiles, int32_t frac_x256);
+
 /* Shows that the index checks of the bounds-checking build (librap_b200_dbg.so, compiled with -DRAP_DEBUG_BOUNDS) are
  * live, without any access leaving a buffer: the next shape-specialised scan launch is told that the split-KV
  * workspace holds only n_floats floats (it is as large as ever).  In the bounds-checking build the writes of partials

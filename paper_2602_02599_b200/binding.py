@@ -27,7 +27,7 @@ EXPORTS = [
     "rap_get_last_device_status", "rap_kernel_launch_count", "rap_set_attn_variant",
     "rap_decode_attn_noalloc", "rap_profile_attn", "rap_profile_attn_read",
     "rap_pack_wo", "rap_out_proj", "rap_budget_alloc", "rap_prefill_attn", "rap_build_tables_hybrid",
-    "rap_build_tables_partial", "rap_build_tables_freq", "rap_set_proj_variant", "rap_debug_arm_wait_timeout", "rap_debug_claim_scan_workspace",
+    "rap_build_tables_partial", "rap_build_tables_freq", "rap_set_proj_variant", "rap_debug_arm_wait_timeout", "rap_debug_claim_scan_workspace", "rap_debug_set_scan_pieces",
     "rap_q8_row_bytes", "rap_quantize_rows", "rap_qkv_rope_append_q8", "rap_decode_attn_q8", "rap_decode_step_q8",
 ]
 
@@ -85,6 +85,7 @@ def _lib():
     lib.rap_set_attn_variant.argtypes = [P, c_int32]
     lib.rap_set_proj_variant.argtypes = [P, c_int32]
     lib.rap_debug_arm_wait_timeout.argtypes = [P]
+    lib.rap_debug_set_scan_pieces.argtypes = [P, c_int32, c_int32]
     lib.rap_debug_claim_scan_workspace.argtypes = [P, c_int64]
     lib.rap_q8_row_bytes.argtypes = [c_int32]
     lib.rap_q8_row_bytes.restype = c_size_t
@@ -348,6 +349,9 @@ class RapContext:
 
     def rap_debug_arm_wait_timeout(self):
         self._check(_lib().rap_debug_arm_wait_timeout(self._ctx), "rap_debug_arm_wait_timeout")
+
+    def rap_debug_set_scan_pieces(self, piece_tiles, frac_x256):
+        self._check(_lib().rap_debug_set_scan_pieces(self._ctx, piece_tiles, frac_x256), "rap_debug_set_scan_pieces")
 
     def rap_set_proj_variant(self, variant):
         self._check(_lib().rap_set_proj_variant(self._ctx, variant), "rap_set_proj_variant")

@@ -86,6 +86,13 @@ rap_status rap_debug_arm_wait_timeout(rap_ctx* ctx) {
   return RAP_OK;
 }
 
+rap_status rap_debug_set_scan_pieces(rap_ctx* ctx, int32_t piece_tiles, int32_t frac_x256) {
+  if (!ctx || piece_tiles < -1 || frac_x256 < 0 || frac_x256 > 256) return RAP_EINVAL;
+  ctx->dbg_dyn_piece = piece_tiles;
+  ctx->dbg_dyn_frac = frac_x256;
+  return RAP_OK;
+}
+
 rap_status rap_set_proj_variant(rap_ctx* ctx, int32_t variant) {
   if (!ctx || variant < 0 || variant > 1) return RAP_EINVAL;
   ctx->proj_variant = variant;
@@ -206,8 +213,9 @@ rap_status rap_create(const rap_model_desc* desc, rap_ctx** out) {
   RAP_CUDA_TRY(c, cudaMalloc(&c->d_status, 2 * sizeof(int32_t)));
   RAP_CUDA_TRY(c, cudaMemset(c->d_status, 0, 2 * sizeof(int32_t)));
   RAP_CUDA_TRY(c, cudaMalloc(&c->d_attn_ws, c->attn_ws_bytes));
-  RAP_CUDA_TRY(c, cudaMalloc(&c->d_unit_cnt, 2 * (size_t)d.max_batch * d.n_kv_heads * sizeof(int32_t)));
-  RAP_CUDA_TRY(c, cudaMemset(c->d_unit_cnt, 0, 2 * (size_t)d.max_batch * d.n_kv_heads * sizeof(int32_t)));
+  // two sets of unit arrival counters, then the two piece counters of the scans that hand out their last tiles at run time
+  RAP_CUDA_TRY(c, cudaMalloc(&c->d_unit_cnt, (2 * (size_t)d.max_batch * d.n_kv_heads + 2) * sizeof(int32_t)));
+  RAP_CUDA_TRY(c, cudaMemset(c->d_unit_cnt, 0, (2 * (size_t)d.max_batch * d.n_kv_heads + 2) * sizeof(int32_t)));
   RAP_CUDA_TRY(c, cudaMalloc(&c->d_proj_ws, c->proj_ws_bytes));
   c->proj_cnt_n = 4 * (int)((n_out_max + 127) / 128);
   RAP_CUDA_TRY(c, cudaMalloc(&c->d_proj_cnt, 2 * (size_t)c->proj_cnt_n * sizeof(int32_t)));
@@ -794,7 +802,7 @@ rap_status rap_get_last_device_status(rap_ctx* ctx, int32_t* code, int32_t* deta
   RAP_CUDA_TRY(ctx, cudaStreamSynchronize(st));
   if (h[0] != 0) {   // a kernel that gave up may have left arrival counters behind (the next launches clear them too)
     const rap_model_desc& d = ctx->desc;
-    RAP_CUDA_TRY(ctx, cudaMemsetAsync(ctx->d_unit_cnt, 0, 2 * (size_t)d.max_batch * d.n_kv_heads * sizeof(int32_t), st));
+    RAP_CUDA_TRY(ctx, cudaMemsetAsync(ctx->d_unit_cnt, 0, (2 * (size_t)d.max_batch * d.n_kv_heads + 2) * sizeof(int32_t), st));
     RAP_CUDA_TRY(ctx, cudaMemsetAsync(ctx->d_proj_cnt, 0, 2 * (size_t)ctx->proj_cnt_n * sizeof(int32_t), st));
     RAP_CUDA_TRY(ctx, cudaStreamSynchronize(st));
   }

@@ -161,6 +161,7 @@ __global__ void __launch_bounds__(STHREADS, 2) attn_scan_kernel(const ScanParams
     pdl_launch_dependents();
     if (blockIdx.x == 0) {   // sequences without any row are scanned by nobody: their output is zero
       for (int i = tid; i < p.B * p.Hkv; i += STHREADS) p.unit_cnt_other[i] = 0;   // counters a launch that gave up left behind
+      if (tid == 0) *p.dyn_next_other = 0;          // and the piece counter a tensor-core launch before this one used
       for (int bb = 0; bb < p.B; ++bb)
         if (sk_tiles_of(p.seq_len, bb, p.len_add, p.S_cap, ST) == 0)
           for (int i = tid; i < p.Hq * DV; i += STHREADS) p.out[(size_t)bb * p.Hq * DV + i] = 0.f;

@@ -64,6 +64,7 @@ struct rap_ctx {
   size_t tmap_next = 0;
   int32_t attn_variant = 0;
   long long dbg_ws_floats = 0;    // > 0: the next scan launch is told its workspace holds only this many floats (rap_debug.h)
+  int32_t dbg_dyn_piece = -1, dbg_dyn_frac = 0;   // test hook: pieces claimed at run time, forced (-1: the launcher decides; rap_debug.h)
   int32_t dbg_arm_timeout = 0;    // the next tensor-core scan launch runs into a bounded wait on purpose (rap_debug.h)
   int32_t proj_variant = 0;       // 1: rap_qkv_rope_append always takes the two-stage path (GEMM, then the epilogue kernel)
   int64_t launches = 0;
@@ -125,6 +126,12 @@ struct rap_scan_params {
   int dbg_skip_copy;   // test hook: the first warp of the first CTA arms its first stage and issues no copy for it
   int B;               // sequences (used by the balanced mode)
   int balanced;        // 0: grid (n_split, H_kv, B), equal tile ranges per split; 1: grid (CTAs), see SkPlan
+  // Balanced mode, tensor-core form: the last tiles of the tile sequence are not assigned up front but cut into pieces
+  // of dyn_piece tiles that the CTAs claim from a counter as they finish (0: everything is assigned up front)
+  int dyn_piece;       // tiles per piece
+  int dyn_frac_x256;   // share of all tiles handed out that way, in 256ths
+  int32_t* dyn_next;   // next unclaimed piece of this launch (zero on entry)
+  int32_t* dyn_next_other;   // the counter the previous launch used; cleared by this launch
 };
 struct rap_scan_entry {
   int G, WK, DV;       // query heads per KV head, K words per row (= P), V channels (= d_v')

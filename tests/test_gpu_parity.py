@@ -191,11 +191,14 @@ def test_adjacent_pairing_end_to_end():
     _end_to_end(w, [40])
 
 
-def _random_attn_case(w, lens, n_split, seed=0, variant=0, q_gain=1.0, ramp=0.0):
+def _random_attn_case(w, lens, n_split, seed=0, variant=0, q_gain=1.0, ramp=0.0, pieces=None):
     """rap_decode_attn alone on random caches (no projection), every unit checked.  q_gain scales q (peaked
-    softmax); ramp > 0 makes the K rows grow with the position (the running maximum keeps moving)."""
+    softmax); ramp > 0 makes the K rows grow with the position (the running maximum keeps moving); pieces =
+    (tiles per piece, 256ths of all tiles) forces the tensor-core scan to hand that share out at run time."""
     st = DecodeStack(w, s_cap=((max(lens) + 8 + 7) // 8) * 8)
     st.ctx.rap_set_attn_variant(variant)
+    if pieces is not None:
+        st.ctx.rap_debug_set_scan_pieces(*pieces)
     ks, vs = synth.draw_scores(w)
     st.build_tables(ks, vs)
     g = torch.Generator(device=st.device).manual_seed(seed)
@@ -230,6 +233,46 @@ def _random_attn_case(w, lens, n_split, seed=0, variant=0, q_gain=1.0, ramp=0.0)
 def test_attention_only_longer_sequences(name, n_split):
     w = synth.scaled_down(synth.CONFIGS[name], n_layers=1, batch=3, seq=4096)
     _random_attn_case(w, [4096, 2500, 1], n_split)
+
+
+@pytest.mark.parametrize("name", ["3b", "8b", "14b", "sweep1.0", "sweep0.5"])
+@pytest.mark.parametrize("pieces", [(1, 128), (2, 64), (3, 200), (7, 38), (1, 256)])
+def test_attention_pieces_claimed_at_run_time(name, pieces):
+    """The tensor-core scan with a share of its tiles handed out at run time (long launches do that by themselves;
+    here it is forced on small ones, down to pieces of one tile, up to every tile): pieces are fixed tile ranges and
+    partials are merged in tile order, so the result is the one the oracle defines whoever scans what -- ragged
+    lengths, an empty sequence, units cut by several pieces, twice in a row on the same context (the counters of the
+    first launch are cleared by the second)."""
+    w = synth.scaled_down(synth.CONFIGS[name], n_layers=2, batch=4, seq=4096)
+    _random_attn_case(w, [4096, 2500, 1, 700], 0, seed=sum(pieces), variant=4, pieces=pieces)
+    _random_attn_case(w, [300, 0, 3999, 129], 0, seed=pieces[0], variant=4, pieces=pieces)
+
+
+def test_attention_pieces_and_tiers_take_turns():
+    """Launches that hand pieces out at run time use a counter that the NEXT balanced launch on the context clears,
+    whichever kernel that is: tensor-core scan with pieces, FP32-pipe scan, tensor-core scan again, explicit splits in
+    between -- every result against the oracle."""
+    w = synth.scaled_down(synth.CONFIGS["8b"], n_layers=1, batch=3, seq=4096)
+    lens = [4096, 1500, 77]
+    st = DecodeStack(w, s_cap=4104)
+    st.build_tables(*synth.draw_scores(w))
+    g = torch.Generator(device=st.device).manual_seed(4)
+    sig = float(np.sqrt(w.hidden) * 0.02)
+    st.k_cache[0].normal_(0, sig, generator=g)
+    st.v_cache[0].normal_(0, sig, generator=g)
+    q = torch.empty((w.batch, w.n_q_heads, 2 * w.n_pairs), dtype=st.dt, device=st.device).normal_(0, sig, generator=g)
+    dl = torch.tensor(lens, dtype=torch.int32, device=st.device)
+    want = O.decode_attn(util.to_np64(q), util.to_np64(st.k_cache[0]), util.to_np64(st.v_cache[0]), lens, w.head_dim)
+    st.ctx.rap_debug_set_scan_pieces(2, 100)
+    for variant, n_split in ((4, 0), (3, 0), (4, 0), (4, 3), (4, 0), (3, 0), (3, 0), (4, 0), (4, 0)):
+        st.ctx.rap_set_attn_variant(variant)
+        st.out.fill_(float("nan"))
+        out = st.decode_attn(0, q, dl, max(lens), n_split=n_split)
+        torch.cuda.synchronize()
+        got = util.to_np64(out[: w.batch * w.n_q_heads * w.n_vch]).reshape(w.batch, w.n_q_heads, w.n_vch)
+        util.check_attn(got, want, w.dtype)
+    assert st.ctx.rap_get_last_device_status() == (0, 0)
+    st.close()
 
 
 @pytest.mark.parametrize("name", ["3b", "8b", "14b", "sweep1.0", "sweep0.5"])
