@@ -46,7 +46,8 @@ rap_status rap_set_proj_variant(rap_ctx* ctx, int32_t variant);
  * used, so nothing has to be reset by hand.  The hook disarms itself when it is used. */
 rap_status rap_debug_arm_wait_timeout(rap_ctx* ctx);
 
-/* The tensor-core scan of rap_decode_attn normally decides by the size of a launch whether its last tiles are handed
+/* The tensor-core scan of rap_decode_attn (head shapes of the shaped workloads: the five retain ratios at D = 128,
+ * 3 to 5 query heads per KV head) normally decides by the size of a launch whether its last tiles are handed
  * out at run time (pieces of some tiles, claimed from a counter by the CTAs as they finish) or assigned up front like
  * the rest.  This forces the choice for every later launch on the context, so that small test cases take the run-time
  * path: piece_tiles > 0 tiles per piece and frac_x256 / 256 of all tiles handed out that way; piece_tiles = 0: nothing

@@ -125,7 +125,8 @@ __device__ __forceinline__ uint32_t mma_prmt(uint32_t a, uint32_t b, uint32_t se
   return r;
 }
 
-template <int G, int WK, int DV>
+// DYN: the instantiation that can hand the last tiles of a launch out at run time (long launches; rap_scan_params)
+template <int G, int WK, int DV, bool DYN>
 __global__ void __launch_bounds__(MmaCfg<G, WK, DV>::THREADS, 2) attn_mma_kernel(const ScanParams p,
                                                                                  const __grid_constant__ CUtensorMap map_k,
                                                                                  const __grid_constant__ CUtensorMap map_v) {
@@ -158,7 +159,10 @@ __global__ void __launch_bounds__(MmaCfg<G, WK, DV>::THREADS, 2) attn_mma_kernel
   splan.T = 0; splan.nc = 0;
   bool shared_plan = false;
   int* const pref = reinterpret_cast<int*>(red);
-  auto piece_of = [&](int tile) { return tile < T_s ? sk_cta_of(tile, splan) : splan.nc + (tile - T_s) / DC; };
+  auto piece_of = [&](int tile) {
+    if constexpr (DYN) return tile < T_s ? sk_cta_of(tile, splan) : splan.nc + (tile - T_s) / DC;
+    else return sk_cta_of(tile, plan);
+  };
   auto locate = [&](int tile) {      // the unit that holds this tile: b, h, unit_start
     int pb = 0;
     if (shared_plan) {
@@ -181,7 +185,7 @@ __global__ void __launch_bounds__(MmaCfg<G, WK, DV>::THREADS, 2) attn_mma_kernel
     shared_plan = sk_plan_shared(p.seq_len, p.B, p.Hkv, p.len_add, p.S_cap, ST, (int)gridDim.x, pref, C::RED_BYTES / 4, &plan);
     if (!shared_plan) plan = sk_plan(p.seq_len, p.B, p.Hkv, p.len_add, p.S_cap, ST, (int)gridDim.x);
     T_s = plan.T;
-    if (shared_plan && DC > 0 && plan.T > 0) {
+    if (DYN && shared_plan && DC > 0 && plan.T > 0) {
       const int n_max = pref[C::RED_BYTES / 4 - 1];     // tiles of the longest sequence
       const int nd = (int)((long long)plan.T * p.dyn_frac_x256 / 256 / DC);
       const int ts = plan.T - nd * DC;
@@ -210,14 +214,21 @@ __global__ void __launch_bounds__(MmaCfg<G, WK, DV>::THREADS, 2) attn_mma_kernel
       }
     }
     if ((int)blockIdx.x >= plan.nc) return;
-    if ((int)blockIdx.x < splan.nc) {
-      cur = (int)((long long)blockIdx.x * T_s / splan.nc);
-      hi = (int)((long long)(blockIdx.x + 1) * T_s / splan.nc);
-    }
-    if (cur < hi) {
+    if constexpr (DYN) {
+      if ((int)blockIdx.x < splan.nc) {
+        cur = (int)((long long)blockIdx.x * T_s / splan.nc);
+        hi = (int)((long long)(blockIdx.x + 1) * T_s / splan.nc);
+      }
+      if (cur < hi) {
+        locate(cur);
+      } else if (n_dyn == 0) {
+        return;
+      }
+    } else {
+      cur = (int)((long long)blockIdx.x * plan.T / plan.nc);
+      hi = (int)((long long)(blockIdx.x + 1) * plan.T / plan.nc);
+      if (cur >= hi) return;
       locate(cur);
-    } else if (n_dyn == 0) {
-      return;
     }
   } else {
     pdl_wait();
@@ -277,7 +288,9 @@ __global__ void __launch_bounds__(MmaCfg<G, WK, DV>::THREADS, 2) attn_mma_kernel
     __syncthreads();                   // every thread has read the prefix before the buffer is reused
     return true;
   };
-  if (p.balanced && cur >= hi && !claim()) return;      // a CTA without a part assigned up front starts with a piece
+  if constexpr (DYN) {
+    if (p.balanced && cur >= hi && !claim()) return;    // a CTA without a part assigned up front starts with a piece
+  }
 
   for (;;) {   // one pass per segment (a single one unless the mode is balanced)
     int seg_tiles;
@@ -662,18 +675,28 @@ __global__ void __launch_bounds__(MmaCfg<G, WK, DV>::THREADS, 2) attn_mma_kernel
     // ---- next segment: the following unit, from its first tile ----
     if (!p.balanced) break;
     cur += n_my;
-    bool more = cur < hi;
-    if (more) {
+    if constexpr (DYN) {
+      bool more = cur < hi;
+      if (more) {
+        unit_start += seg_tiles;
+        if (++h == p.Hkv) {
+          h = 0;
+          do { ++b; } while (b < p.B && sk_tiles_of(p.seq_len, b, p.len_add, p.S_cap, ST) == 0);
+          if (b >= p.B) more = false;
+        }
+      }
+      if (!more) {
+        // this piece is done: claim the next of the pieces that are handed out at run time, if there is one left
+        if (n_dyn == 0 || !claim()) break;
+      }
+    } else {
+      if (cur >= hi) break;
       unit_start += seg_tiles;
       if (++h == p.Hkv) {
         h = 0;
         do { ++b; } while (b < p.B && sk_tiles_of(p.seq_len, b, p.len_add, p.S_cap, ST) == 0);
-        if (b >= p.B) more = false;
+        if (b >= p.B) break;
       }
-    }
-    if (!more) {
-      // this piece is done: claim the next of the pieces that are handed out at run time, if there is one left
-      if (n_dyn == 0 || !claim()) break;
     }
     __syncthreads();   // the reduction buffer and the merge scalars are reused by the next segment
   }   // segment loop

@@ -125,50 +125,13 @@ __global__ void __launch_bounds__(Q8Cfg<G, WK, DV>::THREADS, 2) attn_q8_kernel(c
   SkPlan plan;
   plan.T = 0; plan.nc = 0;
   int cur = 0, hi = 0, unit_start = 0;
-  // Pieces claimed at run time (see rap_scan_params and rap_attn_mma_kernel.cuh): the tiles [T_s, T) in n_dyn pieces of
-  // DC tiles; a piece's index in tile order is the CTA's number for the part assigned up front, nc + j for piece j
-  int T_s = 0, n_dyn = 0, my_piece = (int)blockIdx.x;
-  const int DC = p.dyn_piece;
-  SkPlan splan;
-  splan.T = 0; splan.nc = 0;
-  bool shared_plan = false;
-  int* const pref = reinterpret_cast<int*>(red);
-  auto piece_of = [&](int tile) { return tile < T_s ? sk_cta_of(tile, splan) : splan.nc + (tile - T_s) / DC; };
-  auto locate = [&](int tile) {      // the unit that holds this tile: b, h, unit_start
-    int pb = 0;
-    if (shared_plan) {
-      b = sk_seq_of(pref, p.B, tile);
-      pb = b > 0 ? pref[b - 1] : 0;
-    } else {
-      for (b = 0; b < p.B; ++b) {
-        const int nb = sk_tiles_of(p.seq_len, b, p.len_add, p.S_cap, ST) * p.Hkv;
-        if (tile < pb + nb) break;
-        pb += nb;
-      }
-    }
-    const int ntb = sk_tiles_of(p.seq_len, b, p.len_add, p.S_cap, ST);
-    h = (tile - pb) / ntb;
-    unit_start = pb + h * ntb;
-  };
   if (p.balanced) {
     // the plan (reads the lengths only): computed by the first warp into the reduction buffer, which is free until
     // the first merge; batches too large for that buffer are planned by every thread on its own
-    shared_plan = sk_plan_shared(p.seq_len, p.B, p.Hkv, p.len_add, p.S_cap, ST, (int)gridDim.x, pref, C::RED_BYTES / 4, &plan);
+    int* pref = reinterpret_cast<int*>(red);
+    const bool shared_plan = sk_plan_shared(p.seq_len, p.B, p.Hkv, p.len_add, p.S_cap, ST, (int)gridDim.x, pref,
+                                            C::RED_BYTES / 4, &plan);
     if (!shared_plan) plan = sk_plan(p.seq_len, p.B, p.Hkv, p.len_add, p.S_cap, ST, (int)gridDim.x);
-    T_s = plan.T;
-    if (shared_plan && DC > 0 && plan.T > 0) {
-      const int n_max = pref[C::RED_BYTES / 4 - 1];     // tiles of the longest sequence
-      const int nd = (int)((long long)plan.T * p.dyn_frac_x256 / 256 / DC);
-      const int ts = plan.T - nd * DC;
-      const int ncs = min(plan.nc, ts);                  // CTAs with a part assigned up front
-      // no unit may get more than RAP_MAX_SPLIT partials: pieces of either kind that can touch it, ragged ends included
-      if (nd > 0 && (ts == 0 ? 0LL : (long long)n_max * ncs / ts) + n_max / DC + 4 <= RAP_MAX_SPLIT) {
-        n_dyn = nd;
-        T_s = ts;
-      }
-    }
-    splan.T = T_s;
-    splan.nc = min(plan.nc, T_s);
     // Everything below reads q~ and the cache rows the previous kernel in the stream wrote, and writes what the next
     // one may depend on: wait for the predecessor first, and only then let the successor start (it may begin to
     // stream its weights while this scan runs, and waits for this kernel before it writes anything this one reads).
@@ -176,7 +139,7 @@ __global__ void __launch_bounds__(Q8Cfg<G, WK, DV>::THREADS, 2) attn_q8_kernel(c
     pdl_launch_dependents();
     if (blockIdx.x == 0) {   // sequences without any row are scanned by nobody: their output is zero
       for (int i = tid; i < p.B * p.Hkv; i += THREADS) p.unit_cnt_other[i] = 0;   // counters a launch that gave up left behind
-      if (tid == 0) *p.dyn_next_other = 0;                                        // and the piece counter of the previous launch
+      if (tid == 0) *p.dyn_next_other = 0;          // and the piece counter a bf16 tensor-core launch before this one used
       for (int bb = 0; bb < p.B; ++bb) {
         const bool empty = shared_plan ? pref[bb] == (bb > 0 ? pref[bb - 1] : 0)
                                        : sk_tiles_of(p.seq_len, bb, p.len_add, p.S_cap, ST) == 0;
@@ -185,15 +148,23 @@ __global__ void __launch_bounds__(Q8Cfg<G, WK, DV>::THREADS, 2) attn_q8_kernel(c
       }
     }
     if ((int)blockIdx.x >= plan.nc) return;
-    if ((int)blockIdx.x < splan.nc) {
-      cur = (int)((long long)blockIdx.x * T_s / splan.nc);
-      hi = (int)((long long)(blockIdx.x + 1) * T_s / splan.nc);
+    cur = (int)((long long)blockIdx.x * plan.T / plan.nc);
+    hi = (int)((long long)(blockIdx.x + 1) * plan.T / plan.nc);
+    if (cur >= hi) return;
+    int pb = 0;
+    if (shared_plan) {       // the unit that holds tile `cur`
+      b = sk_seq_of(pref, p.B, cur);
+      pb = b > 0 ? pref[b - 1] : 0;
+    } else {
+      for (b = 0; b < p.B; ++b) {
+        const int nb = sk_tiles_of(p.seq_len, b, p.len_add, p.S_cap, ST) * p.Hkv;
+        if (cur < pb + nb) break;
+        pb += nb;
+      }
     }
-    if (cur < hi) {
-      locate(cur);
-    } else if (n_dyn == 0) {
-      return;
-    }
+    const int ntb = sk_tiles_of(p.seq_len, b, p.len_add, p.S_cap, ST);
+    h = (cur - pb) / ntb;
+    unit_start = pb + h * ntb;
   } else {
     pdl_wait();
     pdl_launch_dependents();
@@ -221,24 +192,6 @@ __global__ void __launch_bounds__(Q8Cfg<G, WK, DV>::THREADS, 2) attn_q8_kernel(c
   bool timed_out = false;
   const float cs = p.qscale;   // log2(e) / sqrt(D)
 
-  // claims the next of the pieces that are handed out at run time; false when none is left (every thread calls it)
-  auto claim = [&]() -> bool {
-    __syncthreads();                   // the merge scalars and the reduction buffer are free
-    if (tid == 0) *s_last = atomicAdd(p.dyn_next, 1);
-    __syncthreads();
-    const int j = *s_last;
-    if (j >= n_dyn) return false;
-    my_piece = splan.nc + j;
-    cur = T_s + j * DC;
-    hi = cur + DC;
-    SkPlan again;                      // the prefix of the plan once more: the reduction buffer held sums in between
-    sk_plan_shared(p.seq_len, p.B, p.Hkv, p.len_add, p.S_cap, ST, (int)gridDim.x, pref, C::RED_BYTES / 4, &again);
-    locate(cur);
-    __syncthreads();                   // every thread has read the prefix before the buffer is reused
-    return true;
-  };
-  if (p.balanced && cur >= hi && !claim()) return;      // a CTA without a part assigned up front starts with a piece
-
   for (;;) {   // one pass per segment (a single one unless the mode is balanced)
     int seg_tiles;
     {
@@ -247,7 +200,7 @@ __global__ void __launch_bounds__(Q8Cfg<G, WK, DV>::THREADS, 2) attn_q8_kernel(c
       if (p.balanced) {
         t_begin = cur - unit_start;
         n_my = min(seg_tiles - t_begin, hi - cur);
-        const int seg = my_piece - piece_of(unit_start);
+        const int seg = (int)blockIdx.x - sk_cta_of(unit_start, plan);
         ws_head = (size_t)RAP_MAX_SPLIT * (DV + 2);
         ws_base = p.ws + (((size_t)b * p.Hq + (size_t)h * G) * RAP_MAX_SPLIT + seg) * (size_t)(DV + 2);
       } else {
@@ -502,8 +455,8 @@ __global__ void __launch_bounds__(Q8Cfg<G, WK, DV>::THREADS, 2) attn_q8_kernel(c
       // ---- the CTA that delivers a unit's last partial merges them (no separate combine launch) ----
       __threadfence();           // this CTA's partials are visible before its arrival is counted
       __syncthreads();
-      const int first = piece_of(unit_start);
-      const int nseg = piece_of(unit_start + seg_tiles - 1) - first + 1;
+      const int first = sk_cta_of(unit_start, plan);
+      const int nseg = sk_cta_of(unit_start + seg_tiles - 1, plan) - first + 1;
       const int u = b * p.Hkv + h;
       if (tid == 0) *s_last = RAP_BOUNDS(u, p.B * p.Hkv, p.status, 0x20a) && atomicAdd(&p.unit_cnt[u], 1) == nseg - 1;
       __syncthreads();
@@ -582,18 +535,12 @@ __global__ void __launch_bounds__(Q8Cfg<G, WK, DV>::THREADS, 2) attn_q8_kernel(c
     // ---- next segment: the following unit, from its first tile ----
     if (!p.balanced) break;
     cur += n_my;
-    bool more = cur < hi;
-    if (more) {
-      unit_start += seg_tiles;
-      if (++h == p.Hkv) {
-        h = 0;
-        do { ++b; } while (b < p.B && sk_tiles_of(p.seq_len, b, p.len_add, p.S_cap, ST) == 0);
-        if (b >= p.B) more = false;
-      }
-    }
-    if (!more) {
-      // this piece is done: claim the next of the pieces that are handed out at run time, if there is one left
-      if (n_dyn == 0 || !claim()) break;
+    if (cur >= hi) break;
+    unit_start += seg_tiles;
+    if (++h == p.Hkv) {
+      h = 0;
+      do { ++b; } while (b < p.B && sk_tiles_of(p.seq_len, b, p.len_add, p.S_cap, ST) == 0);
+      if (b >= p.B) break;
     }
     __syncthreads();   // the reduction buffer and the merge scalars are reused by the next segment
   }   // segment loop

@@ -61,7 +61,7 @@ __global__ void __launch_bounds__(128) attn_scan_combine_kernel(const float* __r
 }  // namespace
 
 static rap_status launch_split_kv(rap_ctx* ctx, const rap_attn_args& a, int n_split_req, cudaStream_t st,
-                                  const rap_scan_entry* e, bool is_mma, bool pieces = false) {
+                                  const rap_scan_entry* e, bool is_mma) {
   // n_split = 0: balanced mode, one CTA per resident slot; an explicit n_split keeps equal ranges per split
   const bool balanced = n_split_req <= 0 && (long long)a.B * a.Hkv * ((a.S_cap + 63) / 64) < (1LL << 31);
   int n_split = balanced ? RAP_MAX_SPLIT : n_split_req;
@@ -88,13 +88,16 @@ static rap_status launch_split_kv(rap_ctx* ctx, const rap_attn_args& a, int n_sp
     p.dyn_next = ctx->d_unit_cnt + 2 * n_units + set;
     p.dyn_next_other = ctx->d_unit_cnt + 2 * n_units + (set ^ 1u);
   }
-  // Long launches of the tensor-core forms (bf16 and quantised cache): the CTAs do not stream at the same pace (the memory system shares its
+  // Long launches of the tensor-core form: the CTAs do not stream at the same pace (the memory system shares its
   // bandwidth unevenly), so the last tenth of the tiles is not assigned up front but claimed piece by piece by
   // whoever is done.  A piece costs a pipeline refill and a partial, so short launches (under ~100 tiles per CTA)
-  // keep the fixed split; a piece is long enough that no unit gets more than ~24 of them.
+  // keep the fixed split -- and the kernel without that logic, which starts and ends a microsecond or two sooner; a
+  // piece is long enough that no unit gets more than ~24 of them.  (Measured on the quantised cache: no gain, a
+  // piece's overhead weighs twice as much there.)
   p.dyn_piece = 0;
   p.dyn_frac_x256 = 0;
-  if (balanced && (is_mma || pieces)) {
+  const void* fn = e->fn;
+  if (balanced && is_mma && e->fn_dyn) {
     const long long unit_tiles = (a.h_len_max + e->tile - 1) / e->tile;
     const long long per_cta = (long long)a.B * a.Hkv * unit_tiles / (2 * ctx->sm_count);
     if (ctx->dbg_dyn_piece >= 0) {
@@ -104,6 +107,7 @@ static rap_status launch_split_kv(rap_ctx* ctx, const rap_attn_args& a, int n_sp
       p.dyn_piece = (int)(unit_tiles / 24 > 16 ? unit_tiles / 24 : 16);
       p.dyn_frac_x256 = 26;
     }
+    if (p.dyn_piece > 0 && p.dyn_frac_x256 > 0) fn = e->fn_dyn;
   }
   p.out = a.out;
   p.wait_limit = WAIT_LIMIT;
@@ -115,7 +119,7 @@ static rap_status launch_split_kv(rap_ctx* ctx, const rap_attn_args& a, int n_sp
     p.dbg_skip_copy = 1;
     ctx->dbg_arm_timeout = 0;
   }
-  RAP_CUDA_TRY(ctx, rap_raise_smem(ctx, e->fn, e->smem));
+  RAP_CUDA_TRY(ctx, rap_raise_smem(ctx, fn, e->smem));
   const int scan_grid = 2 * ctx->sm_count;
   dim3 grid(n_split, a.Hkv, a.B);
   if (balanced) grid = dim3(scan_grid, 1, 1);
@@ -137,7 +141,7 @@ static rap_status launch_split_kv(rap_ctx* ctx, const rap_attn_args& a, int n_sp
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = a.pdl ? 1 : 0;      // the kernel waits for its predecessor before it reads q~ or a cache row
-  RAP_CUDA_TRY(ctx, cudaLaunchKernelExC(&cfg, e->fn, args));
+  RAP_CUDA_TRY(ctx, cudaLaunchKernelExC(&cfg, fn, args));
   ctx->launches++;
   RAP_CUDA_TRY(ctx, cudaGetLastError());
   if (balanced) {
@@ -166,5 +170,5 @@ rap_status rap_launch_attn_mma(rap_ctx* ctx, const rap_attn_args& a, int n_split
 rap_status rap_launch_attn_q8_mma(rap_ctx* ctx, const rap_attn_args& a, int n_split_req, cudaStream_t st) {
   if (a.dtype != RAP_BF16 || (a.P2 & 1)) return RAP_EUNSUPPORTED;
   const rap_scan_entry* e = rap_q8_find(a.Hq / a.Hkv, a.P2 / 2, a.dv);
-  return e ? launch_split_kv(ctx, a, n_split_req, st, e, false, true) : RAP_EUNSUPPORTED;
+  return e ? launch_split_kv(ctx, a, n_split_req, st, e, false) : RAP_EUNSUPPORTED;
 }

@@ -139,6 +139,7 @@ struct rap_scan_entry {
   int threads;         // CTA size
   int tma;             // 1: the kernel takes tensor maps of the K and V caches (boxes of 32 rows x 64 elements)
   const void* fn;      // the kernel, launched with cudaLaunchKernel
+  const void* fn_dyn;  // tensor-core scan only: the instantiation that can hand tiles out at run time, or nullptr
 };
 // the instantiation built for this head shape, or nullptr (generated at build time):
 // the FP32-pipe scan (rap_attn_scan_kernel.cuh) and the mma.sync scan (rap_attn_mma_kernel.cuh)

@@ -121,13 +121,10 @@ def test_q8_append_and_attention_end_to_end(name):
     st.close()
 
 
-def _random_q8_case(w, lens, n_split, seed=0, variant=0, q_gain=1.0, pieces=None):
-    """rap_decode_attn_q8 alone on caches quantised by rap_quantize_rows from random rows, every unit checked.
-    pieces = (tiles per piece, 256ths of all tiles) forces the scan to hand that share of its tiles out at run time."""
+def _random_q8_case(w, lens, n_split, seed=0, variant=0, q_gain=1.0):
+    """rap_decode_attn_q8 alone on caches quantised by rap_quantize_rows from random rows, every unit checked."""
     st = DecodeStack(w, s_cap=((max(lens) + 8 + 7) // 8) * 8)
     st.ctx.rap_set_attn_variant(variant)
-    if pieces is not None:
-        st.ctx.rap_debug_set_scan_pieces(*pieces)
     st.build_tables(*synth.draw_scores(w))
     g = torch.Generator(device=st.device).manual_seed(seed)
     P2, dv = 2 * w.n_pairs, w.n_vch
@@ -157,15 +154,6 @@ def _random_q8_case(w, lens, n_split, seed=0, variant=0, q_gain=1.0, pieces=None
             want[b] = 0.0
     util.check_attn(util.to_np64(out), want, w.dtype)
     st.close()
-
-
-@pytest.mark.parametrize("name", ["3b", "8b", "14b"])
-@pytest.mark.parametrize("pieces", [(1, 128), (2, 64), (5, 40), (1, 256)])
-def test_q8_attention_pieces_claimed_at_run_time(name, pieces):
-    """The scan over the quantised cache with a share of its tiles handed out at run time (forced on a small case)."""
-    w = synth.scaled_down(synth.CONFIGS[name], n_layers=1, batch=4, seq=4096)
-    _random_q8_case(w, [4096, 2500, 1, 700], 0, seed=sum(pieces), pieces=pieces)
-    _random_q8_case(w, [300, 0, 3999, 129], 0, seed=pieces[0], pieces=pieces)
 
 
 @pytest.mark.parametrize("name", ["3b", "8b", "14b", "sweep1.0", "sweep0.8", "sweep0.5"])
