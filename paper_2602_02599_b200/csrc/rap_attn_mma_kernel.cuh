@@ -275,7 +275,14 @@ __global__ void __launch_bounds__(MmaCfg<G, WK, DV>::THREADS, 2) attn_mma_kernel
   // claims the next of the pieces that are handed out at run time; false when none is left (every thread calls it)
   auto claim = [&]() -> bool {
     __syncthreads();                   // the merge scalars and the reduction buffer are free
-    if (tid == 0) *s_last = atomicAdd(p.dyn_next, 1);
+    if (tid == 0) {
+      const int got = atomicAdd(p.dyn_next, 1);
+      *s_last = got;
+      // Every CTA that takes part claims until it is refused once: n_dyn + nc claims per launch.  Whoever makes the
+      // last one leaves the counter at zero for the next launch that uses it (a replayed CUDA graph may run two
+      // launches in a row on the same counter, so clearing "the other one" at the start of a launch is not enough).
+      if (got == n_dyn + plan.nc - 1) *p.dyn_next = 0;
+    }
     __syncthreads();
     const int j = *s_last;
     if (j >= n_dyn) return false;

@@ -520,12 +520,17 @@ def test_layer_adaptive_head_shapes_attention(P, dv):
     _random_attn_case(w, [3000, 1777, 1], 3, seed=P)
 
 
-def test_decode_step_replays_from_a_cuda_graph():
+@pytest.mark.parametrize("n_layers,pieces", [(2, None), (3, (1, 128)), (2, (2, 256))])
+def test_decode_step_replays_from_a_cuda_graph(n_layers, pieces):
     """rap_decode_step reads the sequence lengths on the device and its balanced scan has a fixed grid, so a
-    step captured once can be replayed as the lengths advance: two replays equal two eager steps bit for bit."""
-    w = synth.scaled_down(synth.LLAMA_8B, n_layers=2, batch=2, seq=300, hidden=256)
+    step captured once can be replayed as the lengths advance: two replays equal two eager steps bit for bit.  Also
+    with the scan handing tiles out at run time (forced on this small case): with an odd number of layers two
+    consecutive launches of the replay use the same piece counter, which the launch before must have left at zero."""
+    w = synth.scaled_down(synth.LLAMA_8B, n_layers=n_layers, batch=2, seq=300, hidden=256)
     ks, vs = synth.draw_scores(w)
     st, tabs, w_host = util.build_small_stack(w, ks, vs, full_weights=False)
+    if pieces is not None:
+        st.ctx.rap_debug_set_scan_pieces(*pieces)
     g = torch.Generator(device=st.device).manual_seed(5)
     for l in range(w.n_layers):
         st.k_cache[l].normal_(0, 1.0, generator=g)
@@ -556,6 +561,11 @@ def test_decode_step_replays_from_a_cuda_graph():
         graph.replay()
         torch.cuda.synchronize()
         assert torch.equal(st.out, eager[i])
+    P2, dv = 2 * st.n_pairs[n_layers - 1], st.n_vch[n_layers - 1]
+    q_last = st.q_scratch.flatten()[: w.batch * w.n_q_heads * P2].reshape(w.batch, w.n_q_heads, P2)
+    want = O.decode_attn(util.to_np64(q_last), util.to_np64(st.k_cache[n_layers - 1]), util.to_np64(st.v_cache[n_layers - 1]),
+                         [302, 125], w.head_dim)      # the last layer of the last replay against the definition
+    util.check_attn(util.to_np64(st.out[n_layers - 1][: w.batch * w.n_q_heads * dv]).reshape(w.batch, w.n_q_heads, dv), want, w.dtype)
     assert st.seq_len.cpu().tolist() == [302, 125]
     assert st.ctx.rap_get_last_device_status() == (0, 0)
     st.close()
