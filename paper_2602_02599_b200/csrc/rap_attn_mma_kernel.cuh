@@ -191,7 +191,10 @@ __global__ void __launch_bounds__(MmaCfg<G, WK, DV>::THREADS, 2) attn_mma_kernel
       const int ts = plan.T - nd * DC;
       // no unit may get more than RAP_MAX_SPLIT partials: pieces of either kind that can touch it, ragged ends included
       const int ncs = min(plan.nc, ts);                  // CTAs with a part assigned up front
-      if (nd > 0 && (ts == 0 ? 0LL : (long long)n_max * ncs / ts) + n_max / DC + 4 <= RAP_MAX_SPLIT) {
+      // ... and a piece must be small against a CTA's own part (the launcher judged by the longest sequence; a batch of
+      // mostly short ones has far fewer tiles), unless the test hook chose the sizes
+      const bool small_pieces = !p.dyn_guard || (long long)DC * plan.nc * 6 <= (long long)plan.T;
+      if (nd > 0 && small_pieces && (ts == 0 ? 0LL : (long long)n_max * ncs / ts) + n_max / DC + 4 <= RAP_MAX_SPLIT) {
         n_dyn = nd;
         T_s = ts;
       }

@@ -96,6 +96,7 @@ static rap_status launch_split_kv(rap_ctx* ctx, const rap_attn_args& a, int n_sp
   // piece's overhead weighs twice as much there.)
   p.dyn_piece = 0;
   p.dyn_frac_x256 = 0;
+  p.dyn_guard = 0;
   const void* fn = e->fn;
   if (balanced && is_mma && e->fn_dyn) {
     const long long unit_tiles = (a.h_len_max + e->tile - 1) / e->tile;
@@ -106,6 +107,7 @@ static rap_status launch_split_kv(rap_ctx* ctx, const rap_attn_args& a, int n_sp
     } else if (per_cta >= 96) {
       p.dyn_piece = (int)(unit_tiles / 24 > 16 ? unit_tiles / 24 : 16);
       p.dyn_frac_x256 = 26;
+      p.dyn_guard = 1;
     }
     if (p.dyn_piece > 0 && p.dyn_frac_x256 > 0) fn = e->fn_dyn;
   }

@@ -130,6 +130,7 @@ struct rap_scan_params {
   // of dyn_piece tiles that the CTAs claim from a counter as they finish (0: everything is assigned up front)
   int dyn_piece;       // tiles per piece
   int dyn_frac_x256;   // share of all tiles handed out that way, in 256ths
+  int dyn_guard;       // 1: the kernel drops the pieces when they turn out large against a CTA's own part (automatic mode)
   int32_t* dyn_next;   // next unclaimed piece of this launch (zero on entry)
   int32_t* dyn_next_other;   // the counter the previous launch used; cleared by this launch
 };
